@@ -1,0 +1,233 @@
+"""fp64 CPU oracle for the SAPO policy-scoring path.  TEST INFRASTRUCTURE ONLY.
+
+This file is the slow, plain definition the CUDA library is checked against.  Only the
+test-suite, the smoke check and the benchmark's CPU-baseline leg may import it; the
+product path never does.  It shares no code with the CUDA sources.
+
+What it computes, and where the method states it:
+
+  pack_rollouts       the training set T^n = {I local samples} U {J external samples}
+                      (paper Section 3.2, training-set equation; Algorithm 1
+                      "Assemble training set"), as a varlen token layout
+  group_advantages    GRPO's group-relative advantage (paper Section 4.2 names GRPO);
+                      A = (r - mean_group) / (std_group + eps)
+  token_logprobs      log-prob of each chosen token under the policy's LM head
+                      (Section 3.2: nodes "re-encode and compute token-level values" for
+                      any rollout as if it were their own)
+  policy_loss_fwd     the clipped-ratio surrogate with KL weight 0 and separate lower /
+                      upper clip thresholds (Section 4.2)
+  policy_loss_bwd     its gradient with respect to the final hidden states and the
+                      LM-head weight (Algorithm 1 "Policy update")
+
+All floating point is float64; inputs (bf16 or fp32 values) are widened exactly.
+Every function here is pinned by tests/test_oracle_pins.py against closed forms,
+library routines, invariants, finite differences and brute force; none is unpinned.
+"""
+from __future__ import annotations
+
+from typing import Dict, Optional
+
+import numpy as np
+
+
+# --------------------------------------------------------------------------------------
+def pack_rollouts(local: Dict[str, np.ndarray], ext: Dict[str, np.ndarray],
+                  sel: Dict[str, np.ndarray]) -> Dict[str, np.ndarray]:
+    """Merge the selected local and external rollouts into one token-major batch.
+
+    Section 3.2 builds the training set as the union of I samples of the node's own
+    rollouts and J samples shared by the swarm.  The paper writes a set; the order used
+    here (and required bit for bit of any implementation) is: questions in order, and
+    inside a question first its local picks in list order, then its external picks in
+    list order.
+
+    `local` / `ext`: dicts with hidden [n_tok,H], ids [n_tok], old_logp [n_tok],
+    offsets [n+1], rewards [n].  `sel`: q_offsets_local [Q+1], local_idx,
+    q_offsets_ext [Q+1], ext_idx.
+    """
+    Q = len(sel["q_offsets_local"]) - 1
+    rows_hidden, rows_ids, rows_old = [], [], []
+    rewards, seq_group, seq_is_ext, seq_src, lengths = [], [], [], [], []
+    group_offsets = [0]
+    for q in range(Q):
+        picks = [(0, int(sel["local_idx"][k]))
+                 for k in range(sel["q_offsets_local"][q], sel["q_offsets_local"][q + 1])]
+        picks += [(1, int(sel["ext_idx"][k]))
+                  for k in range(sel["q_offsets_ext"][q], sel["q_offsets_ext"][q + 1])]
+        for is_ext, idx in picks:
+            buf = ext if is_ext else local
+            a, b = int(buf["offsets"][idx]), int(buf["offsets"][idx + 1])
+            rows_hidden.append(buf["hidden"][a:b])
+            rows_ids.append(buf["ids"][a:b])
+            rows_old.append(buf["old_logp"][a:b])
+            rewards.append(buf["rewards"][idx])
+            seq_group.append(q)
+            seq_is_ext.append(is_ext)
+            seq_src.append(idx)
+            lengths.append(b - a)
+        group_offsets.append(len(seq_group))
+    S = len(lengths)
+    cu = np.zeros(S + 1, dtype=np.int32)
+    for s in range(S):
+        cu[s + 1] = cu[s] + lengths[s]
+    T = int(cu[S])
+    tok_seq = np.zeros(T, dtype=np.int32)
+    for s in range(S):
+        tok_seq[cu[s]:cu[s + 1]] = s
+    H = local["hidden"].shape[1]
+    cat = lambda rows, like, shape: (np.concatenate(rows, axis=0) if rows
+                                     else np.zeros(shape, dtype=like.dtype))
+    return {
+        "hidden": cat(rows_hidden, local["hidden"], (0, H)),
+        "ids": cat(rows_ids, local["ids"], (0,)),
+        "old_logp": cat(rows_old, local["old_logp"], (0,)),
+        "rewards": np.asarray(rewards, dtype=np.float32),
+        "cu_seqlens": cu,
+        "seq_group": np.asarray(seq_group, dtype=np.int32),
+        "seq_is_ext": np.asarray(seq_is_ext, dtype=np.uint8),
+        "seq_src": np.asarray(seq_src, dtype=np.int32),
+        "tok_seq": tok_seq,
+        "group_offsets": np.asarray(group_offsets, dtype=np.int32),
+        "n_tokens": T,
+    }
+
+
+# --------------------------------------------------------------------------------------
+def group_advantages(rewards: np.ndarray, group_offsets: np.ndarray,
+                     adv_eps: float = 1e-6, ddof: int = 0) -> Dict[str, np.ndarray]:
+    """Group-relative advantage of GRPO (the update rule named in Section 4.2).
+
+    For every question g with member rewards r_1..r_G:
+        mean_g = (1/G) sum r,   std_g = sqrt( sum (r-mean_g)^2 / (G - ddof) ),
+        A_s    = (r_s - mean_g) / (std_g + adv_eps).
+    The group runs over every completion of the question, local or external.
+    A group with G - ddof <= 0 has std 0.
+    """
+    r = np.asarray(rewards, dtype=np.float64)
+    Q = len(group_offsets) - 1
+    adv = np.zeros_like(r)
+    mean = np.zeros(Q)
+    std = np.zeros(Q)
+    for g in range(Q):
+        a, b = int(group_offsets[g]), int(group_offsets[g + 1])
+        if b == a:
+            continue
+        mu = r[a:b].sum() / (b - a)
+        denom = (b - a) - ddof
+        sd = np.sqrt(((r[a:b] - mu) ** 2).sum() / denom) if denom > 0 else 0.0
+        mean[g], std[g] = mu, sd
+        adv[a:b] = (r[a:b] - mu) / (sd + adv_eps)
+    return {"adv": adv, "mean": mean, "std": std}
+
+
+# --------------------------------------------------------------------------------------
+def logits(hidden: np.ndarray, W: np.ndarray) -> np.ndarray:
+    """z[t, v] = sum_k hidden[t, k] * W[v, k]  (LM head, no bias, temperature 1)."""
+    return np.asarray(hidden, dtype=np.float64) @ np.asarray(W, dtype=np.float64).T
+
+
+def token_logprobs(hidden: np.ndarray, W: np.ndarray, ids: np.ndarray) -> Dict[str, np.ndarray]:
+    """lse_t = log sum_v exp z[t,v];  logp_t = z[t, ids_t] - lse_t."""
+    z = logits(hidden, W)
+    m = z.max(axis=1)
+    lse = m + np.log(np.exp(z - m[:, None]).sum(axis=1))
+    zy = z[np.arange(z.shape[0]), np.asarray(ids, dtype=np.int64)]
+    return {"lse": lse, "logp": zy - lse, "z": z}
+
+
+def _seq_of_token(cu_seqlens: np.ndarray) -> np.ndarray:
+    S = len(cu_seqlens) - 1
+    return np.repeat(np.arange(S), np.diff(np.asarray(cu_seqlens, dtype=np.int64)))
+
+
+def surrogate_from_logp(logp: np.ndarray, old_logp: np.ndarray, adv: np.ndarray,
+                        cu_seqlens: np.ndarray, eps_low: float, eps_high: float,
+                        grad_scale: float = 1.0, n_seqs_total: Optional[int] = None
+                        ) -> Dict[str, np.ndarray]:
+    """Clipped-ratio surrogate and its derivative with respect to logp (Section 4.2).
+
+        rho_t = exp(logp_t - old_t)
+        u_t   = min( rho_t * A_s , clip(rho_t, 1-eps_low, 1+eps_high) * A_s )
+        L     = - (1/S) sum_s (1/T_s) sum_{t in s} u_t            (KL weight 0)
+        g_t   = dL/dlogp_t = -(1/(S*T_s)) * A_s * rho_t * [unclipped term is the min]
+    The min is taken as "unclipped <= clipped" (ties count as unclipped).
+    `n_seqs_total` overrides S in the 1/S factor when the rows given are only part of
+    a batch (used to score sampled sequences of a large batch).
+    """
+    logp = np.asarray(logp, dtype=np.float64)
+    old = np.asarray(old_logp, dtype=np.float64)
+    A = np.asarray(adv, dtype=np.float64)
+    cu = np.asarray(cu_seqlens, dtype=np.int64)
+    S = len(cu) - 1
+    S_norm = S if n_seqs_total is None else n_seqs_total
+    seq = _seq_of_token(cu)
+    T_s = np.diff(cu).astype(np.float64)
+    A_t = A[seq]
+    rho = np.exp(logp - old)
+    unclipped = rho * A_t
+    clipped = np.clip(rho, 1.0 - eps_low, 1.0 + eps_high) * A_t
+    u = np.minimum(unclipped, clipped)
+    active = (unclipped <= clipped).astype(np.float64)
+    seq_surr = np.zeros(S)
+    for s in range(S):
+        seq_surr[s] = u[cu[s]:cu[s + 1]].sum() / T_s[s]
+    loss = -seq_surr.sum() / S_norm
+    g = -(1.0 / (S_norm * T_s[seq])) * A_t * rho * active * grad_scale
+    return {"ratio": rho, "surr": u, "gscale": g, "seq_surr": seq_surr, "loss": loss,
+            "active": active}
+
+
+def policy_loss_fwd(hidden, W, ids, old_logp, adv, cu_seqlens, eps_low=0.2, eps_high=0.2,
+                    grad_scale=1.0) -> Dict[str, np.ndarray]:
+    """Forward of the policy loss: log-probs at the LM head, then the surrogate."""
+    lp = token_logprobs(hidden, W, ids)
+    out = surrogate_from_logp(lp["logp"], old_logp, adv, cu_seqlens, eps_low, eps_high,
+                              grad_scale)
+    out["logp"], out["lse"] = lp["logp"], lp["lse"]
+    return out
+
+
+def dlogits(hidden, W, ids, lse, gscale) -> np.ndarray:
+    """dz[t,v] = g_t * ( [v == ids_t] - exp(z[t,v] - lse_t) )."""
+    z = logits(hidden, W)
+    dz = -np.exp(z - np.asarray(lse, dtype=np.float64)[:, None])
+    dz[np.arange(z.shape[0]), np.asarray(ids, dtype=np.int64)] += 1.0
+    return dz * np.asarray(gscale, dtype=np.float64)[:, None]
+
+
+def policy_loss_bwd(hidden, W, ids, lse, gscale) -> Dict[str, np.ndarray]:
+    """dhidden[t,:] = sum_v dz[t,v] W[v,:];   dW[v,:] = sum_t dz[t,v] hidden[t,:]."""
+    dz = dlogits(hidden, W, ids, lse, gscale)
+    return {"dhidden": dz @ np.asarray(W, dtype=np.float64),
+            "dW": dz.T @ np.asarray(hidden, dtype=np.float64)}
+
+
+# --------------------------------------------------------------------------------------
+def policy_loss_fwd_bwd_rows(hidden, W, ids, old_logp, adv, cu_seqlens, eps_low=0.2,
+                             eps_high=0.2, grad_scale=1.0, rows_per_block: int = 1024,
+                             want_dW: bool = True) -> Dict[str, np.ndarray]:
+    """Same results as policy_loss_fwd + policy_loss_bwd, evaluated a block of token rows
+    at a time so that the [tokens x vocab] float64 logits never exceed a few GB of host
+    memory.  Rows are independent in every formula above except the sum over t in dW,
+    which is accumulated block by block; nothing else is reordered.
+    """
+    T = hidden.shape[0]
+    W64 = np.asarray(W, dtype=np.float64)
+    lse = np.zeros(T)
+    logp = np.zeros(T)
+    for a in range(0, T, rows_per_block):
+        b = min(T, a + rows_per_block)
+        lp = token_logprobs(hidden[a:b], W64, ids[a:b])
+        lse[a:b], logp[a:b] = lp["lse"], lp["logp"]
+    out = surrogate_from_logp(logp, old_logp, adv, cu_seqlens, eps_low, eps_high, grad_scale)
+    out["logp"], out["lse"] = logp, lse
+    dH = np.zeros((T, hidden.shape[1]))
+    dW = np.zeros_like(W64) if want_dW else None
+    for a in range(0, T, rows_per_block):
+        b = min(T, a + rows_per_block)
+        dz = dlogits(hidden[a:b], W64, ids[a:b], lse[a:b], out["gscale"][a:b])
+        dH[a:b] = dz @ W64
+        if want_dW:
+            dW += dz.T @ np.asarray(hidden[a:b], dtype=np.float64)
+    out["dhidden"], out["dW"] = dH, dW
+    return out
