@@ -311,5 +311,7 @@ def test_generator_recipes_have_the_stated_shapes():
     assert set(np.unique(b4.built.rewards)) <= {0.0, 0.5, 1.0}
     for f, J in ((0.0, 0), (0.25, 2), (0.5, 4), (0.75, 6)):
         assert gen.config(5, ext_fraction=f).J == J
-    x = np.array([1.0, 1.00390625, -3.140625, 1e-3], np.float32)
-    assert np.array_equal(gen.bf16_bits_to_f32(gen.f32_to_bf16_bits(x))[:3], x[:3])
+    x = np.array([1.0, 1.0078125, -3.140625], np.float32)          # exactly representable
+    assert np.array_equal(gen.bf16_bits_to_f32(gen.f32_to_bf16_bits(x)), x)
+    ties = np.array([1.00390625, 1.01171875], np.float32)          # halfway: round to even
+    assert gen.bf16_bits_to_f32(gen.f32_to_bf16_bits(ties)).tolist() == [1.0, 1.015625]
