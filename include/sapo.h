@@ -1,0 +1,207 @@
+/*
+ * sapo.h — C ABI of the SAPO policy-scoring library for NVIDIA B200 (sm_100a).
+ *
+ * One SAPO node's policy update (paper Algorithm 1, "Assemble training set" and
+ * "Policy update") scores a batch made of I locally generated and J swarm-sampled
+ * rollouts per question.  This library runs the data-parallel part of that update:
+ *
+ *   sapo_pack_rollouts     training set T^n = {local picks} U {external picks}
+ *                          (Section 3.2, training-set equation) as a varlen layout
+ *   sapo_group_advantages  GRPO group-relative advantages (Section 4.2)
+ *   sapo_policy_loss_fwd   LM-head log-probs of the chosen tokens (Section 3.2: rollouts
+ *                          are re-encoded and their token-level values computed under the
+ *                          node's own policy) + clipped-ratio surrogate, KL weight 0,
+ *                          separate lower/upper clip thresholds (Section 4.2)
+ *   sapo_policy_loss_bwd   gradient of that loss w.r.t. the final hidden states and the
+ *                          LM-head weight (Algorithm 1, PolicyGradient)
+ *
+ * General rules
+ *   - Every pointer is a DEVICE pointer unless its name starts with h_.  The caller owns
+ *     all buffers; the library allocates and frees nothing and keeps no pointer after a
+ *     call returns.  Scratch memory is passed in as `workspace`.
+ *   - Calls enqueue work on `stream` (a cudaStream_t passed as void*) and return without
+ *     synchronising.  Results are valid once the stream has drained.
+ *   - Return value: SAPO_OK or a negative host-detected error.  Conditions only the device
+ *     can see (capacity overflow, index out of range, a bounded wait that ran out) are
+ *     OR-ed as SAPO_ST_* bits into *status (int32 in device memory, zeroed by the caller);
+ *     the kernels never trap and never spin without a limit.
+ *   - Matrices are row-major with the H (hidden) index contiguous.  Base pointers of
+ *     hidden / W_head / dhidden / dW_head / workspace must be 16-byte aligned and the
+ *     leading dimensions, in bytes, multiples of 16.
+ *   - There is no CPU fallback: without a CUDA device every call returns SAPO_ERR_CUDA.
+ */
+#ifndef SAPO_H_
+#define SAPO_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* host-detected errors (return values) */
+#define SAPO_OK                      0
+#define SAPO_ERR_INVALID_ARG        -1
+#define SAPO_ERR_UNSUPPORTED_SHAPE  -2
+#define SAPO_ERR_WORKSPACE_TOO_SMALL -3
+#define SAPO_ERR_CUDA               -4
+
+/* device-detected conditions (bits of *status) */
+#define SAPO_ST_TOKEN_OVERFLOW   0x01  /* packed tokens exceed max_tokens; output truncated   */
+#define SAPO_ST_SEQ_OVERFLOW     0x02  /* selected sequences exceed max_seqs; nothing packed  */
+#define SAPO_ST_BAD_INDEX        0x04  /* a selection index is outside its rollout buffer     */
+#define SAPO_ST_EMPTY_SEQUENCE   0x08  /* a selected rollout has no tokens                    */
+#define SAPO_ST_BAD_TOKEN_ID     0x10  /* ids[t] outside [0, V): token scored as masked       */
+#define SAPO_ST_WAIT_TIMEOUT     0x20  /* a bounded in-kernel wait ran out; results invalid   */
+#define SAPO_ST_NONFINITE_REWARD 0x40  /* a reward is NaN or infinite                         */
+
+/* element types of hidden / W_head */
+#define SAPO_DTYPE_BF16 0
+#define SAPO_DTYPE_F32  1  /* converted on the device to split bf16; see sapo_policy_loss_fwd */
+
+/* `which` of sapo_workspace_bytes */
+#define SAPO_WS_FWD 0
+#define SAPO_WS_BWD 1
+
+/* A rollout store: n_rollouts completions laid end to end (Section 3.1: a node's answers
+ * to its questions; Section 3.2: the tuples other nodes broadcast).
+ *   hidden   [n_tokens, H]  final hidden state at the position that predicts ids[t]
+ *   ids      [n_tokens]     chosen token
+ *   old_logp [n_tokens]     log-prob of ids[t] under the pre-update policy
+ *   offsets  [n_rollouts+1] token offset of each completion (offsets[0] = 0)
+ *   rewards  [n_rollouts]   reward of each completion */
+typedef struct sapo_rollout_buf {
+  const void*    hidden;
+  const int32_t* ids;
+  const float*   old_logp;
+  const int64_t* offsets;
+  const float*   rewards;
+  int32_t        n_rollouts;
+} sapo_rollout_buf;
+
+/* Which rollouts enter the training set: for question q the local picks are
+ * local_idx[q_offsets_local[q] .. q_offsets_local[q+1]) and the external picks
+ * ext_idx[q_offsets_ext[q] .. q_offsets_ext[q+1]).  Either side may be empty. */
+typedef struct sapo_selection {
+  const int32_t* q_offsets_local;  /* [Q+1] */
+  const int32_t* local_idx;
+  const int32_t* q_offsets_ext;    /* [Q+1] */
+  const int32_t* ext_idx;
+  int32_t        Q;
+} sapo_selection;
+
+/* Output of sapo_pack_rollouts.  Capacities max_tokens / max_seqs are set by the caller.
+ *   hidden [max_tokens, H], ids, old_logp [max_tokens], rewards [max_seqs]
+ *   cu_seqlens [max_seqs+1] exclusive prefix sum of sequence lengths
+ *   seq_group [max_seqs] question of each sequence;  seq_is_ext [max_seqs] 0 local / 1 external
+ *   seq_src [max_seqs] index of the rollout inside its buffer
+ *   tok_seq [max_tokens] sequence of each token;  tok_mask [max_tokens] 1 for t < T else 0
+ *   group_offsets [Q+1] first sequence of each question
+ *   n_tokens, n_seqs: device scalars T and S */
+typedef struct sapo_packed {
+  void*    hidden;
+  int32_t* ids;
+  float*   old_logp;
+  float*   rewards;
+  int32_t* cu_seqlens;
+  int32_t* seq_group;
+  uint8_t* seq_is_ext;
+  int32_t* seq_src;
+  int32_t* tok_seq;
+  uint8_t* tok_mask;
+  int32_t* group_offsets;
+  int32_t* n_tokens;
+  int32_t* n_seqs;
+  int64_t  max_tokens;
+  int32_t  max_seqs;
+} sapo_packed;
+
+/* Loss parameters.  The paper's run uses eps_low 0.2, eps_high 0.28 and no KL term
+ * (Section 4.2).  grad_scale multiplies the per-token gradient factor (upstream dL). */
+typedef struct sapo_loss_cfg {
+  float eps_low;
+  float eps_high;
+  float grad_scale;
+} sapo_loss_cfg;
+
+/* Section 3.2, training-set equation / Algorithm 1 "Assemble training set".
+ * Gathers the selected rollouts into one token-major batch.  Sequence order: questions in
+ * order; inside a question its local picks in list order, then its external picks in list
+ * order.  Copies are byte-exact.  H is the row width in elements, `dtype` a SAPO_DTYPE_*.
+ * Errors: a NULL struct or negative size returns SAPO_ERR_INVALID_ARG; a bad index, an
+ * empty rollout or a capacity overflow sets the matching status bit (bad or empty picks are
+ * packed as length-0 sequences, tokens beyond max_tokens are dropped). */
+int sapo_pack_rollouts(const sapo_rollout_buf* h_local, const sapo_rollout_buf* h_ext,
+                       const sapo_selection* h_sel, int32_t H, int32_t dtype,
+                       const sapo_packed* h_out, int32_t* status, void* stream);
+
+/* Section 4.2 (GRPO): for each question g with members group_offsets[g]..group_offsets[g+1):
+ *   mean_g = average reward, std_g = sqrt(sum (r-mean_g)^2 / (G - ddof)),
+ *   adv[s] = (rewards[s] - mean_g) / (std_g + adv_eps).
+ * The group covers all its completions, local and external alike.  Accumulates in fp64,
+ * stores fp32.  mean / std may be NULL.  A non-finite reward sets SAPO_ST_NONFINITE_REWARD. */
+int sapo_group_advantages(const float* rewards, const int32_t* group_offsets, int32_t Q,
+                          float adv_eps, int32_t ddof, float* adv, float* mean, float* std,
+                          int32_t* status, void* stream);
+
+/* Section 3.2 (token-level values under the node's own policy) + Section 4.2 (clipped
+ * surrogate, KL weight 0).  For T packed tokens in S sequences:
+ *   z[t,v] = <hidden[t,:], W_head[v,:]>,  lse[t] = log sum_v exp z[t,v],
+ *   logp[t] = z[t, ids[t]] - lse[t],      ratio[t] = exp(logp[t] - old_logp[t]),
+ *   surr[t] = min(ratio*A, clip(ratio, 1-eps_low, 1+eps_high)*A),  A = adv[seq of t],
+ *   loss    = -(1/S) sum_s (1/T_s) sum_{t in s} surr[t],
+ *   gscale[t] = dloss/dlogp[t] = -grad_scale * A * ratio / (S*T_s) where the unclipped term
+ *               is the min (ties included), else 0.
+ * The [T,V] logits are never written to memory: the projection runs on the tensor cores and
+ * its epilogue keeps a running max / sum-exp / target logit per token.
+ * hidden [T, ld_hidden], W_head [V, ld_W] of `dtype`; for SAPO_DTYPE_F32 the operands are
+ * split on the device into bf16 high and low parts (3 products), which keeps log-probs at
+ * fp32 accuracy.  adv [S], cu_seqlens [S+1].  Outputs logp, lse, ratio, surr, gscale [T]
+ * and loss [1] (float32); seq_surr [S] (token-mean surrogate per sequence) may be NULL.
+ * workspace: at least sapo_workspace_bytes(SAPO_WS_FWD, ...) bytes.
+ * Errors: bad arguments / unaligned pointers -> SAPO_ERR_INVALID_ARG; H or V beyond the
+ * supported range -> SAPO_ERR_UNSUPPORTED_SHAPE; small workspace ->
+ * SAPO_ERR_WORKSPACE_TOO_SMALL; ids outside [0,V) -> SAPO_ST_BAD_TOKEN_ID and the token
+ * gets logp = 0 contribution (surr = gscale = 0). */
+int sapo_policy_loss_fwd(const void* hidden, const void* W_head, int32_t dtype,
+                         int64_t T, int32_t H, int32_t V, int64_t ld_hidden, int64_t ld_W,
+                         const int32_t* ids, const float* old_logp, const float* adv,
+                         const int32_t* cu_seqlens, int32_t S, const sapo_loss_cfg* h_cfg,
+                         float* logp, float* lse, float* ratio, float* surr, float* gscale,
+                         float* seq_surr, float* loss,
+                         void* workspace, size_t workspace_bytes,
+                         int32_t* status, void* stream);
+
+/* Algorithm 1 "Policy update" (gradient of the loss above through the LM head):
+ *   dz[t,v]      = gscale[t] * ([v == ids[t]] - exp(z[t,v] - lse[t]))
+ *   dhidden[t,:] = sum_v dz[t,v] W_head[v,:]        float32 [T, H]
+ *   dW_head[v,:] = sum_t dz[t,v] hidden[t,:]        float32 [V, H]
+ * Logit tiles are recomputed on the tensor cores; dz is rounded to bf16 and kept in a
+ * bounded panel inside `workspace` (token chunks x padded vocab), from which two tensor-core
+ * contractions form dhidden and dW_head.  accumulate_dW != 0 adds into dW_head instead of
+ * overwriting it.  lse and gscale come from sapo_policy_loss_fwd.  For SAPO_DTYPE_F32 the
+ * operands are rounded to bf16.
+ * workspace: sapo_workspace_bytes(SAPO_WS_BWD, ...) is the preferred size; any size down to
+ * the one for 128 tokens works (smaller panels mean more passes over dW_head). */
+int sapo_policy_loss_bwd(const void* hidden, const void* W_head, int32_t dtype,
+                         int64_t T, int32_t H, int32_t V, int64_t ld_hidden, int64_t ld_W,
+                         const int32_t* ids, const float* lse, const float* gscale,
+                         float* dhidden, float* dW_head, int32_t accumulate_dW,
+                         void* workspace, size_t workspace_bytes,
+                         int32_t* status, void* stream);
+
+/* Bytes of scratch the forward (SAPO_WS_FWD) or backward (SAPO_WS_BWD) call wants for
+ * these sizes.  Returns 0 for invalid arguments. */
+size_t sapo_workspace_bytes(int32_t which, int64_t T, int32_t H, int32_t V, int32_t dtype);
+
+/* Smallest backward workspace that still works (one 128-token panel). */
+size_t sapo_workspace_bytes_min(int32_t which, int64_t T, int32_t H, int32_t V, int32_t dtype);
+
+/* Text for a return code. */
+const char* sapo_status_string(int32_t code);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SAPO_H_ */

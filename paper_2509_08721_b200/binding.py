@@ -1,0 +1,241 @@
+"""ctypes binding of the SAPO B200 library: same names as the C ABI, argument marshalling
+only.  torch supplies device memory and the current stream; every step of the path runs in
+the library's CUDA kernels.  There is no fallback: if the shared library is missing or no
+CUDA device is present, calls raise.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from dataclasses import dataclass
+from typing import Dict, Optional
+
+import torch
+
+from . import build as _build
+
+DTYPE_BF16 = 0
+DTYPE_F32 = 1
+WS_FWD = 0
+WS_BWD = 1
+
+ST_BITS = {
+    0x01: "TOKEN_OVERFLOW", 0x02: "SEQ_OVERFLOW", 0x04: "BAD_INDEX", 0x08: "EMPTY_SEQUENCE",
+    0x10: "BAD_TOKEN_ID", 0x20: "WAIT_TIMEOUT", 0x40: "NONFINITE_REWARD",
+}
+
+EXPORTS = ("sapo_pack_rollouts", "sapo_group_advantages", "sapo_policy_loss_fwd",
+           "sapo_policy_loss_bwd", "sapo_workspace_bytes", "sapo_workspace_bytes_min",
+           "sapo_status_string")
+
+
+class RolloutBufC(C.Structure):
+    _fields_ = [("hidden", C.c_void_p), ("ids", C.c_void_p), ("old_logp", C.c_void_p),
+                ("offsets", C.c_void_p), ("rewards", C.c_void_p), ("n_rollouts", C.c_int32)]
+
+
+class SelectionC(C.Structure):
+    _fields_ = [("q_offsets_local", C.c_void_p), ("local_idx", C.c_void_p),
+                ("q_offsets_ext", C.c_void_p), ("ext_idx", C.c_void_p), ("Q", C.c_int32)]
+
+
+class PackedC(C.Structure):
+    _fields_ = [("hidden", C.c_void_p), ("ids", C.c_void_p), ("old_logp", C.c_void_p),
+                ("rewards", C.c_void_p), ("cu_seqlens", C.c_void_p), ("seq_group", C.c_void_p),
+                ("seq_is_ext", C.c_void_p), ("seq_src", C.c_void_p), ("tok_seq", C.c_void_p),
+                ("tok_mask", C.c_void_p), ("group_offsets", C.c_void_p), ("n_tokens", C.c_void_p),
+                ("n_seqs", C.c_void_p), ("max_tokens", C.c_int64), ("max_seqs", C.c_int32)]
+
+
+class LossCfgC(C.Structure):
+    _fields_ = [("eps_low", C.c_float), ("eps_high", C.c_float), ("grad_scale", C.c_float)]
+
+
+_lib: Optional[C.CDLL] = None
+
+
+def lib_path() -> str:
+    return _build.LIB
+
+
+def load() -> C.CDLL:
+    """Load (building first if the sources are newer) and type the C ABI."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    path = _build.LIB
+    if not os.path.exists(path):
+        path = _build.build()
+    lib = C.CDLL(path)
+    vp, i32, i64, f32, sz = C.c_void_p, C.c_int32, C.c_int64, C.c_float, C.c_size_t
+    lib.sapo_pack_rollouts.restype = C.c_int
+    lib.sapo_pack_rollouts.argtypes = [C.POINTER(RolloutBufC), C.POINTER(RolloutBufC),
+                                       C.POINTER(SelectionC), i32, i32, C.POINTER(PackedC), vp, vp]
+    lib.sapo_group_advantages.restype = C.c_int
+    lib.sapo_group_advantages.argtypes = [vp, vp, i32, f32, i32, vp, vp, vp, vp, vp]
+    lib.sapo_policy_loss_fwd.restype = C.c_int
+    lib.sapo_policy_loss_fwd.argtypes = [vp, vp, i32, i64, i32, i32, i64, i64, vp, vp, vp, vp, i32,
+                                         C.POINTER(LossCfgC), vp, vp, vp, vp, vp, vp, vp, vp, sz,
+                                         vp, vp]
+    lib.sapo_policy_loss_bwd.restype = C.c_int
+    lib.sapo_policy_loss_bwd.argtypes = [vp, vp, i32, i64, i32, i32, i64, i64, vp, vp, vp, vp, vp,
+                                         i32, vp, sz, vp, vp]
+    lib.sapo_workspace_bytes.restype = sz
+    lib.sapo_workspace_bytes.argtypes = [i32, i64, i32, i32, i32]
+    lib.sapo_workspace_bytes_min.restype = sz
+    lib.sapo_workspace_bytes_min.argtypes = [i32, i64, i32, i32, i32]
+    lib.sapo_status_string.restype = C.c_char_p
+    lib.sapo_status_string.argtypes = [i32]
+    _lib = lib
+    return lib
+
+
+class SapoError(RuntimeError):
+    pass
+
+
+def _check(rc: int, what: str) -> None:
+    if rc != 0:
+        raise SapoError(f"{what}: {load().sapo_status_string(rc).decode()} ({rc})")
+
+
+def _require_cuda() -> None:
+    if not torch.cuda.is_available():
+        raise SapoError("the SAPO B200 library needs a CUDA device; there is no CPU path")
+
+
+def _p(t: Optional[torch.Tensor]) -> Optional[int]:
+    return None if t is None else t.data_ptr()
+
+
+def _stream() -> int:
+    return torch.cuda.current_stream().cuda_stream
+
+
+def _dtype_code(t: torch.Tensor) -> int:
+    if t.dtype == torch.bfloat16:
+        return DTYPE_BF16
+    if t.dtype == torch.float32:
+        return DTYPE_F32
+    raise SapoError(f"unsupported element type {t.dtype}")
+
+
+def decode_status(word: int):
+    return [name for bit, name in ST_BITS.items() if word & bit]
+
+
+def new_status(device="cuda") -> torch.Tensor:
+    return torch.zeros(1, dtype=torch.int32, device=device)
+
+
+# ------------------------------------------------------------------------------------------
+@dataclass
+class DeviceRollouts:
+    """Device-resident rollout buffer (tensors named as in the C struct)."""
+    hidden: torch.Tensor
+    ids: torch.Tensor
+    old_logp: torch.Tensor
+    offsets: torch.Tensor
+    rewards: torch.Tensor
+
+    def c(self) -> RolloutBufC:
+        return RolloutBufC(_p(self.hidden), _p(self.ids), _p(self.old_logp), _p(self.offsets),
+                           _p(self.rewards), int(self.offsets.numel() - 1))
+
+
+@dataclass
+class DeviceSelection:
+    q_offsets_local: torch.Tensor
+    local_idx: torch.Tensor
+    q_offsets_ext: torch.Tensor
+    ext_idx: torch.Tensor
+
+    def c(self) -> SelectionC:
+        return SelectionC(_p(self.q_offsets_local), _p(self.local_idx), _p(self.q_offsets_ext),
+                          _p(self.ext_idx), int(self.q_offsets_local.numel() - 1))
+
+
+def alloc_packed(max_tokens: int, max_seqs: int, Q: int, H: int, dtype: torch.dtype,
+                 device="cuda") -> Dict[str, torch.Tensor]:
+    i32, f32, u8 = torch.int32, torch.float32, torch.uint8
+    e = lambda *s, dt: torch.empty(*s, dtype=dt, device=device)
+    return {
+        "hidden": e(max_tokens, H, dt=dtype), "ids": e(max_tokens, dt=i32),
+        "old_logp": e(max_tokens, dt=f32), "rewards": e(max_seqs, dt=f32),
+        "cu_seqlens": e(max_seqs + 1, dt=i32), "seq_group": e(max_seqs, dt=i32),
+        "seq_is_ext": e(max_seqs, dt=u8), "seq_src": e(max_seqs, dt=i32),
+        "tok_seq": e(max_tokens, dt=i32), "tok_mask": e(max_tokens, dt=u8),
+        "group_offsets": e(Q + 1, dt=i32), "n_tokens": e(1, dt=i32), "n_seqs": e(1, dt=i32),
+    }
+
+
+def sapo_pack_rollouts(local: DeviceRollouts, ext: DeviceRollouts, sel: DeviceSelection,
+                       out: Dict[str, torch.Tensor], status: torch.Tensor) -> None:
+    """Enqueue the pack on the current stream; `out` comes from alloc_packed."""
+    _require_cuda()
+    H = int(out["hidden"].shape[1])
+    pc = PackedC(*[_p(out[k]) for k in ("hidden", "ids", "old_logp", "rewards", "cu_seqlens",
+                                        "seq_group", "seq_is_ext", "seq_src", "tok_seq", "tok_mask",
+                                        "group_offsets", "n_tokens", "n_seqs")],
+                 int(out["ids"].numel()), int(out["seq_group"].numel()))
+    lc, ec, sc = local.c(), ext.c(), sel.c()
+    rc = load().sapo_pack_rollouts(C.byref(lc), C.byref(ec), C.byref(sc), H,
+                                   _dtype_code(out["hidden"]), C.byref(pc), _p(status), _stream())
+    _check(rc, "sapo_pack_rollouts")
+
+
+def sapo_group_advantages(rewards: torch.Tensor, group_offsets: torch.Tensor, adv_eps: float,
+                          ddof: int, adv: torch.Tensor, mean: Optional[torch.Tensor],
+                          std: Optional[torch.Tensor], status: torch.Tensor) -> None:
+    _require_cuda()
+    rc = load().sapo_group_advantages(_p(rewards), _p(group_offsets), int(group_offsets.numel() - 1),
+                                      float(adv_eps), int(ddof), _p(adv), _p(mean), _p(std),
+                                      _p(status), _stream())
+    _check(rc, "sapo_group_advantages")
+
+
+def sapo_workspace_bytes(which: int, T: int, H: int, V: int, dtype: int) -> int:
+    return int(load().sapo_workspace_bytes(which, T, H, V, dtype))
+
+
+def sapo_workspace_bytes_min(which: int, T: int, H: int, V: int, dtype: int) -> int:
+    return int(load().sapo_workspace_bytes_min(which, T, H, V, dtype))
+
+
+def alloc_fwd_outputs(T: int, S: int, device="cuda") -> Dict[str, torch.Tensor]:
+    f = lambda n: torch.empty(n, dtype=torch.float32, device=device)
+    return {"logp": f(T), "lse": f(T), "ratio": f(T), "surr": f(T), "gscale": f(T),
+            "seq_surr": f(S), "loss": f(1)}
+
+
+def sapo_policy_loss_fwd(hidden: torch.Tensor, W_head: torch.Tensor, ids: torch.Tensor,
+                         old_logp: torch.Tensor, adv: torch.Tensor, cu_seqlens: torch.Tensor,
+                         eps_low: float, eps_high: float, grad_scale: float,
+                         out: Dict[str, torch.Tensor], workspace: torch.Tensor,
+                         status: torch.Tensor, T: Optional[int] = None) -> None:
+    _require_cuda()
+    T = int(hidden.shape[0]) if T is None else int(T)
+    H, V = int(hidden.shape[1]), int(W_head.shape[0])
+    S = int(cu_seqlens.numel() - 1)
+    cfg = LossCfgC(eps_low, eps_high, grad_scale)
+    rc = load().sapo_policy_loss_fwd(
+        _p(hidden), _p(W_head), _dtype_code(hidden), T, H, V, hidden.stride(0), W_head.stride(0),
+        _p(ids), _p(old_logp), _p(adv), _p(cu_seqlens), S, C.byref(cfg),
+        _p(out["logp"]), _p(out["lse"]), _p(out["ratio"]), _p(out["surr"]), _p(out["gscale"]),
+        _p(out.get("seq_surr")), _p(out["loss"]), _p(workspace), workspace.numel() * workspace.element_size(),
+        _p(status), _stream())
+    _check(rc, "sapo_policy_loss_fwd")
+
+
+def sapo_policy_loss_bwd(hidden: torch.Tensor, W_head: torch.Tensor, ids: torch.Tensor,
+                         lse: torch.Tensor, gscale: torch.Tensor, dhidden: torch.Tensor,
+                         dW_head: torch.Tensor, accumulate_dW: bool, workspace: torch.Tensor,
+                         status: torch.Tensor, T: Optional[int] = None) -> None:
+    _require_cuda()
+    T = int(hidden.shape[0]) if T is None else int(T)
+    H, V = int(hidden.shape[1]), int(W_head.shape[0])
+    rc = load().sapo_policy_loss_bwd(
+        _p(hidden), _p(W_head), _dtype_code(hidden), T, H, V, hidden.stride(0), W_head.stride(0),
+        _p(ids), _p(lse), _p(gscale), _p(dhidden), _p(dW_head), 1 if accumulate_dW else 0,
+        _p(workspace), workspace.numel() * workspace.element_size(), _p(status), _stream())
+    _check(rc, "sapo_policy_loss_bwd")

@@ -1,0 +1,704 @@
+// LM-head projection fused with the policy loss, forward and backward, on the Blackwell
+// tensor cores (tcgen05 MMA, accumulators in tensor memory, operands staged by TMA).
+//
+// One persistent, warp-specialised GEMM kernel (128 x 256 output tiles, 64-deep K blocks)
+// serves four contractions; they differ only in operand majors and in the epilogue that
+// drains the accumulator:
+//   forward      S = hidden . W^T      epilogue: running max / sum-exp / target logit per token
+//   backward dz  S = hidden . W^T      epilogue: dz = g (onehot - exp(S - lse)) -> bf16 panel
+//   backward dH  dH = dz . W           epilogue: fp32 store
+//   backward dW  dW = dz^T . hidden    epilogue: fp32 store / accumulate
+// The [tokens x vocab] logits never reach global memory (paper Section 3.2 asks for the
+// token-level values of every rollout under the node's policy; Section 4.2 gives the
+// clipped objective the epilogue tail evaluates).
+#include <cuda.h>
+#include <cuda_bf16.h>
+
+#include "common.cuh"
+#include "umma.cuh"
+
+namespace sapo {
+using namespace umma;
+
+constexpr int BM = 128;            // accumulator rows  (TMEM lanes)
+constexpr int BN = 256;            // accumulator columns per tile
+constexpr int BK = 64;             // bf16 elements per 128-byte operand row
+constexpr int UMMA_K = 16;
+constexpr int STAGES = 4;
+constexpr int GEMM_THREADS = 192;  // warp 0: TMA, warp 1: MMA, warps 2-5: epilogue
+constexpr uint32_t A_STAGE_BYTES = BM * 128;
+constexpr uint32_t B_STAGE_BYTES = BN * 128;
+constexpr uint32_t CHUNK_BYTES = 64 * 128;   // one 64-row box of an MN-major operand
+constexpr uint32_t TMEM_COLS = 512;          // two accumulators of 256 columns
+constexpr size_t GEMM_SMEM_BYTES = 1024 + STAGES * (A_STAGE_BYTES + B_STAGE_BYTES) + 256;
+constexpr float LOG2E = 1.4426950408889634f;
+constexpr float LN2 = 0.6931471805599453f;
+
+// Static tile schedule: `num_units` work units, each one m-block and a run of n-blocks.
+struct Sched {
+  int32_t num_m_blocks, num_n_blocks, n_per_unit, units_per_m, num_units, num_k_blocks;
+  int32_t m_fastest;  // 1: neighbouring CTAs share the B tile; 0: they share the A tile
+  int32_t N;          // true extent of the n dimension (tail tiles use a narrower MMA)
+};
+
+__device__ __forceinline__ void decode_unit(const Sched& s, int unit, int& mb, int& un,
+                                            int& n_begin, int& n_end) {
+  if (s.m_fastest) { un = unit / s.num_m_blocks; mb = unit - un * s.num_m_blocks; }
+  else             { mb = unit / s.units_per_m;  un = unit - mb * s.units_per_m; }
+  n_begin = un * s.n_per_unit;
+  n_end = min(n_begin + s.n_per_unit, s.num_n_blocks);
+}
+
+// columns of a tile that hold real outputs, rounded up to the MMA's granularity of 16
+__device__ __forceinline__ int tile_n_eff(const Sched& s, int nb) {
+  const int left = s.N - nb * BN;
+  return left >= BN ? BN : ((left + 15) & ~15);
+}
+
+// ---------------------------------------------------------------------------- epilogues
+// Each epilogue thread owns one accumulator row (TMEM lane) of the tile.
+
+// Forward: online log-sum-exp in the base-2 domain plus the logit of the chosen token.
+struct FwdEpi {
+  struct Params {
+    const int32_t* ids; float* pm; float* ps; float* pz;  // partials [n_splits][T]
+    int64_t T; int32_t V;
+  };
+  float m, s, zy; int32_t y; int64_t row;
+  __device__ __forceinline__ void begin_unit(const Params& p, int mb, int r) {
+    row = (int64_t)mb * BM + r;
+    m = -INFINITY; s = 0.f; zy = 0.f;
+    y = row < p.T ? p.ids[row] : -1;
+  }
+  __device__ __forceinline__ void chunk(const Params& p, float (&v)[32], int col0) {
+    if (col0 >= p.V) return;
+    if (col0 + 32 > p.V) {
+      #pragma unroll
+      for (int j = 0; j < 32; ++j) if (col0 + j >= p.V) v[j] = -INFINITY;
+    }
+    const int yr = y - col0;
+    if (yr >= 0 && yr < 32) {
+      #pragma unroll
+      for (int j = 0; j < 32; ++j) if (j == yr) zy = v[j];
+    }
+    float cmax = v[0];
+    #pragma unroll
+    for (int j = 1; j < 32; ++j) cmax = fmaxf(cmax, v[j]);
+    const float m_new = fmaxf(m, cmax * LOG2E);
+    float acc = s * ex2(m - m_new);          // first chunk: ex2(-inf) = 0
+    #pragma unroll
+    for (int j = 0; j < 32; ++j) acc += ex2(fmaf(v[j], LOG2E, -m_new));
+    s = acc; m = m_new;
+  }
+  __device__ __forceinline__ void end_unit(const Params& p, int un) {
+    if (row < p.T) {
+      const int64_t o = (int64_t)un * p.T + row;
+      p.pm[o] = m; p.ps[o] = s; p.pz[o] = zy;
+    }
+  }
+};
+
+// Backward, first contraction: dz[t,v] = g_t ([v == y_t] - exp(z[t,v] - lse_t)), to bf16.
+struct DzEpi {
+  struct Params {
+    const int32_t* ids; const float* lse; const float* gscale; __nv_bfloat16* P;
+    int64_t M; int32_t V; int64_t Vp;   // panel [M, Vp], Vp a multiple of 64
+  };
+  float g, l2; int32_t y; int64_t row; bool valid;
+  __device__ __forceinline__ void begin_unit(const Params& p, int mb, int r) {
+    row = (int64_t)mb * BM + r;
+    valid = row < p.M;
+    g = valid ? p.gscale[row] : 0.f;
+    l2 = valid ? p.lse[row] * LOG2E : 0.f;
+    y = valid ? p.ids[row] : -1;
+  }
+  __device__ __forceinline__ void chunk(const Params& p, float (&v)[32], int col0) {
+    if (!valid || col0 >= p.Vp) return;
+    uint32_t packed[16];
+    if (g == 0.f) {
+      #pragma unroll
+      for (int j = 0; j < 16; ++j) packed[j] = 0u;
+    } else {
+      const float ng = -g;
+      #pragma unroll
+      for (int j = 0; j < 32; ++j) {
+        float d = ng * ex2(fmaf(v[j], LOG2E, -l2));
+        if (col0 + j == y) d += g;
+        if (col0 + j >= p.V) d = 0.f;
+        v[j] = d;
+      }
+      #pragma unroll
+      for (int j = 0; j < 16; ++j) {
+        __nv_bfloat162 h = __floats2bfloat162_rn(v[2 * j], v[2 * j + 1]);
+        packed[j] = *reinterpret_cast<uint32_t*>(&h);
+      }
+    }
+    uint4* dst = reinterpret_cast<uint4*>(p.P + row * p.Vp + col0);
+    #pragma unroll
+    for (int q = 0; q < 4; ++q)
+      dst[q] = make_uint4(packed[4 * q], packed[4 * q + 1], packed[4 * q + 2], packed[4 * q + 3]);
+  }
+  __device__ __forceinline__ void end_unit(const Params&, int) {}
+};
+
+// Plain fp32 output tile, optionally added to what is already there.
+struct StoreEpi {
+  struct Params { float* C; int64_t ldc; int64_t M; int32_t N; int32_t accumulate; };
+  int64_t row; bool valid;
+  __device__ __forceinline__ void begin_unit(const Params& p, int mb, int r) {
+    row = (int64_t)mb * BM + r;
+    valid = row < p.M;
+  }
+  __device__ __forceinline__ void chunk(const Params& p, float (&v)[32], int col0) {
+    if (!valid) return;
+    float4* dst = reinterpret_cast<float4*>(p.C + row * p.ldc + col0);
+    #pragma unroll
+    for (int q = 0; q < 8; ++q) {
+      if (col0 + 4 * q < p.N) {          // N is a multiple of 4
+        float4 o = make_float4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
+        if (p.accumulate) { const float4 c = dst[q]; o.x += c.x; o.y += c.y; o.z += c.z; o.w += c.w; }
+        dst[q] = o;
+      }
+    }
+  }
+  __device__ __forceinline__ void end_unit(const Params&, int) {}
+};
+
+// ---------------------------------------------------------------------------- the GEMM kernel
+// D[m, n] = sum_k A[m, k] * B[n, k].
+//   A_MN = false: A is stored [M, K] with K contiguous; map box {64 k, 128 m}
+//   A_MN = true : A is stored [K, M] with M contiguous; map box {64 m, 64 k}, two boxes per stage
+//   B likewise with N in place of M (256 rows, or four 64-wide boxes).
+template <bool A_MN, bool B_MN, class Epi>
+__global__ void __launch_bounds__(GEMM_THREADS, 1)
+umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+                 const Sched sched, const typename Epi::Params ep, int32_t* status) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  uint8_t* smem_a = smem;
+  uint8_t* smem_b = smem + STAGES * A_STAGE_BYTES;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + STAGES * (A_STAGE_BYTES + B_STAGE_BYTES));
+  uint64_t* full = bars;                 // [STAGES] TMA -> MMA
+  uint64_t* empty = bars + STAGES;       // [STAGES] MMA -> TMA
+  uint64_t* acc_full = bars + 2 * STAGES;      // [2] MMA -> epilogue
+  uint64_t* acc_empty = bars + 2 * STAGES + 2; // [2] epilogue -> MMA
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * STAGES + 4);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < STAGES; ++i) { mbar_init(&full[i], 1); mbar_init(&empty[i], 1); }
+    for (int i = 0; i < 2; ++i) { mbar_init(&acc_full[i], 1); mbar_init(&acc_empty[i], 128); }
+    *abort_flag = 0;
+    fence_mbar_init();
+    prefetch_tensormap(&map_a);
+    prefetch_tensormap(&map_b);
+  }
+  if (warp == 1) { tmem_alloc(tmem_slot, TMEM_COLS); tmem_relinquish(); }
+  fence_before_sync();
+  __syncthreads();
+  fence_after_sync();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0 && lane == 0) {
+    // ------------------------------------------------------------ TMA producer
+    int stage = 0; uint32_t phase = 0;
+    uint32_t in_flight = 0;   // bit i: stage i was filled in the current ring pass
+    bool ok = true;
+    for (int unit = blockIdx.x; ok && unit < sched.num_units; unit += gridDim.x) {
+      int mb, un, n_begin, n_end;
+      decode_unit(sched, unit, mb, un, n_begin, n_end);
+      for (int nb = n_begin; ok && nb < n_end; ++nb) {
+        const int n_eff = tile_n_eff(sched, nb);
+        const int b_chunks = (n_eff + 63) >> 6;
+        const uint32_t tx = A_STAGE_BYTES + (B_MN ? b_chunks * CHUNK_BYTES : B_STAGE_BYTES);
+        for (int kb = 0; kb < sched.num_k_blocks; ++kb) {
+          if (!mbar_wait(&empty[stage], phase ^ 1, abort_flag)) { ok = false; break; }
+          mbar_arrive_expect_tx(&full[stage], tx);
+          uint8_t* sa = smem_a + stage * A_STAGE_BYTES;
+          uint8_t* sb = smem_b + stage * B_STAGE_BYTES;
+          if (A_MN) {
+            tma_load_2d(sa, &map_a, &full[stage], mb * BM, kb * BK);
+            tma_load_2d(sa + CHUNK_BYTES, &map_a, &full[stage], mb * BM + 64, kb * BK);
+          } else {
+            tma_load_2d(sa, &map_a, &full[stage], kb * BK, mb * BM);
+          }
+          if (B_MN) {
+            for (int c = 0; c < b_chunks; ++c)
+              tma_load_2d(sb + c * CHUNK_BYTES, &map_b, &full[stage], nb * BN + 64 * c, kb * BK);
+          } else {
+            tma_load_2d(sb, &map_b, &full[stage], kb * BK, nb * BN);
+          }
+          in_flight |= 1u << stage;
+          if (++stage == STAGES) { stage = 0; phase ^= 1; }
+        }
+      }
+    }
+    if (!ok) {
+      // give copies already issued a bounded chance to land before the CTA leaves
+      for (int i = 0; i < STAGES; ++i) {
+        if (!(in_flight & (1u << i))) continue;
+        const uint32_t ph = (i < stage) ? phase : (phase ^ 1);
+        for (int spin = 0; spin < (1 << 20) && !mbar_try_wait(&full[i], ph); ++spin) {}
+      }
+    }
+  } else if (warp == 1 && lane == 0) {
+    // ------------------------------------------------------------ MMA issuer
+    int stage = 0; uint32_t phase = 0;
+    int acc = 0; uint32_t acc_phase = 0;
+    bool ok = true;
+    for (int unit = blockIdx.x; ok && unit < sched.num_units; unit += gridDim.x) {
+      int mb, un, n_begin, n_end;
+      decode_unit(sched, unit, mb, un, n_begin, n_end);
+      for (int nb = n_begin; ok && nb < n_end; ++nb) {
+        const uint32_t idesc = make_idesc_bf16(BM, tile_n_eff(sched, nb), A_MN, B_MN);
+        if (!mbar_wait(&acc_empty[acc], acc_phase ^ 1, abort_flag)) { ok = false; break; }
+        fence_after_sync();
+        const uint32_t d_tmem = tmem_base + acc * BN;
+        for (int kb = 0; kb < sched.num_k_blocks; ++kb) {
+          if (!mbar_wait(&full[stage], phase, abort_flag)) { ok = false; break; }
+          fence_after_sync();
+          const uint32_t a_addr = smem_u32(smem_a + stage * A_STAGE_BYTES);
+          const uint32_t b_addr = smem_u32(smem_b + stage * B_STAGE_BYTES);
+          #pragma unroll
+          for (int k = 0; k < BK / UMMA_K; ++k) {
+            // K-major: 16 elements = 32 bytes along the row; MN-major: 16 rows = 2048 bytes
+            const uint64_t a_desc = A_MN ? make_smem_desc(a_addr + k * 2048, CHUNK_BYTES, 1024)
+                                         : make_smem_desc(a_addr + k * 32, 16, 1024);
+            const uint64_t b_desc = B_MN ? make_smem_desc(b_addr + k * 2048, CHUNK_BYTES, 1024)
+                                         : make_smem_desc(b_addr + k * 32, 16, 1024);
+            mma_bf16(d_tmem, a_desc, b_desc, idesc, (kb | k) != 0 ? 1u : 0u);
+          }
+          mma_commit(&empty[stage]);              // frees the stage once these MMAs retire
+          if (++stage == STAGES) { stage = 0; phase ^= 1; }
+        }
+        if (ok) mma_commit(&acc_full[acc]);       // accumulator complete
+        if (++acc == 2) { acc = 0; acc_phase ^= 1; }
+      }
+    }
+  } else if (warp >= 2) {
+    // ------------------------------------------------------------ epilogue (128 threads)
+    const int quad = warp & 3;                    // TMEM lane quadrant this warp may read
+    const int r = quad * 32 + lane;
+    int acc = 0; uint32_t acc_phase = 0;
+    bool ok = true;
+    Epi epi;
+    for (int unit = blockIdx.x; ok && unit < sched.num_units; unit += gridDim.x) {
+      int mb, un, n_begin, n_end;
+      decode_unit(sched, unit, mb, un, n_begin, n_end);
+      epi.begin_unit(ep, mb, r);
+      for (int nb = n_begin; ok && nb < n_end; ++nb) {
+        if (!mbar_wait(&acc_full[acc], acc_phase, abort_flag)) { ok = false; break; }
+        fence_after_sync();
+        const uint32_t t_addr = tmem_base + (static_cast<uint32_t>(quad * 32) << 16) + acc * BN;
+        const int n_eff = tile_n_eff(sched, nb);
+        for (int c = 0; c * 32 < n_eff; ++c) {
+          float v[32];
+          tmem_ld32(t_addr + c * 32, v);
+          tmem_ld_wait();
+          epi.chunk(ep, v, nb * BN + c * 32);
+        }
+        fence_before_sync();
+        mbar_arrive(&acc_empty[acc]);
+        if (++acc == 2) { acc = 0; acc_phase ^= 1; }
+      }
+      if (ok) epi.end_unit(ep, un);
+    }
+  }
+
+  fence_before_sync();
+  __syncthreads();
+  if (warp == 1) { fence_after_sync(); tmem_dealloc(tmem_base, TMEM_COLS); }
+  if (threadIdx.x == 0 && *abort_flag) raise_status(status, SAPO_ST_WAIT_TIMEOUT);
+}
+
+// ---------------------------------------------------------------------------- small kernels
+// fp32 -> bf16 operands.  mode 0: [hi | hi | lo] (A side), mode 1: [hi | lo | hi] (B side),
+// so that sum_k A'[k] B'[k] = hi.hi + hi.lo + lo.hi; mode 2: hi only.
+__global__ void __launch_bounds__(256)
+split_bf16_kernel(const float* __restrict__ X, int64_t ld, int64_t R, int32_t H,
+                  __nv_bfloat16* __restrict__ out, int mode) {
+  const int64_t n = R * (int64_t)H;
+  const int64_t ldo = mode == 2 ? H : 3 * (int64_t)H;
+  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n;
+       i += (int64_t)gridDim.x * blockDim.x) {
+    const int64_t r = i / H; const int32_t c = (int32_t)(i - r * H);
+    const float x = X[r * ld + c];
+    const __nv_bfloat16 hi = __float2bfloat16_rn(x);
+    __nv_bfloat16* o = out + r * ldo;
+    o[c] = hi;
+    if (mode != 2) {
+      const __nv_bfloat16 lo = __float2bfloat16_rn(x - __bfloat162float(hi));
+      o[H + c] = mode == 0 ? hi : lo;
+      o[2 * H + c] = mode == 0 ? lo : hi;
+    }
+  }
+}
+
+struct TailArgs {
+  const float* pm; const float* ps; const float* pz; int32_t n_splits; int64_t T;
+  const int32_t* ids; int32_t V; const float* old_logp; const float* adv; const int32_t* cu; int32_t S;
+  float lo_edge, hi_edge, grad_scale;
+  float* logp; float* lse; float* ratio; float* surr; float* gscale; float* seq_surr;
+  int32_t* status;
+};
+
+__device__ __forceinline__ double block_sum_256(double x, double* sh) {
+  #pragma unroll
+  for (int d = 16; d > 0; d >>= 1) x += __shfl_xor_sync(0xffffffffu, x, d);
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  __syncthreads();
+  if (lane == 0) sh[warp] = x;
+  __syncthreads();
+  double t = 0.0;
+  if (threadIdx.x == 0) for (int i = 0; i < 8; ++i) t += sh[i];
+  return t;   // valid in thread 0
+}
+
+// One block per sequence: merge the vocab-split partials, then the clipped surrogate.
+__global__ void __launch_bounds__(256) loss_tail_kernel(TailArgs a) {
+  __shared__ double sh[8];
+  for (int32_t s = blockIdx.x; s < a.S; s += gridDim.x) {
+    const int32_t t0 = a.cu[s], t1 = a.cu[s + 1];
+    const int32_t Ts = t1 - t0;
+    const float A = a.adv[s];
+    const float w = Ts > 0 ? 1.f / ((float)a.S * (float)Ts) : 0.f;
+    double acc = 0.0;
+    for (int32_t t = t0 + threadIdx.x; t < t1; t += 256) {
+      float M = -INFINITY;
+      for (int i = 0; i < a.n_splits; ++i) M = fmaxf(M, a.pm[(int64_t)i * a.T + t]);
+      float sum = 0.f, zy = 0.f;
+      for (int i = 0; i < a.n_splits; ++i) {
+        const int64_t o = (int64_t)i * a.T + t;
+        sum += a.ps[o] * exp2f(a.pm[o] - M);
+        zy += a.pz[o];
+      }
+      const float lse = (M + log2f(sum)) * LN2;
+      const int32_t y = a.ids[t];
+      const bool bad = y < 0 || y >= a.V;
+      if (bad) raise_status(a.status, SAPO_ST_BAD_TOKEN_ID);
+      const float lp = bad ? 0.f : zy - lse;
+      const float rho = bad ? 0.f : expf(lp - a.old_logp[t]);
+      const float un = rho * A;
+      const float cl = fminf(fmaxf(rho, a.lo_edge), a.hi_edge) * A;
+      const float u = bad ? 0.f : fminf(un, cl);
+      const float g = (!bad && un <= cl) ? -a.grad_scale * A * rho * w : 0.f;
+      a.lse[t] = lse; a.logp[t] = lp; a.ratio[t] = rho; a.surr[t] = u; a.gscale[t] = g;
+      acc += (double)u;
+    }
+    const double tot = block_sum_256(acc, sh);
+    if (threadIdx.x == 0) a.seq_surr[s] = Ts > 0 ? (float)(tot / (double)Ts) : 0.f;
+  }
+}
+
+__global__ void __launch_bounds__(256) loss_final_kernel(const float* seq_surr, int32_t S, float* loss) {
+  __shared__ double sh[8];
+  double acc = 0.0;
+  for (int32_t s = threadIdx.x; s < S; s += 256) acc += (double)seq_surr[s];
+  const double tot = block_sum_256(acc, sh);
+  if (threadIdx.x == 0) *loss = S > 0 ? (float)(-tot / (double)S) : 0.f;
+}
+
+// ---------------------------------------------------------------------------- host side
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
+                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                  CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (fn == nullptr) {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(p);
+  }
+  return fn;
+}
+
+// bf16 matrix [outer, inner] with `ld` elements between rows; boxes are 64 elements wide
+// (128 bytes, 128-byte swizzle) and `box_outer` rows high.  Out-of-range elements read as 0.
+static bool make_map(CUtensorMap* map, const void* base, int64_t inner, int64_t outer, int64_t ld,
+                     int box_outer) {
+  EncodeTiledFn fn = encode_fn();
+  if (fn == nullptr || inner <= 0 || outer <= 0) return false;
+  cuuint64_t dims[2] = {(cuuint64_t)inner, (cuuint64_t)outer};
+  cuuint64_t strides[1] = {(cuuint64_t)ld * 2};
+  cuuint32_t box[2] = {64u, (cuuint32_t)box_outer};
+  cuuint32_t estr[2] = {1u, 1u};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+static Sched make_sched(int64_t M, int64_t N, int64_t K, int n_splits, bool m_fastest) {
+  Sched s{};
+  s.num_m_blocks = (int32_t)ceil_div<int64_t>(M, BM);
+  s.num_n_blocks = (int32_t)ceil_div<int64_t>(N, BN);
+  s.n_per_unit = n_splits > 0 ? ceil_div(s.num_n_blocks, n_splits) : 1;
+  s.units_per_m = ceil_div(s.num_n_blocks, s.n_per_unit);
+  s.num_units = s.num_m_blocks * s.units_per_m;
+  s.num_k_blocks = (int32_t)ceil_div<int64_t>(K, BK);
+  s.m_fastest = m_fastest ? 1 : 0;
+  s.N = (int32_t)N;
+  return s;
+}
+
+// Number of vocab splits of the forward pass: enough units to cover the SMs when there are
+// few token blocks, never more than there are vocab tiles.
+static int fwd_splits(int64_t T, int32_t V, int sms) {
+  const int64_t mb = ceil_div<int64_t>(T, BM);
+  const int64_t nb = ceil_div<int64_t>(V, BN);
+  int64_t best = 1; double best_eff = 0.0;
+  for (int64_t sp = 1; sp <= 160 && sp <= nb; ++sp) {
+    const int64_t per = ceil_div(nb, sp);
+    const int64_t units = mb * ceil_div(nb, per);
+    const double eff = (double)units / (double)(ceil_div<int64_t>(units, sms) * sms);
+    if (eff > best_eff + 1e-9) { best_eff = eff; best = sp; }
+    if (units >= 8 * (int64_t)sms) break;
+  }
+  const int64_t per = ceil_div(nb, best);
+  return (int)ceil_div(nb, per);
+}
+
+template <bool A_MN, bool B_MN, class Epi>
+static int launch_gemm(const CUtensorMap& ma, const CUtensorMap& mb, const Sched& sched,
+                       const typename Epi::Params& ep, int32_t* status, cudaStream_t st) {
+  auto kern = umma_gemm_kernel<A_MN, B_MN, Epi>;
+  static bool attr_set = false;
+  if (!attr_set) {
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)GEMM_SMEM_BYTES) !=
+        cudaSuccess)
+      return SAPO_ERR_CUDA;
+    attr_set = true;
+  }
+  const int sms = sm_count();
+  if (sms <= 0) return SAPO_ERR_CUDA;
+  const int grid = sched.num_units < sms ? sched.num_units : sms;
+  if (grid <= 0) return SAPO_OK;
+  kern<<<grid, GEMM_THREADS, GEMM_SMEM_BYTES, st>>>(ma, mb, sched, ep, status);
+  return check_launch();
+}
+
+static int launch_split(const float* X, int64_t ld, int64_t R, int32_t H, __nv_bfloat16* out, int mode,
+                        cudaStream_t st) {
+  const int64_t n = R * (int64_t)H;
+  int64_t blocks = ceil_div<int64_t>(n, 256);
+  const int64_t cap = (int64_t)sm_count() * 16;
+  if (blocks > cap) blocks = cap;
+  if (blocks <= 0) return SAPO_OK;
+  split_bf16_kernel<<<(int)blocks, 256, 0, st>>>(X, ld, R, H, out, mode);
+  return check_launch();
+}
+
+static bool shapes_ok(int64_t T, int32_t H, int32_t V) {
+  return T >= 1 && T <= 0x7fffff00LL && H >= 8 && (H % 8) == 0 && H <= 65536 && V >= 1 && V <= 0x7fffff00;
+}
+static int64_t padded_vocab(int32_t V) { return round_up<int64_t>(V, 64); }
+
+struct FwdLayout { size_t partials, a_split, b_split, total; int n_splits; };
+static FwdLayout fwd_layout(int64_t T, int32_t H, int32_t V, int32_t dtype, int sms) {
+  FwdLayout L{};
+  L.n_splits = fwd_splits(T, V, sms);
+  size_t off = 0;
+  L.partials = off; off += round_up<size_t>((size_t)3 * L.n_splits * T * sizeof(float), 256);
+  if (dtype == SAPO_DTYPE_F32) {
+    L.a_split = off; off += round_up<size_t>((size_t)T * 3 * H * 2, 256);
+    L.b_split = off; off += round_up<size_t>((size_t)V * 3 * H * 2, 256);
+  }
+  L.total = off;
+  return L;
+}
+
+struct BwdLayout { size_t a_hi, b_hi, panel, fixed; size_t bytes_per_row; };
+static BwdLayout bwd_layout(int64_t T, int32_t H, int32_t V, int32_t dtype) {
+  BwdLayout L{};
+  size_t off = 0;
+  if (dtype == SAPO_DTYPE_F32) {
+    L.a_hi = off; off += round_up<size_t>((size_t)T * H * 2, 256);
+    L.b_hi = off; off += round_up<size_t>((size_t)V * H * 2, 256);
+  }
+  L.panel = off; L.fixed = off;
+  L.bytes_per_row = (size_t)padded_vocab(V) * 2;
+  return L;
+}
+constexpr int64_t PANEL_ROWS_PREFERRED = 32768;
+
+}  // namespace sapo
+
+// =============================================================================== C ABI
+extern "C" size_t sapo_workspace_bytes(int32_t which, int64_t T, int32_t H, int32_t V, int32_t dtype) {
+  using namespace sapo;
+  if (!shapes_ok(T, H, V) || (dtype != SAPO_DTYPE_BF16 && dtype != SAPO_DTYPE_F32)) return 0;
+  if (which == SAPO_WS_FWD) {
+    int sms = sm_count();
+    if (sms <= 0) sms = 148;
+    return fwd_layout(T, H, V, dtype, sms).total;
+  }
+  if (which == SAPO_WS_BWD) {
+    const BwdLayout L = bwd_layout(T, H, V, dtype);
+    const int64_t rows = T < PANEL_ROWS_PREFERRED ? T : PANEL_ROWS_PREFERRED;
+    return L.fixed + (size_t)round_up<int64_t>(rows, BM) * L.bytes_per_row;
+  }
+  return 0;
+}
+
+extern "C" size_t sapo_workspace_bytes_min(int32_t which, int64_t T, int32_t H, int32_t V, int32_t dtype) {
+  using namespace sapo;
+  if (which != SAPO_WS_BWD) return sapo_workspace_bytes(which, T, H, V, dtype);
+  if (!shapes_ok(T, H, V) || (dtype != SAPO_DTYPE_BF16 && dtype != SAPO_DTYPE_F32)) return 0;
+  const BwdLayout L = bwd_layout(T, H, V, dtype);
+  return L.fixed + (size_t)BM * L.bytes_per_row;
+}
+
+extern "C" int sapo_policy_loss_fwd(const void* hidden, const void* W_head, int32_t dtype,
+                                    int64_t T, int32_t H, int32_t V, int64_t ld_hidden, int64_t ld_W,
+                                    const int32_t* ids, const float* old_logp, const float* adv,
+                                    const int32_t* cu_seqlens, int32_t S, const sapo_loss_cfg* h_cfg,
+                                    float* logp, float* lse, float* ratio, float* surr, float* gscale,
+                                    float* seq_surr, float* loss,
+                                    void* workspace, size_t workspace_bytes,
+                                    int32_t* status, void* stream) {
+  using namespace sapo;
+  if (!hidden || !W_head || !ids || !old_logp || !adv || !cu_seqlens || !h_cfg || !logp || !lse ||
+      !ratio || !surr || !gscale || !loss || !workspace || !status || S < 1)
+    return SAPO_ERR_INVALID_ARG;
+  if (dtype != SAPO_DTYPE_BF16 && dtype != SAPO_DTYPE_F32) return SAPO_ERR_INVALID_ARG;
+  if (T < 1 || H < 1 || V < 1 || ld_hidden < H || ld_W < H) return SAPO_ERR_INVALID_ARG;
+  if (!shapes_ok(T, H, V)) return SAPO_ERR_UNSUPPORTED_SHAPE;
+  const int esz = dtype == SAPO_DTYPE_BF16 ? 2 : 4;
+  if (!aligned16(hidden) || !aligned16(W_head) || !aligned16(workspace) || (ld_hidden * esz) % 16 ||
+      (ld_W * esz) % 16)
+    return SAPO_ERR_INVALID_ARG;
+  if (!(h_cfg->eps_low >= 0.f) || !(h_cfg->eps_high >= 0.f)) return SAPO_ERR_INVALID_ARG;
+  const int sms = sm_count();
+  if (sms <= 0) return SAPO_ERR_CUDA;
+  const FwdLayout L = fwd_layout(T, H, V, dtype, sms);
+  // seq_surr scratch lives behind the layout when the caller does not want it
+  const size_t need = L.total + (seq_surr ? 0 : round_up<size_t>((size_t)S * sizeof(float), 256));
+  if (workspace_bytes < need) return SAPO_ERR_WORKSPACE_TOO_SMALL;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  uint8_t* ws = static_cast<uint8_t*>(workspace);
+  float* pm = reinterpret_cast<float*>(ws + L.partials);
+  float* ps = pm + (size_t)L.n_splits * T;
+  float* pz = ps + (size_t)L.n_splits * T;
+  float* seq_out = seq_surr ? seq_surr : reinterpret_cast<float*>(ws + L.total);
+
+  const void* A = hidden; const void* B = W_head;
+  int64_t K = H, lda = ld_hidden, ldb = ld_W;
+  if (dtype == SAPO_DTYPE_F32) {
+    __nv_bfloat16* a3 = reinterpret_cast<__nv_bfloat16*>(ws + L.a_split);
+    __nv_bfloat16* b3 = reinterpret_cast<__nv_bfloat16*>(ws + L.b_split);
+    int rc = launch_split(static_cast<const float*>(hidden), ld_hidden, T, H, a3, 0, st);
+    if (rc != SAPO_OK) return rc;
+    rc = launch_split(static_cast<const float*>(W_head), ld_W, V, H, b3, 1, st);
+    if (rc != SAPO_OK) return rc;
+    A = a3; B = b3; K = 3 * (int64_t)H; lda = K; ldb = K;
+  }
+  CUtensorMap map_a, map_b;
+  if (!make_map(&map_a, A, K, T, lda, BM) || !make_map(&map_b, B, K, V, ldb, BN)) return SAPO_ERR_CUDA;
+  const Sched sched = make_sched(T, V, K, L.n_splits, /*m_fastest=*/true);
+  FwdEpi::Params ep{ids, pm, ps, pz, T, V};
+  int rc = launch_gemm<false, false, FwdEpi>(map_a, map_b, sched, ep, status, st);
+  if (rc != SAPO_OK) return rc;
+
+  TailArgs ta{};
+  ta.pm = pm; ta.ps = ps; ta.pz = pz; ta.n_splits = sched.units_per_m; ta.T = T;
+  ta.ids = ids; ta.V = V; ta.old_logp = old_logp; ta.adv = adv; ta.cu = cu_seqlens; ta.S = S;
+  ta.lo_edge = 1.f - h_cfg->eps_low; ta.hi_edge = 1.f + h_cfg->eps_high; ta.grad_scale = h_cfg->grad_scale;
+  ta.logp = logp; ta.lse = lse; ta.ratio = ratio; ta.surr = surr; ta.gscale = gscale; ta.seq_surr = seq_out;
+  ta.status = status;
+  const int tail_blocks = S < sms * 8 ? S : sms * 8;
+  loss_tail_kernel<<<tail_blocks, 256, 0, st>>>(ta);
+  loss_final_kernel<<<1, 256, 0, st>>>(seq_out, S, loss);
+  return check_launch();
+}
+
+extern "C" int sapo_policy_loss_bwd(const void* hidden, const void* W_head, int32_t dtype,
+                                    int64_t T, int32_t H, int32_t V, int64_t ld_hidden, int64_t ld_W,
+                                    const int32_t* ids, const float* lse, const float* gscale,
+                                    float* dhidden, float* dW_head, int32_t accumulate_dW,
+                                    void* workspace, size_t workspace_bytes,
+                                    int32_t* status, void* stream) {
+  using namespace sapo;
+  if (!hidden || !W_head || !ids || !lse || !gscale || !dhidden || !dW_head || !workspace || !status)
+    return SAPO_ERR_INVALID_ARG;
+  if (dtype != SAPO_DTYPE_BF16 && dtype != SAPO_DTYPE_F32) return SAPO_ERR_INVALID_ARG;
+  if (T < 1 || H < 1 || V < 1 || ld_hidden < H || ld_W < H) return SAPO_ERR_INVALID_ARG;
+  if (!shapes_ok(T, H, V)) return SAPO_ERR_UNSUPPORTED_SHAPE;
+  const int esz = dtype == SAPO_DTYPE_BF16 ? 2 : 4;
+  if (!aligned16(hidden) || !aligned16(W_head) || !aligned16(workspace) || !aligned16(dhidden) ||
+      !aligned16(dW_head) || (ld_hidden * esz) % 16 || (ld_W * esz) % 16)
+    return SAPO_ERR_INVALID_ARG;
+  const BwdLayout L = bwd_layout(T, H, V, dtype);
+  if (workspace_bytes < L.fixed + (size_t)BM * L.bytes_per_row) return SAPO_ERR_WORKSPACE_TOO_SMALL;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  uint8_t* ws = static_cast<uint8_t*>(workspace);
+
+  const __nv_bfloat16* A = static_cast<const __nv_bfloat16*>(hidden);
+  const __nv_bfloat16* B = static_cast<const __nv_bfloat16*>(W_head);
+  int64_t lda = ld_hidden, ldb = ld_W;
+  if (dtype == SAPO_DTYPE_F32) {
+    __nv_bfloat16* a1 = reinterpret_cast<__nv_bfloat16*>(ws + L.a_hi);
+    __nv_bfloat16* b1 = reinterpret_cast<__nv_bfloat16*>(ws + L.b_hi);
+    int rc = launch_split(static_cast<const float*>(hidden), ld_hidden, T, H, a1, 2, st);
+    if (rc != SAPO_OK) return rc;
+    rc = launch_split(static_cast<const float*>(W_head), ld_W, V, H, b1, 2, st);
+    if (rc != SAPO_OK) return rc;
+    A = a1; B = b1; lda = H; ldb = H;
+  }
+  const int64_t Vp = padded_vocab(V);
+  __nv_bfloat16* panel = reinterpret_cast<__nv_bfloat16*>(ws + L.panel);
+  int64_t rows_fit = (int64_t)((workspace_bytes - L.fixed) / L.bytes_per_row);
+  int64_t chunk_rows = rows_fit >= T ? T : (rows_fit / BM) * BM;
+  if (chunk_rows <= 0) return SAPO_ERR_WORKSPACE_TOO_SMALL;
+
+  // W as the K-major B operand of the logit recompute and as the MN-major B operand of dH
+  CUtensorMap map_w_kmajor, map_w_mn;
+  if (!make_map(&map_w_kmajor, B, H, V, ldb, BN) || !make_map(&map_w_mn, B, H, V, ldb, 64))
+    return SAPO_ERR_CUDA;
+
+  for (int64_t t0 = 0; t0 < T; t0 += chunk_rows) {
+    const int64_t tc = (T - t0) < chunk_rows ? (T - t0) : chunk_rows;
+    const __nv_bfloat16* A0 = A + t0 * lda;
+    CUtensorMap map_h_kmajor, map_h_mn, map_p_kmajor, map_p_mn;
+    if (!make_map(&map_h_kmajor, A0, H, tc, lda, BM) || !make_map(&map_h_mn, A0, H, tc, lda, 64) ||
+        !make_map(&map_p_kmajor, panel, V, tc, Vp, BM) || !make_map(&map_p_mn, panel, V, tc, Vp, 64))
+      return SAPO_ERR_CUDA;
+    // dz panel: recompute logits tile by tile
+    {
+      const Sched sched = make_sched(tc, V, H, 0, /*m_fastest=*/true);
+      DzEpi::Params ep{ids + t0, lse + t0, gscale + t0, panel, tc, V, Vp};
+      int rc = launch_gemm<false, false, DzEpi>(map_h_kmajor, map_w_kmajor, sched, ep, status, st);
+      if (rc != SAPO_OK) return rc;
+    }
+    // dhidden[t0:t0+tc] = dz . W         (M = tokens, N = H, K = V)
+    {
+      const Sched sched = make_sched(tc, H, V, 0, /*m_fastest=*/false);
+      StoreEpi::Params ep{dhidden + t0 * (int64_t)H, H, tc, H, 0};
+      int rc = launch_gemm<false, true, StoreEpi>(map_p_kmajor, map_w_mn, sched, ep, status, st);
+      if (rc != SAPO_OK) return rc;
+    }
+    // dW (+)= dz^T . hidden               (M = V, N = H, K = tokens)
+    {
+      const Sched sched = make_sched(V, H, tc, 0, /*m_fastest=*/false);
+      StoreEpi::Params ep{dW_head, H, V, H, (t0 > 0 || accumulate_dW) ? 1 : 0};
+      int rc = launch_gemm<true, true, StoreEpi>(map_p_mn, map_h_mn, sched, ep, status, st);
+      if (rc != SAPO_OK) return rc;
+    }
+  }
+  return SAPO_OK;
+}
+
+extern "C" const char* sapo_status_string(int32_t code) {
+  switch (code) {
+    case SAPO_OK: return "ok";
+    case SAPO_ERR_INVALID_ARG: return "invalid argument";
+    case SAPO_ERR_UNSUPPORTED_SHAPE: return "unsupported shape";
+    case SAPO_ERR_WORKSPACE_TOO_SMALL: return "workspace too small";
+    case SAPO_ERR_CUDA: return "CUDA error";
+    default: return "unknown code";
+  }
+}

@@ -1,0 +1,197 @@
+// sapo_pack_rollouts: gather the selected local and external rollouts into one varlen,
+// token-major batch (paper Section 3.2, training-set equation; Algorithm 1 "Assemble
+// training set").  Two kernels: a one-block scan that lays out the sequences, and an
+// HBM-bound row gather.  All integer work and copies are exact.
+#include "common.cuh"
+
+namespace sapo {
+
+struct PackArgs {
+  // selection
+  const int32_t* qol; const int32_t* local_idx; const int32_t* qoe; const int32_t* ext_idx;
+  int32_t Q;
+  // sources
+  const uint8_t* hid[2]; const int32_t* ids[2]; const float* old[2];
+  const int64_t* off[2]; const float* rew[2]; int32_t n_roll[2];
+  // outputs
+  uint8_t* o_hid; int32_t* o_ids; float* o_old; float* o_rew;
+  int32_t* cu; int32_t* seq_group; uint8_t* seq_is_ext; int32_t* seq_src;
+  int32_t* tok_seq; uint8_t* tok_mask; int32_t* group_offsets;
+  int32_t* n_tokens; int32_t* n_seqs;
+  int64_t max_tokens; int32_t max_seqs;
+  int64_t row_bytes;
+  int32_t* status;
+};
+
+constexpr int SCAN_THREADS = 1024;
+
+// first group q with go(q+1) > s, where go(q) = qol[q] + qoe[q] is non-decreasing
+__device__ __forceinline__ int32_t group_of(const PackArgs& a, int32_t s) {
+  int32_t lo = 0, hi = a.Q;            // answer in [0, Q)
+  while (lo < hi) {
+    int32_t mid = (lo + hi) >> 1;
+    if (a.qol[mid + 1] + a.qoe[mid + 1] > s) hi = mid; else lo = mid + 1;
+  }
+  return lo;
+}
+
+__global__ void __launch_bounds__(SCAN_THREADS) pack_scan_kernel(PackArgs a) {
+  __shared__ int64_t warp_sums[SCAN_THREADS / 32];
+  __shared__ int64_t running;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int64_t S64 = (int64_t)a.qol[a.Q] + (int64_t)a.qoe[a.Q];
+  if (S64 > a.max_seqs || S64 < 0) {
+    if (tid == 0) {
+      raise_status(a.status, SAPO_ST_SEQ_OVERFLOW);
+      *a.n_tokens = 0; *a.n_seqs = 0; a.cu[0] = 0;
+    }
+    for (int q = tid; q <= a.Q; q += SCAN_THREADS) a.group_offsets[q] = 0;
+    return;
+  }
+  const int32_t S = (int32_t)S64;
+  for (int q = tid; q <= a.Q; q += SCAN_THREADS) a.group_offsets[q] = a.qol[q] + a.qoe[q];
+  if (tid == 0) { running = 0; a.cu[0] = 0; }
+  __syncthreads();
+
+  for (int32_t base = 0; base < S; base += SCAN_THREADS) {
+    const int32_t s = base + tid;
+    int64_t len = 0;
+    if (s < S) {
+      const int32_t q = group_of(a, s);
+      const int32_t r = s - (a.qol[q] + a.qoe[q]);
+      const int32_t Iq = a.qol[q + 1] - a.qol[q];
+      const int side = r < Iq ? 0 : 1;
+      const int32_t idx = side == 0 ? a.local_idx[a.qol[q] + r] : a.ext_idx[a.qoe[q] + (r - Iq)];
+      float rew = 0.f;
+      if (idx < 0 || idx >= a.n_roll[side]) {
+        raise_status(a.status, SAPO_ST_BAD_INDEX);
+      } else {
+        len = a.off[side][idx + 1] - a.off[side][idx];
+        if (len <= 0) { len = 0; raise_status(a.status, SAPO_ST_EMPTY_SEQUENCE); }
+        rew = a.rew[side][idx];
+      }
+      a.seq_group[s] = q;
+      a.seq_is_ext[s] = (uint8_t)side;
+      a.seq_src[s] = idx;
+      a.o_rew[s] = rew;
+    }
+    // inclusive block scan of len
+    int64_t x = len;
+    #pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+      int64_t y = __shfl_up_sync(0xffffffffu, x, d);
+      if (lane >= d) x += y;
+    }
+    if (lane == 31) warp_sums[warp] = x;
+    __syncthreads();
+    if (warp == 0) {
+      int64_t w = warp_sums[lane];
+      #pragma unroll
+      for (int d = 1; d < 32; d <<= 1) {
+        int64_t y = __shfl_up_sync(0xffffffffu, w, d);
+        if (lane >= d) w += y;
+      }
+      warp_sums[lane] = w;
+    }
+    __syncthreads();
+    const int64_t incl = running + (warp > 0 ? warp_sums[warp - 1] : 0) + x;
+    if (s < S) a.cu[s + 1] = (int32_t)(incl < a.max_tokens ? incl : a.max_tokens);
+    __syncthreads();
+    if (tid == SCAN_THREADS - 1) running = incl;
+    __syncthreads();
+  }
+  if (tid == 0) {
+    int64_t total = running;
+    if (total > a.max_tokens) { raise_status(a.status, SAPO_ST_TOKEN_OVERFLOW); total = a.max_tokens; }
+    *a.n_tokens = (int32_t)total;
+    *a.n_seqs = S;
+  }
+}
+
+// One warp per packed token: locate its sequence, then copy the row.
+__global__ void __launch_bounds__(256) pack_copy_kernel(PackArgs a) {
+  const int lane = threadIdx.x & 31;
+  const int64_t warp0 = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  const int64_t n_warps = ((int64_t)gridDim.x * blockDim.x) >> 5;
+  const int32_t T = *a.n_tokens, S = *a.n_seqs;
+  const bool vec = (a.row_bytes & 15) == 0;
+  for (int64_t t = warp0; t < a.max_tokens; t += n_warps) {
+    if (t >= T) { if (lane == 0) a.tok_mask[t] = 0; continue; }
+    // last s with cu[s] <= t  (zero-length sequences share a start; take the one that owns t)
+    int32_t lo = 0, hi = S;                      // cu has S+1 entries; find first s with cu[s+1] > t
+    while (lo < hi) {
+      int32_t mid = (lo + hi) >> 1;
+      if (a.cu[mid + 1] > t) hi = mid; else lo = mid + 1;
+    }
+    const int32_t s = lo;
+    const int side = a.seq_is_ext[s];
+    const int64_t src = a.off[side][a.seq_src[s]] + (t - a.cu[s]);
+    const uint8_t* from = a.hid[side] + src * a.row_bytes;
+    uint8_t* to = a.o_hid + t * a.row_bytes;
+    if (vec) {
+      const uint4* f4 = reinterpret_cast<const uint4*>(from);
+      uint4* t4 = reinterpret_cast<uint4*>(to);
+      const int n4 = (int)(a.row_bytes >> 4);
+      for (int i = lane; i < n4; i += 32) t4[i] = __ldg(f4 + i);
+    } else {
+      const uint16_t* f2 = reinterpret_cast<const uint16_t*>(from);
+      uint16_t* t2 = reinterpret_cast<uint16_t*>(to);
+      const int n2 = (int)(a.row_bytes >> 1);
+      for (int i = lane; i < n2; i += 32) t2[i] = f2[i];
+    }
+    if (lane == 0) {
+      a.o_ids[t] = a.ids[side][src];
+      a.o_old[t] = a.old[side][src];
+      a.tok_seq[t] = s;
+      a.tok_mask[t] = 1;
+    }
+  }
+}
+
+}  // namespace sapo
+
+extern "C" int sapo_pack_rollouts(const sapo_rollout_buf* h_local, const sapo_rollout_buf* h_ext,
+                                  const sapo_selection* h_sel, int32_t H, int32_t dtype,
+                                  const sapo_packed* h_out, int32_t* status, void* stream) {
+  using namespace sapo;
+  if (!h_local || !h_ext || !h_sel || !h_out || !status) return SAPO_ERR_INVALID_ARG;
+  if (H <= 0 || (dtype != SAPO_DTYPE_BF16 && dtype != SAPO_DTYPE_F32)) return SAPO_ERR_INVALID_ARG;
+  if (h_sel->Q < 0 || h_out->max_tokens < 0 || h_out->max_tokens > 0x7fffff00LL ||
+      h_out->max_seqs < 0 || h_local->n_rollouts < 0 || h_ext->n_rollouts < 0)
+    return SAPO_ERR_INVALID_ARG;
+  if (!h_sel->q_offsets_local || !h_sel->q_offsets_ext || !h_out->cu_seqlens ||
+      !h_out->n_tokens || !h_out->n_seqs || !h_out->group_offsets)
+    return SAPO_ERR_INVALID_ARG;
+  PackArgs a{};
+  a.qol = h_sel->q_offsets_local; a.local_idx = h_sel->local_idx;
+  a.qoe = h_sel->q_offsets_ext;   a.ext_idx = h_sel->ext_idx; a.Q = h_sel->Q;
+  const sapo_rollout_buf* b[2] = {h_local, h_ext};
+  for (int i = 0; i < 2; ++i) {
+    a.hid[i] = static_cast<const uint8_t*>(b[i]->hidden); a.ids[i] = b[i]->ids;
+    a.old[i] = b[i]->old_logp; a.off[i] = b[i]->offsets; a.rew[i] = b[i]->rewards;
+    a.n_roll[i] = b[i]->n_rollouts;
+  }
+  a.o_hid = static_cast<uint8_t*>(h_out->hidden); a.o_ids = h_out->ids; a.o_old = h_out->old_logp;
+  a.o_rew = h_out->rewards; a.cu = h_out->cu_seqlens; a.seq_group = h_out->seq_group;
+  a.seq_is_ext = h_out->seq_is_ext; a.seq_src = h_out->seq_src; a.tok_seq = h_out->tok_seq;
+  a.tok_mask = h_out->tok_mask; a.group_offsets = h_out->group_offsets;
+  a.n_tokens = h_out->n_tokens; a.n_seqs = h_out->n_seqs;
+  a.max_tokens = h_out->max_tokens; a.max_seqs = h_out->max_seqs;
+  a.row_bytes = (int64_t)H * (dtype == SAPO_DTYPE_BF16 ? 2 : 4);
+  if (!aligned16(a.o_hid) || !aligned16(a.hid[0]) || !aligned16(a.hid[1])) {
+    if ((a.row_bytes & 15) == 0) return SAPO_ERR_INVALID_ARG;
+  }
+  a.status = status;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  pack_scan_kernel<<<1, SCAN_THREADS, 0, st>>>(a);
+  if (a.max_tokens > 0) {
+    const int sms = sm_count();
+    if (sms <= 0) return SAPO_ERR_CUDA;
+    const int64_t warps_wanted = a.max_tokens;
+    int blocks = (int)((warps_wanted + 7) / 8);
+    const int max_blocks = sms * 8;                 // 8 resident blocks of 256 threads per SM
+    if (blocks > max_blocks) blocks = max_blocks;
+    pack_copy_kernel<<<blocks, 256, 0, st>>>(a);
+  }
+  return check_launch();
+}

@@ -1,0 +1,45 @@
+"""The shared library builds, loads without a GPU, and exports every entry point the header
+declares.  Only host-side helpers are called here (no kernels)."""
+import ctypes
+import os
+import re
+
+from paper_2509_08721_b200 import binding as B
+from paper_2509_08721_b200 import build
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def declared_functions():
+    text = open(os.path.join(ROOT, "include", "sapo.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(sapo_[a-z_0-9]+)\s*\(", text)))
+
+
+def test_library_exports_every_declared_entry_point():
+    path = build.build()
+    lib = ctypes.CDLL(path)
+    names = declared_functions()
+    assert set(B.EXPORTS) <= set(names)
+    assert {"sapo_pack_rollouts", "sapo_group_advantages", "sapo_policy_loss_fwd",
+            "sapo_policy_loss_bwd"} <= set(names)
+    for n in names:
+        assert hasattr(lib, n), n
+
+
+def test_host_side_helpers():
+    lib = B.load()
+    assert lib.sapo_status_string(0) == b"ok"
+    assert b"workspace" in lib.sapo_status_string(-3)
+    # forward scratch: three partial arrays per vocab split; backward: a bf16 dz panel
+    T, H, V = 18432, 896, 151936
+    fwd = B.sapo_workspace_bytes(B.WS_FWD, T, H, V, B.DTYPE_BF16)
+    assert fwd >= 3 * 4 * T and fwd % 256 == 0
+    bwd = B.sapo_workspace_bytes(B.WS_BWD, T, H, V, B.DTYPE_BF16)
+    assert bwd == T * V * 2                              # V is already a multiple of 64
+    assert B.sapo_workspace_bytes_min(B.WS_BWD, T, H, V, B.DTYPE_BF16) == 128 * V * 2
+    assert B.sapo_workspace_bytes(B.WS_FWD, T, 12, V, B.DTYPE_BF16) == 0      # H % 8 != 0
+    assert B.sapo_workspace_bytes(7, T, H, V, B.DTYPE_BF16) == 0
+    f32 = B.sapo_workspace_bytes(B.WS_FWD, 1024, 64, 1000, B.DTYPE_F32)
+    assert f32 >= (1024 + 1000) * 3 * 64 * 2
+    assert B.decode_status(0x21) == ["TOKEN_OVERFLOW", "WAIT_TIMEOUT"]
