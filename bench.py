@@ -1,0 +1,321 @@
+#!/usr/bin/env python
+"""Benchmark of the SAPO policy-scoring step (pack -> advantages -> loss forward -> backward).
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload 2]
+
+Prints one JSON line.  `value` is scored tokens/s with the inputs resident in device memory;
+`e2e` is the same metric with the rollout buffers starting in pinned host memory every step.
+`--impl reference` times the fp64 CPU oracle on a bounded sample of the same workload.
+Under torchrun every rank scores its own batch (independent replicas, no data-path
+collective) and rank 0 reports the aggregate.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+METRIC = "scored tokens/s (fwd+bwd policy loss)"
+UNIT = "tokens/s"
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return {"bf16_tflops": p["bf16_tflops"], "bf16_tflops_sustained": p["bf16_tflops_sustained"],
+                "hbm_gbs": p["hbm_gbs"], "source": "measured"}
+    return {"bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "hbm_gbs": 6650.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+    QUERY = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+             "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+             "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.proc = None
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={index}", f"--query-gpu={self.QUERY}",
+                 "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except Exception:
+            self.proc.kill()
+            out = ""
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in out.strip().splitlines():
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 7:
+                continue
+            try:
+                sm.append(float(f[0])); mx.append(float(f[1]))
+            except ValueError:
+                continue
+            for n, v in zip(names, f[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": statistics.median(sm) if sm else None,
+                "sm_max_mhz": max(mx) if mx else None, "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def oracle_sample(batch, n_tokens_target):
+    """First whole sequences of the packed batch totalling at least `n_tokens_target` tokens."""
+    cu = batch.built.cu_seqlens
+    s = int(np.searchsorted(cu, n_tokens_target, side="left"))
+    s = max(1, min(s, batch.S))
+    return s, int(cu[s])
+
+
+def time_oracle(batch, n_seqs, repeats=1):
+    """Seconds for the oracle to score the first n_seqs sequences (pack, advantages,
+    forward, backward), as it stands."""
+    from oracle import sapo_oracle as orc
+    from paper_2509_08721_b200 import inputs as gen
+    b = batch.built
+    T = int(b.cu_seqlens[n_seqs])
+    times = []
+    for _ in range(repeats):
+        t0 = time.perf_counter()
+        buf = lambda x: {"hidden": x.hidden, "ids": x.ids, "old_logp": x.old_logp,
+                         "offsets": x.offsets, "rewards": x.rewards}
+        sel = {"q_offsets_local": batch.sel.q_offsets_local, "local_idx": batch.sel.local_idx,
+               "q_offsets_ext": batch.sel.q_offsets_ext, "ext_idx": batch.sel.ext_idx}
+        p = orc.pack_rollouts(buf(batch.local), buf(batch.ext), sel)
+        a = orc.group_advantages(p["rewards"], p["group_offsets"])
+        orc.policy_loss_fwd_bwd_rows(gen.as_f32(p["hidden"][:T]), gen.as_f32(batch.W), p["ids"][:T],
+                                     p["old_logp"][:T], a["adv"][:n_seqs], p["cu_seqlens"][:n_seqs + 1],
+                                     batch.eps_low, batch.eps_high, rows_per_block=512)
+        times.append(time.perf_counter() - t0)
+    return min(times), T
+
+
+def blas_threads():
+    try:
+        from threadpoolctl import threadpool_info
+        n = [d.get("num_threads", 1) for d in threadpool_info() if d.get("user_api") == "blas"]
+        return max(n) if n else os.cpu_count()
+    except Exception:
+        return os.cpu_count()
+
+
+def build_batch(workload: int, seed: int):
+    from paper_2509_08721_b200 import inputs as gen
+    recipe = gen.config(workload)
+    return gen.make_batch(recipe, seed), recipe
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return 0
+    batch, recipe = build_batch(args.workload, 1000 * args.workload)
+    batch.built.old_logp = None
+    # old log-probs: the recipe's noise around zero suffices for timing (values do not change cost)
+    n_seqs, T = oracle_sample(batch, args.ref_tokens)
+    for _ in range(min(args.warmup, 1)):
+        time_oracle(batch, n_seqs)
+    t = []
+    for _ in range(args.steps):
+        dt, T = time_oracle(batch, n_seqs)
+        t.append(dt)
+    ms = 1e3 * sum(t) / len(t)
+    value = T / (ms / 1e3)
+    cores = blas_threads()
+    sample = f"first {n_seqs} sequences ({T} tokens) of the {batch.T}-token batch per step"
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": min(args.warmup, 1), "ms_per_step": ms, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": recipe.name, "H": recipe.H, "V": recipe.V, "questions": recipe.Q,
+                   "local_per_question": recipe.I, "external_per_question": recipe.J,
+                   "tokens_per_step": T},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+    return 0
+
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    from paper_2509_08721_b200 import binding as B
+    from paper_2509_08721_b200 import inputs as gen
+    from paper_2509_08721_b200.pipeline import PolicyScorer, _to_dev
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    peaks = load_peaks()
+
+    batch, recipe = build_batch(args.workload, 1000 * args.workload + rank)
+    T, S, H, V = batch.T, batch.S, batch.H, batch.V
+    W = _to_dev(batch.W, "cuda")
+    scorer = PolicyScorer(W, T, S, recipe.Q, eps_low=batch.eps_low, eps_high=batch.eps_high)
+
+    # old log-probs = current + noise: "current" is one forward pass of the library itself
+    # over the packed tokens (set-up, untimed); the noise comes from the seeded generator.
+    scorer.make_host_batch(batch)
+    res = scorer.step_from_host(T, S)
+    torch.cuda.synchronize()
+    gen.install_old_logp(batch, res.fwd["logp"][:T].cpu().numpy())
+    scorer.make_host_batch(batch)
+    d = scorer._dev
+    for k, t in scorer._host.items():
+        d[k].copy_(t)
+    view = lambda t: t.view(torch.bfloat16) if t.dtype == torch.int16 else t
+    local = B.DeviceRollouts(view(d["local.hidden"]), d["local.ids"], d["local.old_logp"],
+                             d["local.offsets"], d["local.rewards"])
+    ext = B.DeviceRollouts(view(d["ext.hidden"]), d["ext.ids"], d["ext.old_logp"],
+                           d["ext.offsets"], d["ext.rewards"])
+    sel = B.DeviceSelection(d["sel.q_offsets_local"], d["sel.local_idx"], d["sel.q_offsets_ext"],
+                            d["sel.ext_idx"])
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def timed(fn, steps):
+        start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        start.record()
+        for _ in range(steps):
+            fn()
+        stop.record()
+        barrier()
+        ms = start.elapsed_time(stop)
+        if world > 1:
+            t = torch.tensor([ms], device="cuda")
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms = float(t.item())
+        return ms
+
+    dev_step = lambda: scorer.step(local, ext, sel, T, S)
+    host_step = lambda: scorer.step_from_host(T, S)
+
+    for _ in range(args.warmup):
+        dev_step()
+    torch.cuda.synchronize()
+    B.sapo_timing_enable(True)
+    launches0 = B.sapo_launch_count()
+    sampler = ClockSampler(local_rank) if rank == 0 else None
+    ms_total = timed(dev_step, args.steps)
+    clocks = sampler.stop() if sampler else None
+    n_launches = B.sapo_launch_count() - launches0
+    per_kernel = B.sapo_timing_read()
+    B.sapo_timing_enable(False)
+    scorer.check_status()
+
+    for _ in range(min(args.warmup, 3)):
+        host_step()
+    ms_e2e = timed(host_step, args.steps)
+    scorer.check_status()
+
+    tokens = torch.tensor([float(T)], device="cuda")
+    if world > 1:
+        dist.all_reduce(tokens)
+    total_tokens = float(tokens.item())
+    ms_step = ms_total / args.steps
+    value = total_tokens / (ms_step / 1e3)
+    e2e_value = total_tokens / (ms_e2e / args.steps / 1e3)
+
+    if rank == 0:
+        # roofline of the dominant kernel (largest share of the timed region)
+        flops_each = 2.0 * T * V * H
+        gemm = {k: per_kernel[k] for k in ("fwd_gemm", "bwd_dz", "bwd_dh", "bwd_dw")}
+        top = max(gemm, key=lambda k: gemm[k]["ms"])
+        n_top = max(1, gemm[top]["launches"])
+        ms_top = gemm[top]["ms"] / n_top
+        # launches per step of that kernel (the backward runs once per dz panel chunk)
+        per_step = n_top / args.steps
+        achieved = flops_each / per_step / (ms_top / 1e3) / 1e12
+        peak = peaks["bf16_tflops"]
+        kernels = {k: {"ms_per_step": v["ms"] / args.steps, "launches_per_step": v["launches"] / args.steps}
+                   for k, v in per_kernel.items() if v["launches"]}
+        gemm_ms = sum(gemm[k]["ms"] for k in gemm) / args.steps
+        f_alg = 6.0 * T * V * H
+        f_exec = 8.0 * T * V * H
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": recipe.name, "H": H, "V": V, "questions": recipe.Q,
+                       "local_per_question": recipe.I, "external_per_question": recipe.J,
+                       "tokens_per_step": T, "sequences": S, "parallelism": f"replicas x{world}",
+                       "l2": "inputs larger than L2 (W_head alone is %d MB)" % (V * H * 2 // 2**20)},
+            "tflops_algorithmic": f_alg / (ms_step / 1e3) / 1e12,
+            "tflops_executed": f_exec / (ms_step / 1e3) / 1e12,
+            "frac_of_bf16_peak_algorithmic": f_alg / (ms_step / 1e3) / 1e12 / peak,
+            "frac_of_bf16_peak_executed": f_exec / (ms_step / 1e3) / 1e12 / peak,
+            "roofline": {"bound": "tensor", "kernel": top, "achieved": achieved, "peak": peak,
+                         "unit": "TFLOP/s", "frac": achieved / peak, "traffic": None,
+                         "peak_source": peaks["source"] + " (burst bf16 GEMM)",
+                         "flops_per_launch": flops_each / per_step, "ms_per_launch": ms_top,
+                         "all_gemm_kernels_ms_per_step": gemm_ms},
+            "kernels": kernels,
+            "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": scorer.h2d_bytes,
+                    "d2h_bytes_per_step": scorer.d2h_bytes, "ms_per_step": ms_e2e / args.steps},
+            "gpu_launches": int(n_launches),
+            "clocks": clocks,
+        }
+        if world == 1 and not args.no_cpu_baseline:
+            n_seqs, _ = oracle_sample(batch, args.ref_tokens)
+            dt, Ts = time_oracle(batch, n_seqs)
+            line["cpu_baseline"] = {
+                "value": Ts / dt, "unit": UNIT, "cores": blas_threads(), "kind": "oracle",
+                "sample": f"first {n_seqs} sequences ({Ts} tokens) of the {T}-token batch, one pass, {dt:.1f} s"}
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+    return 0
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", type=int, default=2, help="1..5; 2 is the Qwen2.5-0.5B-shaped head")
+    ap.add_argument("--ref-tokens", type=int, default=None,
+                    help="tokens of the bounded oracle sample (default 2048 for cpu_baseline, 512 per reference step)")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.warmup < 3 and args.impl == "ours":
+        args.warmup = 3
+    if args.ref_tokens is None:
+        args.ref_tokens = 512 if args.impl == "reference" else 2048
+    return run_reference(args) if args.impl == "reference" else run_ours(args)
+
+
+if __name__ == "__main__":
+    sys.exit(main())

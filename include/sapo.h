@@ -198,6 +198,27 @@ size_t sapo_workspace_bytes(int32_t which, int64_t T, int32_t H, int32_t V, int3
 /* Smallest backward workspace that still works (one 128-token panel). */
 size_t sapo_workspace_bytes_min(int32_t which, int64_t T, int32_t H, int32_t V, int32_t dtype);
 
+/* Optional per-kernel timing for benchmarks (no counterpart in the paper).  While enabled,
+ * every kernel launch of the library is bracketed by two CUDA events recorded on the call's
+ * stream.  sapo_timing_read waits for the recorded events, writes the summed milliseconds and
+ * the number of launches per kernel id (arrays of SAPO_K_COUNT) and forgets them; at most 512
+ * launches are kept between reads.  The events are created on the first enable.  Not thread-safe.
+ * sapo_launch_count returns how many kernels the library has launched in this process. */
+#define SAPO_K_PACK_SCAN  0
+#define SAPO_K_PACK_COPY  1
+#define SAPO_K_GROUP_ADV  2
+#define SAPO_K_SPLIT_BF16 3
+#define SAPO_K_FWD_GEMM   4
+#define SAPO_K_LOSS_TAIL  5
+#define SAPO_K_LOSS_FINAL 6
+#define SAPO_K_BWD_DZ     7
+#define SAPO_K_BWD_DH     8
+#define SAPO_K_BWD_DW     9
+#define SAPO_K_COUNT      10
+int sapo_timing_enable(int32_t on);
+int sapo_timing_read(float* h_ms, int32_t* h_launches);
+int64_t sapo_launch_count(void);
+
 /* Text for a return code. */
 const char* sapo_status_string(int32_t code);
 

@@ -26,7 +26,9 @@ ST_BITS = {
 
 EXPORTS = ("sapo_pack_rollouts", "sapo_group_advantages", "sapo_policy_loss_fwd",
            "sapo_policy_loss_bwd", "sapo_workspace_bytes", "sapo_workspace_bytes_min",
-           "sapo_status_string")
+           "sapo_status_string", "sapo_timing_enable", "sapo_timing_read", "sapo_launch_count")
+KERNEL_NAMES = ("pack_scan", "pack_copy", "group_adv", "split_bf16", "fwd_gemm", "loss_tail",
+                "loss_final", "bwd_dz", "bwd_dh", "bwd_dw")
 
 
 class RolloutBufC(C.Structure):
@@ -84,6 +86,12 @@ def load() -> C.CDLL:
     lib.sapo_workspace_bytes.argtypes = [i32, i64, i32, i32, i32]
     lib.sapo_workspace_bytes_min.restype = sz
     lib.sapo_workspace_bytes_min.argtypes = [i32, i64, i32, i32, i32]
+    lib.sapo_timing_enable.restype = C.c_int
+    lib.sapo_timing_enable.argtypes = [i32]
+    lib.sapo_timing_read.restype = C.c_int
+    lib.sapo_timing_read.argtypes = [C.POINTER(C.c_float), C.POINTER(C.c_int32)]
+    lib.sapo_launch_count.restype = C.c_int64
+    lib.sapo_launch_count.argtypes = []
     lib.sapo_status_string.restype = C.c_char_p
     lib.sapo_status_string.argtypes = [i32]
     _lib = lib
@@ -118,6 +126,23 @@ def _dtype_code(t: torch.Tensor) -> int:
     if t.dtype == torch.float32:
         return DTYPE_F32
     raise SapoError(f"unsupported element type {t.dtype}")
+
+
+def sapo_timing_enable(on: bool) -> None:
+    _check(load().sapo_timing_enable(1 if on else 0), "sapo_timing_enable")
+
+
+def sapo_timing_read() -> Dict[str, Dict[str, float]]:
+    """Summed milliseconds and launch count per kernel since the last read."""
+    n = len(KERNEL_NAMES)
+    ms = (C.c_float * n)()
+    cnt = (C.c_int32 * n)()
+    _check(load().sapo_timing_read(ms, cnt), "sapo_timing_read")
+    return {KERNEL_NAMES[i]: {"ms": float(ms[i]), "launches": int(cnt[i])} for i in range(n)}
+
+
+def sapo_launch_count() -> int:
+    return int(load().sapo_launch_count())
 
 
 def decode_status(word: int):

@@ -61,7 +61,11 @@ extern "C" int sapo_group_advantages(const float* rewards, const int32_t* group_
   if (sms <= 0) return SAPO_ERR_CUDA;
   int64_t blocks = ((int64_t)Q + 7) / 8;
   if (blocks > (int64_t)sms * 8) blocks = (int64_t)sms * 8;
-  group_adv_kernel<<<(int)blocks, 256, 0, static_cast<cudaStream_t>(stream)>>>(
-      rewards, group_offsets, Q, (double)adv_eps, ddof, adv, mean, std, status);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  {
+    KernelScope scope(SAPO_K_GROUP_ADV, st);
+    group_adv_kernel<<<(int)blocks, 256, 0, st>>>(rewards, group_offsets, Q, (double)adv_eps, ddof, adv,
+                                                  mean, std, status);
+  }
   return check_launch();
 }

@@ -29,6 +29,33 @@ inline int sm_count() {
   return n;
 }
 
+// Optional per-kernel timing and launch counting (see sapo_timing_* in sapo.h).
+// A KernelScope brackets one kernel launch with two CUDA events when timing is on.
+struct KernelTimer {
+  static constexpr int MAX_PAIRS = 512;
+  bool enabled = false;
+  bool created = false;
+  int n = 0;
+  int id[MAX_PAIRS];
+  cudaEvent_t start[MAX_PAIRS], stop[MAX_PAIRS];
+  long long launches = 0;
+};
+KernelTimer& kernel_timer();
+
+struct KernelScope {
+  cudaStream_t st; int slot;
+  KernelScope(int kernel_id, cudaStream_t s) : st(s), slot(-1) {
+    KernelTimer& t = kernel_timer();
+    ++t.launches;
+    if (t.enabled && t.created && t.n < KernelTimer::MAX_PAIRS) {
+      slot = t.n++;
+      t.id[slot] = kernel_id;
+      cudaEventRecord(t.start[slot], st);
+    }
+  }
+  ~KernelScope() { if (slot >= 0) cudaEventRecord(kernel_timer().stop[slot], st); }
+};
+
 template <typename T>
 __host__ __device__ constexpr T ceil_div(T a, T b) { return (a + b - 1) / b; }
 template <typename T>

@@ -465,7 +465,7 @@ static int fwd_splits(int64_t T, int32_t V, int sms) {
 
 template <bool A_MN, bool B_MN, class Epi>
 static int launch_gemm(const CUtensorMap& ma, const CUtensorMap& mb, const Sched& sched,
-                       const typename Epi::Params& ep, int32_t* status, cudaStream_t st) {
+                       const typename Epi::Params& ep, int32_t* status, cudaStream_t st, int kernel_id) {
   auto kern = umma_gemm_kernel<A_MN, B_MN, Epi>;
   static bool attr_set = false;
   if (!attr_set) {
@@ -478,7 +478,10 @@ static int launch_gemm(const CUtensorMap& ma, const CUtensorMap& mb, const Sched
   if (sms <= 0) return SAPO_ERR_CUDA;
   const int grid = sched.num_units < sms ? sched.num_units : sms;
   if (grid <= 0) return SAPO_OK;
-  kern<<<grid, GEMM_THREADS, GEMM_SMEM_BYTES, st>>>(ma, mb, sched, ep, status);
+  {
+    KernelScope scope(kernel_id, st);
+    kern<<<grid, GEMM_THREADS, GEMM_SMEM_BYTES, st>>>(ma, mb, sched, ep, status);
+  }
   return check_launch();
 }
 
@@ -489,6 +492,7 @@ static int launch_split(const float* X, int64_t ld, int64_t R, int32_t H, __nv_b
   const int64_t cap = (int64_t)sm_count() * 16;
   if (blocks > cap) blocks = cap;
   if (blocks <= 0) return SAPO_OK;
+  KernelScope scope(SAPO_K_SPLIT_BF16, st);
   split_bf16_kernel<<<(int)blocks, 256, 0, st>>>(X, ld, R, H, out, mode);
   return check_launch();
 }
@@ -601,7 +605,7 @@ extern "C" int sapo_policy_loss_fwd(const void* hidden, const void* W_head, int3
   if (!make_map(&map_a, A, K, T, lda, BM) || !make_map(&map_b, B, K, V, ldb, BN)) return SAPO_ERR_CUDA;
   const Sched sched = make_sched(T, V, K, L.n_splits, /*m_fastest=*/true);
   FwdEpi::Params ep{ids, pm, ps, pz, T, V};
-  int rc = launch_gemm<false, false, FwdEpi>(map_a, map_b, sched, ep, status, st);
+  int rc = launch_gemm<false, false, FwdEpi>(map_a, map_b, sched, ep, status, st, SAPO_K_FWD_GEMM);
   if (rc != SAPO_OK) return rc;
 
   TailArgs ta{};
@@ -611,8 +615,8 @@ extern "C" int sapo_policy_loss_fwd(const void* hidden, const void* W_head, int3
   ta.logp = logp; ta.lse = lse; ta.ratio = ratio; ta.surr = surr; ta.gscale = gscale; ta.seq_surr = seq_out;
   ta.status = status;
   const int tail_blocks = S < sms * 8 ? S : sms * 8;
-  loss_tail_kernel<<<tail_blocks, 256, 0, st>>>(ta);
-  loss_final_kernel<<<1, 256, 0, st>>>(seq_out, S, loss);
+  { KernelScope scope(SAPO_K_LOSS_TAIL, st); loss_tail_kernel<<<tail_blocks, 256, 0, st>>>(ta); }
+  { KernelScope scope(SAPO_K_LOSS_FINAL, st); loss_final_kernel<<<1, 256, 0, st>>>(seq_out, S, loss); }
   return check_launch();
 }
 
@@ -671,34 +675,23 @@ extern "C" int sapo_policy_loss_bwd(const void* hidden, const void* W_head, int3
     {
       const Sched sched = make_sched(tc, V, H, 0, /*m_fastest=*/true);
       DzEpi::Params ep{ids + t0, lse + t0, gscale + t0, panel, tc, V, Vp};
-      int rc = launch_gemm<false, false, DzEpi>(map_h_kmajor, map_w_kmajor, sched, ep, status, st);
+      int rc = launch_gemm<false, false, DzEpi>(map_h_kmajor, map_w_kmajor, sched, ep, status, st, SAPO_K_BWD_DZ);
       if (rc != SAPO_OK) return rc;
     }
     // dhidden[t0:t0+tc] = dz . W         (M = tokens, N = H, K = V)
     {
       const Sched sched = make_sched(tc, H, V, 0, /*m_fastest=*/false);
       StoreEpi::Params ep{dhidden + t0 * (int64_t)H, H, tc, H, 0};
-      int rc = launch_gemm<false, true, StoreEpi>(map_p_kmajor, map_w_mn, sched, ep, status, st);
+      int rc = launch_gemm<false, true, StoreEpi>(map_p_kmajor, map_w_mn, sched, ep, status, st, SAPO_K_BWD_DH);
       if (rc != SAPO_OK) return rc;
     }
     // dW (+)= dz^T . hidden               (M = V, N = H, K = tokens)
     {
       const Sched sched = make_sched(V, H, tc, 0, /*m_fastest=*/false);
       StoreEpi::Params ep{dW_head, H, V, H, (t0 > 0 || accumulate_dW) ? 1 : 0};
-      int rc = launch_gemm<true, true, StoreEpi>(map_p_mn, map_h_mn, sched, ep, status, st);
+      int rc = launch_gemm<true, true, StoreEpi>(map_p_mn, map_h_mn, sched, ep, status, st, SAPO_K_BWD_DW);
       if (rc != SAPO_OK) return rc;
     }
   }
   return SAPO_OK;
-}
-
-extern "C" const char* sapo_status_string(int32_t code) {
-  switch (code) {
-    case SAPO_OK: return "ok";
-    case SAPO_ERR_INVALID_ARG: return "invalid argument";
-    case SAPO_ERR_UNSUPPORTED_SHAPE: return "unsupported shape";
-    case SAPO_ERR_WORKSPACE_TOO_SMALL: return "workspace too small";
-    case SAPO_ERR_CUDA: return "CUDA error";
-    default: return "unknown code";
-  }
 }

@@ -183,7 +183,7 @@ extern "C" int sapo_pack_rollouts(const sapo_rollout_buf* h_local, const sapo_ro
   }
   a.status = status;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  pack_scan_kernel<<<1, SCAN_THREADS, 0, st>>>(a);
+  { KernelScope scope(SAPO_K_PACK_SCAN, st); pack_scan_kernel<<<1, SCAN_THREADS, 0, st>>>(a); }
   if (a.max_tokens > 0) {
     const int sms = sm_count();
     if (sms <= 0) return SAPO_ERR_CUDA;
@@ -191,6 +191,7 @@ extern "C" int sapo_pack_rollouts(const sapo_rollout_buf* h_local, const sapo_ro
     int blocks = (int)((warps_wanted + 7) / 8);
     const int max_blocks = sms * 8;                 // 8 resident blocks of 256 threads per SM
     if (blocks > max_blocks) blocks = max_blocks;
+    KernelScope scope(SAPO_K_PACK_COPY, st);
     pack_copy_kernel<<<blocks, 256, 0, st>>>(a);
   }
   return check_launch();
