@@ -165,6 +165,7 @@ def run_ours(args):
     import torch.distributed as dist
     from paper_2509_08721_b200 import binding as B
     from paper_2509_08721_b200 import inputs as gen
+    from paper_2509_08721_b200 import replicas
     from paper_2509_08721_b200.pipeline import PolicyScorer, _to_dev
 
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -177,7 +178,7 @@ def run_ours(args):
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
     peaks = load_peaks()
 
-    batch, recipe = build_batch(args.workload, 1000 * args.workload + rank, args.length_div)
+    batch, recipe = build_batch(args.workload, replicas.rank_seed(args.workload, rank), args.length_div)
     T, S, H, V = batch.T, batch.S, batch.H, batch.V
     W = _to_dev(batch.W, "cuda")
     scorer = PolicyScorer(W, T, S, recipe.Q, eps_low=batch.eps_low, eps_high=batch.eps_high)
@@ -213,11 +214,7 @@ def run_ours(args):
             fn()
         stop.record()
         barrier()
-        ms = start.elapsed_time(stop)
-        if world > 1:
-            t = torch.tensor([ms], device="cuda")
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms = float(t.item())
+        ms, _ = replicas.aggregate(start.elapsed_time(stop), 0.0, device="cuda")
         return ms
 
     dev_step = lambda: scorer.step(local, ext, sel, T, S)
@@ -241,13 +238,10 @@ def run_ours(args):
     ms_e2e = timed(host_step, args.steps)
     scorer.check_status()
 
-    tokens = torch.tensor([float(T)], device="cuda")
-    if world > 1:
-        dist.all_reduce(tokens)
-    total_tokens = float(tokens.item())
+    _, total_tokens = replicas.aggregate(0.0, float(T), device="cuda")
     ms_step = ms_total / args.steps
-    value = total_tokens / (ms_step / 1e3)
-    e2e_value = total_tokens / (ms_e2e / args.steps / 1e3)
+    value = replicas.throughput(ms_total, total_tokens, args.steps)
+    e2e_value = replicas.throughput(ms_e2e, total_tokens, args.steps)
 
     if rank == 0:
         # roofline of the dominant kernel (largest share of the timed region)
