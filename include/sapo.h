@@ -46,6 +46,7 @@ extern "C" {
 #define SAPO_ERR_UNSUPPORTED_SHAPE  -2
 #define SAPO_ERR_WORKSPACE_TOO_SMALL -3
 #define SAPO_ERR_CUDA               -4
+#define SAPO_ERR_STATIC_SCRATCH_EXCEEDED -5  /* sizes beyond the built-in scratch of the _static call */
 
 /* device-detected conditions (bits of *status) */
 #define SAPO_ST_TOKEN_OVERFLOW   0x01  /* packed tokens exceed max_tokens; output truncated   */
@@ -197,6 +198,30 @@ size_t sapo_workspace_bytes(int32_t which, int64_t T, int32_t H, int32_t V, int3
 
 /* Smallest backward workspace that still works (one 128-token panel). */
 size_t sapo_workspace_bytes_min(int32_t which, int64_t T, int32_t H, int32_t V, int32_t dtype);
+
+/* Forward pass without caller-provided scratch (the paper has no counterpart; this exists for
+ * hosts that are not allowed to allocate device memory: a component embedded in a process whose
+ * memory pool is fixed once at start-up, or a loop that must never reach cudaMalloc because it
+ * synchronises the whole device).  Same arguments, results and error rules as
+ * sapo_policy_loss_fwd, except that `workspace` is gone: the scratch is an array of
+ * SAPO_STATIC_SCRATCH_BYTES that is part of the library image, so every GPU that loads the
+ * library carries it until the process ends.  The call itself allocates and frees nothing.
+ * Limits: bf16 operands only (SAPO_ERR_UNSUPPORTED_SHAPE otherwise), and the forward scratch for
+ * these sizes — sapo_workspace_bytes(SAPO_WS_FWD, ...), plus 4*S bytes when seq_surr is NULL —
+ * must fit; if not, the call does nothing and returns SAPO_ERR_STATIC_SCRATCH_EXCEEDED.  With one
+ * vocab split (at least as many 128-token blocks as SMs) that is about 340,000 tokens.
+ * The first call on each device looks up the array's device address (that device must be
+ * current); make that first call outside any stream capture.  All calls on a device share the
+ * one array and it keeps whatever the previous call left: nothing in it needs clearing between
+ * calls, but two calls that may run on the GPU at the same time (different streams, or
+ * different threads) race on it and must be ordered by the caller. */
+#define SAPO_STATIC_SCRATCH_BYTES (4 * 1024 * 1024)
+int sapo_policy_loss_fwd_static(const void* hidden, const void* W_head, int32_t dtype,
+                                int64_t T, int32_t H, int32_t V, int64_t ld_hidden, int64_t ld_W,
+                                const int32_t* ids, const float* old_logp, const float* adv,
+                                const int32_t* cu_seqlens, int32_t S, const sapo_loss_cfg* h_cfg,
+                                float* logp, float* lse, float* ratio, float* surr, float* gscale,
+                                float* seq_surr, float* loss, int32_t* status, void* stream);
 
 /* Optional per-kernel timing for benchmarks (no counterpart in the paper).  While enabled,
  * every kernel launch of the library is bracketed by two CUDA events recorded on the call's

@@ -26,7 +26,9 @@ ST_BITS = {
 
 EXPORTS = ("sapo_pack_rollouts", "sapo_group_advantages", "sapo_policy_loss_fwd",
            "sapo_policy_loss_bwd", "sapo_workspace_bytes", "sapo_workspace_bytes_min",
-           "sapo_status_string", "sapo_timing_enable", "sapo_timing_read", "sapo_launch_count")
+           "sapo_status_string", "sapo_timing_enable", "sapo_timing_read", "sapo_launch_count",
+           "sapo_policy_loss_fwd_static")
+STATIC_SCRATCH_BYTES = 4 * 1024 * 1024
 KERNEL_NAMES = ("pack_scan", "pack_copy", "group_adv", "split_bf16", "fwd_gemm", "loss_tail",
                 "loss_final", "bwd_dz", "bwd_dh", "bwd_dw")
 
@@ -79,6 +81,9 @@ def load() -> C.CDLL:
     lib.sapo_policy_loss_fwd.argtypes = [vp, vp, i32, i64, i32, i32, i64, i64, vp, vp, vp, vp, i32,
                                          C.POINTER(LossCfgC), vp, vp, vp, vp, vp, vp, vp, vp, sz,
                                          vp, vp]
+    lib.sapo_policy_loss_fwd_static.restype = C.c_int
+    lib.sapo_policy_loss_fwd_static.argtypes = [vp, vp, i32, i64, i32, i32, i64, i64, vp, vp, vp, vp, i32,
+                                                C.POINTER(LossCfgC), vp, vp, vp, vp, vp, vp, vp, vp, vp]
     lib.sapo_policy_loss_bwd.restype = C.c_int
     lib.sapo_policy_loss_bwd.argtypes = [vp, vp, i32, i64, i32, i32, i64, i64, vp, vp, vp, vp, vp,
                                          i32, vp, sz, vp, vp]
@@ -250,6 +255,27 @@ def sapo_policy_loss_fwd(hidden: torch.Tensor, W_head: torch.Tensor, ids: torch.
         _p(out.get("seq_surr")), _p(out["loss"]), _p(workspace), workspace.numel() * workspace.element_size(),
         _p(status), _stream())
     _check(rc, "sapo_policy_loss_fwd")
+
+
+def sapo_policy_loss_fwd_static(hidden: torch.Tensor, W_head: torch.Tensor, ids: torch.Tensor,
+                                old_logp: torch.Tensor, adv: torch.Tensor, cu_seqlens: torch.Tensor,
+                                eps_low: float, eps_high: float, grad_scale: float,
+                                out: Dict[str, torch.Tensor], status: torch.Tensor,
+                                T: Optional[int] = None) -> None:
+    """sapo_policy_loss_fwd for callers that may not allocate device memory: the scratch is the
+    array built into the library (STATIC_SCRATCH_BYTES), so no workspace tensor is passed.
+    Raises SapoError when the sizes need more scratch than that, or for fp32 operands."""
+    _require_cuda()
+    T = int(hidden.shape[0]) if T is None else int(T)
+    H, V = int(hidden.shape[1]), int(W_head.shape[0])
+    S = int(cu_seqlens.numel() - 1)
+    cfg = LossCfgC(eps_low, eps_high, grad_scale)
+    rc = load().sapo_policy_loss_fwd_static(
+        _p(hidden), _p(W_head), _dtype_code(hidden), T, H, V, hidden.stride(0), W_head.stride(0),
+        _p(ids), _p(old_logp), _p(adv), _p(cu_seqlens), S, C.byref(cfg),
+        _p(out["logp"]), _p(out["lse"]), _p(out["ratio"]), _p(out["surr"]), _p(out["gscale"]),
+        _p(out.get("seq_surr")), _p(out["loss"]), _p(status), _stream())
+    _check(rc, "sapo_policy_loss_fwd_static")
 
 
 def sapo_policy_loss_bwd(hidden: torch.Tensor, W_head: torch.Tensor, ids: torch.Tensor,

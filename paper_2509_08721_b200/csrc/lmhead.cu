@@ -620,6 +620,62 @@ extern "C" int sapo_policy_loss_fwd(const void* hidden, const void* W_head, int3
   return check_launch();
 }
 
+// ------------------------------------------------------------------------------------------
+// Forward pass for callers that cannot obtain device memory of their own.
+//
+// Some hosts of this library may not allocate: a plugin inside a serving process whose
+// memory pool is fixed at start-up, code that runs after the process has handed all of its
+// device memory to another allocator, or a latency-critical loop in which cudaMalloc (which
+// synchronises the device) is forbidden.  For them the forward scratch lives in this array,
+// which belongs to the library image: every GPU that loads the library holds these
+// SAPO_STATIC_SCRATCH_BYTES until the process exits, whether or not the entry point is used.
+static __device__ __align__(256) unsigned char g_static_fwd_scratch[SAPO_STATIC_SCRATCH_BYTES];
+
+namespace sapo {
+constexpr int MAX_DEVICES = 64;
+// Device address of the array on each GPU.  In host code the symbol's name is only a handle;
+// the address a kernel can use has to be asked for, once per device, with that device current.
+static void* g_static_scratch_ptr[MAX_DEVICES] = {nullptr};
+
+static int static_scratch(void** out) {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= MAX_DEVICES) return SAPO_ERR_CUDA;
+  if (g_static_scratch_ptr[dev] == nullptr) {
+    void* p = nullptr;
+    if (cudaGetSymbolAddress(&p, g_static_fwd_scratch) != cudaSuccess || p == nullptr) return SAPO_ERR_CUDA;
+    g_static_scratch_ptr[dev] = p;
+  }
+  *out = g_static_scratch_ptr[dev];
+  return SAPO_OK;
+}
+}  // namespace sapo
+
+extern "C" int sapo_policy_loss_fwd_static(const void* hidden, const void* W_head, int32_t dtype,
+                                           int64_t T, int32_t H, int32_t V, int64_t ld_hidden,
+                                           int64_t ld_W, const int32_t* ids, const float* old_logp,
+                                           const float* adv, const int32_t* cu_seqlens, int32_t S,
+                                           const sapo_loss_cfg* h_cfg, float* logp, float* lse,
+                                           float* ratio, float* surr, float* gscale, float* seq_surr,
+                                           float* loss, int32_t* status, void* stream) {
+  using namespace sapo;
+  // fp32 operands would need bf16 copies of hidden and W_head in the scratch: far beyond it
+  if (dtype != SAPO_DTYPE_BF16) return SAPO_ERR_UNSUPPORTED_SHAPE;
+  if (T < 1 || S < 1 || !shapes_ok(T, H, V)) return SAPO_ERR_INVALID_ARG;
+  int sms = sm_count();
+  if (sms <= 0) return SAPO_ERR_CUDA;
+  const size_t need = fwd_layout(T, H, V, dtype, sms).total +
+                      (seq_surr ? 0 : round_up<size_t>((size_t)S * sizeof(float), 256));
+  if (need > (size_t)SAPO_STATIC_SCRATCH_BYTES) return SAPO_ERR_STATIC_SCRATCH_EXCEEDED;
+  void* scratch = nullptr;
+  const int rc = static_scratch(&scratch);
+  if (rc != SAPO_OK) return rc;
+  // Nothing in the scratch has to start at zero: the vocab-split partials and the per-sequence
+  // sums are written for every token / sequence of this call before anything reads them.
+  return sapo_policy_loss_fwd(hidden, W_head, dtype, T, H, V, ld_hidden, ld_W, ids, old_logp, adv,
+                              cu_seqlens, S, h_cfg, logp, lse, ratio, surr, gscale, seq_surr, loss,
+                              scratch, (size_t)SAPO_STATIC_SCRATCH_BYTES, status, stream);
+}
+
 extern "C" int sapo_policy_loss_bwd(const void* hidden, const void* W_head, int32_t dtype,
                                     int64_t T, int32_t H, int32_t V, int64_t ld_hidden, int64_t ld_W,
                                     const int32_t* ids, const float* lse, const float* gscale,

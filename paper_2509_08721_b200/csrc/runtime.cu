@@ -48,6 +48,7 @@ extern "C" const char* sapo_status_string(int32_t code) {
     case SAPO_ERR_UNSUPPORTED_SHAPE: return "unsupported shape";
     case SAPO_ERR_WORKSPACE_TOO_SMALL: return "workspace too small";
     case SAPO_ERR_CUDA: return "CUDA error";
+    case SAPO_ERR_STATIC_SCRATCH_EXCEEDED: return "sizes exceed the built-in static scratch";
     default: return "unknown code";
   }
 }
