@@ -39,6 +39,7 @@ struct Sched {
   int32_t num_m_blocks, num_n_blocks, n_per_unit, units_per_m, num_units, num_k_blocks;
   int32_t m_fastest;  // 1: neighbouring CTAs share the B tile; 0: they share the A tile
   int32_t N;          // true extent of the n dimension (tail tiles use a narrower MMA)
+  int32_t stats_id;   // row of the wait-cycle counters this launch adds to (instrumented builds)
 };
 
 __device__ __forceinline__ void decode_unit(const Sched& s, int unit, int& mb, int& un,
@@ -164,6 +165,21 @@ struct StoreEpi {
   __device__ __forceinline__ void end_unit(const Params&, int) {}
 };
 
+// Optional instrumentation (compile with -DSAPO_WAIT_STATS): cycles each role spends waiting.
+#ifdef SAPO_WAIT_STATS
+__device__ unsigned long long g_wait_stats[4][8];
+#define SAPO_TIMED(slot, expr) ([&] { const long long t0_ = clock64(); const bool r_ = (expr); \
+                                      wait_cycles[slot] += clock64() - t0_; return r_; }())
+#define SAPO_STATS_DECL long long wait_cycles[8] = {0, 0, 0, 0, 0, 0, 0, 0}; const long long role_t0 = clock64();
+#define SAPO_STATS_FLUSH(total_slot) do { wait_cycles[total_slot] += clock64() - role_t0; \
+    for (int i_ = 0; i_ < 8; ++i_) if (wait_cycles[i_]) \
+      atomicAdd(&g_wait_stats[sched.stats_id & 3][i_], (unsigned long long)wait_cycles[i_]); } while (0)
+#else
+#define SAPO_TIMED(slot, expr) (expr)
+#define SAPO_STATS_DECL
+#define SAPO_STATS_FLUSH(total_slot) do {} while (0)
+#endif
+
 // ---------------------------------------------------------------------------- the GEMM kernel
 // D[m, n] = sum_k A[m, k] * B[n, k].
 //   A_MN = false: A is stored [M, K] with K contiguous; map box {64 k, 128 m}
@@ -201,41 +217,46 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
   fence_after_sync();
   const uint32_t tmem_base = *tmem_slot;
 
-  if (warp == 0 && lane == 0) {
+  if (warp == 0) {
     // ------------------------------------------------------------ TMA producer
+    // The whole warp walks the schedule; lane 0 posts the expected byte count and lane i
+    // issues box i of the stage (one box for a K-major operand, one per 64 columns for an
+    // MN-major one), so that the boxes of a stage are issued by one instruction.
+    SAPO_STATS_DECL
     int stage = 0; uint32_t phase = 0;
     uint32_t in_flight = 0;   // bit i: stage i was filled in the current ring pass
     bool ok = true;
+    constexpr int A_BOXES = A_MN ? 2 : 1;
     for (int unit = blockIdx.x; ok && unit < sched.num_units; unit += gridDim.x) {
       int mb, un, n_begin, n_end;
       decode_unit(sched, unit, mb, un, n_begin, n_end);
       for (int nb = n_begin; ok && nb < n_end; ++nb) {
         const int n_eff = tile_n_eff(sched, nb);
-        const int b_chunks = (n_eff + 63) >> 6;
-        const uint32_t tx = A_STAGE_BYTES + (B_MN ? b_chunks * CHUNK_BYTES : B_STAGE_BYTES);
+        const int b_boxes = B_MN ? ((n_eff + 63) >> 6) : 1;
+        const uint32_t tx = A_STAGE_BYTES + (B_MN ? b_boxes * CHUNK_BYTES : B_STAGE_BYTES);
+        // this lane's box: which map, where in the stage, and its coordinates apart from k
+        const bool mine = lane < A_BOXES + b_boxes;
+        const bool is_a = lane < A_BOXES;
+        const int bi = is_a ? lane : lane - A_BOXES;
+        const CUtensorMap* map = is_a ? &map_a : &map_b;
+        const uint32_t dst_off = is_a ? bi * CHUNK_BYTES : STAGES * A_STAGE_BYTES + bi * CHUNK_BYTES;
+        const bool mn = is_a ? A_MN : B_MN;
+        const int row0 = is_a ? mb * BM + 64 * bi : nb * BN + 64 * bi;   // m or n coordinate
         for (int kb = 0; kb < sched.num_k_blocks; ++kb) {
-          if (!mbar_wait(&empty[stage], phase ^ 1, abort_flag)) { ok = false; break; }
-          mbar_arrive_expect_tx(&full[stage], tx);
-          uint8_t* sa = smem_a + stage * A_STAGE_BYTES;
-          uint8_t* sb = smem_b + stage * B_STAGE_BYTES;
-          if (A_MN) {
-            tma_load_2d(sa, &map_a, &full[stage], mb * BM, kb * BK);
-            tma_load_2d(sa + CHUNK_BYTES, &map_a, &full[stage], mb * BM + 64, kb * BK);
-          } else {
-            tma_load_2d(sa, &map_a, &full[stage], kb * BK, mb * BM);
-          }
-          if (B_MN) {
-            for (int c = 0; c < b_chunks; ++c)
-              tma_load_2d(sb + c * CHUNK_BYTES, &map_b, &full[stage], nb * BN + 64 * c, kb * BK);
-          } else {
-            tma_load_2d(sb, &map_b, &full[stage], kb * BK, nb * BN);
+          if (!SAPO_TIMED(0, mbar_wait(&empty[stage], phase ^ 1, abort_flag))) { ok = false; break; }
+          if (lane == 0) mbar_arrive_expect_tx(&full[stage], tx);
+          if (mine) {
+            uint8_t* dst = smem + dst_off + stage * (is_a ? A_STAGE_BYTES : B_STAGE_BYTES);
+            if (mn) tma_load_2d(dst, map, &full[stage], row0, kb * BK);
+            else    tma_load_2d(dst, map, &full[stage], kb * BK, row0);
           }
           in_flight |= 1u << stage;
           if (++stage == STAGES) { stage = 0; phase ^= 1; }
         }
       }
     }
-    if (!ok) {
+    if (lane == 0) SAPO_STATS_FLUSH(4);
+    if (!ok && lane == 0) {
       // give copies already issued a bounded chance to land before the CTA leaves
       for (int i = 0; i < STAGES; ++i) {
         if (!(in_flight & (1u << i))) continue;
@@ -245,6 +266,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
     }
   } else if (warp == 1 && lane == 0) {
     // ------------------------------------------------------------ MMA issuer
+    SAPO_STATS_DECL
     int stage = 0; uint32_t phase = 0;
     int acc = 0; uint32_t acc_phase = 0;
     bool ok = true;
@@ -253,11 +275,11 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
       decode_unit(sched, unit, mb, un, n_begin, n_end);
       for (int nb = n_begin; ok && nb < n_end; ++nb) {
         const uint32_t idesc = make_idesc_bf16(BM, tile_n_eff(sched, nb), A_MN, B_MN);
-        if (!mbar_wait(&acc_empty[acc], acc_phase ^ 1, abort_flag)) { ok = false; break; }
+        if (!SAPO_TIMED(2, mbar_wait(&acc_empty[acc], acc_phase ^ 1, abort_flag))) { ok = false; break; }
         fence_after_sync();
         const uint32_t d_tmem = tmem_base + acc * BN;
         for (int kb = 0; kb < sched.num_k_blocks; ++kb) {
-          if (!mbar_wait(&full[stage], phase, abort_flag)) { ok = false; break; }
+          if (!SAPO_TIMED(1, mbar_wait(&full[stage], phase, abort_flag))) { ok = false; break; }
           fence_after_sync();
           const uint32_t a_addr = smem_u32(smem_a + stage * A_STAGE_BYTES);
           const uint32_t b_addr = smem_u32(smem_b + stage * B_STAGE_BYTES);
@@ -277,10 +299,12 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
         if (++acc == 2) { acc = 0; acc_phase ^= 1; }
       }
     }
+    SAPO_STATS_FLUSH(5);
   } else if (warp >= 2) {
     // ------------------------------------------------------------ epilogue (128 threads)
     const int quad = warp & 3;                    // TMEM lane quadrant this warp may read
     const int r = quad * 32 + lane;
+    SAPO_STATS_DECL
     int acc = 0; uint32_t acc_phase = 0;
     bool ok = true;
     Epi epi;
@@ -289,7 +313,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
       decode_unit(sched, unit, mb, un, n_begin, n_end);
       epi.begin_unit(ep, mb, r);
       for (int nb = n_begin; ok && nb < n_end; ++nb) {
-        if (!mbar_wait(&acc_full[acc], acc_phase, abort_flag)) { ok = false; break; }
+        if (!SAPO_TIMED(3, mbar_wait(&acc_full[acc], acc_phase, abort_flag))) { ok = false; break; }
         fence_after_sync();
         const uint32_t t_addr = tmem_base + (static_cast<uint32_t>(quad * 32) << 16) + acc * BN;
         const int n_eff = tile_n_eff(sched, nb);
@@ -305,6 +329,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
       }
       if (ok) epi.end_unit(ep, un);
     }
+    if (threadIdx.x == 64) SAPO_STATS_FLUSH(6);
   }
 
   fence_before_sync();
@@ -478,9 +503,11 @@ static int launch_gemm(const CUtensorMap& ma, const CUtensorMap& mb, const Sched
   if (sms <= 0) return SAPO_ERR_CUDA;
   const int grid = sched.num_units < sms ? sched.num_units : sms;
   if (grid <= 0) return SAPO_OK;
+  Sched sc = sched;
+  sc.stats_id = kernel_id == SAPO_K_FWD_GEMM ? 0 : kernel_id - SAPO_K_BWD_DZ + 1;
   {
     KernelScope scope(kernel_id, st);
-    kern<<<grid, GEMM_THREADS, GEMM_SMEM_BYTES, st>>>(ma, mb, sched, ep, status);
+    kern<<<grid, GEMM_THREADS, GEMM_SMEM_BYTES, st>>>(ma, mb, sc, ep, status);
   }
   return check_launch();
 }
@@ -751,3 +778,19 @@ extern "C" int sapo_policy_loss_bwd(const void* hidden, const void* W_head, int3
   }
   return SAPO_OK;
 }
+
+#ifdef SAPO_WAIT_STATS
+// Rows: forward, dz, dH, dW.  Columns: [0] TMA waits on free stages, [1] MMA waits on filled
+// stages, [2] MMA waits on a free accumulator, [3] one epilogue thread's waits on a full
+// accumulator, [4..6] total cycles of the TMA / MMA / that epilogue thread; summed over CTAs
+// and launches since the last reset.
+extern "C" int sapo_debug_wait_stats(unsigned long long* h_out, int32_t reset) {
+  if (h_out && cudaMemcpyFromSymbol(h_out, sapo::g_wait_stats, sizeof(unsigned long long) * 32) != cudaSuccess)
+    return SAPO_ERR_CUDA;
+  if (reset) {
+    unsigned long long z[32] = {0};
+    if (cudaMemcpyToSymbol(sapo::g_wait_stats, z, sizeof(z)) != cudaSuccess) return SAPO_ERR_CUDA;
+  }
+  return SAPO_OK;
+}
+#endif
