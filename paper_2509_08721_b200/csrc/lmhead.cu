@@ -5,7 +5,8 @@
 // serves four contractions; they differ only in operand majors and in the epilogue that
 // drains the accumulator:
 //   forward      S = hidden . W^T      epilogue: running max / sum-exp / target logit per token
-//   backward dz  S = hidden . W^T      epilogue: dz = g (onehot - exp(S - lse)) -> bf16 panel
+//   backward dz  S = hidden . W^T      epilogue: dz = g (onehot - exp(S - lse)) -> bf16 panel,
+//                                      stored as contiguous [128 token x 64 vocab] tiles
 //   backward dH  dH = dz . W           epilogue: fp32 store
 //   backward dW  dW = dz^T . hidden    epilogue: fp32 store / accumulate
 // The [tokens x vocab] logits never reach global memory (paper Section 3.2 asks for the
@@ -39,6 +40,8 @@ struct Sched {
   int32_t num_m_blocks, num_n_blocks, n_per_unit, units_per_m, num_units, num_k_blocks;
   int32_t m_fastest;  // 1: neighbouring CTAs share the B tile; 0: they share the A tile
   int32_t N;          // true extent of the n dimension (tail tiles use a narrower MMA)
+  int32_t n_cover;    // columns the epilogue visits (>= N; the dz panel is padded to 64)
+  int32_t panel_nvt;  // 64-column tiles per token block of the dz panel (tiled A operands)
   int32_t stats_id;   // row of the wait-cycle counters this launch adds to (instrumented builds)
 };
 
@@ -100,21 +103,26 @@ struct FwdEpi {
 };
 
 // Backward, first contraction: dz[t,v] = g_t ([v == y_t] - exp(z[t,v] - lse_t)), to bf16.
+// The panel is a sequence of [128 token x 64 vocab] tiles of 16 KB, tile (tb, vt) at index
+// tb * nvt + vt, each tile row-major: both later contractions then fetch whole contiguous
+// tiles (dH) or half tiles (dW) with one TMA box.  Rows past the last token and columns past
+// V are written as zeros, because those consumers cannot tell them from data.
 struct DzEpi {
   struct Params {
     const int32_t* ids; const float* lse; const float* gscale; __nv_bfloat16* P;
-    int64_t M; int32_t V; int64_t Vp;   // panel [M, Vp], Vp a multiple of 64
+    int64_t M; int32_t V; int32_t nvt;
   };
-  float g, l2; int32_t y; int64_t row; bool valid;
-  __device__ __forceinline__ void begin_unit(const Params& p, int mb, int r) {
-    row = (int64_t)mb * BM + r;
-    valid = row < p.M;
+  float g, l2; int32_t y; int64_t tile_row0; int r;
+  __device__ __forceinline__ void begin_unit(const Params& p, int mb, int r_) {
+    const int64_t row = (int64_t)mb * BM + r_;
+    const bool valid = row < p.M;
+    r = r_;
+    tile_row0 = (int64_t)mb * p.nvt * BM;          // first panel row of this token block
     g = valid ? p.gscale[row] : 0.f;
     l2 = valid ? p.lse[row] * LOG2E : 0.f;
     y = valid ? p.ids[row] : -1;
   }
   __device__ __forceinline__ void chunk(const Params& p, float (&v)[32], int col0) {
-    if (!valid || col0 >= p.Vp) return;
     uint32_t packed[16];
     if (g == 0.f) {
       #pragma unroll
@@ -134,7 +142,9 @@ struct DzEpi {
         packed[j] = *reinterpret_cast<uint32_t*>(&h);
       }
     }
-    uint4* dst = reinterpret_cast<uint4*>(p.P + row * p.Vp + col0);
+    const int vt = col0 >> 6;
+    __nv_bfloat16* at = p.P + ((tile_row0 + (int64_t)vt * BM + r) << 6) + (col0 & 32);
+    uint4* dst = reinterpret_cast<uint4*>(at);
     #pragma unroll
     for (int q = 0; q < 4; ++q)
       dst[q] = make_uint4(packed[4 * q], packed[4 * q + 1], packed[4 * q + 2], packed[4 * q + 3]);
@@ -182,10 +192,12 @@ __device__ unsigned long long g_wait_stats[4][8];
 
 // ---------------------------------------------------------------------------- the GEMM kernel
 // D[m, n] = sum_k A[m, k] * B[n, k].
-//   A_MN = false: A is stored [M, K] with K contiguous; map box {64 k, 128 m}
-//   A_MN = true : A is stored [K, M] with M contiguous; map box {64 m, 64 k}, two boxes per stage
-//   B likewise with N in place of M (256 rows, or four 64-wide boxes).
-template <bool A_MN, bool B_MN, class Epi>
+//   A_KIND 0: A is stored [M, K] with K contiguous; map box {64 k, 128 m}
+//   A_KIND 1: A is stored [K, M] with M contiguous; map box {64 m, 64 k}, two boxes per stage
+//   A_KIND 2: A is the tiled dz panel read K-major  (M = tokens, K = vocab): one 128-row box
+//   A_KIND 3: A is the tiled dz panel read MN-major (M = vocab, K = tokens): two 64-row boxes
+//   B_MN false / true: like kinds 0 / 1 with N in place of M (256 rows, or four 64-wide boxes).
+template <int A_KIND, bool B_MN, class Epi>
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
 umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                  const Sched sched, const typename Epi::Params ep, int32_t* status) {
@@ -202,6 +214,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  constexpr bool A_MN = (A_KIND & 1) != 0;
 
   if (threadIdx.x == 0) {
     for (int i = 0; i < STAGES; ++i) { mbar_init(&full[i], 1); mbar_init(&empty[i], 1); }
@@ -247,8 +260,13 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
           if (lane == 0) mbar_arrive_expect_tx(&full[stage], tx);
           if (mine) {
             uint8_t* dst = smem + dst_off + stage * (is_a ? A_STAGE_BYTES : B_STAGE_BYTES);
-            if (mn) tma_load_2d(dst, map, &full[stage], row0, kb * BK);
-            else    tma_load_2d(dst, map, &full[stage], kb * BK, row0);
+            if (is_a && A_KIND == 2)        // tile (token block mb, vocab tile kb), all 128 rows
+              tma_load_2d(dst, map, &full[stage], 0, (mb * sched.panel_nvt + kb) * BM);
+            else if (is_a && A_KIND == 3)   // tile (token block kb/2, vocab tile 2 mb + bi), one half
+              tma_load_2d(dst, map, &full[stage], 0,
+                          ((kb >> 1) * sched.panel_nvt + 2 * mb + bi) * BM + (kb & 1) * 64);
+            else if (mn) tma_load_2d(dst, map, &full[stage], row0, kb * BK);
+            else         tma_load_2d(dst, map, &full[stage], kb * BK, row0);
           }
           in_flight |= 1u << stage;
           if (++stage == STAGES) { stage = 0; phase ^= 1; }
@@ -316,8 +334,8 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
         if (!SAPO_TIMED(3, mbar_wait(&acc_full[acc], acc_phase, abort_flag))) { ok = false; break; }
         fence_after_sync();
         const uint32_t t_addr = tmem_base + (static_cast<uint32_t>(quad * 32) << 16) + acc * BN;
-        const int n_eff = tile_n_eff(sched, nb);
-        for (int c = 0; c * 32 < n_eff; ++c) {
+        const int n_visit = min(BN, sched.n_cover - nb * BN);
+        for (int c = 0; c * 32 < n_visit; ++c) {
           float v[32];
           tmem_ld32(t_addr + c * 32, v);
           tmem_ld_wait();
@@ -468,6 +486,8 @@ static Sched make_sched(int64_t M, int64_t N, int64_t K, int n_splits, bool m_fa
   s.num_k_blocks = (int32_t)ceil_div<int64_t>(K, BK);
   s.m_fastest = m_fastest ? 1 : 0;
   s.N = (int32_t)N;
+  s.n_cover = (int32_t)N;
+  s.panel_nvt = 0;
   return s;
 }
 
@@ -488,10 +508,10 @@ static int fwd_splits(int64_t T, int32_t V, int sms) {
   return (int)ceil_div(nb, per);
 }
 
-template <bool A_MN, bool B_MN, class Epi>
+template <int A_KIND, bool B_MN, class Epi>
 static int launch_gemm(const CUtensorMap& ma, const CUtensorMap& mb, const Sched& sched,
                        const typename Epi::Params& ep, int32_t* status, cudaStream_t st, int kernel_id) {
-  auto kern = umma_gemm_kernel<A_MN, B_MN, Epi>;
+  auto kern = umma_gemm_kernel<A_KIND, B_MN, Epi>;
   static bool attr_set = false;
   if (!attr_set) {
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)GEMM_SMEM_BYTES) !=
@@ -632,7 +652,7 @@ extern "C" int sapo_policy_loss_fwd(const void* hidden, const void* W_head, int3
   if (!make_map(&map_a, A, K, T, lda, BM) || !make_map(&map_b, B, K, V, ldb, BN)) return SAPO_ERR_CUDA;
   const Sched sched = make_sched(T, V, K, L.n_splits, /*m_fastest=*/true);
   FwdEpi::Params ep{ids, pm, ps, pz, T, V};
-  int rc = launch_gemm<false, false, FwdEpi>(map_a, map_b, sched, ep, status, st, SAPO_K_FWD_GEMM);
+  int rc = launch_gemm<0, false, FwdEpi>(map_a, map_b, sched, ep, status, st, SAPO_K_FWD_GEMM);
   if (rc != SAPO_OK) return rc;
 
   TailArgs ta{};
@@ -737,9 +757,11 @@ extern "C" int sapo_policy_loss_bwd(const void* hidden, const void* W_head, int3
     A = a1; B = b1; lda = H; ldb = H;
   }
   const int64_t Vp = padded_vocab(V);
+  const int32_t nvt = (int32_t)(Vp / 64);
   __nv_bfloat16* panel = reinterpret_cast<__nv_bfloat16*>(ws + L.panel);
-  int64_t rows_fit = (int64_t)((workspace_bytes - L.fixed) / L.bytes_per_row);
-  int64_t chunk_rows = rows_fit >= T ? T : (rows_fit / BM) * BM;
+  // whole 128-token blocks of the panel that fit; a chunk never ends inside a block it cannot hold
+  const int64_t rows_fit = ((int64_t)((workspace_bytes - L.fixed) / L.bytes_per_row) / BM) * BM;
+  const int64_t chunk_rows = rows_fit >= T ? T : rows_fit;
   if (chunk_rows <= 0) return SAPO_ERR_WORKSPACE_TOO_SMALL;
 
   // W as the K-major B operand of the logit recompute and as the MN-major B operand of dH
@@ -750,29 +772,34 @@ extern "C" int sapo_policy_loss_bwd(const void* hidden, const void* W_head, int3
   for (int64_t t0 = 0; t0 < T; t0 += chunk_rows) {
     const int64_t tc = (T - t0) < chunk_rows ? (T - t0) : chunk_rows;
     const __nv_bfloat16* A0 = A + t0 * lda;
-    CUtensorMap map_h_kmajor, map_h_mn, map_p_kmajor, map_p_mn;
+    const int64_t panel_rows = ceil_div<int64_t>(tc, BM) * nvt * BM;   // 128-byte rows of the tiled panel
+    CUtensorMap map_h_kmajor, map_h_mn, map_p_tile, map_p_half;
     if (!make_map(&map_h_kmajor, A0, H, tc, lda, BM) || !make_map(&map_h_mn, A0, H, tc, lda, 64) ||
-        !make_map(&map_p_kmajor, panel, V, tc, Vp, BM) || !make_map(&map_p_mn, panel, V, tc, Vp, 64))
+        !make_map(&map_p_tile, panel, 64, panel_rows, 64, BM) ||
+        !make_map(&map_p_half, panel, 64, panel_rows, 64, 64))
       return SAPO_ERR_CUDA;
     // dz panel: recompute logits tile by tile
     {
-      const Sched sched = make_sched(tc, V, H, 0, /*m_fastest=*/true);
-      DzEpi::Params ep{ids + t0, lse + t0, gscale + t0, panel, tc, V, Vp};
-      int rc = launch_gemm<false, false, DzEpi>(map_h_kmajor, map_w_kmajor, sched, ep, status, st, SAPO_K_BWD_DZ);
+      Sched sched = make_sched(tc, V, H, 0, /*m_fastest=*/true);
+      sched.n_cover = (int32_t)Vp;
+      DzEpi::Params ep{ids + t0, lse + t0, gscale + t0, panel, tc, V, nvt};
+      int rc = launch_gemm<0, false, DzEpi>(map_h_kmajor, map_w_kmajor, sched, ep, status, st, SAPO_K_BWD_DZ);
       if (rc != SAPO_OK) return rc;
     }
     // dhidden[t0:t0+tc] = dz . W         (M = tokens, N = H, K = V)
     {
-      const Sched sched = make_sched(tc, H, V, 0, /*m_fastest=*/false);
+      Sched sched = make_sched(tc, H, Vp, 0, /*m_fastest=*/false);
+      sched.panel_nvt = nvt;
       StoreEpi::Params ep{dhidden + t0 * (int64_t)H, H, tc, H, 0};
-      int rc = launch_gemm<false, true, StoreEpi>(map_p_kmajor, map_w_mn, sched, ep, status, st, SAPO_K_BWD_DH);
+      int rc = launch_gemm<2, true, StoreEpi>(map_p_tile, map_w_mn, sched, ep, status, st, SAPO_K_BWD_DH);
       if (rc != SAPO_OK) return rc;
     }
     // dW (+)= dz^T . hidden               (M = V, N = H, K = tokens)
     {
-      const Sched sched = make_sched(V, H, tc, 0, /*m_fastest=*/false);
+      Sched sched = make_sched(V, H, tc, 0, /*m_fastest=*/false);
+      sched.panel_nvt = nvt;
       StoreEpi::Params ep{dW_head, H, V, H, (t0 > 0 || accumulate_dW) ? 1 : 0};
-      int rc = launch_gemm<true, true, StoreEpi>(map_p_mn, map_h_mn, sched, ep, status, st, SAPO_K_BWD_DW);
+      int rc = launch_gemm<3, true, StoreEpi>(map_p_half, map_h_mn, sched, ep, status, st, SAPO_K_BWD_DW);
       if (rc != SAPO_OK) return rc;
     }
   }
