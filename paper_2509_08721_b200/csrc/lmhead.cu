@@ -21,25 +21,28 @@
 namespace sapo {
 using namespace umma;
 
-constexpr int BM = 128;            // accumulator rows  (TMEM lanes)
-constexpr int BN = 256;            // accumulator columns per tile
+constexpr int BM = 128;            // accumulator rows per CTA (TMEM lanes)
+constexpr int PAIR_M = 256;        // rows of a tile: two CTAs of a cluster share it
+constexpr int BN = 256;            // accumulator columns per tile (at most)
 constexpr int BK = 64;             // bf16 elements per 128-byte operand row
 constexpr int UMMA_K = 16;
-constexpr int STAGES = 4;
+constexpr int STAGES = 6;
 constexpr int GEMM_THREADS = 192;  // warp 0: TMA, warp 1: MMA, warps 2-5: epilogue
-constexpr uint32_t A_STAGE_BYTES = BM * 128;
-constexpr uint32_t B_STAGE_BYTES = BN * 128;
+constexpr uint32_t A_STAGE_BYTES = BM * 128;         // this CTA's 128 rows of A
+constexpr uint32_t B_STAGE_BYTES = (BN / 2) * 128;   // this CTA's half of the tile's B columns
 constexpr uint32_t CHUNK_BYTES = 64 * 128;   // one 64-row box of an MN-major operand
 constexpr uint32_t TMEM_COLS = 512;          // two accumulators of 256 columns
 constexpr size_t GEMM_SMEM_BYTES = 1024 + STAGES * (A_STAGE_BYTES + B_STAGE_BYTES) + 256;
 constexpr float LOG2E = 1.4426950408889634f;
 constexpr float LN2 = 0.6931471805599453f;
 
-// Static tile schedule: `num_units` work units, each one m-block and a run of n-blocks.
+// Static tile schedule: `num_units` work units, each one 256-row block and a run of n-blocks,
+// dealt round-robin to the CTA pairs.
 struct Sched {
   int32_t num_m_blocks, num_n_blocks, n_per_unit, units_per_m, num_units, num_k_blocks;
-  int32_t m_fastest;  // 1: neighbouring CTAs share the B tile; 0: they share the A tile
-  int32_t N;          // true extent of the n dimension (tail tiles use a narrower MMA)
+  int32_t m_fastest;  // 1: neighbouring pairs share the B tile; 0: they share the A tile
+  int32_t N;          // true extent of the n dimension
+  int32_t tile_n;     // columns per tile (a multiple of 32, at most 256)
   int32_t n_cover;    // columns the epilogue visits (>= N; the dz panel is padded to 64)
   int32_t panel_nvt;  // 64-column tiles per token block of the dz panel (tiled A operands)
   int32_t stats_id;   // row of the wait-cycle counters this launch adds to (instrumented builds)
@@ -53,10 +56,11 @@ __device__ __forceinline__ void decode_unit(const Sched& s, int unit, int& mb, i
   n_end = min(n_begin + s.n_per_unit, s.num_n_blocks);
 }
 
-// columns of a tile that hold real outputs, rounded up to the MMA's granularity of 16
+// columns of a tile the MMA computes: the tile width, or on the last tile what is left,
+// rounded up to 32 so that each CTA's half stays a multiple of 16
 __device__ __forceinline__ int tile_n_eff(const Sched& s, int nb) {
-  const int left = s.N - nb * BN;
-  return left >= BN ? BN : ((left + 15) & ~15);
+  const int left = s.N - nb * s.tile_n;
+  return left >= s.tile_n ? s.tile_n : ((left + 31) & ~31);
 }
 
 // ---------------------------------------------------------------------------- epilogues
@@ -112,10 +116,11 @@ struct DzEpi {
     const int32_t* ids; const float* lse; const float* gscale; __nv_bfloat16* P;
     int64_t M; int32_t V; int32_t nvt;
   };
-  float g, l2; int32_t y; int64_t tile_row0; int r;
+  float g, l2; int32_t y; int64_t tile_row0; int r; bool in_panel;
   __device__ __forceinline__ void begin_unit(const Params& p, int mb, int r_) {
     const int64_t row = (int64_t)mb * BM + r_;
     const bool valid = row < p.M;
+    in_panel = (int64_t)mb * BM < p.M;   // the odd CTA of the last pair may own no token block
     r = r_;
     tile_row0 = (int64_t)mb * p.nvt * BM;          // first panel row of this token block
     g = valid ? p.gscale[row] : 0.f;
@@ -123,6 +128,7 @@ struct DzEpi {
     y = valid ? p.ids[row] : -1;
   }
   __device__ __forceinline__ void chunk(const Params& p, float (&v)[32], int col0) {
+    if (!in_panel) return;
     uint32_t packed[16];
     if (g == 0.f) {
       #pragma unroll
@@ -191,12 +197,16 @@ __device__ unsigned long long g_wait_stats[4][8];
 #endif
 
 // ---------------------------------------------------------------------------- the GEMM kernel
-// D[m, n] = sum_k A[m, k] * B[n, k].
+// D[m, n] = sum_k A[m, k] * B[n, k], one 256 x tile_n tile per CTA pair and step.
 //   A_KIND 0: A is stored [M, K] with K contiguous; map box {64 k, 128 m}
 //   A_KIND 1: A is stored [K, M] with M contiguous; map box {64 m, 64 k}, two boxes per stage
 //   A_KIND 2: A is the tiled dz panel read K-major  (M = tokens, K = vocab): one 128-row box
 //   A_KIND 3: A is the tiled dz panel read MN-major (M = vocab, K = tokens): two 64-row boxes
-//   B_MN false / true: like kinds 0 / 1 with N in place of M (256 rows, or four 64-wide boxes).
+//   B_MN false: B is stored [N, K]; map box {64 k, 128 n}.  true: [K, N]; boxes {64 n, 64 k}.
+// CTA `rank` of the pair owns rows [256 mb + 128 rank, +128) of the tile and stages columns
+// [n0 + rank * n_eff / 2, + n_eff / 2) of B.  All TMA completions of a stage are counted on the
+// even CTA's barrier; the even CTA's MMA thread frees stages and publishes accumulators on
+// both CTAs' barriers.
 template <int A_KIND, bool B_MN, class Epi>
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
 umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
@@ -206,67 +216,71 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
   uint8_t* smem_a = smem;
   uint8_t* smem_b = smem + STAGES * A_STAGE_BYTES;
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + STAGES * (A_STAGE_BYTES + B_STAGE_BYTES));
-  uint64_t* full = bars;                 // [STAGES] TMA -> MMA
-  uint64_t* empty = bars + STAGES;       // [STAGES] MMA -> TMA
-  uint64_t* acc_full = bars + 2 * STAGES;      // [2] MMA -> epilogue
-  uint64_t* acc_empty = bars + 2 * STAGES + 2; // [2] epilogue -> MMA
+  uint64_t* full = bars;                 // [STAGES] TMA -> MMA          (even CTA's are used)
+  uint64_t* empty = bars + STAGES;       // [STAGES] MMA -> TMA          (each CTA waits on its own)
+  uint64_t* acc_full = bars + 2 * STAGES;      // [2] MMA -> epilogue    (each CTA waits on its own)
+  uint64_t* acc_empty = bars + 2 * STAGES + 2; // [2] epilogue -> MMA    (even CTA's are used)
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * STAGES + 4);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   constexpr bool A_MN = (A_KIND & 1) != 0;
+  const uint32_t rank = cluster_cta_rank();
+  const int pair = blockIdx.x >> 1, num_pairs = gridDim.x >> 1;
 
   if (threadIdx.x == 0) {
     for (int i = 0; i < STAGES; ++i) { mbar_init(&full[i], 1); mbar_init(&empty[i], 1); }
-    for (int i = 0; i < 2; ++i) { mbar_init(&acc_full[i], 1); mbar_init(&acc_empty[i], 128); }
+    for (int i = 0; i < 2; ++i) { mbar_init(&acc_full[i], 1); mbar_init(&acc_empty[i], 8); }
     *abort_flag = 0;
     fence_mbar_init();
     prefetch_tensormap(&map_a);
     prefetch_tensormap(&map_b);
   }
-  if (warp == 1) { tmem_alloc(tmem_slot, TMEM_COLS); tmem_relinquish(); }
+  if (warp == 1) { tmem_alloc_pair(tmem_slot, TMEM_COLS); tmem_relinquish_pair(); }
   fence_before_sync();
   __syncthreads();
+  cluster_sync_all();
   fence_after_sync();
   const uint32_t tmem_base = *tmem_slot;
 
   if (warp == 0) {
-    // ------------------------------------------------------------ TMA producer
-    // The whole warp walks the schedule; lane 0 posts the expected byte count and lane i
-    // issues box i of the stage (one box for a K-major operand, one per 64 columns for an
-    // MN-major one), so that the boxes of a stage are issued by one instruction.
+    // ------------------------------------------------------------ TMA producer (both CTAs)
+    // The whole warp walks the schedule; lane i issues box i of this CTA's share of the
+    // stage; lane 0 of the even CTA posts the byte count of both CTAs' shares.
     SAPO_STATS_DECL
     int stage = 0; uint32_t phase = 0;
     uint32_t in_flight = 0;   // bit i: stage i was filled in the current ring pass
     bool ok = true;
     constexpr int A_BOXES = A_MN ? 2 : 1;
-    for (int unit = blockIdx.x; ok && unit < sched.num_units; unit += gridDim.x) {
-      int mb, un, n_begin, n_end;
-      decode_unit(sched, unit, mb, un, n_begin, n_end);
+    for (int unit = pair; ok && unit < sched.num_units; unit += num_pairs) {
+      int pmb, un, n_begin, n_end;
+      decode_unit(sched, unit, pmb, un, n_begin, n_end);
+      const int mb = 2 * pmb + (int)rank;                 // this CTA's 128-row block
       for (int nb = n_begin; ok && nb < n_end; ++nb) {
-        const int n_eff = tile_n_eff(sched, nb);
-        const int b_boxes = B_MN ? ((n_eff + 63) >> 6) : 1;
-        const uint32_t tx = A_STAGE_BYTES + (B_MN ? b_boxes * CHUNK_BYTES : B_STAGE_BYTES);
-        // this lane's box: which map, where in the stage, and its coordinates apart from k
+        const int half = tile_n_eff(sched, nb) >> 1;       // B columns this CTA stages
+        const int b_boxes = B_MN ? ((half + 63) >> 6) : 1;
+        const uint32_t tx = 2 * (A_STAGE_BYTES + (B_MN ? b_boxes * CHUNK_BYTES : B_STAGE_BYTES));
         const bool mine = lane < A_BOXES + b_boxes;
         const bool is_a = lane < A_BOXES;
         const int bi = is_a ? lane : lane - A_BOXES;
         const CUtensorMap* map = is_a ? &map_a : &map_b;
         const uint32_t dst_off = is_a ? bi * CHUNK_BYTES : STAGES * A_STAGE_BYTES + bi * CHUNK_BYTES;
         const bool mn = is_a ? A_MN : B_MN;
-        const int row0 = is_a ? mb * BM + 64 * bi : nb * BN + 64 * bi;   // m or n coordinate
+        const int row0 = is_a ? mb * BM + 64 * bi
+                              : nb * sched.tile_n + (int)rank * half + 64 * bi;   // m or n coordinate
         for (int kb = 0; kb < sched.num_k_blocks; ++kb) {
-          if (!SAPO_TIMED(0, mbar_wait(&empty[stage], phase ^ 1, abort_flag))) { ok = false; break; }
-          if (lane == 0) mbar_arrive_expect_tx(&full[stage], tx);
+          if (!SAPO_TIMED(0, mbar_wait_cluster(&empty[stage], phase ^ 1, abort_flag))) { ok = false; break; }
+          if (rank == 0 && lane == 0) mbar_arrive_expect_tx(&full[stage], tx);
           if (mine) {
             uint8_t* dst = smem + dst_off + stage * (is_a ? A_STAGE_BYTES : B_STAGE_BYTES);
+            const uint32_t bar = map_to_cta(smem_u32(&full[stage]), 0);
             if (is_a && A_KIND == 2)        // tile (token block mb, vocab tile kb), all 128 rows
-              tma_load_2d(dst, map, &full[stage], 0, (mb * sched.panel_nvt + kb) * BM);
+              tma_load_2d_pair(dst, map, bar, 0, (mb * sched.panel_nvt + kb) * BM);
             else if (is_a && A_KIND == 3)   // tile (token block kb/2, vocab tile 2 mb + bi), one half
-              tma_load_2d(dst, map, &full[stage], 0,
-                          ((kb >> 1) * sched.panel_nvt + 2 * mb + bi) * BM + (kb & 1) * 64);
-            else if (mn) tma_load_2d(dst, map, &full[stage], row0, kb * BK);
-            else         tma_load_2d(dst, map, &full[stage], kb * BK, row0);
+              tma_load_2d_pair(dst, map, bar, 0,
+                               ((kb >> 1) * sched.panel_nvt + 2 * mb + bi) * BM + (kb & 1) * 64);
+            else if (mn) tma_load_2d_pair(dst, map, bar, row0, kb * BK);
+            else         tma_load_2d_pair(dst, map, bar, kb * BK, row0);
           }
           in_flight |= 1u << stage;
           if (++stage == STAGES) { stage = 0; phase ^= 1; }
@@ -274,30 +288,30 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
       }
     }
     if (lane == 0) SAPO_STATS_FLUSH(4);
-    if (!ok && lane == 0) {
-      // give copies already issued a bounded chance to land before the CTA leaves
+    if (!ok && rank == 0 && lane == 0) {
+      // give copies already issued a bounded chance to land before the pair leaves
       for (int i = 0; i < STAGES; ++i) {
         if (!(in_flight & (1u << i))) continue;
         const uint32_t ph = (i < stage) ? phase : (phase ^ 1);
-        for (int spin = 0; spin < (1 << 20) && !mbar_try_wait(&full[i], ph); ++spin) {}
+        for (int spin = 0; spin < (1 << 20) && !mbar_try_wait_cluster(&full[i], ph); ++spin) {}
       }
     }
-  } else if (warp == 1 && lane == 0) {
-    // ------------------------------------------------------------ MMA issuer
+  } else if (warp == 1 && lane == 0 && rank == 0) {
+    // ------------------------------------------------------------ MMA issuer (even CTA only)
     SAPO_STATS_DECL
     int stage = 0; uint32_t phase = 0;
     int acc = 0; uint32_t acc_phase = 0;
     bool ok = true;
-    for (int unit = blockIdx.x; ok && unit < sched.num_units; unit += gridDim.x) {
-      int mb, un, n_begin, n_end;
-      decode_unit(sched, unit, mb, un, n_begin, n_end);
+    for (int unit = pair; ok && unit < sched.num_units; unit += num_pairs) {
+      int pmb, un, n_begin, n_end;
+      decode_unit(sched, unit, pmb, un, n_begin, n_end);
       for (int nb = n_begin; ok && nb < n_end; ++nb) {
-        const uint32_t idesc = make_idesc_bf16(BM, tile_n_eff(sched, nb), A_MN, B_MN);
-        if (!SAPO_TIMED(2, mbar_wait(&acc_empty[acc], acc_phase ^ 1, abort_flag))) { ok = false; break; }
+        const uint32_t idesc = make_idesc_bf16(PAIR_M, tile_n_eff(sched, nb), A_MN, B_MN);
+        if (!SAPO_TIMED(2, mbar_wait_cluster(&acc_empty[acc], acc_phase ^ 1, abort_flag))) { ok = false; break; }
         fence_after_sync();
         const uint32_t d_tmem = tmem_base + acc * BN;
         for (int kb = 0; kb < sched.num_k_blocks; ++kb) {
-          if (!SAPO_TIMED(1, mbar_wait(&full[stage], phase, abort_flag))) { ok = false; break; }
+          if (!SAPO_TIMED(1, mbar_wait_cluster(&full[stage], phase, abort_flag))) { ok = false; break; }
           fence_after_sync();
           const uint32_t a_addr = smem_u32(smem_a + stage * A_STAGE_BYTES);
           const uint32_t b_addr = smem_u32(smem_b + stage * B_STAGE_BYTES);
@@ -308,41 +322,50 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
                                          : make_smem_desc(a_addr + k * 32, 16, 1024);
             const uint64_t b_desc = B_MN ? make_smem_desc(b_addr + k * 2048, CHUNK_BYTES, 1024)
                                          : make_smem_desc(b_addr + k * 32, 16, 1024);
-            mma_bf16(d_tmem, a_desc, b_desc, idesc, (kb | k) != 0 ? 1u : 0u);
+            mma_bf16_pair(d_tmem, a_desc, b_desc, idesc, (kb | k) != 0 ? 1u : 0u);
           }
-          mma_commit(&empty[stage]);              // frees the stage once these MMAs retire
+          // free the stage in both CTAs once these MMAs retire
+          const uint32_t e = smem_u32(&empty[stage]);
+          mma_commit_pair(map_to_cta(e, 0));
+          mma_commit_pair(map_to_cta(e, 1));
           if (++stage == STAGES) { stage = 0; phase ^= 1; }
         }
-        if (ok) mma_commit(&acc_full[acc]);       // accumulator complete
+        if (ok) {                                  // accumulator complete, in both CTAs
+          const uint32_t f = smem_u32(&acc_full[acc]);
+          mma_commit_pair(map_to_cta(f, 0));
+          mma_commit_pair(map_to_cta(f, 1));
+        }
         if (++acc == 2) { acc = 0; acc_phase ^= 1; }
       }
     }
     SAPO_STATS_FLUSH(5);
   } else if (warp >= 2) {
-    // ------------------------------------------------------------ epilogue (128 threads)
+    // ------------------------------------------------------------ epilogue (128 threads, both CTAs)
     const int quad = warp & 3;                    // TMEM lane quadrant this warp may read
     const int r = quad * 32 + lane;
     SAPO_STATS_DECL
     int acc = 0; uint32_t acc_phase = 0;
     bool ok = true;
     Epi epi;
-    for (int unit = blockIdx.x; ok && unit < sched.num_units; unit += gridDim.x) {
-      int mb, un, n_begin, n_end;
-      decode_unit(sched, unit, mb, un, n_begin, n_end);
-      epi.begin_unit(ep, mb, r);
+    for (int unit = pair; ok && unit < sched.num_units; unit += num_pairs) {
+      int pmb, un, n_begin, n_end;
+      decode_unit(sched, unit, pmb, un, n_begin, n_end);
+      epi.begin_unit(ep, 2 * pmb + (int)rank, r);
       for (int nb = n_begin; ok && nb < n_end; ++nb) {
-        if (!SAPO_TIMED(3, mbar_wait(&acc_full[acc], acc_phase, abort_flag))) { ok = false; break; }
+        if (!SAPO_TIMED(3, mbar_wait_cluster(&acc_full[acc], acc_phase, abort_flag))) { ok = false; break; }
         fence_after_sync();
         const uint32_t t_addr = tmem_base + (static_cast<uint32_t>(quad * 32) << 16) + acc * BN;
-        const int n_visit = min(BN, sched.n_cover - nb * BN);
+        const int n0 = nb * sched.tile_n;
+        const int n_visit = min(sched.tile_n, sched.n_cover - n0);
         for (int c = 0; c * 32 < n_visit; ++c) {
           float v[32];
           tmem_ld32(t_addr + c * 32, v);
           tmem_ld_wait();
-          epi.chunk(ep, v, nb * BN + c * 32);
+          epi.chunk(ep, v, n0 + c * 32);
         }
         fence_before_sync();
-        mbar_arrive(&acc_empty[acc]);
+        __syncwarp();
+        if (lane == 0) mbar_arrive_cluster(map_to_cta(smem_u32(&acc_empty[acc]), 0));
         if (++acc == 2) { acc = 0; acc_phase ^= 1; }
       }
       if (ok) epi.end_unit(ep, un);
@@ -350,9 +373,11 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
     if (threadIdx.x == 64) SAPO_STATS_FLUSH(6);
   }
 
+  // neither CTA may leave while the other can still touch its shared or tensor memory
   fence_before_sync();
   __syncthreads();
-  if (warp == 1) { fence_after_sync(); tmem_dealloc(tmem_base, TMEM_COLS); }
+  cluster_sync_all();
+  if (warp == 1) { fence_after_sync(); tmem_dealloc_pair(tmem_base, TMEM_COLS); }
   if (threadIdx.x == 0 && *abort_flag) raise_status(status, SAPO_ST_WAIT_TIMEOUT);
 }
 
@@ -478,8 +503,10 @@ static bool make_map(CUtensorMap* map, const void* base, int64_t inner, int64_t 
 
 static Sched make_sched(int64_t M, int64_t N, int64_t K, int n_splits, bool m_fastest) {
   Sched s{};
-  s.num_m_blocks = (int32_t)ceil_div<int64_t>(M, BM);
-  s.num_n_blocks = (int32_t)ceil_div<int64_t>(N, BN);
+  s.num_m_blocks = (int32_t)ceil_div<int64_t>(M, PAIR_M);
+  const int64_t tiles = ceil_div<int64_t>(N, BN);
+  s.tile_n = (int32_t)round_up<int64_t>(ceil_div<int64_t>(N, tiles), 32);   // equal-width tiles
+  s.num_n_blocks = (int32_t)ceil_div<int64_t>(N, s.tile_n);
   s.n_per_unit = n_splits > 0 ? ceil_div(s.num_n_blocks, n_splits) : 1;
   s.units_per_m = ceil_div(s.num_n_blocks, s.n_per_unit);
   s.num_units = s.num_m_blocks * s.units_per_m;
@@ -491,18 +518,19 @@ static Sched make_sched(int64_t M, int64_t N, int64_t K, int n_splits, bool m_fa
   return s;
 }
 
-// Number of vocab splits of the forward pass: enough units to cover the SMs when there are
-// few token blocks, never more than there are vocab tiles.
+// Number of vocab splits of the forward pass: enough units to keep every CTA pair busy when
+// there are few token blocks, never more than there are vocab tiles.
 static int fwd_splits(int64_t T, int32_t V, int sms) {
-  const int64_t mb = ceil_div<int64_t>(T, BM);
+  const int64_t pairs = sms / 2 > 0 ? sms / 2 : 1;
+  const int64_t mb = ceil_div<int64_t>(T, PAIR_M);
   const int64_t nb = ceil_div<int64_t>(V, BN);
   int64_t best = 1; double best_eff = 0.0;
   for (int64_t sp = 1; sp <= 160 && sp <= nb; ++sp) {
     const int64_t per = ceil_div(nb, sp);
     const int64_t units = mb * ceil_div(nb, per);
-    const double eff = (double)units / (double)(ceil_div<int64_t>(units, sms) * sms);
+    const double eff = (double)units / (double)(ceil_div<int64_t>(units, pairs) * pairs);
     if (eff > best_eff + 1e-9) { best_eff = eff; best = sp; }
-    if (units >= 8 * (int64_t)sms) break;
+    if (units >= 8 * pairs) break;
   }
   const int64_t per = ceil_div(nb, best);
   return (int)ceil_div(nb, per);
@@ -512,22 +540,35 @@ template <int A_KIND, bool B_MN, class Epi>
 static int launch_gemm(const CUtensorMap& ma, const CUtensorMap& mb, const Sched& sched,
                        const typename Epi::Params& ep, int32_t* status, cudaStream_t st, int kernel_id) {
   auto kern = umma_gemm_kernel<A_KIND, B_MN, Epi>;
-  static bool attr_set = false;
-  if (!attr_set) {
+  static int max_pairs = 0;     // CTA pairs the device can hold at once, found on first use
+  if (sched.num_units <= 0) return SAPO_OK;
+  Sched sc = sched;
+  sc.stats_id = kernel_id == SAPO_K_FWD_GEMM ? 0 : kernel_id - SAPO_K_BWD_DZ + 1;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+  cudaLaunchConfig_t cfg = {};
+  cfg.blockDim = dim3(GEMM_THREADS, 1, 1);
+  cfg.dynamicSmemBytes = GEMM_SMEM_BYTES;
+  cfg.stream = st;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  if (max_pairs == 0) {
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)GEMM_SMEM_BYTES) !=
         cudaSuccess)
       return SAPO_ERR_CUDA;
-    attr_set = true;
+    const int sms = sm_count();
+    if (sms <= 0) return SAPO_ERR_CUDA;
+    cfg.gridDim = dim3(sms & ~1, 1, 1);
+    int n = 0;
+    if (cudaOccupancyMaxActiveClusters(&n, kern, &cfg) != cudaSuccess || n <= 0) return SAPO_ERR_CUDA;
+    max_pairs = n < sms / 2 ? n : sms / 2;
   }
-  const int sms = sm_count();
-  if (sms <= 0) return SAPO_ERR_CUDA;
-  const int grid = sched.num_units < sms ? sched.num_units : sms;
-  if (grid <= 0) return SAPO_OK;
-  Sched sc = sched;
-  sc.stats_id = kernel_id == SAPO_K_FWD_GEMM ? 0 : kernel_id - SAPO_K_BWD_DZ + 1;
+  const int pairs = sched.num_units < max_pairs ? sched.num_units : max_pairs;
+  cfg.gridDim = dim3(2 * pairs, 1, 1);
   {
     KernelScope scope(kernel_id, st);
-    kern<<<grid, GEMM_THREADS, GEMM_SMEM_BYTES, st>>>(ma, mb, sc, ep, status);
+    if (cudaLaunchKernelEx(&cfg, kern, ma, mb, sc, ep, status) != cudaSuccess) return SAPO_ERR_CUDA;
   }
   return check_launch();
 }
@@ -649,7 +690,7 @@ extern "C" int sapo_policy_loss_fwd(const void* hidden, const void* W_head, int3
     A = a3; B = b3; K = 3 * (int64_t)H; lda = K; ldb = K;
   }
   CUtensorMap map_a, map_b;
-  if (!make_map(&map_a, A, K, T, lda, BM) || !make_map(&map_b, B, K, V, ldb, BN)) return SAPO_ERR_CUDA;
+  if (!make_map(&map_a, A, K, T, lda, BM) || !make_map(&map_b, B, K, V, ldb, BN / 2)) return SAPO_ERR_CUDA;
   const Sched sched = make_sched(T, V, K, L.n_splits, /*m_fastest=*/true);
   FwdEpi::Params ep{ids, pm, ps, pz, T, V};
   int rc = launch_gemm<0, false, FwdEpi>(map_a, map_b, sched, ep, status, st, SAPO_K_FWD_GEMM);
@@ -766,7 +807,7 @@ extern "C" int sapo_policy_loss_bwd(const void* hidden, const void* W_head, int3
 
   // W as the K-major B operand of the logit recompute and as the MN-major B operand of dH
   CUtensorMap map_w_kmajor, map_w_mn;
-  if (!make_map(&map_w_kmajor, B, H, V, ldb, BN) || !make_map(&map_w_mn, B, H, V, ldb, 64))
+  if (!make_map(&map_w_kmajor, B, H, V, ldb, BN / 2) || !make_map(&map_w_mn, B, H, V, ldb, 64))
     return SAPO_ERR_CUDA;
 
   for (int64_t t0 = 0; t0 < T; t0 += chunk_rows) {
