@@ -24,13 +24,14 @@ using namespace umma;
 constexpr int BM = 128;            // accumulator rows per CTA (TMEM lanes)
 constexpr int PAIR_M = 256;        // rows of a tile: two CTAs of a cluster share it
 constexpr int BN = 256;            // accumulator columns per tile (at most)
-constexpr int BK = 64;             // bf16 elements per 128-byte operand row
+constexpr int BK = 128;            // K depth of a pipeline stage: two 64-element (128-byte) row segments
 constexpr int UMMA_K = 16;
-constexpr int STAGES = 6;
+constexpr int STAGES = 3;
 constexpr int GEMM_THREADS = 192;  // warp 0: TMA, warp 1: MMA, warps 2-5: epilogue
-constexpr uint32_t A_STAGE_BYTES = BM * 128;         // this CTA's 128 rows of A
-constexpr uint32_t B_STAGE_BYTES = (BN / 2) * 128;   // this CTA's half of the tile's B columns
-constexpr uint32_t CHUNK_BYTES = 64 * 128;   // one 64-row box of an MN-major operand
+constexpr uint32_t A_STAGE_BYTES = BM * BK * 2;         // this CTA's 128 rows of A
+constexpr uint32_t B_STAGE_BYTES = (BN / 2) * BK * 2;   // this CTA's half of the tile's B columns
+constexpr uint32_t BOX_BYTES = 128 * 128;    // one 128-row box: half the K depth of a K-major operand,
+                                             // or 64 columns x full K depth of an MN-major one
 constexpr uint32_t TMEM_COLS = 512;          // two accumulators of 256 columns
 constexpr size_t GEMM_SMEM_BYTES = 1024 + STAGES * (A_STAGE_BYTES + B_STAGE_BYTES) + 256;
 constexpr float LOG2E = 1.4426950408889634f;
@@ -198,11 +199,13 @@ __device__ unsigned long long g_wait_stats[4][8];
 
 // ---------------------------------------------------------------------------- the GEMM kernel
 // D[m, n] = sum_k A[m, k] * B[n, k], one 256 x tile_n tile per CTA pair and step.
-//   A_KIND 0: A is stored [M, K] with K contiguous; map box {64 k, 128 m}
-//   A_KIND 1: A is stored [K, M] with M contiguous; map box {64 m, 64 k}, two boxes per stage
-//   A_KIND 2: A is the tiled dz panel read K-major  (M = tokens, K = vocab): one 128-row box
-//   A_KIND 3: A is the tiled dz panel read MN-major (M = vocab, K = tokens): two 64-row boxes
-//   B_MN false: B is stored [N, K]; map box {64 k, 128 n}.  true: [K, N]; boxes {64 n, 64 k}.
+// A stage holds a K depth of 128.  All boxes are 64 elements (128 bytes) wide.
+//   A_KIND 0: A is stored [M, K] with K contiguous; two boxes {64 k, 128 m} per stage
+//   A_KIND 1: A is stored [K, M] with M contiguous; two boxes {64 m, 128 k} per stage
+//   A_KIND 2: A is the tiled dz panel read K-major  (M = tokens, K = vocab): one 256-row box
+//             (two consecutive vocab tiles of the CTA's token block)
+//   A_KIND 3: A is the tiled dz panel read MN-major (M = vocab, K = tokens): two whole tiles
+//   B_MN false: B is stored [N, K]; two boxes {64 k, 128 n}.  true: [K, N]; boxes {64 n, 128 k}.
 // CTA `rank` of the pair owns rows [256 mb + 128 rank, +128) of the tile and stages columns
 // [n0 + rank * n_eff / 2, + n_eff / 2) of B.  All TMA completions of a stage are counted on the
 // even CTA's barrier; the even CTA's MMA thread frees stages and publishes accumulators on
@@ -242,6 +245,11 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
   cluster_sync_all();
   fence_after_sync();
   const uint32_t tmem_base = *tmem_slot;
+  // cluster addresses of barriers the other CTA signals or that live in the even CTA
+  const uint32_t full0_addr = map_to_cta(smem_u32(full), 0);
+  const uint32_t empty_addr[2] = {map_to_cta(smem_u32(empty), 0), map_to_cta(smem_u32(empty), 1)};
+  const uint32_t acc_full_addr[2] = {map_to_cta(smem_u32(acc_full), 0), map_to_cta(smem_u32(acc_full), 1)};
+  const uint32_t acc_empty0_addr = map_to_cta(smem_u32(acc_empty), 0);
 
   if (warp == 0) {
     // ------------------------------------------------------------ TMA producer (both CTAs)
@@ -251,36 +259,37 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
     int stage = 0; uint32_t phase = 0;
     uint32_t in_flight = 0;   // bit i: stage i was filled in the current ring pass
     bool ok = true;
-    constexpr int A_BOXES = A_MN ? 2 : 1;
+    constexpr int A_BOXES = A_KIND == 2 ? 1 : 2;
     for (int unit = pair; ok && unit < sched.num_units; unit += num_pairs) {
       int pmb, un, n_begin, n_end;
       decode_unit(sched, unit, pmb, un, n_begin, n_end);
       const int mb = 2 * pmb + (int)rank;                 // this CTA's 128-row block
       for (int nb = n_begin; ok && nb < n_end; ++nb) {
         const int half = tile_n_eff(sched, nb) >> 1;       // B columns this CTA stages
-        const int b_boxes = B_MN ? ((half + 63) >> 6) : 1;
-        const uint32_t tx = 2 * (A_STAGE_BYTES + (B_MN ? b_boxes * CHUNK_BYTES : B_STAGE_BYTES));
+        const int b_boxes = B_MN ? ((half + 63) >> 6) : 2;
+        const uint32_t tx = 2 * (A_STAGE_BYTES + b_boxes * BOX_BYTES);
         const bool mine = lane < A_BOXES + b_boxes;
         const bool is_a = lane < A_BOXES;
         const int bi = is_a ? lane : lane - A_BOXES;
         const CUtensorMap* map = is_a ? &map_a : &map_b;
-        const uint32_t dst_off = is_a ? bi * CHUNK_BYTES : STAGES * A_STAGE_BYTES + bi * CHUNK_BYTES;
+        const uint32_t dst_off = is_a ? bi * BOX_BYTES : STAGES * A_STAGE_BYTES + bi * BOX_BYTES;
         const bool mn = is_a ? A_MN : B_MN;
-        const int row0 = is_a ? mb * BM + 64 * bi
-                              : nb * sched.tile_n + (int)rank * half + 64 * bi;   // m or n coordinate
+        // m or n coordinate of the box (an MN-major box covers 64 of them, a K-major one 128)
+        const int row0 = is_a ? mb * BM + (mn ? 64 * bi : 0)
+                              : nb * sched.tile_n + (int)rank * half + (mn ? 64 * bi : 0);
+        const int k_off = mn ? 0 : 64 * bi;                // K-major boxes split the stage's K depth
         for (int kb = 0; kb < sched.num_k_blocks; ++kb) {
-          if (!SAPO_TIMED(0, mbar_wait_cluster(&empty[stage], phase ^ 1, abort_flag))) { ok = false; break; }
+          if (!SAPO_TIMED(0, mbar_wait(&empty[stage], phase ^ 1, abort_flag))) { ok = false; break; }
           if (rank == 0 && lane == 0) mbar_arrive_expect_tx(&full[stage], tx);
           if (mine) {
             uint8_t* dst = smem + dst_off + stage * (is_a ? A_STAGE_BYTES : B_STAGE_BYTES);
-            const uint32_t bar = map_to_cta(smem_u32(&full[stage]), 0);
-            if (is_a && A_KIND == 2)        // tile (token block mb, vocab tile kb), all 128 rows
-              tma_load_2d_pair(dst, map, bar, 0, (mb * sched.panel_nvt + kb) * BM);
-            else if (is_a && A_KIND == 3)   // tile (token block kb/2, vocab tile 2 mb + bi), one half
-              tma_load_2d_pair(dst, map, bar, 0,
-                               ((kb >> 1) * sched.panel_nvt + 2 * mb + bi) * BM + (kb & 1) * 64);
+            const uint32_t bar = full0_addr + stage * 8;
+            if (is_a && A_KIND == 2)        // vocab tiles 2 kb and 2 kb + 1 of token block mb: 256 rows
+              tma_load_2d_pair(dst, map, bar, 0, (mb * sched.panel_nvt + 2 * kb) * BM);
+            else if (is_a && A_KIND == 3)   // token block kb, vocab tile 2 mb + bi: all 128 rows
+              tma_load_2d_pair(dst, map, bar, 0, (kb * sched.panel_nvt + 2 * mb + bi) * BM);
             else if (mn) tma_load_2d_pair(dst, map, bar, row0, kb * BK);
-            else         tma_load_2d_pair(dst, map, bar, kb * BK, row0);
+            else         tma_load_2d_pair(dst, map, bar, kb * BK + k_off, row0);
           }
           in_flight |= 1u << stage;
           if (++stage == STAGES) { stage = 0; phase ^= 1; }
@@ -293,7 +302,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
       for (int i = 0; i < STAGES; ++i) {
         if (!(in_flight & (1u << i))) continue;
         const uint32_t ph = (i < stage) ? phase : (phase ^ 1);
-        for (int spin = 0; spin < (1 << 20) && !mbar_try_wait_cluster(&full[i], ph); ++spin) {}
+        for (int spin = 0; spin < (1 << 20) && !mbar_try_wait(&full[i], ph); ++spin) {}
       }
     }
   } else if (warp == 1 && lane == 0 && rank == 0) {
@@ -307,33 +316,39 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
       decode_unit(sched, unit, pmb, un, n_begin, n_end);
       for (int nb = n_begin; ok && nb < n_end; ++nb) {
         const uint32_t idesc = make_idesc_bf16(PAIR_M, tile_n_eff(sched, nb), A_MN, B_MN);
-        if (!SAPO_TIMED(2, mbar_wait_cluster(&acc_empty[acc], acc_phase ^ 1, abort_flag))) { ok = false; break; }
+        if (!SAPO_TIMED(2, mbar_wait(&acc_empty[acc], acc_phase ^ 1, abort_flag))) { ok = false; break; }
         fence_after_sync();
         const uint32_t d_tmem = tmem_base + acc * BN;
         for (int kb = 0; kb < sched.num_k_blocks; ++kb) {
-          if (!SAPO_TIMED(1, mbar_wait_cluster(&full[stage], phase, abort_flag))) { ok = false; break; }
+          if (!SAPO_TIMED(1, mbar_wait(&full[stage], phase, abort_flag))) { ok = false; break; }
           fence_after_sync();
+#ifdef SAPO_WAIT_STATS
+          const long long issue_t0 = clock64();
+#endif
           const uint32_t a_addr = smem_u32(smem_a + stage * A_STAGE_BYTES);
           const uint32_t b_addr = smem_u32(smem_b + stage * B_STAGE_BYTES);
           #pragma unroll
           for (int k = 0; k < BK / UMMA_K; ++k) {
-            // K-major: 16 elements = 32 bytes along the row; MN-major: 16 rows = 2048 bytes
-            const uint64_t a_desc = A_MN ? make_smem_desc(a_addr + k * 2048, CHUNK_BYTES, 1024)
-                                         : make_smem_desc(a_addr + k * 32, 16, 1024);
-            const uint64_t b_desc = B_MN ? make_smem_desc(b_addr + k * 2048, CHUNK_BYTES, 1024)
-                                         : make_smem_desc(b_addr + k * 32, 16, 1024);
+            // K-major: 16 elements = 32 bytes along the row, the second half of the depth in
+            // the next box; MN-major: 16 rows = 2048 bytes, 64-column chunks one box apart
+            const uint32_t k_major_off = (k >> 2) * BOX_BYTES + (k & 3) * 32;
+            const uint64_t a_desc = A_MN ? make_smem_desc(a_addr + k * 2048, BOX_BYTES, 1024)
+                                         : make_smem_desc(a_addr + k_major_off, 16, 1024);
+            const uint64_t b_desc = B_MN ? make_smem_desc(b_addr + k * 2048, BOX_BYTES, 1024)
+                                         : make_smem_desc(b_addr + k_major_off, 16, 1024);
             mma_bf16_pair(d_tmem, a_desc, b_desc, idesc, (kb | k) != 0 ? 1u : 0u);
           }
           // free the stage in both CTAs once these MMAs retire
-          const uint32_t e = smem_u32(&empty[stage]);
-          mma_commit_pair(map_to_cta(e, 0));
-          mma_commit_pair(map_to_cta(e, 1));
+          mma_commit_pair(empty_addr[0] + stage * 8);
+          mma_commit_pair(empty_addr[1] + stage * 8);
+#ifdef SAPO_WAIT_STATS
+          wait_cycles[7] += clock64() - issue_t0;
+#endif
           if (++stage == STAGES) { stage = 0; phase ^= 1; }
         }
         if (ok) {                                  // accumulator complete, in both CTAs
-          const uint32_t f = smem_u32(&acc_full[acc]);
-          mma_commit_pair(map_to_cta(f, 0));
-          mma_commit_pair(map_to_cta(f, 1));
+          mma_commit_pair(acc_full_addr[0] + acc * 8);
+          mma_commit_pair(acc_full_addr[1] + acc * 8);
         }
         if (++acc == 2) { acc = 0; acc_phase ^= 1; }
       }
@@ -352,20 +367,26 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
       decode_unit(sched, unit, pmb, un, n_begin, n_end);
       epi.begin_unit(ep, 2 * pmb + (int)rank, r);
       for (int nb = n_begin; ok && nb < n_end; ++nb) {
-        if (!SAPO_TIMED(3, mbar_wait_cluster(&acc_full[acc], acc_phase, abort_flag))) { ok = false; break; }
+        if (!SAPO_TIMED(3, mbar_wait(&acc_full[acc], acc_phase, abort_flag))) { ok = false; break; }
         fence_after_sync();
         const uint32_t t_addr = tmem_base + (static_cast<uint32_t>(quad * 32) << 16) + acc * BN;
         const int n0 = nb * sched.tile_n;
-        const int n_visit = min(sched.tile_n, sched.n_cover - n0);
+        // the last tile also visits the padding columns up to n_cover (they hold no accumulator)
+        const int n_visit = nb == sched.num_n_blocks - 1 ? sched.n_cover - n0 : sched.tile_n;
         for (int c = 0; c * 32 < n_visit; ++c) {
           float v[32];
-          tmem_ld32(t_addr + c * 32, v);
-          tmem_ld_wait();
+          if (c * 32 < sched.tile_n) {
+            tmem_ld32(t_addr + c * 32, v);
+            tmem_ld_wait();
+          } else {
+            #pragma unroll
+            for (int j = 0; j < 32; ++j) v[j] = 0.f;
+          }
           epi.chunk(ep, v, n0 + c * 32);
         }
         fence_before_sync();
         __syncwarp();
-        if (lane == 0) mbar_arrive_cluster(map_to_cta(smem_u32(&acc_empty[acc]), 0));
+        if (lane == 0) mbar_arrive_cluster(acc_empty0_addr + acc * 8);
         if (++acc == 2) { acc = 0; acc_phase ^= 1; }
       }
       if (ok) epi.end_unit(ep, un);
@@ -588,7 +609,7 @@ static int launch_split(const float* X, int64_t ld, int64_t R, int32_t H, __nv_b
 static bool shapes_ok(int64_t T, int32_t H, int32_t V) {
   return T >= 1 && T <= 0x7fffff00LL && H >= 8 && (H % 8) == 0 && H <= 65536 && V >= 1 && V <= 0x7fffff00;
 }
-static int64_t padded_vocab(int32_t V) { return round_up<int64_t>(V, 64); }
+static int64_t padded_vocab(int32_t V) { return round_up<int64_t>(V, 128); }
 
 struct FwdLayout { size_t partials, a_split, b_split, total; int n_splits; };
 static FwdLayout fwd_layout(int64_t T, int32_t H, int32_t V, int32_t dtype, int sms) {
@@ -690,7 +711,7 @@ extern "C" int sapo_policy_loss_fwd(const void* hidden, const void* W_head, int3
     A = a3; B = b3; K = 3 * (int64_t)H; lda = K; ldb = K;
   }
   CUtensorMap map_a, map_b;
-  if (!make_map(&map_a, A, K, T, lda, BM) || !make_map(&map_b, B, K, V, ldb, BN / 2)) return SAPO_ERR_CUDA;
+  if (!make_map(&map_a, A, K, T, lda, BM) || !make_map(&map_b, B, K, V, ldb, 128)) return SAPO_ERR_CUDA;
   const Sched sched = make_sched(T, V, K, L.n_splits, /*m_fastest=*/true);
   FwdEpi::Params ep{ids, pm, ps, pz, T, V};
   int rc = launch_gemm<0, false, FwdEpi>(map_a, map_b, sched, ep, status, st, SAPO_K_FWD_GEMM);
@@ -807,17 +828,17 @@ extern "C" int sapo_policy_loss_bwd(const void* hidden, const void* W_head, int3
 
   // W as the K-major B operand of the logit recompute and as the MN-major B operand of dH
   CUtensorMap map_w_kmajor, map_w_mn;
-  if (!make_map(&map_w_kmajor, B, H, V, ldb, BN / 2) || !make_map(&map_w_mn, B, H, V, ldb, 64))
+  if (!make_map(&map_w_kmajor, B, H, V, ldb, 128) || !make_map(&map_w_mn, B, H, V, ldb, 128))
     return SAPO_ERR_CUDA;
 
   for (int64_t t0 = 0; t0 < T; t0 += chunk_rows) {
     const int64_t tc = (T - t0) < chunk_rows ? (T - t0) : chunk_rows;
     const __nv_bfloat16* A0 = A + t0 * lda;
     const int64_t panel_rows = ceil_div<int64_t>(tc, BM) * nvt * BM;   // 128-byte rows of the tiled panel
-    CUtensorMap map_h_kmajor, map_h_mn, map_p_tile, map_p_half;
-    if (!make_map(&map_h_kmajor, A0, H, tc, lda, BM) || !make_map(&map_h_mn, A0, H, tc, lda, 64) ||
-        !make_map(&map_p_tile, panel, 64, panel_rows, 64, BM) ||
-        !make_map(&map_p_half, panel, 64, panel_rows, 64, 64))
+    CUtensorMap map_h_kmajor, map_h_mn, map_p_two, map_p_tile;
+    if (!make_map(&map_h_kmajor, A0, H, tc, lda, BM) || !make_map(&map_h_mn, A0, H, tc, lda, 128) ||
+        !make_map(&map_p_two, panel, 64, panel_rows, 64, 256) ||
+        !make_map(&map_p_tile, panel, 64, panel_rows, 64, BM))
       return SAPO_ERR_CUDA;
     // dz panel: recompute logits tile by tile
     {
@@ -832,7 +853,7 @@ extern "C" int sapo_policy_loss_bwd(const void* hidden, const void* W_head, int3
       Sched sched = make_sched(tc, H, Vp, 0, /*m_fastest=*/false);
       sched.panel_nvt = nvt;
       StoreEpi::Params ep{dhidden + t0 * (int64_t)H, H, tc, H, 0};
-      int rc = launch_gemm<2, true, StoreEpi>(map_p_tile, map_w_mn, sched, ep, status, st, SAPO_K_BWD_DH);
+      int rc = launch_gemm<2, true, StoreEpi>(map_p_two, map_w_mn, sched, ep, status, st, SAPO_K_BWD_DH);
       if (rc != SAPO_OK) return rc;
     }
     // dW (+)= dz^T . hidden               (M = V, N = H, K = tokens)
@@ -840,7 +861,7 @@ extern "C" int sapo_policy_loss_bwd(const void* hidden, const void* W_head, int3
       Sched sched = make_sched(V, H, tc, 0, /*m_fastest=*/false);
       sched.panel_nvt = nvt;
       StoreEpi::Params ep{dW_head, H, V, H, (t0 > 0 || accumulate_dW) ? 1 : 0};
-      int rc = launch_gemm<3, true, StoreEpi>(map_p_half, map_h_mn, sched, ep, status, st, SAPO_K_BWD_DW);
+      int rc = launch_gemm<3, true, StoreEpi>(map_p_tile, map_h_mn, sched, ep, status, st, SAPO_K_BWD_DW);
       if (rc != SAPO_OK) return rc;
     }
   }
