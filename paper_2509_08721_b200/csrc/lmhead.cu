@@ -27,7 +27,7 @@ constexpr int BN = 256;            // accumulator columns per tile (at most)
 constexpr int BK = 128;            // K depth of a pipeline stage: two 64-element (128-byte) row segments
 constexpr int UMMA_K = 16;
 constexpr int STAGES = 3;
-constexpr int GEMM_THREADS = 192;  // warp 0: TMA, warp 1: MMA, warps 2-5: epilogue
+constexpr int GEMM_THREADS = 320;  // warp 0: TMA, warp 1: MMA, warps 2-9: epilogue
 constexpr uint32_t A_STAGE_BYTES = BM * BK * 2;         // this CTA's 128 rows of A
 constexpr uint32_t B_STAGE_BYTES = (BN / 2) * BK * 2;   // this CTA's half of the tile's B columns
 constexpr uint32_t BOX_BYTES = 128 * 128;    // one 128-row box: half the K depth of a K-major operand,
@@ -99,9 +99,10 @@ struct FwdEpi {
     for (int j = 0; j < 32; ++j) acc += ex2(fmaf(v[j], LOG2E, -m_new));
     s = acc; m = m_new;
   }
-  __device__ __forceinline__ void end_unit(const Params& p, int un) {
+  // two threads share a row (one per column half of the tiles): each leaves its own partial
+  __device__ __forceinline__ void end_unit(const Params& p, int un, int col_half) {
     if (row < p.T) {
-      const int64_t o = (int64_t)un * p.T + row;
+      const int64_t o = (int64_t)(2 * un + col_half) * p.T + row;
       p.pm[o] = m; p.ps[o] = s; p.pz[o] = zy;
     }
   }
@@ -137,11 +138,15 @@ struct DzEpi {
     } else {
       const float ng = -g;
       #pragma unroll
-      for (int j = 0; j < 32; ++j) {
-        float d = ng * ex2(fmaf(v[j], LOG2E, -l2));
-        if (col0 + j == y) d += g;
-        if (col0 + j >= p.V) d = 0.f;
-        v[j] = d;
+      for (int j = 0; j < 32; ++j) v[j] = ng * ex2(fmaf(v[j], LOG2E, -l2));
+      const int yr = y - col0;
+      if (yr >= 0 && yr < 32) {            // the chunk that holds the chosen token
+        #pragma unroll
+        for (int j = 0; j < 32; ++j) if (j == yr) v[j] += g;
+      }
+      if (col0 + 32 > p.V) {               // ragged end of the vocabulary
+        #pragma unroll
+        for (int j = 0; j < 32; ++j) if (col0 + j >= p.V) v[j] = 0.f;
       }
       #pragma unroll
       for (int j = 0; j < 16; ++j) {
@@ -156,7 +161,7 @@ struct DzEpi {
     for (int q = 0; q < 4; ++q)
       dst[q] = make_uint4(packed[4 * q], packed[4 * q + 1], packed[4 * q + 2], packed[4 * q + 3]);
   }
-  __device__ __forceinline__ void end_unit(const Params&, int) {}
+  __device__ __forceinline__ void end_unit(const Params&, int, int) {}
 };
 
 // Plain fp32 output tile, optionally added to what is already there.
@@ -179,7 +184,7 @@ struct StoreEpi {
       }
     }
   }
-  __device__ __forceinline__ void end_unit(const Params&, int) {}
+  __device__ __forceinline__ void end_unit(const Params&, int, int) {}
 };
 
 // Optional instrumentation (compile with -DSAPO_WAIT_STATS): cycles each role spends waiting.
@@ -233,7 +238,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
 
   if (threadIdx.x == 0) {
     for (int i = 0; i < STAGES; ++i) { mbar_init(&full[i], 1); mbar_init(&empty[i], 1); }
-    for (int i = 0; i < 2; ++i) { mbar_init(&acc_full[i], 1); mbar_init(&acc_empty[i], 8); }
+    for (int i = 0; i < 2; ++i) { mbar_init(&acc_full[i], 1); mbar_init(&acc_empty[i], 16); }
     *abort_flag = 0;
     fence_mbar_init();
     prefetch_tensormap(&map_a);
@@ -355,8 +360,11 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
     }
     SAPO_STATS_FLUSH(5);
   } else if (warp >= 2) {
-    // ------------------------------------------------------------ epilogue (128 threads, both CTAs)
-    const int quad = warp & 3;                    // TMEM lane quadrant this warp may read
+    // ------------------------------------------------------------ epilogue (8 warps, both CTAs)
+    // Warps 2-5 drain the first four 32-column chunks of a tile, warps 6-9 the rest; a warp
+    // may only read the TMEM lane quadrant warp_id % 4, so each quadrant has one warp of each set.
+    const int quad = warp & 3;
+    const int col_half = (warp - 2) >> 2;
     const int r = quad * 32 + lane;
     SAPO_STATS_DECL
     int acc = 0; uint32_t acc_phase = 0;
@@ -373,23 +381,37 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
         const int n0 = nb * sched.tile_n;
         // the last tile also visits the padding columns up to n_cover (they hold no accumulator)
         const int n_visit = nb == sched.num_n_blocks - 1 ? sched.n_cover - n0 : sched.tile_n;
-        for (int c = 0; c * 32 < n_visit; ++c) {
-          float v[32];
-          if (c * 32 < sched.tile_n) {
-            tmem_ld32(t_addr + c * 32, v);
-            tmem_ld_wait();
-          } else {
+        const int chunks = (n_visit + 31) >> 5;
+        const int c_begin = col_half ? 4 : 0;
+        const int c_end = col_half ? chunks : min(chunks, 4);
+        const int c_tmem = (sched.tile_n + 31) >> 5;      // chunks that exist in tensor memory
+        // two buffers: the load of the next chunk is in flight while this one is processed
+        float va[32], vb[32];
+        if (c_begin < c_end && c_begin < c_tmem) tmem_ld32(t_addr + c_begin * 32, va);
+        for (int c = c_begin; c < c_end; c += 2) {
+          tmem_ld_wait();
+          if (c + 1 < c_end && c + 1 < c_tmem) tmem_ld32(t_addr + (c + 1) * 32, vb);
+          if (c >= c_tmem) {
             #pragma unroll
-            for (int j = 0; j < 32; ++j) v[j] = 0.f;
+            for (int j = 0; j < 32; ++j) va[j] = 0.f;
           }
-          epi.chunk(ep, v, n0 + c * 32);
+          epi.chunk(ep, va, n0 + c * 32);
+          if (c + 1 < c_end) {
+            tmem_ld_wait();
+            if (c + 2 < c_end && c + 2 < c_tmem) tmem_ld32(t_addr + (c + 2) * 32, va);
+            if (c + 1 >= c_tmem) {
+              #pragma unroll
+              for (int j = 0; j < 32; ++j) vb[j] = 0.f;
+            }
+            epi.chunk(ep, vb, n0 + (c + 1) * 32);
+          }
         }
         fence_before_sync();
         __syncwarp();
         if (lane == 0) mbar_arrive_cluster(acc_empty0_addr + acc * 8);
         if (++acc == 2) { acc = 0; acc_phase ^= 1; }
       }
-      if (ok) epi.end_unit(ep, un);
+      if (ok) epi.end_unit(ep, un, col_half);
     }
     if (threadIdx.x == 64) SAPO_STATS_FLUSH(6);
   }
@@ -616,7 +638,7 @@ static FwdLayout fwd_layout(int64_t T, int32_t H, int32_t V, int32_t dtype, int 
   FwdLayout L{};
   L.n_splits = fwd_splits(T, V, sms);
   size_t off = 0;
-  L.partials = off; off += round_up<size_t>((size_t)3 * L.n_splits * T * sizeof(float), 256);
+  L.partials = off; off += round_up<size_t>((size_t)3 * 2 * L.n_splits * T * sizeof(float), 256);
   if (dtype == SAPO_DTYPE_F32) {
     L.a_split = off; off += round_up<size_t>((size_t)T * 3 * H * 2, 256);
     L.b_split = off; off += round_up<size_t>((size_t)V * 3 * H * 2, 256);
@@ -695,8 +717,8 @@ extern "C" int sapo_policy_loss_fwd(const void* hidden, const void* W_head, int3
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   uint8_t* ws = static_cast<uint8_t*>(workspace);
   float* pm = reinterpret_cast<float*>(ws + L.partials);
-  float* ps = pm + (size_t)L.n_splits * T;
-  float* pz = ps + (size_t)L.n_splits * T;
+  float* ps = pm + (size_t)2 * L.n_splits * T;
+  float* pz = ps + (size_t)2 * L.n_splits * T;
   float* seq_out = seq_surr ? seq_surr : reinterpret_cast<float*>(ws + L.total);
 
   const void* A = hidden; const void* B = W_head;
@@ -718,7 +740,8 @@ extern "C" int sapo_policy_loss_fwd(const void* hidden, const void* W_head, int3
   if (rc != SAPO_OK) return rc;
 
   TailArgs ta{};
-  ta.pm = pm; ta.ps = ps; ta.pz = pz; ta.n_splits = sched.units_per_m; ta.T = T;
+  ta.pm = pm; ta.ps = ps; ta.pz = pz; ta.T = T;
+  ta.n_splits = 2 * sched.units_per_m;   // one partial per vocab split and column half
   ta.ids = ids; ta.V = V; ta.old_logp = old_logp; ta.adv = adv; ta.cu = cu_seqlens; ta.S = S;
   ta.lo_edge = 1.f - h_cfg->eps_low; ta.hi_edge = 1.f + h_cfg->eps_high; ta.grad_scale = h_cfg->grad_scale;
   ta.logp = logp; ta.lse = lse; ta.ratio = ratio; ta.surr = surr; ta.gscale = gscale; ta.seq_surr = seq_out;
