@@ -33,6 +33,7 @@ constexpr uint32_t B_STAGE_BYTES = (BN / 2) * BK * 2;   // this CTA's half of th
 constexpr uint32_t BOX_BYTES = 128 * 128;    // one 128-row box: half the K depth of a K-major operand,
                                              // or 64 columns x full K depth of an MN-major one
 constexpr uint32_t TMEM_COLS = 512;          // two accumulators of 256 columns
+constexpr uint32_t STAGING_BYTES = 2 * 128 * 128;   // dz epilogue: one 16 KB panel tile per column half
 constexpr size_t GEMM_SMEM_BYTES = 1024 + STAGES * (A_STAGE_BYTES + B_STAGE_BYTES) + 256;
 constexpr float LOG2E = 1.4426950408889634f;
 constexpr float LN2 = 0.6931471805599453f;
@@ -67,8 +68,17 @@ __device__ __forceinline__ int tile_n_eff(const Sched& s, int nb) {
 // ---------------------------------------------------------------------------- epilogues
 // Each epilogue thread owns one accumulator row (TMEM lane) of the tile.
 
+// What a staged epilogue needs to move finished 64-column groups through shared memory.
+struct StageCtx {
+  uint32_t buf;          // shared address of this column half's 16 KB staging tile
+  int bar_id;            // named barrier of the four warps that share it
+  bool elected;          // the one thread that issues and tracks the TMA stores
+  const CUtensorMap* map;
+};
+
 // Forward: online log-sum-exp in the base-2 domain plus the logit of the chosen token.
 struct FwdEpi {
+  static constexpr bool STAGED = false;
   struct Params {
     const int32_t* ids; float* pm; float* ps; float* pz;  // partials [n_splits][T]
     int64_t T; int32_t V;
@@ -79,7 +89,7 @@ struct FwdEpi {
     m = -INFINITY; s = 0.f; zy = 0.f;
     y = row < p.T ? p.ids[row] : -1;
   }
-  __device__ __forceinline__ void chunk(const Params& p, float (&v)[32], int col0) {
+  __device__ __forceinline__ void chunk(const Params& p, float (&v)[32], int col0, const StageCtx&) {
     if (col0 >= p.V) return;
     if (col0 + 32 > p.V) {
       #pragma unroll
@@ -111,25 +121,33 @@ struct FwdEpi {
 // Backward, first contraction: dz[t,v] = g_t ([v == y_t] - exp(z[t,v] - lse_t)), to bf16.
 // The panel is a sequence of [128 token x 64 vocab] tiles of 16 KB, tile (tb, vt) at index
 // tb * nvt + vt, each tile row-major: both later contractions then fetch whole contiguous
-// tiles (dH) or half tiles (dW) with one TMA box.  Rows past the last token and columns past
-// V are written as zeros, because those consumers cannot tell them from data.
+// tiles with one TMA box.  Rows past the last token and columns past V are written as zeros,
+// because those consumers cannot tell them from data.  A finished 64-column group is staged in
+// shared memory (128-byte swizzle) and leaves as one 16 KB TMA store.
 struct DzEpi {
+  static constexpr bool STAGED = true;
   struct Params {
-    const int32_t* ids; const float* lse; const float* gscale; __nv_bfloat16* P;
+    const int32_t* ids; const float* lse; const float* gscale;
     int64_t M; int32_t V; int32_t nvt;
   };
-  float g, l2; int32_t y; int64_t tile_row0; int r; bool in_panel;
+  float g, l2; int32_t y; int32_t tile_row0; int r; bool in_panel;
   __device__ __forceinline__ void begin_unit(const Params& p, int mb, int r_) {
     const int64_t row = (int64_t)mb * BM + r_;
     const bool valid = row < p.M;
     in_panel = (int64_t)mb * BM < p.M;   // the odd CTA of the last pair may own no token block
     r = r_;
-    tile_row0 = (int64_t)mb * p.nvt * BM;          // first panel row of this token block
+    tile_row0 = mb * p.nvt * BM;          // first panel row of this token block
     g = valid ? p.gscale[row] : 0.f;
     l2 = valid ? p.lse[row] * LOG2E : 0.f;
     y = valid ? p.ids[row] : -1;
   }
-  __device__ __forceinline__ void chunk(const Params& p, float (&v)[32], int col0) {
+  // before the first chunk of a 64-column group: the previous store must have left the buffer
+  __device__ __forceinline__ void group_begin(const StageCtx& cx) {
+    if (!in_panel) return;
+    if (cx.elected) bulk_wait_read_all();
+    named_barrier_sync(cx.bar_id, 128);
+  }
+  __device__ __forceinline__ void chunk(const Params& p, float (&v)[32], int col0, const StageCtx& cx) {
     if (!in_panel) return;
     uint32_t packed[16];
     if (g == 0.f) {
@@ -154,25 +172,36 @@ struct DzEpi {
         packed[j] = *reinterpret_cast<uint32_t*>(&h);
       }
     }
-    const int vt = col0 >> 6;
-    __nv_bfloat16* at = p.P + ((tile_row0 + (int64_t)vt * BM + r) << 6) + (col0 & 32);
-    uint4* dst = reinterpret_cast<uint4*>(at);
+    // row r of the tile, 16-byte pieces q..q+3, stored where the 128-byte swizzle puts them
+    const int q0 = (col0 & 32) >> 3;   // 32 columns = four 16-byte pieces
     #pragma unroll
     for (int q = 0; q < 4; ++q)
-      dst[q] = make_uint4(packed[4 * q], packed[4 * q + 1], packed[4 * q + 2], packed[4 * q + 3]);
+      st_shared_v4(cx.buf + r * 128 + (((q0 + q) ^ (r & 7)) << 4),
+                   packed[4 * q], packed[4 * q + 1], packed[4 * q + 2], packed[4 * q + 3]);
+  }
+  // after the last chunk of the group: hand the tile to the TMA
+  __device__ __forceinline__ void group_end(const Params& p, int col0_of_group, const StageCtx& cx) {
+    if (!in_panel) return;
+    fence_proxy_async_smem();
+    named_barrier_sync(cx.bar_id, 128);
+    if (cx.elected) {
+      tma_store_2d(cx.map, cx.buf, 0, tile_row0 + (col0_of_group >> 6) * BM);
+      bulk_commit_group();
+    }
   }
   __device__ __forceinline__ void end_unit(const Params&, int, int) {}
 };
 
 // Plain fp32 output tile, optionally added to what is already there.
 struct StoreEpi {
+  static constexpr bool STAGED = false;
   struct Params { float* C; int64_t ldc; int64_t M; int32_t N; int32_t accumulate; };
   int64_t row; bool valid;
   __device__ __forceinline__ void begin_unit(const Params& p, int mb, int r) {
     row = (int64_t)mb * BM + r;
     valid = row < p.M;
   }
-  __device__ __forceinline__ void chunk(const Params& p, float (&v)[32], int col0) {
+  __device__ __forceinline__ void chunk(const Params& p, float (&v)[32], int col0, const StageCtx&) {
     if (!valid) return;
     float4* dst = reinterpret_cast<float4*>(p.C + row * p.ldc + col0);
     #pragma unroll
@@ -218,12 +247,14 @@ __device__ unsigned long long g_wait_stats[4][8];
 template <int A_KIND, bool B_MN, class Epi>
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
 umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+                 const __grid_constant__ CUtensorMap map_c,   // output tiles of a staged epilogue
                  const Sched sched, const typename Epi::Params ep, int32_t* status) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint8_t* smem_a = smem;
   uint8_t* smem_b = smem + STAGES * A_STAGE_BYTES;
-  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + STAGES * (A_STAGE_BYTES + B_STAGE_BYTES));
+  uint8_t* staging = smem + STAGES * (A_STAGE_BYTES + B_STAGE_BYTES);   // STAGED epilogues only
+  uint64_t* bars = reinterpret_cast<uint64_t*>(staging + (Epi::STAGED ? STAGING_BYTES : 0));
   uint64_t* full = bars;                 // [STAGES] TMA -> MMA          (even CTA's are used)
   uint64_t* empty = bars + STAGES;       // [STAGES] MMA -> TMA          (each CTA waits on its own)
   uint64_t* acc_full = bars + 2 * STAGES;      // [2] MMA -> epilogue    (each CTA waits on its own)
@@ -370,6 +401,11 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
     int acc = 0; uint32_t acc_phase = 0;
     bool ok = true;
     Epi epi;
+    StageCtx cx;
+    cx.buf = smem_u32(staging) + col_half * (STAGING_BYTES / 2);
+    cx.bar_id = 1 + col_half;
+    cx.elected = quad == 0 && lane == 0;
+    cx.map = &map_c;
     for (int unit = pair; ok && unit < sched.num_units; unit += num_pairs) {
       int pmb, un, n_begin, n_end;
       decode_unit(sched, unit, pmb, un, n_begin, n_end);
@@ -388,14 +424,15 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
         // two buffers: the load of the next chunk is in flight while this one is processed
         float va[32], vb[32];
         if (c_begin < c_end && c_begin < c_tmem) tmem_ld32(t_addr + c_begin * 32, va);
-        for (int c = c_begin; c < c_end; c += 2) {
+        for (int c = c_begin; c < c_end; c += 2) {      // one 64-column group per turn
           tmem_ld_wait();
           if (c + 1 < c_end && c + 1 < c_tmem) tmem_ld32(t_addr + (c + 1) * 32, vb);
           if (c >= c_tmem) {
             #pragma unroll
             for (int j = 0; j < 32; ++j) va[j] = 0.f;
           }
-          epi.chunk(ep, va, n0 + c * 32);
+          if constexpr (Epi::STAGED) epi.group_begin(cx);
+          epi.chunk(ep, va, n0 + c * 32, cx);
           if (c + 1 < c_end) {
             tmem_ld_wait();
             if (c + 2 < c_end && c + 2 < c_tmem) tmem_ld32(t_addr + (c + 2) * 32, va);
@@ -403,8 +440,9 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
               #pragma unroll
               for (int j = 0; j < 32; ++j) vb[j] = 0.f;
             }
-            epi.chunk(ep, vb, n0 + (c + 1) * 32);
+            epi.chunk(ep, vb, n0 + (c + 1) * 32, cx);
           }
+          if constexpr (Epi::STAGED) epi.group_end(ep, n0 + c * 32, cx);
         }
         fence_before_sync();
         __syncwarp();
@@ -413,6 +451,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
       }
       if (ok) epi.end_unit(ep, un, col_half);
     }
+    if (Epi::STAGED && cx.elected) bulk_wait_all();   // stores done before shared memory goes away
     if (threadIdx.x == 64) SAPO_STATS_FLUSH(6);
   }
 
@@ -544,11 +583,11 @@ static bool make_map(CUtensorMap* map, const void* base, int64_t inner, int64_t 
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-static Sched make_sched(int64_t M, int64_t N, int64_t K, int n_splits, bool m_fastest) {
+static Sched make_sched(int64_t M, int64_t N, int64_t K, int n_splits, bool m_fastest, int tile_align = 32) {
   Sched s{};
   s.num_m_blocks = (int32_t)ceil_div<int64_t>(M, PAIR_M);
   const int64_t tiles = ceil_div<int64_t>(N, BN);
-  s.tile_n = (int32_t)round_up<int64_t>(ceil_div<int64_t>(N, tiles), 32);   // equal-width tiles
+  s.tile_n = (int32_t)round_up<int64_t>(ceil_div<int64_t>(N, tiles), tile_align);   // equal-width tiles
   s.num_n_blocks = (int32_t)ceil_div<int64_t>(N, s.tile_n);
   s.n_per_unit = n_splits > 0 ? ceil_div(s.num_n_blocks, n_splits) : 1;
   s.units_per_m = ceil_div(s.num_n_blocks, s.n_per_unit);
@@ -580,7 +619,7 @@ static int fwd_splits(int64_t T, int32_t V, int sms) {
 }
 
 template <int A_KIND, bool B_MN, class Epi>
-static int launch_gemm(const CUtensorMap& ma, const CUtensorMap& mb, const Sched& sched,
+static int launch_gemm(const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& mc, const Sched& sched,
                        const typename Epi::Params& ep, int32_t* status, cudaStream_t st, int kernel_id) {
   auto kern = umma_gemm_kernel<A_KIND, B_MN, Epi>;
   static int max_pairs = 0;     // CTA pairs the device can hold at once, found on first use
@@ -592,12 +631,13 @@ static int launch_gemm(const CUtensorMap& ma, const CUtensorMap& mb, const Sched
   attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
   cudaLaunchConfig_t cfg = {};
   cfg.blockDim = dim3(GEMM_THREADS, 1, 1);
-  cfg.dynamicSmemBytes = GEMM_SMEM_BYTES;
+  constexpr size_t smem_bytes = GEMM_SMEM_BYTES + (Epi::STAGED ? STAGING_BYTES : 0);
+  cfg.dynamicSmemBytes = smem_bytes;
   cfg.stream = st;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
   if (max_pairs == 0) {
-    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)GEMM_SMEM_BYTES) !=
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes) !=
         cudaSuccess)
       return SAPO_ERR_CUDA;
     const int sms = sm_count();
@@ -611,7 +651,7 @@ static int launch_gemm(const CUtensorMap& ma, const CUtensorMap& mb, const Sched
   cfg.gridDim = dim3(2 * pairs, 1, 1);
   {
     KernelScope scope(kernel_id, st);
-    if (cudaLaunchKernelEx(&cfg, kern, ma, mb, sc, ep, status) != cudaSuccess) return SAPO_ERR_CUDA;
+    if (cudaLaunchKernelEx(&cfg, kern, ma, mb, mc, sc, ep, status) != cudaSuccess) return SAPO_ERR_CUDA;
   }
   return check_launch();
 }
@@ -736,7 +776,7 @@ extern "C" int sapo_policy_loss_fwd(const void* hidden, const void* W_head, int3
   if (!make_map(&map_a, A, K, T, lda, BM) || !make_map(&map_b, B, K, V, ldb, 128)) return SAPO_ERR_CUDA;
   const Sched sched = make_sched(T, V, K, L.n_splits, /*m_fastest=*/true);
   FwdEpi::Params ep{ids, pm, ps, pz, T, V};
-  int rc = launch_gemm<0, false, FwdEpi>(map_a, map_b, sched, ep, status, st, SAPO_K_FWD_GEMM);
+  int rc = launch_gemm<0, false, FwdEpi>(map_a, map_b, map_a, sched, ep, status, st, SAPO_K_FWD_GEMM);
   if (rc != SAPO_OK) return rc;
 
   TailArgs ta{};
@@ -865,10 +905,10 @@ extern "C" int sapo_policy_loss_bwd(const void* hidden, const void* W_head, int3
       return SAPO_ERR_CUDA;
     // dz panel: recompute logits tile by tile
     {
-      Sched sched = make_sched(tc, V, H, 0, /*m_fastest=*/true);
+      Sched sched = make_sched(tc, V, H, 0, /*m_fastest=*/true, /*tile_align=*/64);
       sched.n_cover = (int32_t)Vp;
-      DzEpi::Params ep{ids + t0, lse + t0, gscale + t0, panel, tc, V, nvt};
-      int rc = launch_gemm<0, false, DzEpi>(map_h_kmajor, map_w_kmajor, sched, ep, status, st, SAPO_K_BWD_DZ);
+      DzEpi::Params ep{ids + t0, lse + t0, gscale + t0, tc, V, nvt};
+      int rc = launch_gemm<0, false, DzEpi>(map_h_kmajor, map_w_kmajor, map_p_tile, sched, ep, status, st, SAPO_K_BWD_DZ);
       if (rc != SAPO_OK) return rc;
     }
     // dhidden[t0:t0+tc] = dz . W         (M = tokens, N = H, K = V)
@@ -876,7 +916,7 @@ extern "C" int sapo_policy_loss_bwd(const void* hidden, const void* W_head, int3
       Sched sched = make_sched(tc, H, Vp, 0, /*m_fastest=*/false);
       sched.panel_nvt = nvt;
       StoreEpi::Params ep{dhidden + t0 * (int64_t)H, H, tc, H, 0};
-      int rc = launch_gemm<2, true, StoreEpi>(map_p_two, map_w_mn, sched, ep, status, st, SAPO_K_BWD_DH);
+      int rc = launch_gemm<2, true, StoreEpi>(map_p_two, map_w_mn, map_p_two, sched, ep, status, st, SAPO_K_BWD_DH);
       if (rc != SAPO_OK) return rc;
     }
     // dW (+)= dz^T . hidden               (M = V, N = H, K = tokens)
@@ -884,7 +924,7 @@ extern "C" int sapo_policy_loss_bwd(const void* hidden, const void* W_head, int3
       Sched sched = make_sched(V, H, tc, 0, /*m_fastest=*/false);
       sched.panel_nvt = nvt;
       StoreEpi::Params ep{dW_head, H, V, H, (t0 > 0 || accumulate_dW) ? 1 : 0};
-      int rc = launch_gemm<3, true, StoreEpi>(map_p_tile, map_h_mn, sched, ep, status, st, SAPO_K_BWD_DW);
+      int rc = launch_gemm<3, true, StoreEpi>(map_p_tile, map_h_mn, map_p_tile, sched, ep, status, st, SAPO_K_BWD_DW);
       if (rc != SAPO_OK) return rc;
     }
   }
