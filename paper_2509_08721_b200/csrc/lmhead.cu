@@ -89,6 +89,7 @@ struct FwdEpi {
     m = -INFINITY; s = 0.f; zy = 0.f;
     y = row < p.T ? p.ids[row] : -1;
   }
+  template <int HALF>
   __device__ __forceinline__ void chunk(const Params& p, float (&v)[32], int col0, const StageCtx&) {
     if (col0 >= p.V) return;
     if (col0 + 32 > p.V) {
@@ -141,15 +142,13 @@ struct DzEpi {
     l2 = valid ? p.lse[row] * LOG2E : 0.f;
     y = valid ? p.ids[row] : -1;
   }
-  // before the first chunk of a 64-column group: the previous store must have left the buffer
-  __device__ __forceinline__ void group_begin(const StageCtx& cx) {
+  __device__ __forceinline__ void group_begin(const StageCtx&) {}
+  // dz of 32 columns, kept in registers as 16 bf16 pairs until the whole 64-column group is done
+  uint32_t pk[2][16];
+  template <int HALF>   // which 32-column half of the group (a compile-time register choice)
+  __device__ __forceinline__ void chunk(const Params& p, float (&v)[32], int col0, const StageCtx&) {
     if (!in_panel) return;
-    if (cx.elected) bulk_wait_read_all();
-    named_barrier_sync(cx.bar_id, 128);
-  }
-  __device__ __forceinline__ void chunk(const Params& p, float (&v)[32], int col0, const StageCtx& cx) {
-    if (!in_panel) return;
-    uint32_t packed[16];
+    uint32_t (&packed)[16] = pk[HALF];
     if (g == 0.f) {
       #pragma unroll
       for (int j = 0; j < 16; ++j) packed[j] = 0u;
@@ -172,16 +171,18 @@ struct DzEpi {
         packed[j] = *reinterpret_cast<uint32_t*>(&h);
       }
     }
-    // row r of the tile, 16-byte pieces q..q+3, stored where the 128-byte swizzle puts them
-    const int q0 = (col0 & 32) >> 3;   // 32 columns = four 16-byte pieces
-    #pragma unroll
-    for (int q = 0; q < 4; ++q)
-      st_shared_v4(cx.buf + r * 128 + (((q0 + q) ^ (r & 7)) << 4),
-                   packed[4 * q], packed[4 * q + 1], packed[4 * q + 2], packed[4 * q + 3]);
   }
-  // after the last chunk of the group: hand the tile to the TMA
+  // after both chunks of the group: wait until the previous TMA store has read the staging
+  // tile, write this row (128 bytes, in 128-byte-swizzle order) and hand the tile to the TMA
   __device__ __forceinline__ void group_end(const Params& p, int col0_of_group, const StageCtx& cx) {
     if (!in_panel) return;
+    if (cx.elected) bulk_wait_read_all();
+    named_barrier_sync(cx.bar_id, 128);
+    #pragma unroll
+    for (int q = 0; q < 8; ++q)
+      st_shared_v4(cx.buf + r * 128 + ((q ^ (r & 7)) << 4),
+                   pk[q >> 2][4 * (q & 3)], pk[q >> 2][4 * (q & 3) + 1],
+                   pk[q >> 2][4 * (q & 3) + 2], pk[q >> 2][4 * (q & 3) + 3]);
     fence_proxy_async_smem();
     named_barrier_sync(cx.bar_id, 128);
     if (cx.elected) {
@@ -201,6 +202,7 @@ struct StoreEpi {
     row = (int64_t)mb * BM + r;
     valid = row < p.M;
   }
+  template <int HALF>
   __device__ __forceinline__ void chunk(const Params& p, float (&v)[32], int col0, const StageCtx&) {
     if (!valid) return;
     float4* dst = reinterpret_cast<float4*>(p.C + row * p.ldc + col0);
@@ -432,7 +434,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
             for (int j = 0; j < 32; ++j) va[j] = 0.f;
           }
           if constexpr (Epi::STAGED) epi.group_begin(cx);
-          epi.chunk(ep, va, n0 + c * 32, cx);
+          epi.template chunk<0>(ep, va, n0 + c * 32, cx);
           if (c + 1 < c_end) {
             tmem_ld_wait();
             if (c + 2 < c_end && c + 2 < c_tmem) tmem_ld32(t_addr + (c + 2) * 32, va);
@@ -440,7 +442,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
               #pragma unroll
               for (int j = 0; j < 32; ++j) vb[j] = 0.f;
             }
-            epi.chunk(ep, vb, n0 + (c + 1) * 32, cx);
+            epi.template chunk<1>(ep, vb, n0 + (c + 1) * 32, cx);
           }
           if constexpr (Epi::STAGED) epi.group_end(ep, n0 + c * 32, cx);
         }
