@@ -231,3 +231,17 @@ def policy_loss_fwd_bwd_rows(hidden, W, ids, old_logp, adv, cu_seqlens, eps_low=
             dW += dz.T @ np.asarray(hidden[a:b], dtype=np.float64)
     out["dhidden"], out["dW"] = dH, dW
     return out
+
+
+def dW_rows(hidden, W, ids, lse, gscale, rows) -> np.ndarray:
+    """The rows `rows` of dW only: dW[v,:] = sum_t dz[t,v] hidden[t,:] with
+    dz[t,v] = g_t ([v == ids_t] - exp(z[t,v] - lse_t)), z restricted to those vocab rows.
+    Same definition as policy_loss_bwd; used where the full [tokens x vocab] matrix is too
+    large for the host.  lse must cover every token (it depends on the whole vocabulary)."""
+    rows = np.asarray(rows, dtype=np.int64)
+    h = np.asarray(hidden, dtype=np.float64)
+    z = h @ np.asarray(W, dtype=np.float64)[rows].T                     # [T, len(rows)]
+    dz = -np.exp(z - np.asarray(lse, dtype=np.float64)[:, None])
+    dz += (np.asarray(ids, dtype=np.int64)[:, None] == rows[None, :])
+    dz *= np.asarray(gscale, dtype=np.float64)[:, None]
+    return dz.T @ h

@@ -293,6 +293,16 @@ def test_row_blocked_evaluation_equals_the_whole_matrix_form():
     assert np.allclose(r["dW"], g["dW"], rtol=1e-12, atol=1e-16)
 
 
+def test_dW_rows_equals_the_rows_of_the_full_gradient():
+    rng, cu, h, W, ids, adv = _toy(8, T_s=(4, 6, 2, 5))
+    cur = orc.token_logprobs(h, W, ids)["logp"]
+    f = orc.policy_loss_fwd(h, W, ids, cur + rng.normal(size=len(cur)) * 0.1, adv, cu)
+    g = orc.policy_loss_bwd(h, W, ids, f["lse"], f["gscale"])
+    rows = [0, 3, int(ids[0]), 16]
+    assert np.allclose(orc.dW_rows(h, W, ids, f["lse"], f["gscale"], rows), g["dW"][rows],
+                       rtol=1e-12, atol=1e-16)
+
+
 # ------------------------------------------------------------------ the input generator
 def test_generator_recipes_have_the_stated_shapes():
     r = gen.config(1)
