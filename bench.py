@@ -253,6 +253,15 @@ def run_ours(args):
         # launches per step of that kernel (the backward runs once per dz panel chunk)
         per_step = n_top / args.steps
         achieved = flops_each / per_step / (ms_top / 1e3) / 1e12
+        # DRAM bytes per launch from the ncu capture of a small case of the same kernels
+        # (profiles/umma_gemm_kernels_workload2_lengths_div4.md): fixed part + bytes per token.
+        # Only valid for hidden 896 / vocab 151936, the shape that capture ran at.
+        ncu_traffic = {"fwd_gemm": (0.272e9, 13.1e3), "bwd_dz": (0.272e9, 299.6e3),
+                       "bwd_dh": (0.272e9, 311.8e3), "bwd_dw": (0.519e9, 335.9e3)}
+        traffic = None
+        if (H, V) == (896, 151936):
+            fixed, per_token = ncu_traffic[top]
+            traffic = fixed + per_token * T / per_step
         peak = peaks["bf16_tflops_sustained"]      # the kernel is timed inside a long step
         burst = peaks["bf16_tflops"]
         kernels = {k: {"ms_per_step": v["ms"] / args.steps, "launches_per_step": v["launches"] / args.steps}
@@ -274,7 +283,7 @@ def run_ours(args):
             "frac_of_bf16_burst_peak_executed": f_exec / (ms_step / 1e3) / 1e12 / burst,
             "frac_of_bf16_sustained_peak_algorithmic": f_alg / (ms_step / 1e3) / 1e12 / peak,
             "roofline": {"bound": "tensor", "kernel": top, "achieved": achieved, "peak": peak,
-                         "unit": "TFLOP/s", "frac": achieved / peak, "traffic": None,
+                         "unit": "TFLOP/s", "frac": achieved / peak, "traffic": traffic,
                          "peak_source": peaks["source"] + " (sustained bf16 GEMM; burst is %.1f)" % burst,
                          "flops_per_launch": flops_each / per_step, "ms_per_launch": ms_top,
                          "all_gemm_kernels_ms_per_step": gemm_ms},

@@ -179,8 +179,9 @@ int sapo_policy_loss_fwd(const void* hidden, const void* W_head, int32_t dtype,
  *   dhidden[t,:] = sum_v dz[t,v] W_head[v,:]        float32 [T, H]
  *   dW_head[v,:] = sum_t dz[t,v] hidden[t,:]        float32 [V, H]
  * Logit tiles are recomputed on the tensor cores; dz is rounded to bf16 and kept in a
- * bounded panel inside `workspace` (token chunks x padded vocab), from which two tensor-core
- * contractions form dhidden and dW_head.  accumulate_dW != 0 adds into dW_head instead of
+ * bounded panel inside `workspace` (token chunks x vocab padded to 128, stored as 16 KB tiles
+ * of 128 tokens x 64 vocab entries), from which two tensor-core contractions form dhidden and
+ * dW_head.  accumulate_dW != 0 adds into dW_head instead of
  * overwriting it.  lse and gscale come from sapo_policy_loss_fwd.  For SAPO_DTYPE_F32 the
  * operands are rounded to bf16.
  * workspace: sapo_workspace_bytes(SAPO_WS_BWD, ...) is the preferred size; any size down to
@@ -209,7 +210,7 @@ size_t sapo_workspace_bytes_min(int32_t which, int64_t T, int32_t H, int32_t V, 
  * Limits: bf16 operands only (SAPO_ERR_UNSUPPORTED_SHAPE otherwise), and the forward scratch for
  * these sizes — sapo_workspace_bytes(SAPO_WS_FWD, ...), plus 4*S bytes when seq_surr is NULL —
  * must fit; if not, the call does nothing and returns SAPO_ERR_STATIC_SCRATCH_EXCEEDED.  With one
- * vocab split (at least as many 128-token blocks as SMs) that is about 340,000 tokens.
+ * vocab split (at least as many 256-token blocks as SM pairs) that is about 170,000 tokens.
  * The first call on each device looks up the array's device address (that device must be
  * current); make that first call outside any stream capture.  All calls on a device share the
  * one array and it keeps whatever the previous call left: nothing in it needs clearing between
