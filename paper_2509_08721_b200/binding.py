@@ -67,7 +67,7 @@ def load() -> C.CDLL:
     global _lib
     if _lib is not None:
         return _lib
-    path = _build.LIB
+    path = os.environ.get("SAPO_B200_LIB") or _build.LIB      # override: a differently built copy
     if not os.path.exists(path):
         path = _build.build()
     lib = C.CDLL(path)
