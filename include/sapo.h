@@ -240,7 +240,8 @@ int sapo_policy_loss_fwd_static(const void* hidden, const void* W_head, int32_t 
 #define SAPO_K_BWD_DZ     7
 #define SAPO_K_BWD_DH     8
 #define SAPO_K_BWD_DW     9
-#define SAPO_K_COUNT      10
+#define SAPO_K_STREAMK_FIXUP 10
+#define SAPO_K_COUNT      11
 int sapo_timing_enable(int32_t on);
 int sapo_timing_read(float* h_ms, int32_t* h_launches);
 int64_t sapo_launch_count(void);

@@ -30,7 +30,7 @@ EXPORTS = ("sapo_pack_rollouts", "sapo_group_advantages", "sapo_policy_loss_fwd"
            "sapo_policy_loss_fwd_static")
 STATIC_SCRATCH_BYTES = 4 * 1024 * 1024
 KERNEL_NAMES = ("pack_scan", "pack_copy", "group_adv", "split_bf16", "fwd_gemm", "loss_tail",
-                "loss_final", "bwd_dz", "bwd_dh", "bwd_dw")
+                "loss_final", "bwd_dz", "bwd_dh", "bwd_dw", "streamk_fixup")
 
 
 class RolloutBufC(C.Structure):

@@ -47,8 +47,17 @@ struct Sched {
   int32_t tile_n;     // columns per tile (a multiple of 32, at most 256)
   int32_t n_cover;    // columns the epilogue visits (>= N; the dz panel is padded to 64)
   int32_t panel_nvt;  // 64-column tiles per token block of the dz panel (tiled A operands)
+  // Units [0, dp_units) are dealt whole, round-robin, to the pairs.  The sk_tiles units after
+  // them (fewer than there are pairs) are cut along K instead: their sk_tiles * num_k_blocks
+  // stage iterations are shared out evenly, sk_ipp consecutive ones per pair, so the last wave
+  // is as full as the others.  A pair that gets only part of a tile's K range leaves a partial
+  // accumulator in scratch; a small second kernel adds the parts up.
+  int32_t dp_units, sk_tiles, sk_ipp;
   int32_t stats_id;   // row of the wait-cycle counters this launch adds to (instrumented builds)
 };
+
+constexpr int PARTIAL_FLOATS = PAIR_M * BN;   // one partial accumulator tile: 256 x 256 fp32
+constexpr int MAX_PAIRS_SCRATCH = 96;          // CTA pairs the K-split scratch is sized for (a B200 has 74)
 
 __device__ __forceinline__ void decode_unit(const Sched& s, int unit, int& mb, int& un,
                                             int& n_begin, int& n_end) {
@@ -57,6 +66,41 @@ __device__ __forceinline__ void decode_unit(const Sched& s, int unit, int& mb, i
   n_begin = un * s.n_per_unit;
   n_end = min(n_begin + s.n_per_unit, s.num_n_blocks);
 }
+
+// The work of one CTA pair, in order: its whole units, then its share of the K-split units.
+// Every role of both CTAs walks the same list.
+struct WorkList {
+  const Sched& s; int pair, n_pairs, i; long long it, it_end;
+  __device__ __forceinline__ WorkList(const Sched& s_, int pair_, int n_pairs_)
+      : s(s_), pair(pair_), n_pairs(n_pairs_), i(0) {
+    const long long total = (long long)s.sk_tiles * s.num_k_blocks;
+    it = (long long)pair * s.sk_ipp;
+    it_end = it + s.sk_ipp < total ? it + s.sk_ipp : total;
+    if (it > it_end) it = it_end;
+  }
+  // slot: -1 = the tile's whole K range (normal epilogue); otherwise the scratch slot of the part
+  __device__ __forceinline__ bool next(int& pmb, int& un, int& n_begin, int& n_end, int& kb0, int& kb1,
+                                       int& slot) {
+    const int unit = pair + i * n_pairs;
+    if (unit < s.dp_units) {
+      ++i;
+      decode_unit(s, unit, pmb, un, n_begin, n_end);
+      kb0 = 0; kb1 = s.num_k_blocks; slot = -1;
+      return true;
+    }
+    if (it < it_end) {
+      const int t = (int)(it / s.num_k_blocks);
+      decode_unit(s, s.dp_units + t, pmb, un, n_begin, n_end);
+      kb0 = (int)(it - (long long)t * s.num_k_blocks);
+      const long long left = it_end - it;
+      kb1 = (long long)(s.num_k_blocks - kb0) <= left ? s.num_k_blocks : kb0 + (int)left;
+      it += kb1 - kb0;
+      slot = (kb0 == 0 && kb1 == s.num_k_blocks) ? -1 : 2 * pair + (kb0 == 0 ? 1 : 0);
+      return true;
+    }
+    return false;
+  }
+};
 
 // columns of a tile the MMA computes: the tile width, or on the last tile what is left,
 // rounded up to 32 so that each CTA's half stays a multiple of 16
@@ -79,6 +123,8 @@ struct StageCtx {
 // Forward: online log-sum-exp in the base-2 domain plus the logit of the chosen token.
 struct FwdEpi {
   static constexpr bool STAGED = false;
+  static constexpr bool STREAMK = false;
+
   struct Params {
     const int32_t* ids; float* pm; float* ps; float* pz;  // partials [n_splits][T]
     int64_t T; int32_t V;
@@ -127,6 +173,7 @@ struct FwdEpi {
 // shared memory (128-byte swizzle) and leaves as one 16 KB TMA store.
 struct DzEpi {
   static constexpr bool STAGED = true;
+  static constexpr bool STREAMK = false;
   struct Params {
     const int32_t* ids; const float* lse; const float* gscale;
     int64_t M; int32_t V; int32_t nvt;
@@ -196,14 +243,28 @@ struct DzEpi {
 // Plain fp32 output tile, optionally added to what is already there.
 struct StoreEpi {
   static constexpr bool STAGED = false;
-  struct Params { float* C; int64_t ldc; int64_t M; int32_t N; int32_t accumulate; };
-  int64_t row; bool valid;
+  static constexpr bool STREAMK = true;
+  struct Params { float* C; int64_t ldc; int64_t M; int32_t N; int32_t accumulate; float* partials; };
+  int64_t row; bool valid; float* part; int n0;
   __device__ __forceinline__ void begin_unit(const Params& p, int mb, int r) {
     row = (int64_t)mb * BM + r;
     valid = row < p.M;
+    part = nullptr;
+  }
+  // a K-split part of a tile goes to scratch slot `slot` instead: rows [128 rank, +128) of a
+  // 256 x 256 fp32 tile, column 0 = the tile's first column
+  __device__ __forceinline__ void set_dest(const Params& p, int slot, int rank, int r, int n0_) {
+    n0 = n0_;
+    part = slot < 0 ? nullptr : p.partials + (size_t)slot * PARTIAL_FLOATS + (size_t)(rank * BM + r) * BN;
   }
   template <int HALF>
   __device__ __forceinline__ void chunk(const Params& p, float (&v)[32], int col0, const StageCtx&) {
+    if (part != nullptr) {
+      float4* dst = reinterpret_cast<float4*>(part + (col0 - n0));
+      #pragma unroll
+      for (int q = 0; q < 8; ++q) dst[q] = make_float4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
+      return;
+    }
     if (!valid) return;
     float4* dst = reinterpret_cast<float4*>(p.C + row * p.ldc + col0);
     #pragma unroll
@@ -217,6 +278,32 @@ struct StoreEpi {
   }
   __device__ __forceinline__ void end_unit(const Params&, int, int) {}
 };
+
+// Adds up the K-split parts of each tile the GEMM kernel left in scratch and stores the sum.
+// Part order is fixed (by pair index), so the result does not depend on timing.
+__global__ void __launch_bounds__(256)
+streamk_fixup_kernel(const Sched s, const StoreEpi::Params p) {
+  const int t = blockIdx.x >> 5;                 // K-split tile
+  const int row_begin = (blockIdx.x & 31) * 8;   // 8 of its 256 rows per block
+  const long long first_it = (long long)t * s.num_k_blocks;
+  const int p_first = (int)(first_it / s.sk_ipp);
+  const int p_last = (int)((first_it + s.num_k_blocks - 1) / s.sk_ipp);
+  if (p_first == p_last) return;                 // one pair had the whole tile and stored it itself
+  int pmb, un, n_begin, n_end;
+  decode_unit(s, s.dp_units + t, pmb, un, n_begin, n_end);
+  const int n0 = n_begin * s.tile_n;
+  const int col = threadIdx.x;
+  if (col >= s.tile_n || n0 + col >= p.N) return;
+  for (int rr = row_begin; rr < row_begin + 8; ++rr) {
+    const int64_t row = (int64_t)pmb * PAIR_M + rr;
+    if (row >= p.M) break;
+    const size_t off = (size_t)rr * BN + col;
+    float sum = p.partials[(size_t)(2 * p_first + 1) * PARTIAL_FLOATS + off];
+    for (int q = p_first + 1; q <= p_last; ++q) sum += p.partials[(size_t)(2 * q) * PARTIAL_FLOATS + off];
+    float* dst = p.C + row * p.ldc + n0 + col;
+    *dst = p.accumulate ? *dst + sum : sum;
+  }
+}
 
 // Optional instrumentation (compile with -DSAPO_WAIT_STATS): cycles each role spends waiting.
 #ifdef SAPO_WAIT_STATS
@@ -298,9 +385,9 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
     uint32_t in_flight = 0;   // bit i: stage i was filled in the current ring pass
     bool ok = true;
     constexpr int A_BOXES = A_KIND == 2 ? 1 : 2;
-    for (int unit = pair; ok && unit < sched.num_units; unit += num_pairs) {
-      int pmb, un, n_begin, n_end;
-      decode_unit(sched, unit, pmb, un, n_begin, n_end);
+    WorkList work(sched, pair, num_pairs);
+    int pmb, un, n_begin, n_end, kb0, kb1, slot;
+    while (ok && work.next(pmb, un, n_begin, n_end, kb0, kb1, slot)) {
       const int mb = 2 * pmb + (int)rank;                 // this CTA's 128-row block
       for (int nb = n_begin; ok && nb < n_end; ++nb) {
         const int half = tile_n_eff(sched, nb) >> 1;       // B columns this CTA stages
@@ -316,7 +403,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
         const int row0 = is_a ? mb * BM + (mn ? 64 * bi : 0)
                               : nb * sched.tile_n + (int)rank * half + (mn ? 64 * bi : 0);
         const int k_off = mn ? 0 : 64 * bi;                // K-major boxes split the stage's K depth
-        for (int kb = 0; kb < sched.num_k_blocks; ++kb) {
+        for (int kb = kb0; kb < kb1; ++kb) {
           if (!SAPO_TIMED(0, mbar_wait(&empty[stage], phase ^ 1, abort_flag))) { ok = false; break; }
           if (rank == 0 && lane == 0) mbar_arrive_expect_tx(&full[stage], tx);
           if (mine) {
@@ -349,20 +436,17 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
     int stage = 0; uint32_t phase = 0;
     int acc = 0; uint32_t acc_phase = 0;
     bool ok = true;
-    for (int unit = pair; ok && unit < sched.num_units; unit += num_pairs) {
-      int pmb, un, n_begin, n_end;
-      decode_unit(sched, unit, pmb, un, n_begin, n_end);
+    WorkList work(sched, pair, num_pairs);
+    int pmb, un, n_begin, n_end, kb0, kb1, slot;
+    while (ok && work.next(pmb, un, n_begin, n_end, kb0, kb1, slot)) {
       for (int nb = n_begin; ok && nb < n_end; ++nb) {
         const uint32_t idesc = make_idesc_bf16(PAIR_M, tile_n_eff(sched, nb), A_MN, B_MN);
         if (!SAPO_TIMED(2, mbar_wait(&acc_empty[acc], acc_phase ^ 1, abort_flag))) { ok = false; break; }
         fence_after_sync();
         const uint32_t d_tmem = tmem_base + acc * BN;
-        for (int kb = 0; kb < sched.num_k_blocks; ++kb) {
+        for (int kb = kb0; kb < kb1; ++kb) {
           if (!SAPO_TIMED(1, mbar_wait(&full[stage], phase, abort_flag))) { ok = false; break; }
           fence_after_sync();
-#ifdef SAPO_WAIT_STATS
-          const long long issue_t0 = clock64();
-#endif
           const uint32_t a_addr = smem_u32(smem_a + stage * A_STAGE_BYTES);
           const uint32_t b_addr = smem_u32(smem_b + stage * B_STAGE_BYTES);
           #pragma unroll
@@ -374,14 +458,11 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
                                          : make_smem_desc(a_addr + k_major_off, 16, 1024);
             const uint64_t b_desc = B_MN ? make_smem_desc(b_addr + k * 2048, BOX_BYTES, 1024)
                                          : make_smem_desc(b_addr + k_major_off, 16, 1024);
-            mma_bf16_pair(d_tmem, a_desc, b_desc, idesc, (kb | k) != 0 ? 1u : 0u);
+            mma_bf16_pair(d_tmem, a_desc, b_desc, idesc, (kb > kb0 || k != 0) ? 1u : 0u);
           }
           // free the stage in both CTAs once these MMAs retire
           mma_commit_pair(empty_addr[0] + stage * 8);
           mma_commit_pair(empty_addr[1] + stage * 8);
-#ifdef SAPO_WAIT_STATS
-          wait_cycles[7] += clock64() - issue_t0;
-#endif
           if (++stage == STAGES) { stage = 0; phase ^= 1; }
         }
         if (ok) {                                  // accumulator complete, in both CTAs
@@ -391,6 +472,9 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
         if (++acc == 2) { acc = 0; acc_phase ^= 1; }
       }
     }
+#ifdef SAPO_WAIT_STATS
+    atomicMax(&g_wait_stats[sched.stats_id & 3][7], (unsigned long long)(clock64() - role_t0));
+#endif
     SAPO_STATS_FLUSH(5);
   } else if (warp >= 2) {
     // ------------------------------------------------------------ epilogue (8 warps, both CTAs)
@@ -408,10 +492,11 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
     cx.bar_id = 1 + col_half;
     cx.elected = quad == 0 && lane == 0;
     cx.map = &map_c;
-    for (int unit = pair; ok && unit < sched.num_units; unit += num_pairs) {
-      int pmb, un, n_begin, n_end;
-      decode_unit(sched, unit, pmb, un, n_begin, n_end);
+    WorkList work(sched, pair, num_pairs);
+    int pmb, un, n_begin, n_end, kb0, kb1, slot;
+    while (ok && work.next(pmb, un, n_begin, n_end, kb0, kb1, slot)) {
       epi.begin_unit(ep, 2 * pmb + (int)rank, r);
+      if constexpr (Epi::STREAMK) epi.set_dest(ep, slot, (int)rank, r, n_begin * sched.tile_n);
       for (int nb = n_begin; ok && nb < n_end; ++nb) {
         if (!SAPO_TIMED(3, mbar_wait(&acc_full[acc], acc_phase, abort_flag))) { ok = false; break; }
         fence_after_sync();
@@ -599,6 +684,7 @@ static Sched make_sched(int64_t M, int64_t N, int64_t K, int n_splits, bool m_fa
   s.N = (int32_t)N;
   s.n_cover = (int32_t)N;
   s.panel_nvt = 0;
+  s.dp_units = s.num_units; s.sk_tiles = 0; s.sk_ipp = 1;
   return s;
 }
 
@@ -648,12 +734,29 @@ static int launch_gemm(const CUtensorMap& ma, const CUtensorMap& mb, const CUten
     int n = 0;
     if (cudaOccupancyMaxActiveClusters(&n, kern, &cfg) != cudaSuccess || n <= 0) return SAPO_ERR_CUDA;
     max_pairs = n < sms / 2 ? n : sms / 2;
+    if (max_pairs > MAX_PAIRS_SCRATCH) max_pairs = MAX_PAIRS_SCRATCH;
   }
-  const int pairs = sched.num_units < max_pairs ? sched.num_units : max_pairs;
+  int pairs = sched.num_units < max_pairs ? sched.num_units : max_pairs;
+  if constexpr (Epi::STREAMK) {
+    // a ragged last wave of long-K tiles is cut along K over all the pairs
+    const int rem = sched.num_units % max_pairs;
+    if (ep.partials != nullptr && rem != 0 && sched.num_k_blocks >= 8 && sched.n_per_unit == 1) {
+      pairs = max_pairs;
+      sc.dp_units = sched.num_units - rem;
+      sc.sk_tiles = rem;
+      sc.sk_ipp = (int32_t)ceil_div<int64_t>((int64_t)rem * sched.num_k_blocks, pairs);
+    }
+  }
   cfg.gridDim = dim3(2 * pairs, 1, 1);
   {
     KernelScope scope(kernel_id, st);
     if (cudaLaunchKernelEx(&cfg, kern, ma, mb, mc, sc, ep, status) != cudaSuccess) return SAPO_ERR_CUDA;
+  }
+  if constexpr (Epi::STREAMK) {
+    if (sc.sk_tiles > 0) {
+      KernelScope scope(SAPO_K_STREAMK_FIXUP, st);
+      streamk_fixup_kernel<<<sc.sk_tiles * 32, 256, 0, st>>>(sc, ep);
+    }
   }
   return check_launch();
 }
@@ -689,7 +792,7 @@ static FwdLayout fwd_layout(int64_t T, int32_t H, int32_t V, int32_t dtype, int 
   return L;
 }
 
-struct BwdLayout { size_t a_hi, b_hi, panel, fixed; size_t bytes_per_row; };
+struct BwdLayout { size_t a_hi, b_hi, partials, panel, fixed; size_t bytes_per_row; };
 static BwdLayout bwd_layout(int64_t T, int32_t H, int32_t V, int32_t dtype) {
   BwdLayout L{};
   size_t off = 0;
@@ -697,6 +800,7 @@ static BwdLayout bwd_layout(int64_t T, int32_t H, int32_t V, int32_t dtype) {
     L.a_hi = off; off += round_up<size_t>((size_t)T * H * 2, 256);
     L.b_hi = off; off += round_up<size_t>((size_t)V * H * 2, 256);
   }
+  L.partials = off; off += (size_t)2 * MAX_PAIRS_SCRATCH * PARTIAL_FLOATS * sizeof(float);
   L.panel = off; L.fixed = off;
   L.bytes_per_row = (size_t)padded_vocab(V) * 2;
   return L;
@@ -886,6 +990,7 @@ extern "C" int sapo_policy_loss_bwd(const void* hidden, const void* W_head, int3
   const int64_t Vp = padded_vocab(V);
   const int32_t nvt = (int32_t)(Vp / 64);
   __nv_bfloat16* panel = reinterpret_cast<__nv_bfloat16*>(ws + L.panel);
+  float* partials = reinterpret_cast<float*>(ws + L.partials);
   // whole 128-token blocks of the panel that fit; a chunk never ends inside a block it cannot hold
   const int64_t rows_fit = ((int64_t)((workspace_bytes - L.fixed) / L.bytes_per_row) / BM) * BM;
   const int64_t chunk_rows = rows_fit >= T ? T : rows_fit;
@@ -917,7 +1022,7 @@ extern "C" int sapo_policy_loss_bwd(const void* hidden, const void* W_head, int3
     {
       Sched sched = make_sched(tc, H, Vp, 0, /*m_fastest=*/false);
       sched.panel_nvt = nvt;
-      StoreEpi::Params ep{dhidden + t0 * (int64_t)H, H, tc, H, 0};
+      StoreEpi::Params ep{dhidden + t0 * (int64_t)H, H, tc, H, 0, partials};
       int rc = launch_gemm<2, true, StoreEpi>(map_p_two, map_w_mn, map_p_two, sched, ep, status, st, SAPO_K_BWD_DH);
       if (rc != SAPO_OK) return rc;
     }
@@ -925,7 +1030,7 @@ extern "C" int sapo_policy_loss_bwd(const void* hidden, const void* W_head, int3
     {
       Sched sched = make_sched(V, H, tc, 0, /*m_fastest=*/false);
       sched.panel_nvt = nvt;
-      StoreEpi::Params ep{dW_head, H, V, H, (t0 > 0 || accumulate_dW) ? 1 : 0};
+      StoreEpi::Params ep{dW_head, H, V, H, (t0 > 0 || accumulate_dW) ? 1 : 0, partials};
       int rc = launch_gemm<3, true, StoreEpi>(map_p_tile, map_h_mn, map_p_tile, sched, ep, status, st, SAPO_K_BWD_DW);
       if (rc != SAPO_OK) return rc;
     }
@@ -936,8 +1041,8 @@ extern "C" int sapo_policy_loss_bwd(const void* hidden, const void* W_head, int3
 #ifdef SAPO_WAIT_STATS
 // Rows: forward, dz, dH, dW.  Columns: [0] TMA waits on free stages, [1] MMA waits on filled
 // stages, [2] MMA waits on a free accumulator, [3] one epilogue thread's waits on a full
-// accumulator, [4..6] total cycles of the TMA / MMA / that epilogue thread; summed over CTAs
-// and launches since the last reset.
+// accumulator, [4..6] total cycles of the TMA / MMA / that epilogue thread, summed over CTAs
+// and launches since the last reset; [7] the longest MMA-thread time of any CTA.
 extern "C" int sapo_debug_wait_stats(unsigned long long* h_out, int32_t reset) {
   if (h_out && cudaMemcpyFromSymbol(h_out, sapo::g_wait_stats, sizeof(unsigned long long) * 32) != cudaSuccess)
     return SAPO_ERR_CUDA;
