@@ -160,6 +160,57 @@ def run_reference(args):
     return 0
 
 
+def hbm_kernels(torch, B, peaks, H=896, n_rollouts=2048, mean_len=288, n_groups=1 << 22):
+    """Achieved HBM GB/s of the pack and advantage kernels on a scaled case (the workload-size
+    launches take tens of microseconds): about 1.3 GB moved by the pack gather, 2^22 questions
+    of 8 completions for the advantages.  Algorithmic bytes: pack 2*T*(2H+8) (hidden row,
+    id and old log-prob, read and written once), advantages 8 bytes per completion."""
+    g = torch.Generator(device="cuda").manual_seed(1)
+    lens = torch.randint(mean_len // 2, mean_len * 3 // 2, (2, n_rollouts), generator=g, device="cuda")
+    bufs = []
+    for side in range(2):
+        off = torch.zeros(n_rollouts + 1, dtype=torch.int64, device="cuda")
+        off[1:] = torch.cumsum(lens[side], 0)
+        nt = int(off[-1].item())
+        bufs.append(B.DeviceRollouts(
+            torch.randn(nt, H, device="cuda", dtype=torch.bfloat16),
+            torch.randint(0, 1000, (nt,), device="cuda", dtype=torch.int32),
+            torch.randn(nt, device="cuda"), off, torch.rand(n_rollouts, device="cuda")))
+    Q, I = n_rollouts // 4, 4                      # every question: 4 local + 4 external picks
+    qo = (torch.arange(Q + 1, device="cuda", dtype=torch.int32) * I)
+    perm = [torch.randperm(n_rollouts, generator=g, device="cuda").to(torch.int32) for _ in range(2)]
+    sel = B.DeviceSelection(qo, perm[0], qo.clone(), perm[1])
+    T = int(lens.sum().item())
+    out = B.alloc_packed(T, 2 * n_rollouts, Q, H, torch.bfloat16)
+    status = B.new_status()
+    rewards = torch.rand(n_groups * 8, device="cuda")
+    go = (torch.arange(n_groups + 1, device="cuda", dtype=torch.int32) * 8)
+    adv = torch.empty_like(rewards)
+
+    def timed(fn, iters=20, warm=3):
+        for _ in range(warm):
+            fn()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for _ in range(iters):
+            fn()
+        b.record()
+        torch.cuda.synchronize()
+        return a.elapsed_time(b) / iters
+
+    ms_pack = timed(lambda: B.sapo_pack_rollouts(bufs[0], bufs[1], sel, out, status))
+    ms_adv = timed(lambda: B.sapo_group_advantages(rewards, go, 1e-6, 0, adv, None, None, status))
+    assert int(status.item()) == 0 and int(out["n_tokens"].item()) == T
+    bytes_pack = 2.0 * T * (2 * H + 8)
+    bytes_adv = 8.0 * rewards.numel() + 4.0 * n_groups
+    peak = peaks["hbm_gbs"]
+    mk = lambda ms, nbytes, what: {"achieved": nbytes / ms / 1e6, "peak": peak, "unit": "GB/s",
+                                   "frac": nbytes / ms / 1e6 / peak, "ms": ms, "bytes": nbytes, "case": what}
+    return {"pack": mk(ms_pack, bytes_pack, f"{T} tokens of {H} bf16 from {2 * n_rollouts} rollouts"),
+            "advantages": mk(ms_adv, bytes_adv, f"{n_groups} questions x 8 completions"),
+            "peak_source": peaks["source"] + " (copy bandwidth)"}
+
+
 def run_ours(args):
     import torch
     import torch.distributed as dist
@@ -293,6 +344,10 @@ def run_ours(args):
             "gpu_launches": int(n_launches),
             "clocks": clocks,
         }
+        if world == 1:
+            del scorer.workspace
+            torch.cuda.empty_cache()
+            line["hbm_kernels"] = hbm_kernels(torch, B, peaks)
         if world == 1 and not args.no_cpu_baseline:
             n_seqs, _ = oracle_sample(batch, args.ref_tokens)
             dt, Ts = time_oracle(batch, n_seqs)

@@ -108,42 +108,63 @@ __global__ void __launch_bounds__(SCAN_THREADS) pack_scan_kernel(PackArgs a) {
   }
 }
 
-// One warp per packed token: locate its sequence, then copy the row.
+// A warp copies runs of TOKENS_PER_WARP consecutive packed tokens: one binary search per run,
+// then it walks the sequence table; rows move as 16-byte vectors, four loads in flight per lane.
+constexpr int TOKENS_PER_WARP = 8;
+
 __global__ void __launch_bounds__(256) pack_copy_kernel(PackArgs a) {
   const int lane = threadIdx.x & 31;
   const int64_t warp0 = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
   const int64_t n_warps = ((int64_t)gridDim.x * blockDim.x) >> 5;
   const int32_t T = *a.n_tokens, S = *a.n_seqs;
   const bool vec = (a.row_bytes & 15) == 0;
-  for (int64_t t = warp0; t < a.max_tokens; t += n_warps) {
-    if (t >= T) { if (lane == 0) a.tok_mask[t] = 0; continue; }
-    // last s with cu[s] <= t  (zero-length sequences share a start; take the one that owns t)
-    int32_t lo = 0, hi = S;                      // cu has S+1 entries; find first s with cu[s+1] > t
-    while (lo < hi) {
-      int32_t mid = (lo + hi) >> 1;
-      if (a.cu[mid + 1] > t) hi = mid; else lo = mid + 1;
+  const int n4 = (int)(a.row_bytes >> 4);
+  for (int64_t t0 = warp0 * TOKENS_PER_WARP; t0 < a.max_tokens; t0 += n_warps * TOKENS_PER_WARP) {
+    int32_t s = 0;
+    if (t0 < T) {
+      // first s with cu[s+1] > t0 (zero-length sequences share a start; take the one that owns t0)
+      int32_t lo = 0, hi = S;
+      while (lo < hi) {
+        int32_t mid = (lo + hi) >> 1;
+        if (a.cu[mid + 1] > t0) hi = mid; else lo = mid + 1;
+      }
+      s = lo;
     }
-    const int32_t s = lo;
-    const int side = a.seq_is_ext[s];
-    const int64_t src = a.off[side][a.seq_src[s]] + (t - a.cu[s]);
-    const uint8_t* from = a.hid[side] + src * a.row_bytes;
-    uint8_t* to = a.o_hid + t * a.row_bytes;
-    if (vec) {
-      const uint4* f4 = reinterpret_cast<const uint4*>(from);
-      uint4* t4 = reinterpret_cast<uint4*>(to);
-      const int n4 = (int)(a.row_bytes >> 4);
-      for (int i = lane; i < n4; i += 32) t4[i] = __ldg(f4 + i);
-    } else {
-      const uint16_t* f2 = reinterpret_cast<const uint16_t*>(from);
-      uint16_t* t2 = reinterpret_cast<uint16_t*>(to);
-      const int n2 = (int)(a.row_bytes >> 1);
-      for (int i = lane; i < n2; i += 32) t2[i] = f2[i];
-    }
-    if (lane == 0) {
-      a.o_ids[t] = a.ids[side][src];
-      a.o_old[t] = a.old[side][src];
-      a.tok_seq[t] = s;
-      a.tok_mask[t] = 1;
+    for (int i = 0; i < TOKENS_PER_WARP; ++i) {
+      const int64_t t = t0 + i;
+      if (t >= a.max_tokens) break;
+      if (t >= T) { if (lane == 0) a.tok_mask[t] = 0; continue; }
+      while (a.cu[s + 1] <= t) ++s;
+      const int side = a.seq_is_ext[s];
+      const int64_t src = a.off[side][a.seq_src[s]] + (t - a.cu[s]);
+      const uint8_t* from = a.hid[side] + src * a.row_bytes;
+      uint8_t* to = a.o_hid + t * a.row_bytes;
+      if (vec) {
+        const uint4* f4 = reinterpret_cast<const uint4*>(from);
+        uint4* t4 = reinterpret_cast<uint4*>(to);
+        for (int j = lane; j < n4; j += 128) {
+          uint4 v0, v1, v2, v3;
+          v0 = __ldg(f4 + j);
+          if (j + 32 < n4) v1 = __ldg(f4 + j + 32);
+          if (j + 64 < n4) v2 = __ldg(f4 + j + 64);
+          if (j + 96 < n4) v3 = __ldg(f4 + j + 96);
+          t4[j] = v0;
+          if (j + 32 < n4) t4[j + 32] = v1;
+          if (j + 64 < n4) t4[j + 64] = v2;
+          if (j + 96 < n4) t4[j + 96] = v3;
+        }
+      } else {
+        const uint16_t* f2 = reinterpret_cast<const uint16_t*>(from);
+        uint16_t* t2 = reinterpret_cast<uint16_t*>(to);
+        const int n2 = (int)(a.row_bytes >> 1);
+        for (int j = lane; j < n2; j += 32) t2[j] = f2[j];
+      }
+      if (lane == 0) {
+        a.o_ids[t] = a.ids[side][src];
+        a.o_old[t] = a.old[side][src];
+        a.tok_seq[t] = s;
+        a.tok_mask[t] = 1;
+      }
     }
   }
 }
@@ -187,7 +208,7 @@ extern "C" int sapo_pack_rollouts(const sapo_rollout_buf* h_local, const sapo_ro
   if (a.max_tokens > 0) {
     const int sms = sm_count();
     if (sms <= 0) return SAPO_ERR_CUDA;
-    const int64_t warps_wanted = a.max_tokens;
+    const int64_t warps_wanted = (a.max_tokens + TOKENS_PER_WARP - 1) / TOKENS_PER_WARP;
     int blocks = (int)((warps_wanted + 7) / 8);
     const int max_blocks = sms * 8;                 // 8 resident blocks of 256 threads per SM
     if (blocks > max_blocks) blocks = max_blocks;

@@ -105,6 +105,27 @@ def test_advantages_match_oracle(ddof):
         assert abs(a[go[g]:go[g + 1]].sum()) < 1e-5
 
 
+def test_advantages_with_many_questions_take_the_thread_per_question_path():
+    """From 4096 questions on, one thread serves a question (float4 where alignment allows)."""
+    rng = np.random.default_rng(6)
+    sizes = rng.integers(0, 21, size=5003)
+    sizes[:64] = 8
+    go = np.concatenate([[0], np.cumsum(sizes)]).astype(np.int32)
+    r = rng.choice([0.0, 0.5, 1.0], size=go[-1]).astype(np.float32)
+    eps = float(np.float32(1e-6))
+    ref = orc.group_advantages(r, go, adv_eps=eps, ddof=0)
+    adv = torch.empty(len(r), dtype=torch.float32, device="cuda")
+    mean = torch.empty(len(sizes), dtype=torch.float32, device="cuda")
+    std = torch.empty(len(sizes), dtype=torch.float32, device="cuda")
+    status = B.new_status()
+    B.sapo_group_advantages(U.to_torch(r), U.to_torch(go), eps, 0, adv, mean, std, status)
+    torch.cuda.synchronize()
+    assert status.item() == 0
+    assert np.allclose(adv.cpu().numpy(), ref["adv"], rtol=2e-7, atol=1e-9)
+    assert np.allclose(mean.cpu().numpy(), ref["mean"], rtol=2e-7, atol=1e-12)
+    assert np.allclose(std.cpu().numpy(), ref["std"], rtol=2e-7, atol=1e-12)
+
+
 def test_advantages_flag_nonfinite_rewards():
     r = torch.tensor([0.0, float("nan"), 1.0, 1.0], device="cuda")
     go = torch.tensor([0, 2, 4], dtype=torch.int32, device="cuda")
