@@ -232,7 +232,8 @@ def run_ours(args):
     batch, recipe = build_batch(args.workload, replicas.rank_seed(args.workload, rank), args.length_div)
     T, S, H, V = batch.T, batch.S, batch.H, batch.V
     W = _to_dev(batch.W, "cuda")
-    scorer = PolicyScorer(W, T, S, recipe.Q, eps_low=batch.eps_low, eps_high=batch.eps_high)
+    scorer = PolicyScorer(W, T, S, recipe.Q, eps_low=batch.eps_low, eps_high=batch.eps_high,
+                          active_backward=args.backward == "active")
 
     # old log-probs = current + noise: "current" is one forward pass of the library itself
     # over the packed tokens (set-up, untimed); the noise comes from the seeded generator.
@@ -296,13 +297,14 @@ def run_ours(args):
 
     if rank == 0:
         # roofline of the dominant kernel (largest share of the timed region)
-        flops_each = 2.0 * T * V * H
+        t_act = int(scorer.n_active.item()) if args.backward == "active" else T
         gemm = {k: per_kernel[k] for k in ("fwd_gemm", "bwd_dz", "bwd_dh", "bwd_dw")}
         top = max(gemm, key=lambda k: gemm[k]["ms"])
         n_top = max(1, gemm[top]["launches"])
         ms_top = gemm[top]["ms"] / n_top
         # launches per step of that kernel (the backward runs once per dz panel chunk)
         per_step = n_top / args.steps
+        flops_each = 2.0 * (T if top == "fwd_gemm" else t_act) * V * H
         achieved = flops_each / per_step / (ms_top / 1e3) / 1e12
         # DRAM bytes per launch from the ncu capture of a small case of the same kernels
         # (profiles/umma_gemm_kernels_workload2_lengths_div4.md): fixed part + bytes per token.
@@ -318,15 +320,16 @@ def run_ours(args):
         kernels = {k: {"ms_per_step": v["ms"] / args.steps, "launches_per_step": v["launches"] / args.steps}
                    for k, v in per_kernel.items() if v["launches"]}
         gemm_ms = sum(gemm[k]["ms"] for k in gemm) / args.steps
-        f_alg = 6.0 * T * V * H
-        f_exec = 8.0 * T * V * H
+        f_alg = 2.0 * T * V * H + 4.0 * t_act * V * H
+        f_exec = 2.0 * T * V * H + 6.0 * t_act * V * H
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
             "config": {"workload": recipe.name, "H": H, "V": V, "questions": recipe.Q,
                        "local_per_question": recipe.I, "external_per_question": recipe.J,
-                       "tokens_per_step": T, "sequences": S, "parallelism": f"replicas x{world}",
+                       "tokens_per_step": T, "sequences": S, "backward": args.backward,
+                       "active_tokens": t_act, "parallelism": f"replicas x{world}",
                        "l2": "inputs larger than L2 (W_head alone is %d MB)" % (V * H * 2 // 2**20)},
             "tflops_algorithmic": f_alg / (ms_step / 1e3) / 1e12,
             "tflops_executed": f_exec / (ms_step / 1e3) / 1e12,
@@ -370,6 +373,8 @@ def main():
     ap.add_argument("--ref-tokens", type=int, default=None,
                     help="tokens of the bounded oracle sample (default 2048 for cpu_baseline, 512 per reference step)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--backward", default="dense", choices=["dense", "active"],
+                    help="active: contract only the tokens whose gradient factor is non-zero")
     ap.add_argument("--length-div", type=int, default=1,
                     help="divide every completion length (a small case of the same kernels for profiling)")
     args = ap.parse_args()

@@ -64,6 +64,7 @@ extern "C" {
 /* `which` of sapo_workspace_bytes */
 #define SAPO_WS_FWD 0
 #define SAPO_WS_BWD 1
+#define SAPO_WS_BWD_ACTIVE 2
 
 /* A rollout store: n_rollouts completions laid end to end (Section 3.1: a node's answers
  * to its questions; Section 3.2: the tuples other nodes broadcast).
@@ -193,6 +194,24 @@ int sapo_policy_loss_bwd(const void* hidden, const void* W_head, int32_t dtype,
                          void* workspace, size_t workspace_bytes,
                          int32_t* status, void* stream);
 
+/* The same gradient, computed over the active tokens only (gscale[t] != 0).  Sequences of a
+ * zero-advantage group — which the paper's experiments drop from the shared pool as
+ * uninformative (Section 5) — and tokens clipped on the binding side have gscale = 0 and add
+ * nothing to either gradient; this call compacts them away first (order kept), gathers the
+ * hidden rows of the rest, runs the three contractions on those rows and writes dhidden rows
+ * back to their token positions (inactive rows are zero).  The active count is read on the
+ * device by the kernels, so the call does not synchronise; if n_active_out (device int32) is not
+ * NULL the count is also copied there.  Results equal sapo_policy_loss_bwd up to fp32 summation
+ * order.  workspace: sapo_workspace_bytes(SAPO_WS_BWD_ACTIVE, ...) (the regular backward's plus
+ * a compacted copy of hidden and four per-token vectors). */
+int sapo_policy_loss_bwd_active(const void* hidden, const void* W_head, int32_t dtype,
+                                int64_t T, int32_t H, int32_t V, int64_t ld_hidden, int64_t ld_W,
+                                const int32_t* ids, const float* lse, const float* gscale,
+                                float* dhidden, float* dW_head, int32_t accumulate_dW,
+                                int32_t* n_active_out,
+                                void* workspace, size_t workspace_bytes,
+                                int32_t* status, void* stream);
+
 /* Bytes of scratch the forward (SAPO_WS_FWD) or backward (SAPO_WS_BWD) call wants for
  * these sizes.  Returns 0 for invalid arguments. */
 size_t sapo_workspace_bytes(int32_t which, int64_t T, int32_t H, int32_t V, int32_t dtype);
@@ -241,7 +260,8 @@ int sapo_policy_loss_fwd_static(const void* hidden, const void* W_head, int32_t 
 #define SAPO_K_BWD_DH     8
 #define SAPO_K_BWD_DW     9
 #define SAPO_K_STREAMK_FIXUP 10
-#define SAPO_K_COUNT      11
+#define SAPO_K_COMPACT   11
+#define SAPO_K_COUNT      12
 int sapo_timing_enable(int32_t on);
 int sapo_timing_read(float* h_ms, int32_t* h_launches);
 int64_t sapo_launch_count(void);

@@ -18,6 +18,7 @@ DTYPE_BF16 = 0
 DTYPE_F32 = 1
 WS_FWD = 0
 WS_BWD = 1
+WS_BWD_ACTIVE = 2
 
 ST_BITS = {
     0x01: "TOKEN_OVERFLOW", 0x02: "SEQ_OVERFLOW", 0x04: "BAD_INDEX", 0x08: "EMPTY_SEQUENCE",
@@ -27,10 +28,10 @@ ST_BITS = {
 EXPORTS = ("sapo_pack_rollouts", "sapo_group_advantages", "sapo_policy_loss_fwd",
            "sapo_policy_loss_bwd", "sapo_workspace_bytes", "sapo_workspace_bytes_min",
            "sapo_status_string", "sapo_timing_enable", "sapo_timing_read", "sapo_launch_count",
-           "sapo_policy_loss_fwd_static")
+           "sapo_policy_loss_fwd_static", "sapo_policy_loss_bwd_active")
 STATIC_SCRATCH_BYTES = 4 * 1024 * 1024
 KERNEL_NAMES = ("pack_scan", "pack_copy", "group_adv", "split_bf16", "fwd_gemm", "loss_tail",
-                "loss_final", "bwd_dz", "bwd_dh", "bwd_dw", "streamk_fixup")
+                "loss_final", "bwd_dz", "bwd_dh", "bwd_dw", "streamk_fixup", "compact")
 
 
 class RolloutBufC(C.Structure):
@@ -87,6 +88,9 @@ def load() -> C.CDLL:
     lib.sapo_policy_loss_bwd.restype = C.c_int
     lib.sapo_policy_loss_bwd.argtypes = [vp, vp, i32, i64, i32, i32, i64, i64, vp, vp, vp, vp, vp,
                                          i32, vp, sz, vp, vp]
+    lib.sapo_policy_loss_bwd_active.restype = C.c_int
+    lib.sapo_policy_loss_bwd_active.argtypes = [vp, vp, i32, i64, i32, i32, i64, i64, vp, vp, vp, vp, vp,
+                                                i32, vp, vp, sz, vp, vp]
     lib.sapo_workspace_bytes.restype = sz
     lib.sapo_workspace_bytes.argtypes = [i32, i64, i32, i32, i32]
     lib.sapo_workspace_bytes_min.restype = sz
@@ -290,3 +294,19 @@ def sapo_policy_loss_bwd(hidden: torch.Tensor, W_head: torch.Tensor, ids: torch.
         _p(ids), _p(lse), _p(gscale), _p(dhidden), _p(dW_head), 1 if accumulate_dW else 0,
         _p(workspace), workspace.numel() * workspace.element_size(), _p(status), _stream())
     _check(rc, "sapo_policy_loss_bwd")
+
+
+def sapo_policy_loss_bwd_active(hidden: torch.Tensor, W_head: torch.Tensor, ids: torch.Tensor,
+                                lse: torch.Tensor, gscale: torch.Tensor, dhidden: torch.Tensor,
+                                dW_head: torch.Tensor, accumulate_dW: bool, workspace: torch.Tensor,
+                                status: torch.Tensor, n_active: Optional[torch.Tensor] = None,
+                                T: Optional[int] = None) -> None:
+    """Backward over the tokens with a non-zero gradient factor only (same results)."""
+    _require_cuda()
+    T = int(hidden.shape[0]) if T is None else int(T)
+    H, V = int(hidden.shape[1]), int(W_head.shape[0])
+    rc = load().sapo_policy_loss_bwd_active(
+        _p(hidden), _p(W_head), _dtype_code(hidden), T, H, V, hidden.stride(0), W_head.stride(0),
+        _p(ids), _p(lse), _p(gscale), _p(dhidden), _p(dW_head), 1 if accumulate_dW else 0, _p(n_active),
+        _p(workspace), workspace.numel() * workspace.element_size(), _p(status), _stream())
+    _check(rc, "sapo_policy_loss_bwd_active")

@@ -16,6 +16,7 @@
 #include <cuda_bf16.h>
 
 #include "common.cuh"
+#include "compact.cuh"
 #include "umma.cuh"
 
 namespace sapo {
@@ -53,8 +54,40 @@ struct Sched {
   // is as full as the others.  A pair that gets only part of a tile's K range leaves a partial
   // accumulator in scratch; a small second kernel adds the parts up.
   int32_t dp_units, sk_tiles, sk_ipp;
+  int32_t k_split_ok; // the epilogue has scratch for K-split parts
+  // A size only the device knows (the number of active tokens after compaction), read by
+  // every CTA at start-up: dyn_dim 1 = it is M (rows), 2 = it is K (contraction length).
+  const int32_t* dyn_count;
+  int32_t dyn_dim;
+  int32_t skip_if_empty;  // dyn_dim 2 only: a zero-length contraction launches no work at all
   int32_t stats_id;   // row of the wait-cycle counters this launch adds to (instrumented builds)
 };
+
+// Cut a ragged last wave of long-K tiles along K over all the pairs (see Sched).
+__host__ __device__ inline void split_last_wave(Sched& s, int pairs) {
+  s.dp_units = s.num_units; s.sk_tiles = 0; s.sk_ipp = 1;
+  if (!s.k_split_ok || pairs <= 0) return;
+  const int rem = s.num_units % pairs;
+  if (rem != 0 && s.num_k_blocks >= 8 && s.n_per_unit == 1) {
+    s.dp_units = s.num_units - rem;
+    s.sk_tiles = rem;
+    s.sk_ipp = (int32_t)(((int64_t)rem * s.num_k_blocks + pairs - 1) / pairs);
+  }
+}
+
+// Fill in what depends on a device-side size; every CTA (and the fix-up kernel) does the same.
+__device__ __forceinline__ void finalize_sched(Sched& s, int pairs) {
+  if (s.dyn_dim == 0) return;
+  const int32_t n = *s.dyn_count;
+  if (s.dyn_dim == 1) {
+    s.num_m_blocks = (n + PAIR_M - 1) / PAIR_M;
+    s.num_units = s.num_m_blocks * s.units_per_m;
+  } else {
+    s.num_k_blocks = (n + BK - 1) / BK;
+    if (n == 0 && s.skip_if_empty) s.num_units = 0;   // adding an empty sum: leave the output alone
+  }
+  split_last_wave(s, pairs);
+}
 
 constexpr int PARTIAL_FLOATS = PAIR_M * BN;   // one partial accumulator tile: 256 x 256 fp32
 constexpr int MAX_PAIRS_SCRATCH = 96;          // CTA pairs the K-split scratch is sized for (a B200 has 74)
@@ -124,6 +157,7 @@ struct StageCtx {
 struct FwdEpi {
   static constexpr bool STAGED = false;
   static constexpr bool STREAMK = false;
+  template <class P> __device__ static void set_dynamic(P&, const Sched&) {}
 
   struct Params {
     const int32_t* ids; float* pm; float* ps; float* pz;  // partials [n_splits][T]
@@ -174,6 +208,9 @@ struct FwdEpi {
 struct DzEpi {
   static constexpr bool STAGED = true;
   static constexpr bool STREAMK = false;
+  template <class P> __device__ static void set_dynamic(P& p, const Sched& s) {
+    if (s.dyn_dim == 1) p.M = *s.dyn_count;
+  }
   struct Params {
     const int32_t* ids; const float* lse; const float* gscale;
     int64_t M; int32_t V; int32_t nvt;
@@ -244,11 +281,18 @@ struct DzEpi {
 struct StoreEpi {
   static constexpr bool STAGED = false;
   static constexpr bool STREAMK = true;
-  struct Params { float* C; int64_t ldc; int64_t M; int32_t N; int32_t accumulate; float* partials; };
+  // row_map (optional): output row of each accumulator row (rows of compacted tokens go back
+  // to their packed positions)
+  struct Params { float* C; int64_t ldc; int64_t M; int32_t N; int32_t accumulate; float* partials;
+                  const int32_t* row_map; };
+  template <class P> __device__ static void set_dynamic(P& p, const Sched& s) {
+    if (s.dyn_dim == 1) p.M = *s.dyn_count;
+  }
   int64_t row; bool valid; float* part; int n0;
   __device__ __forceinline__ void begin_unit(const Params& p, int mb, int r) {
     row = (int64_t)mb * BM + r;
     valid = row < p.M;
+    if (valid && p.row_map != nullptr) row = p.row_map[row];
     part = nullptr;
   }
   // a K-split part of a tile goes to scratch slot `slot` instead: rows [128 rank, +128) of a
@@ -282,8 +326,13 @@ struct StoreEpi {
 // Adds up the K-split parts of each tile the GEMM kernel left in scratch and stores the sum.
 // Part order is fixed (by pair index), so the result does not depend on timing.
 __global__ void __launch_bounds__(256)
-streamk_fixup_kernel(const Sched s, const StoreEpi::Params p) {
+streamk_fixup_kernel(const Sched s_arg, const StoreEpi::Params p_arg, int pairs) {
+  Sched s = s_arg;
+  StoreEpi::Params p = p_arg;
+  finalize_sched(s, pairs);
+  StoreEpi::set_dynamic(p, s);
   const int t = blockIdx.x >> 5;                 // K-split tile
+  if (t >= s.sk_tiles) return;
   const int row_begin = (blockIdx.x & 31) * 8;   // 8 of its 256 rows per block
   const long long first_it = (long long)t * s.num_k_blocks;
   const int p_first = (int)(first_it / s.sk_ipp);
@@ -295,8 +344,9 @@ streamk_fixup_kernel(const Sched s, const StoreEpi::Params p) {
   const int col = threadIdx.x;
   if (col >= s.tile_n || n0 + col >= p.N) return;
   for (int rr = row_begin; rr < row_begin + 8; ++rr) {
-    const int64_t row = (int64_t)pmb * PAIR_M + rr;
+    int64_t row = (int64_t)pmb * PAIR_M + rr;
     if (row >= p.M) break;
+    if (p.row_map != nullptr) row = p.row_map[row];
     const size_t off = (size_t)rr * BN + col;
     float sum = p.partials[(size_t)(2 * p_first + 1) * PARTIAL_FLOATS + off];
     for (int q = p_first + 1; q <= p_last; ++q) sum += p.partials[(size_t)(2 * q) * PARTIAL_FLOATS + off];
@@ -337,7 +387,11 @@ template <int A_KIND, bool B_MN, class Epi>
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
 umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                  const __grid_constant__ CUtensorMap map_c,   // output tiles of a staged epilogue
-                 const Sched sched, const typename Epi::Params ep, int32_t* status) {
+                 const Sched sched_arg, const typename Epi::Params ep_arg, int32_t* status) {
+  Sched sched = sched_arg;
+  typename Epi::Params ep = ep_arg;
+  finalize_sched(sched, (int)(gridDim.x >> 1));
+  Epi::set_dynamic(ep, sched);
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint8_t* smem_a = smem;
@@ -514,7 +568,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
         for (int c = c_begin; c < c_end; c += 2) {      // one 64-column group per turn
           tmem_ld_wait();
           if (c + 1 < c_end && c + 1 < c_tmem) tmem_ld32(t_addr + (c + 1) * 32, vb);
-          if (c >= c_tmem) {
+          if (c >= c_tmem || kb1 == kb0) {       // padding columns, or an empty contraction
             #pragma unroll
             for (int j = 0; j < 32; ++j) va[j] = 0.f;
           }
@@ -523,7 +577,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
           if (c + 1 < c_end) {
             tmem_ld_wait();
             if (c + 2 < c_end && c + 2 < c_tmem) tmem_ld32(t_addr + (c + 2) * 32, va);
-            if (c + 1 >= c_tmem) {
+            if (c + 1 >= c_tmem || kb1 == kb0) {
               #pragma unroll
               for (int j = 0; j < 32; ++j) vb[j] = 0.f;
             }
@@ -685,6 +739,7 @@ static Sched make_sched(int64_t M, int64_t N, int64_t K, int n_splits, bool m_fa
   s.n_cover = (int32_t)N;
   s.panel_nvt = 0;
   s.dp_units = s.num_units; s.sk_tiles = 0; s.sk_ipp = 1;
+  s.k_split_ok = 0; s.dyn_count = nullptr; s.dyn_dim = 0; s.skip_if_empty = 0;
   return s;
 }
 
@@ -737,14 +792,12 @@ static int launch_gemm(const CUtensorMap& ma, const CUtensorMap& mb, const CUten
     if (max_pairs > MAX_PAIRS_SCRATCH) max_pairs = MAX_PAIRS_SCRATCH;
   }
   int pairs = sched.num_units < max_pairs ? sched.num_units : max_pairs;
+  if (sc.dyn_dim != 0) pairs = max_pairs;          // sized on the device: bring every pair
   if constexpr (Epi::STREAMK) {
-    // a ragged last wave of long-K tiles is cut along K over all the pairs
-    const int rem = sched.num_units % max_pairs;
-    if (ep.partials != nullptr && rem != 0 && sched.num_k_blocks >= 8 && sched.n_per_unit == 1) {
-      pairs = max_pairs;
-      sc.dp_units = sched.num_units - rem;
-      sc.sk_tiles = rem;
-      sc.sk_ipp = (int32_t)ceil_div<int64_t>((int64_t)rem * sched.num_k_blocks, pairs);
+    sc.k_split_ok = ep.partials != nullptr ? 1 : 0;
+    if (sc.dyn_dim == 0) {
+      split_last_wave(sc, max_pairs);
+      if (sc.sk_tiles > 0) pairs = max_pairs;
     }
   }
   cfg.gridDim = dim3(2 * pairs, 1, 1);
@@ -753,9 +806,12 @@ static int launch_gemm(const CUtensorMap& ma, const CUtensorMap& mb, const CUten
     if (cudaLaunchKernelEx(&cfg, kern, ma, mb, mc, sc, ep, status) != cudaSuccess) return SAPO_ERR_CUDA;
   }
   if constexpr (Epi::STREAMK) {
-    if (sc.sk_tiles > 0) {
+    // with a device-side size the number of K-split tiles is not known here: launch for the
+    // most there can be, the kernel drops the blocks it does not need
+    const int fix_tiles = sc.dyn_dim != 0 ? (sc.k_split_ok ? pairs - 1 : 0) : sc.sk_tiles;
+    if (fix_tiles > 0) {
       KernelScope scope(SAPO_K_STREAMK_FIXUP, st);
-      streamk_fixup_kernel<<<sc.sk_tiles * 32, 256, 0, st>>>(sc, ep);
+      streamk_fixup_kernel<<<fix_tiles * 32, 256, 0, st>>>(sc, ep, pairs);
     }
   }
   return check_launch();
@@ -807,6 +863,36 @@ static BwdLayout bwd_layout(int64_t T, int32_t H, int32_t V, int32_t dtype) {
 }
 constexpr int64_t PANEL_ROWS_PREFERRED = 32768;
 
+// Scratch of the compacting backward in front of the regular backward's: scan counters, the
+// active-token list, compacted per-token vectors and hidden rows.
+struct ActiveLayout { size_t counts, n_active, chunk_counts, act_idx, ids, lse, g, hidden, total; };
+constexpr int MAX_ACTIVE_CHUNKS = 4096;
+static ActiveLayout active_layout(int64_t T, int32_t H) {
+  ActiveLayout L{};
+  size_t off = 0;
+  const size_t n_blocks = (size_t)ceil_div<int64_t>(T, COMPACT_BLOCK);
+  auto take = [&](size_t bytes) { const size_t at = off; off += round_up<size_t>(bytes, 256); return at; };
+  L.counts = take(n_blocks * 4);
+  L.n_active = take(4);
+  L.chunk_counts = take((size_t)MAX_ACTIVE_CHUNKS * 4);
+  L.act_idx = take((size_t)T * 4);
+  L.ids = take((size_t)T * 4);
+  L.lse = take((size_t)T * 4);
+  L.g = take((size_t)T * 4);
+  L.hidden = take((size_t)round_up<int64_t>(T, 128) * H * 2);
+  L.total = off;
+  return L;
+}
+
+// chunk_counts[c] = active tokens that fall into chunk c of `chunk_rows` compacted rows
+__global__ void chunk_counts_kernel(const int32_t* n_active, int64_t chunk_rows, int32_t n_chunks,
+                                    int32_t* chunk_counts) {
+  for (int c = threadIdx.x; c < n_chunks; c += blockDim.x) {
+    const int64_t left = (int64_t)*n_active - (int64_t)c * chunk_rows;
+    chunk_counts[c] = (int32_t)(left <= 0 ? 0 : (left < chunk_rows ? left : chunk_rows));
+  }
+}
+
 }  // namespace sapo
 
 // =============================================================================== C ABI
@@ -818,10 +904,11 @@ extern "C" size_t sapo_workspace_bytes(int32_t which, int64_t T, int32_t H, int3
     if (sms <= 0) sms = 148;
     return fwd_layout(T, H, V, dtype, sms).total;
   }
-  if (which == SAPO_WS_BWD) {
+  if (which == SAPO_WS_BWD || which == SAPO_WS_BWD_ACTIVE) {
     const BwdLayout L = bwd_layout(T, H, V, dtype);
     const int64_t rows = T < PANEL_ROWS_PREFERRED ? T : PANEL_ROWS_PREFERRED;
-    return L.fixed + (size_t)round_up<int64_t>(rows, BM) * L.bytes_per_row;
+    const size_t extra = which == SAPO_WS_BWD_ACTIVE ? active_layout(T, H).total : 0;
+    return extra + L.fixed + (size_t)round_up<int64_t>(rows, BM) * L.bytes_per_row;
   }
   return 0;
 }
@@ -1022,7 +1109,7 @@ extern "C" int sapo_policy_loss_bwd(const void* hidden, const void* W_head, int3
     {
       Sched sched = make_sched(tc, H, Vp, 0, /*m_fastest=*/false);
       sched.panel_nvt = nvt;
-      StoreEpi::Params ep{dhidden + t0 * (int64_t)H, H, tc, H, 0, partials};
+      StoreEpi::Params ep{dhidden + t0 * (int64_t)H, H, tc, H, 0, partials, nullptr};
       int rc = launch_gemm<2, true, StoreEpi>(map_p_two, map_w_mn, map_p_two, sched, ep, status, st, SAPO_K_BWD_DH);
       if (rc != SAPO_OK) return rc;
     }
@@ -1030,7 +1117,136 @@ extern "C" int sapo_policy_loss_bwd(const void* hidden, const void* W_head, int3
     {
       Sched sched = make_sched(V, H, tc, 0, /*m_fastest=*/false);
       sched.panel_nvt = nvt;
-      StoreEpi::Params ep{dW_head, H, V, H, (t0 > 0 || accumulate_dW) ? 1 : 0, partials};
+      StoreEpi::Params ep{dW_head, H, V, H, (t0 > 0 || accumulate_dW) ? 1 : 0, partials, nullptr};
+      int rc = launch_gemm<3, true, StoreEpi>(map_p_tile, map_h_mn, map_p_tile, sched, ep, status, st, SAPO_K_BWD_DW);
+      if (rc != SAPO_OK) return rc;
+    }
+  }
+  return SAPO_OK;
+}
+
+// ------------------------------------------------------------------------------------------
+// Backward over the active tokens only (g_t != 0): same results as sapo_policy_loss_bwd, less
+// tensor work when many tokens are inactive.  The number of active tokens stays on the device:
+// the GEMM kernels read it when they start, so the call does not synchronise.
+extern "C" int sapo_policy_loss_bwd_active(const void* hidden, const void* W_head, int32_t dtype,
+                                           int64_t T, int32_t H, int32_t V, int64_t ld_hidden, int64_t ld_W,
+                                           const int32_t* ids, const float* lse, const float* gscale,
+                                           float* dhidden, float* dW_head, int32_t accumulate_dW,
+                                           int32_t* n_active_out,
+                                           void* workspace, size_t workspace_bytes,
+                                           int32_t* status, void* stream) {
+  using namespace sapo;
+  if (!hidden || !W_head || !ids || !lse || !gscale || !dhidden || !dW_head || !workspace || !status)
+    return SAPO_ERR_INVALID_ARG;
+  if (dtype != SAPO_DTYPE_BF16 && dtype != SAPO_DTYPE_F32) return SAPO_ERR_INVALID_ARG;
+  if (T < 1 || H < 1 || V < 1 || ld_hidden < H || ld_W < H) return SAPO_ERR_INVALID_ARG;
+  if (!shapes_ok(T, H, V)) return SAPO_ERR_UNSUPPORTED_SHAPE;
+  const int esz = dtype == SAPO_DTYPE_BF16 ? 2 : 4;
+  if (!aligned16(hidden) || !aligned16(W_head) || !aligned16(workspace) || !aligned16(dhidden) ||
+      !aligned16(dW_head) || (ld_hidden * esz) % 16 || (ld_W * esz) % 16)
+    return SAPO_ERR_INVALID_ARG;
+  const ActiveLayout AL = active_layout(T, H);
+  const BwdLayout L = bwd_layout(T, H, V, dtype);
+  if (workspace_bytes < AL.total + L.fixed + (size_t)BM * L.bytes_per_row) return SAPO_ERR_WORKSPACE_TOO_SMALL;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  uint8_t* ws0 = static_cast<uint8_t*>(workspace);
+  uint8_t* ws = ws0 + AL.total;                                   // the regular backward's layout
+  const size_t ws_bytes = workspace_bytes - AL.total;
+  int32_t* counts = reinterpret_cast<int32_t*>(ws0 + AL.counts);
+  int32_t* n_active = reinterpret_cast<int32_t*>(ws0 + AL.n_active);
+  int32_t* chunk_counts = reinterpret_cast<int32_t*>(ws0 + AL.chunk_counts);
+  int32_t* act_idx = reinterpret_cast<int32_t*>(ws0 + AL.act_idx);
+  int32_t* ids_act = reinterpret_cast<int32_t*>(ws0 + AL.ids);
+  float* lse_act = reinterpret_cast<float*>(ws0 + AL.lse);
+  float* g_act = reinterpret_cast<float*>(ws0 + AL.g);
+  __nv_bfloat16* hidden_act = reinterpret_cast<__nv_bfloat16*>(ws0 + AL.hidden);
+
+  const __nv_bfloat16* A = static_cast<const __nv_bfloat16*>(hidden);
+  const __nv_bfloat16* B = static_cast<const __nv_bfloat16*>(W_head);
+  int64_t lda = ld_hidden, ldb = ld_W;
+  if (dtype == SAPO_DTYPE_F32) {
+    __nv_bfloat16* a1 = reinterpret_cast<__nv_bfloat16*>(ws + L.a_hi);
+    __nv_bfloat16* b1 = reinterpret_cast<__nv_bfloat16*>(ws + L.b_hi);
+    int rc = launch_split(static_cast<const float*>(hidden), ld_hidden, T, H, a1, 2, st);
+    if (rc != SAPO_OK) return rc;
+    rc = launch_split(static_cast<const float*>(W_head), ld_W, V, H, b1, 2, st);
+    if (rc != SAPO_OK) return rc;
+    A = a1; B = b1; lda = H; ldb = H;
+  }
+  const int64_t Vp = padded_vocab(V);
+  const int32_t nvt = (int32_t)(Vp / 64);
+  __nv_bfloat16* panel = reinterpret_cast<__nv_bfloat16*>(ws + L.panel);
+  float* partials = reinterpret_cast<float*>(ws + L.partials);
+  const int64_t rows_fit = ((int64_t)((ws_bytes - L.fixed) / L.bytes_per_row) / BM) * BM;
+  const int64_t chunk_rows = rows_fit >= T ? round_up<int64_t>(T, BM) : rows_fit;
+  if (chunk_rows <= 0) return SAPO_ERR_WORKSPACE_TOO_SMALL;
+  const int64_t n_chunks = ceil_div<int64_t>(T, chunk_rows);
+  if (n_chunks > MAX_ACTIVE_CHUNKS) return SAPO_ERR_WORKSPACE_TOO_SMALL;
+
+  // 1. which tokens take part, in order; compacted copies of what the GEMMs read per token
+  const int sms = sm_count();
+  if (sms <= 0) return SAPO_ERR_CUDA;
+  const int n_blocks = (int)ceil_div<int64_t>(T, COMPACT_BLOCK);
+  {
+    KernelScope scope(SAPO_K_COMPACT, st);
+    active_count_kernel<<<n_blocks, COMPACT_BLOCK, 0, st>>>(gscale, T, counts);
+  }
+  { KernelScope scope(SAPO_K_COMPACT, st); active_scan_kernel<<<1, 1024, 0, st>>>(counts, n_blocks, n_active); }
+  {
+    KernelScope scope(SAPO_K_COMPACT, st);
+    active_assign_kernel<<<n_blocks, COMPACT_BLOCK, 0, st>>>(gscale, lse, ids, T, counts, act_idx, ids_act,
+                                                             lse_act, g_act, dhidden, H);
+  }
+  {
+    KernelScope scope(SAPO_K_COMPACT, st);
+    int64_t blocks = ceil_div<int64_t>(T, 8);
+    if (blocks > (int64_t)sms * 8) blocks = (int64_t)sms * 8;
+    active_gather_kernel<<<(int)blocks, 256, 0, st>>>(A, lda, H, act_idx, n_active, hidden_act);
+  }
+  { KernelScope scope(SAPO_K_COMPACT, st); chunk_counts_kernel<<<1, 256, 0, st>>>(n_active, chunk_rows, (int32_t)n_chunks, chunk_counts); }
+  if (n_active_out != nullptr &&
+      cudaMemcpyAsync(n_active_out, n_active, sizeof(int32_t), cudaMemcpyDeviceToDevice, st) != cudaSuccess)
+    return SAPO_ERR_CUDA;
+
+  // 2. the three contractions over at most T compacted rows; their true count is read on the device
+  CUtensorMap map_w_kmajor, map_w_mn;
+  if (!make_map(&map_w_kmajor, B, H, V, ldb, 128) || !make_map(&map_w_mn, B, H, V, ldb, 128))
+    return SAPO_ERR_CUDA;
+  for (int64_t c = 0; c < n_chunks; ++c) {
+    const int64_t t0 = c * chunk_rows;
+    const int64_t tc = (T - t0) < chunk_rows ? (T - t0) : chunk_rows;     // upper bound of this chunk
+    const int64_t tc_pad = round_up<int64_t>(tc, BM);
+    const __nv_bfloat16* A0 = hidden_act + t0 * (int64_t)H;
+    const int64_t panel_rows = ceil_div<int64_t>(tc, BM) * nvt * BM;
+    CUtensorMap map_h_kmajor, map_h_mn, map_p_two, map_p_tile;
+    if (!make_map(&map_h_kmajor, A0, H, tc_pad, H, BM) || !make_map(&map_h_mn, A0, H, tc_pad, H, 128) ||
+        !make_map(&map_p_two, panel, 64, panel_rows, 64, 256) ||
+        !make_map(&map_p_tile, panel, 64, panel_rows, 64, BM))
+      return SAPO_ERR_CUDA;
+    const int32_t* count = chunk_counts + c;
+    {
+      Sched sched = make_sched(tc, V, H, 0, /*m_fastest=*/true, /*tile_align=*/64);
+      sched.n_cover = (int32_t)Vp;
+      sched.dyn_count = count; sched.dyn_dim = 1;
+      DzEpi::Params ep{ids_act + t0, lse_act + t0, g_act + t0, tc, V, nvt};
+      int rc = launch_gemm<0, false, DzEpi>(map_h_kmajor, map_w_kmajor, map_p_tile, sched, ep, status, st, SAPO_K_BWD_DZ);
+      if (rc != SAPO_OK) return rc;
+    }
+    {
+      Sched sched = make_sched(tc, H, Vp, 0, /*m_fastest=*/false);
+      sched.panel_nvt = nvt;
+      sched.dyn_count = count; sched.dyn_dim = 1;
+      StoreEpi::Params ep{dhidden, H, tc, H, 0, partials, act_idx + t0};   // rows go back to their tokens
+      int rc = launch_gemm<2, true, StoreEpi>(map_p_two, map_w_mn, map_p_two, sched, ep, status, st, SAPO_K_BWD_DH);
+      if (rc != SAPO_OK) return rc;
+    }
+    {
+      const int acc = (c > 0 || accumulate_dW) ? 1 : 0;
+      Sched sched = make_sched(V, H, tc, 0, /*m_fastest=*/false);
+      sched.panel_nvt = nvt;
+      sched.dyn_count = count; sched.dyn_dim = 2; sched.skip_if_empty = acc;
+      StoreEpi::Params ep{dW_head, H, V, H, acc, partials, nullptr};
       int rc = launch_gemm<3, true, StoreEpi>(map_p_tile, map_h_mn, map_p_tile, sched, ep, status, st, SAPO_K_BWD_DW);
       if (rc != SAPO_OK) return rc;
     }

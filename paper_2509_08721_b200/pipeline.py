@@ -43,7 +43,7 @@ class PolicyScorer:
 
     def __init__(self, W_head: torch.Tensor, max_tokens: int, max_seqs: int, max_questions: int,
                  eps_low: float = 0.2, eps_high: float = 0.28, adv_eps: float = 1e-6,
-                 ddof: int = 0, grad_scale: float = 1.0, device="cuda"):
+                 ddof: int = 0, grad_scale: float = 1.0, device="cuda", active_backward: bool = False):
         if not torch.cuda.is_available():
             raise B.SapoError("PolicyScorer needs a CUDA device; there is no CPU path")
         B.load()
@@ -61,7 +61,10 @@ class PolicyScorer:
         self.dhidden = torch.empty(self.max_tokens, self.H, dtype=torch.float32, device=device)
         self.dW = torch.empty(self.V, self.H, dtype=torch.float32, device=device)
         nf = B.sapo_workspace_bytes(B.WS_FWD, self.max_tokens, self.H, self.V, self.dcode)
-        nb = B.sapo_workspace_bytes(B.WS_BWD, self.max_tokens, self.H, self.V, self.dcode)
+        self.active_backward = bool(active_backward)   # contract only tokens with a non-zero gradient factor
+        nb = B.sapo_workspace_bytes(B.WS_BWD_ACTIVE if self.active_backward else B.WS_BWD,
+                                    self.max_tokens, self.H, self.V, self.dcode)
+        self.n_active = torch.zeros(1, dtype=torch.int32, device=device)
         # forward and backward never overlap on the stream, so they share one scratch buffer
         self.workspace = torch.empty(max(nf + 4 * self.max_seqs + 256, nb), dtype=torch.uint8, device=device)
         self.status = B.new_status(device)
@@ -81,8 +84,13 @@ class PolicyScorer:
         B.sapo_policy_loss_fwd(p["hidden"], self.W, p["ids"], p["old_logp"], self.adv, cu,
                                self.eps_low, self.eps_high, self.grad_scale, self.fwd,
                                self.workspace, self.status, T=T)
-        B.sapo_policy_loss_bwd(p["hidden"], self.W, p["ids"], self.fwd["lse"], self.fwd["gscale"],
-                               self.dhidden, self.dW, False, self.workspace, self.status, T=T)
+        if self.active_backward:
+            B.sapo_policy_loss_bwd_active(p["hidden"], self.W, p["ids"], self.fwd["lse"], self.fwd["gscale"],
+                                          self.dhidden, self.dW, False, self.workspace, self.status,
+                                          self.n_active, T=T)
+        else:
+            B.sapo_policy_loss_bwd(p["hidden"], self.W, p["ids"], self.fwd["lse"], self.fwd["gscale"],
+                                   self.dhidden, self.dW, False, self.workspace, self.status, T=T)
         return StepResult(self.fwd["loss"], self.fwd, self.dhidden, self.dW, p, self.adv)
 
     # -- one step from pinned host buffers -----------------------------------------------------
