@@ -120,11 +120,19 @@ typedef struct sapo_packed {
 } sapo_packed;
 
 /* Loss parameters.  The paper's run uses eps_low 0.2, eps_high 0.28 and no KL term
- * (Section 4.2).  grad_scale multiplies the per-token gradient factor (upstream dL). */
+ * (Section 4.2).  grad_scale multiplies the per-token gradient factor (upstream dL).
+ * loss_agg: 0 = mean over sequences of the token mean (the default reading), 1 = mean over all
+ * tokens (the aggregation of DAPO, which Section 4.2 cites).  kl_beta: weight of a penalty
+ * towards a reference policy, per token exp(d) - d - 1 with d = ref_logp[t] - logp[t], aggregated
+ * like the surrogate; 0 (the paper's choice) leaves ref_logp unused.  ref_logp: device pointer,
+ * [T], may be NULL when kl_beta is 0. */
 typedef struct sapo_loss_cfg {
   float eps_low;
   float eps_high;
   float grad_scale;
+  int32_t loss_agg;
+  float kl_beta;
+  const float* ref_logp;
 } sapo_loss_cfg;
 
 /* Section 3.2, training-set equation / Algorithm 1 "Assemble training set".
@@ -152,7 +160,7 @@ int sapo_group_advantages(const float* rewards, const int32_t* group_offsets, in
  *   z[t,v] = <hidden[t,:], W_head[v,:]>,  lse[t] = log sum_v exp z[t,v],
  *   logp[t] = z[t, ids[t]] - lse[t],      ratio[t] = exp(logp[t] - old_logp[t]),
  *   surr[t] = min(ratio*A, clip(ratio, 1-eps_low, 1+eps_high)*A),  A = adv[seq of t],
- *   loss    = -(1/S) sum_s (1/T_s) sum_{t in s} surr[t],
+ *   loss    = -(1/S) sum_s (1/T_s) sum_{t in s} surr[t]   (variants: see sapo_loss_cfg),
  *   gscale[t] = dloss/dlogp[t] = -grad_scale * A * ratio / (S*T_s) where the unclipped term
  *               is the min (ties included), else 0.
  * The [T,V] logits are never written to memory: the projection runs on the tensor cores and

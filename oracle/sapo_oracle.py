@@ -142,17 +142,24 @@ def _seq_of_token(cu_seqlens: np.ndarray) -> np.ndarray:
 
 def surrogate_from_logp(logp: np.ndarray, old_logp: np.ndarray, adv: np.ndarray,
                         cu_seqlens: np.ndarray, eps_low: float, eps_high: float,
-                        grad_scale: float = 1.0, n_seqs_total: Optional[int] = None
-                        ) -> Dict[str, np.ndarray]:
+                        grad_scale: float = 1.0, n_seqs_total: Optional[int] = None,
+                        loss_agg: int = 0, kl_beta: float = 0.0,
+                        ref_logp: Optional[np.ndarray] = None,
+                        n_tokens_total: Optional[int] = None) -> Dict[str, np.ndarray]:
     """Clipped-ratio surrogate and its derivative with respect to logp (Section 4.2).
 
         rho_t = exp(logp_t - old_t)
         u_t   = min( rho_t * A_s , clip(rho_t, 1-eps_low, 1+eps_high) * A_s )
-        L     = - (1/S) sum_s (1/T_s) sum_{t in s} u_t            (KL weight 0)
-        g_t   = dL/dlogp_t = -(1/(S*T_s)) * A_s * rho_t * [unclipped term is the min]
+        o_t   = u_t - beta * kl_t,   kl_t = exp(ref_t - logp_t) - (ref_t - logp_t) - 1
+        L     = - sum_t w_t o_t,     w_t = 1/(S*T_s)  (loss_agg 0: mean over sequences of the
+                                     token mean)  or  1/T  (loss_agg 1: mean over all tokens)
+        g_t   = dL/dlogp_t = -w_t * ( A_s * rho_t * [unclipped term is the min]
+                                      - beta * (1 - exp(ref_t - logp_t)) )
+    The paper's runs use beta = 0 (Section 4.2), the default; kl_t is the non-negative
+    estimator GRPO uses for its penalty towards a reference policy.
     The min is taken as "unclipped <= clipped" (ties count as unclipped).
-    `n_seqs_total` overrides S in the 1/S factor when the rows given are only part of
-    a batch (used to score sampled sequences of a large batch).
+    `n_seqs_total` / `n_tokens_total` override S / T in the weights when the rows given are
+    only part of a batch (used to score sampled sequences of a large batch).
     """
     logp = np.asarray(logp, dtype=np.float64)
     old = np.asarray(old_logp, dtype=np.float64)
@@ -160,6 +167,7 @@ def surrogate_from_logp(logp: np.ndarray, old_logp: np.ndarray, adv: np.ndarray,
     cu = np.asarray(cu_seqlens, dtype=np.int64)
     S = len(cu) - 1
     S_norm = S if n_seqs_total is None else n_seqs_total
+    T_norm = int(cu[-1]) if n_tokens_total is None else n_tokens_total
     seq = _seq_of_token(cu)
     T_s = np.diff(cu).astype(np.float64)
     A_t = A[seq]
@@ -168,21 +176,30 @@ def surrogate_from_logp(logp: np.ndarray, old_logp: np.ndarray, adv: np.ndarray,
     clipped = np.clip(rho, 1.0 - eps_low, 1.0 + eps_high) * A_t
     u = np.minimum(unclipped, clipped)
     active = (unclipped <= clipped).astype(np.float64)
+    if kl_beta != 0.0:
+        d = np.asarray(ref_logp, dtype=np.float64) - logp
+        kl = np.exp(d) - d - 1.0
+        dkl = 1.0 - np.exp(d)                      # d kl_t / d logp_t
+    else:
+        kl = np.zeros_like(logp)
+        dkl = np.zeros_like(logp)
+    o = u - kl_beta * kl
+    w = 1.0 / (S_norm * T_s[seq]) if loss_agg == 0 else np.full(len(logp), 1.0 / T_norm)
     seq_surr = np.zeros(S)
     for s in range(S):
-        seq_surr[s] = u[cu[s]:cu[s + 1]].sum() / T_s[s]
-    loss = -seq_surr.sum() / S_norm
-    g = -(1.0 / (S_norm * T_s[seq])) * A_t * rho * active * grad_scale
+        seq_surr[s] = o[cu[s]:cu[s + 1]].sum() / T_s[s]
+    loss = -(w * o).sum()
+    g = -w * (A_t * rho * active - kl_beta * dkl) * grad_scale
     return {"ratio": rho, "surr": u, "gscale": g, "seq_surr": seq_surr, "loss": loss,
-            "active": active}
+            "active": active, "kl": kl}
 
 
 def policy_loss_fwd(hidden, W, ids, old_logp, adv, cu_seqlens, eps_low=0.2, eps_high=0.2,
-                    grad_scale=1.0) -> Dict[str, np.ndarray]:
+                    grad_scale=1.0, loss_agg=0, kl_beta=0.0, ref_logp=None) -> Dict[str, np.ndarray]:
     """Forward of the policy loss: log-probs at the LM head, then the surrogate."""
     lp = token_logprobs(hidden, W, ids)
     out = surrogate_from_logp(lp["logp"], old_logp, adv, cu_seqlens, eps_low, eps_high,
-                              grad_scale)
+                              grad_scale, loss_agg=loss_agg, kl_beta=kl_beta, ref_logp=ref_logp)
     out["logp"], out["lse"] = lp["logp"], lp["lse"]
     return out
 

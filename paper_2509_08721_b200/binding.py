@@ -53,7 +53,8 @@ class PackedC(C.Structure):
 
 
 class LossCfgC(C.Structure):
-    _fields_ = [("eps_low", C.c_float), ("eps_high", C.c_float), ("grad_scale", C.c_float)]
+    _fields_ = [("eps_low", C.c_float), ("eps_high", C.c_float), ("grad_scale", C.c_float),
+                ("loss_agg", C.c_int32), ("kl_beta", C.c_float), ("ref_logp", C.c_void_p)]
 
 
 _lib: Optional[C.CDLL] = None
@@ -246,12 +247,13 @@ def sapo_policy_loss_fwd(hidden: torch.Tensor, W_head: torch.Tensor, ids: torch.
                          old_logp: torch.Tensor, adv: torch.Tensor, cu_seqlens: torch.Tensor,
                          eps_low: float, eps_high: float, grad_scale: float,
                          out: Dict[str, torch.Tensor], workspace: torch.Tensor,
-                         status: torch.Tensor, T: Optional[int] = None) -> None:
+                         status: torch.Tensor, T: Optional[int] = None, loss_agg: int = 0,
+                         kl_beta: float = 0.0, ref_logp: Optional[torch.Tensor] = None) -> None:
     _require_cuda()
     T = int(hidden.shape[0]) if T is None else int(T)
     H, V = int(hidden.shape[1]), int(W_head.shape[0])
     S = int(cu_seqlens.numel() - 1)
-    cfg = LossCfgC(eps_low, eps_high, grad_scale)
+    cfg = LossCfgC(eps_low, eps_high, grad_scale, int(loss_agg), float(kl_beta), _p(ref_logp))
     rc = load().sapo_policy_loss_fwd(
         _p(hidden), _p(W_head), _dtype_code(hidden), T, H, V, hidden.stride(0), W_head.stride(0),
         _p(ids), _p(old_logp), _p(adv), _p(cu_seqlens), S, C.byref(cfg),
@@ -273,7 +275,7 @@ def sapo_policy_loss_fwd_static(hidden: torch.Tensor, W_head: torch.Tensor, ids:
     T = int(hidden.shape[0]) if T is None else int(T)
     H, V = int(hidden.shape[1]), int(W_head.shape[0])
     S = int(cu_seqlens.numel() - 1)
-    cfg = LossCfgC(eps_low, eps_high, grad_scale)
+    cfg = LossCfgC(eps_low, eps_high, grad_scale, 0, 0.0, None)
     rc = load().sapo_policy_loss_fwd_static(
         _p(hidden), _p(W_head), _dtype_code(hidden), T, H, V, hidden.stride(0), W_head.stride(0),
         _p(ids), _p(old_logp), _p(adv), _p(cu_seqlens), S, C.byref(cfg),

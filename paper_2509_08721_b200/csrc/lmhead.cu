@@ -631,6 +631,7 @@ struct TailArgs {
   const float* pm; const float* ps; const float* pz; int32_t n_splits; int64_t T;
   const int32_t* ids; int32_t V; const float* old_logp; const float* adv; const int32_t* cu; int32_t S;
   float lo_edge, hi_edge, grad_scale;
+  int32_t loss_agg; float kl_beta; const float* ref_logp;   // variants: token-level mean, KL penalty
   float* logp; float* lse; float* ratio; float* surr; float* gscale; float* seq_surr;
   int32_t* status;
 };
@@ -654,7 +655,8 @@ __global__ void __launch_bounds__(256) loss_tail_kernel(TailArgs a) {
     const int32_t t0 = a.cu[s], t1 = a.cu[s + 1];
     const int32_t Ts = t1 - t0;
     const float A = a.adv[s];
-    const float w = Ts > 0 ? 1.f / ((float)a.S * (float)Ts) : 0.f;
+    // weight of a token of this sequence: 1/(S T_s) (mean of token means) or 1/T (token mean)
+    const float w = Ts <= 0 ? 0.f : (a.loss_agg == 0 ? 1.f / ((float)a.S * (float)Ts) : 1.f / (float)a.T);
     double acc = 0.0;
     for (int32_t t = t0 + threadIdx.x; t < t1; t += 256) {
       float M = -INFINITY;
@@ -674,21 +676,33 @@ __global__ void __launch_bounds__(256) loss_tail_kernel(TailArgs a) {
       const float un = rho * A;
       const float cl = fminf(fmaxf(rho, a.lo_edge), a.hi_edge) * A;
       const float u = bad ? 0.f : fminf(un, cl);
-      const float g = (!bad && un <= cl) ? -a.grad_scale * A * rho * w : 0.f;
+      float g = (!bad && un <= cl) ? -a.grad_scale * A * rho * w : 0.f;
+      float obj = u;
+      if (a.kl_beta != 0.f && !bad) {
+        // penalty towards a reference policy: kl = e^d - d - 1, d = ref - logp; d kl / d logp = 1 - e^d
+        const float d = a.ref_logp[t] - lp;
+        const float ed = expf(d);
+        obj -= a.kl_beta * (ed - d - 1.f);
+        g += a.grad_scale * w * a.kl_beta * (1.f - ed);
+      }
       a.lse[t] = lse; a.logp[t] = lp; a.ratio[t] = rho; a.surr[t] = u; a.gscale[t] = g;
-      acc += (double)u;
+      acc += (double)obj;
     }
     const double tot = block_sum_256(acc, sh);
     if (threadIdx.x == 0) a.seq_surr[s] = Ts > 0 ? (float)(tot / (double)Ts) : 0.f;
   }
 }
 
-__global__ void __launch_bounds__(256) loss_final_kernel(const float* seq_surr, int32_t S, float* loss) {
+// loss = -(1/S) sum_s seq_surr[s], or with token-level aggregation -(1/T) sum_s T_s seq_surr[s]
+__global__ void __launch_bounds__(256)
+loss_final_kernel(const float* seq_surr, const int32_t* cu, int32_t S, int64_t T, int32_t loss_agg, float* loss) {
   __shared__ double sh[8];
   double acc = 0.0;
-  for (int32_t s = threadIdx.x; s < S; s += 256) acc += (double)seq_surr[s];
+  for (int32_t s = threadIdx.x; s < S; s += 256)
+    acc += loss_agg == 0 ? (double)seq_surr[s] : (double)seq_surr[s] * (double)(cu[s + 1] - cu[s]);
   const double tot = block_sum_256(acc, sh);
-  if (threadIdx.x == 0) *loss = S > 0 ? (float)(-tot / (double)S) : 0.f;
+  const double n = loss_agg == 0 ? (double)S : (double)T;
+  if (threadIdx.x == 0) *loss = n > 0 ? (float)(-tot / n) : 0.f;
 }
 
 // ---------------------------------------------------------------------------- host side
@@ -941,6 +955,8 @@ extern "C" int sapo_policy_loss_fwd(const void* hidden, const void* W_head, int3
       (ld_W * esz) % 16)
     return SAPO_ERR_INVALID_ARG;
   if (!(h_cfg->eps_low >= 0.f) || !(h_cfg->eps_high >= 0.f)) return SAPO_ERR_INVALID_ARG;
+  if ((h_cfg->loss_agg != 0 && h_cfg->loss_agg != 1) || (h_cfg->kl_beta != 0.f && !h_cfg->ref_logp))
+    return SAPO_ERR_INVALID_ARG;
   const int sms = sm_count();
   if (sms <= 0) return SAPO_ERR_CUDA;
   const FwdLayout L = fwd_layout(T, H, V, dtype, sms);
@@ -977,11 +993,12 @@ extern "C" int sapo_policy_loss_fwd(const void* hidden, const void* W_head, int3
   ta.n_splits = 2 * sched.units_per_m;   // one partial per vocab split and column half
   ta.ids = ids; ta.V = V; ta.old_logp = old_logp; ta.adv = adv; ta.cu = cu_seqlens; ta.S = S;
   ta.lo_edge = 1.f - h_cfg->eps_low; ta.hi_edge = 1.f + h_cfg->eps_high; ta.grad_scale = h_cfg->grad_scale;
+  ta.loss_agg = h_cfg->loss_agg; ta.kl_beta = h_cfg->kl_beta; ta.ref_logp = h_cfg->ref_logp;
   ta.logp = logp; ta.lse = lse; ta.ratio = ratio; ta.surr = surr; ta.gscale = gscale; ta.seq_surr = seq_out;
   ta.status = status;
   const int tail_blocks = S < sms * 8 ? S : sms * 8;
   { KernelScope scope(SAPO_K_LOSS_TAIL, st); loss_tail_kernel<<<tail_blocks, 256, 0, st>>>(ta); }
-  { KernelScope scope(SAPO_K_LOSS_FINAL, st); loss_final_kernel<<<1, 256, 0, st>>>(seq_out, S, loss); }
+  { KernelScope scope(SAPO_K_LOSS_FINAL, st); loss_final_kernel<<<1, 256, 0, st>>>(seq_out, cu_seqlens, S, T, h_cfg->loss_agg, loss); }
   return check_launch();
 }
 

@@ -216,6 +216,59 @@ def test_loss_inside_the_clip_band_and_fully_clipped():
     assert math.isclose(out["loss"], expect, rel_tol=1e-12)
 
 
+def test_token_level_aggregation_and_kl_term():
+    """loss_agg = 1 weighs every token 1/T; the KL penalty is the non-negative estimator
+    exp(d) - d - 1 of d = ref - logp, zero (with zero slope) when the policies agree."""
+    rng, cu, h, W, ids, adv = _toy(3)
+    T_s, S = np.diff(cu), len(adv)
+    T = int(cu[-1])
+    cur = orc.token_logprobs(h, W, ids)["logp"]
+    # rho = 1: token-level loss is -(1/T) sum_s T_s A_s
+    out = orc.policy_loss_fwd(h, W, ids, cur, adv, cu, loss_agg=1)
+    assert math.isclose(out["loss"], -(T_s * adv).sum() / T, rel_tol=1e-13)
+    assert np.allclose(out["gscale"], -np.repeat(adv, T_s) / T, rtol=1e-13)
+    # equal lengths: both aggregations coincide
+    cu_eq = np.array([0, 3, 6, 9, 12], np.int32)
+    d = rng.uniform(-0.1, 0.1, size=12)
+    a0 = orc.surrogate_from_logp(cur[:12], cur[:12] - d, adv, cu_eq, 0.2, 0.28, loss_agg=0)
+    a1 = orc.surrogate_from_logp(cur[:12], cur[:12] - d, adv, cu_eq, 0.2, 0.28, loss_agg=1)
+    assert math.isclose(a0["loss"], a1["loss"], rel_tol=1e-13)
+    # KL: ref = logp gives no penalty and no gradient; otherwise positive, equal to the
+    # importance-weighted form E_q[...] term by term, and added with weight beta
+    k0 = orc.surrogate_from_logp(cur, cur, adv, cu, 0.2, 0.28, kl_beta=0.3, ref_logp=cur)
+    b0 = orc.surrogate_from_logp(cur, cur, adv, cu, 0.2, 0.28)
+    assert np.all(k0["kl"] == 0.0) and math.isclose(k0["loss"], b0["loss"], rel_tol=1e-15)
+    assert np.allclose(k0["gscale"], b0["gscale"], rtol=1e-15)
+    ref = cur + rng.normal(size=T) * 0.3
+    k = orc.surrogate_from_logp(cur, cur, adv, cu, 0.2, 0.28, kl_beta=0.3, ref_logp=ref)
+    ratio = np.exp(ref - cur)
+    assert np.all(k["kl"] > 0) and np.allclose(k["kl"], ratio - np.log(ratio) - 1, rtol=1e-13)
+    pen = sum(k["kl"][cu[s]:cu[s + 1]].mean() for s in range(S)) / S
+    assert math.isclose(k["loss"], b0["loss"] + 0.3 * pen, rel_tol=1e-12)
+
+
+def test_variant_gradients_match_finite_differences():
+    rng, cu, h, W, ids, adv = _toy(5, T_s=(2, 3, 1, 2), V=11, H=4)
+    cur = orc.token_logprobs(h, W, ids)["logp"]
+    old = cur + rng.normal(size=len(cur)) * 0.3
+    ref = cur + rng.normal(size=len(cur)) * 0.2
+    kw = dict(eps_low=0.2, eps_high=0.28, loss_agg=1, kl_beta=0.4, ref_logp=ref)
+    f = orc.policy_loss_fwd(h, W, ids, old, adv, cu, **kw)
+    g = orc.policy_loss_bwd(h, W, ids, f["lse"], f["gscale"])
+    d = 1e-6
+    for (arr, grad) in ((h, g["dhidden"]), (W, g["dW"])):
+        num = np.zeros_like(arr)
+        for idx in np.ndindex(*arr.shape):
+            keep = arr[idx]
+            arr[idx] = keep + d
+            fp = orc.policy_loss_fwd(h, W, ids, old, adv, cu, **kw)["loss"]
+            arr[idx] = keep - d
+            fm = orc.policy_loss_fwd(h, W, ids, old, adv, cu, **kw)["loss"]
+            arr[idx] = keep
+            num[idx] = (fp - fm) / (2 * d)
+        assert np.allclose(grad, num, rtol=1e-6, atol=1e-9)
+
+
 # ------------------------------------------------------------------------------ gradient
 def _loss_only(h, W, ids, old, adv, cu, lo, hi):
     return orc.policy_loss_fwd(h, W, ids, old, adv, cu, lo, hi)["loss"]

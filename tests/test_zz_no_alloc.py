@@ -73,7 +73,7 @@ def test_static_scratch_forward_matches_the_regular_one_twice_in_a_row():
 
 def test_static_scratch_rejects_what_does_not_fit():
     lib = B.load()
-    cfg = B.LossCfgC(0.2, 0.2, 1.0)
+    cfg = B.LossCfgC(0.2, 0.2, 1.0, 0, 0.0, None)
     one = torch.zeros(256, dtype=torch.float32, device="cuda")
     # three floats of scratch per token (and per vocab split): two million tokens need 24 MB
     T, H, V = 2_000_000, 64, 512
