@@ -220,6 +220,22 @@ int sapo_policy_loss_bwd_active(const void* hidden, const void* W_head, int32_t 
                                 void* workspace, size_t workspace_bytes,
                                 int32_t* status, void* stream);
 
+/* Section 3.2 (nodes filter and sample what the swarm shares) / Section 5 (the experiments'
+ * policy: discard rollouts with zero advantage, then sample uniformly from the rest).
+ * The pool holds n_entries rollouts; entry g is a question's group of completions with rewards
+ * rewards[group_offsets[g] .. group_offsets[g+1]).  An entry whose rewards are all equal has zero
+ * advantage throughout and is dropped; of the others, J are drawn uniformly without replacement
+ * (all of them if there are fewer than J): entry g gets the key
+ * (philox4x32-10(counter = (g,0,0,0), key = (seed low, seed high))[0] << 32) | g and the J
+ * smallest keys win, so the draw depends only on the seed and the pool.  selected [J] receives
+ * the chosen entries in pool order, *n_selected how many there are, *n_candidates how many passed
+ * the filter (all device memory).  workspace: sapo_select_workspace_bytes(n_entries), 8-byte
+ * aligned. */
+int sapo_select_external(const float* rewards, const int32_t* group_offsets, int32_t n_entries,
+                         int32_t J, uint64_t seed, int32_t* selected, int32_t* n_selected,
+                         int32_t* n_candidates, void* workspace, size_t workspace_bytes, void* stream);
+size_t sapo_select_workspace_bytes(int32_t n_entries);
+
 /* Bytes of scratch the forward (SAPO_WS_FWD) or backward (SAPO_WS_BWD) call wants for
  * these sizes.  Returns 0 for invalid arguments. */
 size_t sapo_workspace_bytes(int32_t which, int64_t T, int32_t H, int32_t V, int32_t dtype);
@@ -269,7 +285,8 @@ int sapo_policy_loss_fwd_static(const void* hidden, const void* W_head, int32_t 
 #define SAPO_K_BWD_DW     9
 #define SAPO_K_STREAMK_FIXUP 10
 #define SAPO_K_COMPACT   11
-#define SAPO_K_COUNT      12
+#define SAPO_K_SELECT    12
+#define SAPO_K_COUNT      13
 int sapo_timing_enable(int32_t on);
 int sapo_timing_read(float* h_ms, int32_t* h_launches);
 int64_t sapo_launch_count(void);

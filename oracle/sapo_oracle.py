@@ -262,3 +262,52 @@ def dW_rows(hidden, W, ids, lse, gscale, rows) -> np.ndarray:
     dz += (np.asarray(ids, dtype=np.int64)[:, None] == rows[None, :])
     dz *= np.asarray(gscale, dtype=np.float64)[:, None]
     return dz.T @ h
+
+
+# --------------------------------------------------------------------------------------
+# Filtering and sampling the shared pool (Section 3.2, last paragraph before Algorithm 1, and
+# Section 5: nodes first discard rollouts with zero advantage, then sample uniformly from the
+# rest).  A pool entry is one question's rollout, i.e. its group of completions; its
+# advantages are all zero exactly when its rewards are all equal.
+_PHILOX_M0, _PHILOX_M1 = 0xD2511F53, 0xCD9E8D57
+_PHILOX_W0, _PHILOX_W1 = 0x9E3779B9, 0xBB67AE85
+
+
+def philox4x32(counter, key, rounds: int = 10):
+    """Philox-4x32 (Salmon, Moraes, Dror, Shaw: "Parallel random numbers: as easy as 1, 2, 3",
+    SC'11): a counter-based generator, four 32-bit outputs per (128-bit counter, 64-bit key)."""
+    c0, c1, c2, c3 = (int(x) & 0xFFFFFFFF for x in counter)
+    k0, k1 = (int(x) & 0xFFFFFFFF for x in key)
+    for _ in range(rounds):
+        p0 = _PHILOX_M0 * c0
+        p1 = _PHILOX_M1 * c2
+        hi0, lo0 = p0 >> 32, p0 & 0xFFFFFFFF
+        hi1, lo1 = p1 >> 32, p1 & 0xFFFFFFFF
+        c0, c1, c2, c3 = hi1 ^ c1 ^ k0, lo1, hi0 ^ c3 ^ k1, lo0
+        k0 = (k0 + _PHILOX_W0) & 0xFFFFFFFF
+        k1 = (k1 + _PHILOX_W1) & 0xFFFFFFFF
+    return c0, c1, c2, c3
+
+
+def select_external(rewards: np.ndarray, group_offsets: np.ndarray, J: int, seed: int
+                    ) -> Dict[str, np.ndarray]:
+    """Drop the pool entries whose rewards are all equal (zero advantage), then draw J of the
+    rest uniformly without replacement: every candidate g gets the 64-bit key
+    (philox4x32(counter=(g,0,0,0), key=(seed_lo, seed_hi))[0] << 32) | g and the J smallest keys
+    win.  Returns the chosen entries in pool order, the candidate flags and counts.
+    Fewer than J candidates: all of them are taken."""
+    r = np.asarray(rewards)
+    n = len(group_offsets) - 1
+    cand = np.zeros(n, dtype=bool)
+    for g in range(n):
+        a, b = int(group_offsets[g]), int(group_offsets[g + 1])
+        cand[g] = b > a and r[a:b].min() != r[a:b].max()
+    keys = []
+    for g in range(n):
+        if cand[g]:
+            x = philox4x32((g, 0, 0, 0), (seed & 0xFFFFFFFF, (seed >> 32) & 0xFFFFFFFF))[0]
+            keys.append(((x << 32) | g, g))
+    keys.sort()
+    chosen = sorted(g for _, g in keys[:max(0, J)])
+    return {"selected": np.asarray(chosen, dtype=np.int32), "candidates": cand,
+            "n_candidates": int(cand.sum()), "n_selected": len(chosen)}

@@ -28,10 +28,11 @@ ST_BITS = {
 EXPORTS = ("sapo_pack_rollouts", "sapo_group_advantages", "sapo_policy_loss_fwd",
            "sapo_policy_loss_bwd", "sapo_workspace_bytes", "sapo_workspace_bytes_min",
            "sapo_status_string", "sapo_timing_enable", "sapo_timing_read", "sapo_launch_count",
-           "sapo_policy_loss_fwd_static", "sapo_policy_loss_bwd_active")
+           "sapo_policy_loss_fwd_static", "sapo_policy_loss_bwd_active", "sapo_select_external",
+           "sapo_select_workspace_bytes")
 STATIC_SCRATCH_BYTES = 4 * 1024 * 1024
 KERNEL_NAMES = ("pack_scan", "pack_copy", "group_adv", "split_bf16", "fwd_gemm", "loss_tail",
-                "loss_final", "bwd_dz", "bwd_dh", "bwd_dw", "streamk_fixup", "compact")
+                "loss_final", "bwd_dz", "bwd_dh", "bwd_dw", "streamk_fixup", "compact", "select")
 
 
 class RolloutBufC(C.Structure):
@@ -92,6 +93,10 @@ def load() -> C.CDLL:
     lib.sapo_policy_loss_bwd_active.restype = C.c_int
     lib.sapo_policy_loss_bwd_active.argtypes = [vp, vp, i32, i64, i32, i32, i64, i64, vp, vp, vp, vp, vp,
                                                 i32, vp, vp, sz, vp, vp]
+    lib.sapo_select_external.restype = C.c_int
+    lib.sapo_select_external.argtypes = [vp, vp, i32, i32, C.c_uint64, vp, vp, vp, vp, sz, vp]
+    lib.sapo_select_workspace_bytes.restype = sz
+    lib.sapo_select_workspace_bytes.argtypes = [i32]
     lib.sapo_workspace_bytes.restype = sz
     lib.sapo_workspace_bytes.argtypes = [i32, i64, i32, i32, i32]
     lib.sapo_workspace_bytes_min.restype = sz
@@ -312,3 +317,19 @@ def sapo_policy_loss_bwd_active(hidden: torch.Tensor, W_head: torch.Tensor, ids:
         _p(ids), _p(lse), _p(gscale), _p(dhidden), _p(dW_head), 1 if accumulate_dW else 0, _p(n_active),
         _p(workspace), workspace.numel() * workspace.element_size(), _p(status), _stream())
     _check(rc, "sapo_policy_loss_bwd_active")
+
+
+def sapo_select_external(rewards: torch.Tensor, group_offsets: torch.Tensor, J: int, seed: int):
+    """Filter the pool (drop entries with all-equal rewards) and draw J of the rest uniformly.
+    Returns (selected [J] int32, n_selected [1], n_candidates [1]) device tensors."""
+    _require_cuda()
+    n = int(group_offsets.numel() - 1)
+    dev = group_offsets.device
+    selected = torch.empty(max(J, 1), dtype=torch.int32, device=dev)
+    n_sel = torch.zeros(1, dtype=torch.int32, device=dev)
+    n_cand = torch.zeros(1, dtype=torch.int32, device=dev)
+    ws = torch.empty(int(load().sapo_select_workspace_bytes(n)) // 8 + 1, dtype=torch.int64, device=dev)
+    rc = load().sapo_select_external(_p(rewards), _p(group_offsets), n, int(J), int(seed) & (2**64 - 1),
+                                     _p(selected), _p(n_sel), _p(n_cand), _p(ws), ws.numel() * 8, _stream())
+    _check(rc, "sapo_select_external")
+    return selected, n_sel, n_cand

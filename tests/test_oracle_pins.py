@@ -3,6 +3,7 @@ form, a library routine, an invariant, brute force on tiny inputs or finite diff
 so that a dropped term, a wrong sign or index, or a transposed operand fails at least one.
 CPU only."""
 import math
+import os
 
 import numpy as np
 import pytest
@@ -354,6 +355,42 @@ def test_dW_rows_equals_the_rows_of_the_full_gradient():
     rows = [0, 3, int(ids[0]), 16]
     assert np.allclose(orc.dW_rows(h, W, ids, f["lse"], f["gscale"], rows), g["dW"][rows],
                        rtol=1e-12, atol=1e-16)
+
+
+# ------------------------------------------------------------- pool filter and sampling
+def test_philox_matches_the_published_known_answers():
+    path = os.path.join(os.path.dirname(__file__), "golden", "philox4x32_10_known_answers.txt")
+    rows = [l.split() for l in open(path) if l.strip() and not l.startswith("#")]
+    assert len(rows) == 3
+    for r in rows:
+        v = [int(x, 16) for x in r]
+        assert list(orc.philox4x32(v[0:4], v[4:6])) == v[6:10]
+
+
+def test_select_external_filters_zero_advantage_and_samples_uniformly():
+    rng = np.random.default_rng(0)
+    sizes = rng.integers(1, 9, size=60)
+    go = np.concatenate([[0], np.cumsum(sizes)]).astype(np.int32)
+    r = rng.integers(0, 2, size=go[-1]).astype(np.float32)
+    const = np.array([len(set(r[go[g]:go[g + 1]])) == 1 for g in range(60)])
+    out = orc.select_external(r, go, 10, seed=123)
+    assert np.array_equal(out["candidates"], ~const)            # brute-force filter
+    sel = out["selected"]
+    assert len(sel) == 10 == len(set(sel.tolist())) and np.all(np.diff(sel) > 0)
+    assert not const[sel].any()                                 # only informative rollouts
+    # fewer candidates than asked for: all of them; J = 0: none
+    assert np.array_equal(orc.select_external(r, go, 1000, seed=5)["selected"], np.nonzero(~const)[0])
+    assert orc.select_external(r, go, 0, seed=5)["n_selected"] == 0
+    # same seed, same draw; the draw is uniform over the candidates (frequency test over seeds)
+    assert np.array_equal(orc.select_external(r, go, 10, seed=123)["selected"], sel)
+    cand = np.nonzero(~const)[0]
+    hits = np.zeros(60)
+    n_seeds = 600
+    for seed in range(n_seeds):
+        hits[orc.select_external(r, go, 10, seed=seed)["selected"]] += 1
+    p = 10 / len(cand)
+    sd = math.sqrt(n_seeds * p * (1 - p))
+    assert np.all(np.abs(hits[cand] - n_seeds * p) < 5 * sd) and hits[const].sum() == 0
 
 
 # ------------------------------------------------------------------ the input generator
