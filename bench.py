@@ -201,6 +201,14 @@ def hbm_kernels(torch, B, peaks, H=896, n_rollouts=2048, mean_len=288, n_groups=
     ms_pack = timed(lambda: B.sapo_pack_rollouts(bufs[0], bufs[1], sel, out, status))
     ms_adv = timed(lambda: B.sapo_group_advantages(rewards, go, 1e-6, 0, adv, None, None, status))
     assert int(status.item()) == 0 and int(out["n_tokens"].item()) == T
+    # Adam step on an LM-head-sized weight: 16 bytes read + 14 written per element
+    V_adam = 151936
+    master = torch.randn(V_adam, H, device="cuda") * 0.02
+    mom, var = torch.zeros_like(master), torch.zeros_like(master)
+    grad = torch.randn(V_adam, H, device="cuda") * 1e-3
+    w16 = torch.empty(V_adam, H, device="cuda", dtype=torch.bfloat16)
+    ms_adam = timed(lambda: B.sapo_adam_step(master, mom, var, grad, w16, 1))
+    bytes_adam = 30.0 * V_adam * H
     bytes_pack = 2.0 * T * (2 * H + 8)
     bytes_adv = 8.0 * rewards.numel() + 4.0 * n_groups
     peak = peaks["hbm_gbs"]
@@ -208,6 +216,7 @@ def hbm_kernels(torch, B, peaks, H=896, n_rollouts=2048, mean_len=288, n_groups=
                                    "frac": nbytes / ms / 1e6 / peak, "ms": ms, "bytes": nbytes, "case": what}
     return {"pack": mk(ms_pack, bytes_pack, f"{T} tokens of {H} bf16 from {2 * n_rollouts} rollouts"),
             "advantages": mk(ms_adv, bytes_adv, f"{n_groups} questions x 8 completions"),
+            "adam": mk(ms_adam, bytes_adam, f"weight [{V_adam}, {H}] fp32 master + moments + bf16 copy"),
             "peak_source": peaks["source"] + " (copy bandwidth)"}
 
 

@@ -236,6 +236,18 @@ int sapo_select_external(const float* rewards, const int32_t* group_offsets, int
                          int32_t* n_candidates, void* workspace, size_t workspace_bytes, void* stream);
 size_t sapo_select_workspace_bytes(int32_t n_entries);
 
+/* Section 4.2: the policy is updated with Adam (default hyper-parameters, learning rate 0.001).
+ * One Adam step (Kingma & Ba, Algorithm 1) on a [rows, cols] weight such as W_head, from the
+ * fp32 gradient sapo_policy_loss_bwd wrote:
+ *   m <- beta1 m + (1-beta1) g;  v <- beta2 v + (1-beta2) g^2;
+ *   master <- master - lr * (m / (1-beta1^step)) / (sqrt(v / (1-beta2^step)) + eps).
+ * master, m, v, grad: fp32 [rows, cols], contiguous, 16-byte aligned, updated in place (grad is
+ * only read).  w_bf16 (may be NULL): bf16 [rows, ld_w] copy of the new master weight, rounded to
+ * nearest even — the operand the next forward reads.  step counts from 1.  cols % 4 == 0. */
+int sapo_adam_step(float* master, float* m, float* v, const float* grad, void* w_bf16,
+                   int64_t rows, int32_t cols, int64_t ld_w, int32_t step,
+                   float lr, float beta1, float beta2, float eps, void* stream);
+
 /* Bytes of scratch the forward (SAPO_WS_FWD) or backward (SAPO_WS_BWD) call wants for
  * these sizes.  Returns 0 for invalid arguments. */
 size_t sapo_workspace_bytes(int32_t which, int64_t T, int32_t H, int32_t V, int32_t dtype);
@@ -286,7 +298,8 @@ int sapo_policy_loss_fwd_static(const void* hidden, const void* W_head, int32_t 
 #define SAPO_K_STREAMK_FIXUP 10
 #define SAPO_K_COMPACT   11
 #define SAPO_K_SELECT    12
-#define SAPO_K_COUNT      13
+#define SAPO_K_ADAM      13
+#define SAPO_K_COUNT      14
 int sapo_timing_enable(int32_t on);
 int sapo_timing_read(float* h_ms, int32_t* h_launches);
 int64_t sapo_launch_count(void);

@@ -311,3 +311,19 @@ def select_external(rewards: np.ndarray, group_offsets: np.ndarray, J: int, seed
     chosen = sorted(g for _, g in keys[:max(0, J)])
     return {"selected": np.asarray(chosen, dtype=np.int32), "candidates": cand,
             "n_candidates": int(cand.sum()), "n_selected": len(chosen)}
+
+
+# --------------------------------------------------------------------------------------
+def adam_step(theta, grad, m, v, step: int, lr=1e-3, beta1=0.9, beta2=0.999, eps=1e-8):
+    """One Adam update (Kingma & Ba, Algorithm 1) with the default hyper-parameters the paper's
+    runs use (Section 4.2: Adam, learning rate 0.001), in float64:
+        m <- b1 m + (1-b1) g;  v <- b2 v + (1-b2) g^2;
+        theta <- theta - lr * (m / (1-b1^t)) / (sqrt(v / (1-b2^t)) + eps).
+    Returns the new (theta, m, v)."""
+    theta = np.asarray(theta, dtype=np.float64)
+    g = np.asarray(grad, dtype=np.float64)
+    m = beta1 * np.asarray(m, dtype=np.float64) + (1.0 - beta1) * g
+    v = beta2 * np.asarray(v, dtype=np.float64) + (1.0 - beta2) * g * g
+    m_hat = m / (1.0 - beta1 ** step)
+    v_hat = v / (1.0 - beta2 ** step)
+    return theta - lr * m_hat / (np.sqrt(v_hat) + eps), m, v

@@ -29,10 +29,10 @@ EXPORTS = ("sapo_pack_rollouts", "sapo_group_advantages", "sapo_policy_loss_fwd"
            "sapo_policy_loss_bwd", "sapo_workspace_bytes", "sapo_workspace_bytes_min",
            "sapo_status_string", "sapo_timing_enable", "sapo_timing_read", "sapo_launch_count",
            "sapo_policy_loss_fwd_static", "sapo_policy_loss_bwd_active", "sapo_select_external",
-           "sapo_select_workspace_bytes")
+           "sapo_select_workspace_bytes", "sapo_adam_step")
 STATIC_SCRATCH_BYTES = 4 * 1024 * 1024
 KERNEL_NAMES = ("pack_scan", "pack_copy", "group_adv", "split_bf16", "fwd_gemm", "loss_tail",
-                "loss_final", "bwd_dz", "bwd_dh", "bwd_dw", "streamk_fixup", "compact", "select")
+                "loss_final", "bwd_dz", "bwd_dh", "bwd_dw", "streamk_fixup", "compact", "select", "adam")
 
 
 class RolloutBufC(C.Structure):
@@ -97,6 +97,8 @@ def load() -> C.CDLL:
     lib.sapo_select_external.argtypes = [vp, vp, i32, i32, C.c_uint64, vp, vp, vp, vp, sz, vp]
     lib.sapo_select_workspace_bytes.restype = sz
     lib.sapo_select_workspace_bytes.argtypes = [i32]
+    lib.sapo_adam_step.restype = C.c_int
+    lib.sapo_adam_step.argtypes = [vp, vp, vp, vp, vp, i64, i32, i64, i32, f32, f32, f32, f32, vp]
     lib.sapo_workspace_bytes.restype = sz
     lib.sapo_workspace_bytes.argtypes = [i32, i64, i32, i32, i32]
     lib.sapo_workspace_bytes_min.restype = sz
@@ -333,3 +335,15 @@ def sapo_select_external(rewards: torch.Tensor, group_offsets: torch.Tensor, J: 
                                      _p(selected), _p(n_sel), _p(n_cand), _p(ws), ws.numel() * 8, _stream())
     _check(rc, "sapo_select_external")
     return selected, n_sel, n_cand
+
+
+def sapo_adam_step(master: torch.Tensor, m: torch.Tensor, v: torch.Tensor, grad: torch.Tensor,
+                   w_bf16: Optional[torch.Tensor], step: int, lr: float = 1e-3, beta1: float = 0.9,
+                   beta2: float = 0.999, eps: float = 1e-8) -> None:
+    """One Adam step on a 2-D fp32 master weight; rewrites its bf16 copy if given."""
+    _require_cuda()
+    rows, cols = int(master.shape[0]), int(master.shape[1])
+    ld = int(w_bf16.stride(0)) if w_bf16 is not None else cols
+    rc = load().sapo_adam_step(_p(master), _p(m), _p(v), _p(grad), _p(w_bf16), rows, cols, ld, int(step),
+                               lr, beta1, beta2, eps, _stream())
+    _check(rc, "sapo_adam_step")

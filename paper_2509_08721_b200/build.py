@@ -10,7 +10,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libsapo_b200.so")
-SOURCES = ["runtime.cu", "pack.cu", "advantages.cu", "select.cu", "lmhead.cu"]
+SOURCES = ["runtime.cu", "pack.cu", "advantages.cu", "select.cu", "adam.cu", "lmhead.cu"]
 FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
          "--shared", "-Xcompiler", "-fPIC", "-Xcompiler", "-fvisibility=default"]
 

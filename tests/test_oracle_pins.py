@@ -393,6 +393,24 @@ def test_select_external_filters_zero_advantage_and_samples_uniformly():
     assert np.all(np.abs(hits[cand] - n_seeds * p) < 5 * sd) and hits[const].sum() == 0
 
 
+def test_adam_step_matches_the_library_optimizer():
+    import torch
+    rng = np.random.default_rng(2)
+    theta0 = rng.normal(size=(7, 5))
+    p = torch.nn.Parameter(torch.tensor(theta0, dtype=torch.float64))
+    opt = torch.optim.Adam([p], lr=1e-3)                     # library defaults: 0.9, 0.999, 1e-8
+    theta, m, v = theta0.copy(), np.zeros_like(theta0), np.zeros_like(theta0)
+    for t in range(1, 4):
+        g = rng.normal(size=theta0.shape) * (10.0 ** -t)
+        p.grad = torch.tensor(g, dtype=torch.float64)
+        opt.step()
+        theta, m, v = orc.adam_step(theta, g, m, v, t)
+        assert np.allclose(theta, p.detach().numpy(), rtol=1e-12, atol=1e-15)
+    # first step of Adam moves every weight by lr against the sign of its gradient
+    th1, _, _ = orc.adam_step(np.zeros(4), np.array([3.0, -2.0, 1e-3, -5e2]), np.zeros(4), np.zeros(4), 1)
+    assert np.allclose(th1, [-1e-3, 1e-3, -1e-3, 1e-3], rtol=1e-4)
+
+
 # ------------------------------------------------------------------ the input generator
 def test_generator_recipes_have_the_stated_shapes():
     r = gen.config(1)
