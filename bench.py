@@ -49,7 +49,7 @@ class ClockSampler:
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", f"--id={index}", f"--query-gpu={self.QUERY}",
-                 "--format=csv,noheader,nounits", "-lms", "100"],
+                 "--format=csv,noheader,nounits", "-lms", "25"],
                 stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
         except Exception:
             self.proc = None
@@ -281,10 +281,16 @@ def run_ours(args):
     dev_step = lambda: scorer.step(local, ext, sel, T, S)
     host_step = lambda: scorer.step_from_host(T, S)
 
-    sampler = ClockSampler(local_rank) if rank == 0 else None
     for _ in range(args.warmup):
         dev_step()
     torch.cuda.synchronize()
+    sampler = ClockSampler(local_rank) if rank == 0 else None
+    if sampler is not None:
+        # nvidia-smi needs a moment to start: keep the GPU under the same load until it reports
+        t_end = time.perf_counter() + 0.5
+        while time.perf_counter() < t_end:
+            dev_step()
+        torch.cuda.synchronize()
     B.sapo_timing_enable(True)
     launches0 = B.sapo_launch_count()
     ms_total = timed(dev_step, args.steps)
@@ -375,7 +381,7 @@ def run_ours(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", type=int, default=2, help="1..5; 2 is the Qwen2.5-0.5B-shaped head")

@@ -282,7 +282,7 @@ int sapo_policy_loss_fwd_static(const void* hidden, const void* W_head, int32_t 
 /* Optional per-kernel timing for benchmarks (no counterpart in the paper).  While enabled,
  * every kernel launch of the library is bracketed by two CUDA events recorded on the call's
  * stream.  sapo_timing_read waits for the recorded events, writes the summed milliseconds and
- * the number of launches per kernel id (arrays of SAPO_K_COUNT) and forgets them; at most 512
+ * the number of launches per kernel id (arrays of SAPO_K_COUNT) and forgets them; at most 16384
  * launches are kept between reads.  The events are created on the first enable.  Not thread-safe.
  * sapo_launch_count returns how many kernels the library has launched in this process. */
 #define SAPO_K_PACK_SCAN  0

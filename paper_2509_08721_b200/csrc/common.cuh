@@ -32,7 +32,7 @@ inline int sm_count() {
 // Optional per-kernel timing and launch counting (see sapo_timing_* in sapo.h).
 // A KernelScope brackets one kernel launch with two CUDA events when timing is on.
 struct KernelTimer {
-  static constexpr int MAX_PAIRS = 512;
+  static constexpr int MAX_PAIRS = 16384;
   bool enabled = false;
   bool created = false;
   int n = 0;
