@@ -237,6 +237,11 @@ def run_ours(args):
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
     peaks = load_peaks()
+    if args.hbm_only:            # only the bandwidth-bound kernels, on their scaled case (for profiling)
+        B.load()
+        if rank == 0:
+            print(json.dumps({"hbm_kernels": hbm_kernels(torch, B, peaks)}))
+        return 0
 
     batch, recipe = build_batch(args.workload, replicas.rank_seed(args.workload, rank), args.length_div)
     T, S, H, V = batch.T, batch.S, batch.H, batch.V
@@ -388,6 +393,8 @@ def main():
     ap.add_argument("--ref-tokens", type=int, default=None,
                     help="tokens of the bounded oracle sample (default 2048 for cpu_baseline, 512 per reference step)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--hbm-only", action="store_true",
+                    help="run only the scaled pack / advantages / Adam bandwidth measurement")
     ap.add_argument("--backward", default="dense", choices=["dense", "active"],
                     help="active: contract only the tokens whose gradient factor is non-zero")
     ap.add_argument("--length-div", type=int, default=1,

@@ -48,12 +48,13 @@ struct Sched {
   int32_t tile_n;     // columns per tile (a multiple of 32, at most 256)
   int32_t n_cover;    // columns the epilogue visits (>= N; the dz panel is padded to 64)
   int32_t panel_nvt;  // 64-column tiles per token block of the dz panel (tiled A operands)
-  // Units [0, dp_units) are dealt whole, round-robin, to the pairs.  The sk_tiles units after
-  // them (fewer than there are pairs) are cut along K instead: their sk_tiles * num_k_blocks
-  // stage iterations are shared out evenly, sk_ipp consecutive ones per pair, so the last wave
-  // is as full as the others.  A pair that gets only part of a tile's K range leaves a partial
-  // accumulator in scratch; a small second kernel adds the parts up.
-  int32_t dp_units, sk_tiles, sk_ipp;
+  // Units [0, dp_units) are dealt whole, round-robin, to the pairs.  If the sk_tiles units
+  // after them would fill less than half of a last wave, each of them is cut along K into
+  // sk_parts equal ranges (sk_tiles * sk_parts <= pairs), one range per pair: the last wave is
+  // shorter, and pairs that work on the same K range still share the B tiles they stream
+  // through L2.  A range leaves a partial accumulator in scratch; a small second kernel adds
+  // the parts of each tile in order.
+  int32_t dp_units, sk_tiles, sk_parts;
   int32_t k_split_ok; // the epilogue has scratch for K-split parts
   // A size only the device knows (the number of active tokens after compaction), read by
   // every CTA at start-up: dyn_dim 1 = it is M (rows), 2 = it is K (contraction length).
@@ -63,15 +64,18 @@ struct Sched {
   int32_t stats_id;   // row of the wait-cycle counters this launch adds to (instrumented builds)
 };
 
-// Cut a ragged last wave of long-K tiles along K over all the pairs (see Sched).
+// Decide whether (and how finely) to cut a thin last wave of long-K tiles along K (see Sched).
 __host__ __device__ inline void split_last_wave(Sched& s, int pairs) {
-  s.dp_units = s.num_units; s.sk_tiles = 0; s.sk_ipp = 1;
+  s.dp_units = s.num_units; s.sk_tiles = 0; s.sk_parts = 1;
   if (!s.k_split_ok || pairs <= 0) return;
   const int rem = s.num_units % pairs;
-  if (rem != 0 && s.num_k_blocks >= 8 && s.n_per_unit == 1) {
+  if (rem != 0 && 2 * rem <= pairs && s.n_per_unit == 1) {
+    int parts = pairs / rem;
+    if (parts > 8) parts = 8;
+    if (s.num_k_blocks / parts < 16) return;      // keep every range long enough to be worth a pipeline fill
     s.dp_units = s.num_units - rem;
     s.sk_tiles = rem;
-    s.sk_ipp = (int32_t)(((int64_t)rem * s.num_k_blocks + pairs - 1) / pairs);
+    s.sk_parts = parts;
   }
 }
 
@@ -103,14 +107,9 @@ __device__ __forceinline__ void decode_unit(const Sched& s, int unit, int& mb, i
 // The work of one CTA pair, in order: its whole units, then its share of the K-split units.
 // Every role of both CTAs walks the same list.
 struct WorkList {
-  const Sched& s; int pair, n_pairs, i; long long it, it_end;
+  const Sched& s; int pair, n_pairs, i; bool tail_done;
   __device__ __forceinline__ WorkList(const Sched& s_, int pair_, int n_pairs_)
-      : s(s_), pair(pair_), n_pairs(n_pairs_), i(0) {
-    const long long total = (long long)s.sk_tiles * s.num_k_blocks;
-    it = (long long)pair * s.sk_ipp;
-    it_end = it + s.sk_ipp < total ? it + s.sk_ipp : total;
-    if (it > it_end) it = it_end;
-  }
+      : s(s_), pair(pair_), n_pairs(n_pairs_), i(0), tail_done(false) {}
   // slot: -1 = the tile's whole K range (normal epilogue); otherwise the scratch slot of the part
   __device__ __forceinline__ bool next(int& pmb, int& un, int& n_begin, int& n_end, int& kb0, int& kb1,
                                        int& slot) {
@@ -121,14 +120,13 @@ struct WorkList {
       kb0 = 0; kb1 = s.num_k_blocks; slot = -1;
       return true;
     }
-    if (it < it_end) {
-      const int t = (int)(it / s.num_k_blocks);
+    if (!tail_done && pair < s.sk_tiles * s.sk_parts) {
+      tail_done = true;
+      const int t = pair / s.sk_parts, j = pair - t * s.sk_parts;
       decode_unit(s, s.dp_units + t, pmb, un, n_begin, n_end);
-      kb0 = (int)(it - (long long)t * s.num_k_blocks);
-      const long long left = it_end - it;
-      kb1 = (long long)(s.num_k_blocks - kb0) <= left ? s.num_k_blocks : kb0 + (int)left;
-      it += kb1 - kb0;
-      slot = (kb0 == 0 && kb1 == s.num_k_blocks) ? -1 : 2 * pair + (kb0 == 0 ? 1 : 0);
+      kb0 = (int)((long long)s.num_k_blocks * j / s.sk_parts);
+      kb1 = (int)((long long)s.num_k_blocks * (j + 1) / s.sk_parts);
+      slot = s.sk_parts > 1 ? pair : -1;
       return true;
     }
     return false;
@@ -334,10 +332,7 @@ streamk_fixup_kernel(const Sched s_arg, const StoreEpi::Params p_arg, int pairs)
   const int t = blockIdx.x >> 5;                 // K-split tile
   if (t >= s.sk_tiles) return;
   const int row_begin = (blockIdx.x & 31) * 8;   // 8 of its 256 rows per block
-  const long long first_it = (long long)t * s.num_k_blocks;
-  const int p_first = (int)(first_it / s.sk_ipp);
-  const int p_last = (int)((first_it + s.num_k_blocks - 1) / s.sk_ipp);
-  if (p_first == p_last) return;                 // one pair had the whole tile and stored it itself
+  if (s.sk_parts <= 1) return;                   // whole tiles were stored by their pair
   int pmb, un, n_begin, n_end;
   decode_unit(s, s.dp_units + t, pmb, un, n_begin, n_end);
   const int n0 = n_begin * s.tile_n;
@@ -348,8 +343,8 @@ streamk_fixup_kernel(const Sched s_arg, const StoreEpi::Params p_arg, int pairs)
     if (row >= p.M) break;
     if (p.row_map != nullptr) row = p.row_map[row];
     const size_t off = (size_t)rr * BN + col;
-    float sum = p.partials[(size_t)(2 * p_first + 1) * PARTIAL_FLOATS + off];
-    for (int q = p_first + 1; q <= p_last; ++q) sum += p.partials[(size_t)(2 * q) * PARTIAL_FLOATS + off];
+    float sum = 0.f;
+    for (int j = 0; j < s.sk_parts; ++j) sum += p.partials[(size_t)(t * s.sk_parts + j) * PARTIAL_FLOATS + off];
     float* dst = p.C + row * p.ldc + n0 + col;
     *dst = p.accumulate ? *dst + sum : sum;
   }
@@ -752,7 +747,7 @@ static Sched make_sched(int64_t M, int64_t N, int64_t K, int n_splits, bool m_fa
   s.N = (int32_t)N;
   s.n_cover = (int32_t)N;
   s.panel_nvt = 0;
-  s.dp_units = s.num_units; s.sk_tiles = 0; s.sk_ipp = 1;
+  s.dp_units = s.num_units; s.sk_tiles = 0; s.sk_parts = 1;
   s.k_split_ok = 0; s.dyn_count = nullptr; s.dyn_dim = 0; s.skip_if_empty = 0;
   return s;
 }

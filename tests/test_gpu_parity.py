@@ -180,6 +180,8 @@ SHAPES = [
     ("bf16_single_tokens", small_recipe(H=128, V=300, Q=4, length_law=("fixed", 1)), None),
     ("bf16_one_group", small_recipe(H=64, V=520, Q=1, I=3, J=0), None),
     ("fp32_small", small_recipe(dtype=gen.DTYPE_F32, H=40, V=333, Q=3), None),
+    # two dH tiles with a long vocabulary contraction: the thin last wave is cut along K
+    ("bf16_k_split", small_recipe(H=128, V=20000, Q=2, length_law=("uniform", 50, 90)), None),
 ]
 
 
