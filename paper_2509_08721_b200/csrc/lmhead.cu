@@ -44,6 +44,8 @@ constexpr float LN2 = 0.6931471805599453f;
 struct Sched {
   int32_t num_m_blocks, num_n_blocks, n_per_unit, units_per_m, num_units, num_k_blocks;
   int32_t m_fastest;  // 1: neighbouring pairs share the B tile; 0: they share the A tile
+  int32_t group_m;    // m_fastest only: row blocks per group; a group's A rows are meant to stay in L2
+                      // while the schedule walks all n-units for it
   int32_t N;          // true extent of the n dimension
   int32_t tile_n;     // columns per tile (a multiple of 32, at most 256)
   int32_t n_cover;    // columns the epilogue visits (>= N; the dz panel is padded to 64)
@@ -98,7 +100,14 @@ constexpr int MAX_PAIRS_SCRATCH = 96;          // CTA pairs the K-split scratch 
 
 __device__ __forceinline__ void decode_unit(const Sched& s, int unit, int& mb, int& un,
                                             int& n_begin, int& n_end) {
-  if (s.m_fastest) { un = unit / s.num_m_blocks; mb = unit - un * s.num_m_blocks; }
+  if (s.m_fastest) {
+    // groups of group_m row blocks; inside a group the row block runs fastest, then the n-unit
+    const int per_group = s.group_m * s.units_per_m;
+    const int g = unit / per_group, r = unit - g * per_group;
+    const int rows_here = min(s.group_m, s.num_m_blocks - g * s.group_m);
+    un = r / rows_here;
+    mb = g * s.group_m + (r - un * rows_here);
+  }
   else             { mb = unit / s.units_per_m;  un = unit - mb * s.units_per_m; }
   n_begin = un * s.n_per_unit;
   n_end = min(n_begin + s.n_per_unit, s.num_n_blocks);
@@ -744,6 +753,12 @@ static Sched make_sched(int64_t M, int64_t N, int64_t K, int n_splits, bool m_fa
   s.num_units = s.num_m_blocks * s.units_per_m;
   s.num_k_blocks = (int32_t)ceil_div<int64_t>(K, BK);
   s.m_fastest = m_fastest ? 1 : 0;
+  // row blocks whose A rows (256 x K bf16 each) fit in about 48 MB of the 126 MB L2
+  {
+    const int64_t fit = (48ll << 20) / (PAIR_M * (int64_t)K * 2);
+    s.group_m = (int32_t)(fit < 1 ? 1 : (fit > s.num_m_blocks ? s.num_m_blocks : fit));
+    if (s.group_m < 1) s.group_m = 1;
+  }
   s.N = (int32_t)N;
   s.n_cover = (int32_t)N;
   s.panel_nvt = 0;
@@ -754,7 +769,7 @@ static Sched make_sched(int64_t M, int64_t N, int64_t K, int n_splits, bool m_fa
 
 // Number of vocab splits of the forward pass: enough units to keep every CTA pair busy when
 // there are few token blocks, never more than there are vocab tiles.
-static int fwd_splits(int64_t T, int32_t V, int sms) {
+static int fwd_splits(int64_t T, int32_t V, int64_t K, int sms) {
   const int64_t pairs = sms / 2 > 0 ? sms / 2 : 1;
   const int64_t mb = ceil_div<int64_t>(T, PAIR_M);
   const int64_t nb = ceil_div<int64_t>(V, BN);
@@ -765,6 +780,13 @@ static int fwd_splits(int64_t T, int32_t V, int sms) {
     const double eff = (double)units / (double)(ceil_div<int64_t>(units, pairs) * pairs);
     if (eff > best_eff + 1e-9) { best_eff = eff; best = sp; }
     if (units >= 8 * pairs) break;
+  }
+  // a wave of pairs should not span more row blocks than stay resident in L2 (see Sched::group_m)
+  const int64_t fit = (48ll << 20) / (PAIR_M * (int64_t)K * 2);
+  const int64_t group = fit < 1 ? 1 : fit;
+  if (group < pairs && group < mb) {
+    const int64_t want = ceil_div(pairs, group);
+    if (best < want) best = want < nb ? want : nb;
   }
   const int64_t per = ceil_div(nb, best);
   return (int)ceil_div(nb, per);
@@ -846,7 +868,7 @@ static int64_t padded_vocab(int32_t V) { return round_up<int64_t>(V, 128); }
 struct FwdLayout { size_t partials, a_split, b_split, total; int n_splits; };
 static FwdLayout fwd_layout(int64_t T, int32_t H, int32_t V, int32_t dtype, int sms) {
   FwdLayout L{};
-  L.n_splits = fwd_splits(T, V, sms);
+  L.n_splits = fwd_splits(T, V, dtype == SAPO_DTYPE_F32 ? 3 * (int64_t)H : (int64_t)H, sms);
   size_t off = 0;
   L.partials = off; off += round_up<size_t>((size_t)3 * 2 * L.n_splits * T * sizeof(float), 256);
   if (dtype == SAPO_DTYPE_F32) {
