@@ -329,8 +329,8 @@ def run_ours(args):
         # DRAM bytes per launch from the ncu capture of a small case of the same kernels
         # (profiles/umma_gemm_kernels_workload2_lengths_div4.md): fixed part + bytes per token.
         # Only valid for hidden 896 / vocab 151936, the shape that capture ran at.
-        ncu_traffic = {"fwd_gemm": (0.272e9, 13.1e3), "bwd_dz": (0.272e9, 299.6e3),
-                       "bwd_dh": (0.272e9, 311.8e3), "bwd_dw": (0.519e9, 335.9e3)}
+        ncu_traffic = {"fwd_gemm": (0.272e9, 12.4e3), "bwd_dz": (0.272e9, 299.6e3),
+                       "bwd_dh": (0.272e9, 310.8e3), "bwd_dw": (0.515e9, 332.3e3)}
         traffic = None
         if (H, V) == (896, 151936):
             fixed, per_token = ncu_traffic[top]
