@@ -50,12 +50,13 @@ struct Sched {
   int32_t tile_n;     // columns per tile (a multiple of 32, at most 256)
   int32_t n_cover;    // columns the epilogue visits (>= N; the dz panel is padded to 64)
   int32_t panel_nvt;  // 64-column tiles per token block of the dz panel (tiled A operands)
-  // Units [0, dp_units) are dealt whole, round-robin, to the pairs.  If the sk_tiles units
-  // after them would fill less than half of a last wave, each of them is cut along K into
-  // sk_parts equal ranges (sk_tiles * sk_parts <= pairs), one range per pair: the last wave is
-  // shorter, and pairs that work on the same K range still share the B tiles they stream
-  // through L2.  A range leaves a partial accumulator in scratch; a small second kernel adds
-  // the parts of each tile in order.
+  // Units [0, dp_units) are dealt whole, round-robin, to the pairs.  The sk_tiles units after
+  // them would leave a last wave partly empty; when cutting helps, each of them is cut along K
+  // into sk_parts equal ranges and the sk_tiles * sk_parts parts are dealt round-robin, K range
+  // slowest: the last wave gets shorter, and pairs that work at the same time are on the same
+  // K range of different tiles, so they still share the B tiles they stream through L2.  A part
+  // leaves a partial accumulator in scratch; a small second kernel adds the parts of each tile
+  // in order.
   int32_t dp_units, sk_tiles, sk_parts;
   int32_t k_split_ok; // the epilogue has scratch for K-split parts
   // A size only the device knows (the number of active tokens after compaction), read by
@@ -66,19 +67,31 @@ struct Sched {
   int32_t stats_id;   // row of the wait-cycle counters this launch adds to (instrumented builds)
 };
 
-// Decide whether (and how finely) to cut a thin last wave of long-K tiles along K (see Sched).
+constexpr int PARTIAL_FLOATS = PAIR_M * BN;   // one partial accumulator tile: 256 x 256 fp32
+constexpr int MAX_PAIRS_SCRATCH = 96;          // CTA pairs a launch may use (a B200 has 74)
+constexpr int MAX_PARTS_SCRATCH = 3 * MAX_PAIRS_SCRATCH;   // K-split parts the scratch holds
+
+// Decide whether (and how finely) to cut the tiles of a ragged last wave along K (see Sched).
+// With `rem` tiles left over and s parts per tile the tail takes ceil(rem s / pairs) / s of a
+// tile's time instead of 1; every part also pays a pipeline fill and an exposed epilogue,
+// counted here as 2 % of a tile.
 __host__ __device__ inline void split_last_wave(Sched& s, int pairs) {
   s.dp_units = s.num_units; s.sk_tiles = 0; s.sk_parts = 1;
-  if (!s.k_split_ok || pairs <= 0) return;
+  if (!s.k_split_ok || pairs <= 0 || s.n_per_unit != 1) return;
   const int rem = s.num_units % pairs;
-  if (rem != 0 && 2 * rem <= pairs && s.n_per_unit == 1) {
-    int parts = pairs / rem;
-    if (parts > 8) parts = 8;
-    if (s.num_k_blocks / parts < 16) return;      // keep every range long enough to be worth a pipeline fill
-    s.dp_units = s.num_units - rem;
-    s.sk_tiles = rem;
-    s.sk_parts = parts;
+  if (rem == 0) return;
+  int best = 1; float best_cost = 1.f;
+  for (int parts = 2; parts <= 8; ++parts) {
+    if (s.num_k_blocks / parts < 16) break;       // keep every range long enough to be worth a pipeline fill
+    if (rem * parts > MAX_PARTS_SCRATCH) break;
+    const int rounds = (rem * parts + pairs - 1) / pairs;
+    const float cost = (float)rounds / (float)parts + 0.02f * (float)rounds;
+    if (cost < best_cost - 0.05f) { best_cost = cost; best = parts; }
   }
+  if (best == 1) return;
+  s.dp_units = s.num_units - rem;
+  s.sk_tiles = rem;
+  s.sk_parts = best;
 }
 
 // Fill in what depends on a device-side size; every CTA (and the fix-up kernel) does the same.
@@ -95,9 +108,6 @@ __device__ __forceinline__ void finalize_sched(Sched& s, int pairs) {
   split_last_wave(s, pairs);
 }
 
-constexpr int PARTIAL_FLOATS = PAIR_M * BN;   // one partial accumulator tile: 256 x 256 fp32
-constexpr int MAX_PAIRS_SCRATCH = 96;          // CTA pairs the K-split scratch is sized for (a B200 has 74)
-
 __device__ __forceinline__ void decode_unit(const Sched& s, int unit, int& mb, int& un,
                                             int& n_begin, int& n_end) {
   if (s.m_fastest) {
@@ -113,12 +123,12 @@ __device__ __forceinline__ void decode_unit(const Sched& s, int unit, int& mb, i
   n_end = min(n_begin + s.n_per_unit, s.num_n_blocks);
 }
 
-// The work of one CTA pair, in order: its whole units, then its share of the K-split units.
+// The work of one CTA pair, in order: its whole units, then its share of the K-split parts.
 // Every role of both CTAs walks the same list.
 struct WorkList {
-  const Sched& s; int pair, n_pairs, i; bool tail_done;
+  const Sched& s; int pair, n_pairs, i, tail_i;
   __device__ __forceinline__ WorkList(const Sched& s_, int pair_, int n_pairs_)
-      : s(s_), pair(pair_), n_pairs(n_pairs_), i(0), tail_done(false) {}
+      : s(s_), pair(pair_), n_pairs(n_pairs_), i(0), tail_i(0) {}
   // slot: -1 = the tile's whole K range (normal epilogue); otherwise the scratch slot of the part
   __device__ __forceinline__ bool next(int& pmb, int& un, int& n_begin, int& n_end, int& kb0, int& kb1,
                                        int& slot) {
@@ -129,13 +139,14 @@ struct WorkList {
       kb0 = 0; kb1 = s.num_k_blocks; slot = -1;
       return true;
     }
-    if (!tail_done && pair < s.sk_tiles * s.sk_parts) {
-      tail_done = true;
-      const int t = pair / s.sk_parts, j = pair - t * s.sk_parts;
+    const int part = pair + tail_i * n_pairs;       // part j of tile t has index j * sk_tiles + t
+    if (part < s.sk_tiles * s.sk_parts) {
+      ++tail_i;
+      const int j = part / s.sk_tiles, t = part - j * s.sk_tiles;
       decode_unit(s, s.dp_units + t, pmb, un, n_begin, n_end);
       kb0 = (int)((long long)s.num_k_blocks * j / s.sk_parts);
       kb1 = (int)((long long)s.num_k_blocks * (j + 1) / s.sk_parts);
-      slot = s.sk_parts > 1 ? pair : -1;
+      slot = part;
       return true;
     }
     return false;
@@ -353,7 +364,7 @@ streamk_fixup_kernel(const Sched s_arg, const StoreEpi::Params p_arg, int pairs)
     if (p.row_map != nullptr) row = p.row_map[row];
     const size_t off = (size_t)rr * BN + col;
     float sum = 0.f;
-    for (int j = 0; j < s.sk_parts; ++j) sum += p.partials[(size_t)(t * s.sk_parts + j) * PARTIAL_FLOATS + off];
+    for (int j = 0; j < s.sk_parts; ++j) sum += p.partials[(size_t)(j * s.sk_tiles + t) * PARTIAL_FLOATS + off];
     float* dst = p.C + row * p.ldc + n0 + col;
     *dst = p.accumulate ? *dst + sum : sum;
   }
@@ -887,7 +898,7 @@ static BwdLayout bwd_layout(int64_t T, int32_t H, int32_t V, int32_t dtype) {
     L.a_hi = off; off += round_up<size_t>((size_t)T * H * 2, 256);
     L.b_hi = off; off += round_up<size_t>((size_t)V * H * 2, 256);
   }
-  L.partials = off; off += (size_t)2 * MAX_PAIRS_SCRATCH * PARTIAL_FLOATS * sizeof(float);
+  L.partials = off; off += (size_t)MAX_PARTS_SCRATCH * PARTIAL_FLOATS * sizeof(float);
   L.panel = off; L.fixed = off;
   L.bytes_per_row = (size_t)padded_vocab(V) * 2;
   return L;

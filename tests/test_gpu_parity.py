@@ -182,6 +182,9 @@ SHAPES = [
     ("fp32_small", small_recipe(dtype=gen.DTYPE_F32, H=40, V=333, Q=3), None),
     # two dH tiles with a long vocabulary contraction: the thin last wave is cut along K
     ("bf16_k_split", small_recipe(H=128, V=20000, Q=2, length_law=("uniform", 50, 90)), None),
+    # about 48 dH tiles (fewer than CTA pairs, more than half of them), each cut in three along
+    # the vocabulary: more parts than pairs, so pairs take several parts in turn
+    ("bf16_k_split_rounds", small_recipe(H=512, V=8192, Q=8, length_law=("uniform", 150, 230)), None),
 ]
 
 
