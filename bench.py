@@ -247,7 +247,7 @@ def run_ours(args):
     T, S, H, V = batch.T, batch.S, batch.H, batch.V
     W = _to_dev(batch.W, "cuda")
     scorer = PolicyScorer(W, T, S, recipe.Q, eps_low=batch.eps_low, eps_high=batch.eps_high,
-                          active_backward=args.backward == "active")
+                          backward=args.backward)
 
     # old log-probs = current + noise: "current" is one forward pass of the library itself
     # over the packed tokens (set-up, untimed); the noise comes from the seeded generator.
@@ -318,13 +318,14 @@ def run_ours(args):
     if rank == 0:
         # roofline of the dominant kernel (largest share of the timed region)
         t_act = int(scorer.n_active.item()) if args.backward == "active" else T
-        gemm = {k: per_kernel[k] for k in ("fwd_gemm", "bwd_dz", "bwd_dh", "bwd_dw")}
+        gemm = {k: per_kernel[k] for k in ("fwd_gemm", "fwd_exp", "bwd_dz", "bwd_dh", "bwd_dw")
+                if per_kernel[k]["launches"]}
         top = max(gemm, key=lambda k: gemm[k]["ms"])
         n_top = max(1, gemm[top]["launches"])
         ms_top = gemm[top]["ms"] / n_top
         # launches per step of that kernel (the backward runs once per dz panel chunk)
         per_step = n_top / args.steps
-        flops_each = 2.0 * (T if top == "fwd_gemm" else t_act) * V * H
+        flops_each = 2.0 * (T if top in ("fwd_gemm", "fwd_exp") else t_act) * V * H
         achieved = flops_each / per_step / (ms_top / 1e3) / 1e12
         # DRAM bytes per launch from the ncu capture of a small case of the same kernels
         # (profiles/umma_gemm_kernels_workload2_lengths_div4.md): fixed part + bytes per token.
@@ -332,7 +333,7 @@ def run_ours(args):
         ncu_traffic = {"fwd_gemm": (0.272e9, 12.4e3), "bwd_dz": (0.272e9, 299.6e3),
                        "bwd_dh": (0.272e9, 310.8e3), "bwd_dw": (0.515e9, 332.3e3)}
         traffic = None
-        if (H, V) == (896, 151936):
+        if (H, V) == (896, 151936) and top in ncu_traffic:
             fixed, per_token = ncu_traffic[top]
             traffic = fixed + per_token * T / per_step
         peak = peaks["bf16_tflops_sustained"]      # the kernel is timed inside a long step
@@ -341,7 +342,8 @@ def run_ours(args):
                    for k, v in per_kernel.items() if v["launches"]}
         gemm_ms = sum(gemm[k]["ms"] for k in gemm) / args.steps
         f_alg = 2.0 * T * V * H + 4.0 * t_act * V * H
-        f_exec = 2.0 * T * V * H + 6.0 * t_act * V * H
+        # the separate backward recomputes the logits (one more contraction); the fused call does not
+        f_exec = f_alg if args.backward == "fused" else 2.0 * T * V * H + 6.0 * t_act * V * H
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
@@ -395,8 +397,10 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--hbm-only", action="store_true",
                     help="run only the scaled pack / advantages / Adam bandwidth measurement")
-    ap.add_argument("--backward", default="dense", choices=["dense", "active"],
-                    help="active: contract only the tokens whose gradient factor is non-zero")
+    ap.add_argument("--backward", default="dense", choices=["dense", "active", "fused"],
+                    help="dense: forward call, then the backward call that recomputes the logits; "
+                         "active: the same over the tokens whose gradient factor is non-zero only; "
+                         "fused: one call that passes over the logits once (bf16 workloads)")
     ap.add_argument("--length-div", type=int, default=1,
                     help="divide every completion length (a small case of the same kernels for profiling)")
     args = ap.parse_args()

@@ -56,6 +56,9 @@ extern "C" {
 #define SAPO_ST_BAD_TOKEN_ID     0x10  /* ids[t] outside [0, V): token scored as masked       */
 #define SAPO_ST_WAIT_TIMEOUT     0x20  /* a bounded in-kernel wait ran out; results invalid   */
 #define SAPO_ST_NONFINITE_REWARD 0x40  /* a reward is NaN or infinite                         */
+#define SAPO_ST_EXP_RANGE        0x80  /* fused call: old_logp[t] is so far from the current
+                                          log-prob that exp(z - c_t) left the safe range; the
+                                          token is scored as masked: use the separate calls   */
 
 /* element types of hidden / W_head */
 #define SAPO_DTYPE_BF16 0
@@ -65,6 +68,7 @@ extern "C" {
 #define SAPO_WS_FWD 0
 #define SAPO_WS_BWD 1
 #define SAPO_WS_BWD_ACTIVE 2
+#define SAPO_WS_FUSED 3
 
 /* A rollout store: n_rollouts completions laid end to end (Section 3.1: a node's answers
  * to its questions; Section 3.2: the tuples other nodes broadcast).
@@ -220,6 +224,39 @@ int sapo_policy_loss_bwd_active(const void* hidden, const void* W_head, int32_t 
                                 void* workspace, size_t workspace_bytes,
                                 int32_t* status, void* stream);
 
+/* Loss (Section 3.2 + Section 4.2) and both gradients (Algorithm 1 "Policy update") in ONE call
+ * that passes over the logits once.  Same definitions and outputs as sapo_policy_loss_fwd followed
+ * by sapo_policy_loss_bwd; what changes is how the softmax is carried from the forward to the
+ * backward contraction.  With a per-token reference
+ *   c_t = z[t, ids[t]] - old_logp[t]          (one dot product per token, computed first)
+ * — equal to lse[t] if the policy has not moved since old_logp was taken, and off by
+ * log ratio[t] otherwise — the forward epilogue forms e[t,v] = exp(z[t,v] - c_t), adds it up per
+ * token in fp32 (lse[t] = c_t + log sum_v e[t,v]; no running maximum is needed) and keeps e,
+ * rounded to bf16, in a panel inside `workspace` (token chunks x vocab padded to 128, 16 KB tiles
+ * of 128 tokens x 64 vocab entries).  Then, with sum_t = sum_v e[t,v] and a_t = -gscale[t] / sum_t,
+ *   dz[t,v] = gscale[t] ([v == ids[t]] - e[t,v] / sum_t) = a_t e'[t,v],  e' = e - [v == ids[t]] sum_t,
+ * so after patching one panel entry per token
+ *   dhidden[t,:] = a_t sum_v e'[t,v] W_head[v,:]     (row scale in the epilogue)
+ *   dW_head[v,:] = sum_t e'[t,v] (a_t hidden[t,:])   (scaled bf16 copy of hidden as operand)
+ * are two tensor-core contractions over the panel: 6 T V H flops instead of the 8 T V H of the
+ * separate calls, which recompute the logits.  The price is the range of e: if old_logp[t] is so
+ * stale that |log ratio| approaches 69 (e reaches 2^100 or the sum drops below 2^-100), the token
+ * is scored as masked (surr = gscale = 0) and SAPO_ST_EXP_RANGE is set; such batches need the
+ * separate calls.  bf16 operands only (SAPO_DTYPE_F32 returns SAPO_ERR_UNSUPPORTED_SHAPE).
+ * Arguments as in the two separate calls.  workspace: sapo_workspace_bytes(SAPO_WS_FUSED, ...)
+ * is the preferred size (a panel of up to 32768 tokens); any size down to
+ * sapo_workspace_bytes_min(SAPO_WS_FUSED, ...) works, the batch is then processed in token
+ * chunks and dW_head accumulated over them.  seq_surr may be NULL (then S <= T is required). */
+int sapo_policy_loss_fwd_bwd(const void* hidden, const void* W_head, int32_t dtype,
+                             int64_t T, int32_t H, int32_t V, int64_t ld_hidden, int64_t ld_W,
+                             const int32_t* ids, const float* old_logp, const float* adv,
+                             const int32_t* cu_seqlens, int32_t S, const sapo_loss_cfg* h_cfg,
+                             float* logp, float* lse, float* ratio, float* surr, float* gscale,
+                             float* seq_surr, float* loss,
+                             float* dhidden, float* dW_head, int32_t accumulate_dW,
+                             void* workspace, size_t workspace_bytes,
+                             int32_t* status, void* stream);
+
 /* Section 3.2 (nodes filter and sample what the swarm shares) / Section 5 (the experiments'
  * policy: discard rollouts with zero advantage, then sample uniformly from the rest).
  * The pool holds n_entries rollouts; entry g is a question's group of completions with rewards
@@ -248,11 +285,11 @@ int sapo_adam_step(float* master, float* m, float* v, const float* grad, void* w
                    int64_t rows, int32_t cols, int64_t ld_w, int32_t step,
                    float lr, float beta1, float beta2, float eps, void* stream);
 
-/* Bytes of scratch the forward (SAPO_WS_FWD) or backward (SAPO_WS_BWD) call wants for
- * these sizes.  Returns 0 for invalid arguments. */
+/* Bytes of scratch the forward (SAPO_WS_FWD), backward (SAPO_WS_BWD, SAPO_WS_BWD_ACTIVE) or
+ * fused (SAPO_WS_FUSED) call wants for these sizes.  Returns 0 for invalid arguments. */
 size_t sapo_workspace_bytes(int32_t which, int64_t T, int32_t H, int32_t V, int32_t dtype);
 
-/* Smallest backward workspace that still works (one 128-token panel). */
+/* Smallest backward or fused workspace that still works (one 128-token panel). */
 size_t sapo_workspace_bytes_min(int32_t which, int64_t T, int32_t H, int32_t V, int32_t dtype);
 
 /* Forward pass without caller-provided scratch (the paper has no counterpart; this exists for
@@ -299,7 +336,10 @@ int sapo_policy_loss_fwd_static(const void* hidden, const void* W_head, int32_t 
 #define SAPO_K_COMPACT   11
 #define SAPO_K_SELECT    12
 #define SAPO_K_ADAM      13
-#define SAPO_K_COUNT      14
+#define SAPO_K_TARGET_LOGIT 14
+#define SAPO_K_FWD_EXP   15
+#define SAPO_K_FUSED_TAIL 16
+#define SAPO_K_COUNT      17
 int sapo_timing_enable(int32_t on);
 int sapo_timing_read(float* h_ms, int32_t* h_launches);
 int64_t sapo_launch_count(void);

@@ -19,20 +19,23 @@ DTYPE_F32 = 1
 WS_FWD = 0
 WS_BWD = 1
 WS_BWD_ACTIVE = 2
+WS_FUSED = 3
 
 ST_BITS = {
     0x01: "TOKEN_OVERFLOW", 0x02: "SEQ_OVERFLOW", 0x04: "BAD_INDEX", 0x08: "EMPTY_SEQUENCE",
-    0x10: "BAD_TOKEN_ID", 0x20: "WAIT_TIMEOUT", 0x40: "NONFINITE_REWARD",
+    0x10: "BAD_TOKEN_ID", 0x20: "WAIT_TIMEOUT", 0x40: "NONFINITE_REWARD", 0x80: "EXP_RANGE",
 }
 
 EXPORTS = ("sapo_pack_rollouts", "sapo_group_advantages", "sapo_policy_loss_fwd",
            "sapo_policy_loss_bwd", "sapo_workspace_bytes", "sapo_workspace_bytes_min",
            "sapo_status_string", "sapo_timing_enable", "sapo_timing_read", "sapo_launch_count",
-           "sapo_policy_loss_fwd_static", "sapo_policy_loss_bwd_active", "sapo_select_external",
+           "sapo_policy_loss_fwd_static", "sapo_policy_loss_bwd_active", "sapo_policy_loss_fwd_bwd",
+           "sapo_select_external",
            "sapo_select_workspace_bytes", "sapo_adam_step")
 STATIC_SCRATCH_BYTES = 4 * 1024 * 1024
 KERNEL_NAMES = ("pack_scan", "pack_copy", "group_adv", "split_bf16", "fwd_gemm", "loss_tail",
-                "loss_final", "bwd_dz", "bwd_dh", "bwd_dw", "streamk_fixup", "compact", "select", "adam")
+                "loss_final", "bwd_dz", "bwd_dh", "bwd_dw", "streamk_fixup", "compact", "select", "adam",
+                "target_logit", "fwd_exp", "fused_tail")
 
 
 class RolloutBufC(C.Structure):
@@ -93,6 +96,10 @@ def load() -> C.CDLL:
     lib.sapo_policy_loss_bwd_active.restype = C.c_int
     lib.sapo_policy_loss_bwd_active.argtypes = [vp, vp, i32, i64, i32, i32, i64, i64, vp, vp, vp, vp, vp,
                                                 i32, vp, vp, sz, vp, vp]
+    lib.sapo_policy_loss_fwd_bwd.restype = C.c_int
+    lib.sapo_policy_loss_fwd_bwd.argtypes = [vp, vp, i32, i64, i32, i32, i64, i64, vp, vp, vp, vp, i32,
+                                             C.POINTER(LossCfgC), vp, vp, vp, vp, vp, vp, vp, vp, vp, i32,
+                                             vp, sz, vp, vp]
     lib.sapo_select_external.restype = C.c_int
     lib.sapo_select_external.argtypes = [vp, vp, i32, i32, C.c_uint64, vp, vp, vp, vp, sz, vp]
     lib.sapo_select_workspace_bytes.restype = sz
@@ -319,6 +326,28 @@ def sapo_policy_loss_bwd_active(hidden: torch.Tensor, W_head: torch.Tensor, ids:
         _p(ids), _p(lse), _p(gscale), _p(dhidden), _p(dW_head), 1 if accumulate_dW else 0, _p(n_active),
         _p(workspace), workspace.numel() * workspace.element_size(), _p(status), _stream())
     _check(rc, "sapo_policy_loss_bwd_active")
+
+
+def sapo_policy_loss_fwd_bwd(hidden: torch.Tensor, W_head: torch.Tensor, ids: torch.Tensor,
+                             old_logp: torch.Tensor, adv: torch.Tensor, cu_seqlens: torch.Tensor,
+                             eps_low: float, eps_high: float, grad_scale: float,
+                             out: Dict[str, torch.Tensor], dhidden: torch.Tensor, dW_head: torch.Tensor,
+                             accumulate_dW: bool, workspace: torch.Tensor, status: torch.Tensor,
+                             T: Optional[int] = None, loss_agg: int = 0, kl_beta: float = 0.0,
+                             ref_logp: Optional[torch.Tensor] = None) -> None:
+    """Loss and both gradients in one call with a single pass over the logits (bf16 only)."""
+    _require_cuda()
+    T = int(hidden.shape[0]) if T is None else int(T)
+    H, V = int(hidden.shape[1]), int(W_head.shape[0])
+    S = int(cu_seqlens.numel() - 1)
+    cfg = LossCfgC(eps_low, eps_high, grad_scale, int(loss_agg), float(kl_beta), _p(ref_logp))
+    rc = load().sapo_policy_loss_fwd_bwd(
+        _p(hidden), _p(W_head), _dtype_code(hidden), T, H, V, hidden.stride(0), W_head.stride(0),
+        _p(ids), _p(old_logp), _p(adv), _p(cu_seqlens), S, C.byref(cfg),
+        _p(out["logp"]), _p(out["lse"]), _p(out["ratio"]), _p(out["surr"]), _p(out["gscale"]),
+        _p(out.get("seq_surr")), _p(out["loss"]), _p(dhidden), _p(dW_head), 1 if accumulate_dW else 0,
+        _p(workspace), workspace.numel() * workspace.element_size(), _p(status), _stream())
+    _check(rc, "sapo_policy_loss_fwd_bwd")
 
 
 def sapo_select_external(rewards: torch.Tensor, group_offsets: torch.Tensor, J: int, seed: int):

@@ -38,6 +38,7 @@ constexpr uint32_t STAGING_BYTES = 2 * 128 * 128;   // dz epilogue: one 16 KB pa
 constexpr size_t GEMM_SMEM_BYTES = 1024 + STAGES * (A_STAGE_BYTES + B_STAGE_BYTES) + 256;
 constexpr float LOG2E = 1.4426950408889634f;
 constexpr float LN2 = 0.6931471805599453f;
+constexpr float EXP_CAP = 1.2676506002282294e30f;   // 2^100: cap of a stored exponential (fused call)
 
 // Static tile schedule: `num_units` work units, each one 256-row block and a run of n-blocks,
 // dealt round-robin to the CTA pairs.
@@ -171,6 +172,27 @@ struct StageCtx {
   const CUtensorMap* map;
 };
 
+// A thread's 64 finished bf16 entries of a panel row (two 32-column chunks as 16 pairs each)
+// go to the staging tile, and the tile leaves as one 16 KB TMA store: wait until the previous
+// store has read the staging tile, write this row (128 bytes, in 128-byte-swizzle order) and
+// hand the tile to the TMA.  Called by all 128 threads that share the staging tile.
+__device__ __forceinline__ void store_panel_group(const StageCtx& cx, int r, const uint32_t (&pk)[2][16],
+                                                  int tile_row0, int col0_of_group) {
+  if (cx.elected) bulk_wait_read_all();
+  named_barrier_sync(cx.bar_id, 128);
+  #pragma unroll
+  for (int q = 0; q < 8; ++q)
+    st_shared_v4(cx.buf + r * 128 + ((q ^ (r & 7)) << 4),
+                 pk[q >> 2][4 * (q & 3)], pk[q >> 2][4 * (q & 3) + 1],
+                 pk[q >> 2][4 * (q & 3) + 2], pk[q >> 2][4 * (q & 3) + 3]);
+  fence_proxy_async_smem();
+  named_barrier_sync(cx.bar_id, 128);
+  if (cx.elected) {
+    tma_store_2d(cx.map, cx.buf, 0, tile_row0 + (col0_of_group >> 6) * BM);
+    bulk_commit_group();
+  }
+}
+
 // Forward: online log-sum-exp in the base-2 domain plus the logit of the chosen token.
 struct FwdEpi {
   static constexpr bool STAGED = false;
@@ -274,25 +296,73 @@ struct DzEpi {
       }
     }
   }
-  // after both chunks of the group: wait until the previous TMA store has read the staging
-  // tile, write this row (128 bytes, in 128-byte-swizzle order) and hand the tile to the TMA
-  __device__ __forceinline__ void group_end(const Params& p, int col0_of_group, const StageCtx& cx) {
-    if (!in_panel) return;
-    if (cx.elected) bulk_wait_read_all();
-    named_barrier_sync(cx.bar_id, 128);
-    #pragma unroll
-    for (int q = 0; q < 8; ++q)
-      st_shared_v4(cx.buf + r * 128 + ((q ^ (r & 7)) << 4),
-                   pk[q >> 2][4 * (q & 3)], pk[q >> 2][4 * (q & 3) + 1],
-                   pk[q >> 2][4 * (q & 3) + 2], pk[q >> 2][4 * (q & 3) + 3]);
-    fence_proxy_async_smem();
-    named_barrier_sync(cx.bar_id, 128);
-    if (cx.elected) {
-      tma_store_2d(cx.map, cx.buf, 0, tile_row0 + (col0_of_group >> 6) * BM);
-      bulk_commit_group();
-    }
+  __device__ __forceinline__ void group_end(const Params&, int col0_of_group, const StageCtx& cx) {
+    if (in_panel) store_panel_group(cx, r, pk, tile_row0, col0_of_group);
   }
   __device__ __forceinline__ void end_unit(const Params&, int, int) {}
+};
+
+// Forward of the fused call: e[t,v] = exp(z[t,v] - c_t) against a per-token reference c_t that
+// is known before the pass (see sapo_policy_loss_fwd_bwd), so no running maximum is needed:
+// the epilogue adds the fp32 exponentials up per token and leaves them, rounded to bf16, in
+// the tiled panel (same layout as DzEpi) for the backward contractions, which then need no
+// second pass over the logits.  Exponentials are capped at 2^100, so that sums and products
+// with them stay finite and a zero row scale later still gives zero (a token that reaches the
+// cap is reported, see fused_tail_kernel).  Rows past the last token and columns past V hold zeros.
+struct ExpEpi {
+  static constexpr bool STAGED = true;
+  static constexpr bool STREAMK = false;
+  template <class P> __device__ static void set_dynamic(P&, const Sched&) {}
+  struct Params {
+    const float* c2;      // [M] reference of each token, in the base-2 domain (c_t * log2 e)
+    float* ps;            // [2 * n_splits][M] partial sums of exponentials
+    int64_t M; int32_t V; int32_t nvt;
+  };
+  float c, sum; int32_t tile_row0; int r; bool valid, in_panel; int64_t row;
+  uint32_t pk[2][16];
+  __device__ __forceinline__ void begin_unit(const Params& p, int mb, int r_) {
+    row = (int64_t)mb * BM + r_;
+    valid = row < p.M;
+    in_panel = (int64_t)mb * BM < p.M;
+    r = r_;
+    tile_row0 = mb * p.nvt * BM;
+    c = valid ? p.c2[row] : 0.f;
+    sum = 0.f;
+  }
+  __device__ __forceinline__ void group_begin(const StageCtx&) {}
+  template <int HALF>
+  __device__ __forceinline__ void chunk(const Params& p, float (&v)[32], int col0, const StageCtx&) {
+    if (!in_panel) return;
+    uint32_t (&packed)[16] = pk[HALF];
+    if (!valid || col0 >= p.V) {
+      #pragma unroll
+      for (int j = 0; j < 16; ++j) packed[j] = 0u;
+      return;
+    }
+    const float cap = EXP_CAP;
+    #pragma unroll
+    for (int j = 0; j < 32; ++j) v[j] = fminf(ex2(fmaf(v[j], LOG2E, -c)), cap);
+    if (col0 + 32 > p.V) {               // ragged end of the vocabulary
+      #pragma unroll
+      for (int j = 0; j < 32; ++j) if (col0 + j >= p.V) v[j] = 0.f;
+    }
+    float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+    #pragma unroll
+    for (int j = 0; j < 32; j += 4) { a0 += v[j]; a1 += v[j + 1]; a2 += v[j + 2]; a3 += v[j + 3]; }
+    sum += (a0 + a1) + (a2 + a3);
+    #pragma unroll
+    for (int j = 0; j < 16; ++j) {
+      __nv_bfloat162 h = __floats2bfloat162_rn(v[2 * j], v[2 * j + 1]);
+      packed[j] = *reinterpret_cast<uint32_t*>(&h);
+    }
+  }
+  __device__ __forceinline__ void group_end(const Params&, int col0_of_group, const StageCtx& cx) {
+    if (in_panel) store_panel_group(cx, r, pk, tile_row0, col0_of_group);
+  }
+  // two threads share a row (one per column half of the tiles): each leaves its own partial
+  __device__ __forceinline__ void end_unit(const Params& p, int un, int col_half) {
+    if (valid) p.ps[(int64_t)(2 * un + col_half) * p.M + row] = sum;
+  }
 };
 
 // Plain fp32 output tile, optionally added to what is already there.
@@ -301,15 +371,17 @@ struct StoreEpi {
   static constexpr bool STREAMK = true;
   // row_map (optional): output row of each accumulator row (rows of compacted tokens go back
   // to their packed positions)
+  // row_scale (optional): factor applied to each accumulator row before it is stored
   struct Params { float* C; int64_t ldc; int64_t M; int32_t N; int32_t accumulate; float* partials;
-                  const int32_t* row_map; };
+                  const int32_t* row_map; const float* row_scale; };
   template <class P> __device__ static void set_dynamic(P& p, const Sched& s) {
     if (s.dyn_dim == 1) p.M = *s.dyn_count;
   }
-  int64_t row; bool valid; float* part; int n0;
+  int64_t row; bool valid; float* part; int n0; float scale;
   __device__ __forceinline__ void begin_unit(const Params& p, int mb, int r) {
     row = (int64_t)mb * BM + r;
     valid = row < p.M;
+    scale = (valid && p.row_scale != nullptr) ? p.row_scale[row] : 1.f;
     if (valid && p.row_map != nullptr) row = p.row_map[row];
     part = nullptr;
   }
@@ -332,7 +404,8 @@ struct StoreEpi {
     #pragma unroll
     for (int q = 0; q < 8; ++q) {
       if (col0 + 4 * q < p.N) {          // N is a multiple of 4
-        float4 o = make_float4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
+        float4 o = make_float4(scale * v[4 * q], scale * v[4 * q + 1], scale * v[4 * q + 2],
+                               scale * v[4 * q + 3]);
         if (p.accumulate) { const float4 c = dst[q]; o.x += c.x; o.y += c.y; o.z += c.z; o.w += c.w; }
         dst[q] = o;
       }
@@ -361,10 +434,12 @@ streamk_fixup_kernel(const Sched s_arg, const StoreEpi::Params p_arg, int pairs)
   for (int rr = row_begin; rr < row_begin + 8; ++rr) {
     int64_t row = (int64_t)pmb * PAIR_M + rr;
     if (row >= p.M) break;
+    const float scale = p.row_scale != nullptr ? p.row_scale[row] : 1.f;
     if (p.row_map != nullptr) row = p.row_map[row];
     const size_t off = (size_t)rr * BN + col;
     float sum = 0.f;
     for (int j = 0; j < s.sk_parts; ++j) sum += p.partials[(size_t)(j * s.sk_tiles + t) * PARTIAL_FLOATS + off];
+    sum *= scale;
     float* dst = p.C + row * p.ldc + n0 + col;
     *dst = p.accumulate ? *dst + sum : sum;
   }
@@ -720,6 +795,143 @@ loss_final_kernel(const float* seq_surr, const int32_t* cu, int32_t S, int64_t T
   if (threadIdx.x == 0) *loss = n > 0 ? (float)(-tot / n) : 0.f;
 }
 
+// ---------------------------------------------------------------------------- fused call: small kernels
+// Before the forward pass of the fused call: the logit of the chosen token, z_y[t] = <h_t, W_y>,
+// as a plain fp32 dot product (one warp per token), and the reference of the exponentials
+//   c_t = z_y[t] - old_logp[t],
+// which equals lse_t when the policy has not moved since old_logp was taken and is off by
+// log(ratio_t) otherwise: exp(z - c_t) then stays within a few powers of e of a probability.
+// c2 is c_t * log2(e).  A token id outside [0, V) gets z_y = c = 0 (the tail reports it).
+__global__ void __launch_bounds__(256)
+target_logit_kernel(const __nv_bfloat16* __restrict__ hidden, int64_t ldh, const __nv_bfloat16* __restrict__ W,
+                    int64_t ldw, const int32_t* __restrict__ ids, const float* __restrict__ old_logp,
+                    int64_t T, int32_t H, int32_t V, float* __restrict__ zy, float* __restrict__ c2) {
+  const int lane = threadIdx.x & 31;
+  const int64_t warp = (int64_t)blockIdx.x * 8 + (threadIdx.x >> 5);
+  const int64_t n_warps = (int64_t)gridDim.x * 8;
+  for (int64_t t = warp; t < T; t += n_warps) {
+    const int32_t y = ids[t];
+    float acc = 0.f;
+    if (y >= 0 && y < V) {
+      const uint4* a = reinterpret_cast<const uint4*>(hidden + t * ldh);
+      const uint4* b = reinterpret_cast<const uint4*>(W + (int64_t)y * ldw);
+      for (int i = lane; i < H / 8; i += 32) {
+        const uint4 ua = a[i], ub = b[i];
+        const __nv_bfloat162* pa = reinterpret_cast<const __nv_bfloat162*>(&ua);
+        const __nv_bfloat162* pb = reinterpret_cast<const __nv_bfloat162*>(&ub);
+        #pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          const float2 fa = __bfloat1622float2(pa[j]), fb = __bfloat1622float2(pb[j]);
+          acc = fmaf(fa.x, fb.x, acc); acc = fmaf(fa.y, fb.y, acc);
+        }
+      }
+      #pragma unroll
+      for (int d = 16; d > 0; d >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, d);
+    }
+    if (lane == 0) {
+      const bool ok = y >= 0 && y < V;
+      zy[t] = ok ? acc : 0.f;
+      c2[t] = ok ? (acc - old_logp[t]) * LOG2E : 0.f;
+    }
+  }
+}
+
+struct FusedTailArgs {
+  const float* ps; int32_t n_parts; int64_t t0, tc;        // partial sums [n_parts][tc] of this token chunk
+  const float* zy; const float* c2;                        // [T]
+  const int32_t* ids; int32_t V; const float* old_logp; const float* adv; const int32_t* cu; int32_t S;
+  int64_t T; float lo_edge, hi_edge, grad_scale; int32_t loss_agg; float kl_beta; const float* ref_logp;
+  float* logp; float* lse; float* ratio; float* surr; float* gscale; float* obj;   // [T]
+  float* row_scale;                                        // [tc]
+  __nv_bfloat16* panel; int32_t nvt;                       // exponentials of the chunk
+  const __nv_bfloat16* hidden; int64_t ldh; int32_t H; __nv_bfloat16* hs;   // hs [tc, H] = row_scale * hidden
+  int32_t* status;
+};
+
+// After the forward pass of a token chunk of the fused call, one warp per token:
+//   sum_t = sum_v exp(z - c_t);  lse = c_t + log sum_t;  logp = z_y - lse;  ratio, surrogate and
+//   g_t = dloss/dlogp as in loss_tail_kernel;
+// then what turns the stored exponentials e into dz = g ([v = y] - e / sum_t) = a_t e' with
+//   a_t = -g_t / sum_t,   e'[t,v] = e[t,v] - [v = y_t] sum_t :
+// the panel entry of the chosen token is replaced by e_y - sum_t, a_t becomes the row scale of
+// the dhidden contraction, and hs = a_t * hidden (bf16) the operand of the dW_head contraction.
+__global__ void __launch_bounds__(256) fused_tail_kernel(FusedTailArgs a) {
+  const int lane = threadIdx.x & 31;
+  const int64_t warp = (int64_t)blockIdx.x * 8 + (threadIdx.x >> 5);
+  const int64_t n_warps = (int64_t)gridDim.x * 8;
+  for (int64_t lr = warp; lr < a.tc; lr += n_warps) {
+    const int64_t t = a.t0 + lr;
+    float part = 0.f;
+    for (int i = lane; i < a.n_parts; i += 32) part += a.ps[(int64_t)i * a.tc + lr];
+    #pragma unroll
+    for (int d = 16; d > 0; d >>= 1) part += __shfl_xor_sync(0xffffffffu, part, d);
+    const float sum = part;
+    // the sequence of this token: last s with cu[s] <= t
+    int lo = 0, hi = a.S - 1;
+    while (lo < hi) { const int mid = (lo + hi + 1) >> 1; if ((int64_t)a.cu[mid] <= t) lo = mid; else hi = mid - 1; }
+    const int32_t Ts = a.cu[lo + 1] - a.cu[lo];
+    const float A = a.adv[lo];
+    const float w = Ts <= 0 ? 0.f : (a.loss_agg == 0 ? 1.f / ((float)a.S * (float)Ts) : 1.f / (float)a.T);
+    const int32_t y = a.ids[t];
+    const bool bad_id = y < 0 || y >= a.V;
+    // a capped exponential, or a sum that left the fp32 range: the reference was too far off
+    const bool bad_range = !(sum < EXP_CAP) || !(sum > 1.f / EXP_CAP);
+    const bool bad = bad_id || bad_range;
+    const float c2 = a.c2[t], zy = a.zy[t];
+    const float lse = bad_range ? 0.f : (c2 + log2f(sum)) * LN2;
+    const float lp = bad ? 0.f : zy - lse;
+    const float rho = bad ? 0.f : expf(lp - a.old_logp[t]);
+    const float un = rho * A;
+    const float cl = fminf(fmaxf(rho, a.lo_edge), a.hi_edge) * A;
+    const float u = bad ? 0.f : fminf(un, cl);
+    float g = (!bad && un <= cl) ? -a.grad_scale * A * rho * w : 0.f;
+    float obj = u;
+    if (a.kl_beta != 0.f && !bad) {
+      const float d = a.ref_logp[t] - lp;
+      const float ed = expf(d);
+      obj -= a.kl_beta * (ed - d - 1.f);
+      g += a.grad_scale * w * a.kl_beta * (1.f - ed);
+    }
+    const float scale = (bad || g == 0.f) ? 0.f : -g / sum;
+    if (lane == 0) {
+      if (bad_id) raise_status(a.status, SAPO_ST_BAD_TOKEN_ID);
+      if (bad_range) raise_status(a.status, SAPO_ST_EXP_RANGE);
+      a.lse[t] = lse; a.logp[t] = lp; a.ratio[t] = rho; a.surr[t] = u; a.gscale[t] = g; a.obj[t] = obj;
+      a.row_scale[lr] = scale;
+      if (!bad) {
+        const float ey = ex2(fmaf(zy, LOG2E, -c2));
+        const int64_t tile = (lr >> 7) * a.nvt + (y >> 6);
+        a.panel[(tile * BM + (lr & 127)) * 64 + (y & 63)] = __float2bfloat16_rn(ey - sum);
+      }
+    }
+    const uint4* src = reinterpret_cast<const uint4*>(a.hidden + t * a.ldh);
+    uint4* dst = reinterpret_cast<uint4*>(a.hs + lr * (int64_t)a.H);
+    for (int i = lane; i < a.H / 8; i += 32) {
+      uint4 x = src[i];
+      __nv_bfloat162* px = reinterpret_cast<__nv_bfloat162*>(&x);
+      #pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const float2 f = __bfloat1622float2(px[j]);
+        px[j] = __floats2bfloat162_rn(scale * f.x, scale * f.y);
+      }
+      dst[i] = x;
+    }
+  }
+}
+
+// seq_surr[s] = mean over the tokens of s of obj[t] (same summation order as loss_tail_kernel)
+__global__ void __launch_bounds__(256)
+seq_mean_kernel(const float* __restrict__ obj, const int32_t* __restrict__ cu, int32_t S, float* seq_surr) {
+  __shared__ double sh[8];
+  for (int32_t s = blockIdx.x; s < S; s += gridDim.x) {
+    const int32_t t0 = cu[s], t1 = cu[s + 1];
+    double acc = 0.0;
+    for (int32_t t = t0 + threadIdx.x; t < t1; t += 256) acc += (double)obj[t];
+    const double tot = block_sum_256(acc, sh);
+    if (threadIdx.x == 0) seq_surr[s] = t1 > t0 ? (float)(tot / (double)(t1 - t0)) : 0.f;
+  }
+}
+
 // ---------------------------------------------------------------------------- host side
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
@@ -810,7 +1022,7 @@ static int launch_gemm(const CUtensorMap& ma, const CUtensorMap& mb, const CUten
   static int max_pairs = 0;     // CTA pairs the device can hold at once, found on first use
   if (sched.num_units <= 0) return SAPO_OK;
   Sched sc = sched;
-  sc.stats_id = kernel_id == SAPO_K_FWD_GEMM ? 0 : kernel_id - SAPO_K_BWD_DZ + 1;
+  sc.stats_id = (kernel_id == SAPO_K_FWD_GEMM || kernel_id == SAPO_K_FWD_EXP) ? 0 : kernel_id - SAPO_K_BWD_DZ + 1;
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeClusterDimension;
   attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
@@ -905,6 +1117,39 @@ static BwdLayout bwd_layout(int64_t T, int32_t H, int32_t V, int32_t dtype) {
 }
 constexpr int64_t PANEL_ROWS_PREFERRED = 32768;
 
+// Scratch of the fused call: per-token vectors for all T tokens, then what one token chunk
+// needs (row scales, partial sums, the scaled copy of hidden), the K-split scratch, the
+// per-sequence sums when the caller does not want them, and the panel of exponentials.
+constexpr int FUSED_MAX_SPLITS = 160;
+struct FusedLayout { size_t zy, c2, obj, seq, partials, fixed; size_t bytes_per_row; };
+static FusedLayout fused_layout(int64_t T, int32_t H, int32_t V, int32_t S) {
+  FusedLayout L{};
+  size_t off = 0;
+  auto take = [&](size_t bytes) { const size_t at = off; off += round_up<size_t>(bytes, 256); return at; };
+  L.zy = take((size_t)T * 4);
+  L.c2 = take((size_t)T * 4);
+  L.obj = take((size_t)T * 4);
+  L.seq = take((size_t)(S > 0 ? S : 1) * 4);
+  L.partials = take((size_t)MAX_PARTS_SCRATCH * PARTIAL_FLOATS * sizeof(float));
+  L.fixed = off;
+  // per chunk row: panel row, scaled hidden row, row scale, partial sums
+  L.bytes_per_row = (size_t)padded_vocab(V) * 2 + (size_t)H * 2 + 4 + (size_t)2 * FUSED_MAX_SPLITS * 4;
+  return L;
+}
+// where the per-chunk arrays sit for a chunk capacity of `rows` (a multiple of 128)
+struct FusedChunk { size_t row_scale, ps, hs, panel; };
+static FusedChunk fused_chunk(const FusedLayout& L, int64_t rows, int32_t H) {
+  FusedChunk C{};
+  size_t off = L.fixed;
+  auto take = [&](size_t bytes) { const size_t at = off; off += round_up<size_t>(bytes, 256); return at; };
+  C.row_scale = take((size_t)rows * 4);
+  C.ps = take((size_t)rows * 2 * FUSED_MAX_SPLITS * 4);
+  C.hs = take((size_t)rows * H * 2);
+  C.panel = take(0);
+  return C;
+}
+constexpr size_t FUSED_CHUNK_SLACK = 4 * 256;   // alignment padding between the per-chunk arrays
+
 // Scratch of the compacting backward in front of the regular backward's: scan counters, the
 // active-token list, compacted per-token vectors and hidden rows.
 struct ActiveLayout { size_t counts, n_active, chunk_counts, act_idx, ids, lse, g, hidden, total; };
@@ -946,6 +1191,12 @@ extern "C" size_t sapo_workspace_bytes(int32_t which, int64_t T, int32_t H, int3
     if (sms <= 0) sms = 148;
     return fwd_layout(T, H, V, dtype, sms).total;
   }
+  if (which == SAPO_WS_FUSED) {
+    if (dtype != SAPO_DTYPE_BF16) return 0;
+    const FusedLayout L = fused_layout(T, H, V, /*S=*/(int32_t)(T < 0x7fffffff ? T : 0x7fffffff));
+    const int64_t rows = T < PANEL_ROWS_PREFERRED ? T : PANEL_ROWS_PREFERRED;
+    return L.fixed + FUSED_CHUNK_SLACK + (size_t)round_up<int64_t>(rows, BM) * L.bytes_per_row;
+  }
   if (which == SAPO_WS_BWD || which == SAPO_WS_BWD_ACTIVE) {
     const BwdLayout L = bwd_layout(T, H, V, dtype);
     const int64_t rows = T < PANEL_ROWS_PREFERRED ? T : PANEL_ROWS_PREFERRED;
@@ -957,8 +1208,13 @@ extern "C" size_t sapo_workspace_bytes(int32_t which, int64_t T, int32_t H, int3
 
 extern "C" size_t sapo_workspace_bytes_min(int32_t which, int64_t T, int32_t H, int32_t V, int32_t dtype) {
   using namespace sapo;
-  if (which != SAPO_WS_BWD) return sapo_workspace_bytes(which, T, H, V, dtype);
+  if (which != SAPO_WS_BWD && which != SAPO_WS_FUSED) return sapo_workspace_bytes(which, T, H, V, dtype);
   if (!shapes_ok(T, H, V) || (dtype != SAPO_DTYPE_BF16 && dtype != SAPO_DTYPE_F32)) return 0;
+  if (which == SAPO_WS_FUSED) {
+    if (dtype != SAPO_DTYPE_BF16) return 0;
+    const FusedLayout L = fused_layout(T, H, V, (int32_t)(T < 0x7fffffff ? T : 0x7fffffff));
+    return L.fixed + FUSED_CHUNK_SLACK + (size_t)BM * L.bytes_per_row;
+  }
   const BwdLayout L = bwd_layout(T, H, V, dtype);
   return L.fixed + (size_t)BM * L.bytes_per_row;
 }
@@ -1154,7 +1410,7 @@ extern "C" int sapo_policy_loss_bwd(const void* hidden, const void* W_head, int3
     {
       Sched sched = make_sched(tc, H, Vp, 0, /*m_fastest=*/false);
       sched.panel_nvt = nvt;
-      StoreEpi::Params ep{dhidden + t0 * (int64_t)H, H, tc, H, 0, partials, nullptr};
+      StoreEpi::Params ep{dhidden + t0 * (int64_t)H, H, tc, H, 0, partials, nullptr, nullptr};
       int rc = launch_gemm<2, true, StoreEpi>(map_p_two, map_w_mn, map_p_two, sched, ep, status, st, SAPO_K_BWD_DH);
       if (rc != SAPO_OK) return rc;
     }
@@ -1162,7 +1418,7 @@ extern "C" int sapo_policy_loss_bwd(const void* hidden, const void* W_head, int3
     {
       Sched sched = make_sched(V, H, tc, 0, /*m_fastest=*/false);
       sched.panel_nvt = nvt;
-      StoreEpi::Params ep{dW_head, H, V, H, (t0 > 0 || accumulate_dW) ? 1 : 0, partials, nullptr};
+      StoreEpi::Params ep{dW_head, H, V, H, (t0 > 0 || accumulate_dW) ? 1 : 0, partials, nullptr, nullptr};
       int rc = launch_gemm<3, true, StoreEpi>(map_p_tile, map_h_mn, map_p_tile, sched, ep, status, st, SAPO_K_BWD_DW);
       if (rc != SAPO_OK) return rc;
     }
@@ -1282,7 +1538,7 @@ extern "C" int sapo_policy_loss_bwd_active(const void* hidden, const void* W_hea
       Sched sched = make_sched(tc, H, Vp, 0, /*m_fastest=*/false);
       sched.panel_nvt = nvt;
       sched.dyn_count = count; sched.dyn_dim = 1;
-      StoreEpi::Params ep{dhidden, H, tc, H, 0, partials, act_idx + t0};   // rows go back to their tokens
+      StoreEpi::Params ep{dhidden, H, tc, H, 0, partials, act_idx + t0, nullptr};   // rows go back to their tokens
       int rc = launch_gemm<2, true, StoreEpi>(map_p_two, map_w_mn, map_p_two, sched, ep, status, st, SAPO_K_BWD_DH);
       if (rc != SAPO_OK) return rc;
     }
@@ -1291,12 +1547,134 @@ extern "C" int sapo_policy_loss_bwd_active(const void* hidden, const void* W_hea
       Sched sched = make_sched(V, H, tc, 0, /*m_fastest=*/false);
       sched.panel_nvt = nvt;
       sched.dyn_count = count; sched.dyn_dim = 2; sched.skip_if_empty = acc;
-      StoreEpi::Params ep{dW_head, H, V, H, acc, partials, nullptr};
+      StoreEpi::Params ep{dW_head, H, V, H, acc, partials, nullptr, nullptr};
       int rc = launch_gemm<3, true, StoreEpi>(map_p_tile, map_h_mn, map_p_tile, sched, ep, status, st, SAPO_K_BWD_DW);
       if (rc != SAPO_OK) return rc;
     }
   }
   return SAPO_OK;
+}
+
+// ------------------------------------------------------------------------------------------
+// Loss and both gradients in one call, without a second pass over the logits: the forward
+// epilogue leaves exp(z - c_t) in the panel, and the two backward contractions read it.
+extern "C" int sapo_policy_loss_fwd_bwd(const void* hidden, const void* W_head, int32_t dtype,
+                                        int64_t T, int32_t H, int32_t V, int64_t ld_hidden, int64_t ld_W,
+                                        const int32_t* ids, const float* old_logp, const float* adv,
+                                        const int32_t* cu_seqlens, int32_t S, const sapo_loss_cfg* h_cfg,
+                                        float* logp, float* lse, float* ratio, float* surr, float* gscale,
+                                        float* seq_surr, float* loss,
+                                        float* dhidden, float* dW_head, int32_t accumulate_dW,
+                                        void* workspace, size_t workspace_bytes,
+                                        int32_t* status, void* stream) {
+  using namespace sapo;
+  if (!hidden || !W_head || !ids || !old_logp || !adv || !cu_seqlens || !h_cfg || !logp || !lse ||
+      !ratio || !surr || !gscale || !loss || !dhidden || !dW_head || !workspace || !status || S < 1)
+    return SAPO_ERR_INVALID_ARG;
+  if (dtype != SAPO_DTYPE_BF16 && dtype != SAPO_DTYPE_F32) return SAPO_ERR_INVALID_ARG;
+  if (T < 1 || H < 1 || V < 1 || ld_hidden < H || ld_W < H) return SAPO_ERR_INVALID_ARG;
+  if (!seq_surr && S > T) return SAPO_ERR_INVALID_ARG;   // the built-in per-sequence scratch holds T entries
+  if (!shapes_ok(T, H, V)) return SAPO_ERR_UNSUPPORTED_SHAPE;
+  if (dtype != SAPO_DTYPE_BF16) return SAPO_ERR_UNSUPPORTED_SHAPE;   // fp32 operands: use the separate calls
+  if (!aligned16(hidden) || !aligned16(W_head) || !aligned16(workspace) || !aligned16(dhidden) ||
+      !aligned16(dW_head) || (ld_hidden * 2) % 16 || (ld_W * 2) % 16)
+    return SAPO_ERR_INVALID_ARG;
+  if (!(h_cfg->eps_low >= 0.f) || !(h_cfg->eps_high >= 0.f)) return SAPO_ERR_INVALID_ARG;
+  if ((h_cfg->loss_agg != 0 && h_cfg->loss_agg != 1) || (h_cfg->kl_beta != 0.f && !h_cfg->ref_logp))
+    return SAPO_ERR_INVALID_ARG;
+  const int sms = sm_count();
+  if (sms <= 0) return SAPO_ERR_CUDA;
+  const FusedLayout L = fused_layout(T, H, V, (int32_t)(T < 0x7fffffff ? T : 0x7fffffff));
+  if (workspace_bytes < L.fixed + FUSED_CHUNK_SLACK + (size_t)BM * L.bytes_per_row)
+    return SAPO_ERR_WORKSPACE_TOO_SMALL;
+  const int64_t rows_fit =
+      ((int64_t)((workspace_bytes - L.fixed - FUSED_CHUNK_SLACK) / L.bytes_per_row) / BM) * BM;
+  const int64_t chunk_rows = rows_fit >= T ? round_up<int64_t>(T, BM) : rows_fit;   // capacity, a multiple of 128
+  const FusedChunk CL = fused_chunk(L, chunk_rows, H);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  uint8_t* ws = static_cast<uint8_t*>(workspace);
+  float* zy = reinterpret_cast<float*>(ws + L.zy);
+  float* c2 = reinterpret_cast<float*>(ws + L.c2);
+  float* obj = reinterpret_cast<float*>(ws + L.obj);
+  float* seq_out = seq_surr ? seq_surr : reinterpret_cast<float*>(ws + L.seq);
+  float* partials = reinterpret_cast<float*>(ws + L.partials);
+  float* row_scale = reinterpret_cast<float*>(ws + CL.row_scale);
+  float* ps = reinterpret_cast<float*>(ws + CL.ps);
+  __nv_bfloat16* hs = reinterpret_cast<__nv_bfloat16*>(ws + CL.hs);
+  __nv_bfloat16* panel = reinterpret_cast<__nv_bfloat16*>(ws + CL.panel);
+  const __nv_bfloat16* A = static_cast<const __nv_bfloat16*>(hidden);
+  const __nv_bfloat16* B = static_cast<const __nv_bfloat16*>(W_head);
+  const int64_t Vp = padded_vocab(V);
+  const int32_t nvt = (int32_t)(Vp / 64);
+
+  // 1. chosen-token logits and the reference of the exponentials, all tokens
+  {
+    int64_t blocks = ceil_div<int64_t>(T, 8);
+    if (blocks > (int64_t)sms * 8) blocks = (int64_t)sms * 8;
+    KernelScope scope(SAPO_K_TARGET_LOGIT, st);
+    target_logit_kernel<<<(int)blocks, 256, 0, st>>>(A, ld_hidden, B, ld_W, ids, old_logp, T, H, V, zy, c2);
+  }
+  CUtensorMap map_w_kmajor, map_w_mn;
+  if (!make_map(&map_w_kmajor, B, H, V, ld_W, 128) || !make_map(&map_w_mn, B, H, V, ld_W, 128))
+    return SAPO_ERR_CUDA;
+
+  for (int64_t t0 = 0; t0 < T; t0 += chunk_rows) {
+    const int64_t tc = (T - t0) < chunk_rows ? (T - t0) : chunk_rows;
+    const __nv_bfloat16* A0 = A + t0 * ld_hidden;
+    const int64_t panel_rows = ceil_div<int64_t>(tc, BM) * nvt * BM;
+    CUtensorMap map_h_kmajor, map_hs_mn, map_p_two, map_p_tile;
+    if (!make_map(&map_h_kmajor, A0, H, tc, ld_hidden, BM) || !make_map(&map_hs_mn, hs, H, tc, H, 128) ||
+        !make_map(&map_p_two, panel, 64, panel_rows, 64, 256) ||
+        !make_map(&map_p_tile, panel, 64, panel_rows, 64, BM))
+      return SAPO_ERR_CUDA;
+    // 2. exponentials of the chunk -> panel, their sums per token and vocab split
+    int n_splits = fwd_splits(tc, V, H, sms);
+    if (n_splits > FUSED_MAX_SPLITS) n_splits = FUSED_MAX_SPLITS;
+    Sched fs = make_sched(tc, V, H, n_splits, /*m_fastest=*/true, /*tile_align=*/64);
+    fs.n_cover = (int32_t)Vp;
+    {
+      ExpEpi::Params ep{c2 + t0, ps, tc, V, nvt};
+      int rc = launch_gemm<0, false, ExpEpi>(map_h_kmajor, map_w_kmajor, map_p_tile, fs, ep, status, st, SAPO_K_FWD_EXP);
+      if (rc != SAPO_OK) return rc;
+    }
+    // 3. per-token loss terms, row scales, the chosen-token entries of the panel, scaled hidden rows
+    {
+      FusedTailArgs ta{};
+      ta.ps = ps; ta.n_parts = 2 * fs.units_per_m; ta.t0 = t0; ta.tc = tc;
+      ta.zy = zy; ta.c2 = c2; ta.ids = ids; ta.V = V; ta.old_logp = old_logp; ta.adv = adv;
+      ta.cu = cu_seqlens; ta.S = S; ta.T = T;
+      ta.lo_edge = 1.f - h_cfg->eps_low; ta.hi_edge = 1.f + h_cfg->eps_high; ta.grad_scale = h_cfg->grad_scale;
+      ta.loss_agg = h_cfg->loss_agg; ta.kl_beta = h_cfg->kl_beta; ta.ref_logp = h_cfg->ref_logp;
+      ta.logp = logp; ta.lse = lse; ta.ratio = ratio; ta.surr = surr; ta.gscale = gscale; ta.obj = obj;
+      ta.row_scale = row_scale; ta.panel = panel; ta.nvt = nvt;
+      ta.hidden = A; ta.ldh = ld_hidden; ta.H = H; ta.hs = hs; ta.status = status;
+      int64_t blocks = ceil_div<int64_t>(tc, 8);
+      if (blocks > (int64_t)sms * 8) blocks = (int64_t)sms * 8;
+      KernelScope scope(SAPO_K_FUSED_TAIL, st);
+      fused_tail_kernel<<<(int)blocks, 256, 0, st>>>(ta);
+    }
+    // 4. dhidden[t0:t0+tc] = a_t (e' . W)     (M = tokens, N = H, K = V)
+    {
+      Sched sched = make_sched(tc, H, Vp, 0, /*m_fastest=*/false);
+      sched.panel_nvt = nvt;
+      StoreEpi::Params ep{dhidden + t0 * (int64_t)H, H, tc, H, 0, partials, nullptr, row_scale};
+      int rc = launch_gemm<2, true, StoreEpi>(map_p_two, map_w_mn, map_p_two, sched, ep, status, st, SAPO_K_BWD_DH);
+      if (rc != SAPO_OK) return rc;
+    }
+    // 5. dW (+)= e'^T . (a_t h_t)            (M = V, N = H, K = tokens)
+    {
+      Sched sched = make_sched(V, H, tc, 0, /*m_fastest=*/false);
+      sched.panel_nvt = nvt;
+      StoreEpi::Params ep{dW_head, H, V, H, (t0 > 0 || accumulate_dW) ? 1 : 0, partials, nullptr, nullptr};
+      int rc = launch_gemm<3, true, StoreEpi>(map_p_tile, map_hs_mn, map_p_tile, sched, ep, status, st, SAPO_K_BWD_DW);
+      if (rc != SAPO_OK) return rc;
+    }
+  }
+  // 6. per-sequence means and the loss
+  const int seq_blocks = S < sms * 8 ? S : sms * 8;
+  { KernelScope scope(SAPO_K_LOSS_TAIL, st); seq_mean_kernel<<<seq_blocks, 256, 0, st>>>(obj, cu_seqlens, S, seq_out); }
+  { KernelScope scope(SAPO_K_LOSS_FINAL, st); loss_final_kernel<<<1, 256, 0, st>>>(seq_out, cu_seqlens, S, T, h_cfg->loss_agg, loss); }
+  return check_launch();
 }
 
 #ifdef SAPO_WAIT_STATS

@@ -43,7 +43,8 @@ class PolicyScorer:
 
     def __init__(self, W_head: torch.Tensor, max_tokens: int, max_seqs: int, max_questions: int,
                  eps_low: float = 0.2, eps_high: float = 0.28, adv_eps: float = 1e-6,
-                 ddof: int = 0, grad_scale: float = 1.0, device="cuda", active_backward: bool = False):
+                 ddof: int = 0, grad_scale: float = 1.0, device="cuda", active_backward: bool = False,
+                 backward: Optional[str] = None):
         if not torch.cuda.is_available():
             raise B.SapoError("PolicyScorer needs a CUDA device; there is no CPU path")
         B.load()
@@ -61,9 +62,17 @@ class PolicyScorer:
         self.dhidden = torch.empty(self.max_tokens, self.H, dtype=torch.float32, device=device)
         self.dW = torch.empty(self.V, self.H, dtype=torch.float32, device=device)
         nf = B.sapo_workspace_bytes(B.WS_FWD, self.max_tokens, self.H, self.V, self.dcode)
-        self.active_backward = bool(active_backward)   # contract only tokens with a non-zero gradient factor
-        nb = B.sapo_workspace_bytes(B.WS_BWD_ACTIVE if self.active_backward else B.WS_BWD,
-                                    self.max_tokens, self.H, self.V, self.dcode)
+        # how the gradients are formed: "dense" = forward call, then the backward call that
+        # recomputes the logits; "active" = the same over tokens with a non-zero gradient factor
+        # only; "fused" = one call that passes over the logits once (bf16 operands)
+        self.backward = backward if backward is not None else ("active" if active_backward else "dense")
+        if self.backward not in ("dense", "active", "fused"):
+            raise ValueError(f"unknown backward mode {self.backward!r}")
+        self.active_backward = self.backward == "active"
+        which = {"dense": B.WS_BWD, "active": B.WS_BWD_ACTIVE, "fused": B.WS_FUSED}[self.backward]
+        nb = B.sapo_workspace_bytes(which, self.max_tokens, self.H, self.V, self.dcode)
+        if nb == 0:
+            raise B.SapoError(f"backward mode {self.backward!r} does not support these operands")
         self.n_active = torch.zeros(1, dtype=torch.int32, device=device)
         # forward and backward never overlap on the stream, so they share one scratch buffer
         self.workspace = torch.empty(max(nf + 4 * self.max_seqs + 256, nb), dtype=torch.uint8, device=device)
@@ -81,6 +90,11 @@ class PolicyScorer:
         B.sapo_group_advantages(p["rewards"], go, self.adv_eps, self.ddof, self.adv, None, None,
                                 self.status)
         cu = p["cu_seqlens"][:S + 1]
+        if self.backward == "fused":
+            B.sapo_policy_loss_fwd_bwd(p["hidden"], self.W, p["ids"], p["old_logp"], self.adv, cu,
+                                       self.eps_low, self.eps_high, self.grad_scale, self.fwd,
+                                       self.dhidden, self.dW, False, self.workspace, self.status, T=T)
+            return StepResult(self.fwd["loss"], self.fwd, self.dhidden, self.dW, p, self.adv)
         B.sapo_policy_loss_fwd(p["hidden"], self.W, p["ids"], p["old_logp"], self.adv, cu,
                                self.eps_low, self.eps_high, self.grad_scale, self.fwd,
                                self.workspace, self.status, T=T)

@@ -36,9 +36,14 @@ def test_host_side_helpers():
     fwd = B.sapo_workspace_bytes(B.WS_FWD, T, H, V, B.DTYPE_BF16)
     assert fwd >= 3 * 4 * T and fwd % 256 == 0
     bwd = B.sapo_workspace_bytes(B.WS_BWD, T, H, V, B.DTYPE_BF16)
-    k_split_scratch = 2 * 96 * 256 * 256 * 4              # partial accumulator tiles, two per CTA pair
+    k_split_scratch = 3 * 96 * 256 * 256 * 4              # partial accumulator tiles of K-split parts
     assert bwd == T * V * 2 + k_split_scratch            # V is already a multiple of 128
     assert B.sapo_workspace_bytes_min(B.WS_BWD, T, H, V, B.DTYPE_BF16) == 128 * V * 2 + k_split_scratch
+    # single-pass call: the panel plus, per token, a scaled hidden row and a few floats
+    fused = B.sapo_workspace_bytes(B.WS_FUSED, T, H, V, B.DTYPE_BF16)
+    assert T * (V + H) * 2 + k_split_scratch < fused < T * (V + H) * 2 + k_split_scratch + 2000 * T
+    assert 0 < B.sapo_workspace_bytes_min(B.WS_FUSED, T, H, V, B.DTYPE_BF16) < fused // 10
+    assert B.sapo_workspace_bytes(B.WS_FUSED, T, H, V, B.DTYPE_F32) == 0       # bf16 operands only
     assert B.sapo_workspace_bytes(B.WS_FWD, T, 12, V, B.DTYPE_BF16) == 0      # H % 8 != 0
     assert B.sapo_workspace_bytes(7, T, H, V, B.DTYPE_BF16) == 0
     f32 = B.sapo_workspace_bytes(B.WS_FWD, 1024, 64, 1000, B.DTYPE_F32)

@@ -1,0 +1,160 @@
+"""The single-pass call sapo_policy_loss_fwd_bwd against the fp64 oracle, element by element,
+under the same tolerances as the separate forward and backward calls, and against those
+calls themselves."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import sapo_oracle as orc
+from paper_2509_08721_b200 import binding as B
+from paper_2509_08721_b200 import inputs as gen
+from tests import util as U
+from tests.test_gpu_parity import small_recipe
+
+pytestmark = pytest.mark.gpu
+
+
+def oracle_case(batch, eps_low, eps_high, grad_scale=1.0, noise_scale=1.0, **variant):
+    batch.built.logp_noise *= np.float32(noise_scale)
+    gen.install_old_logp(batch, U.oracle_current_logp(batch))
+    b = batch.built
+    adv = orc.group_advantages(b.rewards, b.group_offsets, adv_eps=float(np.float32(batch.adv_eps)))["adv"]
+    h, W = gen.as_f32(b.hidden), gen.as_f32(batch.W)
+    ref = orc.policy_loss_fwd(h, W, b.ids, b.old_logp, adv, b.cu_seqlens, eps_low, eps_high,
+                              grad_scale=grad_scale, **variant)
+    ref.update(orc.policy_loss_bwd(h, W, b.ids, ref["lse"], ref["gscale"]))
+    return adv, ref
+
+
+def device_inputs(batch, adv):
+    b = batch.built
+    return (U.to_torch(b.hidden), U.to_torch(batch.W), U.to_torch(b.ids), U.to_torch(b.old_logp),
+            U.to_torch(adv.astype(np.float32)), U.to_torch(b.cu_seqlens))
+
+
+def check_all(out, ref, adv, batch, eps_low, eps_high, extra_scale=0.0):
+    assert out["status"] == 0
+    U.check_forward(out, ref, adv, batch.built.cu_seqlens, eps_low, eps_high)
+    seq = out["seq_surr"].cpu().numpy().astype(np.float64)
+    scale = np.abs(adv).max() + extra_scale + 1e-30
+    assert np.max(np.abs(seq - ref["seq_surr"])) <= 1e-3 * scale
+    if extra_scale == 0.0:
+        U.check_loss(float(out["loss"].item()), ref["loss"], adv)
+    else:
+        assert abs(out["loss"].item() - ref["loss"]) <= 1e-3 * abs(ref["loss"]) + 1e-5 * scale
+    e_h = U.rel_fro(out["dhidden"].cpu().numpy(), ref["dhidden"])
+    e_w = U.rel_fro(out["dW"].cpu().numpy(), ref["dW"])
+    assert e_h <= U.TOL_GRAD_FRO and e_w <= U.TOL_GRAD_FRO, (e_h, e_w)
+
+
+SHAPES = [
+    ("one_tile", small_recipe(H=64, V=200, Q=2, length_law=("uniform", 3, 20))),
+    ("vocab_tail", small_recipe(H=64, V=1000)),
+    ("k_tail", small_recipe(H=72, V=777, Q=4, length_law=("uniform", 20, 90))),
+    ("many_tiles", small_recipe(H=328, V=2500, Q=6, I=3, J=3, length_law=("uniform", 30, 120))),
+    ("single_tokens", small_recipe(H=128, V=300, Q=4, length_law=("fixed", 1))),
+    ("one_group", small_recipe(H=64, V=520, Q=1, I=3, J=0)),
+    ("k_split", small_recipe(H=128, V=20000, Q=2, length_law=("uniform", 50, 90))),
+    ("k_split_rounds", small_recipe(H=512, V=8192, Q=8, length_law=("uniform", 150, 230))),
+]
+
+
+@pytest.mark.parametrize("name,recipe", SHAPES, ids=[c[0] for c in SHAPES])
+def test_fused_matches_oracle_small_shapes(name, recipe):
+    batch = gen.make_batch(recipe, 21)
+    adv, ref = oracle_case(batch, 0.2, 0.28, noise_scale=3.0)
+    out = U.gpu_scores_fused(*device_inputs(batch, adv), 0.2, 0.28)
+    check_all(out, ref, adv, batch, 0.2, 0.28)
+
+
+def test_fused_with_a_minimal_workspace_runs_in_token_chunks():
+    """A workspace for one 128-token panel: the batch goes through in chunks, sequences are cut
+    by chunk boundaries and dW_head is accumulated over the chunks."""
+    recipe = small_recipe(H=64, V=520, Q=4, length_law=("uniform", 60, 120))
+    batch = gen.make_batch(recipe, 33)
+    assert batch.T > 512
+    adv, ref = oracle_case(batch, 0.2, 0.28, noise_scale=2.0)
+    nbytes = B.sapo_workspace_bytes_min(B.WS_FUSED, batch.T, 64, 520, B.DTYPE_BF16)
+    assert 0 < nbytes < B.sapo_workspace_bytes(B.WS_FUSED, batch.T, 64, 520, B.DTYPE_BF16)
+    out = U.gpu_scores_fused(*device_inputs(batch, adv), 0.2, 0.28, workspace_bytes=nbytes)
+    check_all(out, ref, adv, batch, 0.2, 0.28)
+    # chunking changes the per-token outputs and dhidden by summation order at most
+    whole = U.gpu_scores_fused(*device_inputs(batch, adv), 0.2, 0.28)
+    for k in ("logp", "lse", "ratio", "surr", "gscale", "seq_surr", "loss", "dhidden"):
+        assert torch.allclose(out[k], whole[k], rtol=1e-5, atol=1e-7), k
+
+
+@pytest.mark.parametrize("loss_agg,kl_beta", [(1, 0.0), (1, 0.25)])
+def test_fused_loss_variants(loss_agg, kl_beta):
+    recipe = gen.Recipe("var", gen.DTYPE_BF16, 128, 2000, 4, 2, 2, ("uniform", 10, 90), ("bernoulli", 0.5))
+    batch = gen.make_batch(recipe, 61)
+    cur = U.oracle_current_logp(batch)
+    rng = np.random.default_rng(3)
+    ref_lp = (cur + rng.normal(size=batch.T).astype(np.float32) * np.float32(0.2)).astype(np.float32)
+    adv, ref = oracle_case(batch, 0.2, 0.28, grad_scale=1.5, loss_agg=loss_agg, kl_beta=kl_beta,
+                           ref_logp=ref_lp)
+    out = U.gpu_scores_fused(*device_inputs(batch, adv), 0.2, 0.28, grad_scale=1.5, loss_agg=loss_agg,
+                             kl_beta=kl_beta, ref_logp=U.to_torch(ref_lp) if kl_beta else None)
+    check_all(out, ref, adv, batch, 0.2, 0.28, extra_scale=kl_beta)
+
+
+def test_fused_agrees_with_the_separate_calls_and_repeats_bit_for_bit():
+    r = gen.config(3, length_div=16)
+    recipe = gen.Recipe(**{**r.__dict__, "H": 128, "V": 3000, "Q": 8, "I": 2, "J": 2})
+    batch = gen.make_batch(recipe, 5)
+    adv, ref = oracle_case(batch, 0.2, 0.2)
+    args = device_inputs(batch, adv)
+    a = U.gpu_scores_fused(*args, 0.2, 0.2)
+    b = U.gpu_scores_fused(*args, 0.2, 0.2)
+    for k in ("logp", "lse", "ratio", "surr", "gscale", "seq_surr", "loss", "dhidden", "dW"):
+        assert torch.equal(a[k], b[k]), k
+    sep = U.gpu_scores(*args, 0.2, 0.2)
+    assert sep["status"] == 0 and a["status"] == 0
+    assert (a["logp"] - sep["logp"]).abs().max().item() <= 1e-4
+    assert U.rel_fro(a["dhidden"].cpu().numpy(), sep["dhidden"].double().cpu().numpy()) <= 1e-2
+    assert U.rel_fro(a["dW"].cpu().numpy(), sep["dW"].double().cpu().numpy()) <= 1e-2
+    # questions with equal rewards: no gradient from their tokens
+    go, cu = batch.built.group_offsets, batch.built.cu_seqlens
+    zero_q = [q for q in range(recipe.Q) if np.all(adv[go[q]:go[q + 1]] == 0)]
+    assert zero_q
+    for q in zero_q:
+        assert torch.all(a["dhidden"][int(cu[go[q]]):int(cu[go[q + 1]])] == 0)
+
+
+def test_fused_flags_bad_ids_and_stale_old_logp():
+    recipe = small_recipe(H=64, V=400, Q=2, length_law=("uniform", 20, 40))
+    batch = gen.make_batch(recipe, 9)
+    adv, ref = oracle_case(batch, 0.2, 0.28)
+    hidden, W, ids, old, advd, cu = device_inputs(batch, adv)
+    ids_bad = ids.clone(); ids_bad[3] = 400; ids_bad[7] = -1
+    out = U.gpu_scores_fused(hidden, W, ids_bad, old, advd, cu, 0.2, 0.28)
+    assert out["status"] == 0x10
+    assert out["gscale"][3].item() == 0 and out["gscale"][7].item() == 0
+    assert torch.all(out["dhidden"][3] == 0) and torch.all(out["dhidden"][7] == 0)
+    assert torch.isfinite(out["dW"]).all() and torch.isfinite(out["dhidden"]).all()
+    keep = np.ones(batch.T, dtype=bool); keep[[3, 7]] = False
+    assert np.max(np.abs(out["logp"].cpu().numpy()[keep] - ref["logp"][keep])) <= U.TOL_LOGP_ABS
+    # an old log-prob 200 nats below the current one: exp(z - c) leaves the safe range
+    old_stale = old.clone(); old_stale[5] -= 200.0
+    out = U.gpu_scores_fused(hidden, W, ids, old_stale, advd, cu, 0.2, 0.28)
+    assert out["status"] == 0x80
+    assert out["gscale"][5].item() == 0 and torch.all(out["dhidden"][5] == 0)
+    assert torch.isfinite(out["dW"]).all() and torch.isfinite(out["dhidden"]).all()
+
+
+def test_fused_argument_errors():
+    x = torch.zeros(8, 16, dtype=torch.float32, device="cuda")
+    W = torch.zeros(16, 16, dtype=torch.float32, device="cuda")
+    i = torch.zeros(8, dtype=torch.int32, device="cuda")
+    f = torch.zeros(8, device="cuda")
+    cu = torch.tensor([0, 8], dtype=torch.int32, device="cuda")
+    ws = torch.empty(1 << 20, dtype=torch.uint8, device="cuda")
+    out = B.alloc_fwd_outputs(8, 1)
+    dH, dW = torch.empty(8, 16, device="cuda"), torch.empty(16, 16, device="cuda")
+    with pytest.raises(B.SapoError, match="unsupported shape"):      # fp32 operands
+        B.sapo_policy_loss_fwd_bwd(x, W, i, f, f[:1], cu, 0.2, 0.2, 1.0, out, dH, dW, False, ws, B.new_status())
+    xb, Wb = x.bfloat16(), W.bfloat16()
+    with pytest.raises(B.SapoError, match="workspace too small"):
+        B.sapo_policy_loss_fwd_bwd(xb, Wb, i, f, f[:1], cu, 0.2, 0.2, 1.0, out, dH, dW, False, ws[:1024],
+                                   B.new_status())
+    assert B.sapo_workspace_bytes(B.WS_FUSED, 8, 16, 16, B.DTYPE_F32) == 0

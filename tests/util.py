@@ -108,6 +108,24 @@ def gpu_scores(hidden, W, ids, old_logp, adv, cu, eps_low, eps_high, grad_scale=
     return out
 
 
+def gpu_scores_fused(hidden, W, ids, old_logp, adv, cu, eps_low, eps_high, grad_scale=1.0,
+                     workspace_bytes: Optional[int] = None, **variant):
+    """Loss and gradients through the single-pass call; returns device tensors."""
+    T, H, V, S = hidden.shape[0], hidden.shape[1], W.shape[0], cu.numel() - 1
+    status = B.new_status()
+    out = B.alloc_fwd_outputs(T, S)
+    nbytes = (B.sapo_workspace_bytes(B.WS_FUSED, T, H, V, B.DTYPE_BF16)
+              if workspace_bytes is None else workspace_bytes)
+    ws = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
+    out["dhidden"] = torch.empty(T, H, dtype=torch.float32, device="cuda")
+    out["dW"] = torch.empty(V, H, dtype=torch.float32, device="cuda")
+    B.sapo_policy_loss_fwd_bwd(hidden, W, ids, old_logp, adv, cu, eps_low, eps_high, grad_scale, out,
+                               out["dhidden"], out["dW"], False, ws, status, **variant)
+    torch.cuda.synchronize()
+    out["status"] = int(status.item())
+    return out
+
+
 def rel_fro(x: np.ndarray, ref: np.ndarray) -> float:
     d = np.linalg.norm(np.asarray(x, dtype=np.float64) - ref)
     n = np.linalg.norm(ref)
