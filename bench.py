@@ -310,6 +310,22 @@ def run_ours(args):
     ms_e2e = timed(host_step, args.steps)
     scorer.check_status()
 
+    # beside the single-pass call: the same step through the separate forward and backward calls
+    # (the backward recomputes the logits), on the same device-resident inputs
+    separate = None
+    if args.backward == "fused":
+        scorer2 = PolicyScorer(W, T, S, recipe.Q, eps_low=batch.eps_low, eps_high=batch.eps_high,
+                               backward="dense")
+        sep_step = lambda: scorer2.step(local, ext, sel, T, S)
+        for _ in range(args.warmup):
+            sep_step()
+        n_sep = min(args.steps, 30)
+        ms_sep = timed(sep_step, n_sep)
+        scorer2.check_status()
+        separate = (ms_sep, n_sep)
+        del scorer2
+        torch.cuda.empty_cache()
+
     _, total_tokens = replicas.aggregate(0.0, float(T), device="cuda")
     ms_step = ms_total / args.steps
     value = replicas.throughput(ms_total, total_tokens, args.steps)
@@ -369,6 +385,14 @@ def run_ours(args):
             "gpu_launches": int(n_launches),
             "clocks": clocks,
         }
+        if separate is not None:
+            ms_sep, n_sep = separate
+            line["separate_calls"] = {
+                "what": "sapo_policy_loss_fwd then sapo_policy_loss_bwd (logits recomputed), same inputs",
+                "value": replicas.throughput(ms_sep, total_tokens, n_sep), "unit": UNIT,
+                "ms_per_step": ms_sep / n_sep, "steps": n_sep,
+                "tflops_algorithmic": f_alg / (ms_sep / n_sep / 1e3) / 1e12,
+                "tflops_executed": (2.0 * T * V * H + 6.0 * T * V * H) / (ms_sep / n_sep / 1e3) / 1e12}
         if world == 1:
             del scorer.workspace
             torch.cuda.empty_cache()
@@ -397,13 +421,16 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--hbm-only", action="store_true",
                     help="run only the scaled pack / advantages / Adam bandwidth measurement")
-    ap.add_argument("--backward", default="dense", choices=["dense", "active", "fused"],
+    ap.add_argument("--backward", default=None, choices=["dense", "active", "fused"],
                     help="dense: forward call, then the backward call that recomputes the logits; "
                          "active: the same over the tokens whose gradient factor is non-zero only; "
-                         "fused: one call that passes over the logits once (bf16 workloads)")
+                         "fused: one call that passes over the logits once (bf16 workloads; the default "
+                         "for them, with the separate calls timed beside it)")
     ap.add_argument("--length-div", type=int, default=1,
                     help="divide every completion length (a small case of the same kernels for profiling)")
     args = ap.parse_args()
+    if args.backward is None:
+        args.backward = "dense" if args.workload == 1 else "fused"
     if args.warmup < 3 and args.impl == "ours":
         args.warmup = 3
     if args.ref_tokens is None:

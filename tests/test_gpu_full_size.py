@@ -1,5 +1,6 @@
-"""Parity at the full workload sizes, in the launch configuration bench.py times
-(PolicyScorer: pack -> advantages -> forward -> backward with the default workspace).
+"""Parity at the full workload sizes, in the launch configurations bench.py times
+(PolicyScorer: pack -> advantages -> forward -> backward with the default workspace, and
+pack -> advantages -> the single-pass call).
 
 Workload 2 is small enough for the oracle to score every token's forward pass; gradients are
 checked on sampled rows.  Workloads 3-5 are checked on sampled whole sequences, on properties
@@ -18,9 +19,12 @@ from tests import util as U
 pytestmark = pytest.mark.gpu
 
 
-def run_scorer(batch, recipe):
+MODES = ["dense", "fused"]     # separate forward / backward calls; the single-pass call
+
+
+def run_scorer(batch, recipe, backward="dense"):
     scorer = PolicyScorer(_to_dev(batch.W, "cuda"), batch.T, batch.S, recipe.Q,
-                          eps_low=batch.eps_low, eps_high=batch.eps_high)
+                          eps_low=batch.eps_low, eps_high=batch.eps_high, backward=backward)
     scorer.make_host_batch(batch)
     res = scorer.step_from_host(batch.T, batch.S)
     torch.cuda.synchronize()
@@ -41,25 +45,38 @@ def check_gradient_invariants(res, hidden_dev, W_dev, T):
     assert abs(a - b) <= 2e-3 * size, (a, b, size)
 
 
-def test_workload2_full_size():
-    recipe = gen.config(2)
-    batch = gen.make_batch(recipe, 2000)
-    T, S = batch.T, batch.S
-    b = batch.built
-    h = gen.as_f32(b.hidden)
-    W = gen.as_f32(batch.W)
-    W64 = W.astype(np.float64)
-    lse, logp = np.zeros(T), np.zeros(T)
-    for a in range(0, T, 1024):
-        e = min(T, a + 1024)
-        lp = orc.token_logprobs(h[a:e], W64, b.ids[a:e])
-        lse[a:e], logp[a:e] = lp["lse"], lp["logp"]
-    gen.install_old_logp(batch, logp.astype(np.float32))
-    adv = orc.group_advantages(b.rewards, b.group_offsets, adv_eps=float(np.float32(1e-6)))["adv"]
-    ref = orc.surrogate_from_logp(logp, b.old_logp, adv, b.cu_seqlens, batch.eps_low, batch.eps_high)
-    ref["logp"], ref["lse"] = logp, lse
+_W2 = {}
 
-    scorer, res = run_scorer(batch, recipe)
+
+def workload2_reference():
+    """The batch and the oracle's forward pass over all of its tokens (computed once per run)."""
+    if not _W2:
+        recipe = gen.config(2)
+        batch = gen.make_batch(recipe, 2000)
+        T, b = batch.T, batch.built
+        h = gen.as_f32(b.hidden)
+        W64 = gen.as_f32(batch.W).astype(np.float64)
+        lse, logp = np.zeros(T), np.zeros(T)
+        for a in range(0, T, 1024):
+            e = min(T, a + 1024)
+            lp = orc.token_logprobs(h[a:e], W64, b.ids[a:e])
+            lse[a:e], logp[a:e] = lp["lse"], lp["logp"]
+        gen.install_old_logp(batch, logp.astype(np.float32))
+        adv = orc.group_advantages(b.rewards, b.group_offsets, adv_eps=float(np.float32(1e-6)))["adv"]
+        ref = orc.surrogate_from_logp(logp, b.old_logp, adv, b.cu_seqlens, batch.eps_low, batch.eps_high)
+        ref["logp"], ref["lse"] = logp, lse
+        _W2.update(recipe=recipe, batch=batch, h=h, W64=W64, adv=adv, ref=ref)
+    return _W2
+
+
+@pytest.mark.parametrize("backward", MODES)
+def test_workload2_full_size(backward):
+    w2 = workload2_reference()
+    recipe, batch, h, W64, adv, ref = (w2[k] for k in ("recipe", "batch", "h", "W64", "adv", "ref"))
+    T, S, b = batch.T, batch.S, batch.built
+    lse = ref["lse"]
+
+    scorer, res = run_scorer(batch, recipe, backward)
     # pack, bit for bit
     assert np.array_equal(U.to_numpy(res.packed["hidden"])[:T], b.hidden)
     assert np.array_equal(U.to_numpy(res.packed["ids"])[:T], b.ids)
@@ -85,9 +102,10 @@ def test_workload2_full_size():
 FULL = [(3, None, 1200), (4, None, 500), (5, 0.75, 1500), (5, 0.0, 1500)]
 
 
+@pytest.mark.parametrize("backward", MODES)
 @pytest.mark.parametrize("number,ext_fraction,sample_tokens", FULL,
                          ids=["cfg3", "cfg4", "cfg5_J6", "cfg5_J0"])
-def test_workloads_3_to_5_full_size_sampled(number, ext_fraction, sample_tokens):
+def test_workloads_3_to_5_full_size_sampled(number, ext_fraction, sample_tokens, backward):
     recipe = gen.config(number, ext_fraction=ext_fraction)
     batch = gen.make_batch(recipe, 1000 * number)
     T, S = batch.T, batch.S
@@ -98,7 +116,7 @@ def test_workloads_3_to_5_full_size_sampled(number, ext_fraction, sample_tokens)
     gen.install_old_logp(batch, cur)
     adv = orc.group_advantages(b.rewards, b.group_offsets, adv_eps=float(np.float32(1e-6)))["adv"]
 
-    scorer, res = run_scorer(batch, recipe)
+    scorer, res = run_scorer(batch, recipe, backward)
     assert np.array_equal(U.to_numpy(res.packed["ids"])[:T], b.ids)
     assert np.array_equal(U.to_numpy(res.packed["cu_seqlens"])[:S + 1], b.cu_seqlens)
     assert np.allclose(res.adv[:S].cpu().numpy(), adv, rtol=2e-7, atol=1e-9)
