@@ -344,10 +344,11 @@ def run_ours(args):
         flops_each = 2.0 * (T if top in ("fwd_gemm", "fwd_exp") else t_act) * V * H
         achieved = flops_each / per_step / (ms_top / 1e3) / 1e12
         # DRAM bytes per launch from the ncu capture of a small case of the same kernels
-        # (profiles/umma_gemm_kernels_workload2_lengths_div4.md): fixed part + bytes per token.
+        # (profiles/umma_gemm_kernels_*_workload2_lengths_div4.md): fixed part + bytes per token.
         # Only valid for hidden 896 / vocab 151936, the shape that capture ran at.
         ncu_traffic = {"fwd_gemm": (0.272e9, 12.4e3), "bwd_dz": (0.272e9, 299.6e3),
-                       "bwd_dh": (0.272e9, 310.8e3), "bwd_dw": (0.515e9, 332.3e3)}
+                       "fwd_exp": (0.272e9, 309.0e3), "bwd_dh": (0.272e9, 310.7e3),
+                       "bwd_dw": (0.515e9, 327.4e3)}
         traffic = None
         if (H, V) == (896, 151936) and top in ncu_traffic:
             fixed, per_token = ncu_traffic[top]
