@@ -60,6 +60,9 @@ struct Sched {
   // in order.
   int32_t dp_units, sk_tiles, sk_parts;
   int32_t k_split_ok; // the epilogue has scratch for K-split parts
+  int32_t part_ld;    // columns of a partial tile in scratch (256, or 512 for the two-accumulator kernel)
+  int32_t max_parts;  // partial tiles of that width the scratch holds
+  int32_t min_part_k; // shortest K range (in stages) worth a part
   // A size only the device knows (the number of active tokens after compaction), read by
   // every CTA at start-up: dyn_dim 1 = it is M (rows), 2 = it is K (contraction length).
   const int32_t* dyn_count;
@@ -71,6 +74,8 @@ struct Sched {
 constexpr int PARTIAL_FLOATS = PAIR_M * BN;   // one partial accumulator tile: 256 x 256 fp32
 constexpr int MAX_PAIRS_SCRATCH = 96;          // CTA pairs a launch may use (a B200 has 74)
 constexpr int MAX_PARTS_SCRATCH = 3 * MAX_PAIRS_SCRATCH;   // K-split parts the scratch holds
+// partial tiles are 256 rows by 256 columns, or by 512 for the wide-tile kernel: sized for those
+constexpr size_t KSPLIT_SCRATCH_BYTES = (size_t)MAX_PARTS_SCRATCH * 2 * PARTIAL_FLOATS * sizeof(float);
 
 // Decide whether (and how finely) to cut the tiles of a ragged last wave along K (see Sched).
 // With `rem` tiles left over and s parts per tile the tail takes ceil(rem s / pairs) / s of a
@@ -83,8 +88,8 @@ __host__ __device__ inline void split_last_wave(Sched& s, int pairs) {
   if (rem == 0) return;
   int best = 1; float best_cost = 1.f;
   for (int parts = 2; parts <= 8; ++parts) {
-    if (s.num_k_blocks / parts < 16) break;       // keep every range long enough to be worth a pipeline fill
-    if (rem * parts > MAX_PARTS_SCRATCH) break;
+    if (s.num_k_blocks / parts < s.min_part_k) break;   // keep every range long enough to be worth a pipeline fill
+    if (rem * parts > s.max_parts) break;
     const int rounds = (rem * parts + pairs - 1) / pairs;
     const float cost = (float)rounds / (float)parts + 0.02f * (float)rounds;
     if (cost < best_cost - 0.05f) { best_cost = cost; best = parts; }
@@ -387,9 +392,10 @@ struct StoreEpi {
   }
   // a K-split part of a tile goes to scratch slot `slot` instead: rows [128 rank, +128) of a
   // 256 x 256 fp32 tile, column 0 = the tile's first column
-  __device__ __forceinline__ void set_dest(const Params& p, int slot, int rank, int r, int n0_) {
+  __device__ __forceinline__ void set_dest(const Params& p, int slot, int rank, int r, int n0_, int part_ld) {
     n0 = n0_;
-    part = slot < 0 ? nullptr : p.partials + (size_t)slot * PARTIAL_FLOATS + (size_t)(rank * BM + r) * BN;
+    part = slot < 0 ? nullptr
+                    : p.partials + ((size_t)slot * PAIR_M + (size_t)(rank * BM + r)) * part_ld;
   }
   template <int HALF>
   __device__ __forceinline__ void chunk(const Params& p, float (&v)[32], int col0, const StageCtx&) {
@@ -429,19 +435,20 @@ streamk_fixup_kernel(const Sched s_arg, const StoreEpi::Params p_arg, int pairs)
   int pmb, un, n_begin, n_end;
   decode_unit(s, s.dp_units + t, pmb, un, n_begin, n_end);
   const int n0 = n_begin * s.tile_n;
-  const int col = threadIdx.x;
-  if (col >= s.tile_n || n0 + col >= p.N) return;
-  for (int rr = row_begin; rr < row_begin + 8; ++rr) {
-    int64_t row = (int64_t)pmb * PAIR_M + rr;
-    if (row >= p.M) break;
-    const float scale = p.row_scale != nullptr ? p.row_scale[row] : 1.f;
-    if (p.row_map != nullptr) row = p.row_map[row];
-    const size_t off = (size_t)rr * BN + col;
-    float sum = 0.f;
-    for (int j = 0; j < s.sk_parts; ++j) sum += p.partials[(size_t)(j * s.sk_tiles + t) * PARTIAL_FLOATS + off];
-    sum *= scale;
-    float* dst = p.C + row * p.ldc + n0 + col;
-    *dst = p.accumulate ? *dst + sum : sum;
+  const size_t part_floats = (size_t)PAIR_M * s.part_ld;
+  for (int col = threadIdx.x; col < s.tile_n && n0 + col < p.N; col += blockDim.x) {
+    for (int rr = row_begin; rr < row_begin + 8; ++rr) {
+      int64_t row = (int64_t)pmb * PAIR_M + rr;
+      if (row >= p.M) break;
+      const float scale = p.row_scale != nullptr ? p.row_scale[row] : 1.f;
+      if (p.row_map != nullptr) row = p.row_map[row];
+      const size_t off = (size_t)rr * s.part_ld + col;
+      float sum = 0.f;
+      for (int j = 0; j < s.sk_parts; ++j) sum += p.partials[(size_t)(j * s.sk_tiles + t) * part_floats + off];
+      sum *= scale;
+      float* dst = p.C + row * p.ldc + n0 + col;
+      *dst = p.accumulate ? *dst + sum : sum;
+    }
   }
 }
 
@@ -640,7 +647,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
     int pmb, un, n_begin, n_end, kb0, kb1, slot;
     while (ok && work.next(pmb, un, n_begin, n_end, kb0, kb1, slot)) {
       epi.begin_unit(ep, 2 * pmb + (int)rank, r);
-      if constexpr (Epi::STREAMK) epi.set_dest(ep, slot, (int)rank, r, n_begin * sched.tile_n);
+      if constexpr (Epi::STREAMK) epi.set_dest(ep, slot, (int)rank, r, n_begin * sched.tile_n, sched.part_ld);
       for (int nb = n_begin; ok && nb < n_end; ++nb) {
         if (!SAPO_TIMED(3, mbar_wait(&acc_full[acc], acc_phase, abort_flag))) { ok = false; break; }
         fence_after_sync();
@@ -687,6 +694,206 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
   }
 
   // neither CTA may leave while the other can still touch its shared or tensor memory
+  fence_before_sync();
+  __syncthreads();
+  cluster_sync_all();
+  if (warp == 1) { fence_after_sync(); tmem_dealloc_pair(tmem_base, TMEM_COLS); }
+  if (threadIdx.x == 0 && *abort_flag) raise_status(status, SAPO_ST_WAIT_TIMEOUT);
+}
+
+// ---------------------------------------------------------------------------- the wide-tile GEMM kernel
+// The two long-K contractions of the backward pass (dhidden: K = vocabulary, dW_head: K = tokens)
+// read the panel as A and an [K, N] matrix (W_head or hidden rows) as B, and store fp32.  Their
+// tiles are long enough that the epilogue need not overlap the next tile's MMAs, so both
+// accumulators of tensor memory can serve one tile: a pair works on a 256 x (2 tn) tile
+// (tn <= 256) whose two halves share every A stage.  Per flop that is a quarter fewer operand
+// bytes into shared memory than 256 x 256 tiles, which is what bounds these contractions.
+//   A_KIND 2: A = panel read K-major  (M = tokens, K = vocab): one [128 token x 64 vocab] tile per stage
+//   A_KIND 3: A = panel read MN-major (M = vocab, K = tokens): 64-token halves of two tiles per stage
+//   B is stored [K, N], N contiguous: per accumulator, this CTA's tn/2 columns as 64-column boxes.
+// A stage holds a K depth of 64; four stages.  Work units, K-split parts and barriers as in
+// umma_gemm_kernel, with one accumulator barrier pair instead of two.
+constexpr int BK2 = 64;
+constexpr int STAGES2 = 4;
+constexpr uint32_t A2_STAGE_BYTES = BM * BK2 * 2;          // 16 KB
+constexpr uint32_t BOX2_BYTES = 64 * 128;                  // a 64-row box of 128-byte rows
+constexpr uint32_t B2_ACC_BYTES = 2 * BOX2_BYTES;          // up to 128 columns per accumulator and CTA
+constexpr uint32_t B2_STAGE_BYTES = 2 * B2_ACC_BYTES;      // 32 KB
+constexpr size_t GEMM2_SMEM_BYTES = 1024 + STAGES2 * (A2_STAGE_BYTES + B2_STAGE_BYTES) + 256;
+
+template <int A_KIND>
+__global__ void __launch_bounds__(GEMM_THREADS, 1)
+umma_gemm2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+                  const Sched sched_arg, const StoreEpi::Params ep_arg, int32_t* status) {
+  static_assert(A_KIND == 2 || A_KIND == 3, "panel operands only");
+  Sched sched = sched_arg;
+  StoreEpi::Params ep = ep_arg;
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  uint8_t* smem_a = smem;
+  uint8_t* smem_b = smem + STAGES2 * A2_STAGE_BYTES;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + STAGES2 * (A2_STAGE_BYTES + B2_STAGE_BYTES));
+  uint64_t* full = bars;                  // [STAGES2] TMA -> MMA          (even CTA's are used)
+  uint64_t* empty = bars + STAGES2;       // [STAGES2] MMA -> TMA          (each CTA waits on its own)
+  uint64_t* acc_full = bars + 2 * STAGES2;      // MMA -> epilogue         (each CTA waits on its own)
+  uint64_t* acc_empty = bars + 2 * STAGES2 + 1; // epilogue -> MMA         (even CTA's is used)
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * STAGES2 + 2);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  constexpr bool A_MN = A_KIND == 3;
+  const uint32_t rank = cluster_cta_rank();
+  const int pair = blockIdx.x >> 1, num_pairs = gridDim.x >> 1;
+  const int tn = sched.tile_n >> 1;       // columns per accumulator
+  const int half = tn >> 1;               // B columns per accumulator this CTA stages
+  const int b_boxes = (half + 63) >> 6;   // 64-column boxes per accumulator (1 or 2)
+
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < STAGES2; ++i) { mbar_init(&full[i], 1); mbar_init(&empty[i], 1); }
+    mbar_init(acc_full, 1); mbar_init(acc_empty, 16);
+    *abort_flag = 0;
+    fence_mbar_init();
+    prefetch_tensormap(&map_a);
+    prefetch_tensormap(&map_b);
+  }
+  if (warp == 1) { tmem_alloc_pair(tmem_slot, TMEM_COLS); tmem_relinquish_pair(); }
+  fence_before_sync();
+  __syncthreads();
+  cluster_sync_all();
+  fence_after_sync();
+  const uint32_t tmem_base = *tmem_slot;
+  const uint32_t full0_addr = map_to_cta(smem_u32(full), 0);
+  const uint32_t empty_addr[2] = {map_to_cta(smem_u32(empty), 0), map_to_cta(smem_u32(empty), 1)};
+  const uint32_t acc_full_addr[2] = {map_to_cta(smem_u32(acc_full), 0), map_to_cta(smem_u32(acc_full), 1)};
+  const uint32_t acc_empty0_addr = map_to_cta(smem_u32(acc_empty), 0);
+
+  if (warp == 0) {
+    // ------------------------------------------------------------ TMA producer (both CTAs)
+    int stage = 0; uint32_t phase = 0;
+    uint32_t in_flight = 0;
+    bool ok = true;
+    constexpr int A_BOXES = A_KIND == 2 ? 1 : 2;
+    const uint32_t tx = 2 * (A2_STAGE_BYTES + 2 * b_boxes * BOX2_BYTES);
+    const bool is_a = lane < A_BOXES;
+    const int bidx = lane - A_BOXES;                  // B box: accumulator bidx / b_boxes, box bidx % b_boxes
+    const bool mine = lane < A_BOXES + 2 * b_boxes;
+    const int bj = is_a ? 0 : bidx / b_boxes, bb = is_a ? 0 : bidx - bj * b_boxes;
+    WorkList work(sched, pair, num_pairs);
+    int pmb, un, n_begin, n_end, kb0, kb1, slot;
+    while (ok && work.next(pmb, un, n_begin, n_end, kb0, kb1, slot)) {
+      const int mb = 2 * pmb + (int)rank;
+      const int n0 = n_begin * sched.tile_n;
+      const int bcol = n0 + bj * tn + (int)rank * half + 64 * bb;      // first column of this lane's B box
+      for (int kb = kb0; kb < kb1; ++kb) {
+        if (!mbar_wait(&empty[stage], phase ^ 1, abort_flag)) { ok = false; break; }
+        if (rank == 0 && lane == 0) mbar_arrive_expect_tx(&full[stage], tx);
+        if (mine) {
+          const uint32_t bar = full0_addr + stage * 8;
+          if (is_a) {
+            uint8_t* dst = smem_a + stage * A2_STAGE_BYTES + lane * BOX2_BYTES;
+            if (A_KIND == 2)      // vocab tile kb of token block mb
+              tma_load_2d_pair(dst, &map_a, bar, 0, (mb * sched.panel_nvt + kb) * BM);
+            else                  // tokens [64 kb, +64): half of token block kb / 2, vocab tile 2 mb + lane
+              tma_load_2d_pair(dst, &map_a, bar, 0,
+                               ((kb >> 1) * sched.panel_nvt + 2 * mb + lane) * BM + (kb & 1) * 64);
+          } else {
+            uint8_t* dst = smem_b + stage * B2_STAGE_BYTES + bj * B2_ACC_BYTES + bb * BOX2_BYTES;
+            tma_load_2d_pair(dst, &map_b, bar, bcol, kb * BK2);
+          }
+        }
+        in_flight |= 1u << stage;
+        if (++stage == STAGES2) { stage = 0; phase ^= 1; }
+      }
+    }
+    if (!ok && rank == 0 && lane == 0) {
+      for (int i = 0; i < STAGES2; ++i) {
+        if (!(in_flight & (1u << i))) continue;
+        const uint32_t ph = (i < stage) ? phase : (phase ^ 1);
+        for (int spin = 0; spin < (1 << 20) && !mbar_try_wait(&full[i], ph); ++spin) {}
+      }
+    }
+  } else if (warp == 1 && lane == 0 && rank == 0) {
+    // ------------------------------------------------------------ MMA issuer (even CTA only)
+    int stage = 0; uint32_t phase = 0;
+    uint32_t acc_phase = 0;
+    bool ok = true;
+    const uint32_t idesc = make_idesc_bf16(PAIR_M, tn, A_MN, true);
+    WorkList work(sched, pair, num_pairs);
+    int pmb, un, n_begin, n_end, kb0, kb1, slot;
+    while (ok && work.next(pmb, un, n_begin, n_end, kb0, kb1, slot)) {
+      if (!mbar_wait(acc_empty, acc_phase ^ 1, abort_flag)) { ok = false; break; }
+      fence_after_sync();
+      for (int kb = kb0; kb < kb1; ++kb) {
+        if (!mbar_wait(&full[stage], phase, abort_flag)) { ok = false; break; }
+        fence_after_sync();
+        const uint32_t a_addr = smem_u32(smem_a + stage * A2_STAGE_BYTES);
+        const uint32_t b_addr = smem_u32(smem_b + stage * B2_STAGE_BYTES);
+        #pragma unroll
+        for (int k = 0; k < BK2 / UMMA_K; ++k) {
+          const uint64_t a_desc = A_MN ? make_smem_desc(a_addr + k * 2048, BOX2_BYTES, 1024)
+                                       : make_smem_desc(a_addr + k * 32, 16, 1024);
+          const uint32_t acc_on = (kb > kb0 || k != 0) ? 1u : 0u;
+          mma_bf16_pair(tmem_base, a_desc, make_smem_desc(b_addr + k * 2048, BOX2_BYTES, 1024), idesc, acc_on);
+          mma_bf16_pair(tmem_base + BN, a_desc,
+                        make_smem_desc(b_addr + B2_ACC_BYTES + k * 2048, BOX2_BYTES, 1024), idesc, acc_on);
+        }
+        mma_commit_pair(empty_addr[0] + stage * 8);
+        mma_commit_pair(empty_addr[1] + stage * 8);
+        if (++stage == STAGES2) { stage = 0; phase ^= 1; }
+      }
+      if (ok) {
+        mma_commit_pair(acc_full_addr[0]);
+        mma_commit_pair(acc_full_addr[1]);
+      }
+      acc_phase ^= 1;
+    }
+  } else if (warp >= 2) {
+    // ------------------------------------------------------------ epilogue (8 warps, both CTAs)
+    // warps 2-5 drain the first accumulator, warps 6-9 the second; one TMEM lane quadrant each
+    const int quad = warp & 3;
+    const int j = (warp - 2) >> 2;
+    const int r = quad * 32 + lane;
+    uint32_t acc_phase = 0;
+    bool ok = true;
+    StoreEpi epi;
+    StageCtx cx{};
+    WorkList work(sched, pair, num_pairs);
+    int pmb, un, n_begin, n_end, kb0, kb1, slot;
+    while (ok && work.next(pmb, un, n_begin, n_end, kb0, kb1, slot)) {
+      const int n0 = n_begin * sched.tile_n;
+      epi.begin_unit(ep, 2 * pmb + (int)rank, r);
+      epi.set_dest(ep, slot, (int)rank, r, n0, sched.part_ld);
+      if (!mbar_wait(acc_full, acc_phase, abort_flag)) { ok = false; break; }
+      fence_after_sync();
+      const uint32_t t_addr = tmem_base + (static_cast<uint32_t>(quad * 32) << 16) + j * BN;
+      const int chunks = (tn + 31) >> 5;
+      float va[32], vb[32];
+      tmem_ld32(t_addr, va);
+      for (int c = 0; c < chunks; c += 2) {
+        tmem_ld_wait();
+        if (c + 1 < chunks) tmem_ld32(t_addr + (c + 1) * 32, vb);
+        if (kb1 == kb0) {
+          #pragma unroll
+          for (int q = 0; q < 32; ++q) va[q] = 0.f;
+        }
+        epi.template chunk<0>(ep, va, n0 + j * tn + c * 32, cx);
+        if (c + 1 < chunks) {
+          tmem_ld_wait();
+          if (c + 2 < chunks) tmem_ld32(t_addr + (c + 2) * 32, va);
+          if (kb1 == kb0) {
+            #pragma unroll
+            for (int q = 0; q < 32; ++q) vb[q] = 0.f;
+          }
+          epi.template chunk<1>(ep, vb, n0 + j * tn + (c + 1) * 32, cx);
+        }
+      }
+      fence_before_sync();
+      __syncwarp();
+      if (lane == 0) mbar_arrive_cluster(acc_empty0_addr);
+      acc_phase ^= 1;
+    }
+  }
+
   fence_before_sync();
   __syncthreads();
   cluster_sync_all();
@@ -987,6 +1194,7 @@ static Sched make_sched(int64_t M, int64_t N, int64_t K, int n_splits, bool m_fa
   s.panel_nvt = 0;
   s.dp_units = s.num_units; s.sk_tiles = 0; s.sk_parts = 1;
   s.k_split_ok = 0; s.dyn_count = nullptr; s.dyn_dim = 0; s.skip_if_empty = 0;
+  s.part_ld = BN; s.max_parts = MAX_PARTS_SCRATCH; s.min_part_k = 16;
   return s;
 }
 
@@ -1071,6 +1279,105 @@ static int launch_gemm(const CUtensorMap& ma, const CUtensorMap& mb, const CUten
   return check_launch();
 }
 
+// Schedule of the wide-tile kernel: equal-width tiles of up to 512 columns (two accumulators),
+// 64-deep stages, partial tiles of 512 columns in the K-split scratch.
+static Sched make_sched_wide(int64_t M, int64_t N, int64_t K) {
+  Sched s = make_sched(M, N, K, 0, /*m_fastest=*/false);
+  const int64_t tiles = ceil_div<int64_t>(N, 2 * BN);
+  s.tile_n = (int32_t)round_up<int64_t>(ceil_div<int64_t>(N, tiles), 64);
+  s.num_n_blocks = (int32_t)ceil_div<int64_t>(N, s.tile_n);
+  s.n_per_unit = 1;
+  s.units_per_m = s.num_n_blocks;
+  s.num_units = s.num_m_blocks * s.units_per_m;
+  s.num_k_blocks = (int32_t)ceil_div<int64_t>(K, BK2);
+  s.dp_units = s.num_units;
+  s.part_ld = 2 * BN; s.max_parts = MAX_PARTS_SCRATCH; s.min_part_k = 32;
+  return s;
+}
+// the wide tiles pay off once the output is at least one full accumulator wide
+static bool use_wide_tiles(int32_t N) { return N >= BN; }
+
+template <int A_KIND>
+static int launch_gemm_wide(const CUtensorMap& ma, const CUtensorMap& mb, const Sched& sched,
+                            const StoreEpi::Params& ep, int32_t* status, cudaStream_t st, int kernel_id) {
+  auto kern = umma_gemm2_kernel<A_KIND>;
+  static int max_pairs = 0;
+  if (sched.num_units <= 0) return SAPO_OK;
+  Sched sc = sched;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+  cudaLaunchConfig_t cfg = {};
+  cfg.blockDim = dim3(GEMM_THREADS, 1, 1);
+  cfg.dynamicSmemBytes = GEMM2_SMEM_BYTES;
+  cfg.stream = st;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  if (max_pairs == 0) {
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)GEMM2_SMEM_BYTES) !=
+        cudaSuccess)
+      return SAPO_ERR_CUDA;
+    const int sms = sm_count();
+    if (sms <= 0) return SAPO_ERR_CUDA;
+    cfg.gridDim = dim3(sms & ~1, 1, 1);
+    int n = 0;
+    if (cudaOccupancyMaxActiveClusters(&n, kern, &cfg) != cudaSuccess || n <= 0) return SAPO_ERR_CUDA;
+    max_pairs = n < sms / 2 ? n : sms / 2;
+    if (max_pairs > MAX_PAIRS_SCRATCH) max_pairs = MAX_PAIRS_SCRATCH;
+  }
+  int pairs = sched.num_units < max_pairs ? sched.num_units : max_pairs;
+  sc.k_split_ok = ep.partials != nullptr ? 1 : 0;
+  split_last_wave(sc, max_pairs);
+  if (sc.sk_tiles > 0) pairs = max_pairs;
+  cfg.gridDim = dim3(2 * pairs, 1, 1);
+  {
+    KernelScope scope(kernel_id, st);
+    if (cudaLaunchKernelEx(&cfg, kern, ma, mb, sc, ep, status) != cudaSuccess) return SAPO_ERR_CUDA;
+  }
+  if (sc.sk_tiles > 0) {
+    KernelScope scope(SAPO_K_STREAMK_FIXUP, st);
+    streamk_fixup_kernel<<<sc.sk_tiles * 32, 256, 0, st>>>(sc, ep, pairs);
+  }
+  return check_launch();
+}
+
+// The two contractions over a filled panel (dz, or the exponentials of the single-pass call):
+//   dhidden[0:tc] = row_scale . (panel . W)       (M = tokens, N = H, K = vocabulary)
+//   dW_head   (+)= panel^T . X                    (M = vocabulary, N = H, K = tokens)
+// X is hidden (or its row-scaled copy), [tc, ldx].  Wide tiles when H allows.
+static int launch_grad_gemms(const __nv_bfloat16* panel, int64_t panel_rows, int32_t nvt,
+                             const __nv_bfloat16* W, int64_t ldw, const __nv_bfloat16* X, int64_t ldx,
+                             int64_t tc, int32_t H, int32_t V, int64_t Vp, float* dhidden,
+                             const float* row_scale, float* dW_head, int accumulate, float* partials,
+                             int32_t* status, cudaStream_t st) {
+  StoreEpi::Params ep_h{dhidden, H, tc, H, 0, partials, nullptr, row_scale};
+  StoreEpi::Params ep_w{dW_head, H, V, H, accumulate, partials, nullptr, nullptr};
+  if (use_wide_tiles(H)) {
+    CUtensorMap map_p_tile, map_p_half, map_w64, map_x64;
+    if (!make_map(&map_p_tile, panel, 64, panel_rows, 64, BM) || !make_map(&map_p_half, panel, 64, panel_rows, 64, 64) ||
+        !make_map(&map_w64, W, H, V, ldw, 64) || !make_map(&map_x64, X, H, tc, ldx, 64))
+      return SAPO_ERR_CUDA;
+    Sched sh = make_sched_wide(tc, H, Vp);
+    sh.panel_nvt = nvt;
+    int rc = launch_gemm_wide<2>(map_p_tile, map_w64, sh, ep_h, status, st, SAPO_K_BWD_DH);
+    if (rc != SAPO_OK) return rc;
+    Sched sw = make_sched_wide(V, H, tc);
+    sw.panel_nvt = nvt;
+    return launch_gemm_wide<3>(map_p_half, map_x64, sw, ep_w, status, st, SAPO_K_BWD_DW);
+  }
+  CUtensorMap map_p_two, map_p_tile, map_w_mn, map_x_mn;
+  if (!make_map(&map_p_two, panel, 64, panel_rows, 64, 256) || !make_map(&map_p_tile, panel, 64, panel_rows, 64, BM) ||
+      !make_map(&map_w_mn, W, H, V, ldw, 128) || !make_map(&map_x_mn, X, H, tc, ldx, 128))
+    return SAPO_ERR_CUDA;
+  Sched sh = make_sched(tc, H, Vp, 0, /*m_fastest=*/false);
+  sh.panel_nvt = nvt;
+  int rc = launch_gemm<2, true, StoreEpi>(map_p_two, map_w_mn, map_p_two, sh, ep_h, status, st, SAPO_K_BWD_DH);
+  if (rc != SAPO_OK) return rc;
+  Sched sw = make_sched(V, H, tc, 0, /*m_fastest=*/false);
+  sw.panel_nvt = nvt;
+  return launch_gemm<3, true, StoreEpi>(map_p_tile, map_x_mn, map_p_tile, sw, ep_w, status, st, SAPO_K_BWD_DW);
+}
+
 static int launch_split(const float* X, int64_t ld, int64_t R, int32_t H, __nv_bfloat16* out, int mode,
                         cudaStream_t st) {
   const int64_t n = R * (int64_t)H;
@@ -1110,7 +1417,7 @@ static BwdLayout bwd_layout(int64_t T, int32_t H, int32_t V, int32_t dtype) {
     L.a_hi = off; off += round_up<size_t>((size_t)T * H * 2, 256);
     L.b_hi = off; off += round_up<size_t>((size_t)V * H * 2, 256);
   }
-  L.partials = off; off += (size_t)MAX_PARTS_SCRATCH * PARTIAL_FLOATS * sizeof(float);
+  L.partials = off; off += KSPLIT_SCRATCH_BYTES;
   L.panel = off; L.fixed = off;
   L.bytes_per_row = (size_t)padded_vocab(V) * 2;
   return L;
@@ -1130,7 +1437,7 @@ static FusedLayout fused_layout(int64_t T, int32_t H, int32_t V, int32_t S) {
   L.c2 = take((size_t)T * 4);
   L.obj = take((size_t)T * 4);
   L.seq = take((size_t)(S > 0 ? S : 1) * 4);
-  L.partials = take((size_t)MAX_PARTS_SCRATCH * PARTIAL_FLOATS * sizeof(float));
+  L.partials = take(KSPLIT_SCRATCH_BYTES);
   L.fixed = off;
   // per chunk row: panel row, scaled hidden row, row scale, partial sums
   L.bytes_per_row = (size_t)padded_vocab(V) * 2 + (size_t)H * 2 + 4 + (size_t)2 * FUSED_MAX_SPLITS * 4;
@@ -1384,19 +1691,16 @@ extern "C" int sapo_policy_loss_bwd(const void* hidden, const void* W_head, int3
   const int64_t chunk_rows = rows_fit >= T ? T : rows_fit;
   if (chunk_rows <= 0) return SAPO_ERR_WORKSPACE_TOO_SMALL;
 
-  // W as the K-major B operand of the logit recompute and as the MN-major B operand of dH
-  CUtensorMap map_w_kmajor, map_w_mn;
-  if (!make_map(&map_w_kmajor, B, H, V, ldb, 128) || !make_map(&map_w_mn, B, H, V, ldb, 128))
-    return SAPO_ERR_CUDA;
+  // W as the K-major B operand of the logit recompute
+  CUtensorMap map_w_kmajor;
+  if (!make_map(&map_w_kmajor, B, H, V, ldb, 128)) return SAPO_ERR_CUDA;
 
   for (int64_t t0 = 0; t0 < T; t0 += chunk_rows) {
     const int64_t tc = (T - t0) < chunk_rows ? (T - t0) : chunk_rows;
     const __nv_bfloat16* A0 = A + t0 * lda;
     const int64_t panel_rows = ceil_div<int64_t>(tc, BM) * nvt * BM;   // 128-byte rows of the tiled panel
-    CUtensorMap map_h_kmajor, map_h_mn, map_p_two, map_p_tile;
-    if (!make_map(&map_h_kmajor, A0, H, tc, lda, BM) || !make_map(&map_h_mn, A0, H, tc, lda, 128) ||
-        !make_map(&map_p_two, panel, 64, panel_rows, 64, 256) ||
-        !make_map(&map_p_tile, panel, 64, panel_rows, 64, BM))
+    CUtensorMap map_h_kmajor, map_p_tile;
+    if (!make_map(&map_h_kmajor, A0, H, tc, lda, BM) || !make_map(&map_p_tile, panel, 64, panel_rows, 64, BM))
       return SAPO_ERR_CUDA;
     // dz panel: recompute logits tile by tile
     {
@@ -1407,21 +1711,11 @@ extern "C" int sapo_policy_loss_bwd(const void* hidden, const void* W_head, int3
       if (rc != SAPO_OK) return rc;
     }
     // dhidden[t0:t0+tc] = dz . W         (M = tokens, N = H, K = V)
-    {
-      Sched sched = make_sched(tc, H, Vp, 0, /*m_fastest=*/false);
-      sched.panel_nvt = nvt;
-      StoreEpi::Params ep{dhidden + t0 * (int64_t)H, H, tc, H, 0, partials, nullptr, nullptr};
-      int rc = launch_gemm<2, true, StoreEpi>(map_p_two, map_w_mn, map_p_two, sched, ep, status, st, SAPO_K_BWD_DH);
-      if (rc != SAPO_OK) return rc;
-    }
     // dW (+)= dz^T . hidden               (M = V, N = H, K = tokens)
-    {
-      Sched sched = make_sched(V, H, tc, 0, /*m_fastest=*/false);
-      sched.panel_nvt = nvt;
-      StoreEpi::Params ep{dW_head, H, V, H, (t0 > 0 || accumulate_dW) ? 1 : 0, partials, nullptr, nullptr};
-      int rc = launch_gemm<3, true, StoreEpi>(map_p_tile, map_h_mn, map_p_tile, sched, ep, status, st, SAPO_K_BWD_DW);
-      if (rc != SAPO_OK) return rc;
-    }
+    const int rc = launch_grad_gemms(panel, panel_rows, nvt, B, ldb, A0, lda, tc, H, V, Vp,
+                                     dhidden + t0 * (int64_t)H, nullptr, dW_head,
+                                     (t0 > 0 || accumulate_dW) ? 1 : 0, partials, status, st);
+    if (rc != SAPO_OK) return rc;
   }
   return SAPO_OK;
 }
@@ -1614,18 +1908,15 @@ extern "C" int sapo_policy_loss_fwd_bwd(const void* hidden, const void* W_head, 
     KernelScope scope(SAPO_K_TARGET_LOGIT, st);
     target_logit_kernel<<<(int)blocks, 256, 0, st>>>(A, ld_hidden, B, ld_W, ids, old_logp, T, H, V, zy, c2);
   }
-  CUtensorMap map_w_kmajor, map_w_mn;
-  if (!make_map(&map_w_kmajor, B, H, V, ld_W, 128) || !make_map(&map_w_mn, B, H, V, ld_W, 128))
-    return SAPO_ERR_CUDA;
+  CUtensorMap map_w_kmajor;
+  if (!make_map(&map_w_kmajor, B, H, V, ld_W, 128)) return SAPO_ERR_CUDA;
 
   for (int64_t t0 = 0; t0 < T; t0 += chunk_rows) {
     const int64_t tc = (T - t0) < chunk_rows ? (T - t0) : chunk_rows;
     const __nv_bfloat16* A0 = A + t0 * ld_hidden;
     const int64_t panel_rows = ceil_div<int64_t>(tc, BM) * nvt * BM;
-    CUtensorMap map_h_kmajor, map_hs_mn, map_p_two, map_p_tile;
-    if (!make_map(&map_h_kmajor, A0, H, tc, ld_hidden, BM) || !make_map(&map_hs_mn, hs, H, tc, H, 128) ||
-        !make_map(&map_p_two, panel, 64, panel_rows, 64, 256) ||
-        !make_map(&map_p_tile, panel, 64, panel_rows, 64, BM))
+    CUtensorMap map_h_kmajor, map_p_tile;
+    if (!make_map(&map_h_kmajor, A0, H, tc, ld_hidden, BM) || !make_map(&map_p_tile, panel, 64, panel_rows, 64, BM))
       return SAPO_ERR_CUDA;
     // 2. exponentials of the chunk -> panel, their sums per token and vocab split
     int n_splits = fwd_splits(tc, V, H, sms);
@@ -1654,21 +1945,11 @@ extern "C" int sapo_policy_loss_fwd_bwd(const void* hidden, const void* W_head, 
       fused_tail_kernel<<<(int)blocks, 256, 0, st>>>(ta);
     }
     // 4. dhidden[t0:t0+tc] = a_t (e' . W)     (M = tokens, N = H, K = V)
-    {
-      Sched sched = make_sched(tc, H, Vp, 0, /*m_fastest=*/false);
-      sched.panel_nvt = nvt;
-      StoreEpi::Params ep{dhidden + t0 * (int64_t)H, H, tc, H, 0, partials, nullptr, row_scale};
-      int rc = launch_gemm<2, true, StoreEpi>(map_p_two, map_w_mn, map_p_two, sched, ep, status, st, SAPO_K_BWD_DH);
-      if (rc != SAPO_OK) return rc;
-    }
     // 5. dW (+)= e'^T . (a_t h_t)            (M = V, N = H, K = tokens)
-    {
-      Sched sched = make_sched(V, H, tc, 0, /*m_fastest=*/false);
-      sched.panel_nvt = nvt;
-      StoreEpi::Params ep{dW_head, H, V, H, (t0 > 0 || accumulate_dW) ? 1 : 0, partials, nullptr, nullptr};
-      int rc = launch_gemm<3, true, StoreEpi>(map_p_tile, map_hs_mn, map_p_tile, sched, ep, status, st, SAPO_K_BWD_DW);
-      if (rc != SAPO_OK) return rc;
-    }
+    const int rc = launch_grad_gemms(panel, panel_rows, nvt, B, ld_W, hs, H, tc, H, V, Vp,
+                                     dhidden + t0 * (int64_t)H, row_scale, dW_head,
+                                     (t0 > 0 || accumulate_dW) ? 1 : 0, partials, status, st);
+    if (rc != SAPO_OK) return rc;
   }
   // 6. per-sequence means and the loss
   const int seq_blocks = S < sms * 8 ? S : sms * 8;

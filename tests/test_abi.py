@@ -36,7 +36,7 @@ def test_host_side_helpers():
     fwd = B.sapo_workspace_bytes(B.WS_FWD, T, H, V, B.DTYPE_BF16)
     assert fwd >= 3 * 4 * T and fwd % 256 == 0
     bwd = B.sapo_workspace_bytes(B.WS_BWD, T, H, V, B.DTYPE_BF16)
-    k_split_scratch = 3 * 96 * 256 * 256 * 4              # partial accumulator tiles of K-split parts
+    k_split_scratch = 3 * 96 * 256 * 512 * 4              # partial accumulator tiles of K-split parts
     assert bwd == T * V * 2 + k_split_scratch            # V is already a multiple of 128
     assert B.sapo_workspace_bytes_min(B.WS_BWD, T, H, V, B.DTYPE_BF16) == 128 * V * 2 + k_split_scratch
     # single-pass call: the panel plus, per token, a scaled hidden row and a few floats
