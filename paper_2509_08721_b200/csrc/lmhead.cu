@@ -436,19 +436,25 @@ streamk_fixup_kernel(const Sched s_arg, const StoreEpi::Params p_arg, int pairs)
   decode_unit(s, s.dp_units + t, pmb, un, n_begin, n_end);
   const int n0 = n_begin * s.tile_n;
   const size_t part_floats = (size_t)PAIR_M * s.part_ld;
-  for (int col = threadIdx.x; col < s.tile_n && n0 + col < p.N; col += blockDim.x) {
-    for (int rr = row_begin; rr < row_begin + 8; ++rr) {
-      int64_t row = (int64_t)pmb * PAIR_M + rr;
-      if (row >= p.M) break;
-      const float scale = p.row_scale != nullptr ? p.row_scale[row] : 1.f;
-      if (p.row_map != nullptr) row = p.row_map[row];
-      const size_t off = (size_t)rr * s.part_ld + col;
-      float sum = 0.f;
-      for (int j = 0; j < s.sk_parts; ++j) sum += p.partials[(size_t)(j * s.sk_tiles + t) * part_floats + off];
-      sum *= scale;
-      float* dst = p.C + row * p.ldc + n0 + col;
-      *dst = p.accumulate ? *dst + sum : sum;
+  // 8 rows x (columns / 4) float4 items per block; N, tile widths and leading dimensions are multiples of 4
+  const int n4 = min(s.tile_n, p.N - n0) >> 2;
+  for (int item = threadIdx.x; item < 8 * n4; item += blockDim.x) {
+    const int rr = row_begin + item / n4, c4 = item - (item / n4) * n4;
+    int64_t row = (int64_t)pmb * PAIR_M + rr;
+    if (row >= p.M) continue;
+    const float scale = p.row_scale != nullptr ? p.row_scale[row] : 1.f;
+    if (p.row_map != nullptr) row = p.row_map[row];
+    const float* src = p.partials + (size_t)t * part_floats + (size_t)rr * s.part_ld + 4 * c4;
+    float4 sum = make_float4(0.f, 0.f, 0.f, 0.f);
+    #pragma unroll 4
+    for (int j = 0; j < s.sk_parts; ++j) {
+      const float4 v = *reinterpret_cast<const float4*>(src + (size_t)j * s.sk_tiles * part_floats);
+      sum.x += v.x; sum.y += v.y; sum.z += v.z; sum.w += v.w;
     }
+    float4* dst = reinterpret_cast<float4*>(p.C + row * p.ldc + n0 + 4 * c4);
+    float4 o = make_float4(scale * sum.x, scale * sum.y, scale * sum.z, scale * sum.w);
+    if (p.accumulate) { const float4 c = *dst; o.x += c.x; o.y += c.y; o.z += c.z; o.w += c.w; }
+    *dst = o;
   }
 }
 
