@@ -333,7 +333,20 @@ def run_ours(args):
 
     if rank == 0:
         # roofline of the dominant kernel (largest share of the timed region)
-        t_act = int(scorer.n_active.item()) if args.backward == "active" else T
+        # tokens with a non-zero gradient factor: the algorithmic backward work (zero-advantage
+        # groups and tokens clipped on the binding side contribute nothing to either gradient);
+        # t_exec = tokens the backward contractions actually run over in this mode
+        g = scorer.fwd["gscale"][:T]
+        t_act = int((g != 0).sum().item())
+        if args.backward == "active":
+            t_exec = int(scorer.n_active.item())
+        elif args.backward == "fused" and H >= 256:
+            # whole 128-token blocks without any gradient are left out
+            pad = (-T) % 128
+            gp = torch.nn.functional.pad(g, (0, pad)).view(-1, 128)
+            t_exec = min(T, 128 * int((gp != 0).any(dim=1).sum().item()))
+        else:
+            t_exec = T
         gemm = {k: per_kernel[k] for k in ("fwd_gemm", "fwd_exp", "bwd_dz", "bwd_dh", "bwd_dw")
                 if per_kernel[k]["launches"]}
         top = max(gemm, key=lambda k: gemm[k]["ms"])
@@ -341,7 +354,7 @@ def run_ours(args):
         ms_top = gemm[top]["ms"] / n_top
         # launches per step of that kernel (the backward runs once per dz panel chunk)
         per_step = n_top / args.steps
-        flops_each = 2.0 * (T if top in ("fwd_gemm", "fwd_exp") else t_act) * V * H
+        flops_each = 2.0 * (T if top in ("fwd_gemm", "fwd_exp") else t_exec if top == "bwd_dz" else t_act) * V * H
         achieved = flops_each / per_step / (ms_top / 1e3) / 1e12
         # DRAM bytes per launch from the ncu capture of a small case of the same kernels
         # (profiles/umma_gemm_kernels_*_workload2_lengths_div4.md): fixed part + bytes per token.
@@ -360,7 +373,7 @@ def run_ours(args):
         gemm_ms = sum(gemm[k]["ms"] for k in gemm) / args.steps
         f_alg = 2.0 * T * V * H + 4.0 * t_act * V * H
         # the separate backward recomputes the logits (one more contraction); the fused call does not
-        f_exec = f_alg if args.backward == "fused" else 2.0 * T * V * H + 6.0 * t_act * V * H
+        f_exec = 2.0 * T * V * H + (4.0 if args.backward == "fused" else 6.0) * t_exec * V * H
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
@@ -368,7 +381,8 @@ def run_ours(args):
             "config": {"workload": recipe.name, "H": H, "V": V, "questions": recipe.Q,
                        "local_per_question": recipe.I, "external_per_question": recipe.J,
                        "tokens_per_step": T, "sequences": S, "backward": args.backward,
-                       "active_tokens": t_act, "parallelism": f"replicas x{world}",
+                       "active_tokens": t_act, "backward_tokens_executed": t_exec,
+                       "parallelism": f"replicas x{world}",
                        "l2": "inputs larger than L2 (W_head alone is %d MB)" % (V * H * 2 // 2**20)},
             "tflops_algorithmic": f_alg / (ms_step / 1e3) / 1e12,
             "tflops_executed": f_exec / (ms_step / 1e3) / 1e12,

@@ -63,6 +63,12 @@ struct Sched {
   int32_t part_ld;    // columns of a partial tile in scratch (256, or 512 for the two-accumulator kernel)
   int32_t max_parts;  // partial tiles of that width the scratch holds
   int32_t min_part_k; // shortest K range (in stages) worth a part
+  // Wide-tile kernel only: one bit per 128-token block, set when any of its tokens has a
+  // non-zero gradient factor (nullptr: every block counts).  mask_dim 1: the blocks are rows of
+  // the output (a tile whose two blocks are both clear is stored as zeros without any MMA);
+  // mask_dim 2: they are slices of the contraction (stages of a clear block are left out).
+  const uint32_t* active_mask;
+  int32_t mask_words, mask_dim;
   // A size only the device knows (the number of active tokens after compaction), read by
   // every CTA at start-up: dyn_dim 1 = it is M (rows), 2 = it is K (contraction length).
   const int32_t* dyn_count;
@@ -725,7 +731,8 @@ constexpr uint32_t A2_STAGE_BYTES = BM * BK2 * 2;          // 16 KB
 constexpr uint32_t BOX2_BYTES = 64 * 128;                  // a 64-row box of 128-byte rows
 constexpr uint32_t B2_ACC_BYTES = 2 * BOX2_BYTES;          // up to 128 columns per accumulator and CTA
 constexpr uint32_t B2_STAGE_BYTES = 2 * B2_ACC_BYTES;      // 32 KB
-constexpr size_t GEMM2_SMEM_BYTES = 1024 + STAGES2 * (A2_STAGE_BYTES + B2_STAGE_BYTES) + 256;
+constexpr int MASK_WORDS_MAX = 1024;                       // active-block bits kept in shared memory
+constexpr size_t GEMM2_SMEM_BYTES = 1024 + STAGES2 * (A2_STAGE_BYTES + B2_STAGE_BYTES) + 256 + 4 * MASK_WORDS_MAX;
 
 template <int A_KIND>
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
@@ -745,6 +752,32 @@ umma_gemm2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
   uint64_t* acc_empty = bars + 2 * STAGES2 + 1; // epilogue -> MMA         (even CTA's is used)
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * STAGES2 + 2);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  uint32_t* mask_s = reinterpret_cast<uint32_t*>(reinterpret_cast<uint8_t*>(bars) + 256);
+  // the mask only matters if some block of the chunk is clear: decided once, by every thread alike
+  bool has_mask = false;
+  if (sched.active_mask != nullptr) {
+    const int n_blocks = sched.mask_dim == 1 ? (int)((ep.M + BM - 1) / BM) : (sched.num_k_blocks + 1) >> 1;
+    for (int w = 0; w < sched.mask_words && !has_mask; ++w) {
+      const int left = n_blocks - 32 * w;
+      const uint32_t want = left >= 32 ? 0xffffffffu : (left > 0 ? (1u << left) - 1u : 0u);
+      has_mask = (sched.active_mask[w] & want) != want;
+    }
+  }
+  for (int i = threadIdx.x; has_mask && i < sched.mask_words; i += blockDim.x) mask_s[i] = sched.active_mask[i];
+  // bit of 128-token block b (blocks past the mask count as clear)
+  auto blk_active = [&](int b) -> bool {
+    return !has_mask || (b < 32 * sched.mask_words && ((mask_s[b >> 5] >> (b & 31)) & 1u));
+  };
+  // A_KIND 2: an output tile none of whose rows is active needs no contraction at all
+  auto rows_active = [&](int pmb) -> bool { return blk_active(2 * pmb) || blk_active(2 * pmb + 1); };
+  // A_KIND 3: stage kb holds tokens [64 kb, 64 kb + 64) of block kb / 2.  The loops over stages
+  // keep the mask word of the current 32 blocks in a register (`word`, reloaded every 64 stages).
+  const bool skip_stages = A_KIND == 3 && has_mask;
+  auto stage_active = [&](int kb, int kb_first, uint32_t& word) -> bool {
+    if (!skip_stages) return true;
+    if (kb == kb_first || (kb & 63) == 0) word = (kb >> 6) < sched.mask_words ? mask_s[kb >> 6] : 0u;
+    return (word >> ((kb >> 1) & 31)) & 1u;
+  };
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   constexpr bool A_MN = A_KIND == 3;
@@ -790,7 +823,10 @@ umma_gemm2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
       const int mb = 2 * pmb + (int)rank;
       const int n0 = n_begin * sched.tile_n;
       const int bcol = n0 + bj * tn + (int)rank * half + 64 * bb;      // first column of this lane's B box
+      if (A_KIND == 2 && !rows_active(pmb)) kb1 = kb0;
+      uint32_t word = 0;
       for (int kb = kb0; kb < kb1; ++kb) {
+        if (!stage_active(kb, kb0, word)) continue;
         if (!mbar_wait(&empty[stage], phase ^ 1, abort_flag)) { ok = false; break; }
         if (rank == 0 && lane == 0) mbar_arrive_expect_tx(&full[stage], tx);
         if (mine) {
@@ -829,7 +865,11 @@ umma_gemm2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
     while (ok && work.next(pmb, un, n_begin, n_end, kb0, kb1, slot)) {
       if (!mbar_wait(acc_empty, acc_phase ^ 1, abort_flag)) { ok = false; break; }
       fence_after_sync();
+      if (A_KIND == 2 && !rows_active(pmb)) kb1 = kb0;
+      bool first = true;                       // the first stage that runs overwrites the accumulators
+      uint32_t word = 0;
       for (int kb = kb0; kb < kb1; ++kb) {
+        if (!stage_active(kb, kb0, word)) continue;
         if (!mbar_wait(&full[stage], phase, abort_flag)) { ok = false; break; }
         fence_after_sync();
         const uint32_t a_addr = smem_u32(smem_a + stage * A2_STAGE_BYTES);
@@ -838,11 +878,12 @@ umma_gemm2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
         for (int k = 0; k < BK2 / UMMA_K; ++k) {
           const uint64_t a_desc = A_MN ? make_smem_desc(a_addr + k * 2048, BOX2_BYTES, 1024)
                                        : make_smem_desc(a_addr + k * 32, 16, 1024);
-          const uint32_t acc_on = (kb > kb0 || k != 0) ? 1u : 0u;
+          const uint32_t acc_on = (!first || k != 0) ? 1u : 0u;
           mma_bf16_pair(tmem_base, a_desc, make_smem_desc(b_addr + k * 2048, BOX2_BYTES, 1024), idesc, acc_on);
           mma_bf16_pair(tmem_base + BN, a_desc,
                         make_smem_desc(b_addr + B2_ACC_BYTES + k * 2048, BOX2_BYTES, 1024), idesc, acc_on);
         }
+        first = false;
         mma_commit_pair(empty_addr[0] + stage * 8);
         mma_commit_pair(empty_addr[1] + stage * 8);
         if (++stage == STAGES2) { stage = 0; phase ^= 1; }
@@ -869,6 +910,13 @@ umma_gemm2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
       const int n0 = n_begin * sched.tile_n;
       epi.begin_unit(ep, 2 * pmb + (int)rank, r);
       epi.set_dest(ep, slot, (int)rank, r, n0, sched.part_ld);
+      // did any stage run?  if not the accumulators hold nothing of this tile: store zeros
+      bool any = kb1 > kb0;
+      if (A_KIND == 2 && !rows_active(pmb)) any = false;
+      if (A_KIND == 3 && has_mask && any) {
+        any = false;
+        for (int b = kb0 >> 1; b <= (kb1 - 1) >> 1 && !any; ++b) any = blk_active(b);
+      }
       if (!mbar_wait(acc_full, acc_phase, abort_flag)) { ok = false; break; }
       fence_after_sync();
       const uint32_t t_addr = tmem_base + (static_cast<uint32_t>(quad * 32) << 16) + j * BN;
@@ -878,7 +926,7 @@ umma_gemm2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
       for (int c = 0; c < chunks; c += 2) {
         tmem_ld_wait();
         if (c + 1 < chunks) tmem_ld32(t_addr + (c + 1) * 32, vb);
-        if (kb1 == kb0) {
+        if (!any) {
           #pragma unroll
           for (int q = 0; q < 32; ++q) va[q] = 0.f;
         }
@@ -886,7 +934,7 @@ umma_gemm2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
         if (c + 1 < chunks) {
           tmem_ld_wait();
           if (c + 2 < chunks) tmem_ld32(t_addr + (c + 2) * 32, va);
-          if (kb1 == kb0) {
+          if (!any) {
             #pragma unroll
             for (int q = 0; q < 32; ++q) vb[q] = 0.f;
           }
@@ -1058,6 +1106,7 @@ struct FusedTailArgs {
   float* row_scale;                                        // [tc]
   __nv_bfloat16* panel; int32_t nvt;                       // exponentials of the chunk
   const __nv_bfloat16* hidden; int64_t ldh; int32_t H; __nv_bfloat16* hs;   // hs [tc, H] = row_scale * hidden
+  uint32_t* active_mask;   // one bit per 128-token block of the chunk (zeroed by the caller), or nullptr
   int32_t* status;
 };
 
@@ -1111,6 +1160,8 @@ __global__ void __launch_bounds__(256) fused_tail_kernel(FusedTailArgs a) {
       if (bad_range) raise_status(a.status, SAPO_ST_EXP_RANGE);
       a.lse[t] = lse; a.logp[t] = lp; a.ratio[t] = rho; a.surr[t] = u; a.gscale[t] = g; a.obj[t] = obj;
       a.row_scale[lr] = scale;
+      if (scale != 0.f && a.active_mask != nullptr)
+        atomicOr(&a.active_mask[lr >> 12], 1u << ((lr >> 7) & 31));
       if (!bad) {
         const float ey = ex2(fmaf(zy, LOG2E, -c2));
         const int64_t tile = (lr >> 7) * a.nvt + (y >> 6);
@@ -1201,6 +1252,7 @@ static Sched make_sched(int64_t M, int64_t N, int64_t K, int n_splits, bool m_fa
   s.dp_units = s.num_units; s.sk_tiles = 0; s.sk_parts = 1;
   s.k_split_ok = 0; s.dyn_count = nullptr; s.dyn_dim = 0; s.skip_if_empty = 0;
   s.part_ld = BN; s.max_parts = MAX_PARTS_SCRATCH; s.min_part_k = 16;
+  s.active_mask = nullptr; s.mask_words = 0; s.mask_dim = 0;
   return s;
 }
 
@@ -1355,7 +1407,7 @@ static int launch_grad_gemms(const __nv_bfloat16* panel, int64_t panel_rows, int
                              const __nv_bfloat16* W, int64_t ldw, const __nv_bfloat16* X, int64_t ldx,
                              int64_t tc, int32_t H, int32_t V, int64_t Vp, float* dhidden,
                              const float* row_scale, float* dW_head, int accumulate, float* partials,
-                             int32_t* status, cudaStream_t st) {
+                             const uint32_t* active_mask, int32_t* status, cudaStream_t st) {
   StoreEpi::Params ep_h{dhidden, H, tc, H, 0, partials, nullptr, row_scale};
   StoreEpi::Params ep_w{dW_head, H, V, H, accumulate, partials, nullptr, nullptr};
   if (use_wide_tiles(H)) {
@@ -1363,12 +1415,18 @@ static int launch_grad_gemms(const __nv_bfloat16* panel, int64_t panel_rows, int
     if (!make_map(&map_p_tile, panel, 64, panel_rows, 64, BM) || !make_map(&map_p_half, panel, 64, panel_rows, 64, 64) ||
         !make_map(&map_w64, W, H, V, ldw, 64) || !make_map(&map_x64, X, H, tc, ldx, 64))
       return SAPO_ERR_CUDA;
+    // blocks of tokens without any gradient (zero-advantage groups, runs of clipped tokens) are
+    // left out of both contractions when the caller knows them
+    const int32_t mask_words = (int32_t)ceil_div<int64_t>(ceil_div<int64_t>(tc, BM), 32);
+    const bool masked = active_mask != nullptr && mask_words <= MASK_WORDS_MAX;
     Sched sh = make_sched_wide(tc, H, Vp);
     sh.panel_nvt = nvt;
+    if (masked) { sh.active_mask = active_mask; sh.mask_words = mask_words; sh.mask_dim = 1; }
     int rc = launch_gemm_wide<2>(map_p_tile, map_w64, sh, ep_h, status, st, SAPO_K_BWD_DH);
     if (rc != SAPO_OK) return rc;
     Sched sw = make_sched_wide(V, H, tc);
     sw.panel_nvt = nvt;
+    if (masked) { sw.active_mask = active_mask; sw.mask_words = mask_words; sw.mask_dim = 2; }
     return launch_gemm_wide<3>(map_p_half, map_x64, sw, ep_w, status, st, SAPO_K_BWD_DW);
   }
   CUtensorMap map_p_two, map_p_tile, map_w_mn, map_x_mn;
@@ -1434,7 +1492,7 @@ constexpr int64_t PANEL_ROWS_PREFERRED = 32768;
 // needs (row scales, partial sums, the scaled copy of hidden), the K-split scratch, the
 // per-sequence sums when the caller does not want them, and the panel of exponentials.
 constexpr int FUSED_MAX_SPLITS = 160;
-struct FusedLayout { size_t zy, c2, obj, seq, partials, fixed; size_t bytes_per_row; };
+struct FusedLayout { size_t zy, c2, obj, seq, mask, partials, fixed; size_t bytes_per_row; };
 static FusedLayout fused_layout(int64_t T, int32_t H, int32_t V, int32_t S) {
   FusedLayout L{};
   size_t off = 0;
@@ -1443,6 +1501,7 @@ static FusedLayout fused_layout(int64_t T, int32_t H, int32_t V, int32_t S) {
   L.c2 = take((size_t)T * 4);
   L.obj = take((size_t)T * 4);
   L.seq = take((size_t)(S > 0 ? S : 1) * 4);
+  L.mask = take((size_t)MASK_WORDS_MAX * 4);
   L.partials = take(KSPLIT_SCRATCH_BYTES);
   L.fixed = off;
   // per chunk row: panel row, scaled hidden row, row scale, partial sums
@@ -1720,7 +1779,7 @@ extern "C" int sapo_policy_loss_bwd(const void* hidden, const void* W_head, int3
     // dW (+)= dz^T . hidden               (M = V, N = H, K = tokens)
     const int rc = launch_grad_gemms(panel, panel_rows, nvt, B, ldb, A0, lda, tc, H, V, Vp,
                                      dhidden + t0 * (int64_t)H, nullptr, dW_head,
-                                     (t0 > 0 || accumulate_dW) ? 1 : 0, partials, status, st);
+                                     (t0 > 0 || accumulate_dW) ? 1 : 0, partials, nullptr, status, st);
     if (rc != SAPO_OK) return rc;
   }
   return SAPO_OK;
@@ -1898,6 +1957,7 @@ extern "C" int sapo_policy_loss_fwd_bwd(const void* hidden, const void* W_head, 
   float* obj = reinterpret_cast<float*>(ws + L.obj);
   float* seq_out = seq_surr ? seq_surr : reinterpret_cast<float*>(ws + L.seq);
   float* partials = reinterpret_cast<float*>(ws + L.partials);
+  uint32_t* active_mask = reinterpret_cast<uint32_t*>(ws + L.mask);
   float* row_scale = reinterpret_cast<float*>(ws + CL.row_scale);
   float* ps = reinterpret_cast<float*>(ws + CL.ps);
   __nv_bfloat16* hs = reinterpret_cast<__nv_bfloat16*>(ws + CL.hs);
@@ -1945,6 +2005,10 @@ extern "C" int sapo_policy_loss_fwd_bwd(const void* hidden, const void* W_head, 
       ta.logp = logp; ta.lse = lse; ta.ratio = ratio; ta.surr = surr; ta.gscale = gscale; ta.obj = obj;
       ta.row_scale = row_scale; ta.panel = panel; ta.nvt = nvt;
       ta.hidden = A; ta.ldh = ld_hidden; ta.H = H; ta.hs = hs; ta.status = status;
+      // one bit per 128-token block of the chunk that has a token with a gradient
+      const bool masked = ceil_div<int64_t>(ceil_div<int64_t>(tc, BM), 32) <= MASK_WORDS_MAX;
+      ta.active_mask = masked ? active_mask : nullptr;
+      if (masked && cudaMemsetAsync(active_mask, 0, (size_t)MASK_WORDS_MAX * 4, st) != cudaSuccess) return SAPO_ERR_CUDA;
       int64_t blocks = ceil_div<int64_t>(tc, 8);
       if (blocks > (int64_t)sms * 8) blocks = (int64_t)sms * 8;
       KernelScope scope(SAPO_K_FUSED_TAIL, st);
@@ -1954,7 +2018,7 @@ extern "C" int sapo_policy_loss_fwd_bwd(const void* hidden, const void* W_head, 
     // 5. dW (+)= e'^T . (a_t h_t)            (M = V, N = H, K = tokens)
     const int rc = launch_grad_gemms(panel, panel_rows, nvt, B, ld_W, hs, H, tc, H, V, Vp,
                                      dhidden + t0 * (int64_t)H, row_scale, dW_head,
-                                     (t0 > 0 || accumulate_dW) ? 1 : 0, partials, status, st);
+                                     (t0 > 0 || accumulate_dW) ? 1 : 0, partials, active_mask, status, st);
     if (rc != SAPO_OK) return rc;
   }
   // 6. per-sequence means and the loss

@@ -98,11 +98,16 @@ def test_fused_loss_variants(loss_agg, kl_beta):
     check_all(out, ref, adv, batch, 0.2, 0.28, extra_scale=kl_beta)
 
 
-def test_fused_agrees_with_the_separate_calls_and_repeats_bit_for_bit():
+@pytest.mark.parametrize("H,I", [(128, 2), (256, 8)], ids=["narrow_tiles", "wide_tiles_block_skipping"])
+def test_fused_agrees_with_the_separate_calls_and_repeats_bit_for_bit(H, I):
+    """A quarter of the questions have equal rewards (no gradient).  With H = 256 the wide-tile
+    backward kernels run and whole 128-token blocks of such questions are left out of both
+    contractions; the results must not change."""
     r = gen.config(3, length_div=16)
-    recipe = gen.Recipe(**{**r.__dict__, "H": 128, "V": 3000, "Q": 8, "I": 2, "J": 2})
+    recipe = gen.Recipe(**{**r.__dict__, "H": H, "V": 3000, "Q": 8, "I": I, "J": I})
     batch = gen.make_batch(recipe, 5)
     adv, ref = oracle_case(batch, 0.2, 0.2)
+    check_all(U.gpu_scores_fused(*device_inputs(batch, adv), 0.2, 0.2), ref, adv, batch, 0.2, 0.2)
     args = device_inputs(batch, adv)
     a = U.gpu_scores_fused(*args, 0.2, 0.2)
     b = U.gpu_scores_fused(*args, 0.2, 0.2)
