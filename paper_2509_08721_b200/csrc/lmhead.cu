@@ -731,12 +731,20 @@ constexpr uint32_t A2_STAGE_BYTES = BM * BK2 * 2;          // 16 KB
 constexpr uint32_t BOX2_BYTES = 64 * 128;                  // a 64-row box of 128-byte rows
 constexpr uint32_t B2_ACC_BYTES = 2 * BOX2_BYTES;          // up to 128 columns per accumulator and CTA
 constexpr uint32_t B2_STAGE_BYTES = 2 * B2_ACC_BYTES;      // 32 KB
-constexpr int MASK_WORDS_MAX = 1024;                       // active-block bits kept in shared memory
-constexpr size_t GEMM2_SMEM_BYTES = 1024 + STAGES2 * (A2_STAGE_BYTES + B2_STAGE_BYTES) + 256 + 4 * MASK_WORDS_MAX;
+// after the stages: 256 bytes of barriers, the active-block bits, then (1024-byte aligned) one
+// fp32 staging tile of 128 rows x 32 columns per accumulator for the TMA stores of the epilogue
+constexpr int MASK_WORDS_MAX = 448;                        // active-block bits kept in shared memory
+constexpr uint32_t GEMM2_TAIL_BYTES = 2048;                // barriers + mask
+constexpr uint32_t OUT_STAGING_BYTES = 128 * 128;          // per accumulator
+constexpr size_t GEMM2_SMEM_BYTES =
+    1024 + STAGES2 * (A2_STAGE_BYTES + B2_STAGE_BYTES) + GEMM2_TAIL_BYTES + 2 * OUT_STAGING_BYTES;
+static_assert(256 + 4 * MASK_WORDS_MAX <= GEMM2_TAIL_BYTES, "barriers and mask overflow their region");
+static_assert(GEMM2_SMEM_BYTES <= 232448, "more shared memory than a CTA can have");
 
 template <int A_KIND>
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
 umma_gemm2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+                  const __grid_constant__ CUtensorMap map_c,   // the fp32 output, boxes of 32 columns x 128 rows
                   const Sched sched_arg, const StoreEpi::Params ep_arg, int32_t* status) {
   static_assert(A_KIND == 2 || A_KIND == 3, "panel operands only");
   Sched sched = sched_arg;
@@ -753,6 +761,7 @@ umma_gemm2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * STAGES2 + 2);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
   uint32_t* mask_s = reinterpret_cast<uint32_t*>(reinterpret_cast<uint8_t*>(bars) + 256);
+  uint8_t* out_staging = reinterpret_cast<uint8_t*>(bars) + GEMM2_TAIL_BYTES;
   // the mask only matters if some block of the chunk is clear: decided once, by every thread alike
   bool has_mask = false;
   if (sched.active_mask != nullptr) {
@@ -904,6 +913,8 @@ umma_gemm2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
     bool ok = true;
     StoreEpi epi;
     StageCtx cx{};
+    const uint32_t buf = smem_u32(out_staging) + j * OUT_STAGING_BYTES;
+    const bool elected = quad == 0 && lane == 0;     // issues and tracks this accumulator's TMA stores
     WorkList work(sched, pair, num_pairs);
     int pmb, un, n_begin, n_end, kb0, kb1, slot;
     while (ok && work.next(pmb, un, n_begin, n_end, kb0, kb1, slot)) {
@@ -921,24 +932,43 @@ umma_gemm2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
       fence_after_sync();
       const uint32_t t_addr = tmem_base + (static_cast<uint32_t>(quad * 32) << 16) + j * BN;
       const int chunks = (tn + 31) >> 5;
+      const int row0 = (2 * pmb + (int)rank) * BM;      // first output row of this CTA's half of the tile
+      // One 32-column chunk of this thread's row.  A K-split part goes to scratch with plain
+      // stores.  A whole tile goes through the staging tile of this accumulator (128-byte rows,
+      // 128-byte swizzle) and leaves as one TMA store, or TMA add when accumulating, of
+      // 128 rows x 32 columns: full lines, and rows / columns outside the output are clipped.
+      auto emit = [&](float (&v)[32], int col0) {
+        if (!any) {
+          #pragma unroll
+          for (int q = 0; q < 32; ++q) v[q] = 0.f;
+        }
+        if (epi.part != nullptr) { epi.template chunk<0>(ep, v, col0, cx); return; }
+        if (col0 >= ep.N || row0 >= ep.M) return;      // nothing of this box lies inside the output
+        if (elected) bulk_wait_read_all();
+        named_barrier_sync(1 + j, 128);
+        #pragma unroll
+        for (int q = 0; q < 8; ++q)
+          st_shared_v4(buf + r * 128 + ((q ^ (r & 7)) << 4),
+                       __float_as_uint(epi.scale * v[4 * q]), __float_as_uint(epi.scale * v[4 * q + 1]),
+                       __float_as_uint(epi.scale * v[4 * q + 2]), __float_as_uint(epi.scale * v[4 * q + 3]));
+        fence_proxy_async_smem();
+        named_barrier_sync(1 + j, 128);
+        if (elected) {
+          if (ep.accumulate) tma_reduce_add_2d(&map_c, buf, col0, row0);
+          else               tma_store_2d(&map_c, buf, col0, row0);
+          bulk_commit_group();
+        }
+      };
       float va[32], vb[32];
       tmem_ld32(t_addr, va);
       for (int c = 0; c < chunks; c += 2) {
         tmem_ld_wait();
         if (c + 1 < chunks) tmem_ld32(t_addr + (c + 1) * 32, vb);
-        if (!any) {
-          #pragma unroll
-          for (int q = 0; q < 32; ++q) va[q] = 0.f;
-        }
-        epi.template chunk<0>(ep, va, n0 + j * tn + c * 32, cx);
+        emit(va, n0 + j * tn + c * 32);
         if (c + 1 < chunks) {
           tmem_ld_wait();
           if (c + 2 < chunks) tmem_ld32(t_addr + (c + 2) * 32, va);
-          if (!any) {
-            #pragma unroll
-            for (int q = 0; q < 32; ++q) vb[q] = 0.f;
-          }
-          epi.template chunk<1>(ep, vb, n0 + j * tn + (c + 1) * 32, cx);
+          emit(vb, n0 + j * tn + (c + 1) * 32);
         }
       }
       fence_before_sync();
@@ -946,6 +976,7 @@ umma_gemm2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
       if (lane == 0) mbar_arrive_cluster(acc_empty0_addr);
       acc_phase ^= 1;
     }
+    if (elected) bulk_wait_all();     // stores done before shared memory goes away
   }
 
   fence_before_sync();
@@ -1229,6 +1260,20 @@ static bool make_map(CUtensorMap* map, const void* base, int64_t inner, int64_t 
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// fp32 matrix [outer, inner] with `ld` elements between rows, for stores of 32-column x 128-row
+// boxes (128 bytes wide, 128-byte swizzle); elements outside the matrix are not written.
+static bool make_map_f32_out(CUtensorMap* map, const float* base, int64_t inner, int64_t outer, int64_t ld) {
+  EncodeTiledFn fn = encode_fn();
+  if (fn == nullptr || inner <= 0 || outer <= 0) return false;
+  cuuint64_t dims[2] = {(cuuint64_t)inner, (cuuint64_t)outer};
+  cuuint64_t strides[1] = {(cuuint64_t)ld * 4};
+  cuuint32_t box[2] = {32u, 128u};
+  cuuint32_t estr[2] = {1u, 1u};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<float*>(base), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 static Sched make_sched(int64_t M, int64_t N, int64_t K, int n_splits, bool m_fastest, int tile_align = 32) {
   Sched s{};
   s.num_m_blocks = (int32_t)ceil_div<int64_t>(M, PAIR_M);
@@ -1358,6 +1403,8 @@ static bool use_wide_tiles(int32_t N) { return N >= BN; }
 template <int A_KIND>
 static int launch_gemm_wide(const CUtensorMap& ma, const CUtensorMap& mb, const Sched& sched,
                             const StoreEpi::Params& ep, int32_t* status, cudaStream_t st, int kernel_id) {
+  CUtensorMap mc;
+  if (!make_map_f32_out(&mc, ep.C, ep.N, ep.M, ep.ldc)) return SAPO_ERR_CUDA;
   auto kern = umma_gemm2_kernel<A_KIND>;
   static int max_pairs = 0;
   if (sched.num_units <= 0) return SAPO_OK;
@@ -1390,7 +1437,7 @@ static int launch_gemm_wide(const CUtensorMap& ma, const CUtensorMap& mb, const 
   cfg.gridDim = dim3(2 * pairs, 1, 1);
   {
     KernelScope scope(kernel_id, st);
-    if (cudaLaunchKernelEx(&cfg, kern, ma, mb, sc, ep, status) != cudaSuccess) return SAPO_ERR_CUDA;
+    if (cudaLaunchKernelEx(&cfg, kern, ma, mb, mc, sc, ep, status) != cudaSuccess) return SAPO_ERR_CUDA;
   }
   if (sc.sk_tiles > 0) {
     KernelScope scope(SAPO_K_STREAMK_FIXUP, st);
