@@ -160,10 +160,10 @@ def run_reference(args):
     return 0
 
 
-def hbm_kernels(torch, B, peaks, H=896, n_rollouts=2048, mean_len=288, n_groups=1 << 22):
+def hbm_kernels(torch, B, peaks, H=896, n_rollouts=2048, mean_len=288, n_groups=1 << 24):
     """Achieved HBM GB/s of the pack and advantage kernels on a scaled case (the workload-size
-    launches take tens of microseconds): about 1.3 GB moved by the pack gather, 2^22 questions
-    of 8 completions for the advantages.  Algorithmic bytes: pack 2*T*(2H+8) (hidden row,
+    launches take tens of microseconds): about 4.2 GB moved by the pack gather, 2^24 questions
+    of 8 completions (1.1 GB) for the advantages, an LM-head-sized weight for Adam.  Algorithmic bytes: pack 2*T*(2H+8) (hidden row,
     id and old log-prob, read and written once), advantages 8 bytes per completion."""
     g = torch.Generator(device="cuda").manual_seed(1)
     lens = torch.randint(mean_len // 2, mean_len * 3 // 2, (2, n_rollouts), generator=g, device="cuda")
@@ -360,8 +360,10 @@ def run_ours(args):
         # (profiles/umma_gemm_kernels_*_workload2_lengths_div4.md): fixed part + bytes per token.
         # Only valid for hidden 896 / vocab 151936, the shape that capture ran at.
         ncu_traffic = {"fwd_gemm": (0.272e9, 12.4e3), "bwd_dz": (0.272e9, 299.6e3),
-                       "fwd_exp": (0.272e9, 309.0e3), "bwd_dh": (0.272e9, 310.7e3),
-                       "bwd_dw": (0.515e9, 327.4e3)}
+                       "fwd_exp": (0.272e9, 309.5e3), "bwd_dh": (0.405e9, 310.7e3),
+                       "bwd_dw": (0.663e9, 310.7e3)}
+        if args.backward != "fused":     # the separate backward's dH / dW launches were captured earlier
+            ncu_traffic.update({"bwd_dh": (0.272e9, 310.8e3), "bwd_dw": (0.515e9, 332.3e3)})
         traffic = None
         if (H, V) == (896, 151936) and top in ncu_traffic:
             fixed, per_token = ncu_traffic[top]

@@ -126,6 +126,36 @@ def test_fused_agrees_with_the_separate_calls_and_repeats_bit_for_bit(H, I):
         assert torch.all(a["dhidden"][int(cu[go[q]]):int(cu[go[q + 1]])] == 0)
 
 
+# Output widths around the tile shapes of the wide backward kernels (H >= 256: tiles of up to
+# 2 x 256 columns, ragged last tile, columns past H clipped by the store) with token and vocabulary
+# counts around the 128 / 256-row blocks.
+EDGE = [
+    ("h256_few_tokens", small_recipe(H=256, V=130, Q=2, length_law=("uniform", 2, 8))),
+    ("h264_ragged_tile", small_recipe(H=264, V=1000, Q=4, length_law=("uniform", 10, 30))),
+    ("h320_t_over_512", small_recipe(H=320, V=777, Q=6, length_law=("uniform", 20, 40))),
+    ("h520_two_tiles", small_recipe(H=520, V=4100, Q=8, length_law=("uniform", 20, 45))),
+    ("h1024_one_block", small_recipe(H=1024, V=2000, Q=2, length_law=("uniform", 20, 40))),
+    ("h1032_three_tiles", small_recipe(H=1032, V=650, Q=4, length_law=("uniform", 30, 34))),
+]
+
+
+@pytest.mark.parametrize("name,recipe", EDGE, ids=[c[0] for c in EDGE])
+def test_edge_shapes_of_the_wide_backward_kernels(name, recipe):
+    """Both ways through the gradients (the separate backward uses the same wide kernels)."""
+    batch = gen.make_batch(recipe, 77)
+    adv, ref = oracle_case(batch, 0.2, 0.28, noise_scale=2.0)
+    args = device_inputs(batch, adv)
+    check_all(U.gpu_scores_fused(*args, 0.2, 0.28), ref, adv, batch, 0.2, 0.28)
+    check_all(U.gpu_scores(*args, 0.2, 0.28), ref, adv, batch, 0.2, 0.28)
+    # a one-panel workspace: token chunks, dW_head accumulated by TMA adds
+    T, H, V = batch.T, recipe.H, recipe.V
+    if T > 128:
+        small = B.sapo_workspace_bytes_min(B.WS_FUSED, T, H, V, B.DTYPE_BF16)
+        check_all(U.gpu_scores_fused(*args, 0.2, 0.28, workspace_bytes=small), ref, adv, batch, 0.2, 0.28)
+        small_b = B.sapo_workspace_bytes_min(B.WS_BWD, T, H, V, B.DTYPE_BF16)
+        check_all(U.gpu_scores(*args, 0.2, 0.28, bwd_workspace_bytes=small_b), ref, adv, batch, 0.2, 0.28)
+
+
 def test_fused_flags_bad_ids_and_stale_old_logp():
     recipe = small_recipe(H=64, V=400, Q=2, length_law=("uniform", 20, 40))
     batch = gen.make_batch(recipe, 9)
