@@ -156,6 +156,56 @@ def test_edge_shapes_of_the_wide_backward_kernels(name, recipe):
         check_all(U.gpu_scores(*args, 0.2, 0.28, bwd_workspace_bytes=small_b), ref, adv, batch, 0.2, 0.28)
 
 
+def _random_recipe(seed):
+    rng = np.random.default_rng(1000 + seed)
+    H = int(rng.choice([8, 16, 24, 64, 72, 248, 256, 264, 392, 512, 776, 1024, 1096]))
+    V = int(rng.choice([1, 2, 63, 64, 65, 127, 129, 500, 1000, 2049, 4097]))
+    Q = int(rng.integers(1, 7))
+    lo = int(rng.choice([1, 1, 5, 30]))
+    hi = lo + int(rng.choice([0, 3, 40, 90]))
+    return small_recipe(H=H, V=V, Q=Q, I=int(rng.integers(1, 4)), J=int(rng.integers(0, 4)),
+                        length_law=("uniform", lo, hi))
+
+
+@pytest.mark.parametrize("seed", range(24))
+def test_random_shapes_single_pass_against_separate_calls(seed):
+    """Shapes drawn around the tile, block and box sizes of the kernels (hidden sizes on both
+    sides of the wide-tile threshold, vocabularies of one entry and up, one token and up): the
+    two ways through the loss and its gradients must agree with each other.  The old log-probs
+    come from the separate forward itself, so no oracle pass is needed here."""
+    recipe = _random_recipe(seed)
+    batch = gen.make_batch(recipe, 300 + seed)
+    b = batch.built
+    hidden, W, ids = U.to_torch(b.hidden), U.to_torch(batch.W), U.to_torch(b.ids)
+    cu = U.to_torch(b.cu_seqlens)
+    adv_np = orc.group_advantages(b.rewards, b.group_offsets, adv_eps=1e-6)["adv"].astype(np.float32)
+    adv = U.to_torch(adv_np)
+    zero = torch.zeros(batch.T, device="cuda")
+    cur = U.gpu_scores(hidden, W, ids, zero, adv, cu, 0.2, 0.28, want_bwd=False)["logp"]
+    old = cur + U.to_torch(b.logp_noise.astype(np.float32)) * 2.0
+    sep = U.gpu_scores(hidden, W, ids, old, adv, cu, 0.2, 0.28)
+    one = U.gpu_scores_fused(hidden, W, ids, old, adv, cu, 0.2, 0.28)
+    assert sep["status"] == 0 and one["status"] == 0, (recipe, sep["status"], one["status"])
+    assert (one["logp"] - sep["logp"]).abs().max().item() <= 2e-4
+    assert (one["lse"] - sep["lse"]).abs().max().item() <= 2e-4
+    assert torch.allclose(one["ratio"], sep["ratio"], rtol=1e-3, atol=0)
+    # the clip decision may differ for ratios within rounding of an edge
+    rho = sep["ratio"]
+    near = torch.minimum((rho - 0.8).abs(), (rho - 1.28).abs()) < 1e-3
+    gmax = sep["gscale"].abs().max().item() + 1e-30
+    assert ((one["gscale"] - sep["gscale"]).abs()[~near]).max().item() <= 2e-3 * gmax if (~near).any() else True
+    if not near.any():
+        scale = np.abs(adv_np).max() + 1e-30
+        assert (one["seq_surr"] - sep["seq_surr"]).abs().max().item() <= 1e-3 * scale
+        for k in ("dhidden", "dW"):
+            ref = sep[k].double().cpu().numpy()
+            diff = np.linalg.norm(one[k].double().cpu().numpy() - ref)
+            # the floor covers degenerate cases (a vocabulary of one entry: both gradients are
+            # rounding noise around zero)
+            assert diff <= 1.5e-2 * np.linalg.norm(ref) + 1e-5 * gmax * np.sqrt(ref.size), (recipe, k)
+    assert torch.isfinite(one["dhidden"]).all() and torch.isfinite(one["dW"]).all()
+
+
 def test_fused_flags_bad_ids_and_stale_old_logp():
     recipe = small_recipe(H=64, V=400, Q=2, length_law=("uniform", 20, 40))
     batch = gen.make_batch(recipe, 9)
