@@ -1,0 +1,318 @@
+// What happens to an accumulator tile once the tensor cores have finished it: the four epilogues
+// of the GEMM kernels (online log-sum-exp of the forward, dz of the separate backward, the
+// exponential panel of the single-pass call, plain fp32 stores) and the fix-up of K-split tiles.
+#pragma once
+
+#include "gemm_sched.cuh"
+
+namespace sapo {
+using namespace umma;
+
+// ---------------------------------------------------------------------------- epilogues
+// Each epilogue thread owns one accumulator row (TMEM lane) of the tile.
+
+// What a staged epilogue needs to move finished 64-column groups through shared memory.
+struct StageCtx {
+  uint32_t buf;          // shared address of this column half's 16 KB staging tile
+  int bar_id;            // named barrier of the four warps that share it
+  bool elected;          // the one thread that issues and tracks the TMA stores
+  const CUtensorMap* map;
+};
+
+// A thread's 64 finished bf16 entries of a panel row (two 32-column chunks as 16 pairs each)
+// go to the staging tile, and the tile leaves as one 16 KB TMA store: wait until the previous
+// store has read the staging tile, write this row (128 bytes, in 128-byte-swizzle order) and
+// hand the tile to the TMA.  Called by all 128 threads that share the staging tile.
+__device__ __forceinline__ void store_panel_group(const StageCtx& cx, int r, const uint32_t (&pk)[2][16],
+                                                  int tile_row0, int col0_of_group) {
+  if (cx.elected) bulk_wait_read_all();
+  named_barrier_sync(cx.bar_id, 128);
+  #pragma unroll
+  for (int q = 0; q < 8; ++q)
+    st_shared_v4(cx.buf + r * 128 + ((q ^ (r & 7)) << 4),
+                 pk[q >> 2][4 * (q & 3)], pk[q >> 2][4 * (q & 3) + 1],
+                 pk[q >> 2][4 * (q & 3) + 2], pk[q >> 2][4 * (q & 3) + 3]);
+  fence_proxy_async_smem();
+  named_barrier_sync(cx.bar_id, 128);
+  if (cx.elected) {
+    tma_store_2d(cx.map, cx.buf, 0, tile_row0 + (col0_of_group >> 6) * BM);
+    bulk_commit_group();
+  }
+}
+
+// Forward: online log-sum-exp in the base-2 domain plus the logit of the chosen token.
+struct FwdEpi {
+  static constexpr bool STAGED = false;
+  static constexpr bool STREAMK = false;
+  template <class P> __device__ static void set_dynamic(P&, const Sched&) {}
+
+  struct Params {
+    const int32_t* ids; float* pm; float* ps; float* pz;  // partials [n_splits][T]
+    int64_t T; int32_t V;
+  };
+  float m, s, zy; int32_t y; int64_t row;
+  __device__ __forceinline__ void begin_unit(const Params& p, int mb, int r) {
+    row = (int64_t)mb * BM + r;
+    m = -INFINITY; s = 0.f; zy = 0.f;
+    y = row < p.T ? p.ids[row] : -1;
+  }
+  template <int HALF>
+  __device__ __forceinline__ void chunk(const Params& p, float (&v)[32], int col0, const StageCtx&) {
+    if (col0 >= p.V) return;
+    if (col0 + 32 > p.V) {
+      #pragma unroll
+      for (int j = 0; j < 32; ++j) if (col0 + j >= p.V) v[j] = -INFINITY;
+    }
+    const int yr = y - col0;
+    if (yr >= 0 && yr < 32) {
+      #pragma unroll
+      for (int j = 0; j < 32; ++j) if (j == yr) zy = v[j];
+    }
+    float cmax = v[0];
+    #pragma unroll
+    for (int j = 1; j < 32; ++j) cmax = fmaxf(cmax, v[j]);
+    const float m_new = fmaxf(m, cmax * LOG2E);
+    float acc = s * ex2(m - m_new);          // first chunk: ex2(-inf) = 0
+    #pragma unroll
+    for (int j = 0; j < 32; ++j) acc += ex2(fmaf(v[j], LOG2E, -m_new));
+    s = acc; m = m_new;
+  }
+  // two threads share a row (one per column half of the tiles): each leaves its own partial
+  __device__ __forceinline__ void end_unit(const Params& p, int un, int col_half) {
+    if (row < p.T) {
+      const int64_t o = (int64_t)(2 * un + col_half) * p.T + row;
+      p.pm[o] = m; p.ps[o] = s; p.pz[o] = zy;
+    }
+  }
+};
+
+// Backward, first contraction: dz[t,v] = g_t ([v == y_t] - exp(z[t,v] - lse_t)), to bf16.
+// The panel is a sequence of [128 token x 64 vocab] tiles of 16 KB, tile (tb, vt) at index
+// tb * nvt + vt, each tile row-major: both later contractions then fetch whole contiguous
+// tiles with one TMA box.  Rows past the last token and columns past V are written as zeros,
+// because those consumers cannot tell them from data.  A finished 64-column group is staged in
+// shared memory (128-byte swizzle) and leaves as one 16 KB TMA store.
+struct DzEpi {
+  static constexpr bool STAGED = true;
+  static constexpr bool STREAMK = false;
+  template <class P> __device__ static void set_dynamic(P& p, const Sched& s) {
+    if (s.dyn_dim == 1) p.M = *s.dyn_count;
+  }
+  struct Params {
+    const int32_t* ids; const float* lse; const float* gscale;
+    int64_t M; int32_t V; int32_t nvt;
+  };
+  float g, l2; int32_t y; int32_t tile_row0; int r; bool in_panel;
+  __device__ __forceinline__ void begin_unit(const Params& p, int mb, int r_) {
+    const int64_t row = (int64_t)mb * BM + r_;
+    const bool valid = row < p.M;
+    in_panel = (int64_t)mb * BM < p.M;   // the odd CTA of the last pair may own no token block
+    r = r_;
+    tile_row0 = mb * p.nvt * BM;          // first panel row of this token block
+    g = valid ? p.gscale[row] : 0.f;
+    l2 = valid ? p.lse[row] * LOG2E : 0.f;
+    y = valid ? p.ids[row] : -1;
+  }
+  __device__ __forceinline__ void group_begin(const StageCtx&) {}
+  // dz of 32 columns, kept in registers as 16 bf16 pairs until the whole 64-column group is done
+  uint32_t pk[2][16];
+  template <int HALF>   // which 32-column half of the group (a compile-time register choice)
+  __device__ __forceinline__ void chunk(const Params& p, float (&v)[32], int col0, const StageCtx&) {
+    if (!in_panel) return;
+    uint32_t (&packed)[16] = pk[HALF];
+    if (g == 0.f) {
+      #pragma unroll
+      for (int j = 0; j < 16; ++j) packed[j] = 0u;
+    } else {
+      const float ng = -g;
+      #pragma unroll
+      for (int j = 0; j < 32; ++j) v[j] = ng * ex2(fmaf(v[j], LOG2E, -l2));
+      const int yr = y - col0;
+      if (yr >= 0 && yr < 32) {            // the chunk that holds the chosen token
+        #pragma unroll
+        for (int j = 0; j < 32; ++j) if (j == yr) v[j] += g;
+      }
+      if (col0 + 32 > p.V) {               // ragged end of the vocabulary
+        #pragma unroll
+        for (int j = 0; j < 32; ++j) if (col0 + j >= p.V) v[j] = 0.f;
+      }
+      #pragma unroll
+      for (int j = 0; j < 16; ++j) {
+        __nv_bfloat162 h = __floats2bfloat162_rn(v[2 * j], v[2 * j + 1]);
+        packed[j] = *reinterpret_cast<uint32_t*>(&h);
+      }
+    }
+  }
+  __device__ __forceinline__ void group_end(const Params&, int col0_of_group, const StageCtx& cx) {
+    if (in_panel) store_panel_group(cx, r, pk, tile_row0, col0_of_group);
+  }
+  __device__ __forceinline__ void end_unit(const Params&, int, int) {}
+};
+
+// Forward of the fused call: e[t,v] = exp(z[t,v] - c_t) against a per-token reference c_t that
+// is known before the pass (see sapo_policy_loss_fwd_bwd), so no running maximum is needed:
+// the epilogue adds the fp32 exponentials up per token and leaves them, rounded to bf16, in
+// the tiled panel (same layout as DzEpi) for the backward contractions, which then need no
+// second pass over the logits.  Exponentials are capped at 2^100, so that sums and products
+// with them stay finite and a zero row scale later still gives zero (a token that reaches the
+// cap is reported, see fused_tail_kernel).  Rows past the last token and columns past V hold zeros.
+struct ExpEpi {
+  static constexpr bool STAGED = true;
+  static constexpr bool STREAMK = false;
+  template <class P> __device__ static void set_dynamic(P&, const Sched&) {}
+  struct Params {
+    const float* c2;      // [M] reference of each token, in the base-2 domain (c_t * log2 e)
+    float* ps;            // [2 * n_splits][M] partial sums of exponentials
+    int64_t M; int32_t V; int32_t nvt;
+  };
+  float c, sum; int32_t tile_row0; int r; bool valid, in_panel; int64_t row;
+  uint32_t pk[2][16];
+  __device__ __forceinline__ void begin_unit(const Params& p, int mb, int r_) {
+    row = (int64_t)mb * BM + r_;
+    valid = row < p.M;
+    in_panel = (int64_t)mb * BM < p.M;
+    r = r_;
+    tile_row0 = mb * p.nvt * BM;
+    c = valid ? p.c2[row] : 0.f;
+    sum = 0.f;
+  }
+  __device__ __forceinline__ void group_begin(const StageCtx&) {}
+  template <int HALF>
+  __device__ __forceinline__ void chunk(const Params& p, float (&v)[32], int col0, const StageCtx&) {
+    if (!in_panel) return;
+    uint32_t (&packed)[16] = pk[HALF];
+    if (!valid || col0 >= p.V) {
+      #pragma unroll
+      for (int j = 0; j < 16; ++j) packed[j] = 0u;
+      return;
+    }
+    const float cap = EXP_CAP;
+    #pragma unroll
+    for (int j = 0; j < 32; ++j) v[j] = fminf(ex2(fmaf(v[j], LOG2E, -c)), cap);
+    if (col0 + 32 > p.V) {               // ragged end of the vocabulary
+      #pragma unroll
+      for (int j = 0; j < 32; ++j) if (col0 + j >= p.V) v[j] = 0.f;
+    }
+    float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+    #pragma unroll
+    for (int j = 0; j < 32; j += 4) { a0 += v[j]; a1 += v[j + 1]; a2 += v[j + 2]; a3 += v[j + 3]; }
+    sum += (a0 + a1) + (a2 + a3);
+    #pragma unroll
+    for (int j = 0; j < 16; ++j) {
+      __nv_bfloat162 h = __floats2bfloat162_rn(v[2 * j], v[2 * j + 1]);
+      packed[j] = *reinterpret_cast<uint32_t*>(&h);
+    }
+  }
+  __device__ __forceinline__ void group_end(const Params&, int col0_of_group, const StageCtx& cx) {
+    if (in_panel) store_panel_group(cx, r, pk, tile_row0, col0_of_group);
+  }
+  // two threads share a row (one per column half of the tiles): each leaves its own partial
+  __device__ __forceinline__ void end_unit(const Params& p, int un, int col_half) {
+    if (valid) p.ps[(int64_t)(2 * un + col_half) * p.M + row] = sum;
+  }
+};
+
+// Plain fp32 output tile, optionally added to what is already there.
+struct StoreEpi {
+  static constexpr bool STAGED = false;
+  static constexpr bool STREAMK = true;
+  // row_map (optional): output row of each accumulator row (rows of compacted tokens go back
+  // to their packed positions)
+  // row_scale (optional): factor applied to each accumulator row before it is stored
+  struct Params { float* C; int64_t ldc; int64_t M; int32_t N; int32_t accumulate; float* partials;
+                  const int32_t* row_map; const float* row_scale; };
+  template <class P> __device__ static void set_dynamic(P& p, const Sched& s) {
+    if (s.dyn_dim == 1) p.M = *s.dyn_count;
+  }
+  int64_t row; bool valid; float* part; int n0; float scale;
+  __device__ __forceinline__ void begin_unit(const Params& p, int mb, int r) {
+    row = (int64_t)mb * BM + r;
+    valid = row < p.M;
+    scale = (valid && p.row_scale != nullptr) ? p.row_scale[row] : 1.f;
+    if (valid && p.row_map != nullptr) row = p.row_map[row];
+    part = nullptr;
+  }
+  // a K-split part of a tile goes to scratch slot `slot` instead: rows [128 rank, +128) of a
+  // 256 x 256 fp32 tile, column 0 = the tile's first column
+  __device__ __forceinline__ void set_dest(const Params& p, int slot, int rank, int r, int n0_, int part_ld) {
+    n0 = n0_;
+    part = slot < 0 ? nullptr
+                    : p.partials + ((size_t)slot * PAIR_M + (size_t)(rank * BM + r)) * part_ld;
+  }
+  template <int HALF>
+  __device__ __forceinline__ void chunk(const Params& p, float (&v)[32], int col0, const StageCtx&) {
+    if (part != nullptr) {
+      float4* dst = reinterpret_cast<float4*>(part + (col0 - n0));
+      #pragma unroll
+      for (int q = 0; q < 8; ++q) dst[q] = make_float4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
+      return;
+    }
+    if (!valid) return;
+    float4* dst = reinterpret_cast<float4*>(p.C + row * p.ldc + col0);
+    #pragma unroll
+    for (int q = 0; q < 8; ++q) {
+      if (col0 + 4 * q < p.N) {          // N is a multiple of 4
+        float4 o = make_float4(scale * v[4 * q], scale * v[4 * q + 1], scale * v[4 * q + 2],
+                               scale * v[4 * q + 3]);
+        if (p.accumulate) { const float4 c = dst[q]; o.x += c.x; o.y += c.y; o.z += c.z; o.w += c.w; }
+        dst[q] = o;
+      }
+    }
+  }
+  __device__ __forceinline__ void end_unit(const Params&, int, int) {}
+};
+
+// Adds up the K-split parts of each tile the GEMM kernel left in scratch and stores the sum.
+// Part order is fixed (by pair index), so the result does not depend on timing.
+__global__ void __launch_bounds__(256)
+streamk_fixup_kernel(const Sched s_arg, const StoreEpi::Params p_arg, int pairs) {
+  Sched s = s_arg;
+  StoreEpi::Params p = p_arg;
+  finalize_sched(s, pairs);
+  StoreEpi::set_dynamic(p, s);
+  const int t = blockIdx.x >> 5;                 // K-split tile
+  if (t >= s.sk_tiles) return;
+  const int row_begin = (blockIdx.x & 31) * 8;   // 8 of its 256 rows per block
+  if (s.sk_parts <= 1) return;                   // whole tiles were stored by their pair
+  int pmb, un, n_begin, n_end;
+  decode_unit(s, s.dp_units + t, pmb, un, n_begin, n_end);
+  const int n0 = n_begin * s.tile_n;
+  const size_t part_floats = (size_t)PAIR_M * s.part_ld;
+  // 8 rows x (columns / 4) float4 items per block; N, tile widths and leading dimensions are multiples of 4
+  const int n4 = min(s.tile_n, p.N - n0) >> 2;
+  for (int item = threadIdx.x; item < 8 * n4; item += blockDim.x) {
+    const int rr = row_begin + item / n4, c4 = item - (item / n4) * n4;
+    int64_t row = (int64_t)pmb * PAIR_M + rr;
+    if (row >= p.M) continue;
+    const float scale = p.row_scale != nullptr ? p.row_scale[row] : 1.f;
+    if (p.row_map != nullptr) row = p.row_map[row];
+    const float* src = p.partials + (size_t)t * part_floats + (size_t)rr * s.part_ld + 4 * c4;
+    float4 sum = make_float4(0.f, 0.f, 0.f, 0.f);
+    #pragma unroll 4
+    for (int j = 0; j < s.sk_parts; ++j) {
+      const float4 v = *reinterpret_cast<const float4*>(src + (size_t)j * s.sk_tiles * part_floats);
+      sum.x += v.x; sum.y += v.y; sum.z += v.z; sum.w += v.w;
+    }
+    float4* dst = reinterpret_cast<float4*>(p.C + row * p.ldc + n0 + 4 * c4);
+    float4 o = make_float4(scale * sum.x, scale * sum.y, scale * sum.z, scale * sum.w);
+    if (p.accumulate) { const float4 c = *dst; o.x += c.x; o.y += c.y; o.z += c.z; o.w += c.w; }
+    *dst = o;
+  }
+}
+
+// Optional instrumentation (compile with -DSAPO_WAIT_STATS): cycles each role spends waiting.
+#ifdef SAPO_WAIT_STATS
+__device__ unsigned long long g_wait_stats[4][8];
+#define SAPO_TIMED(slot, expr) ([&] { const long long t0_ = clock64(); const bool r_ = (expr); \
+                                      wait_cycles[slot] += clock64() - t0_; return r_; }())
+#define SAPO_STATS_DECL long long wait_cycles[8] = {0, 0, 0, 0, 0, 0, 0, 0}; const long long role_t0 = clock64();
+#define SAPO_STATS_FLUSH(total_slot) do { wait_cycles[total_slot] += clock64() - role_t0; \
+    for (int i_ = 0; i_ < 8; ++i_) if (wait_cycles[i_]) \
+      atomicAdd(&g_wait_stats[sched.stats_id & 3][i_], (unsigned long long)wait_cycles[i_]); } while (0)
+#else
+#define SAPO_TIMED(slot, expr) (expr)
+#define SAPO_STATS_DECL
+#define SAPO_STATS_FLUSH(total_slot) do {} while (0)
+#endif
+
+}  // namespace sapo

@@ -1,0 +1,251 @@
+// The per-token and per-sequence kernels around the GEMMs: bf16 splitting of fp32 operands, the
+// loss tail of the separate forward, and the small kernels of the single-pass call.
+#pragma once
+
+#include "gemm_sched.cuh"
+
+namespace sapo {
+using namespace umma;
+
+// ---------------------------------------------------------------------------- small kernels
+// fp32 -> bf16 operands.  mode 0: [hi | hi | lo] (A side), mode 1: [hi | lo | hi] (B side),
+// so that sum_k A'[k] B'[k] = hi.hi + hi.lo + lo.hi; mode 2: hi only.
+__global__ void __launch_bounds__(256)
+split_bf16_kernel(const float* __restrict__ X, int64_t ld, int64_t R, int32_t H,
+                  __nv_bfloat16* __restrict__ out, int mode) {
+  const int64_t n = R * (int64_t)H;
+  const int64_t ldo = mode == 2 ? H : 3 * (int64_t)H;
+  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n;
+       i += (int64_t)gridDim.x * blockDim.x) {
+    const int64_t r = i / H; const int32_t c = (int32_t)(i - r * H);
+    const float x = X[r * ld + c];
+    const __nv_bfloat16 hi = __float2bfloat16_rn(x);
+    __nv_bfloat16* o = out + r * ldo;
+    o[c] = hi;
+    if (mode != 2) {
+      const __nv_bfloat16 lo = __float2bfloat16_rn(x - __bfloat162float(hi));
+      o[H + c] = mode == 0 ? hi : lo;
+      o[2 * H + c] = mode == 0 ? lo : hi;
+    }
+  }
+}
+
+struct TailArgs {
+  const float* pm; const float* ps; const float* pz; int32_t n_splits; int64_t T;
+  const int32_t* ids; int32_t V; const float* old_logp; const float* adv; const int32_t* cu; int32_t S;
+  float lo_edge, hi_edge, grad_scale;
+  int32_t loss_agg; float kl_beta; const float* ref_logp;   // variants: token-level mean, KL penalty
+  float* logp; float* lse; float* ratio; float* surr; float* gscale; float* seq_surr;
+  int32_t* status;
+};
+
+__device__ __forceinline__ double block_sum_256(double x, double* sh) {
+  #pragma unroll
+  for (int d = 16; d > 0; d >>= 1) x += __shfl_xor_sync(0xffffffffu, x, d);
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  __syncthreads();
+  if (lane == 0) sh[warp] = x;
+  __syncthreads();
+  double t = 0.0;
+  if (threadIdx.x == 0) for (int i = 0; i < 8; ++i) t += sh[i];
+  return t;   // valid in thread 0
+}
+
+// One block per sequence: merge the vocab-split partials, then the clipped surrogate.
+__global__ void __launch_bounds__(256) loss_tail_kernel(TailArgs a) {
+  __shared__ double sh[8];
+  for (int32_t s = blockIdx.x; s < a.S; s += gridDim.x) {
+    const int32_t t0 = a.cu[s], t1 = a.cu[s + 1];
+    const int32_t Ts = t1 - t0;
+    const float A = a.adv[s];
+    // weight of a token of this sequence: 1/(S T_s) (mean of token means) or 1/T (token mean)
+    const float w = Ts <= 0 ? 0.f : (a.loss_agg == 0 ? 1.f / ((float)a.S * (float)Ts) : 1.f / (float)a.T);
+    double acc = 0.0;
+    for (int32_t t = t0 + threadIdx.x; t < t1; t += 256) {
+      float M = -INFINITY;
+      for (int i = 0; i < a.n_splits; ++i) M = fmaxf(M, a.pm[(int64_t)i * a.T + t]);
+      float sum = 0.f, zy = 0.f;
+      for (int i = 0; i < a.n_splits; ++i) {
+        const int64_t o = (int64_t)i * a.T + t;
+        sum += a.ps[o] * exp2f(a.pm[o] - M);
+        zy += a.pz[o];
+      }
+      const float lse = (M + log2f(sum)) * LN2;
+      const int32_t y = a.ids[t];
+      const bool bad = y < 0 || y >= a.V;
+      if (bad) raise_status(a.status, SAPO_ST_BAD_TOKEN_ID);
+      const float lp = bad ? 0.f : zy - lse;
+      const float rho = bad ? 0.f : expf(lp - a.old_logp[t]);
+      const float un = rho * A;
+      const float cl = fminf(fmaxf(rho, a.lo_edge), a.hi_edge) * A;
+      const float u = bad ? 0.f : fminf(un, cl);
+      float g = (!bad && un <= cl) ? -a.grad_scale * A * rho * w : 0.f;
+      float obj = u;
+      if (a.kl_beta != 0.f && !bad) {
+        // penalty towards a reference policy: kl = e^d - d - 1, d = ref - logp; d kl / d logp = 1 - e^d
+        const float d = a.ref_logp[t] - lp;
+        const float ed = expf(d);
+        obj -= a.kl_beta * (ed - d - 1.f);
+        g += a.grad_scale * w * a.kl_beta * (1.f - ed);
+      }
+      a.lse[t] = lse; a.logp[t] = lp; a.ratio[t] = rho; a.surr[t] = u; a.gscale[t] = g;
+      acc += (double)obj;
+    }
+    const double tot = block_sum_256(acc, sh);
+    if (threadIdx.x == 0) a.seq_surr[s] = Ts > 0 ? (float)(tot / (double)Ts) : 0.f;
+  }
+}
+
+// loss = -(1/S) sum_s seq_surr[s], or with token-level aggregation -(1/T) sum_s T_s seq_surr[s]
+__global__ void __launch_bounds__(256)
+loss_final_kernel(const float* seq_surr, const int32_t* cu, int32_t S, int64_t T, int32_t loss_agg, float* loss) {
+  __shared__ double sh[8];
+  double acc = 0.0;
+  for (int32_t s = threadIdx.x; s < S; s += 256)
+    acc += loss_agg == 0 ? (double)seq_surr[s] : (double)seq_surr[s] * (double)(cu[s + 1] - cu[s]);
+  const double tot = block_sum_256(acc, sh);
+  const double n = loss_agg == 0 ? (double)S : (double)T;
+  if (threadIdx.x == 0) *loss = n > 0 ? (float)(-tot / n) : 0.f;
+}
+
+// ---------------------------------------------------------------------------- fused call: small kernels
+// Before the forward pass of the fused call: the logit of the chosen token, z_y[t] = <h_t, W_y>,
+// as a plain fp32 dot product (one warp per token), and the reference of the exponentials
+//   c_t = z_y[t] - old_logp[t],
+// which equals lse_t when the policy has not moved since old_logp was taken and is off by
+// log(ratio_t) otherwise: exp(z - c_t) then stays within a few powers of e of a probability.
+// c2 is c_t * log2(e).  A token id outside [0, V) gets z_y = c = 0 (the tail reports it).
+__global__ void __launch_bounds__(256)
+target_logit_kernel(const __nv_bfloat16* __restrict__ hidden, int64_t ldh, const __nv_bfloat16* __restrict__ W,
+                    int64_t ldw, const int32_t* __restrict__ ids, const float* __restrict__ old_logp,
+                    int64_t T, int32_t H, int32_t V, float* __restrict__ zy, float* __restrict__ c2) {
+  const int lane = threadIdx.x & 31;
+  const int64_t warp = (int64_t)blockIdx.x * 8 + (threadIdx.x >> 5);
+  const int64_t n_warps = (int64_t)gridDim.x * 8;
+  for (int64_t t = warp; t < T; t += n_warps) {
+    const int32_t y = ids[t];
+    float acc = 0.f;
+    if (y >= 0 && y < V) {
+      const uint4* a = reinterpret_cast<const uint4*>(hidden + t * ldh);
+      const uint4* b = reinterpret_cast<const uint4*>(W + (int64_t)y * ldw);
+      for (int i = lane; i < H / 8; i += 32) {
+        const uint4 ua = a[i], ub = b[i];
+        const __nv_bfloat162* pa = reinterpret_cast<const __nv_bfloat162*>(&ua);
+        const __nv_bfloat162* pb = reinterpret_cast<const __nv_bfloat162*>(&ub);
+        #pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          const float2 fa = __bfloat1622float2(pa[j]), fb = __bfloat1622float2(pb[j]);
+          acc = fmaf(fa.x, fb.x, acc); acc = fmaf(fa.y, fb.y, acc);
+        }
+      }
+      #pragma unroll
+      for (int d = 16; d > 0; d >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, d);
+    }
+    if (lane == 0) {
+      const bool ok = y >= 0 && y < V;
+      zy[t] = ok ? acc : 0.f;
+      c2[t] = ok ? (acc - old_logp[t]) * LOG2E : 0.f;
+    }
+  }
+}
+
+struct FusedTailArgs {
+  const float* ps; int32_t n_parts; int64_t t0, tc;        // partial sums [n_parts][tc] of this token chunk
+  const float* zy; const float* c2;                        // [T]
+  const int32_t* ids; int32_t V; const float* old_logp; const float* adv; const int32_t* cu; int32_t S;
+  int64_t T; float lo_edge, hi_edge, grad_scale; int32_t loss_agg; float kl_beta; const float* ref_logp;
+  float* logp; float* lse; float* ratio; float* surr; float* gscale; float* obj;   // [T]
+  float* row_scale;                                        // [tc]
+  __nv_bfloat16* panel; int32_t nvt;                       // exponentials of the chunk
+  const __nv_bfloat16* hidden; int64_t ldh; int32_t H; __nv_bfloat16* hs;   // hs [tc, H] = row_scale * hidden
+  uint32_t* active_mask;   // one bit per 128-token block of the chunk (zeroed by the caller), or nullptr
+  int32_t* status;
+};
+
+// After the forward pass of a token chunk of the fused call, one warp per token:
+//   sum_t = sum_v exp(z - c_t);  lse = c_t + log sum_t;  logp = z_y - lse;  ratio, surrogate and
+//   g_t = dloss/dlogp as in loss_tail_kernel;
+// then what turns the stored exponentials e into dz = g ([v = y] - e / sum_t) = a_t e' with
+//   a_t = -g_t / sum_t,   e'[t,v] = e[t,v] - [v = y_t] sum_t :
+// the panel entry of the chosen token is replaced by e_y - sum_t, a_t becomes the row scale of
+// the dhidden contraction, and hs = a_t * hidden (bf16) the operand of the dW_head contraction.
+__global__ void __launch_bounds__(256) fused_tail_kernel(FusedTailArgs a) {
+  const int lane = threadIdx.x & 31;
+  const int64_t warp = (int64_t)blockIdx.x * 8 + (threadIdx.x >> 5);
+  const int64_t n_warps = (int64_t)gridDim.x * 8;
+  for (int64_t lr = warp; lr < a.tc; lr += n_warps) {
+    const int64_t t = a.t0 + lr;
+    float part = 0.f;
+    for (int i = lane; i < a.n_parts; i += 32) part += a.ps[(int64_t)i * a.tc + lr];
+    #pragma unroll
+    for (int d = 16; d > 0; d >>= 1) part += __shfl_xor_sync(0xffffffffu, part, d);
+    const float sum = part;
+    // the sequence of this token: last s with cu[s] <= t
+    int lo = 0, hi = a.S - 1;
+    while (lo < hi) { const int mid = (lo + hi + 1) >> 1; if ((int64_t)a.cu[mid] <= t) lo = mid; else hi = mid - 1; }
+    const int32_t Ts = a.cu[lo + 1] - a.cu[lo];
+    const float A = a.adv[lo];
+    const float w = Ts <= 0 ? 0.f : (a.loss_agg == 0 ? 1.f / ((float)a.S * (float)Ts) : 1.f / (float)a.T);
+    const int32_t y = a.ids[t];
+    const bool bad_id = y < 0 || y >= a.V;
+    // a capped exponential, or a sum that left the fp32 range: the reference was too far off
+    const bool bad_range = !(sum < EXP_CAP) || !(sum > 1.f / EXP_CAP);
+    const bool bad = bad_id || bad_range;
+    const float c2 = a.c2[t], zy = a.zy[t];
+    const float lse = bad_range ? 0.f : (c2 + log2f(sum)) * LN2;
+    const float lp = bad ? 0.f : zy - lse;
+    const float rho = bad ? 0.f : expf(lp - a.old_logp[t]);
+    const float un = rho * A;
+    const float cl = fminf(fmaxf(rho, a.lo_edge), a.hi_edge) * A;
+    const float u = bad ? 0.f : fminf(un, cl);
+    float g = (!bad && un <= cl) ? -a.grad_scale * A * rho * w : 0.f;
+    float obj = u;
+    if (a.kl_beta != 0.f && !bad) {
+      const float d = a.ref_logp[t] - lp;
+      const float ed = expf(d);
+      obj -= a.kl_beta * (ed - d - 1.f);
+      g += a.grad_scale * w * a.kl_beta * (1.f - ed);
+    }
+    const float scale = (bad || g == 0.f) ? 0.f : -g / sum;
+    if (lane == 0) {
+      if (bad_id) raise_status(a.status, SAPO_ST_BAD_TOKEN_ID);
+      if (bad_range) raise_status(a.status, SAPO_ST_EXP_RANGE);
+      a.lse[t] = lse; a.logp[t] = lp; a.ratio[t] = rho; a.surr[t] = u; a.gscale[t] = g; a.obj[t] = obj;
+      a.row_scale[lr] = scale;
+      if (scale != 0.f && a.active_mask != nullptr)
+        atomicOr(&a.active_mask[lr >> 12], 1u << ((lr >> 7) & 31));
+      if (!bad) {
+        const float ey = ex2(fmaf(zy, LOG2E, -c2));
+        const int64_t tile = (lr >> 7) * a.nvt + (y >> 6);
+        a.panel[(tile * BM + (lr & 127)) * 64 + (y & 63)] = __float2bfloat16_rn(ey - sum);
+      }
+    }
+    const uint4* src = reinterpret_cast<const uint4*>(a.hidden + t * a.ldh);
+    uint4* dst = reinterpret_cast<uint4*>(a.hs + lr * (int64_t)a.H);
+    for (int i = lane; i < a.H / 8; i += 32) {
+      uint4 x = src[i];
+      __nv_bfloat162* px = reinterpret_cast<__nv_bfloat162*>(&x);
+      #pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const float2 f = __bfloat1622float2(px[j]);
+        px[j] = __floats2bfloat162_rn(scale * f.x, scale * f.y);
+      }
+      dst[i] = x;
+    }
+  }
+}
+
+// seq_surr[s] = mean over the tokens of s of obj[t] (same summation order as loss_tail_kernel)
+__global__ void __launch_bounds__(256)
+seq_mean_kernel(const float* __restrict__ obj, const int32_t* __restrict__ cu, int32_t S, float* seq_surr) {
+  __shared__ double sh[8];
+  for (int32_t s = blockIdx.x; s < S; s += gridDim.x) {
+    const int32_t t0 = cu[s], t1 = cu[s + 1];
+    double acc = 0.0;
+    for (int32_t t = t0 + threadIdx.x; t < t1; t += 256) acc += (double)obj[t];
+    const double tot = block_sum_256(acc, sh);
+    if (threadIdx.x == 0) seq_surr[s] = t1 > t0 ? (float)(tot / (double)(t1 - t0)) : 0.f;
+  }
+}
+
+}  // namespace sapo
