@@ -49,3 +49,20 @@ def test_host_side_helpers():
     f32 = B.sapo_workspace_bytes(B.WS_FWD, 1024, 64, 1000, B.DTYPE_F32)
     assert f32 >= (1024 + 1000) * 3 * 64 * 2
     assert B.decode_status(0x21) == ["TOKEN_OVERFLOW", "WAIT_TIMEOUT"]
+
+
+def test_header_is_plain_c(tmp_path):
+    """include/sapo.h is the boundary: it must compile as C99 on its own (no C++, no CUDA or
+    torch types), and every status / error code it defines must have a text."""
+    import subprocess
+    src = tmp_path / "use_header.c"
+    src.write_text('#include "sapo.h"\n'
+                   "int main(void) { sapo_loss_cfg c; c.eps_low = 0.2f; (void)c;\n"
+                   "  return sizeof(sapo_packed) > 0 && SAPO_WS_FUSED == 3 ? 0 : 1; }\n")
+    inc = os.path.join(ROOT, "include")
+    res = subprocess.run(["gcc", "-std=c99", "-Wall", "-Werror", "-pedantic", "-fsyntax-only", "-I", inc, str(src)],
+                         capture_output=True, text=True)
+    assert res.returncode == 0, res.stderr
+    lib = B.load()
+    for code in range(0, -6, -1):
+        assert lib.sapo_status_string(code) != b"unknown code"
