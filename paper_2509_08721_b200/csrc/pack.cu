@@ -20,6 +20,7 @@ struct PackArgs {
   int32_t* n_tokens; int32_t* n_seqs;
   int64_t max_tokens; int32_t max_seqs;
   int64_t row_bytes;
+  int32_t tokens_per_warp;   // length of the runs of packed tokens a warp copies (even)
   int32_t* status;
 };
 
@@ -108,9 +109,13 @@ __global__ void __launch_bounds__(SCAN_THREADS) pack_scan_kernel(PackArgs a) {
   }
 }
 
-// A warp copies runs of TOKENS_PER_WARP consecutive packed tokens: one binary search per run,
-// then it walks the sequence table; rows move as 16-byte vectors, four loads in flight per lane.
-constexpr int TOKENS_PER_WARP = 8;
+// A warp copies runs of tokens_per_warp consecutive packed tokens (16 for batches that fill
+// the device several times over, 8 below that, so that small batches still spread over all
+// SMs): one binary search per run,
+// then it walks the sequence table, re-reading a sequence's source only when the run crosses
+// into the next sequence.  Rows move as 16-byte vectors; the loads of two tokens (up to eight
+// per lane) are issued before the first store.
+constexpr int ROW_VECS_PER_LANE = 4;     // 16-byte vectors of one row a lane holds at a time
 
 __global__ void __launch_bounds__(256) pack_copy_kernel(PackArgs a) {
   const int lane = threadIdx.x & 31;
@@ -119,7 +124,9 @@ __global__ void __launch_bounds__(256) pack_copy_kernel(PackArgs a) {
   const int32_t T = *a.n_tokens, S = *a.n_seqs;
   const bool vec = (a.row_bytes & 15) == 0;
   const int n4 = (int)(a.row_bytes >> 4);
-  for (int64_t t0 = warp0 * TOKENS_PER_WARP; t0 < a.max_tokens; t0 += n_warps * TOKENS_PER_WARP) {
+  const bool two_at_once = vec && n4 <= 32 * ROW_VECS_PER_LANE;
+  const int tpw = a.tokens_per_warp;
+  for (int64_t t0 = warp0 * tpw; t0 < a.max_tokens; t0 += n_warps * tpw) {
     int32_t s = 0;
     if (t0 < T) {
       // first s with cu[s+1] > t0 (zero-length sequences share a start; take the one that owns t0)
@@ -130,40 +137,90 @@ __global__ void __launch_bounds__(256) pack_copy_kernel(PackArgs a) {
       }
       s = lo;
     }
-    for (int i = 0; i < TOKENS_PER_WARP; ++i) {
-      const int64_t t = t0 + i;
-      if (t >= a.max_tokens) break;
-      if (t >= T) { if (lane == 0) a.tok_mask[t] = 0; continue; }
-      while (a.cu[s + 1] <= t) ++s;
-      const int side = a.seq_is_ext[s];
-      const int64_t src = a.off[side][a.seq_src[s]] + (t - a.cu[s]);
-      const uint8_t* from = a.hid[side] + src * a.row_bytes;
-      uint8_t* to = a.o_hid + t * a.row_bytes;
-      if (vec) {
-        const uint4* f4 = reinterpret_cast<const uint4*>(from);
-        uint4* t4 = reinterpret_cast<uint4*>(to);
-        for (int j = lane; j < n4; j += 128) {
-          uint4 v0, v1, v2, v3;
-          v0 = __ldg(f4 + j);
-          if (j + 32 < n4) v1 = __ldg(f4 + j + 32);
-          if (j + 64 < n4) v2 = __ldg(f4 + j + 64);
-          if (j + 96 < n4) v3 = __ldg(f4 + j + 96);
-          t4[j] = v0;
-          if (j + 32 < n4) t4[j + 32] = v1;
-          if (j + 64 < n4) t4[j + 64] = v2;
-          if (j + 96 < n4) t4[j + 96] = v3;
-        }
-      } else {
-        const uint16_t* f2 = reinterpret_cast<const uint16_t*>(from);
-        uint16_t* t2 = reinterpret_cast<uint16_t*>(to);
-        const int n2 = (int)(a.row_bytes >> 1);
-        for (int j = lane; j < n2; j += 32) t2[j] = f2[j];
+    // the sequence the walk is in: its end, its side and the source token of its first token
+    int32_t seq_end = -1, seq_begin = 0, side = 0;
+    int64_t src0 = 0;
+    auto locate = [&](int64_t t) -> int64_t {       // source token of packed token t (t < T)
+      if (t >= seq_end) {
+        while (a.cu[s + 1] <= t) ++s;
+        seq_begin = a.cu[s]; seq_end = a.cu[s + 1];
+        side = a.seq_is_ext[s];
+        src0 = a.off[side][a.seq_src[s]];
       }
+      return src0 + (t - seq_begin);
+    };
+    auto finish = [&](int64_t t, int64_t src) {     // the per-token scalars
       if (lane == 0) {
         a.o_ids[t] = a.ids[side][src];
         a.o_old[t] = a.old[side][src];
         a.tok_seq[t] = s;
         a.tok_mask[t] = 1;
+      }
+    };
+    for (int i = 0; i < tpw; i += 2) {
+      const int64_t ta = t0 + i, tb = ta + 1;
+      if (ta >= a.max_tokens) break;
+      const bool have_a = ta < T, have_b = tb < T && tb < a.max_tokens;
+      if (!have_a) {
+        if (lane == 0) { a.tok_mask[ta] = 0; if (tb < a.max_tokens) a.tok_mask[tb] = 0; }
+        continue;
+      }
+      if (two_at_once) {
+        const int64_t sa = locate(ta);
+        const uint4* fa = reinterpret_cast<const uint4*>(a.hid[side] + sa * a.row_bytes);
+        uint4 va[ROW_VECS_PER_LANE], vb[ROW_VECS_PER_LANE];
+        #pragma unroll
+        for (int q = 0; q < ROW_VECS_PER_LANE; ++q) if (lane + 32 * q < n4) va[q] = __ldg(fa + lane + 32 * q);
+        finish(ta, sa);
+        int64_t sb = 0;
+        if (have_b) {
+          sb = locate(tb);
+          const uint4* fb = reinterpret_cast<const uint4*>(a.hid[side] + sb * a.row_bytes);
+          #pragma unroll
+          for (int q = 0; q < ROW_VECS_PER_LANE; ++q) if (lane + 32 * q < n4) vb[q] = __ldg(fb + lane + 32 * q);
+        }
+        uint4* oa = reinterpret_cast<uint4*>(a.o_hid + ta * a.row_bytes);
+        #pragma unroll
+        for (int q = 0; q < ROW_VECS_PER_LANE; ++q) if (lane + 32 * q < n4) oa[lane + 32 * q] = va[q];
+        if (have_b) {
+          uint4* ob = reinterpret_cast<uint4*>(a.o_hid + tb * a.row_bytes);
+          #pragma unroll
+          for (int q = 0; q < ROW_VECS_PER_LANE; ++q) if (lane + 32 * q < n4) ob[lane + 32 * q] = vb[q];
+          finish(tb, sb);
+        } else if (tb < a.max_tokens && lane == 0) {
+          a.tok_mask[tb] = 0;
+        }
+        continue;
+      }
+      // wide or unaligned rows: one token at a time
+      for (int k = 0; k < 2; ++k) {
+        const int64_t t = ta + k;
+        if (t >= a.max_tokens) break;
+        if (t >= T) { if (lane == 0) a.tok_mask[t] = 0; continue; }
+        const int64_t src = locate(t);
+        const uint8_t* from = a.hid[side] + src * a.row_bytes;
+        uint8_t* to = a.o_hid + t * a.row_bytes;
+        if (vec) {
+          const uint4* f4 = reinterpret_cast<const uint4*>(from);
+          uint4* t4 = reinterpret_cast<uint4*>(to);
+          for (int j = lane; j < n4; j += 128) {
+            uint4 v0, v1, v2, v3;
+            v0 = __ldg(f4 + j);
+            if (j + 32 < n4) v1 = __ldg(f4 + j + 32);
+            if (j + 64 < n4) v2 = __ldg(f4 + j + 64);
+            if (j + 96 < n4) v3 = __ldg(f4 + j + 96);
+            t4[j] = v0;
+            if (j + 32 < n4) t4[j + 32] = v1;
+            if (j + 64 < n4) t4[j + 64] = v2;
+            if (j + 96 < n4) t4[j + 96] = v3;
+          }
+        } else {
+          const uint16_t* f2 = reinterpret_cast<const uint16_t*>(from);
+          uint16_t* t2 = reinterpret_cast<uint16_t*>(to);
+          const int n2 = (int)(a.row_bytes >> 1);
+          for (int j = lane; j < n2; j += 32) t2[j] = f2[j];
+        }
+        finish(t, src);
       }
     }
   }
@@ -208,7 +265,8 @@ extern "C" int sapo_pack_rollouts(const sapo_rollout_buf* h_local, const sapo_ro
   if (a.max_tokens > 0) {
     const int sms = sm_count();
     if (sms <= 0) return SAPO_ERR_CUDA;
-    const int64_t warps_wanted = (a.max_tokens + TOKENS_PER_WARP - 1) / TOKENS_PER_WARP;
+    a.tokens_per_warp = a.max_tokens >= (int64_t)sms * 64 * 16 ? 16 : 8;
+    const int64_t warps_wanted = (a.max_tokens + a.tokens_per_warp - 1) / a.tokens_per_warp;
     int blocks = (int)((warps_wanted + 7) / 8);
     const int max_blocks = sms * 8;                 // 8 resident blocks of 256 threads per SM
     if (blocks > max_blocks) blocks = max_blocks;
