@@ -57,6 +57,26 @@ group_adv_kernel(const float* __restrict__ rewards, const int32_t* __restrict__ 
   }
 }
 
+// 1/n for the small integers a group size (or size minus ddof) can be on the register path
+__constant__ double c_inv_small[17] = {0.0, 1.0, 1.0 / 2, 1.0 / 3, 1.0 / 4, 1.0 / 5, 1.0 / 6, 1.0 / 7, 1.0 / 8, 1.0 / 9,
+                                       1.0 / 10, 1.0 / 11, 1.0 / 12, 1.0 / 13, 1.0 / 14, 1.0 / 15, 1.0 / 16};
+
+// sqrt and reciprocal in fp64 from an fp32 estimate and one Newton step (relative error about
+// 1e-14, far below the fp32 rounding of the results); arguments outside the comfortable fp32
+// range take the library routine.  The library's fp64 division and square root cost several
+// times more fp64 instructions, and this kernel is bound by them.
+__device__ __forceinline__ double sqrt_newton(double v) {
+  if (!(v > 1e-30 && v < 1e30)) return v > 0.0 ? sqrt(v) : 0.0;
+  double r = (double)rsqrtf((float)v);
+  r = r * (1.5 - 0.5 * v * r * r);
+  return v * r;
+}
+__device__ __forceinline__ double rcp_newton(double x) {
+  if (!(x > 1e-30 && x < 1e30)) return 1.0 / x;
+  double r = (double)(1.f / (float)x);
+  return r * (2.0 - x * r);
+}
+
 // One thread per question, for batches of very many small groups: no shuffles, and the three
 // passes over a group hit L1 after the first.  Groups whose start and size are multiples of
 // four move as float4.
@@ -84,7 +104,7 @@ group_adv_thread_kernel(const float* __restrict__ rewards, const int32_t* __rest
         sum += (double)buf[i].x; sum += (double)buf[i].y; sum += (double)buf[i].z; sum += (double)buf[i].w;
       }
       if (bad) raise_status(status, SAPO_ST_NONFINITE_REWARD);
-      const double mu = sum / (double)G;
+      const double mu = sum * c_inv_small[G];
       double ss = 0.0;
       #pragma unroll
       for (int i = 0; i < 4; ++i) {
@@ -95,8 +115,8 @@ group_adv_thread_kernel(const float* __restrict__ rewards, const int32_t* __rest
         }
       }
       const int32_t denom = G - ddof;
-      const double sd = denom > 0 ? sqrt(ss / (double)denom) : 0.0;
-      const double inv = 1.0 / (sd + adv_eps);
+      const double sd = denom > 0 ? sqrt_newton(ss * c_inv_small[denom]) : 0.0;
+      const double inv = rcp_newton(sd + adv_eps);
       float4* a4 = reinterpret_cast<float4*>(adv + a);
       #pragma unroll
       for (int i = 0; i < 4; ++i)
