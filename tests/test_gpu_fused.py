@@ -206,6 +206,37 @@ def test_random_shapes_single_pass_against_separate_calls(seed):
     assert torch.isfinite(one["dhidden"]).all() and torch.isfinite(one["dW"]).all()
 
 
+@pytest.mark.parametrize("H", [64, 256], ids=["narrow_tiles", "wide_tiles"])
+def test_accumulate_dW_adds_to_what_the_caller_holds(H):
+    """Gradient accumulation over micro-batches: with accumulate_dW set, both the separate
+    backward and the single-pass call add this batch's dW_head to the buffer's contents."""
+    recipe = small_recipe(H=H, V=700, Q=3, length_law=("uniform", 20, 60))
+    batch = gen.make_batch(recipe, 12)
+    adv, ref = oracle_case(batch, 0.2, 0.28)
+    hidden, W, ids, old, advd, cu = device_inputs(batch, adv)
+    T, V = batch.T, recipe.V
+    base = torch.randn(V, H, device="cuda") * ref["dW"].std()
+    want = base.double().cpu().numpy() + ref["dW"]
+    # separate calls
+    out = U.gpu_scores(hidden, W, ids, old, advd, cu, 0.2, 0.28, want_bwd=False)
+    dH, dW = torch.empty(T, H, device="cuda"), base.clone()
+    ws = torch.empty(B.sapo_workspace_bytes(B.WS_BWD, T, H, V, B.DTYPE_BF16), dtype=torch.uint8, device="cuda")
+    status = B.new_status()
+    B.sapo_policy_loss_bwd(hidden, W, ids, out["lse"], out["gscale"], dH, dW, True, ws, status)
+    torch.cuda.synchronize()
+    assert status.item() == 0
+    assert np.linalg.norm(dW.double().cpu().numpy() - want) <= U.TOL_GRAD_FRO * np.linalg.norm(ref["dW"])
+    # single-pass call
+    out2 = B.alloc_fwd_outputs(T, batch.S)
+    dH2, dW2 = torch.empty(T, H, device="cuda"), base.clone()
+    ws2 = torch.empty(B.sapo_workspace_bytes(B.WS_FUSED, T, H, V, B.DTYPE_BF16), dtype=torch.uint8, device="cuda")
+    B.sapo_policy_loss_fwd_bwd(hidden, W, ids, old, advd, cu, 0.2, 0.28, 1.0, out2, dH2, dW2, True, ws2, status)
+    torch.cuda.synchronize()
+    assert status.item() == 0
+    assert np.linalg.norm(dW2.double().cpu().numpy() - want) <= U.TOL_GRAD_FRO * np.linalg.norm(ref["dW"])
+    assert U.rel_fro(dH2.cpu().numpy(), ref["dhidden"]) <= U.TOL_GRAD_FRO
+
+
 def test_fused_flags_bad_ids_and_stale_old_logp():
     recipe = small_recipe(H=64, V=400, Q=2, length_law=("uniform", 20, 40))
     batch = gen.make_batch(recipe, 9)
