@@ -237,6 +237,23 @@ def test_accumulate_dW_adds_to_what_the_caller_holds(H):
     assert U.rel_fro(dH2.cpu().numpy(), ref["dhidden"]) <= U.TOL_GRAD_FRO
 
 
+@pytest.mark.parametrize("H", [72, 264], ids=["narrow_tiles", "wide_tiles"])
+def test_padded_leading_dimensions(H):
+    """hidden and W_head as column slices of wider buffers (leading dimension > H)."""
+    recipe = small_recipe(H=H, V=900, Q=3, length_law=("uniform", 20, 60))
+    batch = gen.make_batch(recipe, 14)
+    adv, ref = oracle_case(batch, 0.2, 0.28)
+    hidden, W, ids, old, advd, cu = device_inputs(batch, adv)
+    big_h = torch.full((batch.T, H + 40), 7.0, dtype=torch.bfloat16, device="cuda")
+    big_W = torch.full((recipe.V, H + 16), -3.0, dtype=torch.bfloat16, device="cuda")
+    big_h[:, :H] = hidden
+    big_W[:, :H] = W
+    hv, Wv = big_h[:, :H], big_W[:, :H]
+    assert hv.stride(0) == H + 40 and Wv.stride(0) == H + 16
+    check_all(U.gpu_scores_fused(hv, Wv, ids, old, advd, cu, 0.2, 0.28), ref, adv, batch, 0.2, 0.28)
+    check_all(U.gpu_scores(hv, Wv, ids, old, advd, cu, 0.2, 0.28), ref, adv, batch, 0.2, 0.28)
+
+
 def test_fused_flags_bad_ids_and_stale_old_logp():
     recipe = small_recipe(H=64, V=400, Q=2, length_law=("uniform", 20, 40))
     batch = gen.make_batch(recipe, 9)
