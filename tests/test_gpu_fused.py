@@ -254,6 +254,28 @@ def test_padded_leading_dimensions(H):
     check_all(U.gpu_scores(hv, Wv, ids, old, advd, cu, 0.2, 0.28), ref, adv, batch, 0.2, 0.28)
 
 
+@pytest.mark.parametrize("H", [64, 256], ids=["narrow_tiles", "wide_tiles"])
+def test_peaked_distributions(H):
+    """Logits with a standard deviation of about 8, as a trained head has, instead of the
+    near-uniform softmax of a freshly drawn one: half of the chosen tokens are the arg-max
+    (probability close to 1, so 1 - p is a difference of nearly equal numbers), the other half
+    are random (log-probs of -20 and below)."""
+    recipe = small_recipe(H=H, V=2000, Q=4, length_law=("uniform", 30, 60))
+    batch = gen.make_batch(recipe, 41)
+    rng = np.random.default_rng(5)
+    batch.W = gen.draw_W(rng, recipe.V, H, recipe.dtype, std=8.0 / np.sqrt(H))
+    b = batch.built
+    z = gen.as_f32(b.hidden).astype(np.float64) @ gen.as_f32(batch.W).astype(np.float64).T
+    top = z.argmax(axis=1).astype(np.int32)
+    pick = rng.random(batch.T) < 0.5
+    b.ids[pick] = top[pick]
+    adv, ref = oracle_case(batch, 0.2, 0.28)
+    assert np.exp(ref["logp"]).max() > 0.99 and ref["logp"].min() < -20
+    args = device_inputs(batch, adv)
+    check_all(U.gpu_scores(*args, 0.2, 0.28), ref, adv, batch, 0.2, 0.28)
+    check_all(U.gpu_scores_fused(*args, 0.2, 0.28), ref, adv, batch, 0.2, 0.28)
+
+
 def test_fused_flags_bad_ids_and_stale_old_logp():
     recipe = small_recipe(H=64, V=400, Q=2, length_law=("uniform", 20, 40))
     batch = gen.make_batch(recipe, 9)
