@@ -14,6 +14,12 @@
  *                          separate lower/upper clip thresholds (Section 4.2)
  *   sapo_policy_loss_bwd   gradient of that loss w.r.t. the final hidden states and the
  *                          LM-head weight (Algorithm 1, PolicyGradient)
+ *   sapo_policy_loss_fwd_bwd  the two above in one call that passes over the logits once
+ *                          (bf16 operands; the fastest way through a training step)
+ *
+ * and, around them, sapo_select_external (filter and sample the shared pool, Section 3.2 /
+ * Section 5), sapo_policy_loss_bwd_active (backward over tokens with a gradient only) and
+ * sapo_adam_step (the optimiser step of Section 4.2 on the LM head).
  *
  * General rules
  *   - Every pointer is a DEVICE pointer unless its name starts with h_.  The caller owns
