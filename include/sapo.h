@@ -246,7 +246,7 @@ int sapo_policy_loss_bwd_active(const void* hidden, const void* W_head, int32_t 
  *   dW_head[v,:] = sum_t e'[t,v] (a_t hidden[t,:])   (scaled bf16 copy of hidden as operand)
  * are two tensor-core contractions over the panel: 6 T V H flops instead of the 8 T V H of the
  * separate calls, which recompute the logits.  The price is the range of e: if old_logp[t] is so
- * stale that |log ratio| approaches 69 (e reaches 2^100 or the sum drops below 2^-100), the token
+ * stale that |log ratio| approaches 69 (the sum of e reaches 2^100 or drops below 2^-100), the token
  * is scored as masked (surr = gscale = 0) and SAPO_ST_EXP_RANGE is set; such batches need the
  * separate calls.  bf16 operands only (SAPO_DTYPE_F32 returns SAPO_ERR_UNSUPPORTED_SHAPE).
  * Arguments as in the two separate calls.  workspace: sapo_workspace_bytes(SAPO_WS_FUSED, ...)

@@ -153,9 +153,10 @@ struct DzEpi {
 // is known before the pass (see sapo_policy_loss_fwd_bwd), so no running maximum is needed:
 // the epilogue adds the fp32 exponentials up per token and leaves them, rounded to bf16, in
 // the tiled panel (same layout as DzEpi) for the backward contractions, which then need no
-// second pass over the logits.  Exponentials are capped at 2^100, so that sums and products
-// with them stay finite and a zero row scale later still gives zero (a token that reaches the
-// cap is reported, see fused_tail_kernel).  Rows past the last token and columns past V hold zeros.
+// second pass over the logits.  Nothing is clamped here: a token whose exponentials leave the
+// safe range (2^100 and beyond, infinite or NaN) shows in its sum, and fused_tail_kernel then
+// reports it and clears its panel row, so that the backward contractions only ever see finite
+// entries.  Rows past the last token and columns past V hold zeros.
 struct ExpEpi {
   static constexpr bool STAGED = true;
   static constexpr bool STREAMK = false;
@@ -186,9 +187,8 @@ struct ExpEpi {
       for (int j = 0; j < 16; ++j) packed[j] = 0u;
       return;
     }
-    const float cap = EXP_CAP;
     #pragma unroll
-    for (int j = 0; j < 32; ++j) v[j] = fminf(ex2(fmaf(v[j], LOG2E, -c)), cap);
+    for (int j = 0; j < 32; ++j) v[j] = ex2(fmaf(v[j], LOG2E, -c));
     if (col0 + 32 > p.V) {               // ragged end of the vocabulary
       #pragma unroll
       for (int j = 0; j < 32; ++j) if (col0 + j >= p.V) v[j] = 0.f;

@@ -29,7 +29,7 @@ constexpr uint32_t STAGING_BYTES = 2 * 128 * 128;   // dz epilogue: one 16 KB pa
 constexpr size_t GEMM_SMEM_BYTES = 1024 + STAGES * (A_STAGE_BYTES + B_STAGE_BYTES) + 256;
 constexpr float LOG2E = 1.4426950408889634f;
 constexpr float LN2 = 0.6931471805599453f;
-constexpr float EXP_CAP = 1.2676506002282294e30f;   // 2^100: cap of a stored exponential (fused call)
+constexpr float EXP_CAP = 1.2676506002282294e30f;   // 2^100: a row sum of exponentials at or beyond this is out of range (fused call)
 
 // Static tile schedule: `num_units` work units, each one 256-row block and a run of n-blocks,
 // dealt round-robin to the CTA pairs.

@@ -188,7 +188,7 @@ __global__ void __launch_bounds__(256) fused_tail_kernel(FusedTailArgs a) {
     const float w = Ts <= 0 ? 0.f : (a.loss_agg == 0 ? 1.f / ((float)a.S * (float)Ts) : 1.f / (float)a.T);
     const int32_t y = a.ids[t];
     const bool bad_id = y < 0 || y >= a.V;
-    // a capped exponential, or a sum that left the fp32 range: the reference was too far off
+    // a sum of exponentials that left the safe range (or is not a number): the reference was too far off
     const bool bad_range = !(sum < EXP_CAP) || !(sum > 1.f / EXP_CAP);
     const bool bad = bad_id || bad_range;
     const float c2 = a.c2[t], zy = a.zy[t];
@@ -219,6 +219,13 @@ __global__ void __launch_bounds__(256) fused_tail_kernel(FusedTailArgs a) {
         const int64_t tile = (lr >> 7) * a.nvt + (y >> 6);
         a.panel[(tile * BM + (lr & 127)) * 64 + (y & 63)] = __float2bfloat16_rn(ey - sum);
       }
+    }
+    if (!(sum < EXP_CAP)) {
+      // huge, infinite or NaN exponentials in this row: clear it (the row scale is zero, but
+      // zero times a non-finite entry would still poison dW_head); rare, so one warp does it
+      uint32_t* row32 = reinterpret_cast<uint32_t*>(a.panel);
+      for (int vt = 0; vt < a.nvt; ++vt)
+        row32[((((lr >> 7) * (int64_t)a.nvt + vt) * BM + (lr & 127)) * 64 >> 1) + lane] = 0u;
     }
     const uint4* src = reinterpret_cast<const uint4*>(a.hidden + t * a.ldh);
     uint4* dst = reinterpret_cast<uint4*>(a.hs + lr * (int64_t)a.H);

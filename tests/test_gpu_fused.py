@@ -295,6 +295,18 @@ def test_fused_flags_bad_ids_and_stale_old_logp():
     assert out["status"] == 0x80
     assert out["gscale"][5].item() == 0 and torch.all(out["dhidden"][5] == 0)
     assert torch.isfinite(out["dW"]).all() and torch.isfinite(out["dhidden"]).all()
+    # and 200 nats above it: the exponentials overflow; the row is flagged and cleared, and the
+    # other tokens' results are untouched
+    old_stale = old.clone(); old_stale[6] += 200.0
+    out = U.gpu_scores_fused(hidden, W, ids, old_stale, advd, cu, 0.2, 0.28)
+    assert out["status"] == 0x80
+    assert out["gscale"][6].item() == 0 and torch.all(out["dhidden"][6] == 0)
+    assert torch.isfinite(out["dW"]).all() and torch.isfinite(out["dhidden"]).all()
+    keep = np.ones(batch.T, dtype=bool); keep[6] = False
+    assert np.max(np.abs(out["logp"].cpu().numpy()[keep] - ref["logp"][keep])) <= U.TOL_LOGP_ABS
+    clean = U.gpu_scores_fused(hidden, W, ids, old, advd, cu, 0.2, 0.28)
+    rows = torch.from_numpy(np.nonzero(keep)[0]).cuda()
+    assert torch.equal(out["dhidden"][rows], clean["dhidden"][rows])
 
 
 def test_fused_argument_errors():
