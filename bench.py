@@ -360,8 +360,8 @@ def run_ours(args):
         # (profiles/umma_gemm_kernels_*_workload2_lengths_div4.md): fixed part + bytes per token.
         # Only valid for hidden 896 / vocab 151936, the shape that capture ran at.
         ncu_traffic = {"fwd_gemm": (0.272e9, 12.4e3), "bwd_dz": (0.272e9, 299.6e3),
-                       "fwd_exp": (0.272e9, 309.5e3), "bwd_dh": (0.405e9, 310.7e3),
-                       "bwd_dw": (0.663e9, 310.7e3)}
+                       "fwd_exp": (0.272e9, 309.5e3), "bwd_dh": (0.52e9, 310.7e3),
+                       "bwd_dw": (0.60e9, 310.7e3)}
         if args.backward != "fused":     # the separate backward's dH / dW launches were captured earlier
             ncu_traffic.update({"bwd_dh": (0.272e9, 310.8e3), "bwd_dw": (0.515e9, 332.3e3)})
         traffic = None

@@ -19,14 +19,22 @@ inline int check_launch() {
 
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
+constexpr int MAX_DEVICES = 64;   // devices of one process the per-device caches below cover
+
+// index of the current device, or -1 (no device, or more devices than the caches cover)
+inline int current_device() {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= MAX_DEVICES) return -1;
+  return dev;
+}
+
+// SM count of the current device (looked up once per device)
 inline int sm_count() {
-  static int n = 0;
-  if (n == 0) {
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess) return 0;
-    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) n = 0;
-  }
-  return n;
+  static int n[MAX_DEVICES] = {0};
+  const int dev = current_device();
+  if (dev < 0) return 0;
+  if (n[dev] == 0 && cudaDeviceGetAttribute(&n[dev], cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) n[dev] = 0;
+  return n[dev];
 }
 
 // Optional per-kernel timing and launch counting (see sapo_timing_* in sapo.h).

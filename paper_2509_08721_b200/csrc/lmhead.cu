@@ -128,7 +128,12 @@ template <int A_KIND, bool B_MN, class Epi>
 static int launch_gemm(const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& mc, const Sched& sched,
                        const typename Epi::Params& ep, int32_t* status, cudaStream_t st, int kernel_id) {
   auto kern = umma_gemm_kernel<A_KIND, B_MN, Epi>;
-  static int max_pairs = 0;     // CTA pairs the device can hold at once, found on first use
+  // CTA pairs the device can hold at once; found, together with the kernel's shared-memory
+  // opt-in, on the first use on each device
+  static int max_pairs_of[MAX_DEVICES] = {0};
+  const int dev = current_device();
+  if (dev < 0) return SAPO_ERR_CUDA;
+  int& max_pairs = max_pairs_of[dev];
   if (sched.num_units <= 0) return SAPO_OK;
   Sched sc = sched;
   sc.stats_id = (kernel_id == SAPO_K_FWD_GEMM || kernel_id == SAPO_K_FWD_EXP) ? 0 : kernel_id - SAPO_K_BWD_DZ + 1;
@@ -204,7 +209,10 @@ static int launch_gemm_wide(const CUtensorMap& ma, const CUtensorMap& mb, const 
   CUtensorMap mc;
   if (!make_map_f32_out(&mc, ep.C, ep.N, ep.M, ep.ldc)) return SAPO_ERR_CUDA;
   auto kern = umma_gemm2_kernel<A_KIND>;
-  static int max_pairs = 0;
+  static int max_pairs_of[MAX_DEVICES] = {0};   // as in launch_gemm: per device, found on first use
+  const int dev = current_device();
+  if (dev < 0) return SAPO_ERR_CUDA;
+  int& max_pairs = max_pairs_of[dev];
   if (sched.num_units <= 0) return SAPO_OK;
   Sched sc = sched;
   cudaLaunchAttribute attr[1];
@@ -515,7 +523,6 @@ extern "C" int sapo_policy_loss_fwd(const void* hidden, const void* W_head, int3
 static __device__ __align__(256) unsigned char g_static_fwd_scratch[SAPO_STATIC_SCRATCH_BYTES];
 
 namespace sapo {
-constexpr int MAX_DEVICES = 64;
 // Device address of the array on each GPU.  In host code the symbol's name is only a handle;
 // the address a kernel can use has to be asked for, once per device, with that device current.
 static void* g_static_scratch_ptr[MAX_DEVICES] = {nullptr};
