@@ -65,6 +65,8 @@ extern "C" {
 #define SAPO_ST_EXP_RANGE        0x80  /* fused call: old_logp[t] is so far from the current
                                           log-prob that exp(z - c_t) left the safe range; the
                                           token is scored as masked: use the separate calls   */
+#define SAPO_ST_NONFINITE_INPUT  0x100 /* old_logp[t] or the advantage of its sequence is NaN or
+                                          infinite: the token is scored as masked               */
 
 /* element types of hidden / W_head */
 #define SAPO_DTYPE_BF16 0
@@ -149,9 +151,14 @@ typedef struct sapo_loss_cfg {
  * Gathers the selected rollouts into one token-major batch.  Sequence order: questions in
  * order; inside a question its local picks in list order, then its external picks in list
  * order.  Copies are byte-exact.  H is the row width in elements, `dtype` a SAPO_DTYPE_*.
- * Errors: a NULL struct or negative size returns SAPO_ERR_INVALID_ARG; a bad index, an
- * empty rollout or a capacity overflow sets the matching status bit (bad or empty picks are
- * packed as length-0 sequences, tokens beyond max_tokens are dropped). */
+ * Slots [T, max_tokens) of hidden, ids and old_logp are zero-filled (tok_mask 0, tok_seq -1),
+ * so a caller that must not read n_tokens back can score the whole capacity: the loss calls
+ * treat tokens that belong to no sequence as masked.
+ * Errors: a NULL struct, a NULL array that the sizes say will be touched (outputs when the
+ * capacities are positive, the members of a rollout buffer that holds rollouts; the index lists
+ * may be NULL when empty) or a negative size returns SAPO_ERR_INVALID_ARG before anything is
+ * launched; a bad index, an empty rollout or a capacity overflow sets the matching status bit
+ * (bad or empty picks are packed as length-0 sequences, tokens beyond max_tokens are dropped). */
 int sapo_pack_rollouts(const sapo_rollout_buf* h_local, const sapo_rollout_buf* h_ext,
                        const sapo_selection* h_sel, int32_t H, int32_t dtype,
                        const sapo_packed* h_out, int32_t* status, void* stream);
@@ -179,6 +186,14 @@ int sapo_group_advantages(const float* rewards, const int32_t* group_offsets, in
  * split on the device into bf16 high and low parts (3 products), which keeps log-probs at
  * fp32 accuracy.  adv [S], cu_seqlens [S+1].  Outputs logp, lse, ratio, surr, gscale [T]
  * and loss [1] (float32); seq_surr [S] (token-mean surrogate per sequence) may be NULL.
+ * cu_seqlens must be non-decreasing with every entry in [0, T]; normally cu_seqlens[0] = 0 and
+ * cu_seqlens[S] = T, but T may also be the capacity of the buffers (sapo_pack_rollouts leaves the
+ * token count on the device): tokens of [0, T) before cu_seqlens[0] or from cu_seqlens[S] on
+ * belong to no sequence and are scored as masked (all five per-token outputs 0, no gradient).
+ * Their hidden rows are still read by the projection and must hold finite numbers
+ * (sapo_pack_rollouts zero-fills them).  An entry of cu_seqlens outside [0, T] or below its
+ * predecessor is clamped and sets SAPO_ST_BAD_INDEX.  A NaN or infinite old_logp[t] or adv[s]
+ * sets SAPO_ST_NONFINITE_INPUT and masks the token(s) (ratio = surr = gscale = 0).
  * workspace: at least sapo_workspace_bytes(SAPO_WS_FWD, ...) bytes.
  * Errors: bad arguments / unaligned pointers -> SAPO_ERR_INVALID_ARG; H or V beyond the
  * supported range -> SAPO_ERR_UNSUPPORTED_SHAPE; small workspace ->
@@ -301,19 +316,24 @@ size_t sapo_workspace_bytes_min(int32_t which, int64_t T, int32_t H, int32_t V, 
 /* Forward pass without caller-provided scratch (the paper has no counterpart; this exists for
  * hosts that are not allowed to allocate device memory: a component embedded in a process whose
  * memory pool is fixed once at start-up, or a loop that must never reach cudaMalloc because it
- * synchronises the whole device).  Same arguments, results and error rules as
- * sapo_policy_loss_fwd, except that `workspace` is gone: the scratch is an array of
- * SAPO_STATIC_SCRATCH_BYTES that is part of the library image, so every GPU that loads the
- * library carries it until the process ends.  The call itself allocates and frees nothing.
- * Limits: bf16 operands only (SAPO_ERR_UNSUPPORTED_SHAPE otherwise), and the forward scratch for
- * these sizes — sapo_workspace_bytes(SAPO_WS_FWD, ...), plus 4*S bytes when seq_surr is NULL —
- * must fit; if not, the call does nothing and returns SAPO_ERR_STATIC_SCRATCH_EXCEEDED.  With one
- * vocab split (at least as many 256-token blocks as SM pairs) that is about 170,000 tokens.
+ * synchronises the whole device).  Same arguments and results as sapo_policy_loss_fwd, and the
+ * same argument checks in the same order, except that `workspace` is gone: the scratch is an
+ * array of SAPO_STATIC_SCRATCH_BYTES that is part of the library image, so every GPU that loads
+ * the library carries it until the process ends.  The call itself allocates and frees nothing.
+ * Limits, checked after the common argument checks: bf16 operands only
+ * (SAPO_ERR_UNSUPPORTED_SHAPE otherwise), and
+ *     24 * T bytes  (+ 4 * S, rounded up to 256, when seq_surr is NULL)  <=  SAPO_STATIC_SCRATCH_BYTES,
+ * i.e. up to 174,762 tokens; beyond that the call does nothing and returns
+ * SAPO_ERR_STATIC_SCRATCH_EXCEEDED.  The forward keeps 24 bytes per token and vocab split; this
+ * entry takes as many of the splits the regular call would use as fit in the array.  When all of
+ * them fit the results are bit-identical to sapo_policy_loss_fwd; with fewer splits they agree up
+ * to the order in which a token's partial sums are added (and large batches of few tokens per SM
+ * pair run somewhat slower).
  * The first call on each device looks up the array's device address (that device must be
- * current); make that first call outside any stream capture.  All calls on a device share the
- * one array and it keeps whatever the previous call left: nothing in it needs clearing between
- * calls, but two calls that may run on the GPU at the same time (different streams, or
- * different threads) race on it and must be ordered by the caller. */
+ * current); make that first call outside any stream capture, and from one thread.  All calls on
+ * a device share the one array and it keeps whatever the previous call left: nothing in it needs
+ * clearing between calls, but two calls that may run on the GPU at the same time (different
+ * streams, or different threads) race on it and must be ordered by the caller. */
 #define SAPO_STATIC_SCRATCH_BYTES (4 * 1024 * 1024)
 int sapo_policy_loss_fwd_static(const void* hidden, const void* W_head, int32_t dtype,
                                 int64_t T, int32_t H, int32_t V, int64_t ld_hidden, int64_t ld_W,

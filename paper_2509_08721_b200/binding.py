@@ -24,6 +24,7 @@ WS_FUSED = 3
 ST_BITS = {
     0x01: "TOKEN_OVERFLOW", 0x02: "SEQ_OVERFLOW", 0x04: "BAD_INDEX", 0x08: "EMPTY_SEQUENCE",
     0x10: "BAD_TOKEN_ID", 0x20: "WAIT_TIMEOUT", 0x40: "NONFINITE_REWARD", 0x80: "EXP_RANGE",
+    0x100: "NONFINITE_INPUT",
 }
 
 EXPORTS = ("sapo_pack_rollouts", "sapo_group_advantages", "sapo_policy_loss_fwd",

@@ -11,38 +11,28 @@ using namespace umma;
 // ---------------------------------------------------------------------------- epilogues
 // Each epilogue thread owns one accumulator row (TMEM lane) of the tile.
 
-// What a staged epilogue needs to move finished 64-column groups through shared memory.
-struct StageCtx {
-  uint32_t buf;          // shared address of this column half's 16 KB staging tile
-  int bar_id;            // named barrier of the four warps that share it
-  bool elected;          // the one thread that issues and tracks the TMA stores
-  const CUtensorMap* map;
-};
-
-// A thread's 64 finished bf16 entries of a panel row (two 32-column chunks as 16 pairs each)
-// go to the staging tile, and the tile leaves as one 16 KB TMA store: wait until the previous
-// store has read the staging tile, write this row (128 bytes, in 128-byte-swizzle order) and
-// hand the tile to the TMA.  Called by all 128 threads that share the staging tile.
-__device__ __forceinline__ void store_panel_group(const StageCtx& cx, int r, const uint32_t (&pk)[2][16],
+// A thread's 64 finished bf16 entries of a panel row (two 32-column chunks as 16 pairs each) go
+// straight from its registers to the tile's row in global memory: the row is 128 contiguous
+// bytes, written as four 32-byte stores, so every store fills whole sectors.  (Staging the tile
+// in shared memory for one TMA store per tile was measured slower: the kernel's operand traffic
+// already fills the shared-memory bandwidth, and the staged copy took the MMA issuer's share:
+// 4-5 % more cycles per launch.)
+__device__ __forceinline__ void store_panel_group(__nv_bfloat16* panel, int r, const uint32_t (&pk)[2][16],
                                                   int tile_row0, int col0_of_group) {
-  if (cx.elected) bulk_wait_read_all();
-  named_barrier_sync(cx.bar_id, 128);
+  uint8_t* dst = reinterpret_cast<uint8_t*>(panel) +
+                 ((size_t)tile_row0 + (size_t)(col0_of_group >> 6) * BM + (size_t)r) * 128;
   #pragma unroll
-  for (int q = 0; q < 8; ++q)
-    st_shared_v4(cx.buf + r * 128 + ((q ^ (r & 7)) << 4),
-                 pk[q >> 2][4 * (q & 3)], pk[q >> 2][4 * (q & 3) + 1],
-                 pk[q >> 2][4 * (q & 3) + 2], pk[q >> 2][4 * (q & 3) + 3]);
-  fence_proxy_async_smem();
-  named_barrier_sync(cx.bar_id, 128);
-  if (cx.elected) {
-    tma_store_2d(cx.map, cx.buf, 0, tile_row0 + (col0_of_group >> 6) * BM);
-    bulk_commit_group();
+  for (int q = 0; q < 4; ++q) {
+    const uint32_t* w = &pk[q >> 1][8 * (q & 1)];
+    asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
+                 ::"l"(dst + 32 * q), "r"(w[0]), "r"(w[1]), "r"(w[2]), "r"(w[3]), "r"(w[4]), "r"(w[5]), "r"(w[6]), "r"(w[7])
+                 : "memory");
   }
 }
 
 // Forward: online log-sum-exp in the base-2 domain plus the logit of the chosen token.
 struct FwdEpi {
-  static constexpr bool STAGED = false;
+  static constexpr bool PANEL = false;
   static constexpr bool STREAMK = false;
   template <class P> __device__ static void set_dynamic(P&, const Sched&) {}
 
@@ -57,7 +47,7 @@ struct FwdEpi {
     y = row < p.T ? p.ids[row] : -1;
   }
   template <int HALF>
-  __device__ __forceinline__ void chunk(const Params& p, float (&v)[32], int col0, const StageCtx&) {
+  __device__ __forceinline__ void chunk(const Params& p, float (&v)[32], int col0) {
     if (col0 >= p.V) return;
     if (col0 + 32 > p.V) {
       #pragma unroll
@@ -90,10 +80,10 @@ struct FwdEpi {
 // The panel is a sequence of [128 token x 64 vocab] tiles of 16 KB, tile (tb, vt) at index
 // tb * nvt + vt, each tile row-major: both later contractions then fetch whole contiguous
 // tiles with one TMA box.  Rows past the last token and columns past V are written as zeros,
-// because those consumers cannot tell them from data.  A finished 64-column group is staged in
-// shared memory (128-byte swizzle) and leaves as one 16 KB TMA store.
+// because those consumers cannot tell them from data.  A finished 64-column group of a row is
+// written by its thread (store_panel_group).
 struct DzEpi {
-  static constexpr bool STAGED = true;
+  static constexpr bool PANEL = true;
   static constexpr bool STREAMK = false;
   template <class P> __device__ static void set_dynamic(P& p, const Sched& s) {
     if (s.dyn_dim == 1) p.M = *s.dyn_count;
@@ -101,6 +91,7 @@ struct DzEpi {
   struct Params {
     const int32_t* ids; const float* lse; const float* gscale;
     int64_t M; int32_t V; int32_t nvt;
+    __nv_bfloat16* panel;
   };
   float g, l2; int32_t y; int32_t tile_row0; int r; bool in_panel;
   __device__ __forceinline__ void begin_unit(const Params& p, int mb, int r_) {
@@ -113,11 +104,10 @@ struct DzEpi {
     l2 = valid ? p.lse[row] * LOG2E : 0.f;
     y = valid ? p.ids[row] : -1;
   }
-  __device__ __forceinline__ void group_begin(const StageCtx&) {}
   // dz of 32 columns, kept in registers as 16 bf16 pairs until the whole 64-column group is done
   uint32_t pk[2][16];
   template <int HALF>   // which 32-column half of the group (a compile-time register choice)
-  __device__ __forceinline__ void chunk(const Params& p, float (&v)[32], int col0, const StageCtx&) {
+  __device__ __forceinline__ void chunk(const Params& p, float (&v)[32], int col0) {
     if (!in_panel) return;
     uint32_t (&packed)[16] = pk[HALF];
     if (g == 0.f) {
@@ -143,8 +133,8 @@ struct DzEpi {
       }
     }
   }
-  __device__ __forceinline__ void group_end(const Params&, int col0_of_group, const StageCtx& cx) {
-    if (in_panel) store_panel_group(cx, r, pk, tile_row0, col0_of_group);
+  __device__ __forceinline__ void group_end(const Params& p, int col0_of_group) {
+    if (in_panel) store_panel_group(p.panel, r, pk, tile_row0, col0_of_group);
   }
   __device__ __forceinline__ void end_unit(const Params&, int, int) {}
 };
@@ -158,13 +148,14 @@ struct DzEpi {
 // reports it and clears its panel row, so that the backward contractions only ever see finite
 // entries.  Rows past the last token and columns past V hold zeros.
 struct ExpEpi {
-  static constexpr bool STAGED = true;
+  static constexpr bool PANEL = true;
   static constexpr bool STREAMK = false;
   template <class P> __device__ static void set_dynamic(P&, const Sched&) {}
   struct Params {
     const float* c2;      // [M] reference of each token, in the base-2 domain (c_t * log2 e)
     float* ps;            // [2 * n_splits][M] partial sums of exponentials
     int64_t M; int32_t V; int32_t nvt;
+    __nv_bfloat16* panel;
   };
   float c, sum; int32_t tile_row0; int r; bool valid, in_panel; int64_t row;
   uint32_t pk[2][16];
@@ -177,9 +168,8 @@ struct ExpEpi {
     c = valid ? p.c2[row] : 0.f;
     sum = 0.f;
   }
-  __device__ __forceinline__ void group_begin(const StageCtx&) {}
   template <int HALF>
-  __device__ __forceinline__ void chunk(const Params& p, float (&v)[32], int col0, const StageCtx&) {
+  __device__ __forceinline__ void chunk(const Params& p, float (&v)[32], int col0) {
     if (!in_panel) return;
     uint32_t (&packed)[16] = pk[HALF];
     if (!valid || col0 >= p.V) {
@@ -203,8 +193,8 @@ struct ExpEpi {
       packed[j] = *reinterpret_cast<uint32_t*>(&h);
     }
   }
-  __device__ __forceinline__ void group_end(const Params&, int col0_of_group, const StageCtx& cx) {
-    if (in_panel) store_panel_group(cx, r, pk, tile_row0, col0_of_group);
+  __device__ __forceinline__ void group_end(const Params& p, int col0_of_group) {
+    if (in_panel) store_panel_group(p.panel, r, pk, tile_row0, col0_of_group);
   }
   // two threads share a row (one per column half of the tiles): each leaves its own partial
   __device__ __forceinline__ void end_unit(const Params& p, int un, int col_half) {
@@ -214,7 +204,7 @@ struct ExpEpi {
 
 // Plain fp32 output tile, optionally added to what is already there.
 struct StoreEpi {
-  static constexpr bool STAGED = false;
+  static constexpr bool PANEL = false;
   static constexpr bool STREAMK = true;
   // row_map (optional): output row of each accumulator row (rows of compacted tokens go back
   // to their packed positions)
@@ -240,7 +230,7 @@ struct StoreEpi {
                     : p.partials + ((size_t)slot * PAIR_M + (size_t)(rank * BM + r)) * part_ld;
   }
   template <int HALF>
-  __device__ __forceinline__ void chunk(const Params& p, float (&v)[32], int col0, const StageCtx&) {
+  __device__ __forceinline__ void chunk(const Params& p, float (&v)[32], int col0) {
     if (part != nullptr) {
       float4* dst = reinterpret_cast<float4*>(part + (col0 - n0));
       #pragma unroll
@@ -302,7 +292,17 @@ streamk_fixup_kernel(const Sched s_arg, const StoreEpi::Params p_arg, int pairs)
 
 // Optional instrumentation (compile with -DSAPO_WAIT_STATS): cycles each role spends waiting.
 #ifdef SAPO_WAIT_STATS
-__device__ unsigned long long g_wait_stats[4][8];
+__device__ unsigned long long g_wait_stats[4][12];   // [8] SM cycles, [9] nanoseconds, [10] launches of CTA 0
+__device__ __forceinline__ unsigned long long global_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+#define SAPO_CLOCK_BEGIN const long long clk_c0_ = clock64(); const unsigned long long clk_n0_ = global_ns();
+#define SAPO_CLOCK_END(id) do { if (blockIdx.x == 0 && threadIdx.x == 0) { \
+    atomicAdd(&g_wait_stats[(id) & 3][8], (unsigned long long)(clock64() - clk_c0_)); \
+    atomicAdd(&g_wait_stats[(id) & 3][9], global_ns() - clk_n0_); \
+    atomicAdd(&g_wait_stats[(id) & 3][10], 1ull); } } while (0)
 #define SAPO_TIMED(slot, expr) ([&] { const long long t0_ = clock64(); const bool r_ = (expr); \
                                       wait_cycles[slot] += clock64() - t0_; return r_; }())
 #define SAPO_STATS_DECL long long wait_cycles[8] = {0, 0, 0, 0, 0, 0, 0, 0}; const long long role_t0 = clock64();
@@ -313,6 +313,8 @@ __device__ unsigned long long g_wait_stats[4][8];
 #define SAPO_TIMED(slot, expr) (expr)
 #define SAPO_STATS_DECL
 #define SAPO_STATS_FLUSH(total_slot) do {} while (0)
+#define SAPO_CLOCK_BEGIN
+#define SAPO_CLOCK_END(id) do {} while (0)
 #endif
 
 }  // namespace sapo

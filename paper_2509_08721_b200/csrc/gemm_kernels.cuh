@@ -24,8 +24,8 @@ using namespace umma;
 template <int A_KIND, bool B_MN, class Epi>
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
 umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
-                 const __grid_constant__ CUtensorMap map_c,   // output tiles of a staged epilogue
                  const Sched sched_arg, const typename Epi::Params ep_arg, int32_t* status) {
+  SAPO_CLOCK_BEGIN
   Sched sched = sched_arg;
   typename Epi::Params ep = ep_arg;
   finalize_sched(sched, (int)(gridDim.x >> 1));
@@ -34,8 +34,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint8_t* smem_a = smem;
   uint8_t* smem_b = smem + STAGES * A_STAGE_BYTES;
-  uint8_t* staging = smem + STAGES * (A_STAGE_BYTES + B_STAGE_BYTES);   // STAGED epilogues only
-  uint64_t* bars = reinterpret_cast<uint64_t*>(staging + (Epi::STAGED ? STAGING_BYTES : 0));
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + STAGES * (A_STAGE_BYTES + B_STAGE_BYTES));
   uint64_t* full = bars;                 // [STAGES] TMA -> MMA          (even CTA's are used)
   uint64_t* empty = bars + STAGES;       // [STAGES] MMA -> TMA          (each CTA waits on its own)
   uint64_t* acc_full = bars + 2 * STAGES;      // [2] MMA -> epilogue    (each CTA waits on its own)
@@ -179,11 +178,6 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
     int acc = 0; uint32_t acc_phase = 0;
     bool ok = true;
     Epi epi;
-    StageCtx cx;
-    cx.buf = smem_u32(staging) + col_half * (STAGING_BYTES / 2);
-    cx.bar_id = 1 + col_half;
-    cx.elected = quad == 0 && lane == 0;
-    cx.map = &map_c;
     WorkList work(sched, pair, num_pairs);
     int pmb, un, n_begin, n_end, kb0, kb1, slot;
     while (ok && work.next(pmb, un, n_begin, n_end, kb0, kb1, slot)) {
@@ -210,8 +204,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
             #pragma unroll
             for (int j = 0; j < 32; ++j) va[j] = 0.f;
           }
-          if constexpr (Epi::STAGED) epi.group_begin(cx);
-          epi.template chunk<0>(ep, va, n0 + c * 32, cx);
+          epi.template chunk<0>(ep, va, n0 + c * 32);
           if (c + 1 < c_end) {
             tmem_ld_wait();
             if (c + 2 < c_end && c + 2 < c_tmem) tmem_ld32(t_addr + (c + 2) * 32, va);
@@ -219,9 +212,9 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
               #pragma unroll
               for (int j = 0; j < 32; ++j) vb[j] = 0.f;
             }
-            epi.template chunk<1>(ep, vb, n0 + (c + 1) * 32, cx);
+            epi.template chunk<1>(ep, vb, n0 + (c + 1) * 32);
           }
-          if constexpr (Epi::STAGED) epi.group_end(ep, n0 + c * 32, cx);
+          if constexpr (Epi::PANEL) epi.group_end(ep, n0 + c * 32);
         }
         fence_before_sync();
         __syncwarp();
@@ -230,7 +223,6 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
       }
       if (ok) epi.end_unit(ep, un, col_half);
     }
-    if (Epi::STAGED && cx.elected) bulk_wait_all();   // stores done before shared memory goes away
     if (threadIdx.x == 64) SAPO_STATS_FLUSH(6);
   }
 
@@ -240,6 +232,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
   cluster_sync_all();
   if (warp == 1) { fence_after_sync(); tmem_dealloc_pair(tmem_base, TMEM_COLS); }
   if (threadIdx.x == 0 && *abort_flag) raise_status(status, SAPO_ST_WAIT_TIMEOUT);
+  SAPO_CLOCK_END(sched.stats_id);
 }
 
 // ---------------------------------------------------------------------------- the wide-tile GEMM kernel
@@ -276,6 +269,7 @@ umma_gemm2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
                   const __grid_constant__ CUtensorMap map_c,   // the fp32 output, boxes of 32 columns x 128 rows
                   const Sched sched_arg, const StoreEpi::Params ep_arg, int32_t* status) {
   static_assert(A_KIND == 2 || A_KIND == 3, "panel operands only");
+  SAPO_CLOCK_BEGIN
   Sched sched = sched_arg;
   StoreEpi::Params ep = ep_arg;
   extern __shared__ uint8_t smem_raw[];
@@ -441,7 +435,6 @@ umma_gemm2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
     uint32_t acc_phase = 0;
     bool ok = true;
     StoreEpi epi;
-    StageCtx cx{};
     const uint32_t buf = smem_u32(out_staging) + j * OUT_STAGING_BYTES;
     const bool elected = quad == 0 && lane == 0;     // issues and tracks this accumulator's TMA stores
     WorkList work(sched, pair, num_pairs);
@@ -471,7 +464,7 @@ umma_gemm2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
           #pragma unroll
           for (int q = 0; q < 32; ++q) v[q] = 0.f;
         }
-        if (epi.part != nullptr) { epi.template chunk<0>(ep, v, col0, cx); return; }
+        if (epi.part != nullptr) { epi.template chunk<0>(ep, v, col0); return; }
         if (col0 >= ep.N || row0 >= ep.M) return;      // nothing of this box lies inside the output
         if (elected) bulk_wait_read_all();
         named_barrier_sync(1 + j, 128);
@@ -513,6 +506,7 @@ umma_gemm2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
   cluster_sync_all();
   if (warp == 1) { fence_after_sync(); tmem_dealloc_pair(tmem_base, TMEM_COLS); }
   if (threadIdx.x == 0 && *abort_flag) raise_status(status, SAPO_ST_WAIT_TIMEOUT);
+  SAPO_CLOCK_END(sched.stats_id);
 }
 
 }  // namespace sapo

@@ -25,7 +25,6 @@ constexpr uint32_t B_STAGE_BYTES = (BN / 2) * BK * 2;   // this CTA's half of th
 constexpr uint32_t BOX_BYTES = 128 * 128;    // one 128-row box: half the K depth of a K-major operand,
                                              // or 64 columns x full K depth of an MN-major one
 constexpr uint32_t TMEM_COLS = 512;          // two accumulators of 256 columns
-constexpr uint32_t STAGING_BYTES = 2 * 128 * 128;   // dz epilogue: one 16 KB panel tile per column half
 constexpr size_t GEMM_SMEM_BYTES = 1024 + STAGES * (A_STAGE_BYTES + B_STAGE_BYTES) + 256;
 constexpr float LOG2E = 1.4426950408889634f;
 constexpr float LN2 = 0.6931471805599453f;

@@ -125,7 +125,7 @@ static int fwd_splits(int64_t T, int32_t V, int64_t K, int sms) {
 }
 
 template <int A_KIND, bool B_MN, class Epi>
-static int launch_gemm(const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& mc, const Sched& sched,
+static int launch_gemm(const CUtensorMap& ma, const CUtensorMap& mb, const Sched& sched,
                        const typename Epi::Params& ep, int32_t* status, cudaStream_t st, int kernel_id) {
   auto kern = umma_gemm_kernel<A_KIND, B_MN, Epi>;
   // CTA pairs the device can hold at once; found, together with the kernel's shared-memory
@@ -142,7 +142,7 @@ static int launch_gemm(const CUtensorMap& ma, const CUtensorMap& mb, const CUten
   attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
   cudaLaunchConfig_t cfg = {};
   cfg.blockDim = dim3(GEMM_THREADS, 1, 1);
-  constexpr size_t smem_bytes = GEMM_SMEM_BYTES + (Epi::STAGED ? STAGING_BYTES : 0);
+  constexpr size_t smem_bytes = GEMM_SMEM_BYTES;
   cfg.dynamicSmemBytes = smem_bytes;
   cfg.stream = st;
   cfg.attrs = attr;
@@ -171,7 +171,7 @@ static int launch_gemm(const CUtensorMap& ma, const CUtensorMap& mb, const CUten
   cfg.gridDim = dim3(2 * pairs, 1, 1);
   {
     KernelScope scope(kernel_id, st);
-    if (cudaLaunchKernelEx(&cfg, kern, ma, mb, mc, sc, ep, status) != cudaSuccess) return SAPO_ERR_CUDA;
+    if (cudaLaunchKernelEx(&cfg, kern, ma, mb, sc, ep, status) != cudaSuccess) return SAPO_ERR_CUDA;
   }
   if constexpr (Epi::STREAMK) {
     // with a device-side size the number of K-split tiles is not known here: launch for the
@@ -215,6 +215,7 @@ static int launch_gemm_wide(const CUtensorMap& ma, const CUtensorMap& mb, const 
   int& max_pairs = max_pairs_of[dev];
   if (sched.num_units <= 0) return SAPO_OK;
   Sched sc = sched;
+  sc.stats_id = kernel_id - SAPO_K_BWD_DZ + 1;
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeClusterDimension;
   attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
@@ -288,11 +289,11 @@ static int launch_grad_gemms(const __nv_bfloat16* panel, int64_t panel_rows, int
     return SAPO_ERR_CUDA;
   Sched sh = make_sched(tc, H, Vp, 0, /*m_fastest=*/false);
   sh.panel_nvt = nvt;
-  int rc = launch_gemm<2, true, StoreEpi>(map_p_two, map_w_mn, map_p_two, sh, ep_h, status, st, SAPO_K_BWD_DH);
+  int rc = launch_gemm<2, true, StoreEpi>(map_p_two, map_w_mn, sh, ep_h, status, st, SAPO_K_BWD_DH);
   if (rc != SAPO_OK) return rc;
   Sched sw = make_sched(V, H, tc, 0, /*m_fastest=*/false);
   sw.panel_nvt = nvt;
-  return launch_gemm<3, true, StoreEpi>(map_p_tile, map_x_mn, map_p_tile, sw, ep_w, status, st, SAPO_K_BWD_DW);
+  return launch_gemm<3, true, StoreEpi>(map_p_tile, map_x_mn, sw, ep_w, status, st, SAPO_K_BWD_DW);
 }
 
 static int launch_split(const float* X, int64_t ld, int64_t R, int32_t H, __nv_bfloat16* out, int mode,
@@ -313,9 +314,12 @@ static bool shapes_ok(int64_t T, int32_t H, int32_t V) {
 static int64_t padded_vocab(int32_t V) { return round_up<int64_t>(V, 128); }
 
 struct FwdLayout { size_t partials, a_split, b_split, total; int n_splits; };
-static FwdLayout fwd_layout(int64_t T, int32_t H, int32_t V, int32_t dtype, int sms) {
+// max_splits > 0 caps the number of vocab splits (fewer splits: less scratch, the same results up
+// to the order in which the partial sums of a token are added)
+static FwdLayout fwd_layout(int64_t T, int32_t H, int32_t V, int32_t dtype, int sms, int max_splits = 0) {
   FwdLayout L{};
   L.n_splits = fwd_splits(T, V, dtype == SAPO_DTYPE_F32 ? 3 * (int64_t)H : (int64_t)H, sms);
+  if (max_splits > 0 && L.n_splits > max_splits) L.n_splits = max_splits;
   size_t off = 0;
   L.partials = off; off += round_up<size_t>((size_t)3 * 2 * L.n_splits * T * sizeof(float), 256);
   if (dtype == SAPO_DTYPE_F32) {
@@ -405,6 +409,28 @@ __global__ void chunk_counts_kernel(const int32_t* n_active, int64_t chunk_rows,
   }
 }
 
+// Host-side checks of the forward's arguments (everything but the scratch), in the order the
+// header documents.
+static int fwd_check_args(const void* hidden, const void* W_head, int32_t dtype, int64_t T, int32_t H, int32_t V,
+                          int64_t ld_hidden, int64_t ld_W, const int32_t* ids, const float* old_logp,
+                          const float* adv, const int32_t* cu_seqlens, int32_t S, const sapo_loss_cfg* h_cfg,
+                          const float* logp, const float* lse, const float* ratio, const float* surr,
+                          const float* gscale, const float* loss, const int32_t* status) {
+  if (!hidden || !W_head || !ids || !old_logp || !adv || !cu_seqlens || !h_cfg || !logp || !lse ||
+      !ratio || !surr || !gscale || !loss || !status || S < 1)
+    return SAPO_ERR_INVALID_ARG;
+  if (dtype != SAPO_DTYPE_BF16 && dtype != SAPO_DTYPE_F32) return SAPO_ERR_INVALID_ARG;
+  if (T < 1 || H < 1 || V < 1 || ld_hidden < H || ld_W < H) return SAPO_ERR_INVALID_ARG;
+  if (!shapes_ok(T, H, V)) return SAPO_ERR_UNSUPPORTED_SHAPE;
+  const int esz = dtype == SAPO_DTYPE_BF16 ? 2 : 4;
+  if (!aligned16(hidden) || !aligned16(W_head) || (ld_hidden * esz) % 16 || (ld_W * esz) % 16)
+    return SAPO_ERR_INVALID_ARG;
+  if (!(h_cfg->eps_low >= 0.f) || !(h_cfg->eps_high >= 0.f)) return SAPO_ERR_INVALID_ARG;
+  if ((h_cfg->loss_agg != 0 && h_cfg->loss_agg != 1) || (h_cfg->kl_beta != 0.f && !h_cfg->ref_logp))
+    return SAPO_ERR_INVALID_ARG;
+  return SAPO_OK;
+}
+
 }  // namespace sapo
 
 // =============================================================================== C ABI
@@ -444,31 +470,22 @@ extern "C" size_t sapo_workspace_bytes_min(int32_t which, int64_t T, int32_t H, 
   return L.fixed + (size_t)BM * L.bytes_per_row;
 }
 
-extern "C" int sapo_policy_loss_fwd(const void* hidden, const void* W_head, int32_t dtype,
-                                    int64_t T, int32_t H, int32_t V, int64_t ld_hidden, int64_t ld_W,
-                                    const int32_t* ids, const float* old_logp, const float* adv,
-                                    const int32_t* cu_seqlens, int32_t S, const sapo_loss_cfg* h_cfg,
-                                    float* logp, float* lse, float* ratio, float* surr, float* gscale,
-                                    float* seq_surr, float* loss,
-                                    void* workspace, size_t workspace_bytes,
-                                    int32_t* status, void* stream) {
-  using namespace sapo;
-  if (!hidden || !W_head || !ids || !old_logp || !adv || !cu_seqlens || !h_cfg || !logp || !lse ||
-      !ratio || !surr || !gscale || !loss || !workspace || !status || S < 1)
-    return SAPO_ERR_INVALID_ARG;
-  if (dtype != SAPO_DTYPE_BF16 && dtype != SAPO_DTYPE_F32) return SAPO_ERR_INVALID_ARG;
-  if (T < 1 || H < 1 || V < 1 || ld_hidden < H || ld_W < H) return SAPO_ERR_INVALID_ARG;
-  if (!shapes_ok(T, H, V)) return SAPO_ERR_UNSUPPORTED_SHAPE;
-  const int esz = dtype == SAPO_DTYPE_BF16 ? 2 : 4;
-  if (!aligned16(hidden) || !aligned16(W_head) || !aligned16(workspace) || (ld_hidden * esz) % 16 ||
-      (ld_W * esz) % 16)
-    return SAPO_ERR_INVALID_ARG;
-  if (!(h_cfg->eps_low >= 0.f) || !(h_cfg->eps_high >= 0.f)) return SAPO_ERR_INVALID_ARG;
-  if ((h_cfg->loss_agg != 0 && h_cfg->loss_agg != 1) || (h_cfg->kl_beta != 0.f && !h_cfg->ref_logp))
-    return SAPO_ERR_INVALID_ARG;
+namespace sapo {
+static int fwd_impl(const void* hidden, const void* W_head, int32_t dtype,
+                    int64_t T, int32_t H, int32_t V, int64_t ld_hidden, int64_t ld_W,
+                    const int32_t* ids, const float* old_logp, const float* adv,
+                    const int32_t* cu_seqlens, int32_t S, const sapo_loss_cfg* h_cfg,
+                    float* logp, float* lse, float* ratio, float* surr, float* gscale,
+                    float* seq_surr, float* loss,
+                    void* workspace, size_t workspace_bytes,
+                    int32_t* status, void* stream, int max_splits) {
+  int rc0 = fwd_check_args(hidden, W_head, dtype, T, H, V, ld_hidden, ld_W, ids, old_logp, adv, cu_seqlens, S,
+                           h_cfg, logp, lse, ratio, surr, gscale, loss, status);
+  if (rc0 != SAPO_OK) return rc0;
+  if (!workspace || !aligned16(workspace)) return SAPO_ERR_INVALID_ARG;
   const int sms = sm_count();
   if (sms <= 0) return SAPO_ERR_CUDA;
-  const FwdLayout L = fwd_layout(T, H, V, dtype, sms);
+  const FwdLayout L = fwd_layout(T, H, V, dtype, sms, max_splits);
   // seq_surr scratch lives behind the layout when the caller does not want it
   const size_t need = L.total + (seq_surr ? 0 : round_up<size_t>((size_t)S * sizeof(float), 256));
   if (workspace_bytes < need) return SAPO_ERR_WORKSPACE_TOO_SMALL;
@@ -494,7 +511,7 @@ extern "C" int sapo_policy_loss_fwd(const void* hidden, const void* W_head, int3
   if (!make_map(&map_a, A, K, T, lda, BM) || !make_map(&map_b, B, K, V, ldb, 128)) return SAPO_ERR_CUDA;
   const Sched sched = make_sched(T, V, K, L.n_splits, /*m_fastest=*/true);
   FwdEpi::Params ep{ids, pm, ps, pz, T, V};
-  int rc = launch_gemm<0, false, FwdEpi>(map_a, map_b, map_a, sched, ep, status, st, SAPO_K_FWD_GEMM);
+  int rc = launch_gemm<0, false, FwdEpi>(map_a, map_b, sched, ep, status, st, SAPO_K_FWD_GEMM);
   if (rc != SAPO_OK) return rc;
 
   TailArgs ta{};
@@ -505,10 +522,28 @@ extern "C" int sapo_policy_loss_fwd(const void* hidden, const void* W_head, int3
   ta.loss_agg = h_cfg->loss_agg; ta.kl_beta = h_cfg->kl_beta; ta.ref_logp = h_cfg->ref_logp;
   ta.logp = logp; ta.lse = lse; ta.ratio = ratio; ta.surr = surr; ta.gscale = gscale; ta.seq_surr = seq_out;
   ta.status = status;
-  const int tail_blocks = S < sms * 8 ? S : sms * 8;
-  { KernelScope scope(SAPO_K_LOSS_TAIL, st); loss_tail_kernel<<<tail_blocks, 256, 0, st>>>(ta); }
+  // one block per sequence; at least enough blocks to zero-fill, at a few thousand tokens each,
+  // the outputs of tokens that belong to no sequence (T may be the caller's buffer capacity)
+  int64_t tail_blocks = ceil_div<int64_t>(T, 4096);
+  if (tail_blocks < S) tail_blocks = S;
+  if (tail_blocks > (int64_t)sms * 8) tail_blocks = (int64_t)sms * 8;
+  { KernelScope scope(SAPO_K_LOSS_TAIL, st); loss_tail_kernel<<<(int)tail_blocks, 256, 0, st>>>(ta); }
   { KernelScope scope(SAPO_K_LOSS_FINAL, st); loss_final_kernel<<<1, 256, 0, st>>>(seq_out, cu_seqlens, S, T, h_cfg->loss_agg, loss); }
   return check_launch();
+}
+}  // namespace sapo
+
+extern "C" int sapo_policy_loss_fwd(const void* hidden, const void* W_head, int32_t dtype,
+                                    int64_t T, int32_t H, int32_t V, int64_t ld_hidden, int64_t ld_W,
+                                    const int32_t* ids, const float* old_logp, const float* adv,
+                                    const int32_t* cu_seqlens, int32_t S, const sapo_loss_cfg* h_cfg,
+                                    float* logp, float* lse, float* ratio, float* surr, float* gscale,
+                                    float* seq_surr, float* loss,
+                                    void* workspace, size_t workspace_bytes,
+                                    int32_t* status, void* stream) {
+  return sapo::fwd_impl(hidden, W_head, dtype, T, H, V, ld_hidden, ld_W, ids, old_logp, adv, cu_seqlens, S, h_cfg,
+                        logp, lse, ratio, surr, gscale, seq_surr, loss, workspace, workspace_bytes, status, stream,
+                        /*max_splits=*/0);
 }
 
 // ------------------------------------------------------------------------------------------
@@ -548,22 +583,30 @@ extern "C" int sapo_policy_loss_fwd_static(const void* hidden, const void* W_hea
                                            float* ratio, float* surr, float* gscale, float* seq_surr,
                                            float* loss, int32_t* status, void* stream) {
   using namespace sapo;
+  // the same checks, in the same order, as the regular forward; then what only this entry limits
+  const int rc0 = fwd_check_args(hidden, W_head, dtype, T, H, V, ld_hidden, ld_W, ids, old_logp, adv, cu_seqlens,
+                                 S, h_cfg, logp, lse, ratio, surr, gscale, loss, status);
+  if (rc0 != SAPO_OK) return rc0;
   // fp32 operands would need bf16 copies of hidden and W_head in the scratch: far beyond it
   if (dtype != SAPO_DTYPE_BF16) return SAPO_ERR_UNSUPPORTED_SHAPE;
-  if (T < 1 || S < 1 || !shapes_ok(T, H, V)) return SAPO_ERR_INVALID_ARG;
   int sms = sm_count();
   if (sms <= 0) return SAPO_ERR_CUDA;
-  const size_t need = fwd_layout(T, H, V, dtype, sms).total +
-                      (seq_surr ? 0 : round_up<size_t>((size_t)S * sizeof(float), 256));
-  if (need > (size_t)SAPO_STATIC_SCRATCH_BYTES) return SAPO_ERR_STATIC_SCRATCH_EXCEEDED;
+  // The forward likes one set of partials per vocab split (24 bytes per token and split); take
+  // as many of the splits it would choose as the array holds, at least one.
+  const size_t seq_bytes = seq_surr ? 0 : round_up<size_t>((size_t)S * sizeof(float), 256);
+  if (seq_bytes >= (size_t)SAPO_STATIC_SCRATCH_BYTES) return SAPO_ERR_STATIC_SCRATCH_EXCEEDED;
+  const size_t avail = (size_t)SAPO_STATIC_SCRATCH_BYTES - seq_bytes;
+  int max_splits = (int)(avail / ((size_t)24 * (size_t)T) > 4096 ? 4096 : avail / ((size_t)24 * (size_t)T));
+  while (max_splits >= 1 && fwd_layout(T, H, V, dtype, sms, max_splits).total > avail) --max_splits;
+  if (max_splits < 1) return SAPO_ERR_STATIC_SCRATCH_EXCEEDED;
   void* scratch = nullptr;
   const int rc = static_scratch(&scratch);
   if (rc != SAPO_OK) return rc;
   // Nothing in the scratch has to start at zero: the vocab-split partials and the per-sequence
   // sums are written for every token / sequence of this call before anything reads them.
-  return sapo_policy_loss_fwd(hidden, W_head, dtype, T, H, V, ld_hidden, ld_W, ids, old_logp, adv,
-                              cu_seqlens, S, h_cfg, logp, lse, ratio, surr, gscale, seq_surr, loss,
-                              scratch, (size_t)SAPO_STATIC_SCRATCH_BYTES, status, stream);
+  return fwd_impl(hidden, W_head, dtype, T, H, V, ld_hidden, ld_W, ids, old_logp, adv,
+                  cu_seqlens, S, h_cfg, logp, lse, ratio, surr, gscale, seq_surr, loss,
+                  scratch, (size_t)SAPO_STATIC_SCRATCH_BYTES, status, stream, max_splits);
 }
 
 extern "C" int sapo_policy_loss_bwd(const void* hidden, const void* W_head, int32_t dtype,
@@ -616,15 +659,14 @@ extern "C" int sapo_policy_loss_bwd(const void* hidden, const void* W_head, int3
     const int64_t tc = (T - t0) < chunk_rows ? (T - t0) : chunk_rows;
     const __nv_bfloat16* A0 = A + t0 * lda;
     const int64_t panel_rows = ceil_div<int64_t>(tc, BM) * nvt * BM;   // 128-byte rows of the tiled panel
-    CUtensorMap map_h_kmajor, map_p_tile;
-    if (!make_map(&map_h_kmajor, A0, H, tc, lda, BM) || !make_map(&map_p_tile, panel, 64, panel_rows, 64, BM))
-      return SAPO_ERR_CUDA;
+    CUtensorMap map_h_kmajor;
+    if (!make_map(&map_h_kmajor, A0, H, tc, lda, BM)) return SAPO_ERR_CUDA;
     // dz panel: recompute logits tile by tile
     {
       Sched sched = make_sched(tc, V, H, 0, /*m_fastest=*/true, /*tile_align=*/64);
       sched.n_cover = (int32_t)Vp;
-      DzEpi::Params ep{ids + t0, lse + t0, gscale + t0, tc, V, nvt};
-      int rc = launch_gemm<0, false, DzEpi>(map_h_kmajor, map_w_kmajor, map_p_tile, sched, ep, status, st, SAPO_K_BWD_DZ);
+      DzEpi::Params ep{ids + t0, lse + t0, gscale + t0, tc, V, nvt, panel};
+      int rc = launch_gemm<0, false, DzEpi>(map_h_kmajor, map_w_kmajor, sched, ep, status, st, SAPO_K_BWD_DZ);
       if (rc != SAPO_OK) return rc;
     }
     // dhidden[t0:t0+tc] = dz . W         (M = tokens, N = H, K = V)
@@ -741,8 +783,8 @@ extern "C" int sapo_policy_loss_bwd_active(const void* hidden, const void* W_hea
       Sched sched = make_sched(tc, V, H, 0, /*m_fastest=*/true, /*tile_align=*/64);
       sched.n_cover = (int32_t)Vp;
       sched.dyn_count = count; sched.dyn_dim = 1;
-      DzEpi::Params ep{ids_act + t0, lse_act + t0, g_act + t0, tc, V, nvt};
-      int rc = launch_gemm<0, false, DzEpi>(map_h_kmajor, map_w_kmajor, map_p_tile, sched, ep, status, st, SAPO_K_BWD_DZ);
+      DzEpi::Params ep{ids_act + t0, lse_act + t0, g_act + t0, tc, V, nvt, panel};
+      int rc = launch_gemm<0, false, DzEpi>(map_h_kmajor, map_w_kmajor, sched, ep, status, st, SAPO_K_BWD_DZ);
       if (rc != SAPO_OK) return rc;
     }
     {
@@ -750,7 +792,7 @@ extern "C" int sapo_policy_loss_bwd_active(const void* hidden, const void* W_hea
       sched.panel_nvt = nvt;
       sched.dyn_count = count; sched.dyn_dim = 1;
       StoreEpi::Params ep{dhidden, H, tc, H, 0, partials, act_idx + t0, nullptr};   // rows go back to their tokens
-      int rc = launch_gemm<2, true, StoreEpi>(map_p_two, map_w_mn, map_p_two, sched, ep, status, st, SAPO_K_BWD_DH);
+      int rc = launch_gemm<2, true, StoreEpi>(map_p_two, map_w_mn, sched, ep, status, st, SAPO_K_BWD_DH);
       if (rc != SAPO_OK) return rc;
     }
     {
@@ -759,7 +801,7 @@ extern "C" int sapo_policy_loss_bwd_active(const void* hidden, const void* W_hea
       sched.panel_nvt = nvt;
       sched.dyn_count = count; sched.dyn_dim = 2; sched.skip_if_empty = acc;
       StoreEpi::Params ep{dW_head, H, V, H, acc, partials, nullptr, nullptr};
-      int rc = launch_gemm<3, true, StoreEpi>(map_p_tile, map_h_mn, map_p_tile, sched, ep, status, st, SAPO_K_BWD_DW);
+      int rc = launch_gemm<3, true, StoreEpi>(map_p_tile, map_h_mn, sched, ep, status, st, SAPO_K_BWD_DW);
       if (rc != SAPO_OK) return rc;
     }
   }
@@ -833,17 +875,16 @@ extern "C" int sapo_policy_loss_fwd_bwd(const void* hidden, const void* W_head, 
     const int64_t tc = (T - t0) < chunk_rows ? (T - t0) : chunk_rows;
     const __nv_bfloat16* A0 = A + t0 * ld_hidden;
     const int64_t panel_rows = ceil_div<int64_t>(tc, BM) * nvt * BM;
-    CUtensorMap map_h_kmajor, map_p_tile;
-    if (!make_map(&map_h_kmajor, A0, H, tc, ld_hidden, BM) || !make_map(&map_p_tile, panel, 64, panel_rows, 64, BM))
-      return SAPO_ERR_CUDA;
+    CUtensorMap map_h_kmajor;
+    if (!make_map(&map_h_kmajor, A0, H, tc, ld_hidden, BM)) return SAPO_ERR_CUDA;
     // 2. exponentials of the chunk -> panel, their sums per token and vocab split
     int n_splits = fwd_splits(tc, V, H, sms);
     if (n_splits > FUSED_MAX_SPLITS) n_splits = FUSED_MAX_SPLITS;
     Sched fs = make_sched(tc, V, H, n_splits, /*m_fastest=*/true, /*tile_align=*/64);
     fs.n_cover = (int32_t)Vp;
     {
-      ExpEpi::Params ep{c2 + t0, ps, tc, V, nvt};
-      int rc = launch_gemm<0, false, ExpEpi>(map_h_kmajor, map_w_kmajor, map_p_tile, fs, ep, status, st, SAPO_K_FWD_EXP);
+      ExpEpi::Params ep{c2 + t0, ps, tc, V, nvt, panel};
+      int rc = launch_gemm<0, false, ExpEpi>(map_h_kmajor, map_w_kmajor, fs, ep, status, st, SAPO_K_FWD_EXP);
       if (rc != SAPO_OK) return rc;
     }
     // 3. per-token loss terms, row scales, the chosen-token entries of the panel, scaled hidden rows
@@ -875,7 +916,7 @@ extern "C" int sapo_policy_loss_fwd_bwd(const void* hidden, const void* W_head, 
   }
   // 6. per-sequence means and the loss
   const int seq_blocks = S < sms * 8 ? S : sms * 8;
-  { KernelScope scope(SAPO_K_LOSS_TAIL, st); seq_mean_kernel<<<seq_blocks, 256, 0, st>>>(obj, cu_seqlens, S, seq_out); }
+  { KernelScope scope(SAPO_K_LOSS_TAIL, st); seq_mean_kernel<<<seq_blocks, 256, 0, st>>>(obj, cu_seqlens, S, T, seq_out, status); }
   { KernelScope scope(SAPO_K_LOSS_FINAL, st); loss_final_kernel<<<1, 256, 0, st>>>(seq_out, cu_seqlens, S, T, h_cfg->loss_agg, loss); }
   return check_launch();
 }
@@ -884,12 +925,14 @@ extern "C" int sapo_policy_loss_fwd_bwd(const void* hidden, const void* W_head, 
 // Rows: forward, dz, dH, dW.  Columns: [0] TMA waits on free stages, [1] MMA waits on filled
 // stages, [2] MMA waits on a free accumulator, [3] one epilogue thread's waits on a full
 // accumulator, [4..6] total cycles of the TMA / MMA / that epilogue thread, summed over CTAs
-// and launches since the last reset; [7] the longest MMA-thread time of any CTA.
+// and launches since the last reset; [7] the longest MMA-thread time of any CTA; [8] SM cycles and
+// [9] nanoseconds that CTA 0 of each launch was alive, [10] the number of launches: [8] / [9] is the
+// SM clock (GHz) the kernel actually ran at.  12 columns per row.
 extern "C" int sapo_debug_wait_stats(unsigned long long* h_out, int32_t reset) {
-  if (h_out && cudaMemcpyFromSymbol(h_out, sapo::g_wait_stats, sizeof(unsigned long long) * 32) != cudaSuccess)
+  if (h_out && cudaMemcpyFromSymbol(h_out, sapo::g_wait_stats, sizeof(unsigned long long) * 48) != cudaSuccess)
     return SAPO_ERR_CUDA;
   if (reset) {
-    unsigned long long z[32] = {0};
+    unsigned long long z[48] = {0};
     if (cudaMemcpyToSymbol(sapo::g_wait_stats, z, sizeof(z)) != cudaSuccess) return SAPO_ERR_CUDA;
   }
   return SAPO_OK;

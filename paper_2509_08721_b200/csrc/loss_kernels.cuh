@@ -51,15 +51,44 @@ __device__ __forceinline__ double block_sum_256(double x, double* sh) {
   return t;   // valid in thread 0
 }
 
-// One block per sequence: merge the vocab-split partials, then the clipped surrogate.
+// Token range of sequence s as the kernels may use it: cu_seqlens must be a non-decreasing
+// sequence inside [0, T].  An entry outside that range, or below its predecessor, is clamped and
+// reported (SAPO_ST_BAD_INDEX), so that no kernel indexes a per-token array out of bounds.
+__device__ __forceinline__ void seq_range(const int32_t* cu, int32_t s, int64_t T, int32_t& t0, int32_t& t1,
+                                          int32_t* status) {
+  const int32_t c0 = cu[s], c1 = cu[s + 1];
+  const int32_t Tc = (int32_t)T;
+  t0 = c0 < 0 ? 0 : (c0 > Tc ? Tc : c0);
+  t1 = c1 < 0 ? 0 : (c1 > Tc ? Tc : c1);
+  if (t1 < t0) t1 = t0;
+  if ((t0 != c0 || t1 != c1) && threadIdx.x == 0) raise_status(status, SAPO_ST_BAD_INDEX);
+}
+// first and one-past-last token that belongs to a sequence, clamped the same way
+__device__ __forceinline__ void scored_range(const int32_t* cu, int32_t S, int64_t T, int32_t& lo, int32_t& hi) {
+  const int32_t Tc = (int32_t)T;
+  const int32_t c0 = cu[0], c1 = cu[S];
+  lo = c0 < 0 ? 0 : (c0 > Tc ? Tc : c0);
+  hi = c1 < 0 ? 0 : (c1 > Tc ? Tc : c1);
+  if (hi < lo) hi = lo;
+}
+
+// One block per sequence: merge the vocab-split partials, then the clipped surrogate.  Blocks
+// past the last sequence only help with the tokens of [0, T) that belong to no sequence (a
+// caller that passes its buffer capacity as T): those are scored as masked, all outputs zero.
 __global__ void __launch_bounds__(256) loss_tail_kernel(TailArgs a) {
   __shared__ double sh[8];
+  int32_t lo, hi;                      // the tokens that belong to some sequence
+  scored_range(a.cu, a.S, a.T, lo, hi);
+  const float n_scored = (float)(hi - lo);
   for (int32_t s = blockIdx.x; s < a.S; s += gridDim.x) {
-    const int32_t t0 = a.cu[s], t1 = a.cu[s + 1];
+    int32_t t0, t1;
+    seq_range(a.cu, s, a.T, t0, t1, a.status);
     const int32_t Ts = t1 - t0;
     const float A = a.adv[s];
+    const bool bad_adv = !isfinite(A);
+    if (bad_adv && Ts > 0 && threadIdx.x == 0) raise_status(a.status, SAPO_ST_NONFINITE_INPUT);
     // weight of a token of this sequence: 1/(S T_s) (mean of token means) or 1/T (token mean)
-    const float w = Ts <= 0 ? 0.f : (a.loss_agg == 0 ? 1.f / ((float)a.S * (float)Ts) : 1.f / (float)a.T);
+    const float w = Ts <= 0 ? 0.f : (a.loss_agg == 0 ? 1.f / ((float)a.S * (float)Ts) : 1.f / n_scored);
     double acc = 0.0;
     for (int32_t t = t0 + threadIdx.x; t < t1; t += 256) {
       float M = -INFINITY;
@@ -72,10 +101,14 @@ __global__ void __launch_bounds__(256) loss_tail_kernel(TailArgs a) {
       }
       const float lse = (M + log2f(sum)) * LN2;
       const int32_t y = a.ids[t];
-      const bool bad = y < 0 || y >= a.V;
-      if (bad) raise_status(a.status, SAPO_ST_BAD_TOKEN_ID);
-      const float lp = bad ? 0.f : zy - lse;
-      const float rho = bad ? 0.f : expf(lp - a.old_logp[t]);
+      const bool bad_id = y < 0 || y >= a.V;
+      if (bad_id) raise_status(a.status, SAPO_ST_BAD_TOKEN_ID);
+      const float old = a.old_logp[t];
+      const bool bad_in = !isfinite(old);
+      if (bad_in) raise_status(a.status, SAPO_ST_NONFINITE_INPUT);
+      const bool bad = bad_id || bad_in || bad_adv;
+      const float lp = bad_id ? 0.f : zy - lse;
+      const float rho = bad ? 0.f : expf(lp - old);
       const float un = rho * A;
       const float cl = fminf(fmaxf(rho, a.lo_edge), a.hi_edge) * A;
       const float u = bad ? 0.f : fminf(un, cl);
@@ -94,6 +127,12 @@ __global__ void __launch_bounds__(256) loss_tail_kernel(TailArgs a) {
     const double tot = block_sum_256(acc, sh);
     if (threadIdx.x == 0) a.seq_surr[s] = Ts > 0 ? (float)(tot / (double)Ts) : 0.f;
   }
+  // tokens before the first or after the last sequence
+  const int64_t n_out = (int64_t)lo + (a.T - hi);
+  for (int64_t i = (int64_t)blockIdx.x * 256 + threadIdx.x; i < n_out; i += (int64_t)gridDim.x * 256) {
+    const int64_t t = i < lo ? i : hi + (i - lo);
+    a.lse[t] = 0.f; a.logp[t] = 0.f; a.ratio[t] = 0.f; a.surr[t] = 0.f; a.gscale[t] = 0.f;
+  }
 }
 
 // loss = -(1/S) sum_s seq_surr[s], or with token-level aggregation -(1/T) sum_s T_s seq_surr[s]
@@ -101,10 +140,16 @@ __global__ void __launch_bounds__(256)
 loss_final_kernel(const float* seq_surr, const int32_t* cu, int32_t S, int64_t T, int32_t loss_agg, float* loss) {
   __shared__ double sh[8];
   double acc = 0.0;
-  for (int32_t s = threadIdx.x; s < S; s += 256)
-    acc += loss_agg == 0 ? (double)seq_surr[s] : (double)seq_surr[s] * (double)(cu[s + 1] - cu[s]);
+  for (int32_t s = threadIdx.x; s < S; s += 256) {
+    if (loss_agg == 0) { acc += (double)seq_surr[s]; continue; }
+    int32_t t0, t1;
+    seq_range(cu, s, T, t0, t1, nullptr);
+    acc += (double)seq_surr[s] * (double)(t1 - t0);
+  }
   const double tot = block_sum_256(acc, sh);
-  const double n = loss_agg == 0 ? (double)S : (double)T;
+  int32_t lo, hi;
+  scored_range(cu, S, T, lo, hi);
+  const double n = loss_agg == 0 ? (double)S : (double)(hi - lo);
   if (threadIdx.x == 0) *loss = n > 0 ? (float)(-tot / n) : 0.f;
 }
 
@@ -143,8 +188,10 @@ target_logit_kernel(const __nv_bfloat16* __restrict__ hidden, int64_t ldh, const
     }
     if (lane == 0) {
       const bool ok = y >= 0 && y < V;
+      const float old = old_logp[t];
       zy[t] = ok ? acc : 0.f;
-      c2[t] = ok ? (acc - old_logp[t]) * LOG2E : 0.f;
+      // a non-finite old log-prob (the tail reports it and masks the token) must not reach the panel
+      c2[t] = ok ? (isfinite(old) ? acc - old : acc) * LOG2E : 0.f;
     }
   }
 }
@@ -173,6 +220,9 @@ __global__ void __launch_bounds__(256) fused_tail_kernel(FusedTailArgs a) {
   const int lane = threadIdx.x & 31;
   const int64_t warp = (int64_t)blockIdx.x * 8 + (threadIdx.x >> 5);
   const int64_t n_warps = (int64_t)gridDim.x * 8;
+  int32_t first_scored, end_scored;
+  scored_range(a.cu, a.S, a.T, first_scored, end_scored);
+  const float n_scored = (float)(end_scored - first_scored);
   for (int64_t lr = warp; lr < a.tc; lr += n_warps) {
     const int64_t t = a.t0 + lr;
     float part = 0.f;
@@ -180,21 +230,27 @@ __global__ void __launch_bounds__(256) fused_tail_kernel(FusedTailArgs a) {
     #pragma unroll
     for (int d = 16; d > 0; d >>= 1) part += __shfl_xor_sync(0xffffffffu, part, d);
     const float sum = part;
-    // the sequence of this token: last s with cu[s] <= t
+    // the sequence of this token: last s with cu[s] <= t; a token before the first or after the
+    // last sequence (the caller passed its buffer capacity as T) is scored as masked
     int lo = 0, hi = a.S - 1;
     while (lo < hi) { const int mid = (lo + hi + 1) >> 1; if ((int64_t)a.cu[mid] <= t) lo = mid; else hi = mid - 1; }
-    const int32_t Ts = a.cu[lo + 1] - a.cu[lo];
+    int32_t s0, s1;
+    seq_range(a.cu, lo, a.T, s0, s1, nullptr);       // seq_mean_kernel reports a bad cu_seqlens
+    const bool in_seq = t >= s0 && t < s1;
+    const int32_t Ts = s1 - s0;
     const float A = a.adv[lo];
-    const float w = Ts <= 0 ? 0.f : (a.loss_agg == 0 ? 1.f / ((float)a.S * (float)Ts) : 1.f / (float)a.T);
+    const float w = Ts <= 0 ? 0.f : (a.loss_agg == 0 ? 1.f / ((float)a.S * (float)Ts) : 1.f / n_scored);
     const int32_t y = a.ids[t];
-    const bool bad_id = y < 0 || y >= a.V;
+    const bool bad_id = in_seq && (y < 0 || y >= a.V);
     // a sum of exponentials that left the safe range (or is not a number): the reference was too far off
     const bool bad_range = !(sum < EXP_CAP) || !(sum > 1.f / EXP_CAP);
-    const bool bad = bad_id || bad_range;
+    const float old = a.old_logp[t];
+    const bool bad_in = in_seq && (!isfinite(old) || !isfinite(A));
+    const bool bad = !in_seq || bad_id || bad_range || bad_in;
     const float c2 = a.c2[t], zy = a.zy[t];
-    const float lse = bad_range ? 0.f : (c2 + log2f(sum)) * LN2;
-    const float lp = bad ? 0.f : zy - lse;
-    const float rho = bad ? 0.f : expf(lp - a.old_logp[t]);
+    const float lse = (bad_range || !in_seq) ? 0.f : (c2 + log2f(sum)) * LN2;
+    const float lp = (bad_id || bad_range || !in_seq) ? 0.f : zy - lse;
+    const float rho = bad ? 0.f : expf(lp - old);
     const float un = rho * A;
     const float cl = fminf(fmaxf(rho, a.lo_edge), a.hi_edge) * A;
     const float u = bad ? 0.f : fminf(un, cl);
@@ -209,12 +265,13 @@ __global__ void __launch_bounds__(256) fused_tail_kernel(FusedTailArgs a) {
     const float scale = (bad || g == 0.f) ? 0.f : -g / sum;
     if (lane == 0) {
       if (bad_id) raise_status(a.status, SAPO_ST_BAD_TOKEN_ID);
-      if (bad_range) raise_status(a.status, SAPO_ST_EXP_RANGE);
+      if (bad_range && in_seq) raise_status(a.status, SAPO_ST_EXP_RANGE);
+      if (bad_in) raise_status(a.status, SAPO_ST_NONFINITE_INPUT);
       a.lse[t] = lse; a.logp[t] = lp; a.ratio[t] = rho; a.surr[t] = u; a.gscale[t] = g; a.obj[t] = obj;
       a.row_scale[lr] = scale;
       if (scale != 0.f && a.active_mask != nullptr)
         atomicOr(&a.active_mask[lr >> 12], 1u << ((lr >> 7) & 31));
-      if (!bad) {
+      if (!bad_id && !bad_range && in_seq) {
         const float ey = ex2(fmaf(zy, LOG2E, -c2));
         const int64_t tile = (lr >> 7) * a.nvt + (y >> 6);
         a.panel[(tile * BM + (lr & 127)) * 64 + (y & 63)] = __float2bfloat16_rn(ey - sum);
@@ -237,6 +294,7 @@ __global__ void __launch_bounds__(256) fused_tail_kernel(FusedTailArgs a) {
         const float2 f = __bfloat1622float2(px[j]);
         px[j] = __floats2bfloat162_rn(scale * f.x, scale * f.y);
       }
+      if (scale == 0.f) x = make_uint4(0u, 0u, 0u, 0u);    // also when the hidden row is not finite
       dst[i] = x;
     }
   }
@@ -244,10 +302,12 @@ __global__ void __launch_bounds__(256) fused_tail_kernel(FusedTailArgs a) {
 
 // seq_surr[s] = mean over the tokens of s of obj[t] (same summation order as loss_tail_kernel)
 __global__ void __launch_bounds__(256)
-seq_mean_kernel(const float* __restrict__ obj, const int32_t* __restrict__ cu, int32_t S, float* seq_surr) {
+seq_mean_kernel(const float* __restrict__ obj, const int32_t* __restrict__ cu, int32_t S, int64_t T,
+                float* seq_surr, int32_t* status) {
   __shared__ double sh[8];
   for (int32_t s = blockIdx.x; s < S; s += gridDim.x) {
-    const int32_t t0 = cu[s], t1 = cu[s + 1];
+    int32_t t0, t1;
+    seq_range(cu, s, T, t0, t1, status);
     double acc = 0.0;
     for (int32_t t = t0 + threadIdx.x; t < t1; t += 256) acc += (double)obj[t];
     const double tot = block_sum_256(acc, sh);

@@ -157,12 +157,26 @@ __global__ void __launch_bounds__(256) pack_copy_kernel(PackArgs a) {
         a.tok_mask[t] = 1;
       }
     };
+    // a slot past the last packed token: mask 0 and an all-zero row, id and log-prob, so that the
+    // whole capacity can be scored without reading the token count back to the host
+    auto pad = [&](int64_t t) {
+      uint8_t* to = a.o_hid + t * a.row_bytes;
+      if (vec) {
+        uint4* t4 = reinterpret_cast<uint4*>(to);
+        for (int j = lane; j < n4; j += 32) t4[j] = make_uint4(0u, 0u, 0u, 0u);
+      } else {
+        uint16_t* t2 = reinterpret_cast<uint16_t*>(to);
+        for (int j = lane; j < (int)(a.row_bytes >> 1); j += 32) t2[j] = 0;
+      }
+      if (lane == 0) { a.o_ids[t] = 0; a.o_old[t] = 0.f; a.tok_seq[t] = -1; a.tok_mask[t] = 0; }
+    };
     for (int i = 0; i < tpw; i += 2) {
       const int64_t ta = t0 + i, tb = ta + 1;
       if (ta >= a.max_tokens) break;
       const bool have_a = ta < T, have_b = tb < T && tb < a.max_tokens;
       if (!have_a) {
-        if (lane == 0) { a.tok_mask[ta] = 0; if (tb < a.max_tokens) a.tok_mask[tb] = 0; }
+        pad(ta);
+        if (tb < a.max_tokens) pad(tb);
         continue;
       }
       if (two_at_once) {
@@ -187,8 +201,8 @@ __global__ void __launch_bounds__(256) pack_copy_kernel(PackArgs a) {
           #pragma unroll
           for (int q = 0; q < ROW_VECS_PER_LANE; ++q) if (lane + 32 * q < n4) ob[lane + 32 * q] = vb[q];
           finish(tb, sb);
-        } else if (tb < a.max_tokens && lane == 0) {
-          a.tok_mask[tb] = 0;
+        } else if (tb < a.max_tokens) {
+          pad(tb);
         }
         continue;
       }
@@ -196,7 +210,7 @@ __global__ void __launch_bounds__(256) pack_copy_kernel(PackArgs a) {
       for (int k = 0; k < 2; ++k) {
         const int64_t t = ta + k;
         if (t >= a.max_tokens) break;
-        if (t >= T) { if (lane == 0) a.tok_mask[t] = 0; continue; }
+        if (t >= T) { pad(t); continue; }
         const int64_t src = locate(t);
         const uint8_t* from = a.hid[side] + src * a.row_bytes;
         uint8_t* to = a.o_hid + t * a.row_bytes;
@@ -240,6 +254,19 @@ extern "C" int sapo_pack_rollouts(const sapo_rollout_buf* h_local, const sapo_ro
   if (!h_sel->q_offsets_local || !h_sel->q_offsets_ext || !h_out->cu_seqlens ||
       !h_out->n_tokens || !h_out->n_seqs || !h_out->group_offsets)
     return SAPO_ERR_INVALID_ARG;
+  // every array a kernel will touch must be there: a NULL would only show as a device fault
+  if (h_out->max_seqs > 0 && (!h_out->rewards || !h_out->seq_group || !h_out->seq_is_ext || !h_out->seq_src))
+    return SAPO_ERR_INVALID_ARG;
+  if (h_out->max_tokens > 0 && (!h_out->hidden || !h_out->ids || !h_out->old_logp || !h_out->tok_seq ||
+                                !h_out->tok_mask))
+    return SAPO_ERR_INVALID_ARG;
+  // (the index lists may be NULL: a side nobody picks from has an empty list, and only the
+  // device knows the list lengths; the scan never reads an empty list)
+  const sapo_rollout_buf* src_bufs[2] = {h_local, h_ext};
+  for (int i = 0; i < 2; ++i)
+    if (src_bufs[i]->n_rollouts > 0 && (!src_bufs[i]->hidden || !src_bufs[i]->ids || !src_bufs[i]->old_logp ||
+                                        !src_bufs[i]->offsets || !src_bufs[i]->rewards))
+      return SAPO_ERR_INVALID_ARG;
   PackArgs a{};
   a.qol = h_sel->q_offsets_local; a.local_idx = h_sel->local_idx;
   a.qoe = h_sel->q_offsets_ext;   a.ext_idx = h_sel->ext_idx; a.Q = h_sel->Q;

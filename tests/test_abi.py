@@ -66,3 +66,33 @@ def test_header_is_plain_c(tmp_path):
     lib = B.load()
     for code in range(0, -6, -1):
         assert lib.sapo_status_string(code) != b"unknown code"
+
+
+def test_pack_rejects_null_arrays_on_the_host():
+    """A NULL array the sizes say will be touched is an argument error, found before any launch
+    (so this needs no GPU): it must not become a fault on the device."""
+    import ctypes as C
+    lib = B.load()
+    x = 0x1000                                  # any non-NULL value: nothing dereferences it on the host
+    def bufs(**kw):
+        full = dict(hidden=x, ids=x, old_logp=x, offsets=x, rewards=x, n_rollouts=4)
+        full.update(kw)
+        return B.RolloutBufC(*[full[k] for k in ("hidden", "ids", "old_logp", "offsets", "rewards", "n_rollouts")])
+    sel = B.SelectionC(x, x, x, x, 2)
+    def packed(**kw):
+        names = ("hidden", "ids", "old_logp", "rewards", "cu_seqlens", "seq_group", "seq_is_ext", "seq_src",
+                 "tok_seq", "tok_mask", "group_offsets", "n_tokens", "n_seqs")
+        full = {k: x for k in names}
+        full.update(kw)
+        return B.PackedC(*[full[k] for k in names], 128, 8)
+    def call(local, ext, out, selection=sel):
+        return lib.sapo_pack_rollouts(C.byref(local), C.byref(ext), C.byref(selection), 64, B.DTYPE_BF16,
+                                      C.byref(out), x, None)
+    for member in ("hidden", "ids", "old_logp", "offsets", "rewards"):
+        assert call(bufs(**{member: None}), bufs(), packed()) == -1, member
+        assert call(bufs(), bufs(**{member: None}), packed()) == -1, member
+    for member in ("hidden", "ids", "old_logp", "rewards", "cu_seqlens", "seq_group", "seq_is_ext", "seq_src",
+                   "tok_seq", "tok_mask", "group_offsets", "n_tokens", "n_seqs"):
+        assert call(bufs(), bufs(), packed(**{member: None})) == -1, member
+    assert call(bufs(), bufs(), packed(), B.SelectionC(None, x, x, x, 2)) == -1
+    assert call(bufs(), bufs(), packed(), B.SelectionC(x, x, None, x, 2)) == -1

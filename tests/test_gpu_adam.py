@@ -34,7 +34,8 @@ def test_adam_steps_match_the_oracle(rows, cols):
         assert np.max(np.abs(v.cpu().numpy() - vo)) <= 1e-6 * np.abs(vo).max()
         bits = w16.view(torch.int16).cpu().numpy().view(np.uint16)
         assert np.array_equal(bits, gen.f32_to_bf16_bits(master.cpu().numpy()))
-    assert np.array_equal(master.cpu().numpy()[0, :8] , theta0[0, :8]) is False or True
+        if step == 1:        # zero gradient and zero moments: the weight stays bit for bit
+            assert np.array_equal(master.cpu().numpy()[0, :8], theta0[0, :8])
 
 
 def test_adam_rejects_bad_arguments():
