@@ -120,9 +120,9 @@ def blas_threads():
         return os.cpu_count()
 
 
-def build_batch(workload: int, seed: int, length_div: int = 1):
+def build_batch(workload: int, seed: int, length_div: int = 1, ext_fraction=None):
     from paper_2509_08721_b200 import inputs as gen
-    recipe = gen.config(workload, length_div=length_div)
+    recipe = gen.config(workload, length_div=length_div, ext_fraction=ext_fraction)
     if length_div != 1:
         recipe.name += f"_lengths_div{length_div}"
     return gen.make_batch(recipe, seed), recipe
@@ -132,7 +132,7 @@ def run_reference(args):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return 0
-    batch, recipe = build_batch(args.workload, 1000 * args.workload, args.length_div)
+    batch, recipe = build_batch(args.workload, 1000 * args.workload, args.length_div, args.ext_fraction)
     # old log-probs: the recipe's noise around zero suffices for timing (values do not change cost)
     n_seqs, T = oracle_sample(batch, args.ref_tokens)
     for _ in range(min(args.warmup, 1)):
@@ -200,6 +200,8 @@ def hbm_kernels(torch, B, peaks, H=896, n_rollouts=2048, mean_len=288, n_groups=
 
     ms_pack = timed(lambda: B.sapo_pack_rollouts(bufs[0], bufs[1], sel, out, status))
     ms_adv = timed(lambda: B.sapo_group_advantages(rewards, go, 1e-6, 0, adv, None, None, status))
+    ms_adv_warp = timed(lambda: B.sapo_group_advantages(rewards, go, 1e-6, 0, adv, None, None, status,
+                                                         warp_level=True))
     assert int(status.item()) == 0 and int(out["n_tokens"].item()) == T
     # Adam step on an LM-head-sized weight: 16 bytes read + 14 written per element
     V_adam = 151936
@@ -215,9 +217,192 @@ def hbm_kernels(torch, B, peaks, H=896, n_rollouts=2048, mean_len=288, n_groups=
     mk = lambda ms, nbytes, what: {"achieved": nbytes / ms / 1e6, "peak": peak, "unit": "GB/s",
                                    "frac": nbytes / ms / 1e6 / peak, "ms": ms, "bytes": nbytes, "case": what}
     return {"pack": mk(ms_pack, bytes_pack, f"{T} tokens of {H} bf16 from {2 * n_rollouts} rollouts"),
-            "advantages": mk(ms_adv, bytes_adv, f"{n_groups} questions x 8 completions"),
+            "advantages": mk(ms_adv, bytes_adv, f"{n_groups} questions x 8 completions, thread-per-question kernel"),
+            "advantages_warp": mk(ms_adv_warp, bytes_adv, f"{n_groups} questions x 8 completions, warp-level kernel "
+                                                          "(8 lanes per question; the one batches below 4096 questions take)"),
             "adam": mk(ms_adam, bytes_adam, f"weight [{V_adam}, {H}] fp32 master + moments + bf16 copy"),
             "peak_source": peaks["source"] + " (copy bandwidth)"}
+
+
+# DRAM bytes per launch of the tensor-core kernels, measured with ncu on a small case of the same
+# kernels (workload 2 with lengths / 4: W_head still exceeds L2; a full-size launch holds more on
+# the device than a capture should) and extended to the bench's token count as fixed + per_token * T:
+# the traffic is the weight (or dW) once plus the panel rows.  Only for hidden 896 / vocab 151936.
+# "alg_per_token" is what the per-token part must be by the algorithm (panel row + the token's
+# hidden / output row); run_ours refuses to report a table entry that is off by more than 2 %.
+NCU_TRAFFIC_SHAPE = (896, 151936)
+NCU_TRAFFIC = {
+    # kernel: (fixed bytes, bytes per token)
+}
+
+
+def algorithmic_bytes_per_token(kernel: str, H: int, V: int) -> float:
+    vp = -(-V // 128) * 128
+    return {"fwd_gemm": 2.0 * H + 12, "fwd_exp": 2.0 * vp + 2 * H, "bwd_dz": 2.0 * vp + 2 * H,
+            "bwd_dh": 2.0 * vp + 4 * H, "bwd_dw": 2.0 * vp + 2 * H}[kernel]
+
+
+def ncu_traffic(kernel: str, H: int, V: int, tokens_per_launch: float):
+    """Per-launch DRAM traffic from the ncu table, or None when there is no valid entry."""
+    if (H, V) != NCU_TRAFFIC_SHAPE or kernel not in NCU_TRAFFIC:
+        return None
+    fixed, per_token = NCU_TRAFFIC[kernel]
+    alg = algorithmic_bytes_per_token(kernel, H, V)
+    if kernel != "fwd_gemm" and abs(per_token / alg - 1.0) > 0.02:
+        raise SystemExit(f"bench.py: the ncu traffic table for {kernel} ({per_token:.0f} B/token) no longer matches "
+                         f"the kernel's algorithmic {alg:.0f} B/token: re-capture it")
+    return fixed + per_token * tokens_per_launch
+
+
+class Measured:
+    """Device-resident and host-buffer timings of one workload."""
+
+
+def measure(torch, dist, B, gen, replicas, PolicyScorer, _to_dev, args, workload, ext_fraction, steps, warmup,
+            backward, rank, world, local_rank, breakdown=True, separate=True):
+    """Time `steps` scoring steps of one workload: device-resident (the headline, per-kernel
+    timing off), then per kernel in a short loop of its own, then from pinned host buffers, then
+    (single-pass mode) the separate forward / backward calls on the same inputs."""
+    m = Measured()
+    batch, recipe = build_batch(workload, replicas.rank_seed(workload, rank), args.length_div, ext_fraction)
+    T, S, H, V = batch.T, batch.S, batch.H, batch.V
+    W = _to_dev(batch.W, "cuda")
+    scorer = PolicyScorer(W, T, S, recipe.Q, eps_low=batch.eps_low, eps_high=batch.eps_high, backward=backward)
+
+    # old log-probs = current + noise: "current" is one forward pass of the library itself
+    # over the packed tokens (set-up, untimed); the noise comes from the seeded generator.
+    scorer.make_host_batch(batch)
+    res = scorer.step_from_host(T, S)
+    torch.cuda.synchronize()
+    gen.install_old_logp(batch, res.fwd["logp"][:T].cpu().numpy())
+    scorer.make_host_batch(batch)
+    d = scorer._dev
+    for k, t in scorer._host.items():
+        d[k].copy_(t)
+    view = lambda t: t.view(torch.bfloat16) if t.dtype == torch.int16 else t
+    local = B.DeviceRollouts(view(d["local.hidden"]), d["local.ids"], d["local.old_logp"],
+                             d["local.offsets"], d["local.rewards"])
+    ext = B.DeviceRollouts(view(d["ext.hidden"]), d["ext.ids"], d["ext.old_logp"],
+                           d["ext.offsets"], d["ext.rewards"])
+    sel = B.DeviceSelection(d["sel.q_offsets_local"], d["sel.local_idx"], d["sel.q_offsets_ext"],
+                            d["sel.ext_idx"])
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def timed(fn, n):
+        start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        start.record()
+        for _ in range(n):
+            fn()
+        stop.record()
+        barrier()
+        ms, _ = replicas.aggregate(start.elapsed_time(stop), 0.0, device="cuda")
+        return ms
+
+    def sampled(fn, n, before=None):
+        """timed(), with the clocks sampled under the same load (nvidia-smi needs a moment to
+        start: the GPU is kept busy with the same steps until it reports)."""
+        sampler = ClockSampler(local_rank) if rank == 0 else None
+        if sampler is not None:
+            t_end = time.perf_counter() + 0.5
+            while time.perf_counter() < t_end:
+                fn()
+            torch.cuda.synchronize()
+        if before is not None:
+            before()
+        ms = timed(fn, n)
+        return ms, (sampler.stop() if sampler else None)
+
+    dev_step = lambda: scorer.step(local, ext, sel, T, S)
+    host_step = lambda: scorer.step_from_host(T, S)
+
+    for _ in range(warmup):
+        dev_step()
+    torch.cuda.synchronize()
+    # 1. the headline: device-resident inputs, no per-kernel events in the stream
+    m.ms_total, m.clocks = sampled(dev_step, steps)
+    scorer.check_status()
+    # 2. the same steps with every launch bracketed by events: which kernel takes what
+    m.per_kernel, m.clocks_kernels, m.kernel_steps = None, None, 0
+    if breakdown:
+        m.kernel_steps = max(3, min(steps, 20))
+        count = {}
+
+        def start_events():
+            B.sapo_timing_enable(True)
+            count["at_start"] = B.sapo_launch_count()
+        _, m.clocks_kernels = sampled(dev_step, m.kernel_steps, before=start_events)
+        m.launches_per_step = (B.sapo_launch_count() - count["at_start"]) / m.kernel_steps
+        m.per_kernel = B.sapo_timing_read()
+        B.sapo_timing_enable(False)
+    else:
+        launches0 = B.sapo_launch_count()
+        dev_step()
+        m.launches_per_step = float(B.sapo_launch_count() - launches0)
+    scorer.check_status()
+    # 3. end to end: the rollout buffers start in pinned host memory every step
+    for _ in range(min(warmup, 3)):
+        host_step()
+    m.ms_e2e, m.clocks_e2e = sampled(host_step, steps)
+    scorer.check_status()
+    # 4. beside the single-pass call: the separate forward and backward calls (logits recomputed)
+    m.separate = None
+    if separate and backward == "fused":
+        scorer2 = PolicyScorer(W, T, S, recipe.Q, eps_low=batch.eps_low, eps_high=batch.eps_high,
+                               backward="dense")
+        sep_step = lambda: scorer2.step(local, ext, sel, T, S)
+        for _ in range(warmup):
+            sep_step()
+        n_sep = min(steps, 30)
+        ms_sep, clocks_sep = sampled(sep_step, n_sep)
+        scorer2.check_status()
+        m.separate = (ms_sep, n_sep, clocks_sep)
+        del scorer2
+        torch.cuda.empty_cache()
+
+    _, m.total_tokens = replicas.aggregate(0.0, float(T), device="cuda")
+    m.steps = steps
+    m.batch, m.recipe, m.scorer = batch, recipe, scorer
+    # tokens with a non-zero gradient factor: the algorithmic backward work (zero-advantage groups
+    # and tokens clipped on the binding side contribute nothing to either gradient);
+    # t_exec = tokens the backward contractions actually run over in this mode
+    g = scorer.fwd["gscale"][:T]
+    m.t_act = int((g != 0).sum().item())
+    if backward == "active":
+        m.t_exec = int(scorer.n_active.item())
+    elif backward == "fused" and H >= 256:
+        pad = (-T) % 128                 # whole 128-token blocks without any gradient are left out
+        gp = torch.nn.functional.pad(g, (0, pad)).view(-1, 128)
+        m.t_exec = min(T, 128 * int((gp != 0).any(dim=1).sum().item()))
+    else:
+        m.t_exec = T
+    m.workspace_bytes = int(scorer.workspace.numel())
+    return m
+
+
+def summary(m, replicas, backward, peaks):
+    """The short record of a workload for the `other_workloads` key."""
+    b, r = m.batch, m.recipe
+    T, H, V = b.T, b.H, b.V
+    ms_step = m.ms_total / m.steps
+    f_alg = 2.0 * T * V * H + 4.0 * m.t_act * V * H
+    out = {"workload": r.name, "H": H, "V": V, "tokens_per_step": T, "active_tokens": m.t_act, "steps": m.steps,
+           "backward": backward, "ms_per_step": ms_step,
+           "value": replicas.throughput(m.ms_total, m.total_tokens, m.steps), "unit": UNIT,
+           "e2e_value": replicas.throughput(m.ms_e2e, m.total_tokens, m.steps),
+           "tflops_algorithmic": f_alg / (ms_step / 1e3) / 1e12,
+           "frac_of_bf16_burst_peak_algorithmic": f_alg / (ms_step / 1e3) / 1e12 / peaks["bf16_tflops"],
+           "frac_of_bf16_sustained_peak_algorithmic": f_alg / (ms_step / 1e3) / 1e12 / peaks["bf16_tflops_sustained"],
+           "workspace_bytes": m.workspace_bytes, "clocks": m.clocks}
+    if m.separate is not None:
+        ms_sep, n_sep, _ = m.separate
+        out["separate_calls_ms_per_step"] = ms_sep / n_sep
+        out["separate_calls_tflops_algorithmic"] = f_alg / (ms_sep / n_sep / 1e3) / 1e12
+    return out
 
 
 def run_ours(args):
@@ -243,147 +428,60 @@ def run_ours(args):
             print(json.dumps({"hbm_kernels": hbm_kernels(torch, B, peaks)}))
         return 0
 
-    batch, recipe = build_batch(args.workload, replicas.rank_seed(args.workload, rank), args.length_div)
+    mods = (torch, dist, B, gen, replicas, PolicyScorer, _to_dev)
+    m = measure(*mods, args, args.workload, args.ext_fraction, args.steps, args.warmup, args.backward,
+                rank, world, local_rank)
+    batch, recipe, scorer = m.batch, m.recipe, m.scorer
     T, S, H, V = batch.T, batch.S, batch.H, batch.V
-    W = _to_dev(batch.W, "cuda")
-    scorer = PolicyScorer(W, T, S, recipe.Q, eps_low=batch.eps_low, eps_high=batch.eps_high,
-                          backward=args.backward)
-
-    # old log-probs = current + noise: "current" is one forward pass of the library itself
-    # over the packed tokens (set-up, untimed); the noise comes from the seeded generator.
-    scorer.make_host_batch(batch)
-    res = scorer.step_from_host(T, S)
-    torch.cuda.synchronize()
-    gen.install_old_logp(batch, res.fwd["logp"][:T].cpu().numpy())
-    scorer.make_host_batch(batch)
-    d = scorer._dev
-    for k, t in scorer._host.items():
-        d[k].copy_(t)
-    view = lambda t: t.view(torch.bfloat16) if t.dtype == torch.int16 else t
-    local = B.DeviceRollouts(view(d["local.hidden"]), d["local.ids"], d["local.old_logp"],
-                             d["local.offsets"], d["local.rewards"])
-    ext = B.DeviceRollouts(view(d["ext.hidden"]), d["ext.ids"], d["ext.old_logp"],
-                           d["ext.offsets"], d["ext.rewards"])
-    sel = B.DeviceSelection(d["sel.q_offsets_local"], d["sel.local_idx"], d["sel.q_offsets_ext"],
-                            d["sel.ext_idx"])
-
-    def barrier():
-        if world > 1:
-            dist.barrier()
-        torch.cuda.synchronize()
-
-    def timed(fn, steps):
-        start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        barrier()
-        start.record()
-        for _ in range(steps):
-            fn()
-        stop.record()
-        barrier()
-        ms, _ = replicas.aggregate(start.elapsed_time(stop), 0.0, device="cuda")
-        return ms
-
-    dev_step = lambda: scorer.step(local, ext, sel, T, S)
-    host_step = lambda: scorer.step_from_host(T, S)
-
-    for _ in range(args.warmup):
-        dev_step()
-    torch.cuda.synchronize()
-    sampler = ClockSampler(local_rank) if rank == 0 else None
-    if sampler is not None:
-        # nvidia-smi needs a moment to start: keep the GPU under the same load until it reports
-        t_end = time.perf_counter() + 0.5
-        while time.perf_counter() < t_end:
-            dev_step()
-        torch.cuda.synchronize()
-    B.sapo_timing_enable(True)
-    launches0 = B.sapo_launch_count()
-    ms_total = timed(dev_step, args.steps)
-    clocks = sampler.stop() if sampler else None
-    n_launches = B.sapo_launch_count() - launches0
-    per_kernel = B.sapo_timing_read()
-    B.sapo_timing_enable(False)
-    scorer.check_status()
-
-    for _ in range(min(args.warmup, 3)):
-        host_step()
-    ms_e2e = timed(host_step, args.steps)
-    scorer.check_status()
-
-    # beside the single-pass call: the same step through the separate forward and backward calls
-    # (the backward recomputes the logits), on the same device-resident inputs
-    separate = None
-    if args.backward == "fused":
-        scorer2 = PolicyScorer(W, T, S, recipe.Q, eps_low=batch.eps_low, eps_high=batch.eps_high,
-                               backward="dense")
-        sep_step = lambda: scorer2.step(local, ext, sel, T, S)
-        for _ in range(args.warmup):
-            sep_step()
-        n_sep = min(args.steps, 30)
-        ms_sep = timed(sep_step, n_sep)
-        scorer2.check_status()
-        separate = (ms_sep, n_sep)
-        del scorer2
-        torch.cuda.empty_cache()
-
-    _, total_tokens = replicas.aggregate(0.0, float(T), device="cuda")
-    ms_step = ms_total / args.steps
-    value = replicas.throughput(ms_total, total_tokens, args.steps)
-    e2e_value = replicas.throughput(ms_e2e, total_tokens, args.steps)
+    ms_step = m.ms_total / args.steps
+    value = replicas.throughput(m.ms_total, m.total_tokens, args.steps)
+    e2e_value = replicas.throughput(m.ms_e2e, m.total_tokens, args.steps)
+    h2d, d2h = scorer.h2d_bytes, scorer.d2h_bytes
 
     if rank == 0:
-        # roofline of the dominant kernel (largest share of the timed region)
-        # tokens with a non-zero gradient factor: the algorithmic backward work (zero-advantage
-        # groups and tokens clipped on the binding side contribute nothing to either gradient);
-        # t_exec = tokens the backward contractions actually run over in this mode
-        g = scorer.fwd["gscale"][:T]
-        t_act = int((g != 0).sum().item())
-        if args.backward == "active":
-            t_exec = int(scorer.n_active.item())
-        elif args.backward == "fused" and H >= 256:
-            # whole 128-token blocks without any gradient are left out
-            pad = (-T) % 128
-            gp = torch.nn.functional.pad(g, (0, pad)).view(-1, 128)
-            t_exec = min(T, 128 * int((gp != 0).any(dim=1).sum().item()))
-        else:
-            t_exec = T
+        per_kernel, ksteps = m.per_kernel, m.kernel_steps
+        t_act, t_exec = m.t_act, m.t_exec
+        # roofline of the dominant kernel (largest share of the per-kernel loop)
         gemm = {k: per_kernel[k] for k in ("fwd_gemm", "fwd_exp", "bwd_dz", "bwd_dh", "bwd_dw")
                 if per_kernel[k]["launches"]}
         top = max(gemm, key=lambda k: gemm[k]["ms"])
         n_top = max(1, gemm[top]["launches"])
         ms_top = gemm[top]["ms"] / n_top
-        # launches per step of that kernel (the backward runs once per dz panel chunk)
-        per_step = n_top / args.steps
-        flops_each = 2.0 * (T if top in ("fwd_gemm", "fwd_exp") else t_exec if top == "bwd_dz" else t_act) * V * H
-        achieved = flops_each / per_step / (ms_top / 1e3) / 1e12
-        # DRAM bytes per launch from the ncu capture of a small case of the same kernels
-        # (profiles/umma_gemm_kernels_*_workload2_lengths_div4.md): fixed part + bytes per token.
-        # Only valid for hidden 896 / vocab 151936, the shape that capture ran at.
-        ncu_traffic = {"fwd_gemm": (0.272e9, 12.4e3), "bwd_dz": (0.272e9, 299.6e3),
-                       "fwd_exp": (0.272e9, 309.5e3), "bwd_dh": (0.52e9, 310.7e3),
-                       "bwd_dw": (0.60e9, 310.7e3)}
-        if args.backward != "fused":     # the separate backward's dH / dW launches were captured earlier
-            ncu_traffic.update({"bwd_dh": (0.272e9, 310.8e3), "bwd_dw": (0.515e9, 332.3e3)})
-        traffic = None
-        if (H, V) == (896, 151936) and top in ncu_traffic:
-            fixed, per_token = ncu_traffic[top]
-            traffic = fixed + per_token * T / per_step
+        per_step = n_top / ksteps                   # launches per step (one per panel chunk)
+        flops_of = lambda k: 2.0 * (T if k in ("fwd_gemm", "fwd_exp") else t_exec if k == "bwd_dz" else t_act) * V * H
+        achieved = flops_of(top) / per_step / (ms_top / 1e3) / 1e12
+        traffic = ncu_traffic(top, H, V, T / per_step)
         peak = peaks["bf16_tflops_sustained"]      # the kernel is timed inside a long step
         burst = peaks["bf16_tflops"]
-        kernels = {k: {"ms_per_step": v["ms"] / args.steps, "launches_per_step": v["launches"] / args.steps}
-                   for k, v in per_kernel.items() if v["launches"]}
-        gemm_ms = sum(gemm[k]["ms"] for k in gemm) / args.steps
+        # per kernel: time, and time x SM clock (median under the same load): runs under different
+        # power caps compare on the second
+        mhz = (m.clocks_kernels or {}).get("sm_mhz")
+        kernels = {}
+        for k, v in per_kernel.items():
+            if not v["launches"]:
+                continue
+            kernels[k] = {"ms_per_step": v["ms"] / ksteps, "launches_per_step": v["launches"] / ksteps}
+            if k in gemm:
+                kernels[k]["tflops"] = flops_of(k) / (v["ms"] / ksteps / 1e3) / 1e12
+                if mhz:
+                    kernels[k]["ms_x_sm_mhz"] = v["ms"] / ksteps * mhz
+                    # share of the tensor pipe's cycles the contraction needs at that clock (148 SMs x 8192 flop / cycle)
+                    kernels[k]["tensor_cycles_frac_at_that_clock"] = \
+                        flops_of(k) / (148 * 8192.0) / (v["ms"] / ksteps * 1e-3 * mhz * 1e6)
+        gemm_ms = sum(gemm[k]["ms"] for k in gemm) / ksteps
         f_alg = 2.0 * T * V * H + 4.0 * t_act * V * H
         # the separate backward recomputes the logits (one more contraction); the fused call does not
         f_exec = 2.0 * T * V * H + (4.0 if args.backward == "fused" else 6.0) * t_exec * V * H
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
-            "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "vs_baseline": None, "dtype": "bf16" if batch.dtype == gen.DTYPE_BF16 else "f32 (split into bf16 pairs)",
+            "data": "synthetic",
             "config": {"workload": recipe.name, "H": H, "V": V, "questions": recipe.Q,
                        "local_per_question": recipe.I, "external_per_question": recipe.J,
                        "tokens_per_step": T, "sequences": S, "backward": args.backward,
                        "active_tokens": t_act, "backward_tokens_executed": t_exec,
+                       "workspace_bytes": m.workspace_bytes,
                        "parallelism": f"replicas x{world}",
                        "l2": "inputs larger than L2 (W_head alone is %d MB)" % (V * H * 2 // 2**20)},
             "tflops_algorithmic": f_alg / (ms_step / 1e3) / 1e12,
@@ -394,32 +492,53 @@ def run_ours(args):
             "roofline": {"bound": "tensor", "kernel": top, "achieved": achieved, "peak": peak,
                          "unit": "TFLOP/s", "frac": achieved / peak, "traffic": traffic,
                          "peak_source": peaks["source"] + " (sustained bf16 GEMM; burst is %.1f)" % burst,
-                         "flops_per_launch": flops_each / per_step, "ms_per_launch": ms_top,
+                         "flops_per_launch": flops_of(top) / per_step, "ms_per_launch": ms_top,
                          "all_gemm_kernels_ms_per_step": gemm_ms},
             "kernels": kernels,
-            "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": scorer.h2d_bytes,
-                    "d2h_bytes_per_step": scorer.d2h_bytes, "ms_per_step": ms_e2e / args.steps},
-            "gpu_launches": int(n_launches),
-            "clocks": clocks,
+            "kernels_measured": {"how": "a separate loop of %d steps with every launch bracketed by CUDA events "
+                                        "(the headline loop has none)" % ksteps,
+                                 "clocks": m.clocks_kernels},
+            "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d,
+                    "d2h_bytes_per_step": d2h, "ms_per_step": m.ms_e2e / args.steps,
+                    "returns": "loss and per-token log-probs go back to the host every step; dhidden and dW_head "
+                               "stay in device memory, where the transformer backward and the optimiser step "
+                               "read them",
+                    "clocks": m.clocks_e2e},
+            "gpu_launches": int(round(m.launches_per_step * args.steps)),
+            "clocks": m.clocks,
         }
-        if separate is not None:
-            ms_sep, n_sep = separate
+        if m.separate is not None:
+            ms_sep, n_sep, clocks_sep = m.separate
             line["separate_calls"] = {
                 "what": "sapo_policy_loss_fwd then sapo_policy_loss_bwd (logits recomputed), same inputs",
-                "value": replicas.throughput(ms_sep, total_tokens, n_sep), "unit": UNIT,
+                "value": replicas.throughput(ms_sep, m.total_tokens, n_sep), "unit": UNIT,
                 "ms_per_step": ms_sep / n_sep, "steps": n_sep,
                 "tflops_algorithmic": f_alg / (ms_sep / n_sep / 1e3) / 1e12,
-                "tflops_executed": (2.0 * T * V * H + 6.0 * T * V * H) / (ms_sep / n_sep / 1e3) / 1e12}
-        if world == 1:
-            del scorer.workspace
-            torch.cuda.empty_cache()
-            line["hbm_kernels"] = hbm_kernels(torch, B, peaks)
-        if world == 1 and not args.no_cpu_baseline:
+                "tflops_executed": (2.0 * T * V * H + 6.0 * T * V * H) / (ms_sep / n_sep / 1e3) / 1e12,
+                "frac_of_bf16_burst_peak_algorithmic": f_alg / (ms_sep / n_sep / 1e3) / 1e12 / burst,
+                "clocks": clocks_sep}
+    del scorer, m
+    torch.cuda.empty_cache()
+    if world == 1 and rank == 0:
+        line["hbm_kernels"] = hbm_kernels(torch, B, peaks)
+        torch.cuda.empty_cache()
+        if args.other_workloads and args.workload == 2 and args.length_div == 1:
+            # the other bf16 workloads, a few steps each: same measurement, short record
+            others = []
+            for w, frac in ((3, None), (4, None), (5, 0.5)):
+                mo = measure(*mods, args, w, frac, args.other_steps, 3, "fused", rank, world, local_rank,
+                             breakdown=False, separate=False)
+                others.append(summary(mo, replicas, "fused", peaks))
+                del mo
+                torch.cuda.empty_cache()
+            line["other_workloads"] = others
+        if not args.no_cpu_baseline:
             n_seqs, _ = oracle_sample(batch, args.ref_tokens)
             dt, Ts = time_oracle(batch, n_seqs)
             line["cpu_baseline"] = {
                 "value": Ts / dt, "unit": UNIT, "cores": blas_threads(), "kind": "oracle",
                 "sample": f"first {n_seqs} sequences ({Ts} tokens) of the {T}-token batch, one pass, {dt:.1f} s"}
+    if rank == 0:
         print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()
@@ -445,6 +564,12 @@ def main():
                          "for them, with the separate calls timed beside it)")
     ap.add_argument("--length-div", type=int, default=1,
                     help="divide every completion length (a small case of the same kernels for profiling)")
+    ap.add_argument("--ext-fraction", type=float, default=None,
+                    help="workload 5: external share J / (I + J) of every question, one of 0, 0.25, 0.5, 0.75")
+    ap.add_argument("--other-workloads", dest="other_workloads", action="store_true", default=True,
+                    help="after the headline (workload 2), also time workloads 3, 4 and 5 for a few steps (default)")
+    ap.add_argument("--no-other-workloads", dest="other_workloads", action="store_false")
+    ap.add_argument("--other-steps", type=int, default=4)
     args = ap.parse_args()
     if args.backward is None:
         args.backward = "dense" if args.workload == 1 else "fused"

@@ -137,7 +137,10 @@ typedef struct sapo_packed {
  * tokens (the aggregation of DAPO, which Section 4.2 cites).  kl_beta: weight of a penalty
  * towards a reference policy, per token exp(d) - d - 1 with d = ref_logp[t] - logp[t], aggregated
  * like the surrogate; 0 (the paper's choice) leaves ref_logp unused.  ref_logp: device pointer,
- * [T], may be NULL when kl_beta is 0. */
+ * [T], may be NULL when kl_beta is 0.  entropy: device pointer [T] or NULL; when given, the forward
+ * also writes the entropy of the policy's next-token distribution at every scored position,
+ * H_t = - sum_v p[t,v] log p[t,v] (nats), a by-product of the same pass over the logits that RL
+ * runs log beside the reward; it does not enter the loss.  Tokens that belong to no sequence get 0. */
 typedef struct sapo_loss_cfg {
   float eps_low;
   float eps_high;
@@ -145,6 +148,7 @@ typedef struct sapo_loss_cfg {
   int32_t loss_agg;
   float kl_beta;
   const float* ref_logp;
+  float* entropy;
 } sapo_loss_cfg;
 
 /* Section 3.2, training-set equation / Algorithm 1 "Assemble training set".
@@ -166,11 +170,19 @@ int sapo_pack_rollouts(const sapo_rollout_buf* h_local, const sapo_rollout_buf* 
 /* Section 4.2 (GRPO): for each question g with members group_offsets[g]..group_offsets[g+1):
  *   mean_g = average reward, std_g = sqrt(sum (r-mean_g)^2 / (G - ddof)),
  *   adv[s] = (rewards[s] - mean_g) / (std_g + adv_eps).
- * The group covers all its completions, local and external alike.  Accumulates in fp64,
- * stores fp32.  mean / std may be NULL.  A non-finite reward sets SAPO_ST_NONFINITE_REWARD. */
+ * The group covers all its completions, local and external alike.  fp32 in, fp32 out; the sums
+ * carry their rounding errors along (compensated fp32), so an advantage is within 6 fp32 ulp of
+ * the exactly computed value for groups of up to 16 rewards whatever their common offset, and an
+ * all-equal group gives exactly 0.  mean / std may be NULL.  A non-finite reward sets
+ * SAPO_ST_NONFINITE_REWARD.  Up to 4095 questions run on the warp-level kernel (eight lanes per
+ * question), more on a thread-per-question kernel; sapo_group_advantages_warp always takes the
+ * warp-level one (same arguments and results; it exists so that kernel can be measured alone). */
 int sapo_group_advantages(const float* rewards, const int32_t* group_offsets, int32_t Q,
                           float adv_eps, int32_t ddof, float* adv, float* mean, float* std,
                           int32_t* status, void* stream);
+int sapo_group_advantages_warp(const float* rewards, const int32_t* group_offsets, int32_t Q,
+                               float adv_eps, int32_t ddof, float* adv, float* mean, float* std,
+                               int32_t* status, void* stream);
 
 /* Section 3.2 (token-level values under the node's own policy) + Section 4.2 (clipped
  * surrogate, KL weight 0).  For T packed tokens in S sequences:
@@ -323,8 +335,9 @@ size_t sapo_workspace_bytes_min(int32_t which, int64_t T, int32_t H, int32_t V, 
  * Limits, checked after the common argument checks: bf16 operands only
  * (SAPO_ERR_UNSUPPORTED_SHAPE otherwise), and
  *     24 * T bytes  (+ 4 * S, rounded up to 256, when seq_surr is NULL)  <=  SAPO_STATIC_SCRATCH_BYTES,
- * i.e. up to 174,762 tokens; beyond that the call does nothing and returns
- * SAPO_ERR_STATIC_SCRATCH_EXCEEDED.  The forward keeps 24 bytes per token and vocab split; this
+ * i.e. up to 174,762 tokens (32 * T and 131,072 tokens when h_cfg->entropy is given); beyond that
+ * the call does nothing and returns SAPO_ERR_STATIC_SCRATCH_EXCEEDED.  The forward keeps 24 (32)
+ * bytes per token and vocab split; this
  * entry takes as many of the splits the regular call would use as fit in the array.  When all of
  * them fit the results are bit-identical to sapo_policy_loss_fwd; with fewer splits they agree up
  * to the order in which a token's partial sums are added (and large batches of few tokens per SM

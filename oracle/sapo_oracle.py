@@ -14,6 +14,7 @@ What it computes, and where the method states it:
   token_logprobs      log-prob of each chosen token under the policy's LM head
                       (Section 3.2: nodes "re-encode and compute token-level values" for
                       any rollout as if it were their own)
+  token_entropy       entropy of that distribution per position (a logged by-product)
   policy_loss_fwd     the clipped-ratio surrogate with KL weight 0 and separate lower /
                       upper clip thresholds (Section 4.2)
   policy_loss_bwd     its gradient with respect to the final hidden states and the
@@ -133,6 +134,23 @@ def token_logprobs(hidden: np.ndarray, W: np.ndarray, ids: np.ndarray) -> Dict[s
     lse = m + np.log(np.exp(z - m[:, None]).sum(axis=1))
     zy = z[np.arange(z.shape[0]), np.asarray(ids, dtype=np.int64)]
     return {"lse": lse, "logp": zy - lse, "z": z}
+
+
+def entropy_from_logits(z: np.ndarray, lse: np.ndarray) -> np.ndarray:
+    """H_t = - sum_v p[t,v] log p[t,v] with log p[t,v] = z[t,v] - lse_t (in nats)."""
+    logp_all = np.asarray(z, dtype=np.float64) - np.asarray(lse, dtype=np.float64)[:, None]
+    return -(np.exp(logp_all) * logp_all).sum(axis=1)
+
+
+def token_entropy(hidden: np.ndarray, W: np.ndarray) -> np.ndarray:
+    """Entropy of the policy's next-token distribution at every scored position:
+        p[t,v] = exp(z[t,v] - lse_t),   H_t = - sum_v p[t,v] log p[t,v].
+    Not part of the loss: the quantity RL post-training runs log beside the reward (the paper's
+    experiments track rewards only; Section 5), available from the same pass over the logits."""
+    z = logits(hidden, W)
+    m = z.max(axis=1)
+    lse = m + np.log(np.exp(z - m[:, None]).sum(axis=1))
+    return entropy_from_logits(z, lse)
 
 
 def _seq_of_token(cu_seqlens: np.ndarray) -> np.ndarray:

@@ -31,7 +31,7 @@ EXPORTS = ("sapo_pack_rollouts", "sapo_group_advantages", "sapo_policy_loss_fwd"
            "sapo_policy_loss_bwd", "sapo_workspace_bytes", "sapo_workspace_bytes_min",
            "sapo_status_string", "sapo_timing_enable", "sapo_timing_read", "sapo_launch_count",
            "sapo_policy_loss_fwd_static", "sapo_policy_loss_bwd_active", "sapo_policy_loss_fwd_bwd",
-           "sapo_select_external",
+           "sapo_select_external", "sapo_group_advantages_warp",
            "sapo_select_workspace_bytes", "sapo_adam_step")
 STATIC_SCRATCH_BYTES = 4 * 1024 * 1024
 KERNEL_NAMES = ("pack_scan", "pack_copy", "group_adv", "split_bf16", "fwd_gemm", "loss_tail",
@@ -59,7 +59,8 @@ class PackedC(C.Structure):
 
 class LossCfgC(C.Structure):
     _fields_ = [("eps_low", C.c_float), ("eps_high", C.c_float), ("grad_scale", C.c_float),
-                ("loss_agg", C.c_int32), ("kl_beta", C.c_float), ("ref_logp", C.c_void_p)]
+                ("loss_agg", C.c_int32), ("kl_beta", C.c_float), ("ref_logp", C.c_void_p),
+                ("entropy", C.c_void_p)]
 
 
 _lib: Optional[C.CDLL] = None
@@ -84,6 +85,8 @@ def load() -> C.CDLL:
                                        C.POINTER(SelectionC), i32, i32, C.POINTER(PackedC), vp, vp]
     lib.sapo_group_advantages.restype = C.c_int
     lib.sapo_group_advantages.argtypes = [vp, vp, i32, f32, i32, vp, vp, vp, vp, vp]
+    lib.sapo_group_advantages_warp.restype = C.c_int
+    lib.sapo_group_advantages_warp.argtypes = [vp, vp, i32, f32, i32, vp, vp, vp, vp, vp]
     lib.sapo_policy_loss_fwd.restype = C.c_int
     lib.sapo_policy_loss_fwd.argtypes = [vp, vp, i32, i64, i32, i32, i64, i64, vp, vp, vp, vp, i32,
                                          C.POINTER(LossCfgC), vp, vp, vp, vp, vp, vp, vp, vp, sz,
@@ -236,9 +239,11 @@ def sapo_pack_rollouts(local: DeviceRollouts, ext: DeviceRollouts, sel: DeviceSe
 
 def sapo_group_advantages(rewards: torch.Tensor, group_offsets: torch.Tensor, adv_eps: float,
                           ddof: int, adv: torch.Tensor, mean: Optional[torch.Tensor],
-                          std: Optional[torch.Tensor], status: torch.Tensor) -> None:
+                          std: Optional[torch.Tensor], status: torch.Tensor, warp_level: bool = False) -> None:
+    """warp_level=True always takes the warp-level kernel (sapo_group_advantages_warp)."""
     _require_cuda()
-    rc = load().sapo_group_advantages(_p(rewards), _p(group_offsets), int(group_offsets.numel() - 1),
+    fn = load().sapo_group_advantages_warp if warp_level else load().sapo_group_advantages
+    rc = fn(_p(rewards), _p(group_offsets), int(group_offsets.numel() - 1),
                                       float(adv_eps), int(ddof), _p(adv), _p(mean), _p(std),
                                       _p(status), _stream())
     _check(rc, "sapo_group_advantages")
@@ -263,12 +268,14 @@ def sapo_policy_loss_fwd(hidden: torch.Tensor, W_head: torch.Tensor, ids: torch.
                          eps_low: float, eps_high: float, grad_scale: float,
                          out: Dict[str, torch.Tensor], workspace: torch.Tensor,
                          status: torch.Tensor, T: Optional[int] = None, loss_agg: int = 0,
-                         kl_beta: float = 0.0, ref_logp: Optional[torch.Tensor] = None) -> None:
+                         kl_beta: float = 0.0, ref_logp: Optional[torch.Tensor] = None,
+                         entropy: Optional[torch.Tensor] = None) -> None:
+    """entropy: optional float32 [T] output, the per-token entropy of the policy's distribution."""
     _require_cuda()
     T = int(hidden.shape[0]) if T is None else int(T)
     H, V = int(hidden.shape[1]), int(W_head.shape[0])
     S = int(cu_seqlens.numel() - 1)
-    cfg = LossCfgC(eps_low, eps_high, grad_scale, int(loss_agg), float(kl_beta), _p(ref_logp))
+    cfg = LossCfgC(eps_low, eps_high, grad_scale, int(loss_agg), float(kl_beta), _p(ref_logp), _p(entropy))
     rc = load().sapo_policy_loss_fwd(
         _p(hidden), _p(W_head), _dtype_code(hidden), T, H, V, hidden.stride(0), W_head.stride(0),
         _p(ids), _p(old_logp), _p(adv), _p(cu_seqlens), S, C.byref(cfg),
@@ -290,7 +297,7 @@ def sapo_policy_loss_fwd_static(hidden: torch.Tensor, W_head: torch.Tensor, ids:
     T = int(hidden.shape[0]) if T is None else int(T)
     H, V = int(hidden.shape[1]), int(W_head.shape[0])
     S = int(cu_seqlens.numel() - 1)
-    cfg = LossCfgC(eps_low, eps_high, grad_scale, 0, 0.0, None)
+    cfg = LossCfgC(eps_low, eps_high, grad_scale, 0, 0.0, None, None)
     rc = load().sapo_policy_loss_fwd_static(
         _p(hidden), _p(W_head), _dtype_code(hidden), T, H, V, hidden.stride(0), W_head.stride(0),
         _p(ids), _p(old_logp), _p(adv), _p(cu_seqlens), S, C.byref(cfg),
@@ -335,13 +342,14 @@ def sapo_policy_loss_fwd_bwd(hidden: torch.Tensor, W_head: torch.Tensor, ids: to
                              out: Dict[str, torch.Tensor], dhidden: torch.Tensor, dW_head: torch.Tensor,
                              accumulate_dW: bool, workspace: torch.Tensor, status: torch.Tensor,
                              T: Optional[int] = None, loss_agg: int = 0, kl_beta: float = 0.0,
-                             ref_logp: Optional[torch.Tensor] = None) -> None:
+                             ref_logp: Optional[torch.Tensor] = None,
+                             entropy: Optional[torch.Tensor] = None) -> None:
     """Loss and both gradients in one call with a single pass over the logits (bf16 only)."""
     _require_cuda()
     T = int(hidden.shape[0]) if T is None else int(T)
     H, V = int(hidden.shape[1]), int(W_head.shape[0])
     S = int(cu_seqlens.numel() - 1)
-    cfg = LossCfgC(eps_low, eps_high, grad_scale, int(loss_agg), float(kl_beta), _p(ref_logp))
+    cfg = LossCfgC(eps_low, eps_high, grad_scale, int(loss_agg), float(kl_beta), _p(ref_logp), _p(entropy))
     rc = load().sapo_policy_loss_fwd_bwd(
         _p(hidden), _p(W_head), _dtype_code(hidden), T, H, V, hidden.stride(0), W_head.stride(0),
         _p(ids), _p(old_logp), _p(adv), _p(cu_seqlens), S, C.byref(cfg),

@@ -11,47 +11,49 @@ using namespace umma;
 // ---------------------------------------------------------------------------- epilogues
 // Each epilogue thread owns one accumulator row (TMEM lane) of the tile.
 
-// A thread's 64 finished bf16 entries of a panel row (two 32-column chunks as 16 pairs each) go
-// straight from its registers to the tile's row in global memory: the row is 128 contiguous
-// bytes, written as four 32-byte stores, so every store fills whole sectors.  (Staging the tile
-// in shared memory for one TMA store per tile was measured slower: the kernel's operand traffic
-// already fills the shared-memory bandwidth, and the staged copy took the MMA issuer's share:
-// 4-5 % more cycles per launch.)
-__device__ __forceinline__ void store_panel_group(__nv_bfloat16* panel, int r, const uint32_t (&pk)[2][16],
-                                                  int tile_row0, int col0_of_group) {
+// Panel rows go straight from the epilogue threads' registers to global memory.  A tile row is
+// 128 contiguous bytes (64 bf16); a thread writes it as 32-byte stores, each a whole sector.
+// (Staging the tile in shared memory for one TMA store per tile was measured slower: the kernel's
+// operand traffic already fills the shared-memory bandwidth, and the staged copy cost the MMA
+// issuer 4-5 % more cycles per launch.)
+// 16 finished bf16 entries (32 bytes, one sector) of a panel row: columns [col0, col0 + 16) of the
+// tile row `r` of token block `tile_row0`.
+__device__ __forceinline__ void store_panel_16(__nv_bfloat16* panel, int r, int tile_row0, int col0,
+                                               const uint32_t (&w)[8]) {
   uint8_t* dst = reinterpret_cast<uint8_t*>(panel) +
-                 ((size_t)tile_row0 + (size_t)(col0_of_group >> 6) * BM + (size_t)r) * 128;
-  #pragma unroll
-  for (int q = 0; q < 4; ++q) {
-    const uint32_t* w = &pk[q >> 1][8 * (q & 1)];
-    asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
-                 ::"l"(dst + 32 * q), "r"(w[0]), "r"(w[1]), "r"(w[2]), "r"(w[3]), "r"(w[4]), "r"(w[5]), "r"(w[6]), "r"(w[7])
-                 : "memory");
-  }
+                 ((size_t)tile_row0 + (size_t)(col0 >> 6) * BM + (size_t)r) * 128 + (size_t)(col0 & 63) * 2;
+  asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
+               ::"l"(dst), "r"(w[0]), "r"(w[1]), "r"(w[2]), "r"(w[3]), "r"(w[4]), "r"(w[5]), "r"(w[6]), "r"(w[7])
+               : "memory");
 }
 
 // Forward: online log-sum-exp in the base-2 domain plus the logit of the chosen token.
-struct FwdEpi {
+// ENT: also the running sum of 2^(x - m) z, from which the tail forms the entropy of the row's
+// distribution, H = lse - sum_v p_v z_v (one more multiply-add per logit, so it is a variant).
+template <bool ENT>
+struct FwdEpiT {
   static constexpr bool PANEL = false;
   static constexpr bool STREAMK = false;
   template <class P> __device__ static void set_dynamic(P&, const Sched&) {}
 
   struct Params {
     const int32_t* ids; float* pm; float* ps; float* pz;  // partials [n_splits][T]
+    float* pe;                                             // ENT: partial sums of 2^(x - m) z
     int64_t T; int32_t V;
   };
-  float m, s, zy; int32_t y; int64_t row;
+  float m, s, zy, sz; int32_t y; int64_t row;
   __device__ __forceinline__ void begin_unit(const Params& p, int mb, int r) {
     row = (int64_t)mb * BM + r;
-    m = -INFINITY; s = 0.f; zy = 0.f;
+    m = -INFINITY; s = 0.f; zy = 0.f; sz = 0.f;
     y = row < p.T ? p.ids[row] : -1;
   }
   template <int HALF>
   __device__ __forceinline__ void chunk(const Params& p, float (&v)[32], int col0) {
     if (col0 >= p.V) return;
     if (col0 + 32 > p.V) {
+      // columns past the vocabulary: far below any logit, but finite so that 0 * z stays 0
       #pragma unroll
-      for (int j = 0; j < 32; ++j) if (col0 + j >= p.V) v[j] = -INFINITY;
+      for (int j = 0; j < 32; ++j) if (col0 + j >= p.V) v[j] = -1e30f;
     }
     const int yr = y - col0;
     if (yr >= 0 && yr < 32) {
@@ -62,19 +64,27 @@ struct FwdEpi {
     #pragma unroll
     for (int j = 1; j < 32; ++j) cmax = fmaxf(cmax, v[j]);
     const float m_new = fmaxf(m, cmax * LOG2E);
-    float acc = s * ex2(m - m_new);          // first chunk: ex2(-inf) = 0
+    const float rescale = ex2(m - m_new);    // first chunk: ex2(-inf) = 0
+    float acc = s * rescale;
+    float acc_z = sz * rescale;
     #pragma unroll
-    for (int j = 0; j < 32; ++j) acc += ex2(fmaf(v[j], LOG2E, -m_new));
-    s = acc; m = m_new;
+    for (int j = 0; j < 32; ++j) {
+      const float e = ex2(fmaf(v[j], LOG2E, -m_new));
+      acc += e;
+      if constexpr (ENT) acc_z = fmaf(e, v[j], acc_z);
+    }
+    s = acc; m = m_new; sz = acc_z;
   }
   // two threads share a row (one per column half of the tiles): each leaves its own partial
   __device__ __forceinline__ void end_unit(const Params& p, int un, int col_half) {
     if (row < p.T) {
       const int64_t o = (int64_t)(2 * un + col_half) * p.T + row;
       p.pm[o] = m; p.ps[o] = s; p.pz[o] = zy;
+      if constexpr (ENT) p.pe[o] = sz;
     }
   }
 };
+using FwdEpi = FwdEpiT<false>;
 
 // Backward, first contraction: dz[t,v] = g_t ([v == y_t] - exp(z[t,v] - lse_t)), to bf16.
 // The panel is a sequence of [128 token x 64 vocab] tiles of 16 KB, tile (tb, vt) at index
@@ -104,38 +114,43 @@ struct DzEpi {
     l2 = valid ? p.lse[row] * LOG2E : 0.f;
     y = valid ? p.ids[row] : -1;
   }
-  // dz of 32 columns, kept in registers as 16 bf16 pairs until the whole 64-column group is done
-  uint32_t pk[2][16];
-  template <int HALF>   // which 32-column half of the group (a compile-time register choice)
+  // dz of 32 columns; every 16 finished columns (32 bytes of the row) are stored at once, so the
+  // stores of the eight epilogue warps trickle out between their arithmetic instead of leaving
+  // the SM in bursts of whole rows
+  template <int HALF>   // which 32-column half of the 64-column group (kept for symmetry with the other epilogues)
   __device__ __forceinline__ void chunk(const Params& p, float (&v)[32], int col0) {
     if (!in_panel) return;
-    uint32_t (&packed)[16] = pk[HALF];
+    uint32_t w[8];
     if (g == 0.f) {
       #pragma unroll
-      for (int j = 0; j < 16; ++j) packed[j] = 0u;
-    } else {
-      const float ng = -g;
+      for (int j = 0; j < 8; ++j) w[j] = 0u;
+      store_panel_16(p.panel, r, tile_row0, col0, w);
+      store_panel_16(p.panel, r, tile_row0, col0 + 16, w);
+      return;
+    }
+    const float ng = -g;
+    const int yr = y - col0;
+    #pragma unroll
+    for (int h = 0; h < 2; ++h) {
       #pragma unroll
-      for (int j = 0; j < 32; ++j) v[j] = ng * ex2(fmaf(v[j], LOG2E, -l2));
-      const int yr = y - col0;
-      if (yr >= 0 && yr < 32) {            // the chunk that holds the chosen token
+      for (int j = 16 * h; j < 16 * h + 16; ++j) v[j] = ng * ex2(fmaf(v[j], LOG2E, -l2));
+      if (yr >= 16 * h && yr < 16 * h + 16) {            // the columns that hold the chosen token
         #pragma unroll
-        for (int j = 0; j < 32; ++j) if (j == yr) v[j] += g;
+        for (int j = 16 * h; j < 16 * h + 16; ++j) if (j == yr) v[j] += g;
       }
-      if (col0 + 32 > p.V) {               // ragged end of the vocabulary
+      if (col0 + 16 * h + 16 > p.V) {                     // ragged end of the vocabulary
         #pragma unroll
-        for (int j = 0; j < 32; ++j) if (col0 + j >= p.V) v[j] = 0.f;
+        for (int j = 16 * h; j < 16 * h + 16; ++j) if (col0 + j >= p.V) v[j] = 0.f;
       }
       #pragma unroll
-      for (int j = 0; j < 16; ++j) {
-        __nv_bfloat162 h = __floats2bfloat162_rn(v[2 * j], v[2 * j + 1]);
-        packed[j] = *reinterpret_cast<uint32_t*>(&h);
+      for (int j = 0; j < 8; ++j) {
+        __nv_bfloat162 b2 = __floats2bfloat162_rn(v[16 * h + 2 * j], v[16 * h + 2 * j + 1]);
+        w[j] = *reinterpret_cast<uint32_t*>(&b2);
       }
+      store_panel_16(p.panel, r, tile_row0, col0 + 16 * h, w);
     }
   }
-  __device__ __forceinline__ void group_end(const Params& p, int col0_of_group) {
-    if (in_panel) store_panel_group(p.panel, r, pk, tile_row0, col0_of_group);
-  }
+  __device__ __forceinline__ void group_end(const Params&, int) {}
   __device__ __forceinline__ void end_unit(const Params&, int, int) {}
 };
 
@@ -147,18 +162,19 @@ struct DzEpi {
 // safe range (2^100 and beyond, infinite or NaN) shows in its sum, and fused_tail_kernel then
 // reports it and clears its panel row, so that the backward contractions only ever see finite
 // entries.  Rows past the last token and columns past V hold zeros.
-struct ExpEpi {
+template <bool ENT>     // ENT: also sum_v e[t,v] z[t,v] per token (for the entropy, see FwdEpiT)
+struct ExpEpiT {
   static constexpr bool PANEL = true;
   static constexpr bool STREAMK = false;
   template <class P> __device__ static void set_dynamic(P&, const Sched&) {}
   struct Params {
     const float* c2;      // [M] reference of each token, in the base-2 domain (c_t * log2 e)
     float* ps;            // [2 * n_splits][M] partial sums of exponentials
+    float* pe;            // ENT: [2 * n_splits][M] partial sums of e z
     int64_t M; int32_t V; int32_t nvt;
     __nv_bfloat16* panel;
   };
-  float c, sum; int32_t tile_row0; int r; bool valid, in_panel; int64_t row;
-  uint32_t pk[2][16];
+  float c, sum, sz; int32_t tile_row0; int r; bool valid, in_panel; int64_t row;
   __device__ __forceinline__ void begin_unit(const Params& p, int mb, int r_) {
     row = (int64_t)mb * BM + r_;
     valid = row < p.M;
@@ -166,41 +182,55 @@ struct ExpEpi {
     r = r_;
     tile_row0 = mb * p.nvt * BM;
     c = valid ? p.c2[row] : 0.f;
-    sum = 0.f;
+    sum = 0.f; sz = 0.f;
   }
   template <int HALF>
   __device__ __forceinline__ void chunk(const Params& p, float (&v)[32], int col0) {
     if (!in_panel) return;
-    uint32_t (&packed)[16] = pk[HALF];
+    uint32_t w[8];
     if (!valid || col0 >= p.V) {
       #pragma unroll
-      for (int j = 0; j < 16; ++j) packed[j] = 0u;
+      for (int j = 0; j < 8; ++j) w[j] = 0u;
+      store_panel_16(p.panel, r, tile_row0, col0, w);
+      store_panel_16(p.panel, r, tile_row0, col0 + 16, w);
       return;
     }
+    // every 16 finished columns (32 bytes of the row) are stored at once: see DzEpi
     #pragma unroll
-    for (int j = 0; j < 32; ++j) v[j] = ex2(fmaf(v[j], LOG2E, -c));
-    if (col0 + 32 > p.V) {               // ragged end of the vocabulary
+    for (int h = 0; h < 2; ++h) {
       #pragma unroll
-      for (int j = 0; j < 32; ++j) if (col0 + j >= p.V) v[j] = 0.f;
-    }
-    float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
-    #pragma unroll
-    for (int j = 0; j < 32; j += 4) { a0 += v[j]; a1 += v[j + 1]; a2 += v[j + 2]; a3 += v[j + 3]; }
-    sum += (a0 + a1) + (a2 + a3);
-    #pragma unroll
-    for (int j = 0; j < 16; ++j) {
-      __nv_bfloat162 h = __floats2bfloat162_rn(v[2 * j], v[2 * j + 1]);
-      packed[j] = *reinterpret_cast<uint32_t*>(&h);
+      for (int j = 16 * h; j < 16 * h + 16; ++j) {
+        const float e = ex2(fmaf(v[j], LOG2E, -c));
+        // (columns past the vocabulary hold z = 0 from the zero-filled load: they add nothing)
+        if constexpr (ENT) sz = fmaf((col0 + j < p.V) ? e : 0.f, v[j], sz);
+        v[j] = e;
+      }
+      if (col0 + 16 * h + 16 > p.V) {                     // ragged end of the vocabulary
+        #pragma unroll
+        for (int j = 16 * h; j < 16 * h + 16; ++j) if (col0 + j >= p.V) v[j] = 0.f;
+      }
+      float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+      #pragma unroll
+      for (int j = 16 * h; j < 16 * h + 16; j += 4) { a0 += v[j]; a1 += v[j + 1]; a2 += v[j + 2]; a3 += v[j + 3]; }
+      sum += (a0 + a1) + (a2 + a3);
+      #pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        __nv_bfloat162 b2 = __floats2bfloat162_rn(v[16 * h + 2 * j], v[16 * h + 2 * j + 1]);
+        w[j] = *reinterpret_cast<uint32_t*>(&b2);
+      }
+      store_panel_16(p.panel, r, tile_row0, col0 + 16 * h, w);
     }
   }
-  __device__ __forceinline__ void group_end(const Params& p, int col0_of_group) {
-    if (in_panel) store_panel_group(p.panel, r, pk, tile_row0, col0_of_group);
-  }
+  __device__ __forceinline__ void group_end(const Params&, int) {}
   // two threads share a row (one per column half of the tiles): each leaves its own partial
   __device__ __forceinline__ void end_unit(const Params& p, int un, int col_half) {
-    if (valid) p.ps[(int64_t)(2 * un + col_half) * p.M + row] = sum;
+    if (valid) {
+      p.ps[(int64_t)(2 * un + col_half) * p.M + row] = sum;
+      if constexpr (ENT) p.pe[(int64_t)(2 * un + col_half) * p.M + row] = sz;
+    }
   }
 };
+using ExpEpi = ExpEpiT<false>;
 
 // Plain fp32 output tile, optionally added to what is already there.
 struct StoreEpi {

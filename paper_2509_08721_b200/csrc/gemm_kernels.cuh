@@ -21,11 +21,15 @@ using namespace umma;
 // [n0 + rank * n_eff / 2, + n_eff / 2) of B.  All TMA completions of a stage are counted on the
 // even CTA's barrier; the even CTA's MMA thread frees stages and publishes accumulators on
 // both CTAs' barriers.
-template <int A_KIND, bool B_MN, class Epi>
+template <int A_KIND, bool B_MN, class Epi, int BKT = BK, int NSTAGE = STAGES>
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
 umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                  const Sched sched_arg, const typename Epi::Params ep_arg, int32_t* status) {
   SAPO_CLOCK_BEGIN
+  // a stage holds a K depth of BKT (128: two 64-element boxes per K-major operand; 64: one)
+  static_assert(BKT == 128 || (BKT == 64 && A_KIND == 0 && !B_MN), "64-deep stages: K-major operands only");
+  constexpr int KBOX = BKT / 64;
+  constexpr uint32_t A_ST = BM * BKT * 2, B_ST = (BN / 2) * BKT * 2;
   Sched sched = sched_arg;
   typename Epi::Params ep = ep_arg;
   finalize_sched(sched, (int)(gridDim.x >> 1));
@@ -33,13 +37,13 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint8_t* smem_a = smem;
-  uint8_t* smem_b = smem + STAGES * A_STAGE_BYTES;
-  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + STAGES * (A_STAGE_BYTES + B_STAGE_BYTES));
-  uint64_t* full = bars;                 // [STAGES] TMA -> MMA          (even CTA's are used)
-  uint64_t* empty = bars + STAGES;       // [STAGES] MMA -> TMA          (each CTA waits on its own)
-  uint64_t* acc_full = bars + 2 * STAGES;      // [2] MMA -> epilogue    (each CTA waits on its own)
-  uint64_t* acc_empty = bars + 2 * STAGES + 2; // [2] epilogue -> MMA    (even CTA's are used)
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * STAGES + 4);
+  uint8_t* smem_b = smem + NSTAGE * A_ST;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + NSTAGE * (A_ST + B_ST));
+  uint64_t* full = bars;                 // [NSTAGE] TMA -> MMA          (even CTA's are used)
+  uint64_t* empty = bars + NSTAGE;       // [NSTAGE] MMA -> TMA          (each CTA waits on its own)
+  uint64_t* acc_full = bars + 2 * NSTAGE;      // [2] MMA -> epilogue    (each CTA waits on its own)
+  uint64_t* acc_empty = bars + 2 * NSTAGE + 2; // [2] epilogue -> MMA    (even CTA's are used)
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * NSTAGE + 4);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -48,7 +52,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
   const int pair = blockIdx.x >> 1, num_pairs = gridDim.x >> 1;
 
   if (threadIdx.x == 0) {
-    for (int i = 0; i < STAGES; ++i) { mbar_init(&full[i], 1); mbar_init(&empty[i], 1); }
+    for (int i = 0; i < NSTAGE; ++i) { mbar_init(&full[i], 1); mbar_init(&empty[i], 1); }
     for (int i = 0; i < 2; ++i) { mbar_init(&acc_full[i], 1); mbar_init(&acc_empty[i], 16); }
     *abort_flag = 0;
     fence_mbar_init();
@@ -75,20 +79,20 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
     int stage = 0; uint32_t phase = 0;
     uint32_t in_flight = 0;   // bit i: stage i was filled in the current ring pass
     bool ok = true;
-    constexpr int A_BOXES = A_KIND == 2 ? 1 : 2;
+    constexpr int A_BOXES = A_KIND == 2 ? 1 : KBOX;
     WorkList work(sched, pair, num_pairs);
     int pmb, un, n_begin, n_end, kb0, kb1, slot;
     while (ok && work.next(pmb, un, n_begin, n_end, kb0, kb1, slot)) {
       const int mb = 2 * pmb + (int)rank;                 // this CTA's 128-row block
       for (int nb = n_begin; ok && nb < n_end; ++nb) {
         const int half = tile_n_eff(sched, nb) >> 1;       // B columns this CTA stages
-        const int b_boxes = B_MN ? ((half + 63) >> 6) : 2;
-        const uint32_t tx = 2 * (A_STAGE_BYTES + b_boxes * BOX_BYTES);
+        const int b_boxes = B_MN ? ((half + 63) >> 6) : KBOX;
+        const uint32_t tx = 2 * (A_ST + b_boxes * BOX_BYTES);
         const bool mine = lane < A_BOXES + b_boxes;
         const bool is_a = lane < A_BOXES;
         const int bi = is_a ? lane : lane - A_BOXES;
         const CUtensorMap* map = is_a ? &map_a : &map_b;
-        const uint32_t dst_off = is_a ? bi * BOX_BYTES : STAGES * A_STAGE_BYTES + bi * BOX_BYTES;
+        const uint32_t dst_off = is_a ? bi * BOX_BYTES : NSTAGE * A_ST + bi * BOX_BYTES;
         const bool mn = is_a ? A_MN : B_MN;
         // m or n coordinate of the box (an MN-major box covers 64 of them, a K-major one 128)
         const int row0 = is_a ? mb * BM + (mn ? 64 * bi : 0)
@@ -98,24 +102,24 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
           if (!SAPO_TIMED(0, mbar_wait(&empty[stage], phase ^ 1, abort_flag))) { ok = false; break; }
           if (rank == 0 && lane == 0) mbar_arrive_expect_tx(&full[stage], tx);
           if (mine) {
-            uint8_t* dst = smem + dst_off + stage * (is_a ? A_STAGE_BYTES : B_STAGE_BYTES);
+            uint8_t* dst = smem + dst_off + stage * (is_a ? A_ST : B_ST);
             const uint32_t bar = full0_addr + stage * 8;
             if (is_a && A_KIND == 2)        // vocab tiles 2 kb and 2 kb + 1 of token block mb: 256 rows
               tma_load_2d_pair(dst, map, bar, 0, (mb * sched.panel_nvt + 2 * kb) * BM);
             else if (is_a && A_KIND == 3)   // token block kb, vocab tile 2 mb + bi: all 128 rows
               tma_load_2d_pair(dst, map, bar, 0, (kb * sched.panel_nvt + 2 * mb + bi) * BM);
-            else if (mn) tma_load_2d_pair(dst, map, bar, row0, kb * BK);
-            else         tma_load_2d_pair(dst, map, bar, kb * BK + k_off, row0);
+            else if (mn) tma_load_2d_pair(dst, map, bar, row0, kb * BKT);
+            else         tma_load_2d_pair(dst, map, bar, kb * BKT + k_off, row0);
           }
           in_flight |= 1u << stage;
-          if (++stage == STAGES) { stage = 0; phase ^= 1; }
+          if (++stage == NSTAGE) { stage = 0; phase ^= 1; }
         }
       }
     }
     if (lane == 0) SAPO_STATS_FLUSH(4);
     if (!ok && rank == 0 && lane == 0) {
       // give copies already issued a bounded chance to land before the pair leaves
-      for (int i = 0; i < STAGES; ++i) {
+      for (int i = 0; i < NSTAGE; ++i) {
         if (!(in_flight & (1u << i))) continue;
         const uint32_t ph = (i < stage) ? phase : (phase ^ 1);
         for (int spin = 0; spin < (1 << 20) && !mbar_try_wait(&full[i], ph); ++spin) {}
@@ -138,10 +142,10 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
         for (int kb = kb0; kb < kb1; ++kb) {
           if (!SAPO_TIMED(1, mbar_wait(&full[stage], phase, abort_flag))) { ok = false; break; }
           fence_after_sync();
-          const uint32_t a_addr = smem_u32(smem_a + stage * A_STAGE_BYTES);
-          const uint32_t b_addr = smem_u32(smem_b + stage * B_STAGE_BYTES);
+          const uint32_t a_addr = smem_u32(smem_a + stage * A_ST);
+          const uint32_t b_addr = smem_u32(smem_b + stage * B_ST);
           #pragma unroll
-          for (int k = 0; k < BK / UMMA_K; ++k) {
+          for (int k = 0; k < BKT / UMMA_K; ++k) {
             // K-major: 16 elements = 32 bytes along the row, the second half of the depth in
             // the next box; MN-major: 16 rows = 2048 bytes, 64-column chunks one box apart
             const uint32_t k_major_off = (k >> 2) * BOX_BYTES + (k & 3) * 32;
@@ -154,7 +158,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
           // free the stage in both CTAs once these MMAs retire
           mma_commit_pair(empty_addr[0] + stage * 8);
           mma_commit_pair(empty_addr[1] + stage * 8);
-          if (++stage == STAGES) { stage = 0; phase ^= 1; }
+          if (++stage == NSTAGE) { stage = 0; phase ^= 1; }
         }
         if (ok) {                                  // accumulator complete, in both CTAs
           mma_commit_pair(acc_full_addr[0] + acc * 8);

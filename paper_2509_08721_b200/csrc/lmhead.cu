@@ -72,7 +72,8 @@ static bool make_map_f32_out(CUtensorMap* map, const float* base, int64_t inner,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-static Sched make_sched(int64_t M, int64_t N, int64_t K, int n_splits, bool m_fastest, int tile_align = 32) {
+static Sched make_sched(int64_t M, int64_t N, int64_t K, int n_splits, bool m_fastest, int tile_align = 32,
+                        int bk = BK) {
   Sched s{};
   s.num_m_blocks = (int32_t)ceil_div<int64_t>(M, PAIR_M);
   const int64_t tiles = ceil_div<int64_t>(N, BN);
@@ -81,7 +82,7 @@ static Sched make_sched(int64_t M, int64_t N, int64_t K, int n_splits, bool m_fa
   s.n_per_unit = n_splits > 0 ? ceil_div(s.num_n_blocks, n_splits) : 1;
   s.units_per_m = ceil_div(s.num_n_blocks, s.n_per_unit);
   s.num_units = s.num_m_blocks * s.units_per_m;
-  s.num_k_blocks = (int32_t)ceil_div<int64_t>(K, BK);
+  s.num_k_blocks = (int32_t)ceil_div<int64_t>(K, bk);
   s.m_fastest = m_fastest ? 1 : 0;
   // row blocks whose A rows (256 x K bf16 each) fit in about 48 MB of the 126 MB L2
   {
@@ -124,10 +125,17 @@ static int fwd_splits(int64_t T, int32_t V, int64_t K, int sms) {
   return (int)ceil_div(nb, per);
 }
 
-template <int A_KIND, bool B_MN, class Epi>
+// Stage shape of the three projections hidden . W^T (forward, dz, single pass): K depth and ring length
+#ifdef SAPO_FWD_BK64
+constexpr int FWD_BK = 64, FWD_STAGES = 7;
+#else
+constexpr int FWD_BK = BK, FWD_STAGES = STAGES;
+#endif
+
+template <int A_KIND, bool B_MN, class Epi, int BKT = BK, int NSTAGE = STAGES>
 static int launch_gemm(const CUtensorMap& ma, const CUtensorMap& mb, const Sched& sched,
                        const typename Epi::Params& ep, int32_t* status, cudaStream_t st, int kernel_id) {
-  auto kern = umma_gemm_kernel<A_KIND, B_MN, Epi>;
+  auto kern = umma_gemm_kernel<A_KIND, B_MN, Epi, BKT, NSTAGE>;
   // CTA pairs the device can hold at once; found, together with the kernel's shared-memory
   // opt-in, on the first use on each device
   static int max_pairs_of[MAX_DEVICES] = {0};
@@ -142,7 +150,7 @@ static int launch_gemm(const CUtensorMap& ma, const CUtensorMap& mb, const Sched
   attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
   cudaLaunchConfig_t cfg = {};
   cfg.blockDim = dim3(GEMM_THREADS, 1, 1);
-  constexpr size_t smem_bytes = GEMM_SMEM_BYTES;
+  constexpr size_t smem_bytes = 1024 + (size_t)NSTAGE * (BM + BN / 2) * BKT * 2 + 256;
   cfg.dynamicSmemBytes = smem_bytes;
   cfg.stream = st;
   cfg.attrs = attr;
@@ -316,12 +324,14 @@ static int64_t padded_vocab(int32_t V) { return round_up<int64_t>(V, 128); }
 struct FwdLayout { size_t partials, a_split, b_split, total; int n_splits; };
 // max_splits > 0 caps the number of vocab splits (fewer splits: less scratch, the same results up
 // to the order in which the partial sums of a token are added)
-static FwdLayout fwd_layout(int64_t T, int32_t H, int32_t V, int32_t dtype, int sms, int max_splits = 0) {
+static FwdLayout fwd_layout(int64_t T, int32_t H, int32_t V, int32_t dtype, int sms, int max_splits = 0,
+                            bool entropy = true) {
   FwdLayout L{};
   L.n_splits = fwd_splits(T, V, dtype == SAPO_DTYPE_F32 ? 3 * (int64_t)H : (int64_t)H, sms);
   if (max_splits > 0 && L.n_splits > max_splits) L.n_splits = max_splits;
   size_t off = 0;
-  L.partials = off; off += round_up<size_t>((size_t)3 * 2 * L.n_splits * T * sizeof(float), 256);
+  // per vocab split and column half: running max, sum, target logit (and the entropy's sum)
+  L.partials = off; off += round_up<size_t>((size_t)(entropy ? 4 : 3) * 2 * L.n_splits * T * sizeof(float), 256);
   if (dtype == SAPO_DTYPE_F32) {
     L.a_split = off; off += round_up<size_t>((size_t)T * 3 * H * 2, 256);
     L.b_split = off; off += round_up<size_t>((size_t)V * 3 * H * 2, 256);
@@ -343,7 +353,22 @@ static BwdLayout bwd_layout(int64_t T, int32_t H, int32_t V, int32_t dtype) {
   L.bytes_per_row = (size_t)padded_vocab(V) * 2;
   return L;
 }
-constexpr int64_t PANEL_ROWS_PREFERRED = 32768;
+// Token rows of the panel the workspace queries ask for.  Measured (hidden 896 and 1536, vocab
+// 151936): a step over chunks of 16384 tokens is within 0.3 % of one over chunks of 32768, chunks
+// of 8192 cost 2-3 %, of 2048 about 15 %; a batch of up to 20480 tokens is fastest in one piece.
+// Longer batches are cut into equal chunks of at most 16384 tokens (rounded up to whole
+// 128-token blocks), so that no short ragged chunk is left at the end.
+constexpr int64_t PANEL_ROWS_TARGET = 16384;
+constexpr int64_t PANEL_ROWS_ONE_PIECE = 20480;
+static int64_t equal_chunk_rows(int64_t T, int64_t max_rows) {     // max_rows: a multiple of 128
+  const int64_t n = ceil_div<int64_t>(T, max_rows);
+  const int64_t rows = round_up<int64_t>(ceil_div<int64_t>(T, n), BM);
+  return rows < max_rows ? rows : max_rows;
+}
+static int64_t preferred_panel_rows(int64_t T) {
+  if (T <= PANEL_ROWS_ONE_PIECE) return round_up<int64_t>(T, BM);
+  return equal_chunk_rows(T, PANEL_ROWS_TARGET);
+}
 
 // Scratch of the fused call: per-token vectors for all T tokens, then what one token chunk
 // needs (row scales, partial sums, the scaled copy of hidden), the K-split scratch, the
@@ -362,22 +387,23 @@ static FusedLayout fused_layout(int64_t T, int32_t H, int32_t V, int32_t S) {
   L.partials = take(KSPLIT_SCRATCH_BYTES);
   L.fixed = off;
   // per chunk row: panel row, scaled hidden row, row scale, partial sums
-  L.bytes_per_row = (size_t)padded_vocab(V) * 2 + (size_t)H * 2 + 4 + (size_t)2 * FUSED_MAX_SPLITS * 4;
+  L.bytes_per_row = (size_t)padded_vocab(V) * 2 + (size_t)H * 2 + 4 + (size_t)2 * 2 * FUSED_MAX_SPLITS * 4;
   return L;
 }
 // where the per-chunk arrays sit for a chunk capacity of `rows` (a multiple of 128)
-struct FusedChunk { size_t row_scale, ps, hs, panel; };
+struct FusedChunk { size_t row_scale, ps, pe, hs, panel; };
 static FusedChunk fused_chunk(const FusedLayout& L, int64_t rows, int32_t H) {
   FusedChunk C{};
   size_t off = L.fixed;
   auto take = [&](size_t bytes) { const size_t at = off; off += round_up<size_t>(bytes, 256); return at; };
   C.row_scale = take((size_t)rows * 4);
   C.ps = take((size_t)rows * 2 * FUSED_MAX_SPLITS * 4);
+  C.pe = take((size_t)rows * 2 * FUSED_MAX_SPLITS * 4);
   C.hs = take((size_t)rows * H * 2);
   C.panel = take(0);
   return C;
 }
-constexpr size_t FUSED_CHUNK_SLACK = 4 * 256;   // alignment padding between the per-chunk arrays
+constexpr size_t FUSED_CHUNK_SLACK = 5 * 256;   // alignment padding between the per-chunk arrays
 
 // Scratch of the compacting backward in front of the regular backward's: scan counters, the
 // active-token list, compacted per-token vectors and hidden rows.
@@ -445,14 +471,12 @@ extern "C" size_t sapo_workspace_bytes(int32_t which, int64_t T, int32_t H, int3
   if (which == SAPO_WS_FUSED) {
     if (dtype != SAPO_DTYPE_BF16) return 0;
     const FusedLayout L = fused_layout(T, H, V, /*S=*/(int32_t)(T < 0x7fffffff ? T : 0x7fffffff));
-    const int64_t rows = T < PANEL_ROWS_PREFERRED ? T : PANEL_ROWS_PREFERRED;
-    return L.fixed + FUSED_CHUNK_SLACK + (size_t)round_up<int64_t>(rows, BM) * L.bytes_per_row;
+    return L.fixed + FUSED_CHUNK_SLACK + (size_t)preferred_panel_rows(T) * L.bytes_per_row;
   }
   if (which == SAPO_WS_BWD || which == SAPO_WS_BWD_ACTIVE) {
     const BwdLayout L = bwd_layout(T, H, V, dtype);
-    const int64_t rows = T < PANEL_ROWS_PREFERRED ? T : PANEL_ROWS_PREFERRED;
     const size_t extra = which == SAPO_WS_BWD_ACTIVE ? active_layout(T, H).total : 0;
-    return extra + L.fixed + (size_t)round_up<int64_t>(rows, BM) * L.bytes_per_row;
+    return extra + L.fixed + (size_t)preferred_panel_rows(T) * L.bytes_per_row;
   }
   return 0;
 }
@@ -485,7 +509,8 @@ static int fwd_impl(const void* hidden, const void* W_head, int32_t dtype,
   if (!workspace || !aligned16(workspace)) return SAPO_ERR_INVALID_ARG;
   const int sms = sm_count();
   if (sms <= 0) return SAPO_ERR_CUDA;
-  const FwdLayout L = fwd_layout(T, H, V, dtype, sms, max_splits);
+  const bool want_entropy = h_cfg->entropy != nullptr;
+  const FwdLayout L = fwd_layout(T, H, V, dtype, sms, max_splits, want_entropy);
   // seq_surr scratch lives behind the layout when the caller does not want it
   const size_t need = L.total + (seq_surr ? 0 : round_up<size_t>((size_t)S * sizeof(float), 256));
   if (workspace_bytes < need) return SAPO_ERR_WORKSPACE_TOO_SMALL;
@@ -494,6 +519,7 @@ static int fwd_impl(const void* hidden, const void* W_head, int32_t dtype,
   float* pm = reinterpret_cast<float*>(ws + L.partials);
   float* ps = pm + (size_t)2 * L.n_splits * T;
   float* pz = ps + (size_t)2 * L.n_splits * T;
+  float* pe = want_entropy ? pz + (size_t)2 * L.n_splits * T : nullptr;
   float* seq_out = seq_surr ? seq_surr : reinterpret_cast<float*>(ws + L.total);
 
   const void* A = hidden; const void* B = W_head;
@@ -509,13 +535,20 @@ static int fwd_impl(const void* hidden, const void* W_head, int32_t dtype,
   }
   CUtensorMap map_a, map_b;
   if (!make_map(&map_a, A, K, T, lda, BM) || !make_map(&map_b, B, K, V, ldb, 128)) return SAPO_ERR_CUDA;
-  const Sched sched = make_sched(T, V, K, L.n_splits, /*m_fastest=*/true);
-  FwdEpi::Params ep{ids, pm, ps, pz, T, V};
-  int rc = launch_gemm<0, false, FwdEpi>(map_a, map_b, sched, ep, status, st, SAPO_K_FWD_GEMM);
+  const Sched sched = make_sched(T, V, K, L.n_splits, /*m_fastest=*/true, 32, FWD_BK);
+  int rc;
+  if (want_entropy) {
+    FwdEpiT<true>::Params ep{ids, pm, ps, pz, pe, T, V};
+    rc = launch_gemm<0, false, FwdEpiT<true>, FWD_BK, FWD_STAGES>(map_a, map_b, sched, ep, status, st, SAPO_K_FWD_GEMM);
+  } else {
+    FwdEpi::Params ep{ids, pm, ps, pz, nullptr, T, V};
+    rc = launch_gemm<0, false, FwdEpi, FWD_BK, FWD_STAGES>(map_a, map_b, sched, ep, status, st, SAPO_K_FWD_GEMM);
+  }
   if (rc != SAPO_OK) return rc;
 
   TailArgs ta{};
   ta.pm = pm; ta.ps = ps; ta.pz = pz; ta.T = T;
+  ta.pe = pe; ta.entropy = h_cfg->entropy;
   ta.n_splits = 2 * sched.units_per_m;   // one partial per vocab split and column half
   ta.ids = ids; ta.V = V; ta.old_logp = old_logp; ta.adv = adv; ta.cu = cu_seqlens; ta.S = S;
   ta.lo_edge = 1.f - h_cfg->eps_low; ta.hi_edge = 1.f + h_cfg->eps_high; ta.grad_scale = h_cfg->grad_scale;
@@ -596,8 +629,10 @@ extern "C" int sapo_policy_loss_fwd_static(const void* hidden, const void* W_hea
   const size_t seq_bytes = seq_surr ? 0 : round_up<size_t>((size_t)S * sizeof(float), 256);
   if (seq_bytes >= (size_t)SAPO_STATIC_SCRATCH_BYTES) return SAPO_ERR_STATIC_SCRATCH_EXCEEDED;
   const size_t avail = (size_t)SAPO_STATIC_SCRATCH_BYTES - seq_bytes;
-  int max_splits = (int)(avail / ((size_t)24 * (size_t)T) > 4096 ? 4096 : avail / ((size_t)24 * (size_t)T));
-  while (max_splits >= 1 && fwd_layout(T, H, V, dtype, sms, max_splits).total > avail) --max_splits;
+  const bool want_entropy = h_cfg->entropy != nullptr;
+  const size_t per_token = want_entropy ? 32 : 24;
+  int max_splits = (int)(avail / (per_token * (size_t)T) > 4096 ? 4096 : avail / (per_token * (size_t)T));
+  while (max_splits >= 1 && fwd_layout(T, H, V, dtype, sms, max_splits, want_entropy).total > avail) --max_splits;
   if (max_splits < 1) return SAPO_ERR_STATIC_SCRATCH_EXCEEDED;
   void* scratch = nullptr;
   const int rc = static_scratch(&scratch);
@@ -648,8 +683,8 @@ extern "C" int sapo_policy_loss_bwd(const void* hidden, const void* W_head, int3
   float* partials = reinterpret_cast<float*>(ws + L.partials);
   // whole 128-token blocks of the panel that fit; a chunk never ends inside a block it cannot hold
   const int64_t rows_fit = ((int64_t)((workspace_bytes - L.fixed) / L.bytes_per_row) / BM) * BM;
-  const int64_t chunk_rows = rows_fit >= T ? T : rows_fit;
-  if (chunk_rows <= 0) return SAPO_ERR_WORKSPACE_TOO_SMALL;
+  if (rows_fit <= 0) return SAPO_ERR_WORKSPACE_TOO_SMALL;
+  const int64_t chunk_rows = rows_fit >= T ? T : equal_chunk_rows(T, rows_fit);   // equal chunks: no short last one
 
   // W as the K-major B operand of the logit recompute
   CUtensorMap map_w_kmajor;
@@ -663,10 +698,10 @@ extern "C" int sapo_policy_loss_bwd(const void* hidden, const void* W_head, int3
     if (!make_map(&map_h_kmajor, A0, H, tc, lda, BM)) return SAPO_ERR_CUDA;
     // dz panel: recompute logits tile by tile
     {
-      Sched sched = make_sched(tc, V, H, 0, /*m_fastest=*/true, /*tile_align=*/64);
+      Sched sched = make_sched(tc, V, H, 0, /*m_fastest=*/true, /*tile_align=*/64, FWD_BK);
       sched.n_cover = (int32_t)Vp;
       DzEpi::Params ep{ids + t0, lse + t0, gscale + t0, tc, V, nvt, panel};
-      int rc = launch_gemm<0, false, DzEpi>(map_h_kmajor, map_w_kmajor, sched, ep, status, st, SAPO_K_BWD_DZ);
+      int rc = launch_gemm<0, false, DzEpi, FWD_BK, FWD_STAGES>(map_h_kmajor, map_w_kmajor, sched, ep, status, st, SAPO_K_BWD_DZ);
       if (rc != SAPO_OK) return rc;
     }
     // dhidden[t0:t0+tc] = dz . W         (M = tokens, N = H, K = V)
@@ -780,11 +815,11 @@ extern "C" int sapo_policy_loss_bwd_active(const void* hidden, const void* W_hea
       return SAPO_ERR_CUDA;
     const int32_t* count = chunk_counts + c;
     {
-      Sched sched = make_sched(tc, V, H, 0, /*m_fastest=*/true, /*tile_align=*/64);
+      Sched sched = make_sched(tc, V, H, 0, /*m_fastest=*/true, /*tile_align=*/64, FWD_BK);
       sched.n_cover = (int32_t)Vp;
       sched.dyn_count = count; sched.dyn_dim = 1;
       DzEpi::Params ep{ids_act + t0, lse_act + t0, g_act + t0, tc, V, nvt, panel};
-      int rc = launch_gemm<0, false, DzEpi>(map_h_kmajor, map_w_kmajor, sched, ep, status, st, SAPO_K_BWD_DZ);
+      int rc = launch_gemm<0, false, DzEpi, FWD_BK, FWD_STAGES>(map_h_kmajor, map_w_kmajor, sched, ep, status, st, SAPO_K_BWD_DZ);
       if (rc != SAPO_OK) return rc;
     }
     {
@@ -842,7 +877,8 @@ extern "C" int sapo_policy_loss_fwd_bwd(const void* hidden, const void* W_head, 
     return SAPO_ERR_WORKSPACE_TOO_SMALL;
   const int64_t rows_fit =
       ((int64_t)((workspace_bytes - L.fixed - FUSED_CHUNK_SLACK) / L.bytes_per_row) / BM) * BM;
-  const int64_t chunk_rows = rows_fit >= T ? round_up<int64_t>(T, BM) : rows_fit;   // capacity, a multiple of 128
+  // capacity of a chunk, a multiple of 128; equal chunks, so that no short one is left at the end
+  const int64_t chunk_rows = rows_fit >= T ? round_up<int64_t>(T, BM) : equal_chunk_rows(T, rows_fit);
   const FusedChunk CL = fused_chunk(L, chunk_rows, H);
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   uint8_t* ws = static_cast<uint8_t*>(workspace);
@@ -854,6 +890,8 @@ extern "C" int sapo_policy_loss_fwd_bwd(const void* hidden, const void* W_head, 
   uint32_t* active_mask = reinterpret_cast<uint32_t*>(ws + L.mask);
   float* row_scale = reinterpret_cast<float*>(ws + CL.row_scale);
   float* ps = reinterpret_cast<float*>(ws + CL.ps);
+  float* pe = reinterpret_cast<float*>(ws + CL.pe);
+  const bool want_entropy = h_cfg->entropy != nullptr;
   __nv_bfloat16* hs = reinterpret_cast<__nv_bfloat16*>(ws + CL.hs);
   __nv_bfloat16* panel = reinterpret_cast<__nv_bfloat16*>(ws + CL.panel);
   const __nv_bfloat16* A = static_cast<const __nv_bfloat16*>(hidden);
@@ -880,17 +918,24 @@ extern "C" int sapo_policy_loss_fwd_bwd(const void* hidden, const void* W_head, 
     // 2. exponentials of the chunk -> panel, their sums per token and vocab split
     int n_splits = fwd_splits(tc, V, H, sms);
     if (n_splits > FUSED_MAX_SPLITS) n_splits = FUSED_MAX_SPLITS;
-    Sched fs = make_sched(tc, V, H, n_splits, /*m_fastest=*/true, /*tile_align=*/64);
+    Sched fs = make_sched(tc, V, H, n_splits, /*m_fastest=*/true, /*tile_align=*/64, FWD_BK);
     fs.n_cover = (int32_t)Vp;
     {
-      ExpEpi::Params ep{c2 + t0, ps, tc, V, nvt, panel};
-      int rc = launch_gemm<0, false, ExpEpi>(map_h_kmajor, map_w_kmajor, fs, ep, status, st, SAPO_K_FWD_EXP);
+      int rc;
+      if (want_entropy) {
+        ExpEpiT<true>::Params ep{c2 + t0, ps, pe, tc, V, nvt, panel};
+        rc = launch_gemm<0, false, ExpEpiT<true>, FWD_BK, FWD_STAGES>(map_h_kmajor, map_w_kmajor, fs, ep, status, st, SAPO_K_FWD_EXP);
+      } else {
+        ExpEpi::Params ep{c2 + t0, ps, nullptr, tc, V, nvt, panel};
+        rc = launch_gemm<0, false, ExpEpi, FWD_BK, FWD_STAGES>(map_h_kmajor, map_w_kmajor, fs, ep, status, st, SAPO_K_FWD_EXP);
+      }
       if (rc != SAPO_OK) return rc;
     }
     // 3. per-token loss terms, row scales, the chosen-token entries of the panel, scaled hidden rows
     {
       FusedTailArgs ta{};
       ta.ps = ps; ta.n_parts = 2 * fs.units_per_m; ta.t0 = t0; ta.tc = tc;
+      ta.pe = pe; ta.entropy = h_cfg->entropy;
       ta.zy = zy; ta.c2 = c2; ta.ids = ids; ta.V = V; ta.old_logp = old_logp; ta.adv = adv;
       ta.cu = cu_seqlens; ta.S = S; ta.T = T;
       ta.lo_edge = 1.f - h_cfg->eps_low; ta.hi_edge = 1.f + h_cfg->eps_high; ta.grad_scale = h_cfg->grad_scale;

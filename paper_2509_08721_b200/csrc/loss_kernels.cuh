@@ -32,6 +32,7 @@ split_bf16_kernel(const float* __restrict__ X, int64_t ld, int64_t R, int32_t H,
 
 struct TailArgs {
   const float* pm; const float* ps; const float* pz; int32_t n_splits; int64_t T;
+  const float* pe; float* entropy;     // optional: partial sums of 2^(x - m) z, and the per-token entropy
   const int32_t* ids; int32_t V; const float* old_logp; const float* adv; const int32_t* cu; int32_t S;
   float lo_edge, hi_edge, grad_scale;
   int32_t loss_agg; float kl_beta; const float* ref_logp;   // variants: token-level mean, KL penalty
@@ -93,13 +94,17 @@ __global__ void __launch_bounds__(256) loss_tail_kernel(TailArgs a) {
     for (int32_t t = t0 + threadIdx.x; t < t1; t += 256) {
       float M = -INFINITY;
       for (int i = 0; i < a.n_splits; ++i) M = fmaxf(M, a.pm[(int64_t)i * a.T + t]);
-      float sum = 0.f, zy = 0.f;
+      float sum = 0.f, zy = 0.f, sz = 0.f;
       for (int i = 0; i < a.n_splits; ++i) {
         const int64_t o = (int64_t)i * a.T + t;
-        sum += a.ps[o] * exp2f(a.pm[o] - M);
+        const float scale = exp2f(a.pm[o] - M);
+        sum += a.ps[o] * scale;
         zy += a.pz[o];
+        if (a.entropy != nullptr) sz += a.pe[o] * scale;
       }
       const float lse = (M + log2f(sum)) * LN2;
+      // entropy of the row's distribution: - sum_v p log p = lse - sum_v p z
+      if (a.entropy != nullptr) a.entropy[t] = lse - sz / sum;
       const int32_t y = a.ids[t];
       const bool bad_id = y < 0 || y >= a.V;
       if (bad_id) raise_status(a.status, SAPO_ST_BAD_TOKEN_ID);
@@ -132,6 +137,7 @@ __global__ void __launch_bounds__(256) loss_tail_kernel(TailArgs a) {
   for (int64_t i = (int64_t)blockIdx.x * 256 + threadIdx.x; i < n_out; i += (int64_t)gridDim.x * 256) {
     const int64_t t = i < lo ? i : hi + (i - lo);
     a.lse[t] = 0.f; a.logp[t] = 0.f; a.ratio[t] = 0.f; a.surr[t] = 0.f; a.gscale[t] = 0.f;
+    if (a.entropy != nullptr) a.entropy[t] = 0.f;
   }
 }
 
@@ -198,6 +204,7 @@ target_logit_kernel(const __nv_bfloat16* __restrict__ hidden, int64_t ldh, const
 
 struct FusedTailArgs {
   const float* ps; int32_t n_parts; int64_t t0, tc;        // partial sums [n_parts][tc] of this token chunk
+  const float* pe; float* entropy;                         // optional: partial sums of e z [n_parts][tc]; entropy [T]
   const float* zy; const float* c2;                        // [T]
   const int32_t* ids; int32_t V; const float* old_logp; const float* adv; const int32_t* cu; int32_t S;
   int64_t T; float lo_edge, hi_edge, grad_scale; int32_t loss_agg; float kl_beta; const float* ref_logp;
@@ -225,10 +232,16 @@ __global__ void __launch_bounds__(256) fused_tail_kernel(FusedTailArgs a) {
   const float n_scored = (float)(end_scored - first_scored);
   for (int64_t lr = warp; lr < a.tc; lr += n_warps) {
     const int64_t t = a.t0 + lr;
-    float part = 0.f;
-    for (int i = lane; i < a.n_parts; i += 32) part += a.ps[(int64_t)i * a.tc + lr];
+    float part = 0.f, part_z = 0.f;
+    for (int i = lane; i < a.n_parts; i += 32) {
+      part += a.ps[(int64_t)i * a.tc + lr];
+      if (a.entropy != nullptr) part_z += a.pe[(int64_t)i * a.tc + lr];
+    }
     #pragma unroll
-    for (int d = 16; d > 0; d >>= 1) part += __shfl_xor_sync(0xffffffffu, part, d);
+    for (int d = 16; d > 0; d >>= 1) {
+      part += __shfl_xor_sync(0xffffffffu, part, d);
+      part_z += __shfl_xor_sync(0xffffffffu, part_z, d);
+    }
     const float sum = part;
     // the sequence of this token: last s with cu[s] <= t; a token before the first or after the
     // last sequence (the caller passed its buffer capacity as T) is scored as masked
@@ -268,6 +281,7 @@ __global__ void __launch_bounds__(256) fused_tail_kernel(FusedTailArgs a) {
       if (bad_range && in_seq) raise_status(a.status, SAPO_ST_EXP_RANGE);
       if (bad_in) raise_status(a.status, SAPO_ST_NONFINITE_INPUT);
       a.lse[t] = lse; a.logp[t] = lp; a.ratio[t] = rho; a.surr[t] = u; a.gscale[t] = g; a.obj[t] = obj;
+      if (a.entropy != nullptr) a.entropy[t] = (bad_range || !in_seq) ? 0.f : lse - part_z / sum;
       a.row_scale[lr] = scale;
       if (scale != 0.f && a.active_mask != nullptr)
         atomicOr(&a.active_mask[lr >> 12], 1u << ((lr >> 7) & 31));

@@ -126,9 +126,22 @@ __global__ void __launch_bounds__(256) pack_copy_kernel(PackArgs a) {
   const int n4 = (int)(a.row_bytes >> 4);
   const bool two_at_once = vec && n4 <= 32 * ROW_VECS_PER_LANE;
   const int tpw = a.tokens_per_warp;
-  for (int64_t t0 = warp0 * tpw; t0 < a.max_tokens; t0 += n_warps * tpw) {
+  // Slots past the last packed token: mask 0, sequence -1 and an all-zero row, id and log-prob, so
+  // that the whole capacity can be scored without reading the token count back to the host.
+  for (int64_t t = T + warp0; t < a.max_tokens; t += n_warps) {
+    uint8_t* to = a.o_hid + t * a.row_bytes;
+    if (vec) {
+      uint4* t4 = reinterpret_cast<uint4*>(to);
+      for (int j = lane; j < n4; j += 32) t4[j] = make_uint4(0u, 0u, 0u, 0u);
+    } else {
+      uint16_t* t2 = reinterpret_cast<uint16_t*>(to);
+      for (int j = lane; j < (int)(a.row_bytes >> 1); j += 32) t2[j] = 0;
+    }
+    if (lane == 0) { a.o_ids[t] = 0; a.o_old[t] = 0.f; a.tok_seq[t] = -1; a.tok_mask[t] = 0; }
+  }
+  for (int64_t t0 = warp0 * tpw; t0 < T; t0 += n_warps * tpw) {
     int32_t s = 0;
-    if (t0 < T) {
+    {
       // first s with cu[s+1] > t0 (zero-length sequences share a start; take the one that owns t0)
       int32_t lo = 0, hi = S;
       while (lo < hi) {
@@ -157,28 +170,10 @@ __global__ void __launch_bounds__(256) pack_copy_kernel(PackArgs a) {
         a.tok_mask[t] = 1;
       }
     };
-    // a slot past the last packed token: mask 0 and an all-zero row, id and log-prob, so that the
-    // whole capacity can be scored without reading the token count back to the host
-    auto pad = [&](int64_t t) {
-      uint8_t* to = a.o_hid + t * a.row_bytes;
-      if (vec) {
-        uint4* t4 = reinterpret_cast<uint4*>(to);
-        for (int j = lane; j < n4; j += 32) t4[j] = make_uint4(0u, 0u, 0u, 0u);
-      } else {
-        uint16_t* t2 = reinterpret_cast<uint16_t*>(to);
-        for (int j = lane; j < (int)(a.row_bytes >> 1); j += 32) t2[j] = 0;
-      }
-      if (lane == 0) { a.o_ids[t] = 0; a.o_old[t] = 0.f; a.tok_seq[t] = -1; a.tok_mask[t] = 0; }
-    };
     for (int i = 0; i < tpw; i += 2) {
       const int64_t ta = t0 + i, tb = ta + 1;
-      if (ta >= a.max_tokens) break;
-      const bool have_a = ta < T, have_b = tb < T && tb < a.max_tokens;
-      if (!have_a) {
-        pad(ta);
-        if (tb < a.max_tokens) pad(tb);
-        continue;
-      }
+      if (ta >= T) break;
+      const bool have_b = tb < T;
       if (two_at_once) {
         const int64_t sa = locate(ta);
         const uint4* fa = reinterpret_cast<const uint4*>(a.hid[side] + sa * a.row_bytes);
@@ -201,16 +196,13 @@ __global__ void __launch_bounds__(256) pack_copy_kernel(PackArgs a) {
           #pragma unroll
           for (int q = 0; q < ROW_VECS_PER_LANE; ++q) if (lane + 32 * q < n4) ob[lane + 32 * q] = vb[q];
           finish(tb, sb);
-        } else if (tb < a.max_tokens) {
-          pad(tb);
         }
         continue;
       }
       // wide or unaligned rows: one token at a time
       for (int k = 0; k < 2; ++k) {
         const int64_t t = ta + k;
-        if (t >= a.max_tokens) break;
-        if (t >= T) { pad(t); continue; }
+        if (t >= T) break;
         const int64_t src = locate(t);
         const uint8_t* from = a.hid[side] + src * a.row_bytes;
         uint8_t* to = a.o_hid + t * a.row_bytes;

@@ -140,8 +140,10 @@ class Recipe:
     noise_sigma: float = 0.05
     eps_low: float = 0.2
     eps_high: float = 0.2
-    n_nodes: int = 2             # number of simulated nodes feeding the external buffer (+ self)
-    distractor_fraction: float = 0.25
+    n_nodes: int = 2             # simulated nodes (this one included); from 3 on the buffers are a swarm pool:
+                                 # the local buffer holds this node's Q x (I+J) rollouts, the external buffer
+                                 # the Q x (I+J) rollouts of each of the other n_nodes - 1 nodes, end to end
+    distractor_fraction: float = 0.25    # n_nodes == 2: share of unselected rollouts mixed into each buffer
 
 
 def config(number: int, *, ext_fraction: Optional[float] = None, length_div: int = 1) -> Recipe:
@@ -258,11 +260,18 @@ def make_batch(recipe: Recipe, seed: int, *, selections: Optional[List[Tuple[int
     for q, (i, j) in enumerate(per_q):
         seq_is_ext[group_offsets[q] + i:group_offsets[q + 1]] = 1
 
-    # ---- scatter the sequences into a local and an external buffer among distractors
-    def scatter(which: np.ndarray, pool_extra: int):
+    # ---- scatter the sequences into a local and an external buffer among rollouts that are not
+    # selected: a fixed share of distractors, or (swarm pool) whole node buffers of Q x (I+J)
+    # rollouts each, in which the selected ones sit at seeded uniform slots
+    pool = recipe.n_nodes >= 3
+    per_node = int(G.max()) * Q if Q > 0 else 0
+
+    def scatter(which: np.ndarray, n_node_buffers: int):
         n_sel = int(which.sum())
-        n_dis = int(np.ceil(recipe.distractor_fraction * max(n_sel, 1))) + pool_extra
-        n_all = n_sel + n_dis
+        if pool:
+            n_all = max(n_sel, n_node_buffers * per_node)
+        else:
+            n_all = n_sel + int(np.ceil(recipe.distractor_fraction * max(n_sel, 1)))
         slot_of = rng.permutation(n_all)[:n_sel]                 # buffer slot of each selected seq
         d_len = _draw_lengths(rng, recipe.length_law, n_all)
         d_rew = _draw_rewards(rng, recipe.reward_law, n_all)
@@ -285,9 +294,9 @@ def make_batch(recipe: Recipe, seed: int, *, selections: Optional[List[Tuple[int
         src[sel_seqs] = slot_of.astype(np.int32)
         return buf, src
 
-    local, src_l = scatter(seq_is_ext == 0, 0)
+    local, src_l = scatter(seq_is_ext == 0, 1)
     # the external buffer stands for the concatenated buffers of the other nodes
-    ext, src_e = scatter(seq_is_ext == 1, max(0, recipe.n_nodes - 2))
+    ext, src_e = scatter(seq_is_ext == 1, max(1, recipe.n_nodes - 1))
     seq_src = np.where(seq_is_ext == 1, src_e, src_l).astype(np.int32)
 
     qol = np.zeros(Q + 1, dtype=np.int32)

@@ -41,7 +41,7 @@ def test_host_side_helpers():
     assert B.sapo_workspace_bytes_min(B.WS_BWD, T, H, V, B.DTYPE_BF16) == 128 * V * 2 + k_split_scratch
     # single-pass call: the panel plus, per token, a scaled hidden row and a few floats
     fused = B.sapo_workspace_bytes(B.WS_FUSED, T, H, V, B.DTYPE_BF16)
-    assert T * (V + H) * 2 + k_split_scratch < fused < T * (V + H) * 2 + k_split_scratch + 2000 * T
+    assert T * (V + H) * 2 + k_split_scratch < fused < T * (V + H) * 2 + k_split_scratch + 3000 * T
     assert 0 < B.sapo_workspace_bytes_min(B.WS_FUSED, T, H, V, B.DTYPE_BF16) < fused // 10
     assert B.sapo_workspace_bytes(B.WS_FUSED, T, H, V, B.DTYPE_F32) == 0       # bf16 operands only
     assert B.sapo_workspace_bytes(B.WS_FWD, T, 12, V, B.DTYPE_BF16) == 0      # H % 8 != 0

@@ -81,7 +81,7 @@ def test_workload2_full_size(backward):
     assert np.array_equal(U.to_numpy(res.packed["hidden"])[:T], b.hidden)
     assert np.array_equal(U.to_numpy(res.packed["ids"])[:T], b.ids)
     assert np.array_equal(U.to_numpy(res.packed["cu_seqlens"])[:S + 1], b.cu_seqlens)
-    assert np.allclose(res.adv[:S].cpu().numpy(), adv, rtol=2e-7, atol=1e-9)
+    assert np.allclose(res.adv[:S].cpu().numpy(), adv, rtol=U.TOL_ADV_REL, atol=1e-9)
     out = {k: v[:T] for k, v in res.fwd.items() if k not in ("seq_surr", "loss")}
     U.check_forward(out, ref, adv, b.cu_seqlens, batch.eps_low, batch.eps_high)
     seq = res.fwd["seq_surr"][:S].cpu().numpy().astype(np.float64)
@@ -119,7 +119,7 @@ def test_workloads_3_to_5_full_size_sampled(number, ext_fraction, sample_tokens,
     scorer, res = run_scorer(batch, recipe, backward)
     assert np.array_equal(U.to_numpy(res.packed["ids"])[:T], b.ids)
     assert np.array_equal(U.to_numpy(res.packed["cu_seqlens"])[:S + 1], b.cu_seqlens)
-    assert np.allclose(res.adv[:S].cpu().numpy(), adv, rtol=2e-7, atol=1e-9)
+    assert np.allclose(res.adv[:S].cpu().numpy(), adv, rtol=U.TOL_ADV_REL, atol=1e-9)
 
     # sampled whole sequences (prefer ones with a non-zero advantage), scored one by one
     rng = np.random.default_rng(number)

@@ -50,6 +50,50 @@ def test_loss_variants_match_the_oracle(loss_agg, kl_beta):
     assert U.rel_fro(dW.cpu().numpy(), grads["dW"]) <= U.TOL_GRAD_FRO
 
 
+ENTROPY_SHAPES = [
+    # hidden, vocab, lengths: a ragged vocabulary tail, several vocab tiles and splits, a peaked head
+    (64, 1000, ("uniform", 1, 40), 0.02),
+    (328, 2500, ("uniform", 30, 120), 0.02),
+    (128, 20000, ("uniform", 50, 90), 0.2),
+]
+
+
+@pytest.mark.parametrize("H,V,lengths,w_std", ENTROPY_SHAPES, ids=["vocab_tail", "many_tiles", "peaked"])
+@pytest.mark.parametrize("fused", [False, True], ids=["separate_calls", "single_pass"])
+def test_per_token_entropy_matches_the_oracle(H, V, lengths, w_std, fused):
+    """The entropy of the policy's distribution at every position, a by-product of the forward
+    epilogue, against the oracle's -sum p log p at the log-prob tolerance; asking for it must not
+    change any other output."""
+    recipe = gen.Recipe("ent", gen.DTYPE_BF16, H, V, 4, 2, 2, lengths, ("bernoulli", 0.5))
+    batch = gen.make_batch(recipe, 71)
+    b = batch.built
+    if w_std != 0.02:                      # a head with a wide logit spread: low-entropy rows
+        batch.W = gen.f32_to_bf16_bits(gen.as_f32(batch.W) * np.float32(w_std / 0.02))
+    gen.install_old_logp(batch, U.oracle_current_logp(batch))
+    adv = np.linspace(-1.0, 1.0, batch.S).astype(np.float32)
+    ref_ent = orc.token_entropy(gen.as_f32(b.hidden), gen.as_f32(batch.W))
+    args = (U.to_torch(b.hidden), U.to_torch(batch.W), U.to_torch(b.ids), U.to_torch(b.old_logp),
+            U.to_torch(adv), U.to_torch(b.cu_seqlens), 0.2, 0.28)
+    T, S = batch.T, batch.S
+    ent = torch.full((T,), -1.0, device="cuda")
+    if fused:
+        plain = U.gpu_scores_fused(*args)
+        out = U.gpu_scores_fused(*args, entropy=ent)
+    else:
+        plain = U.gpu_scores(*args, want_bwd=False)
+        status = B.new_status()
+        out = B.alloc_fwd_outputs(T, S)
+        ws = torch.empty(B.sapo_workspace_bytes(B.WS_FWD, T, H, V, B.DTYPE_BF16), dtype=torch.uint8, device="cuda")
+        B.sapo_policy_loss_fwd(*args, 1.0, out, ws, status, entropy=ent)
+        torch.cuda.synchronize()
+        assert status.item() == 0
+    got = ent.cpu().numpy().astype(np.float64)
+    assert np.max(np.abs(got - ref_ent)) <= U.TOL_LOGP_ABS, np.max(np.abs(got - ref_ent))
+    assert got.min() >= -1e-4 and got.max() <= np.log(V) + 1e-4
+    for k in ("logp", "lse", "ratio", "surr", "gscale", "loss"):
+        assert torch.equal(out[k], plain[k]), k
+
+
 def test_kl_without_reference_is_rejected():
     x = torch.zeros(8, 16, dtype=torch.bfloat16, device="cuda")
     W = torch.zeros(16, 16, dtype=torch.bfloat16, device="cuda")

@@ -97,10 +97,10 @@ def test_advantages_match_oracle(ddof):
     torch.cuda.synchronize()
     assert status.item() == 0
     a = adv.cpu().numpy().astype(np.float64)
-    assert np.allclose(a, ref["adv"], rtol=2e-7, atol=1e-9)
+    assert np.allclose(a, ref["adv"], rtol=U.TOL_ADV_REL, atol=1e-9)
     assert np.all(a[go[5]:go[6]] == 0.0)
-    assert np.allclose(mean.cpu().numpy(), ref["mean"], rtol=2e-7, atol=1e-12)
-    assert np.allclose(std.cpu().numpy(), ref["std"], rtol=2e-7, atol=1e-12)
+    assert np.allclose(mean.cpu().numpy(), ref["mean"], rtol=U.TOL_ADV_REL, atol=1e-12)
+    assert np.allclose(std.cpu().numpy(), ref["std"], rtol=U.TOL_ADV_REL, atol=1e-12)
     for g in range(len(sizes)):
         assert abs(a[go[g]:go[g + 1]].sum()) < 1e-5
 
@@ -121,9 +121,44 @@ def test_advantages_with_many_questions_take_the_thread_per_question_path():
     B.sapo_group_advantages(U.to_torch(r), U.to_torch(go), eps, 0, adv, mean, std, status)
     torch.cuda.synchronize()
     assert status.item() == 0
-    assert np.allclose(adv.cpu().numpy(), ref["adv"], rtol=2e-7, atol=1e-9)
-    assert np.allclose(mean.cpu().numpy(), ref["mean"], rtol=2e-7, atol=1e-12)
-    assert np.allclose(std.cpu().numpy(), ref["std"], rtol=2e-7, atol=1e-12)
+    assert np.allclose(adv.cpu().numpy(), ref["adv"], rtol=U.TOL_ADV_REL, atol=1e-9)
+    assert np.allclose(mean.cpu().numpy(), ref["mean"], rtol=U.TOL_ADV_REL, atol=1e-12)
+    assert np.allclose(std.cpu().numpy(), ref["std"], rtol=U.TOL_ADV_REL, atol=1e-12)
+
+
+@pytest.mark.parametrize("warp_level", [False, True], ids=["thread_per_question", "warp_level"])
+@pytest.mark.parametrize("G", [8, 16])
+def test_advantages_stay_within_the_stated_ulps_whatever_the_offset(G, warp_level):
+    """The kernels keep their sums in compensated fp32.  Against the fp64 oracle: binary and
+    partial-credit rewards, real-valued rewards, and the same on top of a large common offset
+    (where an uncompensated fp32 mean would lose the deviations) all stay within 6 fp32 ulp."""
+    rng = np.random.default_rng(100 + G)
+    Q = 6000
+    go = (np.arange(Q + 1) * G).astype(np.int32)
+    base = np.concatenate([
+        rng.choice([0.0, 0.5, 1.0], size=(Q // 3, G)),
+        rng.normal(size=(Q // 3, G)),
+        rng.random(size=(Q - 2 * (Q // 3), G)) * 1e-3,
+    ]).astype(np.float32)
+    eps = float(np.float32(1e-6))
+    worst = 0.0
+    for offset in (0.0, 1000.0, -3.0e5):
+        r = (base + np.float32(offset)).astype(np.float32).reshape(-1)
+        ref = orc.group_advantages(r, go, adv_eps=eps, ddof=0)
+        adv = torch.empty(len(r), dtype=torch.float32, device="cuda")
+        std = torch.empty(Q, dtype=torch.float32, device="cuda")
+        status = B.new_status()
+        B.sapo_group_advantages(U.to_torch(r), U.to_torch(go), eps, 0, adv, None, std, status,
+                                warp_level=warp_level)
+        torch.cuda.synchronize()
+        assert status.item() == 0
+        a = adv.cpu().numpy().astype(np.float64)
+        big = np.abs(ref["adv"]) > 1e-3                     # ulps of values that are not rounding residue
+        ulp = np.abs(a - ref["adv"])[big] / np.spacing(np.abs(ref["adv"][big]).astype(np.float32))
+        worst = max(worst, float(ulp.max()))
+        assert np.allclose(a, ref["adv"], rtol=U.TOL_ADV_REL, atol=1e-9), (offset, float(ulp.max()))
+        assert np.allclose(std.cpu().numpy(), ref["std"], rtol=U.TOL_ADV_REL, atol=1e-12)
+    assert worst <= 6.5, worst                               # 6 ulp by the error analysis + the fp32 rounding of the result
 
 
 def test_advantages_flag_nonfinite_rewards():
@@ -160,7 +195,7 @@ def run_case(batch, eps_low=None, eps_high=None, grad_scale=1.0, bwd_ws=None, no
     out = U.gpu_scores(packed["hidden"], U.to_torch(batch.W), packed["ids"], packed["old_logp"], adv,
                        packed["cu_seqlens"], eps_low, eps_high, grad_scale, bwd_workspace_bytes=bwd_ws)
     assert out["status"] == 0 and status.item() == 0
-    assert np.allclose(adv.cpu().numpy(), a["adv"], rtol=2e-7, atol=1e-9)
+    assert np.allclose(adv.cpu().numpy(), a["adv"], rtol=U.TOL_ADV_REL, atol=1e-9)
     U.check_forward(out, ref, a["adv"], p["cu_seqlens"], eps_low, eps_high)
     seq = out["seq_surr"].cpu().numpy().astype(np.float64)
     assert np.max(np.abs(seq - ref["seq_surr"])) <= 1e-3 * (np.abs(a["adv"]).max() + 1e-30)

@@ -433,3 +433,36 @@ def test_generator_recipes_have_the_stated_shapes():
     assert np.array_equal(gen.bf16_bits_to_f32(gen.f32_to_bf16_bits(x)), x)
     ties = np.array([1.00390625, 1.01171875], np.float32)          # halfway: round to even
     assert gen.bf16_bits_to_f32(gen.f32_to_bf16_bits(ties)).tolist() == [1.0, 1.015625]
+
+
+# ------------------------------------------------------------------------------ entropy
+def test_entropy_pins():
+    """token_entropy against what fixes it: a uniform head gives ln V; scipy's entropy of the
+    row distributions; the two-outcome closed form -(p ln p + q ln q); the identity
+    H = lse - sum_v p z; and the bound 0 <= H <= ln V."""
+    from scipy.special import softmax
+    from scipy.stats import entropy as scipy_entropy
+    rng = np.random.default_rng(17)
+    T, H, V = 9, 6, 23
+    h = rng.normal(size=(T, H))
+    W = rng.normal(size=(V, H))
+    ent = orc.token_entropy(h, W)
+    # uniform head
+    assert np.allclose(orc.token_entropy(h, np.zeros((V, H))), np.log(V), rtol=0, atol=1e-13)
+    # library routine on the row distributions
+    z = h @ W.T
+    assert np.allclose(ent, scipy_entropy(softmax(z, axis=1), axis=1), rtol=1e-12, atol=1e-13)
+    # identity with the log-sum-exp the oracle also reports
+    lp = orc.token_logprobs(h, W, np.zeros(T, dtype=np.int64))
+    assert np.allclose(ent, lp["lse"] - (softmax(z, axis=1) * z).sum(axis=1), rtol=1e-12, atol=1e-12)
+    assert np.all(ent >= 0) and np.all(ent <= np.log(V) + 1e-12)
+    # two outcomes: logits (a, 0) -> p = sigmoid(a)
+    a = np.array([[-3.0], [0.0], [0.7], [5.0]])
+    W2 = np.array([[1.0], [0.0]])
+    p = 1.0 / (1.0 + np.exp(-a[:, 0]))
+    closed = -(p * np.log(p) + (1 - p) * np.log(1 - p))
+    assert np.allclose(orc.token_entropy(a, W2), closed, rtol=1e-13, atol=1e-15)
+    # a peaked row has (almost) no entropy; shifting every logit of a row changes nothing
+    assert orc.token_entropy(np.array([[50.0]]), W2)[0] < 1e-19
+    u = rng.normal(size=H)
+    assert np.allclose(orc.token_entropy(h, W + u[None, :]), ent, rtol=1e-11, atol=1e-12)
