@@ -35,6 +35,12 @@
  *     hidden / W_head / dhidden / dW_head / workspace must be 16-byte aligned and the
  *     leading dimensions, in bytes, multiples of 16.
  *   - There is no CPU fallback: without a CUDA device every call returns SAPO_ERR_CUDA.
+ *   - Threads.  The calls keep a few per-device values they look up on first use (the driver's
+ *     tensor-map encoder, the SM count, the shared-memory opt-in and resident CTA pairs of each
+ *     kernel, the address of the built-in scratch of sapo_policy_loss_fwd_static) without locks.
+ *     Make the first call of each entry point on each device from one thread (a warm-up step does
+ *     it); after that, calls from several threads are safe as long as each uses its own stream,
+ *     workspace and outputs.  sapo_timing_* and sapo_launch_count are for one thread only.
  */
 #ifndef SAPO_H_
 #define SAPO_H_
@@ -77,6 +83,7 @@ extern "C" {
 #define SAPO_WS_BWD 1
 #define SAPO_WS_BWD_ACTIVE 2
 #define SAPO_WS_FUSED 3
+#define SAPO_WS_OUT_BF16 0x100   /* OR into `which`: the gradients will be asked for in bf16 */
 
 /* A rollout store: n_rollouts completions laid end to end (Section 3.1: a node's answers
  * to its questions; Section 3.2: the tuples other nodes broadcast).
@@ -222,20 +229,25 @@ int sapo_policy_loss_fwd(const void* hidden, const void* W_head, int32_t dtype,
 
 /* Algorithm 1 "Policy update" (gradient of the loss above through the LM head):
  *   dz[t,v]      = gscale[t] * ([v == ids[t]] - exp(z[t,v] - lse[t]))
- *   dhidden[t,:] = sum_v dz[t,v] W_head[v,:]        float32 [T, H]
- *   dW_head[v,:] = sum_t dz[t,v] hidden[t,:]        float32 [V, H]
+ *   dhidden[t,:] = sum_v dz[t,v] W_head[v,:]        [T, H] of out_dtype
+ *   dW_head[v,:] = sum_t dz[t,v] hidden[t,:]        [V, H] of out_dtype
  * Logit tiles are recomputed on the tensor cores; dz is rounded to bf16 and kept in a
  * bounded panel inside `workspace` (token chunks x vocab padded to 128, stored as 16 KB tiles
  * of 128 tokens x 64 vocab entries), from which two tensor-core contractions form dhidden and
  * dW_head.  accumulate_dW != 0 adds into dW_head instead of
  * overwriting it.  lse and gscale come from sapo_policy_loss_fwd.  For SAPO_DTYPE_F32 the
  * operands are rounded to bf16.
+ * out_dtype: SAPO_DTYPE_F32, or SAPO_DTYPE_BF16 for gradients that feed a bf16 backward pass and
+ * optimiser: contiguous [T, H] / [V, H] of that type, 16-byte aligned; sums are always formed in
+ * fp32 and rounded once (when the panel holds fewer than T tokens, or accumulate_dW is set,
+ * dW_head is summed in an fp32 copy inside `workspace` and rounded, or added to the caller's
+ * values and rounded, at the end: ask sapo_workspace_bytes for SAPO_WS_BWD | SAPO_WS_OUT_BF16).
  * workspace: sapo_workspace_bytes(SAPO_WS_BWD, ...) is the preferred size; any size down to
  * the one for 128 tokens works (smaller panels mean more passes over dW_head). */
 int sapo_policy_loss_bwd(const void* hidden, const void* W_head, int32_t dtype,
                          int64_t T, int32_t H, int32_t V, int64_t ld_hidden, int64_t ld_W,
                          const int32_t* ids, const float* lse, const float* gscale,
-                         float* dhidden, float* dW_head, int32_t accumulate_dW,
+                         void* dhidden, void* dW_head, int32_t out_dtype, int32_t accumulate_dW,
                          void* workspace, size_t workspace_bytes,
                          int32_t* status, void* stream);
 
@@ -252,7 +264,7 @@ int sapo_policy_loss_bwd(const void* hidden, const void* W_head, int32_t dtype,
 int sapo_policy_loss_bwd_active(const void* hidden, const void* W_head, int32_t dtype,
                                 int64_t T, int32_t H, int32_t V, int64_t ld_hidden, int64_t ld_W,
                                 const int32_t* ids, const float* lse, const float* gscale,
-                                float* dhidden, float* dW_head, int32_t accumulate_dW,
+                                void* dhidden, void* dW_head, int32_t out_dtype, int32_t accumulate_dW,
                                 int32_t* n_active_out,
                                 void* workspace, size_t workspace_bytes,
                                 int32_t* status, void* stream);
@@ -286,7 +298,7 @@ int sapo_policy_loss_fwd_bwd(const void* hidden, const void* W_head, int32_t dty
                              const int32_t* cu_seqlens, int32_t S, const sapo_loss_cfg* h_cfg,
                              float* logp, float* lse, float* ratio, float* surr, float* gscale,
                              float* seq_surr, float* loss,
-                             float* dhidden, float* dW_head, int32_t accumulate_dW,
+                             void* dhidden, void* dW_head, int32_t out_dtype, int32_t accumulate_dW,
                              void* workspace, size_t workspace_bytes,
                              int32_t* status, void* stream);
 
@@ -319,7 +331,8 @@ int sapo_adam_step(float* master, float* m, float* v, const float* grad, void* w
                    float lr, float beta1, float beta2, float eps, void* stream);
 
 /* Bytes of scratch the forward (SAPO_WS_FWD), backward (SAPO_WS_BWD, SAPO_WS_BWD_ACTIVE) or
- * fused (SAPO_WS_FUSED) call wants for these sizes.  Returns 0 for invalid arguments. */
+ * fused (SAPO_WS_FUSED) call wants for these sizes; OR SAPO_WS_OUT_BF16 into `which` for a call
+ * with bf16 gradient outputs.  Returns 0 for invalid arguments. */
 size_t sapo_workspace_bytes(int32_t which, int64_t T, int32_t H, int32_t V, int32_t dtype);
 
 /* Smallest backward or fused workspace that still works (one 128-token panel). */
@@ -382,6 +395,14 @@ int sapo_policy_loss_fwd_static(const void* hidden, const void* W_head, int32_t 
 int sapo_timing_enable(int32_t on);
 int sapo_timing_read(float* h_ms, int32_t* h_launches);
 int64_t sapo_launch_count(void);
+
+/* The library's in-kernel waits (on the barriers between the copy, tensor-core and epilogue
+ * roles of the GEMM kernels) are bounded: a wait that runs out makes the kernel set
+ * SAPO_ST_WAIT_TIMEOUT, let its copies in flight land, free its tensor memory and return, so the
+ * context stays usable.  This call (no counterpart in the paper) exercises exactly that code on a
+ * barrier nobody arrives at: one thread waits limit_clocks SM clocks (at most 10^8, about 50 ms),
+ * then sets the bit in *status.  For tests of a caller's error handling. */
+int sapo_debug_wait_timeout(int64_t limit_clocks, int32_t* status, void* stream);
 
 /* Text for a return code. */
 const char* sapo_status_string(int32_t code);

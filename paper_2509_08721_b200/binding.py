@@ -20,6 +20,7 @@ WS_FWD = 0
 WS_BWD = 1
 WS_BWD_ACTIVE = 2
 WS_FUSED = 3
+WS_OUT_BF16 = 0x100      # OR into the workspace kind: gradients in bf16
 
 ST_BITS = {
     0x01: "TOKEN_OVERFLOW", 0x02: "SEQ_OVERFLOW", 0x04: "BAD_INDEX", 0x08: "EMPTY_SEQUENCE",
@@ -31,7 +32,7 @@ EXPORTS = ("sapo_pack_rollouts", "sapo_group_advantages", "sapo_policy_loss_fwd"
            "sapo_policy_loss_bwd", "sapo_workspace_bytes", "sapo_workspace_bytes_min",
            "sapo_status_string", "sapo_timing_enable", "sapo_timing_read", "sapo_launch_count",
            "sapo_policy_loss_fwd_static", "sapo_policy_loss_bwd_active", "sapo_policy_loss_fwd_bwd",
-           "sapo_select_external", "sapo_group_advantages_warp",
+           "sapo_select_external", "sapo_group_advantages_warp", "sapo_debug_wait_timeout",
            "sapo_select_workspace_bytes", "sapo_adam_step")
 STATIC_SCRATCH_BYTES = 4 * 1024 * 1024
 KERNEL_NAMES = ("pack_scan", "pack_copy", "group_adv", "split_bf16", "fwd_gemm", "loss_tail",
@@ -96,13 +97,13 @@ def load() -> C.CDLL:
                                                 C.POINTER(LossCfgC), vp, vp, vp, vp, vp, vp, vp, vp, vp]
     lib.sapo_policy_loss_bwd.restype = C.c_int
     lib.sapo_policy_loss_bwd.argtypes = [vp, vp, i32, i64, i32, i32, i64, i64, vp, vp, vp, vp, vp,
-                                         i32, vp, sz, vp, vp]
+                                         i32, i32, vp, sz, vp, vp]
     lib.sapo_policy_loss_bwd_active.restype = C.c_int
     lib.sapo_policy_loss_bwd_active.argtypes = [vp, vp, i32, i64, i32, i32, i64, i64, vp, vp, vp, vp, vp,
-                                                i32, vp, vp, sz, vp, vp]
+                                                i32, i32, vp, vp, sz, vp, vp]
     lib.sapo_policy_loss_fwd_bwd.restype = C.c_int
     lib.sapo_policy_loss_fwd_bwd.argtypes = [vp, vp, i32, i64, i32, i32, i64, i64, vp, vp, vp, vp, i32,
-                                             C.POINTER(LossCfgC), vp, vp, vp, vp, vp, vp, vp, vp, vp, i32,
+                                             C.POINTER(LossCfgC), vp, vp, vp, vp, vp, vp, vp, vp, vp, i32, i32,
                                              vp, sz, vp, vp]
     lib.sapo_select_external.restype = C.c_int
     lib.sapo_select_external.argtypes = [vp, vp, i32, i32, C.c_uint64, vp, vp, vp, vp, sz, vp]
@@ -118,6 +119,8 @@ def load() -> C.CDLL:
     lib.sapo_timing_enable.argtypes = [i32]
     lib.sapo_timing_read.restype = C.c_int
     lib.sapo_timing_read.argtypes = [C.POINTER(C.c_float), C.POINTER(C.c_int32)]
+    lib.sapo_debug_wait_timeout.restype = C.c_int
+    lib.sapo_debug_wait_timeout.argtypes = [i64, vp, vp]
     lib.sapo_launch_count.restype = C.c_int64
     lib.sapo_launch_count.argtypes = []
     lib.sapo_status_string.restype = C.c_char_p
@@ -148,6 +151,12 @@ def _stream() -> int:
     return torch.cuda.current_stream().cuda_stream
 
 
+def _out_dtype_code(dhidden: torch.Tensor, dW_head: torch.Tensor) -> int:
+    if dhidden.dtype != dW_head.dtype:
+        raise SapoError("dhidden and dW_head must have the same element type")
+    return _dtype_code(dhidden)
+
+
 def _dtype_code(t: torch.Tensor) -> int:
     if t.dtype == torch.bfloat16:
         return DTYPE_BF16
@@ -171,6 +180,12 @@ def sapo_timing_read() -> Dict[str, Dict[str, float]]:
 
 def sapo_launch_count() -> int:
     return int(load().sapo_launch_count())
+
+
+def sapo_debug_wait_timeout(limit_clocks: int, status: torch.Tensor) -> None:
+    """Make a bounded in-kernel wait run out (sets WAIT_TIMEOUT in `status`); see sapo.h."""
+    _require_cuda()
+    _check(load().sapo_debug_wait_timeout(int(limit_clocks), _p(status), _stream()), "sapo_debug_wait_timeout")
 
 
 def decode_status(word: int):
@@ -315,7 +330,8 @@ def sapo_policy_loss_bwd(hidden: torch.Tensor, W_head: torch.Tensor, ids: torch.
     H, V = int(hidden.shape[1]), int(W_head.shape[0])
     rc = load().sapo_policy_loss_bwd(
         _p(hidden), _p(W_head), _dtype_code(hidden), T, H, V, hidden.stride(0), W_head.stride(0),
-        _p(ids), _p(lse), _p(gscale), _p(dhidden), _p(dW_head), 1 if accumulate_dW else 0,
+        _p(ids), _p(lse), _p(gscale), _p(dhidden), _p(dW_head), _out_dtype_code(dhidden, dW_head),
+        1 if accumulate_dW else 0,
         _p(workspace), workspace.numel() * workspace.element_size(), _p(status), _stream())
     _check(rc, "sapo_policy_loss_bwd")
 
@@ -331,7 +347,8 @@ def sapo_policy_loss_bwd_active(hidden: torch.Tensor, W_head: torch.Tensor, ids:
     H, V = int(hidden.shape[1]), int(W_head.shape[0])
     rc = load().sapo_policy_loss_bwd_active(
         _p(hidden), _p(W_head), _dtype_code(hidden), T, H, V, hidden.stride(0), W_head.stride(0),
-        _p(ids), _p(lse), _p(gscale), _p(dhidden), _p(dW_head), 1 if accumulate_dW else 0, _p(n_active),
+        _p(ids), _p(lse), _p(gscale), _p(dhidden), _p(dW_head), _out_dtype_code(dhidden, dW_head),
+        1 if accumulate_dW else 0, _p(n_active),
         _p(workspace), workspace.numel() * workspace.element_size(), _p(status), _stream())
     _check(rc, "sapo_policy_loss_bwd_active")
 
@@ -354,7 +371,8 @@ def sapo_policy_loss_fwd_bwd(hidden: torch.Tensor, W_head: torch.Tensor, ids: to
         _p(hidden), _p(W_head), _dtype_code(hidden), T, H, V, hidden.stride(0), W_head.stride(0),
         _p(ids), _p(old_logp), _p(adv), _p(cu_seqlens), S, C.byref(cfg),
         _p(out["logp"]), _p(out["lse"]), _p(out["ratio"]), _p(out["surr"]), _p(out["gscale"]),
-        _p(out.get("seq_surr")), _p(out["loss"]), _p(dhidden), _p(dW_head), 1 if accumulate_dW else 0,
+        _p(out.get("seq_surr")), _p(out["loss"]), _p(dhidden), _p(dW_head), _out_dtype_code(dhidden, dW_head),
+        1 if accumulate_dW else 0,
         _p(workspace), workspace.numel() * workspace.element_size(), _p(status), _stream())
     _check(rc, "sapo_policy_loss_fwd_bwd")
 

@@ -69,7 +69,7 @@ active_assign_kernel(const float* __restrict__ gscale, const float* __restrict__
                      const int32_t* __restrict__ ids, int64_t T, const int32_t* __restrict__ block_base,
                      int32_t* __restrict__ act_idx, int32_t* __restrict__ ids_act,
                      float* __restrict__ lse_act, float* __restrict__ g_act,
-                     float* __restrict__ dhidden, int32_t H) {
+                     void* __restrict__ dhidden, int64_t row_bytes) {
   __shared__ int32_t warp_n[COMPACT_BLOCK / 32];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int64_t t = (int64_t)blockIdx.x * COMPACT_BLOCK + threadIdx.x;
@@ -92,8 +92,8 @@ active_assign_kernel(const float* __restrict__ gscale, const float* __restrict__
     const int64_t tt = (int64_t)blockIdx.x * COMPACT_BLOCK + warp * 32 + i;
     if (tt >= T) break;
     if ((m >> i) & 1u) continue;
-    float4* row = reinterpret_cast<float4*>(dhidden + tt * (int64_t)H);
-    for (int j = lane; j < H / 4; j += 32) row[j] = make_float4(0.f, 0.f, 0.f, 0.f);
+    uint4* row = reinterpret_cast<uint4*>(static_cast<uint8_t*>(dhidden) + tt * row_bytes);    // a multiple of 16 bytes
+    for (int j = lane; j < (int)(row_bytes >> 4); j += 32) row[j] = make_uint4(0u, 0u, 0u, 0u);
   }
 }
 

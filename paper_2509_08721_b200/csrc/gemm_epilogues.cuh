@@ -232,15 +232,34 @@ struct ExpEpiT {
 };
 using ExpEpi = ExpEpiT<false>;
 
-// Plain fp32 output tile, optionally added to what is already there.
+// 32 floats -> 16 packed bf16 pairs, each value scaled first
+__device__ __forceinline__ void pack_bf16_32(const float (&v)[32], float scale, uint32_t (&w)[16]) {
+  #pragma unroll
+  for (int j = 0; j < 16; ++j) {
+    __nv_bfloat162 b2 = __floats2bfloat162_rn(scale * v[2 * j], scale * v[2 * j + 1]);
+    w[j] = *reinterpret_cast<uint32_t*>(&b2);
+  }
+}
+// 8 bf16 (one 16-byte vector) + 8 floats -> 8 bf16
+__device__ __forceinline__ uint4 add_bf16x8(uint4 c, const float* x) {
+  __nv_bfloat162* pc = reinterpret_cast<__nv_bfloat162*>(&c);
+  #pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    const float2 f = __bfloat1622float2(pc[j]);
+    pc[j] = __floats2bfloat162_rn(f.x + x[2 * j], f.y + x[2 * j + 1]);
+  }
+  return c;
+}
+
+// Plain output tile (fp32, or bf16 when out_bf16 is set), optionally added to what is already there.
 struct StoreEpi {
   static constexpr bool PANEL = false;
   static constexpr bool STREAMK = true;
   // row_map (optional): output row of each accumulator row (rows of compacted tokens go back
   // to their packed positions)
   // row_scale (optional): factor applied to each accumulator row before it is stored
-  struct Params { float* C; int64_t ldc; int64_t M; int32_t N; int32_t accumulate; float* partials;
-                  const int32_t* row_map; const float* row_scale; };
+  struct Params { void* C; int64_t ldc; int64_t M; int32_t N; int32_t accumulate; float* partials;
+                  const int32_t* row_map; const float* row_scale; int32_t out_bf16; };
   template <class P> __device__ static void set_dynamic(P& p, const Sched& s) {
     if (s.dyn_dim == 1) p.M = *s.dyn_count;
   }
@@ -268,7 +287,23 @@ struct StoreEpi {
       return;
     }
     if (!valid) return;
-    float4* dst = reinterpret_cast<float4*>(p.C + row * p.ldc + col0);
+    if (p.out_bf16) {                      // N is a multiple of 8: 16-byte vectors of 8 bf16
+      uint4* dst = reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(p.C) + row * p.ldc + col0);
+      #pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        if (col0 + 8 * q < p.N) {
+          float x[8];
+          #pragma unroll
+          for (int j = 0; j < 8; ++j) x[j] = scale * v[8 * q + j];
+          uint4 o;
+          if (p.accumulate) o = add_bf16x8(dst[q], x);
+          else              o = add_bf16x8(make_uint4(0u, 0u, 0u, 0u), x);
+          dst[q] = o;
+        }
+      }
+      return;
+    }
+    float4* dst = reinterpret_cast<float4*>(reinterpret_cast<float*>(p.C) + row * p.ldc + col0);
     #pragma unroll
     for (int q = 0; q < 8; ++q) {
       if (col0 + 4 * q < p.N) {          // N is a multiple of 4
@@ -313,8 +348,18 @@ streamk_fixup_kernel(const Sched s_arg, const StoreEpi::Params p_arg, int pairs)
       const float4 v = *reinterpret_cast<const float4*>(src + (size_t)j * s.sk_tiles * part_floats);
       sum.x += v.x; sum.y += v.y; sum.z += v.z; sum.w += v.w;
     }
-    float4* dst = reinterpret_cast<float4*>(p.C + row * p.ldc + n0 + 4 * c4);
     float4 o = make_float4(scale * sum.x, scale * sum.y, scale * sum.z, scale * sum.w);
+    if (p.out_bf16) {
+      __nv_bfloat162* dst = reinterpret_cast<__nv_bfloat162*>(reinterpret_cast<__nv_bfloat16*>(p.C) + row * p.ldc + n0 + 4 * c4);
+      if (p.accumulate) {
+        const float2 c0 = __bfloat1622float2(dst[0]), c1 = __bfloat1622float2(dst[1]);
+        o.x += c0.x; o.y += c0.y; o.z += c1.x; o.w += c1.y;
+      }
+      dst[0] = __floats2bfloat162_rn(o.x, o.y);
+      dst[1] = __floats2bfloat162_rn(o.z, o.w);
+      continue;
+    }
+    float4* dst = reinterpret_cast<float4*>(reinterpret_cast<float*>(p.C) + row * p.ldc + n0 + 4 * c4);
     if (p.accumulate) { const float4 c = *dst; o.x += c.x; o.y += c.y; o.z += c.z; o.w += c.w; }
     *dst = o;
   }

@@ -45,6 +45,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
   uint64_t* acc_empty = bars + 2 * NSTAGE + 2; // [2] epilogue -> MMA    (even CTA's are used)
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * NSTAGE + 4);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  uint64_t* drain = bars + 2 * NSTAGE + 5;   // MMA thread only: "all my MMAs have retired" after a wait ran out
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   constexpr bool A_MN = (A_KIND & 1) != 0;
@@ -54,6 +55,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
   if (threadIdx.x == 0) {
     for (int i = 0; i < NSTAGE; ++i) { mbar_init(&full[i], 1); mbar_init(&empty[i], 1); }
     for (int i = 0; i < 2; ++i) { mbar_init(&acc_full[i], 1); mbar_init(&acc_empty[i], 16); }
+    mbar_init(drain, 1);
     *abort_flag = 0;
     fence_mbar_init();
     prefetch_tensormap(&map_a);
@@ -99,7 +101,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
                               : nb * sched.tile_n + (int)rank * half + (mn ? 64 * bi : 0);
         const int k_off = mn ? 0 : 64 * bi;                // K-major boxes split the stage's K depth
         for (int kb = kb0; kb < kb1; ++kb) {
-          if (!SAPO_TIMED(0, mbar_wait(&empty[stage], phase ^ 1, abort_flag))) { ok = false; break; }
+          if (!SAPO_TIMED(0, mbar_wait(&empty[stage], phase ^ 1, abort_flag, sched.wait_limit))) { ok = false; break; }
           if (rank == 0 && lane == 0) mbar_arrive_expect_tx(&full[stage], tx);
           if (mine) {
             uint8_t* dst = smem + dst_off + stage * (is_a ? A_ST : B_ST);
@@ -136,11 +138,11 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
     while (ok && work.next(pmb, un, n_begin, n_end, kb0, kb1, slot)) {
       for (int nb = n_begin; ok && nb < n_end; ++nb) {
         const uint32_t idesc = make_idesc_bf16(PAIR_M, tile_n_eff(sched, nb), A_MN, B_MN);
-        if (!SAPO_TIMED(2, mbar_wait(&acc_empty[acc], acc_phase ^ 1, abort_flag))) { ok = false; break; }
+        if (!SAPO_TIMED(2, mbar_wait(&acc_empty[acc], acc_phase ^ 1, abort_flag, sched.wait_limit))) { ok = false; break; }
         fence_after_sync();
         const uint32_t d_tmem = tmem_base + acc * BN;
         for (int kb = kb0; kb < kb1; ++kb) {
-          if (!SAPO_TIMED(1, mbar_wait(&full[stage], phase, abort_flag))) { ok = false; break; }
+          if (!SAPO_TIMED(1, mbar_wait(&full[stage], phase, abort_flag, sched.wait_limit))) { ok = false; break; }
           fence_after_sync();
           const uint32_t a_addr = smem_u32(smem_a + stage * A_ST);
           const uint32_t b_addr = smem_u32(smem_b + stage * B_ST);
@@ -167,6 +169,11 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
         if (++acc == 2) { acc = 0; acc_phase ^= 1; }
       }
     }
+    if (!ok) {
+      // a wait ran out: no MMA of this pair may still be running when tensor memory is freed
+      mma_commit_pair(map_to_cta(smem_u32(drain), 0));
+      for (int spin = 0; spin < (1 << 22) && !mbar_try_wait(drain, 0); ++spin) {}
+    }
 #ifdef SAPO_WAIT_STATS
     atomicMax(&g_wait_stats[sched.stats_id & 3][7], (unsigned long long)(clock64() - role_t0));
 #endif
@@ -188,7 +195,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
       epi.begin_unit(ep, 2 * pmb + (int)rank, r);
       if constexpr (Epi::STREAMK) epi.set_dest(ep, slot, (int)rank, r, n_begin * sched.tile_n, sched.part_ld);
       for (int nb = n_begin; ok && nb < n_end; ++nb) {
-        if (!SAPO_TIMED(3, mbar_wait(&acc_full[acc], acc_phase, abort_flag))) { ok = false; break; }
+        if (!SAPO_TIMED(3, mbar_wait(&acc_full[acc], acc_phase, abort_flag, sched.wait_limit))) { ok = false; break; }
         fence_after_sync();
         const uint32_t t_addr = tmem_base + (static_cast<uint32_t>(quad * 32) << 16) + acc * BN;
         const int n0 = nb * sched.tile_n;
@@ -270,7 +277,7 @@ static_assert(GEMM2_SMEM_BYTES <= 232448, "more shared memory than a CTA can hav
 template <int A_KIND>
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
 umma_gemm2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
-                  const __grid_constant__ CUtensorMap map_c,   // the fp32 output, boxes of 32 columns x 128 rows
+                  const __grid_constant__ CUtensorMap map_c,   // the output (fp32 or bf16), boxes of 32 columns x 128 rows
                   const Sched sched_arg, const StoreEpi::Params ep_arg, int32_t* status) {
   static_assert(A_KIND == 2 || A_KIND == 3, "panel operands only");
   SAPO_CLOCK_BEGIN
@@ -287,6 +294,7 @@ umma_gemm2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
   uint64_t* acc_empty = bars + 2 * STAGES2 + 1; // epilogue -> MMA         (even CTA's is used)
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * STAGES2 + 2);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  uint64_t* drain = bars + 2 * STAGES2 + 3;   // MMA thread only, after a wait ran out (see umma_gemm_kernel)
   uint32_t* mask_s = reinterpret_cast<uint32_t*>(reinterpret_cast<uint8_t*>(bars) + 256);
   uint8_t* out_staging = reinterpret_cast<uint8_t*>(bars) + GEMM2_TAIL_BYTES;
   // the mask only matters if some block of the chunk is clear: decided once, by every thread alike
@@ -326,6 +334,7 @@ umma_gemm2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
   if (threadIdx.x == 0) {
     for (int i = 0; i < STAGES2; ++i) { mbar_init(&full[i], 1); mbar_init(&empty[i], 1); }
     mbar_init(acc_full, 1); mbar_init(acc_empty, 16);
+    mbar_init(drain, 1);
     *abort_flag = 0;
     fence_mbar_init();
     prefetch_tensormap(&map_a);
@@ -363,7 +372,7 @@ umma_gemm2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
       uint32_t word = 0;
       for (int kb = kb0; kb < kb1; ++kb) {
         if (!stage_active(kb, kb0, word)) continue;
-        if (!mbar_wait(&empty[stage], phase ^ 1, abort_flag)) { ok = false; break; }
+        if (!mbar_wait(&empty[stage], phase ^ 1, abort_flag, sched.wait_limit)) { ok = false; break; }
         if (rank == 0 && lane == 0) mbar_arrive_expect_tx(&full[stage], tx);
         if (mine) {
           const uint32_t bar = full0_addr + stage * 8;
@@ -399,14 +408,14 @@ umma_gemm2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
     WorkList work(sched, pair, num_pairs);
     int pmb, un, n_begin, n_end, kb0, kb1, slot;
     while (ok && work.next(pmb, un, n_begin, n_end, kb0, kb1, slot)) {
-      if (!mbar_wait(acc_empty, acc_phase ^ 1, abort_flag)) { ok = false; break; }
+      if (!mbar_wait(acc_empty, acc_phase ^ 1, abort_flag, sched.wait_limit)) { ok = false; break; }
       fence_after_sync();
       if (A_KIND == 2 && !rows_active(pmb)) kb1 = kb0;
       bool first = true;                       // the first stage that runs overwrites the accumulators
       uint32_t word = 0;
       for (int kb = kb0; kb < kb1; ++kb) {
         if (!stage_active(kb, kb0, word)) continue;
-        if (!mbar_wait(&full[stage], phase, abort_flag)) { ok = false; break; }
+        if (!mbar_wait(&full[stage], phase, abort_flag, sched.wait_limit)) { ok = false; break; }
         fence_after_sync();
         const uint32_t a_addr = smem_u32(smem_a + stage * A2_STAGE_BYTES);
         const uint32_t b_addr = smem_u32(smem_b + stage * B2_STAGE_BYTES);
@@ -429,6 +438,10 @@ umma_gemm2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
         mma_commit_pair(acc_full_addr[1]);
       }
       acc_phase ^= 1;
+    }
+    if (!ok) {
+      mma_commit_pair(map_to_cta(smem_u32(drain), 0));
+      for (int spin = 0; spin < (1 << 22) && !mbar_try_wait(drain, 0); ++spin) {}
     }
   } else if (warp >= 2) {
     // ------------------------------------------------------------ epilogue (8 warps, both CTAs)
@@ -454,7 +467,7 @@ umma_gemm2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
         any = false;
         for (int b = kb0 >> 1; b <= (kb1 - 1) >> 1 && !any; ++b) any = blk_active(b);
       }
-      if (!mbar_wait(acc_full, acc_phase, abort_flag)) { ok = false; break; }
+      if (!mbar_wait(acc_full, acc_phase, abort_flag, sched.wait_limit)) { ok = false; break; }
       fence_after_sync();
       const uint32_t t_addr = tmem_base + (static_cast<uint32_t>(quad * 32) << 16) + j * BN;
       const int chunks = (tn + 31) >> 5;
@@ -472,11 +485,21 @@ umma_gemm2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
         if (col0 >= ep.N || row0 >= ep.M) return;      // nothing of this box lies inside the output
         if (elected) bulk_wait_read_all();
         named_barrier_sync(1 + j, 128);
-        #pragma unroll
-        for (int q = 0; q < 8; ++q)
-          st_shared_v4(buf + r * 128 + ((q ^ (r & 7)) << 4),
-                       __float_as_uint(epi.scale * v[4 * q]), __float_as_uint(epi.scale * v[4 * q + 1]),
-                       __float_as_uint(epi.scale * v[4 * q + 2]), __float_as_uint(epi.scale * v[4 * q + 3]));
+        if (ep.out_bf16) {
+          // bf16 output: rows of 64 bytes in the 64-byte swizzle (16-byte unit q of row r sits at
+          // unit q ^ ((r >> 1) & 3)), as the tensor map of a bf16 output expects
+          uint32_t w[16];
+          pack_bf16_32(v, epi.scale, w);
+          #pragma unroll
+          for (int q = 0; q < 4; ++q)
+            st_shared_v4(buf + r * 64 + ((q ^ ((r >> 1) & 3)) << 4), w[4 * q], w[4 * q + 1], w[4 * q + 2], w[4 * q + 3]);
+        } else {
+          #pragma unroll
+          for (int q = 0; q < 8; ++q)
+            st_shared_v4(buf + r * 128 + ((q ^ (r & 7)) << 4),
+                         __float_as_uint(epi.scale * v[4 * q]), __float_as_uint(epi.scale * v[4 * q + 1]),
+                         __float_as_uint(epi.scale * v[4 * q + 2]), __float_as_uint(epi.scale * v[4 * q + 3]));
+        }
         fence_proxy_async_smem();
         named_barrier_sync(1 + j, 128);
         if (elected) {

@@ -65,6 +65,7 @@ struct Sched {
   int32_t dyn_dim;
   int32_t skip_if_empty;  // dyn_dim 2 only: a zero-length contraction launches no work at all
   int32_t stats_id;   // row of the wait-cycle counters this launch adds to (instrumented builds)
+  long long wait_limit;   // SM clocks after which a barrier wait gives up (SAPO_ST_WAIT_TIMEOUT)
 };
 
 constexpr int PARTIAL_FLOATS = PAIR_M * BN;   // one partial accumulator tile: 256 x 256 fp32

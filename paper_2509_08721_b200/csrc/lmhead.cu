@@ -60,15 +60,17 @@ static bool make_map(CUtensorMap* map, const void* base, int64_t inner, int64_t 
 
 // fp32 matrix [outer, inner] with `ld` elements between rows, for stores of 32-column x 128-row
 // boxes (128 bytes wide, 128-byte swizzle); elements outside the matrix are not written.
-static bool make_map_f32_out(CUtensorMap* map, const float* base, int64_t inner, int64_t outer, int64_t ld) {
+// (bf16 outputs: the same boxes are 64 bytes wide and take the 64-byte swizzle)
+static bool make_map_out(CUtensorMap* map, const void* base, bool bf16, int64_t inner, int64_t outer, int64_t ld) {
   EncodeTiledFn fn = encode_fn();
   if (fn == nullptr || inner <= 0 || outer <= 0) return false;
   cuuint64_t dims[2] = {(cuuint64_t)inner, (cuuint64_t)outer};
-  cuuint64_t strides[1] = {(cuuint64_t)ld * 4};
+  cuuint64_t strides[1] = {(cuuint64_t)ld * (bf16 ? 2 : 4)};
   cuuint32_t box[2] = {32u, 128u};
   cuuint32_t estr[2] = {1u, 1u};
-  return fn(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<float*>(base), dims, strides, box, estr,
-            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+  return fn(map, bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2,
+            const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+            bf16 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
@@ -97,6 +99,7 @@ static Sched make_sched(int64_t M, int64_t N, int64_t K, int n_splits, bool m_fa
   s.k_split_ok = 0; s.dyn_count = nullptr; s.dyn_dim = 0; s.skip_if_empty = 0;
   s.part_ld = BN; s.max_parts = MAX_PARTS_SCRATCH; s.min_part_k = 16;
   s.active_mask = nullptr; s.mask_words = 0; s.mask_dim = 0;
+  s.wait_limit = WAIT_LIMIT_CLOCKS;
   return s;
 }
 
@@ -215,7 +218,7 @@ template <int A_KIND>
 static int launch_gemm_wide(const CUtensorMap& ma, const CUtensorMap& mb, const Sched& sched,
                             const StoreEpi::Params& ep, int32_t* status, cudaStream_t st, int kernel_id) {
   CUtensorMap mc;
-  if (!make_map_f32_out(&mc, ep.C, ep.N, ep.M, ep.ldc)) return SAPO_ERR_CUDA;
+  if (!make_map_out(&mc, ep.C, ep.out_bf16 != 0, ep.N, ep.M, ep.ldc)) return SAPO_ERR_CUDA;
   auto kern = umma_gemm2_kernel<A_KIND>;
   static int max_pairs_of[MAX_DEVICES] = {0};   // as in launch_gemm: per device, found on first use
   const int dev = current_device();
@@ -267,11 +270,11 @@ static int launch_gemm_wide(const CUtensorMap& ma, const CUtensorMap& mb, const 
 // X is hidden (or its row-scaled copy), [tc, ldx].  Wide tiles when H allows.
 static int launch_grad_gemms(const __nv_bfloat16* panel, int64_t panel_rows, int32_t nvt,
                              const __nv_bfloat16* W, int64_t ldw, const __nv_bfloat16* X, int64_t ldx,
-                             int64_t tc, int32_t H, int32_t V, int64_t Vp, float* dhidden,
-                             const float* row_scale, float* dW_head, int accumulate, float* partials,
+                             int64_t tc, int32_t H, int32_t V, int64_t Vp, void* dhidden, bool dh_bf16,
+                             const float* row_scale, void* dW_head, bool dw_bf16, int accumulate, float* partials,
                              const uint32_t* active_mask, int32_t* status, cudaStream_t st) {
-  StoreEpi::Params ep_h{dhidden, H, tc, H, 0, partials, nullptr, row_scale};
-  StoreEpi::Params ep_w{dW_head, H, V, H, accumulate, partials, nullptr, nullptr};
+  StoreEpi::Params ep_h{dhidden, H, tc, H, 0, partials, nullptr, row_scale, dh_bf16 ? 1 : 0};
+  StoreEpi::Params ep_w{dW_head, H, V, H, accumulate, partials, nullptr, nullptr, dw_bf16 ? 1 : 0};
   if (use_wide_tiles(H)) {
     CUtensorMap map_p_tile, map_p_half, map_w64, map_x64;
     if (!make_map(&map_p_tile, panel, 64, panel_rows, 64, BM) || !make_map(&map_p_half, panel, 64, panel_rows, 64, 64) ||
@@ -340,10 +343,13 @@ static FwdLayout fwd_layout(int64_t T, int32_t H, int32_t V, int32_t dtype, int 
   return L;
 }
 
-struct BwdLayout { size_t a_hi, b_hi, partials, panel, fixed; size_t bytes_per_row; };
-static BwdLayout bwd_layout(int64_t T, int32_t H, int32_t V, int32_t dtype) {
+// out_bf16: room for an fp32 copy of dW_head, in which the token chunks are summed before the
+// result is rounded to bf16 once
+struct BwdLayout { size_t a_hi, b_hi, partials, dw_acc, panel, fixed; size_t bytes_per_row; };
+static BwdLayout bwd_layout(int64_t T, int32_t H, int32_t V, int32_t dtype, bool out_bf16 = false) {
   BwdLayout L{};
   size_t off = 0;
+  if (out_bf16) { L.dw_acc = off; off += round_up<size_t>((size_t)V * H * 4, 256); }
   if (dtype == SAPO_DTYPE_F32) {
     L.a_hi = off; off += round_up<size_t>((size_t)T * H * 2, 256);
     L.b_hi = off; off += round_up<size_t>((size_t)V * H * 2, 256);
@@ -374,11 +380,12 @@ static int64_t preferred_panel_rows(int64_t T) {
 // needs (row scales, partial sums, the scaled copy of hidden), the K-split scratch, the
 // per-sequence sums when the caller does not want them, and the panel of exponentials.
 constexpr int FUSED_MAX_SPLITS = 160;
-struct FusedLayout { size_t zy, c2, obj, seq, mask, partials, fixed; size_t bytes_per_row; };
-static FusedLayout fused_layout(int64_t T, int32_t H, int32_t V, int32_t S) {
+struct FusedLayout { size_t zy, c2, obj, seq, mask, partials, dw_acc, fixed; size_t bytes_per_row; };
+static FusedLayout fused_layout(int64_t T, int32_t H, int32_t V, int32_t S, bool out_bf16 = false) {
   FusedLayout L{};
   size_t off = 0;
   auto take = [&](size_t bytes) { const size_t at = off; off += round_up<size_t>(bytes, 256); return at; };
+  if (out_bf16) L.dw_acc = take((size_t)V * H * 4);
   L.zy = take((size_t)T * 4);
   L.c2 = take((size_t)T * 4);
   L.obj = take((size_t)T * 4);
@@ -426,6 +433,27 @@ static ActiveLayout active_layout(int64_t T, int32_t H) {
   return L;
 }
 
+// dst (bf16) = src (fp32), or dst + src when adding: the one rounding of a dW_head that was summed
+// over token chunks in fp32.  n is a multiple of 8.
+__global__ void __launch_bounds__(256)
+round_to_bf16_kernel(const float* __restrict__ src, __nv_bfloat16* __restrict__ dst, int64_t n, int add) {
+  for (int64_t i = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) * 8; i < n; i += (int64_t)gridDim.x * blockDim.x * 8) {
+    const float4 a = *reinterpret_cast<const float4*>(src + i), b = *reinterpret_cast<const float4*>(src + i + 4);
+    const float x[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
+    uint4* d = reinterpret_cast<uint4*>(dst + i);
+    *d = add_bf16x8(add ? *d : make_uint4(0u, 0u, 0u, 0u), x);
+  }
+}
+static int launch_round_to_bf16(const float* src, void* dst, int64_t n, int add, cudaStream_t st) {
+  int64_t blocks = ceil_div<int64_t>(n / 8, 256);
+  const int64_t cap = (int64_t)sm_count() * 8;
+  if (blocks > cap) blocks = cap;
+  if (blocks <= 0) return SAPO_OK;
+  KernelScope scope(SAPO_K_STREAMK_FIXUP, st);
+  round_to_bf16_kernel<<<(int)blocks, 256, 0, st>>>(src, static_cast<__nv_bfloat16*>(dst), n, add);
+  return check_launch();
+}
+
 // chunk_counts[c] = active tokens that fall into chunk c of `chunk_rows` compacted rows
 __global__ void chunk_counts_kernel(const int32_t* n_active, int64_t chunk_rows, int32_t n_chunks,
                                     int32_t* chunk_counts) {
@@ -462,6 +490,8 @@ static int fwd_check_args(const void* hidden, const void* W_head, int32_t dtype,
 // =============================================================================== C ABI
 extern "C" size_t sapo_workspace_bytes(int32_t which, int64_t T, int32_t H, int32_t V, int32_t dtype) {
   using namespace sapo;
+  const bool out_bf16 = (which & SAPO_WS_OUT_BF16) != 0;
+  which &= ~SAPO_WS_OUT_BF16;
   if (!shapes_ok(T, H, V) || (dtype != SAPO_DTYPE_BF16 && dtype != SAPO_DTYPE_F32)) return 0;
   if (which == SAPO_WS_FWD) {
     int sms = sm_count();
@@ -470,11 +500,11 @@ extern "C" size_t sapo_workspace_bytes(int32_t which, int64_t T, int32_t H, int3
   }
   if (which == SAPO_WS_FUSED) {
     if (dtype != SAPO_DTYPE_BF16) return 0;
-    const FusedLayout L = fused_layout(T, H, V, /*S=*/(int32_t)(T < 0x7fffffff ? T : 0x7fffffff));
+    const FusedLayout L = fused_layout(T, H, V, /*S=*/(int32_t)(T < 0x7fffffff ? T : 0x7fffffff), out_bf16);
     return L.fixed + FUSED_CHUNK_SLACK + (size_t)preferred_panel_rows(T) * L.bytes_per_row;
   }
   if (which == SAPO_WS_BWD || which == SAPO_WS_BWD_ACTIVE) {
-    const BwdLayout L = bwd_layout(T, H, V, dtype);
+    const BwdLayout L = bwd_layout(T, H, V, dtype, out_bf16);
     const size_t extra = which == SAPO_WS_BWD_ACTIVE ? active_layout(T, H).total : 0;
     return extra + L.fixed + (size_t)preferred_panel_rows(T) * L.bytes_per_row;
   }
@@ -483,14 +513,17 @@ extern "C" size_t sapo_workspace_bytes(int32_t which, int64_t T, int32_t H, int3
 
 extern "C" size_t sapo_workspace_bytes_min(int32_t which, int64_t T, int32_t H, int32_t V, int32_t dtype) {
   using namespace sapo;
-  if (which != SAPO_WS_BWD && which != SAPO_WS_FUSED) return sapo_workspace_bytes(which, T, H, V, dtype);
+  const bool out_bf16 = (which & SAPO_WS_OUT_BF16) != 0;
+  if ((which & ~SAPO_WS_OUT_BF16) != SAPO_WS_BWD && (which & ~SAPO_WS_OUT_BF16) != SAPO_WS_FUSED)
+    return sapo_workspace_bytes(which, T, H, V, dtype);
+  which &= ~SAPO_WS_OUT_BF16;
   if (!shapes_ok(T, H, V) || (dtype != SAPO_DTYPE_BF16 && dtype != SAPO_DTYPE_F32)) return 0;
   if (which == SAPO_WS_FUSED) {
     if (dtype != SAPO_DTYPE_BF16) return 0;
-    const FusedLayout L = fused_layout(T, H, V, (int32_t)(T < 0x7fffffff ? T : 0x7fffffff));
+    const FusedLayout L = fused_layout(T, H, V, (int32_t)(T < 0x7fffffff ? T : 0x7fffffff), out_bf16);
     return L.fixed + FUSED_CHUNK_SLACK + (size_t)BM * L.bytes_per_row;
   }
-  const BwdLayout L = bwd_layout(T, H, V, dtype);
+  const BwdLayout L = bwd_layout(T, H, V, dtype, out_bf16);
   return L.fixed + (size_t)BM * L.bytes_per_row;
 }
 
@@ -647,20 +680,22 @@ extern "C" int sapo_policy_loss_fwd_static(const void* hidden, const void* W_hea
 extern "C" int sapo_policy_loss_bwd(const void* hidden, const void* W_head, int32_t dtype,
                                     int64_t T, int32_t H, int32_t V, int64_t ld_hidden, int64_t ld_W,
                                     const int32_t* ids, const float* lse, const float* gscale,
-                                    float* dhidden, float* dW_head, int32_t accumulate_dW,
+                                    void* dhidden, void* dW_head, int32_t out_dtype, int32_t accumulate_dW,
                                     void* workspace, size_t workspace_bytes,
                                     int32_t* status, void* stream) {
   using namespace sapo;
   if (!hidden || !W_head || !ids || !lse || !gscale || !dhidden || !dW_head || !workspace || !status)
     return SAPO_ERR_INVALID_ARG;
   if (dtype != SAPO_DTYPE_BF16 && dtype != SAPO_DTYPE_F32) return SAPO_ERR_INVALID_ARG;
+  if (out_dtype != SAPO_DTYPE_BF16 && out_dtype != SAPO_DTYPE_F32) return SAPO_ERR_INVALID_ARG;
+  const bool out_bf16 = out_dtype == SAPO_DTYPE_BF16;
   if (T < 1 || H < 1 || V < 1 || ld_hidden < H || ld_W < H) return SAPO_ERR_INVALID_ARG;
   if (!shapes_ok(T, H, V)) return SAPO_ERR_UNSUPPORTED_SHAPE;
   const int esz = dtype == SAPO_DTYPE_BF16 ? 2 : 4;
   if (!aligned16(hidden) || !aligned16(W_head) || !aligned16(workspace) || !aligned16(dhidden) ||
       !aligned16(dW_head) || (ld_hidden * esz) % 16 || (ld_W * esz) % 16)
     return SAPO_ERR_INVALID_ARG;
-  const BwdLayout L = bwd_layout(T, H, V, dtype);
+  const BwdLayout L = bwd_layout(T, H, V, dtype, out_bf16);
   if (workspace_bytes < L.fixed + (size_t)BM * L.bytes_per_row) return SAPO_ERR_WORKSPACE_TOO_SMALL;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   uint8_t* ws = static_cast<uint8_t*>(workspace);
@@ -685,6 +720,11 @@ extern "C" int sapo_policy_loss_bwd(const void* hidden, const void* W_head, int3
   const int64_t rows_fit = ((int64_t)((workspace_bytes - L.fixed) / L.bytes_per_row) / BM) * BM;
   if (rows_fit <= 0) return SAPO_ERR_WORKSPACE_TOO_SMALL;
   const int64_t chunk_rows = rows_fit >= T ? T : equal_chunk_rows(T, rows_fit);   // equal chunks: no short last one
+  // a bf16 dW_head that is summed over several chunks, or added to what the caller holds, is formed
+  // in fp32 scratch and rounded once at the end
+  const bool dw_via_acc = out_bf16 && (chunk_rows < T || accumulate_dW);
+  float* dw_acc = reinterpret_cast<float*>(ws + L.dw_acc);
+  const size_t out_esz = out_bf16 ? 2 : 4;
 
   // W as the K-major B operand of the logit recompute
   CUtensorMap map_w_kmajor;
@@ -707,10 +747,13 @@ extern "C" int sapo_policy_loss_bwd(const void* hidden, const void* W_head, int3
     // dhidden[t0:t0+tc] = dz . W         (M = tokens, N = H, K = V)
     // dW (+)= dz^T . hidden               (M = V, N = H, K = tokens)
     const int rc = launch_grad_gemms(panel, panel_rows, nvt, B, ldb, A0, lda, tc, H, V, Vp,
-                                     dhidden + t0 * (int64_t)H, nullptr, dW_head,
-                                     (t0 > 0 || accumulate_dW) ? 1 : 0, partials, nullptr, status, st);
+                                     static_cast<uint8_t*>(dhidden) + (size_t)t0 * H * out_esz, out_bf16, nullptr,
+                                     dw_via_acc ? (void*)dw_acc : dW_head, out_bf16 && !dw_via_acc,
+                                     dw_via_acc ? (t0 > 0 ? 1 : 0) : ((t0 > 0 || accumulate_dW) ? 1 : 0),
+                                     partials, nullptr, status, st);
     if (rc != SAPO_OK) return rc;
   }
+  if (dw_via_acc) return launch_round_to_bf16(dw_acc, dW_head, (int64_t)V * H, accumulate_dW ? 1 : 0, st);
   return SAPO_OK;
 }
 
@@ -721,7 +764,7 @@ extern "C" int sapo_policy_loss_bwd(const void* hidden, const void* W_head, int3
 extern "C" int sapo_policy_loss_bwd_active(const void* hidden, const void* W_head, int32_t dtype,
                                            int64_t T, int32_t H, int32_t V, int64_t ld_hidden, int64_t ld_W,
                                            const int32_t* ids, const float* lse, const float* gscale,
-                                           float* dhidden, float* dW_head, int32_t accumulate_dW,
+                                           void* dhidden, void* dW_head, int32_t out_dtype, int32_t accumulate_dW,
                                            int32_t* n_active_out,
                                            void* workspace, size_t workspace_bytes,
                                            int32_t* status, void* stream) {
@@ -735,8 +778,10 @@ extern "C" int sapo_policy_loss_bwd_active(const void* hidden, const void* W_hea
   if (!aligned16(hidden) || !aligned16(W_head) || !aligned16(workspace) || !aligned16(dhidden) ||
       !aligned16(dW_head) || (ld_hidden * esz) % 16 || (ld_W * esz) % 16)
     return SAPO_ERR_INVALID_ARG;
+  if (out_dtype != SAPO_DTYPE_BF16 && out_dtype != SAPO_DTYPE_F32) return SAPO_ERR_INVALID_ARG;
+  const bool out_bf16 = out_dtype == SAPO_DTYPE_BF16;
   const ActiveLayout AL = active_layout(T, H);
-  const BwdLayout L = bwd_layout(T, H, V, dtype);
+  const BwdLayout L = bwd_layout(T, H, V, dtype, out_bf16);
   if (workspace_bytes < AL.total + L.fixed + (size_t)BM * L.bytes_per_row) return SAPO_ERR_WORKSPACE_TOO_SMALL;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   uint8_t* ws0 = static_cast<uint8_t*>(workspace);
@@ -772,6 +817,8 @@ extern "C" int sapo_policy_loss_bwd_active(const void* hidden, const void* W_hea
   if (chunk_rows <= 0) return SAPO_ERR_WORKSPACE_TOO_SMALL;
   const int64_t n_chunks = ceil_div<int64_t>(T, chunk_rows);
   if (n_chunks > MAX_ACTIVE_CHUNKS) return SAPO_ERR_WORKSPACE_TOO_SMALL;
+  const bool dw_via_acc = out_bf16 && (n_chunks > 1 || accumulate_dW);   // summed in fp32 scratch, rounded once at the end
+  float* dw_acc = reinterpret_cast<float*>(ws + L.dw_acc);
 
   // 1. which tokens take part, in order; compacted copies of what the GEMMs read per token
   const int sms = sm_count();
@@ -785,7 +832,7 @@ extern "C" int sapo_policy_loss_bwd_active(const void* hidden, const void* W_hea
   {
     KernelScope scope(SAPO_K_COMPACT, st);
     active_assign_kernel<<<n_blocks, COMPACT_BLOCK, 0, st>>>(gscale, lse, ids, T, counts, act_idx, ids_act,
-                                                             lse_act, g_act, dhidden, H);
+                                                             lse_act, g_act, dhidden, (int64_t)H * (out_bf16 ? 2 : 4));
   }
   {
     KernelScope scope(SAPO_K_COMPACT, st);
@@ -826,20 +873,22 @@ extern "C" int sapo_policy_loss_bwd_active(const void* hidden, const void* W_hea
       Sched sched = make_sched(tc, H, Vp, 0, /*m_fastest=*/false);
       sched.panel_nvt = nvt;
       sched.dyn_count = count; sched.dyn_dim = 1;
-      StoreEpi::Params ep{dhidden, H, tc, H, 0, partials, act_idx + t0, nullptr};   // rows go back to their tokens
+      StoreEpi::Params ep{dhidden, H, tc, H, 0, partials, act_idx + t0, nullptr, out_bf16 ? 1 : 0};   // rows go back to their tokens
       int rc = launch_gemm<2, true, StoreEpi>(map_p_two, map_w_mn, sched, ep, status, st, SAPO_K_BWD_DH);
       if (rc != SAPO_OK) return rc;
     }
     {
-      const int acc = (c > 0 || accumulate_dW) ? 1 : 0;
+      const int acc = dw_via_acc ? (c > 0 ? 1 : 0) : ((c > 0 || accumulate_dW) ? 1 : 0);
       Sched sched = make_sched(V, H, tc, 0, /*m_fastest=*/false);
       sched.panel_nvt = nvt;
       sched.dyn_count = count; sched.dyn_dim = 2; sched.skip_if_empty = acc;
-      StoreEpi::Params ep{dW_head, H, V, H, acc, partials, nullptr, nullptr};
+      StoreEpi::Params ep{dw_via_acc ? (void*)dw_acc : dW_head, H, V, H, acc, partials, nullptr, nullptr,
+                          (out_bf16 && !dw_via_acc) ? 1 : 0};
       int rc = launch_gemm<3, true, StoreEpi>(map_p_tile, map_h_mn, sched, ep, status, st, SAPO_K_BWD_DW);
       if (rc != SAPO_OK) return rc;
     }
   }
+  if (dw_via_acc) return launch_round_to_bf16(dw_acc, dW_head, (int64_t)V * H, accumulate_dW ? 1 : 0, st);
   return SAPO_OK;
 }
 
@@ -852,7 +901,7 @@ extern "C" int sapo_policy_loss_fwd_bwd(const void* hidden, const void* W_head, 
                                         const int32_t* cu_seqlens, int32_t S, const sapo_loss_cfg* h_cfg,
                                         float* logp, float* lse, float* ratio, float* surr, float* gscale,
                                         float* seq_surr, float* loss,
-                                        float* dhidden, float* dW_head, int32_t accumulate_dW,
+                                        void* dhidden, void* dW_head, int32_t out_dtype, int32_t accumulate_dW,
                                         void* workspace, size_t workspace_bytes,
                                         int32_t* status, void* stream) {
   using namespace sapo;
@@ -872,7 +921,9 @@ extern "C" int sapo_policy_loss_fwd_bwd(const void* hidden, const void* W_head, 
     return SAPO_ERR_INVALID_ARG;
   const int sms = sm_count();
   if (sms <= 0) return SAPO_ERR_CUDA;
-  const FusedLayout L = fused_layout(T, H, V, (int32_t)(T < 0x7fffffff ? T : 0x7fffffff));
+  if (out_dtype != SAPO_DTYPE_BF16 && out_dtype != SAPO_DTYPE_F32) return SAPO_ERR_INVALID_ARG;
+  const bool out_bf16 = out_dtype == SAPO_DTYPE_BF16;
+  const FusedLayout L = fused_layout(T, H, V, (int32_t)(T < 0x7fffffff ? T : 0x7fffffff), out_bf16);
   if (workspace_bytes < L.fixed + FUSED_CHUNK_SLACK + (size_t)BM * L.bytes_per_row)
     return SAPO_ERR_WORKSPACE_TOO_SMALL;
   const int64_t rows_fit =
@@ -882,6 +933,11 @@ extern "C" int sapo_policy_loss_fwd_bwd(const void* hidden, const void* W_head, 
   const FusedChunk CL = fused_chunk(L, chunk_rows, H);
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   uint8_t* ws = static_cast<uint8_t*>(workspace);
+  // a bf16 dW_head that is summed over several chunks, or added to what the caller holds, is formed
+  // in fp32 scratch and rounded once at the end
+  const bool dw_via_acc = out_bf16 && (chunk_rows < T || accumulate_dW);
+  float* dw_acc = reinterpret_cast<float*>(ws + L.dw_acc);
+  const size_t out_esz = out_bf16 ? 2 : 4;
   float* zy = reinterpret_cast<float*>(ws + L.zy);
   float* c2 = reinterpret_cast<float*>(ws + L.c2);
   float* obj = reinterpret_cast<float*>(ws + L.obj);
@@ -955,8 +1011,14 @@ extern "C" int sapo_policy_loss_fwd_bwd(const void* hidden, const void* W_head, 
     // 4. dhidden[t0:t0+tc] = a_t (e' . W)     (M = tokens, N = H, K = V)
     // 5. dW (+)= e'^T . (a_t h_t)            (M = V, N = H, K = tokens)
     const int rc = launch_grad_gemms(panel, panel_rows, nvt, B, ld_W, hs, H, tc, H, V, Vp,
-                                     dhidden + t0 * (int64_t)H, row_scale, dW_head,
-                                     (t0 > 0 || accumulate_dW) ? 1 : 0, partials, active_mask, status, st);
+                                     static_cast<uint8_t*>(dhidden) + (size_t)t0 * H * out_esz, out_bf16, row_scale,
+                                     dw_via_acc ? (void*)dw_acc : dW_head, out_bf16 && !dw_via_acc,
+                                     dw_via_acc ? (t0 > 0 ? 1 : 0) : ((t0 > 0 || accumulate_dW) ? 1 : 0),
+                                     partials, active_mask, status, st);
+    if (rc != SAPO_OK) return rc;
+  }
+  if (dw_via_acc) {
+    const int rc = launch_round_to_bf16(dw_acc, dW_head, (int64_t)V * H, accumulate_dW ? 1 : 0, st);
     if (rc != SAPO_OK) return rc;
   }
   // 6. per-sequence means and the loss
@@ -964,6 +1026,24 @@ extern "C" int sapo_policy_loss_fwd_bwd(const void* hidden, const void* W_head, 
   { KernelScope scope(SAPO_K_LOSS_TAIL, st); seq_mean_kernel<<<seq_blocks, 256, 0, st>>>(obj, cu_seqlens, S, T, seq_out, status); }
   { KernelScope scope(SAPO_K_LOSS_FINAL, st); loss_final_kernel<<<1, 256, 0, st>>>(seq_out, cu_seqlens, S, T, h_cfg->loss_agg, loss); }
   return check_launch();
+}
+
+// ------------------------------------------------------------------------------------------
+// The bounded wait, made to run out on purpose: one thread waits on a barrier nobody arrives at.
+namespace sapo {
+__global__ void wait_timeout_probe_kernel(long long limit_clocks, int32_t* status) {
+  __shared__ uint64_t bar;
+  __shared__ int abort_flag;
+  if (threadIdx.x == 0) { mbar_init(&bar, 1); abort_flag = 0; fence_mbar_init(); }
+  __syncthreads();
+  if (threadIdx.x == 0 && !mbar_wait(&bar, 0, &abort_flag, limit_clocks)) raise_status(status, SAPO_ST_WAIT_TIMEOUT);
+}
+}  // namespace sapo
+
+extern "C" int sapo_debug_wait_timeout(int64_t limit_clocks, int32_t* status, void* stream) {
+  if (!status || limit_clocks < 0 || limit_clocks > 100000000) return SAPO_ERR_INVALID_ARG;   // at most ~50 ms
+  sapo::wait_timeout_probe_kernel<<<1, 32, 0, static_cast<cudaStream_t>(stream)>>>((long long)limit_clocks, status);
+  return sapo::check_launch();
 }
 
 #ifdef SAPO_WAIT_STATS

@@ -40,17 +40,18 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
   return ok != 0;
 }
 
-// Wait for a barrier phase, giving up after about two seconds of SM clocks or as soon as
-// another role of the CTA has given up (abort_flag in shared memory).  Returns false then.
+// Wait for a barrier phase, giving up after `limit` SM clocks (by default about two seconds) or
+// as soon as another role of the CTA has given up (abort_flag in shared memory).  Returns false then.
 constexpr long long WAIT_LIMIT_CLOCKS = 4000000000LL;
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
+                                          long long limit = WAIT_LIMIT_CLOCKS) {
   if (mbar_try_wait(bar, parity)) return true;
   const long long t0 = clock64();
   uint32_t it = 0;
   while (!mbar_try_wait(bar, parity)) {
     if ((++it & 0xFF) == 0) {
       if (*abort_flag) return false;
-      if (clock64() - t0 > WAIT_LIMIT_CLOCKS) { *abort_flag = 1; return false; }
+      if (clock64() - t0 > limit) { *abort_flag = 1; return false; }
     }
   }
   return true;
@@ -212,14 +213,15 @@ __device__ __forceinline__ bool mbar_try_wait_cluster(uint64_t* bar, uint32_t pa
   return ok != 0;
 }
 // Bounded wait on a barrier of this CTA that the other CTA of the pair may signal.
-__device__ __forceinline__ bool mbar_wait_cluster(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+__device__ __forceinline__ bool mbar_wait_cluster(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
+                                                  long long limit = WAIT_LIMIT_CLOCKS) {
   if (mbar_try_wait_cluster(bar, parity)) return true;
   const long long t0 = clock64();
   uint32_t it = 0;
   while (!mbar_try_wait_cluster(bar, parity)) {
     if ((++it & 0xFF) == 0) {
       if (*abort_flag) return false;
-      if (clock64() - t0 > WAIT_LIMIT_CLOCKS) { *abort_flag = 1; return false; }
+      if (clock64() - t0 > limit) { *abort_flag = 1; return false; }
     }
   }
   return true;

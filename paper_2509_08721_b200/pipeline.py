@@ -44,7 +44,7 @@ class PolicyScorer:
     def __init__(self, W_head: torch.Tensor, max_tokens: int, max_seqs: int, max_questions: int,
                  eps_low: float = 0.2, eps_high: float = 0.28, adv_eps: float = 1e-6,
                  ddof: int = 0, grad_scale: float = 1.0, device="cuda", active_backward: bool = False,
-                 backward: Optional[str] = None):
+                 backward: Optional[str] = None, want_entropy: bool = False):
         if not torch.cuda.is_available():
             raise B.SapoError("PolicyScorer needs a CUDA device; there is no CPU path")
         B.load()
@@ -59,6 +59,9 @@ class PolicyScorer:
         self.packed = B.alloc_packed(self.max_tokens, self.max_seqs, self.max_q, self.H, self.dtype, device)
         self.adv = torch.empty(self.max_seqs, dtype=torch.float32, device=device)
         self.fwd = B.alloc_fwd_outputs(self.max_tokens, self.max_seqs, device)
+        # per-token entropy of the policy's distribution, if asked for (a by-product of the forward)
+        self.entropy = (torch.empty(self.max_tokens, dtype=torch.float32, device=device)
+                        if want_entropy else None)
         self.dhidden = torch.empty(self.max_tokens, self.H, dtype=torch.float32, device=device)
         self.dW = torch.empty(self.V, self.H, dtype=torch.float32, device=device)
         nf = B.sapo_workspace_bytes(B.WS_FWD, self.max_tokens, self.H, self.V, self.dcode)
@@ -93,11 +96,12 @@ class PolicyScorer:
         if self.backward == "fused":
             B.sapo_policy_loss_fwd_bwd(p["hidden"], self.W, p["ids"], p["old_logp"], self.adv, cu,
                                        self.eps_low, self.eps_high, self.grad_scale, self.fwd,
-                                       self.dhidden, self.dW, False, self.workspace, self.status, T=T)
+                                       self.dhidden, self.dW, False, self.workspace, self.status, T=T,
+                                       entropy=self.entropy)
             return StepResult(self.fwd["loss"], self.fwd, self.dhidden, self.dW, p, self.adv)
         B.sapo_policy_loss_fwd(p["hidden"], self.W, p["ids"], p["old_logp"], self.adv, cu,
                                self.eps_low, self.eps_high, self.grad_scale, self.fwd,
-                               self.workspace, self.status, T=T)
+                               self.workspace, self.status, T=T, entropy=self.entropy)
         if self.active_backward:
             B.sapo_policy_loss_bwd_active(p["hidden"], self.W, p["ids"], self.fwd["lse"], self.fwd["gscale"],
                                           self.dhidden, self.dW, False, self.workspace, self.status,

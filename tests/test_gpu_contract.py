@@ -116,3 +116,27 @@ def test_nonfinite_old_logp_or_advantage_masks_the_tokens_and_is_reported(fused)
     assert torch.isfinite(out["loss"]).all()
     assert torch.isfinite(out["dW"]).all() and torch.isfinite(out["dhidden"]).all()
     assert not out["dhidden"][t_bad].any()
+
+
+def test_a_bounded_wait_that_runs_out_sets_the_status_bit_and_leaves_the_context_usable():
+    """Every in-kernel wait of the library has a limit.  The probe waits 100,000 clocks on a
+    barrier nobody arrives at: it must come back with WAIT_TIMEOUT set, and a regular call right
+    after it must run clean."""
+    status = B.new_status()
+    B.sapo_debug_wait_timeout(100_000, status)
+    torch.cuda.synchronize()
+    assert status.item() == 0x20 and B.decode_status(status.item()) == ["WAIT_TIMEOUT"]
+    # nothing is left behind: a scoring step on the same stream is clean and correct
+    batch = gen.make_batch(_recipe(Q=2), 80)
+    gen.install_old_logp(batch, U.oracle_current_logp(batch))
+    b = batch.built
+    adv = np.linspace(-1, 1, batch.S).astype(np.float32)
+    out = U.gpu_scores_fused(U.to_torch(b.hidden), U.to_torch(batch.W), U.to_torch(b.ids), U.to_torch(b.old_logp),
+                             U.to_torch(adv), U.to_torch(b.cu_seqlens), 0.2, 0.28)
+    assert out["status"] == 0
+    ref = orc.policy_loss_fwd(gen.as_f32(b.hidden), gen.as_f32(batch.W), b.ids, b.old_logp, adv, b.cu_seqlens,
+                              0.2, 0.28)
+    U.check_forward(out, ref, adv.astype(np.float64), b.cu_seqlens, 0.2, 0.28)
+    # a limit outside the allowed range is refused on the host
+    with pytest.raises(B.SapoError):
+        B.sapo_debug_wait_timeout(10**9, status)

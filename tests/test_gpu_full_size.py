@@ -38,12 +38,21 @@ def check_gradient_invariants(res, hidden_dev, W_dev, T):
     dW, dH = res.dW.double(), res.dhidden[:T].double()
     col = dW.sum(0)
     scale = dW.abs().sum(0) + 1e-30
-    assert (col.abs() / scale).max().item() < 2e-2          # bf16 rounding of dz, summed over V
+    col_ratio = (col.abs() / scale).max().item()
     a = (dW * W_dev.double()).sum().item()
     b = (dH * hidden_dev[:T].double()).sum().item()
     size = (dW.abs() * W_dev.double().abs()).sum().item() + 1e-30
-    assert abs(a - b) <= 2e-3 * size, (a, b, size)
+    print(f"\n[invariants] T={T} max_h |sum_v dW| / sum_v |dW| = {col_ratio:.3e}; "
+          f"|<dW,W> - <dH,h>| / sum |dW||W| = {abs(a - b) / size:.3e}")
+    assert col_ratio < COL_SUM_BOUND                         # bf16 rounding of the panel entries, summed over V
+    assert abs(a - b) <= INNER_PRODUCT_BOUND * size, (a, b, size)
 
+
+# Bounds of the two invariants: twice the largest value measured over workloads 2-5 in both modes
+# (the residue of rounding each panel entry to bf16; a dropped vocab tile or token chunk is
+# orders of magnitude above it).
+COL_SUM_BOUND = 2e-2
+INNER_PRODUCT_BOUND = 2e-3
 
 _W2 = {}
 
@@ -99,70 +108,105 @@ def test_workload2_full_size(backward):
     check_gradient_invariants(res, res.packed["hidden"], scorer.W, T)
 
 
-FULL = [(3, None, 1200), (4, None, 500), (5, 0.75, 1500), (5, 0.0, 1500)]
+# ---------------------------------------------------------------------------------------------
+# Workloads 3, 4 and 5 at full size.  The oracle's forward pass over ALL tokens (lse, log-probs,
+# entropy) is too long for every test run (7e13 - 1.6e14 fp64 flops per workload), so it is
+# written once by tests/golden/write_oracle_cache.py and kept under build/oracle_cache/, keyed by
+# the oracle's code and the inputs; a missing or stale file is recomputed here (minutes).
+# Everything downstream of the log-probs (ratio, surrogate, gradient factor, per-sequence means,
+# loss) is the oracle's, over all tokens; the gradients are compared on sampled rows, which the
+# oracle computes one by one: dhidden on token rows, dW_head on vocab rows (oracle.dW_rows).
+import importlib.util
+import os
+
+_spec = importlib.util.spec_from_file_location(
+    "write_oracle_cache", os.path.join(os.path.dirname(os.path.abspath(__file__)), "golden", "write_oracle_cache.py"))
+oracle_cache = importlib.util.module_from_spec(_spec)
+_spec.loader.exec_module(oracle_cache)
+
+FULL = [(3, None), (4, None), (5, 0.75), (5, 0.0)]
+_FULL = {}
+
+
+def full_size_reference(number, ext_fraction):
+    """Batch, oracle forward over all tokens and the oracle's loss terms; one case is kept."""
+    key = (number, ext_fraction)
+    if _FULL.get("key") != key:
+        _FULL.clear()
+        torch.cuda.empty_cache()
+        recipe = gen.config(number, ext_fraction=ext_fraction)
+        batch = gen.make_batch(recipe, 1000 * number)
+        fwd = oracle_cache.load(number, ext_fraction, batch)
+        if fwd is None:
+            print(f"\n[oracle cache] computing {oracle_cache.case_name(number, ext_fraction)} "
+                  f"({batch.T} tokens): minutes of host BLAS")
+            fwd = oracle_cache.write(number, ext_fraction, batch=batch, progress=False)
+        b = batch.built
+        gen.install_old_logp(batch, fwd["logp"].astype(np.float32))
+        adv = orc.group_advantages(b.rewards, b.group_offsets, adv_eps=float(np.float32(1e-6)))["adv"]
+        ref = orc.surrogate_from_logp(fwd["logp"], b.old_logp, adv, b.cu_seqlens, batch.eps_low, batch.eps_high)
+        ref["logp"], ref["lse"], ref["entropy"] = fwd["logp"], fwd["lse"], fwd["entropy"]
+        _FULL.update(key=key, recipe=recipe, batch=batch, adv=adv, ref=ref,
+                     h=gen.as_f32(b.hidden), W64=gen.as_f32(batch.W).astype(np.float64))
+    return _FULL
 
 
 @pytest.mark.parametrize("backward", MODES)
-@pytest.mark.parametrize("number,ext_fraction,sample_tokens", FULL,
-                         ids=["cfg3", "cfg4", "cfg5_J6", "cfg5_J0"])
-def test_workloads_3_to_5_full_size_sampled(number, ext_fraction, sample_tokens, backward):
-    recipe = gen.config(number, ext_fraction=ext_fraction)
-    batch = gen.make_batch(recipe, 1000 * number)
-    T, S = batch.T, batch.S
+@pytest.mark.parametrize("number,ext_fraction", FULL, ids=["cfg3", "cfg4", "cfg5_J6", "cfg5_J0"])
+def test_workloads_3_to_5_full_size(number, ext_fraction, backward):
+    c = full_size_reference(number, ext_fraction)
+    recipe, batch, adv, ref, h, W64 = (c[k] for k in ("recipe", "batch", "adv", "ref", "h", "W64"))
+    T, S, V = batch.T, batch.S, batch.V
     b = batch.built
-    W_dev = _to_dev(batch.W, "cuda")
-    # old log-probs: noise around a chunked torch estimate of the current ones (an input recipe)
-    cur = U.torch_current_logp(_to_dev(b.hidden, "cuda"), W_dev, U.to_torch(b.ids)).cpu().numpy()
-    gen.install_old_logp(batch, cur)
-    adv = orc.group_advantages(b.rewards, b.group_offsets, adv_eps=float(np.float32(1e-6)))["adv"]
 
-    scorer, res = run_scorer(batch, recipe, backward)
+    scorer = PolicyScorer(_to_dev(batch.W, "cuda"), T, S, recipe.Q, eps_low=batch.eps_low,
+                          eps_high=batch.eps_high, backward=backward, want_entropy=True)
+    scorer.make_host_batch(batch)
+    res = scorer.step_from_host(T, S)
+    torch.cuda.synchronize()
+    scorer.check_status()
+    # pack and advantages
     assert np.array_equal(U.to_numpy(res.packed["ids"])[:T], b.ids)
     assert np.array_equal(U.to_numpy(res.packed["cu_seqlens"])[:S + 1], b.cu_seqlens)
-    assert np.allclose(res.adv[:S].cpu().numpy(), adv, rtol=U.TOL_ADV_REL, atol=1e-9)
-
-    # sampled whole sequences (prefer ones with a non-zero advantage), scored one by one
+    assert np.array_equal(U.to_numpy(res.packed["seq_src"])[:S], b.seq_src)
     rng = np.random.default_rng(number)
-    order = rng.permutation(S)
-    order = np.concatenate([order[adv[order] != 0], order[adv[order] == 0][:1]])
-    W64 = gen.as_f32(batch.W).astype(np.float64)
-    used = 0
-    for s in order:
-        a, e = int(b.cu_seqlens[s]), int(b.cu_seqlens[s + 1])
-        if used + (e - a) > sample_tokens and used > 0:
-            continue
-        used += e - a
-        hs = gen.as_f32(b.hidden[a:e])
-        lp = orc.token_logprobs(hs, W64, b.ids[a:e])
-        ref = orc.surrogate_from_logp(lp["logp"], b.old_logp[a:e], adv[s:s + 1], [0, e - a],
-                                      batch.eps_low, batch.eps_high, n_seqs_total=S)
-        ref["logp"], ref["lse"] = lp["logp"], lp["lse"]
-        out = {k: res.fwd[k][a:e] for k in ("logp", "lse", "ratio", "surr", "gscale")}
-        U.check_forward(out, ref, adv[s:s + 1], np.array([0, e - a]), batch.eps_low, batch.eps_high)
-        assert abs(res.fwd["seq_surr"][s].item() - ref["seq_surr"][0]) <= 1e-3 * (abs(adv[s]) + 1e-12)
-        dz = orc.dlogits(hs, W64, b.ids[a:e], lp["lse"], ref["gscale"])
-        dH_ref = dz @ W64
-        got = res.dhidden[a:e].cpu().numpy()
-        if adv[s] == 0:
-            assert np.all(got == 0.0)
-        else:
-            assert U.rel_fro(got, dH_ref) <= U.TOL_GRAD_FRO
-        if used >= sample_tokens:
-            break
-    # the loss is the mean of the per-sequence surrogates the device reported
-    seq = res.fwd["seq_surr"][:S].double().cpu().numpy()
-    assert abs(res.loss.item() - (-seq.mean())) <= 1e-6 * np.abs(seq).mean() + 1e-9
+    rows = np.sort(rng.choice(T, size=256, replace=False))
+    assert np.array_equal(U.to_numpy(res.packed["hidden"][torch.from_numpy(rows).cuda()]), b.hidden[rows])
+    assert np.allclose(res.adv[:S].cpu().numpy(), adv, rtol=U.TOL_ADV_REL, atol=1e-9)
+    # every token's forward outputs, the per-sequence means and the loss
+    out = {k: v[:T] for k, v in res.fwd.items() if k not in ("seq_surr", "loss")}
+    U.check_forward(out, ref, adv, b.cu_seqlens, batch.eps_low, batch.eps_high)
+    ent = scorer.entropy[:T].cpu().numpy().astype(np.float64)
+    assert np.max(np.abs(ent - ref["entropy"])) <= U.TOL_LOGP_ABS
+    seq = res.fwd["seq_surr"][:S].cpu().numpy().astype(np.float64)
+    assert np.max(np.abs(seq - ref["seq_surr"])) <= 1e-3 * np.abs(adv).max()
+    U.check_loss(float(res.loss.item()), ref["loss"], adv)
+    # dhidden on sampled token rows (zero-advantage rows must be exactly zero)
+    dz = orc.dlogits(h[rows], W64, b.ids[rows], ref["lse"][rows], ref["gscale"][rows])
+    got = res.dhidden[torch.from_numpy(rows).cuda()].cpu().numpy()
+    e_h = U.rel_fro(got, dz @ W64)
+    zero = ref["gscale"][rows] == 0
+    assert not got[zero].any()
+    # dW_head on sampled vocab rows: random ones, rows of chosen ids, and the last vocab tile
+    vrows = np.unique(np.concatenate([rng.choice(V, size=112, replace=False), b.ids[:8], b.ids[-8:],
+                                      np.arange(V - 8, V)]))
+    dW_ref = orc.dW_rows(h, W64, b.ids, ref["lse"], ref["gscale"], vrows)
+    e_w = U.rel_fro(res.dW[torch.from_numpy(vrows).cuda()].cpu().numpy(), dW_ref)
+    assert e_h <= U.TOL_GRAD_FRO and e_w <= U.TOL_GRAD_FRO, (e_h, e_w)
     check_gradient_invariants(res, res.packed["hidden"], scorer.W, T)
     if number == 3:      # a quarter of the questions have equal rewards: no gradient from them
         go = b.group_offsets
-        rows = slice(int(b.cu_seqlens[go[0]]), int(b.cu_seqlens[go[4]]))
-        assert torch.all(res.dhidden[rows] == 0)
+        zrows = slice(int(b.cu_seqlens[go[0]]), int(b.cu_seqlens[go[4]]))
+        assert torch.all(res.dhidden[zrows] == 0)
+    del scorer, res
+    torch.cuda.empty_cache()
 
 
-LITE = [(3, None, 128), (4, None, 128), (5, 0.5, 64)]
+LITE = [(3, None, 128), (4, None, 128), (5, 0.0, 64), (5, 0.25, 64), (5, 0.5, 64), (5, 0.75, 64)]
 
 
-@pytest.mark.parametrize("number,ext_fraction,length_div", LITE, ids=["cfg3", "cfg4", "cfg5"])
+@pytest.mark.parametrize("number,ext_fraction,length_div", LITE,
+                         ids=["cfg3", "cfg4", "cfg5_J0", "cfg5_J2", "cfg5_J4", "cfg5_J6"])
 def test_workloads_3_to_5_lite_end_to_end(number, ext_fraction, length_div):
     """Full H and V, group structure and reward law of the workload, completions shortened so
     that the oracle finishes: every output, dW included, against the oracle."""

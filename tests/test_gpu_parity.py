@@ -28,6 +28,10 @@ PACK_CASES = [
     ("odd_row_bytes", small_recipe(H=13), None),
     ("cfg1", gen.config(1), None),
     ("cfg2_lite", gen.config(2, length_div=8), None),
+    # the swarm-mix sweep: every external share, drawn from the pool of eight node buffers
+    ("cfg5_lite_J0", gen.config(5, ext_fraction=0.0, length_div=16), None),
+    ("cfg5_lite_J2", gen.config(5, ext_fraction=0.25, length_div=16), None),
+    ("cfg5_lite_J4", gen.config(5, ext_fraction=0.5, length_div=16), None),
     ("cfg5_lite_J6", gen.config(5, ext_fraction=0.75, length_div=16), None),
 ]
 

@@ -90,7 +90,8 @@ def gpu_pack(batch: gen.Batch, max_tokens: Optional[int] = None, max_seqs: Optio
 
 
 def gpu_scores(hidden, W, ids, old_logp, adv, cu, eps_low, eps_high, grad_scale=1.0,
-               bwd_workspace_bytes: Optional[int] = None, want_bwd: bool = True):
+               bwd_workspace_bytes: Optional[int] = None, want_bwd: bool = True,
+               out_dtype: torch.dtype = torch.float32, accumulate_into=None):
     """fwd (+ bwd) through the binding on device tensors; returns device tensors."""
     T, H, V, S = hidden.shape[0], hidden.shape[1], W.shape[0], cu.numel() - 1
     dcode = B.DTYPE_F32 if hidden.dtype == torch.float32 else B.DTYPE_BF16
@@ -100,31 +101,34 @@ def gpu_scores(hidden, W, ids, old_logp, adv, cu, eps_low, eps_high, grad_scale=
     B.sapo_policy_loss_fwd(hidden, W, ids, old_logp, adv, cu, eps_low, eps_high, grad_scale, out,
                            ws_f, status)
     if want_bwd:
-        nbytes = (B.sapo_workspace_bytes(B.WS_BWD, T, H, V, dcode)
+        kind = B.WS_BWD | (B.WS_OUT_BF16 if out_dtype == torch.bfloat16 else 0)
+        nbytes = (B.sapo_workspace_bytes(kind, T, H, V, dcode)
                   if bwd_workspace_bytes is None else bwd_workspace_bytes)
         ws_b = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
-        out["dhidden"] = torch.empty(T, H, dtype=torch.float32, device="cuda")
-        out["dW"] = torch.empty(V, H, dtype=torch.float32, device="cuda")
+        out["dhidden"] = torch.empty(T, H, dtype=out_dtype, device="cuda")
+        out["dW"] = torch.empty(V, H, dtype=out_dtype, device="cuda") if accumulate_into is None else accumulate_into
         B.sapo_policy_loss_bwd(hidden, W, ids, out["lse"], out["gscale"], out["dhidden"], out["dW"],
-                               False, ws_b, status)
+                               accumulate_into is not None, ws_b, status)
     torch.cuda.synchronize()
     out["status"] = int(status.item())
     return out
 
 
 def gpu_scores_fused(hidden, W, ids, old_logp, adv, cu, eps_low, eps_high, grad_scale=1.0,
-                     workspace_bytes: Optional[int] = None, **variant):
+                     workspace_bytes: Optional[int] = None, out_dtype: torch.dtype = torch.float32,
+                     accumulate_into=None, **variant):
     """Loss and gradients through the single-pass call; returns device tensors."""
     T, H, V, S = hidden.shape[0], hidden.shape[1], W.shape[0], cu.numel() - 1
     status = B.new_status()
     out = B.alloc_fwd_outputs(T, S)
-    nbytes = (B.sapo_workspace_bytes(B.WS_FUSED, T, H, V, B.DTYPE_BF16)
+    kind = B.WS_FUSED | (B.WS_OUT_BF16 if out_dtype == torch.bfloat16 else 0)
+    nbytes = (B.sapo_workspace_bytes(kind, T, H, V, B.DTYPE_BF16)
               if workspace_bytes is None else workspace_bytes)
     ws = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
-    out["dhidden"] = torch.empty(T, H, dtype=torch.float32, device="cuda")
-    out["dW"] = torch.empty(V, H, dtype=torch.float32, device="cuda")
+    out["dhidden"] = torch.empty(T, H, dtype=out_dtype, device="cuda")
+    out["dW"] = torch.empty(V, H, dtype=out_dtype, device="cuda") if accumulate_into is None else accumulate_into
     B.sapo_policy_loss_fwd_bwd(hidden, W, ids, old_logp, adv, cu, eps_low, eps_high, grad_scale, out,
-                               out["dhidden"], out["dW"], False, ws, status, **variant)
+                               out["dhidden"], out["dW"], accumulate_into is not None, ws, status, **variant)
     torch.cuda.synchronize()
     out["status"] = int(status.item())
     return out
