@@ -84,6 +84,7 @@ extern "C" {
 #define SAPO_WS_BWD_ACTIVE 2
 #define SAPO_WS_FUSED 3
 #define SAPO_WS_OUT_BF16 0x100   /* OR into `which`: the gradients will be asked for in bf16 */
+#define SAPO_WS_GATHER   0x200   /* OR into `which`: for sapo_policy_loss_fwd_bwd_gather          */
 
 /* A rollout store: n_rollouts completions laid end to end (Section 3.1: a node's answers
  * to its questions; Section 3.2: the tuples other nodes broadcast).
@@ -119,7 +120,11 @@ typedef struct sapo_selection {
  *   seq_src [max_seqs] index of the rollout inside its buffer
  *   tok_seq [max_tokens] sequence of each token;  tok_mask [max_tokens] 1 for t < T else 0
  *   group_offsets [Q+1] first sequence of each question
- *   n_tokens, n_seqs: device scalars T and S */
+ *   n_tokens, n_seqs: device scalars T and S
+ *   tok_src [max_tokens] (optional, may be NULL): where each packed token's row lives in its source
+ *     buffer: row index, plus 2^62 when it is the external buffer; -1 for unused slots.  With it the
+ *     loss can read the hidden states in place (sapo_policy_loss_fwd_bwd_gather) and `hidden` may
+ *     be NULL: the pack then copies no hidden rows at all. */
 typedef struct sapo_packed {
   void*    hidden;
   int32_t* ids;
@@ -136,6 +141,7 @@ typedef struct sapo_packed {
   int32_t* n_seqs;
   int64_t  max_tokens;
   int32_t  max_seqs;
+  int64_t* tok_src;
 } sapo_packed;
 
 /* Loss parameters.  The paper's run uses eps_low 0.2, eps_high 0.28 and no KL term
@@ -251,6 +257,38 @@ int sapo_policy_loss_bwd(const void* hidden, const void* W_head, int32_t dtype,
                          void* workspace, size_t workspace_bytes,
                          int32_t* status, void* stream);
 
+/* The loss over a vocabulary that is sharded across ranks (no counterpart in the paper, whose
+ * nodes each hold a whole model; it lets one node's LM head span several GPUs).  Rank r holds
+ * W_shard = rows [vocab_offset, vocab_offset + V_shard) of W_head and every token's hidden state.
+ *   1. sapo_lmhead_lse_partial: the projection of the shard on the tensor cores, reduced per token
+ *      to triple[0][t] = max_v z log2(e), triple[1][t] = sum_v 2^(z log2(e) - max), triple[2][t] =
+ *      z[t, ids[t]] if the chosen token lies in the shard, else 0   (float32 [3][T]).
+ *      workspace: sapo_workspace_bytes(SAPO_WS_FWD, T, H, V_shard, dtype).
+ *   2. the caller gathers the triples of all ranks into local memory, [n_parts][3][T] (one
+ *      all-gather of 12 T bytes per rank);
+ *   3. sapo_policy_loss_from_partials: merges them (log-sum-exp over the parts) and evaluates the
+ *      loss tail exactly as sapo_policy_loss_fwd does; every rank computes the same values.
+ *      ids are the global token ids, V the whole vocabulary.  h_cfg->entropy must be NULL.
+ *   4. sapo_policy_loss_bwd_shard: sapo_policy_loss_bwd on the shard with the global lse:
+ *      dW_shard [V_shard, H] is this rank's rows of dW_head; dhidden is this shard's share of
+ *      the sum over the vocabulary, to be added up over the ranks (one all-reduce of T H values).
+ * The library itself moves nothing between GPUs; a kernel only ever reads local memory. */
+int sapo_lmhead_lse_partial(const void* hidden, const void* W_shard, int32_t dtype,
+                            int64_t T, int32_t H, int32_t V_shard, int64_t ld_hidden, int64_t ld_W,
+                            const int32_t* ids, int32_t vocab_offset, float* triple,
+                            void* workspace, size_t workspace_bytes, int32_t* status, void* stream);
+int sapo_policy_loss_from_partials(const float* triples, int32_t n_parts, int64_t T, int32_t V,
+                                   const int32_t* ids, const float* old_logp, const float* adv,
+                                   const int32_t* cu_seqlens, int32_t S, const sapo_loss_cfg* h_cfg,
+                                   float* logp, float* lse, float* ratio, float* surr, float* gscale,
+                                   float* seq_surr, float* loss, int32_t* status, void* stream);
+int sapo_policy_loss_bwd_shard(const void* hidden, const void* W_shard, int32_t dtype,
+                               int64_t T, int32_t H, int32_t V_shard, int64_t ld_hidden, int64_t ld_W,
+                               const int32_t* ids, int32_t vocab_offset, const float* lse,
+                               const float* gscale, void* dhidden, void* dW_shard, int32_t out_dtype,
+                               int32_t accumulate_dW, void* workspace, size_t workspace_bytes,
+                               int32_t* status, void* stream);
+
 /* The same gradient, computed over the active tokens only (gscale[t] != 0).  Sequences of a
  * zero-advantage group — which the paper's experiments drop from the shared pool as
  * uninformative (Section 5) — and tokens clipped on the binding side have gscale = 0 and add
@@ -301,6 +339,28 @@ int sapo_policy_loss_fwd_bwd(const void* hidden, const void* W_head, int32_t dty
                              void* dhidden, void* dW_head, int32_t out_dtype, int32_t accumulate_dW,
                              void* workspace, size_t workspace_bytes,
                              int32_t* status, void* stream);
+
+/* sapo_policy_loss_fwd_bwd with the hidden states read in place.  The training set is a union of
+ * index picks (Section 3.2, training-set equation), so it need not be copied: every packed token
+ * names its row in the local or the external rollout store (tok_src, written by
+ * sapo_pack_rollouts, which then copies no hidden rows when its `hidden` output is NULL), the
+ * projection's row loads follow the runs of consecutive rows that whole sequences form, and the
+ * per-token kernels read their row through the same map.  local_hidden [n_local_tokens, ld_hidden],
+ * ext_hidden [n_ext_tokens, ld_hidden] (bf16, the same row pitch, 16-byte aligned; fewer than 2^31
+ * rows each); everything else, results included, as in sapo_policy_loss_fwd_bwd.  A packed slot
+ * without a token (tok_src -1) is scored as masked; a tok_src that points outside its store sets
+ * SAPO_ST_BAD_INDEX.  workspace: sapo_workspace_bytes(SAPO_WS_FUSED | SAPO_WS_GATHER, ...). */
+int sapo_policy_loss_fwd_bwd_gather(const void* local_hidden, int64_t n_local_tokens,
+                                    const void* ext_hidden, int64_t n_ext_tokens, const int64_t* tok_src,
+                                    const void* W_head, int32_t dtype,
+                                    int64_t T, int32_t H, int32_t V, int64_t ld_hidden, int64_t ld_W,
+                                    const int32_t* ids, const float* old_logp, const float* adv,
+                                    const int32_t* cu_seqlens, int32_t S, const sapo_loss_cfg* h_cfg,
+                                    float* logp, float* lse, float* ratio, float* surr, float* gscale,
+                                    float* seq_surr, float* loss,
+                                    void* dhidden, void* dW_head, int32_t out_dtype, int32_t accumulate_dW,
+                                    void* workspace, size_t workspace_bytes,
+                                    int32_t* status, void* stream);
 
 /* Section 3.2 (nodes filter and sample what the swarm shares) / Section 5 (the experiments'
  * policy: discard rollouts with zero advantage, then sample uniformly from the rest).

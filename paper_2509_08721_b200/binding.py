@@ -21,6 +21,7 @@ WS_BWD = 1
 WS_BWD_ACTIVE = 2
 WS_FUSED = 3
 WS_OUT_BF16 = 0x100      # OR into the workspace kind: gradients in bf16
+WS_GATHER = 0x200        # OR into the workspace kind: hidden rows read in place (..._gather)
 
 ST_BITS = {
     0x01: "TOKEN_OVERFLOW", 0x02: "SEQ_OVERFLOW", 0x04: "BAD_INDEX", 0x08: "EMPTY_SEQUENCE",
@@ -33,6 +34,7 @@ EXPORTS = ("sapo_pack_rollouts", "sapo_group_advantages", "sapo_policy_loss_fwd"
            "sapo_status_string", "sapo_timing_enable", "sapo_timing_read", "sapo_launch_count",
            "sapo_policy_loss_fwd_static", "sapo_policy_loss_bwd_active", "sapo_policy_loss_fwd_bwd",
            "sapo_select_external", "sapo_group_advantages_warp", "sapo_debug_wait_timeout",
+           "sapo_policy_loss_fwd_bwd_gather", "sapo_lmhead_lse_partial", "sapo_policy_loss_from_partials", "sapo_policy_loss_bwd_shard",
            "sapo_select_workspace_bytes", "sapo_adam_step")
 STATIC_SCRATCH_BYTES = 4 * 1024 * 1024
 KERNEL_NAMES = ("pack_scan", "pack_copy", "group_adv", "split_bf16", "fwd_gemm", "loss_tail",
@@ -55,7 +57,8 @@ class PackedC(C.Structure):
                 ("rewards", C.c_void_p), ("cu_seqlens", C.c_void_p), ("seq_group", C.c_void_p),
                 ("seq_is_ext", C.c_void_p), ("seq_src", C.c_void_p), ("tok_seq", C.c_void_p),
                 ("tok_mask", C.c_void_p), ("group_offsets", C.c_void_p), ("n_tokens", C.c_void_p),
-                ("n_seqs", C.c_void_p), ("max_tokens", C.c_int64), ("max_seqs", C.c_int32)]
+                ("n_seqs", C.c_void_p), ("max_tokens", C.c_int64), ("max_seqs", C.c_int32),
+                ("tok_src", C.c_void_p)]
 
 
 class LossCfgC(C.Structure):
@@ -105,6 +108,10 @@ def load() -> C.CDLL:
     lib.sapo_policy_loss_fwd_bwd.argtypes = [vp, vp, i32, i64, i32, i32, i64, i64, vp, vp, vp, vp, i32,
                                              C.POINTER(LossCfgC), vp, vp, vp, vp, vp, vp, vp, vp, vp, i32, i32,
                                              vp, sz, vp, vp]
+    lib.sapo_policy_loss_fwd_bwd_gather.restype = C.c_int
+    lib.sapo_policy_loss_fwd_bwd_gather.argtypes = [vp, i64, vp, i64, vp, vp, i32, i64, i32, i32, i64, i64, vp, vp, vp,
+                                                    vp, i32, C.POINTER(LossCfgC), vp, vp, vp, vp, vp, vp, vp, vp, vp,
+                                                    i32, i32, vp, sz, vp, vp]
     lib.sapo_select_external.restype = C.c_int
     lib.sapo_select_external.argtypes = [vp, vp, i32, i32, C.c_uint64, vp, vp, vp, vp, sz, vp]
     lib.sapo_select_workspace_bytes.restype = sz
@@ -119,6 +126,14 @@ def load() -> C.CDLL:
     lib.sapo_timing_enable.argtypes = [i32]
     lib.sapo_timing_read.restype = C.c_int
     lib.sapo_timing_read.argtypes = [C.POINTER(C.c_float), C.POINTER(C.c_int32)]
+    lib.sapo_lmhead_lse_partial.restype = C.c_int
+    lib.sapo_lmhead_lse_partial.argtypes = [vp, vp, i32, i64, i32, i32, i64, i64, vp, i32, vp, vp, sz, vp, vp]
+    lib.sapo_policy_loss_from_partials.restype = C.c_int
+    lib.sapo_policy_loss_from_partials.argtypes = [vp, i32, i64, i32, vp, vp, vp, vp, i32, C.POINTER(LossCfgC),
+                                                   vp, vp, vp, vp, vp, vp, vp, vp, vp]
+    lib.sapo_policy_loss_bwd_shard.restype = C.c_int
+    lib.sapo_policy_loss_bwd_shard.argtypes = [vp, vp, i32, i64, i32, i32, i64, i64, vp, i32, vp, vp, vp, vp,
+                                               i32, i32, vp, sz, vp, vp]
     lib.sapo_debug_wait_timeout.restype = C.c_int
     lib.sapo_debug_wait_timeout.argtypes = [i64, vp, vp]
     lib.sapo_launch_count.restype = C.c_int64
@@ -224,11 +239,15 @@ class DeviceSelection:
 
 
 def alloc_packed(max_tokens: int, max_seqs: int, Q: int, H: int, dtype: torch.dtype,
-                 device="cuda") -> Dict[str, torch.Tensor]:
+                 device="cuda", copy_hidden: bool = True, tok_src: bool = False) -> Dict[str, torch.Tensor]:
+    """Output buffers of sapo_pack_rollouts.  copy_hidden=False leaves out the packed copy of the
+    hidden rows (then tok_src is needed: the loss reads the rows in place)."""
     i32, f32, u8 = torch.int32, torch.float32, torch.uint8
     e = lambda *s, dt: torch.empty(*s, dtype=dt, device=device)
+    extra = {"tok_src": e(max_tokens, dt=torch.int64)} if (tok_src or not copy_hidden) else {}
     return {
-        "hidden": e(max_tokens, H, dt=dtype), "ids": e(max_tokens, dt=i32),
+        **extra, "H": H, "dtype": dtype,
+        "hidden": e(max_tokens, H, dt=dtype) if copy_hidden else None, "ids": e(max_tokens, dt=i32),
         "old_logp": e(max_tokens, dt=f32), "rewards": e(max_seqs, dt=f32),
         "cu_seqlens": e(max_seqs + 1, dt=i32), "seq_group": e(max_seqs, dt=i32),
         "seq_is_ext": e(max_seqs, dt=u8), "seq_src": e(max_seqs, dt=i32),
@@ -241,14 +260,14 @@ def sapo_pack_rollouts(local: DeviceRollouts, ext: DeviceRollouts, sel: DeviceSe
                        out: Dict[str, torch.Tensor], status: torch.Tensor) -> None:
     """Enqueue the pack on the current stream; `out` comes from alloc_packed."""
     _require_cuda()
-    H = int(out["hidden"].shape[1])
+    H = int(out["H"])
     pc = PackedC(*[_p(out[k]) for k in ("hidden", "ids", "old_logp", "rewards", "cu_seqlens",
                                         "seq_group", "seq_is_ext", "seq_src", "tok_seq", "tok_mask",
                                         "group_offsets", "n_tokens", "n_seqs")],
-                 int(out["ids"].numel()), int(out["seq_group"].numel()))
+                 int(out["ids"].numel()), int(out["seq_group"].numel()), _p(out.get("tok_src")))
     lc, ec, sc = local.c(), ext.c(), sel.c()
     rc = load().sapo_pack_rollouts(C.byref(lc), C.byref(ec), C.byref(sc), H,
-                                   _dtype_code(out["hidden"]), C.byref(pc), _p(status), _stream())
+                                   _dtype_code(local.hidden), C.byref(pc), _p(status), _stream())
     _check(rc, "sapo_pack_rollouts")
 
 
@@ -375,6 +394,78 @@ def sapo_policy_loss_fwd_bwd(hidden: torch.Tensor, W_head: torch.Tensor, ids: to
         1 if accumulate_dW else 0,
         _p(workspace), workspace.numel() * workspace.element_size(), _p(status), _stream())
     _check(rc, "sapo_policy_loss_fwd_bwd")
+
+
+def sapo_policy_loss_fwd_bwd_gather(local_hidden: torch.Tensor, ext_hidden: torch.Tensor, tok_src: torch.Tensor,
+                                    W_head: torch.Tensor, ids: torch.Tensor, old_logp: torch.Tensor,
+                                    adv: torch.Tensor, cu_seqlens: torch.Tensor, eps_low: float, eps_high: float,
+                                    grad_scale: float, out: Dict[str, torch.Tensor], dhidden: torch.Tensor,
+                                    dW_head: torch.Tensor, accumulate_dW: bool, workspace: torch.Tensor,
+                                    status: torch.Tensor, T: Optional[int] = None, loss_agg: int = 0,
+                                    kl_beta: float = 0.0, ref_logp: Optional[torch.Tensor] = None,
+                                    entropy: Optional[torch.Tensor] = None) -> None:
+    """sapo_policy_loss_fwd_bwd with the hidden rows read in place from the two rollout stores
+    through tok_src (int64 [T], from sapo_pack_rollouts): no packed copy of the hidden states."""
+    _require_cuda()
+    T = int(tok_src.shape[0]) if T is None else int(T)
+    H, V = int(W_head.shape[1]), int(W_head.shape[0])
+    S = int(cu_seqlens.numel() - 1)
+    ld = int(local_hidden.stride(0)) if local_hidden.shape[0] > 0 else int(ext_hidden.stride(0))
+    if local_hidden.shape[0] > 0 and ext_hidden.shape[0] > 0 and local_hidden.stride(0) != ext_hidden.stride(0):
+        raise SapoError("the two rollout stores must have the same row pitch")
+    cfg = LossCfgC(eps_low, eps_high, grad_scale, int(loss_agg), float(kl_beta), _p(ref_logp), _p(entropy))
+    rc = load().sapo_policy_loss_fwd_bwd_gather(
+        _p(local_hidden), int(local_hidden.shape[0]), _p(ext_hidden), int(ext_hidden.shape[0]), _p(tok_src),
+        _p(W_head), _dtype_code(W_head), T, H, V, ld, W_head.stride(0),
+        _p(ids), _p(old_logp), _p(adv), _p(cu_seqlens), S, C.byref(cfg),
+        _p(out["logp"]), _p(out["lse"]), _p(out["ratio"]), _p(out["surr"]), _p(out["gscale"]),
+        _p(out.get("seq_surr")), _p(out["loss"]), _p(dhidden), _p(dW_head), _out_dtype_code(dhidden, dW_head),
+        1 if accumulate_dW else 0,
+        _p(workspace), workspace.numel() * workspace.element_size(), _p(status), _stream())
+    _check(rc, "sapo_policy_loss_fwd_bwd_gather")
+
+
+def sapo_lmhead_lse_partial(hidden: torch.Tensor, W_shard: torch.Tensor, ids: torch.Tensor, vocab_offset: int,
+                            triple: torch.Tensor, workspace: torch.Tensor, status: torch.Tensor) -> None:
+    """(max, sum, target logit) per token over one vocabulary shard; triple is float32 [3, T]."""
+    _require_cuda()
+    T, H, V = int(hidden.shape[0]), int(hidden.shape[1]), int(W_shard.shape[0])
+    rc = load().sapo_lmhead_lse_partial(
+        _p(hidden), _p(W_shard), _dtype_code(hidden), T, H, V, hidden.stride(0), W_shard.stride(0), _p(ids),
+        int(vocab_offset), _p(triple), _p(workspace), workspace.numel() * workspace.element_size(), _p(status),
+        _stream())
+    _check(rc, "sapo_lmhead_lse_partial")
+
+
+def sapo_policy_loss_from_partials(triples: torch.Tensor, V: int, ids: torch.Tensor, old_logp: torch.Tensor,
+                                   adv: torch.Tensor, cu_seqlens: torch.Tensor, eps_low: float, eps_high: float,
+                                   grad_scale: float, out: Dict[str, torch.Tensor], status: torch.Tensor,
+                                   loss_agg: int = 0, kl_beta: float = 0.0,
+                                   ref_logp: Optional[torch.Tensor] = None) -> None:
+    """The loss tail over the gathered triples of all shards, float32 [n_parts, 3, T]."""
+    _require_cuda()
+    n_parts, T = int(triples.shape[0]), int(triples.shape[2])
+    cfg = LossCfgC(eps_low, eps_high, grad_scale, int(loss_agg), float(kl_beta), _p(ref_logp), None)
+    rc = load().sapo_policy_loss_from_partials(
+        _p(triples), n_parts, T, int(V), _p(ids), _p(old_logp), _p(adv), _p(cu_seqlens),
+        int(cu_seqlens.numel() - 1), C.byref(cfg), _p(out["logp"]), _p(out["lse"]), _p(out["ratio"]),
+        _p(out["surr"]), _p(out["gscale"]), _p(out["seq_surr"]), _p(out["loss"]), _p(status), _stream())
+    _check(rc, "sapo_policy_loss_from_partials")
+
+
+def sapo_policy_loss_bwd_shard(hidden: torch.Tensor, W_shard: torch.Tensor, ids: torch.Tensor, vocab_offset: int,
+                               lse: torch.Tensor, gscale: torch.Tensor, dhidden: torch.Tensor,
+                               dW_shard: torch.Tensor, accumulate_dW: bool, workspace: torch.Tensor,
+                               status: torch.Tensor) -> None:
+    """Backward of one vocabulary shard: dW_shard is final, dhidden is to be summed over the shards."""
+    _require_cuda()
+    T, H, V = int(hidden.shape[0]), int(hidden.shape[1]), int(W_shard.shape[0])
+    rc = load().sapo_policy_loss_bwd_shard(
+        _p(hidden), _p(W_shard), _dtype_code(hidden), T, H, V, hidden.stride(0), W_shard.stride(0), _p(ids),
+        int(vocab_offset), _p(lse), _p(gscale), _p(dhidden), _p(dW_shard), _out_dtype_code(dhidden, dW_shard),
+        1 if accumulate_dW else 0, _p(workspace), workspace.numel() * workspace.element_size(), _p(status),
+        _stream())
+    _check(rc, "sapo_policy_loss_bwd_shard")
 
 
 def sapo_select_external(rewards: torch.Tensor, group_offsets: torch.Tensor, J: int, seed: int):

@@ -40,12 +40,13 @@ struct FwdEpiT {
     const int32_t* ids; float* pm; float* ps; float* pz;  // partials [n_splits][T]
     float* pe;                                             // ENT: partial sums of 2^(x - m) z
     int64_t T; int32_t V;
+    int32_t id_offset;                                     // first vocabulary entry of W (a vocab shard), else 0
   };
   float m, s, zy, sz; int32_t y; int64_t row;
   __device__ __forceinline__ void begin_unit(const Params& p, int mb, int r) {
     row = (int64_t)mb * BM + r;
     m = -INFINITY; s = 0.f; zy = 0.f; sz = 0.f;
-    y = row < p.T ? p.ids[row] : -1;
+    y = row < p.T ? p.ids[row] - p.id_offset : -1;          // outside [0, V): the chosen token is not in these columns
   }
   template <int HALF>
   __device__ __forceinline__ void chunk(const Params& p, float (&v)[32], int col0) {
@@ -56,7 +57,7 @@ struct FwdEpiT {
       for (int j = 0; j < 32; ++j) if (col0 + j >= p.V) v[j] = -1e30f;
     }
     const int yr = y - col0;
-    if (yr >= 0 && yr < 32) {
+    if (yr >= 0 && yr < 32 && y < p.V) {
       #pragma unroll
       for (int j = 0; j < 32; ++j) if (j == yr) zy = v[j];
     }
@@ -102,6 +103,7 @@ struct DzEpi {
     const int32_t* ids; const float* lse; const float* gscale;
     int64_t M; int32_t V; int32_t nvt;
     __nv_bfloat16* panel;
+    int32_t id_offset;     // first vocabulary entry of W (a vocab shard), else 0
   };
   float g, l2; int32_t y; int32_t tile_row0; int r; bool in_panel;
   __device__ __forceinline__ void begin_unit(const Params& p, int mb, int r_) {
@@ -112,7 +114,7 @@ struct DzEpi {
     tile_row0 = mb * p.nvt * BM;          // first panel row of this token block
     g = valid ? p.gscale[row] : 0.f;
     l2 = valid ? p.lse[row] * LOG2E : 0.f;
-    y = valid ? p.ids[row] : -1;
+    y = valid ? p.ids[row] - p.id_offset : -1;
   }
   // dz of 32 columns; every 16 finished columns (32 bytes of the row) are stored at once, so the
   // stores of the eight epilogue warps trickle out between their arithmetic instead of leaving

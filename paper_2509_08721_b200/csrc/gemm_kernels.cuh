@@ -3,6 +3,8 @@
 // wide-tile one for the long-K contractions of the backward pass.
 #pragma once
 
+#include <type_traits>
+
 #include "gemm_epilogues.cuh"
 
 namespace sapo {
@@ -21,10 +23,15 @@ using namespace umma;
 // [n0 + rank * n_eff / 2, + n_eff / 2) of B.  All TMA completions of a stage are counted on the
 // even CTA's barrier; the even CTA's MMA thread frees stages and publishes accumulators on
 // both CTAs' barriers.
-template <int A_KIND, bool B_MN, class Epi, int BKT = BK, int NSTAGE = STAGES>
+//   GATHER (A_KIND 0 only): the rows of A come from two source buffers through a per-block box
+//             list (GatherArgs) instead of from one matrix; map_a is unused.
+template <int A_KIND, bool B_MN, class Epi, int BKT = BK, int NSTAGE = STAGES, class Gather = NoGather>
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
 umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
-                 const Sched sched_arg, const typename Epi::Params ep_arg, int32_t* status) {
+                 const Sched sched_arg, const typename Epi::Params ep_arg, int32_t* status,
+                 const __grid_constant__ Gather ga) {
+  constexpr bool GATHER = !std::is_same<Gather, NoGather>::value;
+  static_assert(!GATHER || (A_KIND == 0 && !B_MN), "gathered rows: K-major A only");
   SAPO_CLOCK_BEGIN
   // a stage holds a K depth of BKT (128: two 64-element boxes per K-major operand; 64: one)
   static_assert(BKT == 128 || (BKT == 64 && A_KIND == 0 && !B_MN), "64-deep stages: K-major operands only");
@@ -46,6 +53,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * NSTAGE + 4);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
   uint64_t* drain = bars + 2 * NSTAGE + 5;   // MMA thread only: "all my MMAs have retired" after a wait ran out
+  uint64_t* box_s = reinterpret_cast<uint64_t*>(reinterpret_cast<uint8_t*>(bars) + 256);   // GATHER: this block's box list
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   constexpr bool A_MN = (A_KIND & 1) != 0;
@@ -86,10 +94,20 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
     int pmb, un, n_begin, n_end, kb0, kb1, slot;
     while (ok && work.next(pmb, un, n_begin, n_end, kb0, kb1, slot)) {
       const int mb = 2 * pmb + (int)rank;                 // this CTA's 128-row block
+      int n_box = 0;
+      uint32_t gather_tx = 0;      // bytes of A rows per stage, both CTAs (rows past the end are not fetched)
+      if constexpr (GATHER) {
+        __syncwarp();
+        auto word_of = [&](int b) -> uint32_t { return (int64_t)b * BM < ga.rows ? (uint32_t)ga.n_boxes[b] : 0u; };
+        n_box = (int)(word_of(mb) & 0xffffu);
+        for (int i = lane; i < n_box; i += 32) box_s[i] = ga.boxes[(size_t)mb * 128 + i];
+        __syncwarp();
+        gather_tx = ((word_of(2 * pmb) >> 16) + (word_of(2 * pmb + 1) >> 16)) * 128u * KBOX;
+      }
       for (int nb = n_begin; ok && nb < n_end; ++nb) {
         const int half = tile_n_eff(sched, nb) >> 1;       // B columns this CTA stages
         const int b_boxes = B_MN ? ((half + 63) >> 6) : KBOX;
-        const uint32_t tx = 2 * (A_ST + b_boxes * BOX_BYTES);
+        const uint32_t tx = GATHER ? gather_tx + 2 * b_boxes * BOX_BYTES : 2 * (A_ST + b_boxes * BOX_BYTES);
         const bool mine = lane < A_BOXES + b_boxes;
         const bool is_a = lane < A_BOXES;
         const int bi = is_a ? lane : lane - A_BOXES;
@@ -103,7 +121,20 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
         for (int kb = kb0; kb < kb1; ++kb) {
           if (!SAPO_TIMED(0, mbar_wait(&empty[stage], phase ^ 1, abort_flag, sched.wait_limit))) { ok = false; break; }
           if (rank == 0 && lane == 0) mbar_arrive_expect_tx(&full[stage], tx);
-          if (mine) {
+          if constexpr (GATHER) {
+            // the A rows of this block, box by box (a lane takes every 32nd box, both k boxes of it)
+            const uint32_t bar = full0_addr + stage * 8;
+            for (int i = lane; i < n_box; i += 32) {
+              const uint64_t e = box_s[i];
+              const int dst_row = (int)(e & 127u), lg = (int)((e >> 7) & 7u), side = (int)((e >> 10) & 1u);
+              const int32_t src_row = (int32_t)(e >> 16);
+              #pragma unroll
+              for (int kx = 0; kx < KBOX; ++kx)
+                tma_load_2d_pair(smem_a + stage * A_ST + kx * BOX_BYTES + dst_row * 128, &ga.maps[side][lg], bar,
+                                 kb * BKT + 64 * kx, src_row);
+            }
+          }
+          if (mine && !(GATHER && is_a)) {
             uint8_t* dst = smem + dst_off + stage * (is_a ? A_ST : B_ST);
             const uint32_t bar = full0_addr + stage * 8;
             if (is_a && A_KIND == 2)        // vocab tiles 2 kb and 2 kb + 1 of token block mb: 256 rows

@@ -68,6 +68,18 @@ struct Sched {
   long long wait_limit;   // SM clocks after which a barrier wait gives up (SAPO_ST_WAIT_TIMEOUT)
 };
 
+// A-operand rows fetched in place from two source buffers (the rollout stores) instead of from a
+// packed copy: for every 128-token block a list of boxes, each 2^k consecutive source rows that go
+// to consecutive rows of the block (a run of tokens of one sequence, cut into powers of two).
+struct NoGather {};
+struct GatherArgs {
+  CUtensorMap maps[2][8];     // [buffer][log2 rows]: boxes of 64 columns x 2^k rows, 128-byte swizzle
+  const uint64_t* boxes;      // [blocks][128]: bits 0-6 first row in the block, 7-9 log2 rows, 10 buffer, 16.. source row
+  const int32_t* n_boxes;     // [blocks]: boxes | rows they cover << 16
+  int64_t rows;               // token rows of this launch (those past it are not fetched)
+};
+constexpr uint32_t GATHER_LIST_BYTES = 128 * 8;
+
 constexpr int PARTIAL_FLOATS = PAIR_M * BN;   // one partial accumulator tile: 256 x 256 fp32
 constexpr int MAX_PAIRS_SCRATCH = 96;          // CTA pairs a launch may use (a B200 has 74)
 constexpr int MAX_PARTS_SCRATCH = 3 * MAX_PAIRS_SCRATCH;   // K-split parts the scratch holds

@@ -135,10 +135,11 @@ constexpr int FWD_BK = 64, FWD_STAGES = 7;
 constexpr int FWD_BK = BK, FWD_STAGES = STAGES;
 #endif
 
-template <int A_KIND, bool B_MN, class Epi, int BKT = BK, int NSTAGE = STAGES>
+template <int A_KIND, bool B_MN, class Epi, int BKT = BK, int NSTAGE = STAGES, class Gather = NoGather>
 static int launch_gemm(const CUtensorMap& ma, const CUtensorMap& mb, const Sched& sched,
-                       const typename Epi::Params& ep, int32_t* status, cudaStream_t st, int kernel_id) {
-  auto kern = umma_gemm_kernel<A_KIND, B_MN, Epi, BKT, NSTAGE>;
+                       const typename Epi::Params& ep, int32_t* status, cudaStream_t st, int kernel_id,
+                       const Gather& ga = Gather{}) {
+  auto kern = umma_gemm_kernel<A_KIND, B_MN, Epi, BKT, NSTAGE, Gather>;
   // CTA pairs the device can hold at once; found, together with the kernel's shared-memory
   // opt-in, on the first use on each device
   static int max_pairs_of[MAX_DEVICES] = {0};
@@ -153,7 +154,8 @@ static int launch_gemm(const CUtensorMap& ma, const CUtensorMap& mb, const Sched
   attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
   cudaLaunchConfig_t cfg = {};
   cfg.blockDim = dim3(GEMM_THREADS, 1, 1);
-  constexpr size_t smem_bytes = 1024 + (size_t)NSTAGE * (BM + BN / 2) * BKT * 2 + 256;
+  constexpr size_t smem_bytes = 1024 + (size_t)NSTAGE * (BM + BN / 2) * BKT * 2 + 256 +
+                                (std::is_same<Gather, NoGather>::value ? 0 : GATHER_LIST_BYTES);
   cfg.dynamicSmemBytes = smem_bytes;
   cfg.stream = st;
   cfg.attrs = attr;
@@ -182,7 +184,7 @@ static int launch_gemm(const CUtensorMap& ma, const CUtensorMap& mb, const Sched
   cfg.gridDim = dim3(2 * pairs, 1, 1);
   {
     KernelScope scope(kernel_id, st);
-    if (cudaLaunchKernelEx(&cfg, kern, ma, mb, sc, ep, status) != cudaSuccess) return SAPO_ERR_CUDA;
+    if (cudaLaunchKernelEx(&cfg, kern, ma, mb, sc, ep, status, ga) != cudaSuccess) return SAPO_ERR_CUDA;
   }
   if constexpr (Epi::STREAMK) {
     // with a device-side size the number of K-split tiles is not known here: launch for the
@@ -380,12 +382,18 @@ static int64_t preferred_panel_rows(int64_t T) {
 // needs (row scales, partial sums, the scaled copy of hidden), the K-split scratch, the
 // per-sequence sums when the caller does not want them, and the panel of exponentials.
 constexpr int FUSED_MAX_SPLITS = 160;
-struct FusedLayout { size_t zy, c2, obj, seq, mask, partials, dw_acc, fixed; size_t bytes_per_row; };
-static FusedLayout fused_layout(int64_t T, int32_t H, int32_t V, int32_t S, bool out_bf16 = false) {
+struct FusedLayout { size_t zy, c2, obj, seq, mask, partials, dw_acc, boxes, n_boxes, fixed; size_t bytes_per_row; };
+static FusedLayout fused_layout(int64_t T, int32_t H, int32_t V, int32_t S, bool out_bf16 = false,
+                                bool gather = false) {
   FusedLayout L{};
   size_t off = 0;
   auto take = [&](size_t bytes) { const size_t at = off; off += round_up<size_t>(bytes, 256); return at; };
   if (out_bf16) L.dw_acc = take((size_t)V * H * 4);
+  if (gather) {      // the box list of every 128-token block (hidden rows read in place)
+    const size_t n_blocks = (size_t)ceil_div<int64_t>(T, BM);
+    L.boxes = take(n_blocks * 128 * 8);
+    L.n_boxes = take(n_blocks * 4);
+  }
   L.zy = take((size_t)T * 4);
   L.c2 = take((size_t)T * 4);
   L.obj = take((size_t)T * 4);
@@ -491,7 +499,8 @@ static int fwd_check_args(const void* hidden, const void* W_head, int32_t dtype,
 extern "C" size_t sapo_workspace_bytes(int32_t which, int64_t T, int32_t H, int32_t V, int32_t dtype) {
   using namespace sapo;
   const bool out_bf16 = (which & SAPO_WS_OUT_BF16) != 0;
-  which &= ~SAPO_WS_OUT_BF16;
+  const bool gather = (which & SAPO_WS_GATHER) != 0;
+  which &= ~(SAPO_WS_OUT_BF16 | SAPO_WS_GATHER);
   if (!shapes_ok(T, H, V) || (dtype != SAPO_DTYPE_BF16 && dtype != SAPO_DTYPE_F32)) return 0;
   if (which == SAPO_WS_FWD) {
     int sms = sm_count();
@@ -500,7 +509,7 @@ extern "C" size_t sapo_workspace_bytes(int32_t which, int64_t T, int32_t H, int3
   }
   if (which == SAPO_WS_FUSED) {
     if (dtype != SAPO_DTYPE_BF16) return 0;
-    const FusedLayout L = fused_layout(T, H, V, /*S=*/(int32_t)(T < 0x7fffffff ? T : 0x7fffffff), out_bf16);
+    const FusedLayout L = fused_layout(T, H, V, /*S=*/(int32_t)(T < 0x7fffffff ? T : 0x7fffffff), out_bf16, gather);
     return L.fixed + FUSED_CHUNK_SLACK + (size_t)preferred_panel_rows(T) * L.bytes_per_row;
   }
   if (which == SAPO_WS_BWD || which == SAPO_WS_BWD_ACTIVE) {
@@ -514,13 +523,15 @@ extern "C" size_t sapo_workspace_bytes(int32_t which, int64_t T, int32_t H, int3
 extern "C" size_t sapo_workspace_bytes_min(int32_t which, int64_t T, int32_t H, int32_t V, int32_t dtype) {
   using namespace sapo;
   const bool out_bf16 = (which & SAPO_WS_OUT_BF16) != 0;
-  if ((which & ~SAPO_WS_OUT_BF16) != SAPO_WS_BWD && (which & ~SAPO_WS_OUT_BF16) != SAPO_WS_FUSED)
+  const bool gather = (which & SAPO_WS_GATHER) != 0;
+  const int32_t flags = SAPO_WS_OUT_BF16 | SAPO_WS_GATHER;
+  if ((which & ~flags) != SAPO_WS_BWD && (which & ~flags) != SAPO_WS_FUSED)
     return sapo_workspace_bytes(which, T, H, V, dtype);
-  which &= ~SAPO_WS_OUT_BF16;
+  which &= ~flags;
   if (!shapes_ok(T, H, V) || (dtype != SAPO_DTYPE_BF16 && dtype != SAPO_DTYPE_F32)) return 0;
   if (which == SAPO_WS_FUSED) {
     if (dtype != SAPO_DTYPE_BF16) return 0;
-    const FusedLayout L = fused_layout(T, H, V, (int32_t)(T < 0x7fffffff ? T : 0x7fffffff), out_bf16);
+    const FusedLayout L = fused_layout(T, H, V, (int32_t)(T < 0x7fffffff ? T : 0x7fffffff), out_bf16, gather);
     return L.fixed + FUSED_CHUNK_SLACK + (size_t)BM * L.bytes_per_row;
   }
   const BwdLayout L = bwd_layout(T, H, V, dtype, out_bf16);
@@ -528,6 +539,48 @@ extern "C" size_t sapo_workspace_bytes_min(int32_t which, int64_t T, int32_t H, 
 }
 
 namespace sapo {
+// The LM-head projection of the forward: hidden . W^T on the tensor cores with the online
+// log-sum-exp epilogue, leaving per token one (max, sum, target logit[, entropy sum]) partial per
+// vocab split and column half.  id_offset: first vocabulary entry of W when it is a shard.
+static int fwd_project(const void* hidden, const void* W_head, int32_t dtype, int64_t T, int32_t H, int32_t V,
+                       int64_t ld_hidden, int64_t ld_W, const int32_t* ids, int32_t id_offset, const FwdLayout& L,
+                       uint8_t* ws, float* pm, float* ps, float* pz, float* pe, int32_t* status, cudaStream_t st,
+                       int* n_parts) {
+  const void* A = hidden; const void* B = W_head;
+  int64_t K = H, lda = ld_hidden, ldb = ld_W;
+  if (dtype == SAPO_DTYPE_F32) {
+    __nv_bfloat16* a3 = reinterpret_cast<__nv_bfloat16*>(ws + L.a_split);
+    __nv_bfloat16* b3 = reinterpret_cast<__nv_bfloat16*>(ws + L.b_split);
+    int rc = launch_split(static_cast<const float*>(hidden), ld_hidden, T, H, a3, 0, st);
+    if (rc != SAPO_OK) return rc;
+    rc = launch_split(static_cast<const float*>(W_head), ld_W, V, H, b3, 1, st);
+    if (rc != SAPO_OK) return rc;
+    A = a3; B = b3; K = 3 * (int64_t)H; lda = K; ldb = K;
+  }
+  CUtensorMap map_a, map_b;
+  if (!make_map(&map_a, A, K, T, lda, BM) || !make_map(&map_b, B, K, V, ldb, 128)) return SAPO_ERR_CUDA;
+  const Sched sched = make_sched(T, V, K, L.n_splits, /*m_fastest=*/true, 32, FWD_BK);
+  *n_parts = 2 * sched.units_per_m;   // one partial per vocab split and column half
+  if (pe != nullptr) {
+    FwdEpiT<true>::Params ep{ids, pm, ps, pz, pe, T, V, id_offset};
+    return launch_gemm<0, false, FwdEpiT<true>, FWD_BK, FWD_STAGES>(map_a, map_b, sched, ep, status, st, SAPO_K_FWD_GEMM);
+  }
+  FwdEpi::Params ep{ids, pm, ps, pz, nullptr, T, V, id_offset};
+  return launch_gemm<0, false, FwdEpi, FWD_BK, FWD_STAGES>(map_a, map_b, sched, ep, status, st, SAPO_K_FWD_GEMM);
+}
+
+// The loss tail over merged or unmerged partials, then the loss itself.
+static int launch_tail(const TailArgs& ta, int32_t loss_agg, float* loss, int sms, cudaStream_t st) {
+  // one block per sequence; at least enough blocks to zero-fill, at a few thousand tokens each,
+  // the outputs of tokens that belong to no sequence (T may be the caller's buffer capacity)
+  int64_t tail_blocks = ceil_div<int64_t>(ta.T, 4096);
+  if (tail_blocks < ta.S) tail_blocks = ta.S;
+  if (tail_blocks > (int64_t)sms * 8) tail_blocks = (int64_t)sms * 8;
+  { KernelScope scope(SAPO_K_LOSS_TAIL, st); loss_tail_kernel<<<(int)tail_blocks, 256, 0, st>>>(ta); }
+  { KernelScope scope(SAPO_K_LOSS_FINAL, st); loss_final_kernel<<<1, 256, 0, st>>>(ta.seq_surr, ta.cu, ta.S, ta.T, loss_agg, loss); }
+  return check_launch();
+}
+
 static int fwd_impl(const void* hidden, const void* W_head, int32_t dtype,
                     int64_t T, int32_t H, int32_t V, int64_t ld_hidden, int64_t ld_W,
                     const int32_t* ids, const float* old_logp, const float* adv,
@@ -555,47 +608,21 @@ static int fwd_impl(const void* hidden, const void* W_head, int32_t dtype,
   float* pe = want_entropy ? pz + (size_t)2 * L.n_splits * T : nullptr;
   float* seq_out = seq_surr ? seq_surr : reinterpret_cast<float*>(ws + L.total);
 
-  const void* A = hidden; const void* B = W_head;
-  int64_t K = H, lda = ld_hidden, ldb = ld_W;
-  if (dtype == SAPO_DTYPE_F32) {
-    __nv_bfloat16* a3 = reinterpret_cast<__nv_bfloat16*>(ws + L.a_split);
-    __nv_bfloat16* b3 = reinterpret_cast<__nv_bfloat16*>(ws + L.b_split);
-    int rc = launch_split(static_cast<const float*>(hidden), ld_hidden, T, H, a3, 0, st);
-    if (rc != SAPO_OK) return rc;
-    rc = launch_split(static_cast<const float*>(W_head), ld_W, V, H, b3, 1, st);
-    if (rc != SAPO_OK) return rc;
-    A = a3; B = b3; K = 3 * (int64_t)H; lda = K; ldb = K;
-  }
-  CUtensorMap map_a, map_b;
-  if (!make_map(&map_a, A, K, T, lda, BM) || !make_map(&map_b, B, K, V, ldb, 128)) return SAPO_ERR_CUDA;
-  const Sched sched = make_sched(T, V, K, L.n_splits, /*m_fastest=*/true, 32, FWD_BK);
-  int rc;
-  if (want_entropy) {
-    FwdEpiT<true>::Params ep{ids, pm, ps, pz, pe, T, V};
-    rc = launch_gemm<0, false, FwdEpiT<true>, FWD_BK, FWD_STAGES>(map_a, map_b, sched, ep, status, st, SAPO_K_FWD_GEMM);
-  } else {
-    FwdEpi::Params ep{ids, pm, ps, pz, nullptr, T, V};
-    rc = launch_gemm<0, false, FwdEpi, FWD_BK, FWD_STAGES>(map_a, map_b, sched, ep, status, st, SAPO_K_FWD_GEMM);
-  }
+  int n_parts = 0;
+  int rc = fwd_project(hidden, W_head, dtype, T, H, V, ld_hidden, ld_W, ids, /*id_offset=*/0, L, ws, pm, ps, pz, pe,
+                       status, st, &n_parts);
   if (rc != SAPO_OK) return rc;
 
   TailArgs ta{};
-  ta.pm = pm; ta.ps = ps; ta.pz = pz; ta.T = T;
+  ta.pm = pm; ta.ps = ps; ta.pz = pz; ta.T = T; ta.part_stride = T;
   ta.pe = pe; ta.entropy = h_cfg->entropy;
-  ta.n_splits = 2 * sched.units_per_m;   // one partial per vocab split and column half
+  ta.n_splits = n_parts;
   ta.ids = ids; ta.V = V; ta.old_logp = old_logp; ta.adv = adv; ta.cu = cu_seqlens; ta.S = S;
   ta.lo_edge = 1.f - h_cfg->eps_low; ta.hi_edge = 1.f + h_cfg->eps_high; ta.grad_scale = h_cfg->grad_scale;
   ta.loss_agg = h_cfg->loss_agg; ta.kl_beta = h_cfg->kl_beta; ta.ref_logp = h_cfg->ref_logp;
   ta.logp = logp; ta.lse = lse; ta.ratio = ratio; ta.surr = surr; ta.gscale = gscale; ta.seq_surr = seq_out;
   ta.status = status;
-  // one block per sequence; at least enough blocks to zero-fill, at a few thousand tokens each,
-  // the outputs of tokens that belong to no sequence (T may be the caller's buffer capacity)
-  int64_t tail_blocks = ceil_div<int64_t>(T, 4096);
-  if (tail_blocks < S) tail_blocks = S;
-  if (tail_blocks > (int64_t)sms * 8) tail_blocks = (int64_t)sms * 8;
-  { KernelScope scope(SAPO_K_LOSS_TAIL, st); loss_tail_kernel<<<(int)tail_blocks, 256, 0, st>>>(ta); }
-  { KernelScope scope(SAPO_K_LOSS_FINAL, st); loss_final_kernel<<<1, 256, 0, st>>>(seq_out, cu_seqlens, S, T, h_cfg->loss_agg, loss); }
-  return check_launch();
+  return launch_tail(ta, h_cfg->loss_agg, loss, sms, st);
 }
 }  // namespace sapo
 
@@ -610,6 +637,69 @@ extern "C" int sapo_policy_loss_fwd(const void* hidden, const void* W_head, int3
   return sapo::fwd_impl(hidden, W_head, dtype, T, H, V, ld_hidden, ld_W, ids, old_logp, adv, cu_seqlens, S, h_cfg,
                         logp, lse, ratio, surr, gscale, seq_surr, loss, workspace, workspace_bytes, status, stream,
                         /*max_splits=*/0);
+}
+
+// ------------------------------------------------------------------------------------------
+// The forward in two halves, for a vocabulary that is sharded over ranks (each rank holds rows
+// [vocab_offset, vocab_offset + V_shard) of W_head and all tokens): the projection of one shard,
+// reduced to one (max, sum, target logit) triple per token, and the loss tail over the triples of
+// all shards once they have been gathered into local memory.
+extern "C" int sapo_lmhead_lse_partial(const void* hidden, const void* W_shard, int32_t dtype,
+                                       int64_t T, int32_t H, int32_t V_shard, int64_t ld_hidden, int64_t ld_W,
+                                       const int32_t* ids, int32_t vocab_offset, float* triple,
+                                       void* workspace, size_t workspace_bytes, int32_t* status, void* stream) {
+  using namespace sapo;
+  if (!hidden || !W_shard || !ids || !triple || !workspace || !status) return SAPO_ERR_INVALID_ARG;
+  if (dtype != SAPO_DTYPE_BF16 && dtype != SAPO_DTYPE_F32) return SAPO_ERR_INVALID_ARG;
+  if (T < 1 || H < 1 || V_shard < 1 || ld_hidden < H || ld_W < H || vocab_offset < 0) return SAPO_ERR_INVALID_ARG;
+  if (!shapes_ok(T, H, V_shard)) return SAPO_ERR_UNSUPPORTED_SHAPE;
+  const int esz = dtype == SAPO_DTYPE_BF16 ? 2 : 4;
+  if (!aligned16(hidden) || !aligned16(W_shard) || !aligned16(workspace) || (ld_hidden * esz) % 16 || (ld_W * esz) % 16)
+    return SAPO_ERR_INVALID_ARG;
+  const int sms = sm_count();
+  if (sms <= 0) return SAPO_ERR_CUDA;
+  const FwdLayout L = fwd_layout(T, H, V_shard, dtype, sms, 0, /*entropy=*/false);
+  if (workspace_bytes < L.total) return SAPO_ERR_WORKSPACE_TOO_SMALL;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  uint8_t* ws = static_cast<uint8_t*>(workspace);
+  float* pm = reinterpret_cast<float*>(ws + L.partials);
+  float* ps = pm + (size_t)2 * L.n_splits * T;
+  float* pz = ps + (size_t)2 * L.n_splits * T;
+  int n_parts = 0;
+  int rc = fwd_project(hidden, W_shard, dtype, T, H, V_shard, ld_hidden, ld_W, ids, vocab_offset, L, ws, pm, ps, pz,
+                       nullptr, status, st, &n_parts);
+  if (rc != SAPO_OK) return rc;
+  int64_t blocks = ceil_div<int64_t>(T, 256);
+  if (blocks > (int64_t)sms * 8) blocks = (int64_t)sms * 8;
+  { KernelScope scope(SAPO_K_LOSS_TAIL, st); merge_partials_kernel<<<(int)blocks, 256, 0, st>>>(pm, ps, pz, n_parts, T, triple); }
+  return check_launch();
+}
+
+extern "C" int sapo_policy_loss_from_partials(const float* triples, int32_t n_parts, int64_t T, int32_t V,
+                                              const int32_t* ids, const float* old_logp, const float* adv,
+                                              const int32_t* cu_seqlens, int32_t S, const sapo_loss_cfg* h_cfg,
+                                              float* logp, float* lse, float* ratio, float* surr, float* gscale,
+                                              float* seq_surr, float* loss, int32_t* status, void* stream) {
+  using namespace sapo;
+  if (!triples || !ids || !old_logp || !adv || !cu_seqlens || !h_cfg || !logp || !lse || !ratio || !surr ||
+      !gscale || !seq_surr || !loss || !status || S < 1 || n_parts < 1 || T < 1 || V < 1)
+    return SAPO_ERR_INVALID_ARG;
+  if (!(h_cfg->eps_low >= 0.f) || !(h_cfg->eps_high >= 0.f)) return SAPO_ERR_INVALID_ARG;
+  if ((h_cfg->loss_agg != 0 && h_cfg->loss_agg != 1) || (h_cfg->kl_beta != 0.f && !h_cfg->ref_logp))
+    return SAPO_ERR_INVALID_ARG;
+  if (h_cfg->entropy != nullptr) return SAPO_ERR_UNSUPPORTED_SHAPE;   // the triples do not carry its sum
+  const int sms = sm_count();
+  if (sms <= 0) return SAPO_ERR_CUDA;
+  TailArgs ta{};
+  ta.pm = triples; ta.ps = triples + T; ta.pz = triples + 2 * T; ta.T = T; ta.part_stride = 3 * T;
+  ta.pe = nullptr; ta.entropy = nullptr;
+  ta.n_splits = n_parts;
+  ta.ids = ids; ta.V = V; ta.old_logp = old_logp; ta.adv = adv; ta.cu = cu_seqlens; ta.S = S;
+  ta.lo_edge = 1.f - h_cfg->eps_low; ta.hi_edge = 1.f + h_cfg->eps_high; ta.grad_scale = h_cfg->grad_scale;
+  ta.loss_agg = h_cfg->loss_agg; ta.kl_beta = h_cfg->kl_beta; ta.ref_logp = h_cfg->ref_logp;
+  ta.logp = logp; ta.lse = lse; ta.ratio = ratio; ta.surr = surr; ta.gscale = gscale; ta.seq_surr = seq_surr;
+  ta.status = status;
+  return launch_tail(ta, h_cfg->loss_agg, loss, sms, static_cast<cudaStream_t>(stream));
 }
 
 // ------------------------------------------------------------------------------------------
@@ -677,13 +767,13 @@ extern "C" int sapo_policy_loss_fwd_static(const void* hidden, const void* W_hea
                   scratch, (size_t)SAPO_STATIC_SCRATCH_BYTES, status, stream, max_splits);
 }
 
-extern "C" int sapo_policy_loss_bwd(const void* hidden, const void* W_head, int32_t dtype,
-                                    int64_t T, int32_t H, int32_t V, int64_t ld_hidden, int64_t ld_W,
-                                    const int32_t* ids, const float* lse, const float* gscale,
-                                    void* dhidden, void* dW_head, int32_t out_dtype, int32_t accumulate_dW,
-                                    void* workspace, size_t workspace_bytes,
-                                    int32_t* status, void* stream) {
-  using namespace sapo;
+namespace sapo {
+static int bwd_impl(const void* hidden, const void* W_head, int32_t dtype,
+                    int64_t T, int32_t H, int32_t V, int64_t ld_hidden, int64_t ld_W,
+                    const int32_t* ids, int32_t vocab_offset, const float* lse, const float* gscale,
+                    void* dhidden, void* dW_head, int32_t out_dtype, int32_t accumulate_dW,
+                    void* workspace, size_t workspace_bytes,
+                    int32_t* status, void* stream) {
   if (!hidden || !W_head || !ids || !lse || !gscale || !dhidden || !dW_head || !workspace || !status)
     return SAPO_ERR_INVALID_ARG;
   if (dtype != SAPO_DTYPE_BF16 && dtype != SAPO_DTYPE_F32) return SAPO_ERR_INVALID_ARG;
@@ -740,7 +830,7 @@ extern "C" int sapo_policy_loss_bwd(const void* hidden, const void* W_head, int3
     {
       Sched sched = make_sched(tc, V, H, 0, /*m_fastest=*/true, /*tile_align=*/64, FWD_BK);
       sched.n_cover = (int32_t)Vp;
-      DzEpi::Params ep{ids + t0, lse + t0, gscale + t0, tc, V, nvt, panel};
+      DzEpi::Params ep{ids + t0, lse + t0, gscale + t0, tc, V, nvt, panel, vocab_offset};
       int rc = launch_gemm<0, false, DzEpi, FWD_BK, FWD_STAGES>(map_h_kmajor, map_w_kmajor, sched, ep, status, st, SAPO_K_BWD_DZ);
       if (rc != SAPO_OK) return rc;
     }
@@ -755,6 +845,31 @@ extern "C" int sapo_policy_loss_bwd(const void* hidden, const void* W_head, int3
   }
   if (dw_via_acc) return launch_round_to_bf16(dw_acc, dW_head, (int64_t)V * H, accumulate_dW ? 1 : 0, st);
   return SAPO_OK;
+}
+}  // namespace sapo
+
+extern "C" int sapo_policy_loss_bwd(const void* hidden, const void* W_head, int32_t dtype,
+                                    int64_t T, int32_t H, int32_t V, int64_t ld_hidden, int64_t ld_W,
+                                    const int32_t* ids, const float* lse, const float* gscale,
+                                    void* dhidden, void* dW_head, int32_t out_dtype, int32_t accumulate_dW,
+                                    void* workspace, size_t workspace_bytes,
+                                    int32_t* status, void* stream) {
+  return sapo::bwd_impl(hidden, W_head, dtype, T, H, V, ld_hidden, ld_W, ids, 0, lse, gscale, dhidden, dW_head,
+                        out_dtype, accumulate_dW, workspace, workspace_bytes, status, stream);
+}
+
+// The same for one vocabulary shard: W_shard holds rows [vocab_offset, vocab_offset + V_shard) of
+// W_head, lse is the log-sum-exp over the WHOLE vocabulary; dhidden receives this shard's share of
+// the sum over v (to be added up over the shards), dW_shard the shard's rows of dW_head.
+extern "C" int sapo_policy_loss_bwd_shard(const void* hidden, const void* W_shard, int32_t dtype,
+                                          int64_t T, int32_t H, int32_t V_shard, int64_t ld_hidden, int64_t ld_W,
+                                          const int32_t* ids, int32_t vocab_offset, const float* lse,
+                                          const float* gscale, void* dhidden, void* dW_shard, int32_t out_dtype,
+                                          int32_t accumulate_dW, void* workspace, size_t workspace_bytes,
+                                          int32_t* status, void* stream) {
+  if (vocab_offset < 0) return SAPO_ERR_INVALID_ARG;
+  return sapo::bwd_impl(hidden, W_shard, dtype, T, H, V_shard, ld_hidden, ld_W, ids, vocab_offset, lse, gscale,
+                        dhidden, dW_shard, out_dtype, accumulate_dW, workspace, workspace_bytes, status, stream);
 }
 
 // ------------------------------------------------------------------------------------------
@@ -865,7 +980,7 @@ extern "C" int sapo_policy_loss_bwd_active(const void* hidden, const void* W_hea
       Sched sched = make_sched(tc, V, H, 0, /*m_fastest=*/true, /*tile_align=*/64, FWD_BK);
       sched.n_cover = (int32_t)Vp;
       sched.dyn_count = count; sched.dyn_dim = 1;
-      DzEpi::Params ep{ids_act + t0, lse_act + t0, g_act + t0, tc, V, nvt, panel};
+      DzEpi::Params ep{ids_act + t0, lse_act + t0, g_act + t0, tc, V, nvt, panel, 0};
       int rc = launch_gemm<0, false, DzEpi, FWD_BK, FWD_STAGES>(map_h_kmajor, map_w_kmajor, sched, ep, status, st, SAPO_K_BWD_DZ);
       if (rc != SAPO_OK) return rc;
     }
@@ -895,7 +1010,11 @@ extern "C" int sapo_policy_loss_bwd_active(const void* hidden, const void* W_hea
 // ------------------------------------------------------------------------------------------
 // Loss and both gradients in one call, without a second pass over the logits: the forward
 // epilogue leaves exp(z - c_t) in the panel, and the two backward contractions read it.
-extern "C" int sapo_policy_loss_fwd_bwd(const void* hidden, const void* W_head, int32_t dtype,
+namespace sapo {
+// Where the hidden rows are read in place: the two rollout stores and each packed token's row.
+struct HiddenSource { const void* local; const void* ext; int64_t n_local, n_ext; const int64_t* tok_src; };
+
+static int fused_impl(const void* hidden, const HiddenSource* src, const void* W_head, int32_t dtype,
                                         int64_t T, int32_t H, int32_t V, int64_t ld_hidden, int64_t ld_W,
                                         const int32_t* ids, const float* old_logp, const float* adv,
                                         const int32_t* cu_seqlens, int32_t S, const sapo_loss_cfg* h_cfg,
@@ -904,8 +1023,11 @@ extern "C" int sapo_policy_loss_fwd_bwd(const void* hidden, const void* W_head, 
                                         void* dhidden, void* dW_head, int32_t out_dtype, int32_t accumulate_dW,
                                         void* workspace, size_t workspace_bytes,
                                         int32_t* status, void* stream) {
-  using namespace sapo;
-  if (!hidden || !W_head || !ids || !old_logp || !adv || !cu_seqlens || !h_cfg || !logp || !lse ||
+  const bool gather = src != nullptr;
+  if (gather && (!src->tok_src || src->n_local < 0 || src->n_ext < 0 || (src->n_local > 0 && !src->local) ||
+                 (src->n_ext > 0 && !src->ext) || src->n_local > 0x7fffff00LL || src->n_ext > 0x7fffff00LL))
+    return SAPO_ERR_INVALID_ARG;
+  if ((!gather && !hidden) || !W_head || !ids || !old_logp || !adv || !cu_seqlens || !h_cfg || !logp || !lse ||
       !ratio || !surr || !gscale || !loss || !dhidden || !dW_head || !workspace || !status || S < 1)
     return SAPO_ERR_INVALID_ARG;
   if (dtype != SAPO_DTYPE_BF16 && dtype != SAPO_DTYPE_F32) return SAPO_ERR_INVALID_ARG;
@@ -913,9 +1035,10 @@ extern "C" int sapo_policy_loss_fwd_bwd(const void* hidden, const void* W_head, 
   if (!seq_surr && S > T) return SAPO_ERR_INVALID_ARG;   // the built-in per-sequence scratch holds T entries
   if (!shapes_ok(T, H, V)) return SAPO_ERR_UNSUPPORTED_SHAPE;
   if (dtype != SAPO_DTYPE_BF16) return SAPO_ERR_UNSUPPORTED_SHAPE;   // fp32 operands: use the separate calls
-  if (!aligned16(hidden) || !aligned16(W_head) || !aligned16(workspace) || !aligned16(dhidden) ||
+  if ((!gather && !aligned16(hidden)) || !aligned16(W_head) || !aligned16(workspace) || !aligned16(dhidden) ||
       !aligned16(dW_head) || (ld_hidden * 2) % 16 || (ld_W * 2) % 16)
     return SAPO_ERR_INVALID_ARG;
+  if (gather && (!aligned16(src->local) || !aligned16(src->ext))) return SAPO_ERR_INVALID_ARG;
   if (!(h_cfg->eps_low >= 0.f) || !(h_cfg->eps_high >= 0.f)) return SAPO_ERR_INVALID_ARG;
   if ((h_cfg->loss_agg != 0 && h_cfg->loss_agg != 1) || (h_cfg->kl_beta != 0.f && !h_cfg->ref_logp))
     return SAPO_ERR_INVALID_ARG;
@@ -923,7 +1046,7 @@ extern "C" int sapo_policy_loss_fwd_bwd(const void* hidden, const void* W_head, 
   if (sms <= 0) return SAPO_ERR_CUDA;
   if (out_dtype != SAPO_DTYPE_BF16 && out_dtype != SAPO_DTYPE_F32) return SAPO_ERR_INVALID_ARG;
   const bool out_bf16 = out_dtype == SAPO_DTYPE_BF16;
-  const FusedLayout L = fused_layout(T, H, V, (int32_t)(T < 0x7fffffff ? T : 0x7fffffff), out_bf16);
+  const FusedLayout L = fused_layout(T, H, V, (int32_t)(T < 0x7fffffff ? T : 0x7fffffff), out_bf16, gather);
   if (workspace_bytes < L.fixed + FUSED_CHUNK_SLACK + (size_t)BM * L.bytes_per_row)
     return SAPO_ERR_WORKSPACE_TOO_SMALL;
   const int64_t rows_fit =
@@ -954,23 +1077,49 @@ extern "C" int sapo_policy_loss_fwd_bwd(const void* hidden, const void* W_head, 
   const __nv_bfloat16* B = static_cast<const __nv_bfloat16*>(W_head);
   const int64_t Vp = padded_vocab(V);
   const int32_t nvt = (int32_t)(Vp / 64);
+  RowSource rows{A, nullptr, ld_hidden, nullptr, 0, 0};
+  GatherArgs ga{};
+  uint64_t* boxes = reinterpret_cast<uint64_t*>(ws + L.boxes);
+  int32_t* n_boxes = reinterpret_cast<int32_t*>(ws + L.n_boxes);
+  if (gather) {
+    rows = RowSource{static_cast<const __nv_bfloat16*>(src->local), static_cast<const __nv_bfloat16*>(src->ext),
+                     ld_hidden, src->tok_src, src->n_local, src->n_ext};
+    // boxes of 64 columns x 2^k rows over each rollout store, and the box list of every 128-token block
+    for (int side = 0; side < 2; ++side) {
+      const void* base = side == 0 ? src->local : src->ext;
+      const int64_t n = side == 0 ? src->n_local : src->n_ext;
+      for (int k = 0; k < 8; ++k)
+        if (!make_map(&ga.maps[side][k], n > 0 ? base : (const void*)W_head, H, n > 0 ? n : 1, ld_hidden, 1 << k))
+          return SAPO_ERR_CUDA;
+    }
+    const int64_t n_blocks = ceil_div<int64_t>(T, BM);
+    KernelScope scope(SAPO_K_COMPACT, st);
+    gather_boxes_kernel<<<(int)ceil_div<int64_t>(n_blocks, 128), 128, 0, st>>>(src->tok_src, T, src->n_local,
+                                                                               src->n_ext, boxes, n_boxes, status);
+  }
 
   // 1. chosen-token logits and the reference of the exponentials, all tokens
   {
     int64_t blocks = ceil_div<int64_t>(T, 8);
     if (blocks > (int64_t)sms * 8) blocks = (int64_t)sms * 8;
     KernelScope scope(SAPO_K_TARGET_LOGIT, st);
-    target_logit_kernel<<<(int)blocks, 256, 0, st>>>(A, ld_hidden, B, ld_W, ids, old_logp, T, H, V, zy, c2);
+    target_logit_kernel<<<(int)blocks, 256, 0, st>>>(rows, B, ld_W, ids, old_logp, T, H, V, zy, c2);
   }
   CUtensorMap map_w_kmajor;
   if (!make_map(&map_w_kmajor, B, H, V, ld_W, 128)) return SAPO_ERR_CUDA;
 
   for (int64_t t0 = 0; t0 < T; t0 += chunk_rows) {
     const int64_t tc = (T - t0) < chunk_rows ? (T - t0) : chunk_rows;
-    const __nv_bfloat16* A0 = A + t0 * ld_hidden;
     const int64_t panel_rows = ceil_div<int64_t>(tc, BM) * nvt * BM;
     CUtensorMap map_h_kmajor;
-    if (!make_map(&map_h_kmajor, A0, H, tc, ld_hidden, BM)) return SAPO_ERR_CUDA;
+    if (gather) {
+      map_h_kmajor = ga.maps[0][7];        // unused by the gathering kernel
+      ga.boxes = boxes + (size_t)(t0 / BM) * 128;
+      ga.n_boxes = n_boxes + t0 / BM;
+      ga.rows = tc;
+    } else if (!make_map(&map_h_kmajor, A + t0 * ld_hidden, H, tc, ld_hidden, BM)) {
+      return SAPO_ERR_CUDA;
+    }
     // 2. exponentials of the chunk -> panel, their sums per token and vocab split
     int n_splits = fwd_splits(tc, V, H, sms);
     if (n_splits > FUSED_MAX_SPLITS) n_splits = FUSED_MAX_SPLITS;
@@ -980,10 +1129,12 @@ extern "C" int sapo_policy_loss_fwd_bwd(const void* hidden, const void* W_head, 
       int rc;
       if (want_entropy) {
         ExpEpiT<true>::Params ep{c2 + t0, ps, pe, tc, V, nvt, panel};
-        rc = launch_gemm<0, false, ExpEpiT<true>, FWD_BK, FWD_STAGES>(map_h_kmajor, map_w_kmajor, fs, ep, status, st, SAPO_K_FWD_EXP);
+        rc = gather ? launch_gemm<0, false, ExpEpiT<true>, FWD_BK, FWD_STAGES, GatherArgs>(map_h_kmajor, map_w_kmajor, fs, ep, status, st, SAPO_K_FWD_EXP, ga)
+                    : launch_gemm<0, false, ExpEpiT<true>, FWD_BK, FWD_STAGES>(map_h_kmajor, map_w_kmajor, fs, ep, status, st, SAPO_K_FWD_EXP);
       } else {
         ExpEpi::Params ep{c2 + t0, ps, nullptr, tc, V, nvt, panel};
-        rc = launch_gemm<0, false, ExpEpi, FWD_BK, FWD_STAGES>(map_h_kmajor, map_w_kmajor, fs, ep, status, st, SAPO_K_FWD_EXP);
+        rc = gather ? launch_gemm<0, false, ExpEpi, FWD_BK, FWD_STAGES, GatherArgs>(map_h_kmajor, map_w_kmajor, fs, ep, status, st, SAPO_K_FWD_EXP, ga)
+                    : launch_gemm<0, false, ExpEpi, FWD_BK, FWD_STAGES>(map_h_kmajor, map_w_kmajor, fs, ep, status, st, SAPO_K_FWD_EXP);
       }
       if (rc != SAPO_OK) return rc;
     }
@@ -998,7 +1149,7 @@ extern "C" int sapo_policy_loss_fwd_bwd(const void* hidden, const void* W_head, 
       ta.loss_agg = h_cfg->loss_agg; ta.kl_beta = h_cfg->kl_beta; ta.ref_logp = h_cfg->ref_logp;
       ta.logp = logp; ta.lse = lse; ta.ratio = ratio; ta.surr = surr; ta.gscale = gscale; ta.obj = obj;
       ta.row_scale = row_scale; ta.panel = panel; ta.nvt = nvt;
-      ta.hidden = A; ta.ldh = ld_hidden; ta.H = H; ta.hs = hs; ta.status = status;
+      ta.rows = rows; ta.H = H; ta.hs = hs; ta.status = status;
       // one bit per 128-token block of the chunk that has a token with a gradient
       const bool masked = ceil_div<int64_t>(ceil_div<int64_t>(tc, BM), 32) <= MASK_WORDS_MAX;
       ta.active_mask = masked ? active_mask : nullptr;
@@ -1026,6 +1177,41 @@ extern "C" int sapo_policy_loss_fwd_bwd(const void* hidden, const void* W_head, 
   { KernelScope scope(SAPO_K_LOSS_TAIL, st); seq_mean_kernel<<<seq_blocks, 256, 0, st>>>(obj, cu_seqlens, S, T, seq_out, status); }
   { KernelScope scope(SAPO_K_LOSS_FINAL, st); loss_final_kernel<<<1, 256, 0, st>>>(seq_out, cu_seqlens, S, T, h_cfg->loss_agg, loss); }
   return check_launch();
+}
+}  // namespace sapo
+
+extern "C" int sapo_policy_loss_fwd_bwd(const void* hidden, const void* W_head, int32_t dtype,
+                                        int64_t T, int32_t H, int32_t V, int64_t ld_hidden, int64_t ld_W,
+                                        const int32_t* ids, const float* old_logp, const float* adv,
+                                        const int32_t* cu_seqlens, int32_t S, const sapo_loss_cfg* h_cfg,
+                                        float* logp, float* lse, float* ratio, float* surr, float* gscale,
+                                        float* seq_surr, float* loss,
+                                        void* dhidden, void* dW_head, int32_t out_dtype, int32_t accumulate_dW,
+                                        void* workspace, size_t workspace_bytes,
+                                        int32_t* status, void* stream) {
+  if (!hidden) return SAPO_ERR_INVALID_ARG;
+  return sapo::fused_impl(hidden, nullptr, W_head, dtype, T, H, V, ld_hidden, ld_W, ids, old_logp, adv, cu_seqlens, S,
+                          h_cfg, logp, lse, ratio, surr, gscale, seq_surr, loss, dhidden, dW_head, out_dtype,
+                          accumulate_dW, workspace, workspace_bytes, status, stream);
+}
+
+// The same with the hidden states read in place from the two rollout stores (no packed copy):
+// tok_src is what sapo_pack_rollouts wrote, n_*_tokens the number of token rows of each store.
+extern "C" int sapo_policy_loss_fwd_bwd_gather(const void* local_hidden, int64_t n_local_tokens,
+                                               const void* ext_hidden, int64_t n_ext_tokens, const int64_t* tok_src,
+                                               const void* W_head, int32_t dtype,
+                                               int64_t T, int32_t H, int32_t V, int64_t ld_hidden, int64_t ld_W,
+                                               const int32_t* ids, const float* old_logp, const float* adv,
+                                               const int32_t* cu_seqlens, int32_t S, const sapo_loss_cfg* h_cfg,
+                                               float* logp, float* lse, float* ratio, float* surr, float* gscale,
+                                               float* seq_surr, float* loss,
+                                               void* dhidden, void* dW_head, int32_t out_dtype, int32_t accumulate_dW,
+                                               void* workspace, size_t workspace_bytes,
+                                               int32_t* status, void* stream) {
+  const sapo::HiddenSource src{local_hidden, ext_hidden, n_local_tokens, n_ext_tokens, tok_src};
+  return sapo::fused_impl(nullptr, &src, W_head, dtype, T, H, V, ld_hidden, ld_W, ids, old_logp, adv, cu_seqlens, S,
+                          h_cfg, logp, lse, ratio, surr, gscale, seq_surr, loss, dhidden, dW_head, out_dtype,
+                          accumulate_dW, workspace, workspace_bytes, status, stream);
 }
 
 // ------------------------------------------------------------------------------------------

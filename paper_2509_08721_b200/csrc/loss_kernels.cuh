@@ -32,6 +32,7 @@ split_bf16_kernel(const float* __restrict__ X, int64_t ld, int64_t R, int32_t H,
 
 struct TailArgs {
   const float* pm; const float* ps; const float* pz; int32_t n_splits; int64_t T;
+  int64_t part_stride;                 // elements from one partial of a token to the next (T when packed)
   const float* pe; float* entropy;     // optional: partial sums of 2^(x - m) z, and the per-token entropy
   const int32_t* ids; int32_t V; const float* old_logp; const float* adv; const int32_t* cu; int32_t S;
   float lo_edge, hi_edge, grad_scale;
@@ -93,10 +94,10 @@ __global__ void __launch_bounds__(256) loss_tail_kernel(TailArgs a) {
     double acc = 0.0;
     for (int32_t t = t0 + threadIdx.x; t < t1; t += 256) {
       float M = -INFINITY;
-      for (int i = 0; i < a.n_splits; ++i) M = fmaxf(M, a.pm[(int64_t)i * a.T + t]);
+      for (int i = 0; i < a.n_splits; ++i) M = fmaxf(M, a.pm[(int64_t)i * a.part_stride + t]);
       float sum = 0.f, zy = 0.f, sz = 0.f;
       for (int i = 0; i < a.n_splits; ++i) {
-        const int64_t o = (int64_t)i * a.T + t;
+        const int64_t o = (int64_t)i * a.part_stride + t;
         const float scale = exp2f(a.pm[o] - M);
         sum += a.ps[o] * scale;
         zy += a.pz[o];
@@ -141,6 +142,24 @@ __global__ void __launch_bounds__(256) loss_tail_kernel(TailArgs a) {
   }
 }
 
+// The vocab-split partials of every token merged into one (max, sum, target logit) triple:
+// what a rank that holds one vocabulary shard hands to the others.  out is [3][T].
+__global__ void __launch_bounds__(256)
+merge_partials_kernel(const float* __restrict__ pm, const float* __restrict__ ps, const float* __restrict__ pz,
+                      int32_t n_splits, int64_t T, float* __restrict__ out) {
+  for (int64_t t = (int64_t)blockIdx.x * 256 + threadIdx.x; t < T; t += (int64_t)gridDim.x * 256) {
+    float M = -INFINITY;
+    for (int i = 0; i < n_splits; ++i) M = fmaxf(M, pm[(int64_t)i * T + t]);
+    float sum = 0.f, zy = 0.f;
+    for (int i = 0; i < n_splits; ++i) {
+      const int64_t o = (int64_t)i * T + t;
+      sum += ps[o] * exp2f(pm[o] - M);
+      zy += pz[o];
+    }
+    out[t] = M; out[T + t] = sum; out[2 * T + t] = zy;
+  }
+}
+
 // loss = -(1/S) sum_s seq_surr[s], or with token-level aggregation -(1/T) sum_s T_s seq_surr[s]
 __global__ void __launch_bounds__(256)
 loss_final_kernel(const float* seq_surr, const int32_t* cu, int32_t S, int64_t T, int32_t loss_agg, float* loss) {
@@ -159,6 +178,64 @@ loss_final_kernel(const float* seq_surr, const int32_t* cu, int32_t S, int64_t T
   if (threadIdx.x == 0) *loss = n > 0 ? (float)(-tot / n) : 0.f;
 }
 
+// ---------------------------------------------------------------------------- hidden rows in place
+// Where token t's hidden row is: row t of one matrix, or (tok_src given) a row of one of the two
+// rollout stores: tok_src[t] = source row, plus 2^62 for the external store, or -1 for no row.
+struct RowSource {
+  const __nv_bfloat16* base0; const __nv_bfloat16* base1; int64_t ld; const int64_t* tok_src;
+  int64_t n_rows0, n_rows1;     // rows of the two stores (tok_src given): a row outside them is not read
+  __device__ __forceinline__ const __nv_bfloat16* row(int64_t t) const {
+    if (tok_src == nullptr) return base0 + t * ld;
+    const int64_t s = tok_src[t];
+    if (s < 0) return nullptr;
+    const bool ext = (s >> 62) & 1;
+    const int64_t r = s & ((1ll << 62) - 1);
+    if (r >= (ext ? n_rows1 : n_rows0)) return nullptr;      // gather_boxes_kernel reports it
+    return (ext ? base1 : base0) + r * ld;
+  }
+};
+
+// The box list of every 128-token block for the GEMM that fetches its A rows in place (see
+// GatherArgs): maximal runs of tokens whose source rows are consecutive in one store, each run
+// cut into boxes of 2^k rows, largest first.  One thread per block; at most 128 boxes.
+// n_boxes[b] = number of boxes | rows they cover << 16.
+// A source row outside its store is reported (SAPO_ST_BAD_INDEX) and not fetched.
+__global__ void __launch_bounds__(128)
+gather_boxes_kernel(const int64_t* __restrict__ tok_src, int64_t T, int64_t n_rows0, int64_t n_rows1,
+                    uint64_t* __restrict__ boxes, int32_t* __restrict__ n_boxes, int32_t* status) {
+  const int64_t blk = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  const int64_t t_begin = blk * BM;
+  if (t_begin >= T) return;
+  const int64_t t_end = t_begin + BM < T ? t_begin + BM : T;
+  uint64_t* out = boxes + blk * 128;
+  int n = 0, rows = 0;
+  int64_t t = t_begin;
+  while (t < t_end) {
+    const int64_t s = tok_src[t];
+    if (s < 0) { ++t; continue; }                       // a slot without a token: nothing to fetch
+    const int side = (int)((s >> 62) & 1);
+    const int64_t row = s & ((1ll << 62) - 1);
+    int64_t len = 1;
+    while (t + len < t_end && tok_src[t + len] == s + len) ++len;
+    if (row + len > (side ? n_rows1 : n_rows0)) {        // would read past the store
+      raise_status(status, SAPO_ST_BAD_INDEX);
+      t += len;
+      continue;
+    }
+    int64_t done = 0;
+    while (done < len) {
+      int lg = 7;
+      while ((1ll << lg) > len - done) --lg;
+      out[n++] = (uint64_t)(t - t_begin + done) | ((uint64_t)lg << 7) | ((uint64_t)side << 10) |
+                 ((uint64_t)(row + done) << 16);
+      done += 1ll << lg;
+    }
+    rows += (int)len;
+    t += len;
+  }
+  n_boxes[blk] = n | (rows << 16);      // boxes, and the rows they bring (what the copy barrier must count)
+}
+
 // ---------------------------------------------------------------------------- fused call: small kernels
 // Before the forward pass of the fused call: the logit of the chosen token, z_y[t] = <h_t, W_y>,
 // as a plain fp32 dot product (one warp per token), and the reference of the exponentials
@@ -167,7 +244,7 @@ loss_final_kernel(const float* seq_surr, const int32_t* cu, int32_t S, int64_t T
 // log(ratio_t) otherwise: exp(z - c_t) then stays within a few powers of e of a probability.
 // c2 is c_t * log2(e).  A token id outside [0, V) gets z_y = c = 0 (the tail reports it).
 __global__ void __launch_bounds__(256)
-target_logit_kernel(const __nv_bfloat16* __restrict__ hidden, int64_t ldh, const __nv_bfloat16* __restrict__ W,
+target_logit_kernel(const RowSource rows, const __nv_bfloat16* __restrict__ W,
                     int64_t ldw, const int32_t* __restrict__ ids, const float* __restrict__ old_logp,
                     int64_t T, int32_t H, int32_t V, float* __restrict__ zy, float* __restrict__ c2) {
   const int lane = threadIdx.x & 31;
@@ -176,8 +253,9 @@ target_logit_kernel(const __nv_bfloat16* __restrict__ hidden, int64_t ldh, const
   for (int64_t t = warp; t < T; t += n_warps) {
     const int32_t y = ids[t];
     float acc = 0.f;
-    if (y >= 0 && y < V) {
-      const uint4* a = reinterpret_cast<const uint4*>(hidden + t * ldh);
+    const __nv_bfloat16* hrow = rows.row(t);
+    if (y >= 0 && y < V && hrow != nullptr) {
+      const uint4* a = reinterpret_cast<const uint4*>(hrow);
       const uint4* b = reinterpret_cast<const uint4*>(W + (int64_t)y * ldw);
       for (int i = lane; i < H / 8; i += 32) {
         const uint4 ua = a[i], ub = b[i];
@@ -211,7 +289,7 @@ struct FusedTailArgs {
   float* logp; float* lse; float* ratio; float* surr; float* gscale; float* obj;   // [T]
   float* row_scale;                                        // [tc]
   __nv_bfloat16* panel; int32_t nvt;                       // exponentials of the chunk
-  const __nv_bfloat16* hidden; int64_t ldh; int32_t H; __nv_bfloat16* hs;   // hs [tc, H] = row_scale * hidden
+  RowSource rows; int32_t H; __nv_bfloat16* hs;            // hs [tc, H] = row_scale * hidden row
   uint32_t* active_mask;   // one bit per 128-token block of the chunk (zeroed by the caller), or nullptr
   int32_t* status;
 };
@@ -298,10 +376,11 @@ __global__ void __launch_bounds__(256) fused_tail_kernel(FusedTailArgs a) {
       for (int vt = 0; vt < a.nvt; ++vt)
         row32[((((lr >> 7) * (int64_t)a.nvt + vt) * BM + (lr & 127)) * 64 >> 1) + lane] = 0u;
     }
-    const uint4* src = reinterpret_cast<const uint4*>(a.hidden + t * a.ldh);
+    const __nv_bfloat16* hrow = a.rows.row(t);
+    const uint4* src = reinterpret_cast<const uint4*>(hrow);
     uint4* dst = reinterpret_cast<uint4*>(a.hs + lr * (int64_t)a.H);
     for (int i = lane; i < a.H / 8; i += 32) {
-      uint4 x = src[i];
+      uint4 x = (hrow != nullptr && scale != 0.f) ? src[i] : make_uint4(0u, 0u, 0u, 0u);
       __nv_bfloat162* px = reinterpret_cast<__nv_bfloat162*>(&x);
       #pragma unroll
       for (int j = 0; j < 4; ++j) {

@@ -17,6 +17,7 @@ struct PackArgs {
   uint8_t* o_hid; int32_t* o_ids; float* o_old; float* o_rew;
   int32_t* cu; int32_t* seq_group; uint8_t* seq_is_ext; int32_t* seq_src;
   int32_t* tok_seq; uint8_t* tok_mask; int32_t* group_offsets;
+  int64_t* tok_src;          // optional: source row of every packed token (bit 62: external buffer)
   int32_t* n_tokens; int32_t* n_seqs;
   int64_t max_tokens; int32_t max_seqs;
   int64_t row_bytes;
@@ -129,6 +130,11 @@ __global__ void __launch_bounds__(256) pack_copy_kernel(PackArgs a) {
   // Slots past the last packed token: mask 0, sequence -1 and an all-zero row, id and log-prob, so
   // that the whole capacity can be scored without reading the token count back to the host.
   for (int64_t t = T + warp0; t < a.max_tokens; t += n_warps) {
+    if (lane == 0 && a.tok_src != nullptr) a.tok_src[t] = -1;
+    if (a.o_hid == nullptr) {
+      if (lane == 0) { a.o_ids[t] = 0; a.o_old[t] = 0.f; a.tok_seq[t] = -1; a.tok_mask[t] = 0; }
+      continue;
+    }
     uint8_t* to = a.o_hid + t * a.row_bytes;
     if (vec) {
       uint4* t4 = reinterpret_cast<uint4*>(to);
@@ -168,8 +174,14 @@ __global__ void __launch_bounds__(256) pack_copy_kernel(PackArgs a) {
         a.o_old[t] = a.old[side][src];
         a.tok_seq[t] = s;
         a.tok_mask[t] = 1;
+        if (a.tok_src != nullptr) a.tok_src[t] = src | ((int64_t)side << 62);
       }
     };
+    if (a.o_hid == nullptr) {
+      // no copy of the hidden rows was asked for (the caller reads them in place through tok_src)
+      for (int i = 0; i < tpw && t0 + i < T; ++i) finish(t0 + i, locate(t0 + i));
+      continue;
+    }
     for (int i = 0; i < tpw; i += 2) {
       const int64_t ta = t0 + i, tb = ta + 1;
       if (ta >= T) break;
@@ -249,9 +261,10 @@ extern "C" int sapo_pack_rollouts(const sapo_rollout_buf* h_local, const sapo_ro
   // every array a kernel will touch must be there: a NULL would only show as a device fault
   if (h_out->max_seqs > 0 && (!h_out->rewards || !h_out->seq_group || !h_out->seq_is_ext || !h_out->seq_src))
     return SAPO_ERR_INVALID_ARG;
-  if (h_out->max_tokens > 0 && (!h_out->hidden || !h_out->ids || !h_out->old_logp || !h_out->tok_seq ||
-                                !h_out->tok_mask))
+  if (h_out->max_tokens > 0 && (!h_out->ids || !h_out->old_logp || !h_out->tok_seq || !h_out->tok_mask))
     return SAPO_ERR_INVALID_ARG;
+  // the packed copy of the hidden rows is optional, but then the map to the source rows is not
+  if (h_out->max_tokens > 0 && !h_out->hidden && !h_out->tok_src) return SAPO_ERR_INVALID_ARG;
   // (the index lists may be NULL: a side nobody picks from has an empty list, and only the
   // device knows the list lengths; the scan never reads an empty list)
   const sapo_rollout_buf* src_bufs[2] = {h_local, h_ext};
@@ -271,11 +284,11 @@ extern "C" int sapo_pack_rollouts(const sapo_rollout_buf* h_local, const sapo_ro
   a.o_hid = static_cast<uint8_t*>(h_out->hidden); a.o_ids = h_out->ids; a.o_old = h_out->old_logp;
   a.o_rew = h_out->rewards; a.cu = h_out->cu_seqlens; a.seq_group = h_out->seq_group;
   a.seq_is_ext = h_out->seq_is_ext; a.seq_src = h_out->seq_src; a.tok_seq = h_out->tok_seq;
-  a.tok_mask = h_out->tok_mask; a.group_offsets = h_out->group_offsets;
+  a.tok_mask = h_out->tok_mask; a.group_offsets = h_out->group_offsets; a.tok_src = h_out->tok_src;
   a.n_tokens = h_out->n_tokens; a.n_seqs = h_out->n_seqs;
   a.max_tokens = h_out->max_tokens; a.max_seqs = h_out->max_seqs;
   a.row_bytes = (int64_t)H * (dtype == SAPO_DTYPE_BF16 ? 2 : 4);
-  if (!aligned16(a.o_hid) || !aligned16(a.hid[0]) || !aligned16(a.hid[1])) {
+  if (a.o_hid != nullptr && (!aligned16(a.o_hid) || !aligned16(a.hid[0]) || !aligned16(a.hid[1]))) {
     if ((a.row_bytes & 15) == 0) return SAPO_ERR_INVALID_ARG;
   }
   a.status = status;

@@ -56,7 +56,11 @@ class PolicyScorer:
         self.max_tokens, self.max_seqs, self.max_q = int(max_tokens), int(max_seqs), int(max_questions)
         self.eps_low, self.eps_high = float(eps_low), float(eps_high)
         self.adv_eps, self.ddof, self.grad_scale = float(adv_eps), int(ddof), float(grad_scale)
-        self.packed = B.alloc_packed(self.max_tokens, self.max_seqs, self.max_q, self.H, self.dtype, device)
+        # "gather": the single-pass call with the hidden rows read in place from the rollout stores
+        # (the pack copies no hidden rows)
+        self.backward = backward if backward is not None else ("active" if active_backward else "dense")
+        self.packed = B.alloc_packed(self.max_tokens, self.max_seqs, self.max_q, self.H, self.dtype, device,
+                                     copy_hidden=self.backward != "gather")
         self.adv = torch.empty(self.max_seqs, dtype=torch.float32, device=device)
         self.fwd = B.alloc_fwd_outputs(self.max_tokens, self.max_seqs, device)
         # per-token entropy of the policy's distribution, if asked for (a by-product of the forward)
@@ -68,11 +72,11 @@ class PolicyScorer:
         # how the gradients are formed: "dense" = forward call, then the backward call that
         # recomputes the logits; "active" = the same over tokens with a non-zero gradient factor
         # only; "fused" = one call that passes over the logits once (bf16 operands)
-        self.backward = backward if backward is not None else ("active" if active_backward else "dense")
-        if self.backward not in ("dense", "active", "fused"):
+        if self.backward not in ("dense", "active", "fused", "gather"):
             raise ValueError(f"unknown backward mode {self.backward!r}")
         self.active_backward = self.backward == "active"
-        which = {"dense": B.WS_BWD, "active": B.WS_BWD_ACTIVE, "fused": B.WS_FUSED}[self.backward]
+        which = {"dense": B.WS_BWD, "active": B.WS_BWD_ACTIVE, "fused": B.WS_FUSED,
+                 "gather": B.WS_FUSED | B.WS_GATHER}[self.backward]
         nb = B.sapo_workspace_bytes(which, self.max_tokens, self.H, self.V, self.dcode)
         if nb == 0:
             raise B.SapoError(f"backward mode {self.backward!r} does not support these operands")
@@ -93,6 +97,12 @@ class PolicyScorer:
         B.sapo_group_advantages(p["rewards"], go, self.adv_eps, self.ddof, self.adv, None, None,
                                 self.status)
         cu = p["cu_seqlens"][:S + 1]
+        if self.backward == "gather":
+            B.sapo_policy_loss_fwd_bwd_gather(local.hidden, ext.hidden, p["tok_src"], self.W, p["ids"],
+                                              p["old_logp"], self.adv, cu, self.eps_low, self.eps_high,
+                                              self.grad_scale, self.fwd, self.dhidden, self.dW, False,
+                                              self.workspace, self.status, T=T, entropy=self.entropy)
+            return StepResult(self.fwd["loss"], self.fwd, self.dhidden, self.dW, p, self.adv)
         if self.backward == "fused":
             B.sapo_policy_loss_fwd_bwd(p["hidden"], self.W, p["ids"], p["old_logp"], self.adv, cu,
                                        self.eps_low, self.eps_high, self.grad_scale, self.fwd,

@@ -140,3 +140,42 @@ def test_a_bounded_wait_that_runs_out_sets_the_status_bit_and_leaves_the_context
     # a limit outside the allowed range is refused on the host
     with pytest.raises(B.SapoError):
         B.sapo_debug_wait_timeout(10**9, status)
+
+
+@pytest.mark.parametrize("V,parts", [(2500, 2), (1000, 3)])
+def test_vocabulary_shards_on_one_device_add_up_to_the_unsharded_call(V, parts):
+    """The three shard entry points, run for every shard in turn on one GPU (no rank waits for
+    another): the gathered triples give the same forward outputs as the unsharded call, the
+    shards' dW rows and the sum of their dhidden shares match the oracle."""
+    from paper_2509_08721_b200.vocab_parallel import CudaBackend, shard_bounds
+    batch = gen.make_batch(_recipe(V=V, Q=3), 81)
+    gen.install_old_logp(batch, U.oracle_current_logp(batch))
+    b = batch.built
+    T, S, H = batch.T, batch.S, batch.H
+    adv = np.linspace(-1, 1, S).astype(np.float32)
+    hidden, W, ids = U.to_torch(b.hidden), U.to_torch(batch.W), U.to_torch(b.ids)
+    old, adv_d, cu = U.to_torch(b.old_logp), U.to_torch(adv), U.to_torch(b.cu_seqlens)
+    be, status = CudaBackend(), B.new_status()
+    triples = torch.empty(parts, 3, T, device="cuda")
+    spans = [shard_bounds(V, parts, r) for r in range(parts)]
+    for r, (lo, hi) in enumerate(spans):
+        be.lse_partial(hidden, W[lo:hi], ids, lo, triples[r], status)
+    out = B.alloc_fwd_outputs(T, S)
+    be.loss_from_partials(triples, V, ids, old, adv_d, cu, 0.2, 0.28, 1.0, out, status)
+    dH = torch.zeros(T, H, device="cuda")
+    dW = torch.empty(V, H, device="cuda")
+    for lo, hi in spans:
+        share = torch.empty(T, H, device="cuda")
+        be.bwd_shard(hidden, W[lo:hi], ids, lo, out["lse"], out["gscale"], share, dW[lo:hi], status)
+        dH += share
+    torch.cuda.synchronize()
+    assert status.item() == 0
+    ref = orc.policy_loss_fwd(gen.as_f32(b.hidden), gen.as_f32(batch.W), b.ids, b.old_logp, adv, b.cu_seqlens,
+                              0.2, 0.28)
+    grads = orc.policy_loss_bwd(gen.as_f32(b.hidden), gen.as_f32(batch.W), b.ids, ref["lse"], ref["gscale"])
+    U.check_forward(out, ref, adv.astype(np.float64), b.cu_seqlens, 0.2, 0.28)
+    U.check_loss(float(out["loss"].item()), ref["loss"], adv.astype(np.float64))
+    assert U.rel_fro(dH.cpu().numpy(), grads["dhidden"]) <= U.TOL_GRAD_FRO
+    assert U.rel_fro(dW.cpu().numpy(), grads["dW"]) <= U.TOL_GRAD_FRO
+    whole = U.gpu_scores(hidden, W, ids, old, adv_d, cu, 0.2, 0.28, want_bwd=False)
+    assert (out["logp"] - whole["logp"]).abs().max().item() <= 1e-5
