@@ -374,7 +374,7 @@ def measure(torch, dist, B, gen, replicas, PolicyScorer, _to_dev, args, workload
     m.t_act = int((g != 0).sum().item())
     if backward == "active":
         m.t_exec = int(scorer.n_active.item())
-    elif backward == "fused" and H >= 256:
+    elif backward in ("fused", "gather") and H >= 256:
         pad = (-T) % 128                 # whole 128-token blocks without any gradient are left out
         gp = torch.nn.functional.pad(g, (0, pad)).view(-1, 128)
         m.t_exec = min(T, 128 * int((gp != 0).any(dim=1).sum().item()))
@@ -471,7 +471,7 @@ def run_ours(args):
         gemm_ms = sum(gemm[k]["ms"] for k in gemm) / ksteps
         f_alg = 2.0 * T * V * H + 4.0 * t_act * V * H
         # the separate backward recomputes the logits (one more contraction); the fused call does not
-        f_exec = 2.0 * T * V * H + (4.0 if args.backward == "fused" else 6.0) * t_exec * V * H
+        f_exec = 2.0 * T * V * H + (4.0 if args.backward in ("fused", "gather") else 6.0) * t_exec * V * H
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
@@ -557,11 +557,12 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--hbm-only", action="store_true",
                     help="run only the scaled pack / advantages / Adam bandwidth measurement")
-    ap.add_argument("--backward", default=None, choices=["dense", "active", "fused"],
+    ap.add_argument("--backward", default=None, choices=["dense", "active", "fused", "gather"],
                     help="dense: forward call, then the backward call that recomputes the logits; "
                          "active: the same over the tokens whose gradient factor is non-zero only; "
                          "fused: one call that passes over the logits once (bf16 workloads; the default "
-                         "for them, with the separate calls timed beside it)")
+                         "for them, with the separate calls timed beside it); gather: the same call reading "
+                         "the hidden states in place from the rollout buffers (the pack copies none)")
     ap.add_argument("--length-div", type=int, default=1,
                     help="divide every completion length (a small case of the same kernels for profiling)")
     ap.add_argument("--ext-fraction", type=float, default=None,

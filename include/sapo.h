@@ -464,6 +464,12 @@ int64_t sapo_launch_count(void);
  * then sets the bit in *status.  For tests of a caller's error handling. */
 int sapo_debug_wait_timeout(int64_t limit_clocks, int32_t* status, void* stream);
 
+/* Checked builds (the library compiled with -DSAPO_BOUNDS_CHECK, see build.py): the kernels compare
+ * every index they compute before a global-memory access with the extent of its array, count a
+ * violation and leave the access out.  Returns the number of violations counted so far in this
+ * process, or -1 when the library is a regular build. */
+int64_t sapo_debug_bounds_violations(void);
+
 /* Text for a return code. */
 const char* sapo_status_string(int32_t code);
 

@@ -33,7 +33,7 @@ EXPORTS = ("sapo_pack_rollouts", "sapo_group_advantages", "sapo_policy_loss_fwd"
            "sapo_policy_loss_bwd", "sapo_workspace_bytes", "sapo_workspace_bytes_min",
            "sapo_status_string", "sapo_timing_enable", "sapo_timing_read", "sapo_launch_count",
            "sapo_policy_loss_fwd_static", "sapo_policy_loss_bwd_active", "sapo_policy_loss_fwd_bwd",
-           "sapo_select_external", "sapo_group_advantages_warp", "sapo_debug_wait_timeout",
+           "sapo_select_external", "sapo_group_advantages_warp", "sapo_debug_wait_timeout", "sapo_debug_bounds_violations",
            "sapo_policy_loss_fwd_bwd_gather", "sapo_lmhead_lse_partial", "sapo_policy_loss_from_partials", "sapo_policy_loss_bwd_shard",
            "sapo_select_workspace_bytes", "sapo_adam_step")
 STATIC_SCRATCH_BYTES = 4 * 1024 * 1024
@@ -136,6 +136,8 @@ def load() -> C.CDLL:
                                                i32, i32, vp, sz, vp, vp]
     lib.sapo_debug_wait_timeout.restype = C.c_int
     lib.sapo_debug_wait_timeout.argtypes = [i64, vp, vp]
+    lib.sapo_debug_bounds_violations.restype = C.c_int64
+    lib.sapo_debug_bounds_violations.argtypes = []
     lib.sapo_launch_count.restype = C.c_int64
     lib.sapo_launch_count.argtypes = []
     lib.sapo_status_string.restype = C.c_char_p

@@ -13,6 +13,25 @@ __device__ __forceinline__ void raise_status(int32_t* status, int32_t bit) {
   if (status != nullptr) atomicOr(status, bit);
 }
 
+// Checked builds (-DSAPO_BOUNDS_CHECK; the stand-in for a memory checker): every index a kernel
+// computes from its arguments or its data before a global-memory access is compared with the
+// extent of the array; a violation is counted and the access left out.  Each translation unit
+// counts for itself (sapo_debug_bounds_violations adds the counters up).  In regular builds the
+// macro is constant true and costs nothing.
+#ifdef SAPO_BOUNDS_CHECK
+static __device__ unsigned long long g_bounds_violations = 0;
+#define SAPO_IN_BOUNDS(cond) ((cond) ? true : (atomicAdd(&g_bounds_violations, 1ull), false))
+static inline long long read_bounds_violations() {
+  unsigned long long v = 0;
+  return cudaMemcpyFromSymbol(&v, g_bounds_violations, sizeof(v)) == cudaSuccess ? (long long)v : -1;
+}
+#else
+#define SAPO_IN_BOUNDS(cond) (true)
+static inline long long read_bounds_violations() { return 0; }
+#endif
+long long bounds_violations_pack();
+long long bounds_violations_lmhead();
+
 inline int check_launch() {
   return cudaGetLastError() == cudaSuccess ? SAPO_OK : SAPO_ERR_CUDA;
 }

@@ -18,8 +18,10 @@ using namespace umma;
 // issuer 4-5 % more cycles per launch.)
 // 16 finished bf16 entries (32 bytes, one sector) of a panel row: columns [col0, col0 + 16) of the
 // tile row `r` of token block `tile_row0`.
-__device__ __forceinline__ void store_panel_16(__nv_bfloat16* panel, int r, int tile_row0, int col0,
-                                               const uint32_t (&w)[8]) {
+__device__ __forceinline__ void store_panel_16(__nv_bfloat16* panel, int64_t panel_rows, int r, int tile_row0,
+                                               int col0, const uint32_t (&w)[8]) {
+  const int64_t prow = (int64_t)tile_row0 + (int64_t)(col0 >> 6) * BM + r;
+  if (!SAPO_IN_BOUNDS(prow >= 0 && prow < panel_rows && r < BM)) return;
   uint8_t* dst = reinterpret_cast<uint8_t*>(panel) +
                  ((size_t)tile_row0 + (size_t)(col0 >> 6) * BM + (size_t)r) * 128 + (size_t)(col0 & 63) * 2;
   asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
@@ -41,6 +43,7 @@ struct FwdEpiT {
     float* pe;                                             // ENT: partial sums of 2^(x - m) z
     int64_t T; int32_t V;
     int32_t id_offset;                                     // first vocabulary entry of W (a vocab shard), else 0
+    int32_t parts_cap;                                     // partials per token the arrays hold (checked builds)
   };
   float m, s, zy, sz; int32_t y; int64_t row;
   __device__ __forceinline__ void begin_unit(const Params& p, int mb, int r) {
@@ -78,7 +81,7 @@ struct FwdEpiT {
   }
   // two threads share a row (one per column half of the tiles): each leaves its own partial
   __device__ __forceinline__ void end_unit(const Params& p, int un, int col_half) {
-    if (row < p.T) {
+    if (row < p.T && SAPO_IN_BOUNDS(2 * un + col_half < p.parts_cap)) {
       const int64_t o = (int64_t)(2 * un + col_half) * p.T + row;
       p.pm[o] = m; p.ps[o] = s; p.pz[o] = zy;
       if constexpr (ENT) p.pe[o] = sz;
@@ -104,6 +107,7 @@ struct DzEpi {
     int64_t M; int32_t V; int32_t nvt;
     __nv_bfloat16* panel;
     int32_t id_offset;     // first vocabulary entry of W (a vocab shard), else 0
+    int64_t panel_rows;    // 128-byte rows the panel holds (checked builds)
   };
   float g, l2; int32_t y; int32_t tile_row0; int r; bool in_panel;
   __device__ __forceinline__ void begin_unit(const Params& p, int mb, int r_) {
@@ -126,8 +130,8 @@ struct DzEpi {
     if (g == 0.f) {
       #pragma unroll
       for (int j = 0; j < 8; ++j) w[j] = 0u;
-      store_panel_16(p.panel, r, tile_row0, col0, w);
-      store_panel_16(p.panel, r, tile_row0, col0 + 16, w);
+      store_panel_16(p.panel, p.panel_rows, r, tile_row0, col0, w);
+      store_panel_16(p.panel, p.panel_rows, r, tile_row0, col0 + 16, w);
       return;
     }
     const float ng = -g;
@@ -149,7 +153,7 @@ struct DzEpi {
         __nv_bfloat162 b2 = __floats2bfloat162_rn(v[16 * h + 2 * j], v[16 * h + 2 * j + 1]);
         w[j] = *reinterpret_cast<uint32_t*>(&b2);
       }
-      store_panel_16(p.panel, r, tile_row0, col0 + 16 * h, w);
+      store_panel_16(p.panel, p.panel_rows, r, tile_row0, col0 + 16 * h, w);
     }
   }
   __device__ __forceinline__ void group_end(const Params&, int) {}
@@ -175,6 +179,8 @@ struct ExpEpiT {
     float* pe;            // ENT: [2 * n_splits][M] partial sums of e z
     int64_t M; int32_t V; int32_t nvt;
     __nv_bfloat16* panel;
+    int64_t panel_rows;   // 128-byte rows the panel holds, and
+    int32_t parts_cap;    // partials per token the arrays hold (checked builds)
   };
   float c, sum, sz; int32_t tile_row0; int r; bool valid, in_panel; int64_t row;
   __device__ __forceinline__ void begin_unit(const Params& p, int mb, int r_) {
@@ -193,8 +199,8 @@ struct ExpEpiT {
     if (!valid || col0 >= p.V) {
       #pragma unroll
       for (int j = 0; j < 8; ++j) w[j] = 0u;
-      store_panel_16(p.panel, r, tile_row0, col0, w);
-      store_panel_16(p.panel, r, tile_row0, col0 + 16, w);
+      store_panel_16(p.panel, p.panel_rows, r, tile_row0, col0, w);
+      store_panel_16(p.panel, p.panel_rows, r, tile_row0, col0 + 16, w);
       return;
     }
     // every 16 finished columns (32 bytes of the row) are stored at once: see DzEpi
@@ -220,13 +226,13 @@ struct ExpEpiT {
         __nv_bfloat162 b2 = __floats2bfloat162_rn(v[16 * h + 2 * j], v[16 * h + 2 * j + 1]);
         w[j] = *reinterpret_cast<uint32_t*>(&b2);
       }
-      store_panel_16(p.panel, r, tile_row0, col0 + 16 * h, w);
+      store_panel_16(p.panel, p.panel_rows, r, tile_row0, col0 + 16 * h, w);
     }
   }
   __device__ __forceinline__ void group_end(const Params&, int) {}
   // two threads share a row (one per column half of the tiles): each leaves its own partial
   __device__ __forceinline__ void end_unit(const Params& p, int un, int col_half) {
-    if (valid) {
+    if (valid && SAPO_IN_BOUNDS(2 * un + col_half < p.parts_cap)) {
       p.ps[(int64_t)(2 * un + col_half) * p.M + row] = sum;
       if constexpr (ENT) p.pe[(int64_t)(2 * un + col_half) * p.M + row] = sz;
     }
@@ -261,7 +267,8 @@ struct StoreEpi {
   // to their packed positions)
   // row_scale (optional): factor applied to each accumulator row before it is stored
   struct Params { void* C; int64_t ldc; int64_t M; int32_t N; int32_t accumulate; float* partials;
-                  const int32_t* row_map; const float* row_scale; int32_t out_bf16; };
+                  const int32_t* row_map; const float* row_scale; int32_t out_bf16;
+                  int64_t out_rows; int32_t parts_cap; };   // rows of C, K-split parts the scratch holds (checked builds)
   template <class P> __device__ static void set_dynamic(P& p, const Sched& s) {
     if (s.dyn_dim == 1) p.M = *s.dyn_count;
   }
@@ -271,6 +278,7 @@ struct StoreEpi {
     valid = row < p.M;
     scale = (valid && p.row_scale != nullptr) ? p.row_scale[row] : 1.f;
     if (valid && p.row_map != nullptr) row = p.row_map[row];
+    if (valid && !SAPO_IN_BOUNDS(row >= 0 && row < p.out_rows)) valid = false;
     part = nullptr;
   }
   // a K-split part of a tile goes to scratch slot `slot` instead: rows [128 rank, +128) of a
@@ -279,6 +287,7 @@ struct StoreEpi {
     n0 = n0_;
     part = slot < 0 ? nullptr
                     : p.partials + ((size_t)slot * PAIR_M + (size_t)(rank * BM + r)) * part_ld;
+    if (slot >= 0 && !SAPO_IN_BOUNDS(slot < p.parts_cap)) { part = nullptr; valid = false; }
   }
   template <int HALF>
   __device__ __forceinline__ void chunk(const Params& p, float (&v)[32], int col0) {

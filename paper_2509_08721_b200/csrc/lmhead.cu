@@ -275,8 +275,8 @@ static int launch_grad_gemms(const __nv_bfloat16* panel, int64_t panel_rows, int
                              int64_t tc, int32_t H, int32_t V, int64_t Vp, void* dhidden, bool dh_bf16,
                              const float* row_scale, void* dW_head, bool dw_bf16, int accumulate, float* partials,
                              const uint32_t* active_mask, int32_t* status, cudaStream_t st) {
-  StoreEpi::Params ep_h{dhidden, H, tc, H, 0, partials, nullptr, row_scale, dh_bf16 ? 1 : 0};
-  StoreEpi::Params ep_w{dW_head, H, V, H, accumulate, partials, nullptr, nullptr, dw_bf16 ? 1 : 0};
+  StoreEpi::Params ep_h{dhidden, H, tc, H, 0, partials, nullptr, row_scale, dh_bf16 ? 1 : 0, tc, MAX_PARTS_SCRATCH};
+  StoreEpi::Params ep_w{dW_head, H, V, H, accumulate, partials, nullptr, nullptr, dw_bf16 ? 1 : 0, V, MAX_PARTS_SCRATCH};
   if (use_wide_tiles(H)) {
     CUtensorMap map_p_tile, map_p_half, map_w64, map_x64;
     if (!make_map(&map_p_tile, panel, 64, panel_rows, 64, BM) || !make_map(&map_p_half, panel, 64, panel_rows, 64, 64) ||
@@ -562,10 +562,10 @@ static int fwd_project(const void* hidden, const void* W_head, int32_t dtype, in
   const Sched sched = make_sched(T, V, K, L.n_splits, /*m_fastest=*/true, 32, FWD_BK);
   *n_parts = 2 * sched.units_per_m;   // one partial per vocab split and column half
   if (pe != nullptr) {
-    FwdEpiT<true>::Params ep{ids, pm, ps, pz, pe, T, V, id_offset};
+    FwdEpiT<true>::Params ep{ids, pm, ps, pz, pe, T, V, id_offset, 2 * L.n_splits};
     return launch_gemm<0, false, FwdEpiT<true>, FWD_BK, FWD_STAGES>(map_a, map_b, sched, ep, status, st, SAPO_K_FWD_GEMM);
   }
-  FwdEpi::Params ep{ids, pm, ps, pz, nullptr, T, V, id_offset};
+  FwdEpi::Params ep{ids, pm, ps, pz, nullptr, T, V, id_offset, 2 * L.n_splits};
   return launch_gemm<0, false, FwdEpi, FWD_BK, FWD_STAGES>(map_a, map_b, sched, ep, status, st, SAPO_K_FWD_GEMM);
 }
 
@@ -830,7 +830,7 @@ static int bwd_impl(const void* hidden, const void* W_head, int32_t dtype,
     {
       Sched sched = make_sched(tc, V, H, 0, /*m_fastest=*/true, /*tile_align=*/64, FWD_BK);
       sched.n_cover = (int32_t)Vp;
-      DzEpi::Params ep{ids + t0, lse + t0, gscale + t0, tc, V, nvt, panel, vocab_offset};
+      DzEpi::Params ep{ids + t0, lse + t0, gscale + t0, tc, V, nvt, panel, vocab_offset, panel_rows};
       int rc = launch_gemm<0, false, DzEpi, FWD_BK, FWD_STAGES>(map_h_kmajor, map_w_kmajor, sched, ep, status, st, SAPO_K_BWD_DZ);
       if (rc != SAPO_OK) return rc;
     }
@@ -980,7 +980,7 @@ extern "C" int sapo_policy_loss_bwd_active(const void* hidden, const void* W_hea
       Sched sched = make_sched(tc, V, H, 0, /*m_fastest=*/true, /*tile_align=*/64, FWD_BK);
       sched.n_cover = (int32_t)Vp;
       sched.dyn_count = count; sched.dyn_dim = 1;
-      DzEpi::Params ep{ids_act + t0, lse_act + t0, g_act + t0, tc, V, nvt, panel, 0};
+      DzEpi::Params ep{ids_act + t0, lse_act + t0, g_act + t0, tc, V, nvt, panel, 0, panel_rows};
       int rc = launch_gemm<0, false, DzEpi, FWD_BK, FWD_STAGES>(map_h_kmajor, map_w_kmajor, sched, ep, status, st, SAPO_K_BWD_DZ);
       if (rc != SAPO_OK) return rc;
     }
@@ -988,7 +988,8 @@ extern "C" int sapo_policy_loss_bwd_active(const void* hidden, const void* W_hea
       Sched sched = make_sched(tc, H, Vp, 0, /*m_fastest=*/false);
       sched.panel_nvt = nvt;
       sched.dyn_count = count; sched.dyn_dim = 1;
-      StoreEpi::Params ep{dhidden, H, tc, H, 0, partials, act_idx + t0, nullptr, out_bf16 ? 1 : 0};   // rows go back to their tokens
+      StoreEpi::Params ep{dhidden, H, tc, H, 0, partials, act_idx + t0, nullptr, out_bf16 ? 1 : 0, T,
+                          MAX_PARTS_SCRATCH};   // rows go back to their tokens
       int rc = launch_gemm<2, true, StoreEpi>(map_p_two, map_w_mn, sched, ep, status, st, SAPO_K_BWD_DH);
       if (rc != SAPO_OK) return rc;
     }
@@ -998,7 +999,7 @@ extern "C" int sapo_policy_loss_bwd_active(const void* hidden, const void* W_hea
       sched.panel_nvt = nvt;
       sched.dyn_count = count; sched.dyn_dim = 2; sched.skip_if_empty = acc;
       StoreEpi::Params ep{dw_via_acc ? (void*)dw_acc : dW_head, H, V, H, acc, partials, nullptr, nullptr,
-                          (out_bf16 && !dw_via_acc) ? 1 : 0};
+                          (out_bf16 && !dw_via_acc) ? 1 : 0, V, MAX_PARTS_SCRATCH};
       int rc = launch_gemm<3, true, StoreEpi>(map_p_tile, map_h_mn, sched, ep, status, st, SAPO_K_BWD_DW);
       if (rc != SAPO_OK) return rc;
     }
@@ -1128,11 +1129,11 @@ static int fused_impl(const void* hidden, const HiddenSource* src, const void* W
     {
       int rc;
       if (want_entropy) {
-        ExpEpiT<true>::Params ep{c2 + t0, ps, pe, tc, V, nvt, panel};
+        ExpEpiT<true>::Params ep{c2 + t0, ps, pe, tc, V, nvt, panel, panel_rows, 2 * FUSED_MAX_SPLITS};
         rc = gather ? launch_gemm<0, false, ExpEpiT<true>, FWD_BK, FWD_STAGES, GatherArgs>(map_h_kmajor, map_w_kmajor, fs, ep, status, st, SAPO_K_FWD_EXP, ga)
                     : launch_gemm<0, false, ExpEpiT<true>, FWD_BK, FWD_STAGES>(map_h_kmajor, map_w_kmajor, fs, ep, status, st, SAPO_K_FWD_EXP);
       } else {
-        ExpEpi::Params ep{c2 + t0, ps, nullptr, tc, V, nvt, panel};
+        ExpEpi::Params ep{c2 + t0, ps, nullptr, tc, V, nvt, panel, panel_rows, 2 * FUSED_MAX_SPLITS};
         rc = gather ? launch_gemm<0, false, ExpEpi, FWD_BK, FWD_STAGES, GatherArgs>(map_h_kmajor, map_w_kmajor, fs, ep, status, st, SAPO_K_FWD_EXP, ga)
                     : launch_gemm<0, false, ExpEpi, FWD_BK, FWD_STAGES>(map_h_kmajor, map_w_kmajor, fs, ep, status, st, SAPO_K_FWD_EXP);
       }
@@ -1148,7 +1149,7 @@ static int fused_impl(const void* hidden, const HiddenSource* src, const void* W
       ta.lo_edge = 1.f - h_cfg->eps_low; ta.hi_edge = 1.f + h_cfg->eps_high; ta.grad_scale = h_cfg->grad_scale;
       ta.loss_agg = h_cfg->loss_agg; ta.kl_beta = h_cfg->kl_beta; ta.ref_logp = h_cfg->ref_logp;
       ta.logp = logp; ta.lse = lse; ta.ratio = ratio; ta.surr = surr; ta.gscale = gscale; ta.obj = obj;
-      ta.row_scale = row_scale; ta.panel = panel; ta.nvt = nvt;
+      ta.row_scale = row_scale; ta.panel = panel; ta.nvt = nvt; ta.panel_rows = panel_rows;
       ta.rows = rows; ta.H = H; ta.hs = hs; ta.status = status;
       // one bit per 128-token block of the chunk that has a token with a gradient
       const bool masked = ceil_div<int64_t>(ceil_div<int64_t>(tc, BM), 32) <= MASK_WORDS_MAX;
@@ -1213,6 +1214,10 @@ extern "C" int sapo_policy_loss_fwd_bwd_gather(const void* local_hidden, int64_t
                           h_cfg, logp, lse, ratio, surr, gscale, seq_surr, loss, dhidden, dW_head, out_dtype,
                           accumulate_dW, workspace, workspace_bytes, status, stream);
 }
+
+namespace sapo {
+long long bounds_violations_lmhead() { return read_bounds_violations(); }
+}  // namespace sapo
 
 // ------------------------------------------------------------------------------------------
 // The bounded wait, made to run out on purpose: one thread waits on a barrier nobody arrives at.

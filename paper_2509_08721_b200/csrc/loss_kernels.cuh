@@ -226,6 +226,7 @@ gather_boxes_kernel(const int64_t* __restrict__ tok_src, int64_t T, int64_t n_ro
     while (done < len) {
       int lg = 7;
       while ((1ll << lg) > len - done) --lg;
+      if (!SAPO_IN_BOUNDS(n < 128)) break;
       out[n++] = (uint64_t)(t - t_begin + done) | ((uint64_t)lg << 7) | ((uint64_t)side << 10) |
                  ((uint64_t)(row + done) << 16);
       done += 1ll << lg;
@@ -289,6 +290,7 @@ struct FusedTailArgs {
   float* logp; float* lse; float* ratio; float* surr; float* gscale; float* obj;   // [T]
   float* row_scale;                                        // [tc]
   __nv_bfloat16* panel; int32_t nvt;                       // exponentials of the chunk
+  int64_t panel_rows;                                      // 128-byte rows it holds (checked builds)
   RowSource rows; int32_t H; __nv_bfloat16* hs;            // hs [tc, H] = row_scale * hidden row
   uint32_t* active_mask;   // one bit per 128-token block of the chunk (zeroed by the caller), or nullptr
   int32_t* status;
@@ -366,7 +368,8 @@ __global__ void __launch_bounds__(256) fused_tail_kernel(FusedTailArgs a) {
       if (!bad_id && !bad_range && in_seq) {
         const float ey = ex2(fmaf(zy, LOG2E, -c2));
         const int64_t tile = (lr >> 7) * a.nvt + (y >> 6);
-        a.panel[(tile * BM + (lr & 127)) * 64 + (y & 63)] = __float2bfloat16_rn(ey - sum);
+        if (SAPO_IN_BOUNDS(tile * BM + (lr & 127) < a.panel_rows))
+          a.panel[(tile * BM + (lr & 127)) * 64 + (y & 63)] = __float2bfloat16_rn(ey - sum);
       }
     }
     if (!(sum < EXP_CAP)) {

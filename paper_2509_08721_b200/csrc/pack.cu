@@ -169,7 +169,7 @@ __global__ void __launch_bounds__(256) pack_copy_kernel(PackArgs a) {
       return src0 + (t - seq_begin);
     };
     auto finish = [&](int64_t t, int64_t src) {     // the per-token scalars
-      if (lane == 0) {
+      if (lane == 0 && SAPO_IN_BOUNDS(t >= 0 && t < a.max_tokens && src >= 0 && src < a.off[side][a.n_roll[side]])) {
         a.o_ids[t] = a.ids[side][src];
         a.o_old[t] = a.old[side][src];
         a.tok_seq[t] = s;
@@ -243,6 +243,8 @@ __global__ void __launch_bounds__(256) pack_copy_kernel(PackArgs a) {
     }
   }
 }
+
+long long bounds_violations_pack() { return read_bounds_violations(); }
 
 }  // namespace sapo
 

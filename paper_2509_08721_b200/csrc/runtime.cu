@@ -39,6 +39,15 @@ extern "C" int sapo_timing_read(float* h_ms, int32_t* h_launches) {
   return SAPO_OK;
 }
 
+extern "C" int64_t sapo_debug_bounds_violations(void) {
+#ifdef SAPO_BOUNDS_CHECK
+  const long long a = sapo::bounds_violations_pack(), b = sapo::bounds_violations_lmhead();
+  return (a < 0 || b < 0) ? -2 : a + b;
+#else
+  return -1;      // not a checked build
+#endif
+}
+
 extern "C" int64_t sapo_launch_count(void) { return sapo::kernel_timer().launches; }
 
 extern "C" const char* sapo_status_string(int32_t code) {

@@ -24,3 +24,14 @@ def pytest_collection_modifyitems(config, items):
     for item in items:
         if "gpu" in item.keywords:
             item.add_marker(skip)
+
+
+def pytest_sessionfinish(session, exitstatus):
+    """A run against the bounds-checking build of the library (see test_gpu_bounds_checked.py)
+    leaves the number of violations its kernels counted in the file SAPO_BOUNDS_REPORT names."""
+    path = os.environ.get("SAPO_BOUNDS_REPORT")
+    if not path:
+        return
+    from paper_2509_08721_b200 import binding as B
+    with open(path, "w") as f:
+        f.write(str(int(B.load().sapo_debug_bounds_violations())))
