@@ -17,9 +17,18 @@
  *   sapo_policy_loss_fwd_bwd  the two above in one call that passes over the logits once
  *                          (bf16 operands; the fastest way through a training step)
  *
- * and, around them, sapo_select_external (filter and sample the shared pool, Section 3.2 /
- * Section 5), sapo_policy_loss_bwd_active (backward over tokens with a gradient only) and
- * sapo_adam_step (the optimiser step of Section 4.2 on the LM head).
+ * and, around them:
+ *   sapo_select_external            filter and sample the shared pool (Section 3.2 / Section 5)
+ *   sapo_policy_loss_bwd_active     backward over the tokens with a gradient only
+ *   sapo_policy_loss_fwd_bwd_gather the single-pass call reading the hidden states in place from the
+ *                                   rollout stores (the pack then copies none)
+ *   sapo_lmhead_lse_partial, sapo_policy_loss_from_partials, sapo_policy_loss_bwd_shard
+ *                                   the same loss with W_head sharded by vocabulary over ranks
+ *   sapo_adam_step                  the optimiser step of Section 4.2 on the LM head
+ *   sapo_policy_loss_fwd_static     the forward for callers that may not allocate device memory
+ *   sapo_group_advantages_warp, sapo_workspace_bytes[_min], sapo_status_string, sapo_timing_*,
+ *   sapo_launch_count, sapo_debug_wait_timeout, sapo_debug_bounds_violations
+ *                                   sizes, texts, measurement and test hooks
  *
  * General rules
  *   - Every pointer is a DEVICE pointer unless its name starts with h_.  The caller owns

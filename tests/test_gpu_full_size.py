@@ -48,11 +48,11 @@ def check_gradient_invariants(res, hidden_dev, W_dev, T):
     assert abs(a - b) <= INNER_PRODUCT_BOUND * size, (a, b, size)
 
 
-# Bounds of the two invariants: twice the largest value measured over workloads 2-5 in both modes
-# (the residue of rounding each panel entry to bf16; a dropped vocab tile or token chunk is
-# orders of magnitude above it).
-COL_SUM_BOUND = 2e-2
-INNER_PRODUCT_BOUND = 2e-3
+# Bounds of the two invariants: about twice the largest value measured over workloads 2-5 in both
+# modes (8.7e-5 and 5.6e-7: the residue of rounding each panel entry to bf16; a dropped vocab tile
+# or token chunk is orders of magnitude above it).
+COL_SUM_BOUND = 2e-4
+INNER_PRODUCT_BOUND = 1.2e-6
 
 _W2 = {}
 
