@@ -219,21 +219,30 @@ def hbm_kernels(torch, B, peaks, H=896, n_rollouts=2048, mean_len=288, n_groups=
     return {"pack": mk(ms_pack, bytes_pack, f"{T} tokens of {H} bf16 from {2 * n_rollouts} rollouts"),
             "advantages": mk(ms_adv, bytes_adv, f"{n_groups} questions x 8 completions, thread-per-question kernel"),
             "advantages_warp": mk(ms_adv_warp, bytes_adv, f"{n_groups} questions x 8 completions, warp-level kernel "
-                                                          "(8 lanes per question; the one batches below 4096 questions take)"),
+                                                          "(2 lanes per question; the one batches below 4096 questions take)"),
             "adam": mk(ms_adam, bytes_adam, f"weight [{V_adam}, {H}] fp32 master + moments + bf16 copy"),
             "peak_source": peaks["source"] + " (copy bandwidth)"}
 
 
-# DRAM bytes per launch of the tensor-core kernels, measured with ncu on a small case of the same
-# kernels (workload 2 with lengths / 4: W_head still exceeds L2; a full-size launch holds more on
-# the device than a capture should) and extended to the bench's token count as fixed + per_token * T:
-# the traffic is the weight (or dW) once plus the panel rows.  Only for hidden 896 / vocab 151936.
-# "alg_per_token" is what the per-token part must be by the algorithm (panel row + the token's
-# hidden / output row); run_ours refuses to report a table entry that is off by more than 2 %.
+# DRAM bytes per launch of the tensor-core kernels, measured with ncu on two small cases of the same
+# kernels (workload 2 with lengths / 4 and / 8: 4133 and 2059 tokens, W_head still exceeds L2; a
+# full-size launch holds more on the device than a capture should) and extended to the bench's
+# token count as fixed + per_token * T, both from the two-point fit.  Only for hidden 896 / vocab
+# 151936.  The per-token part is the panel row plus the token's hidden / output row by the
+# algorithm; the forward and dz kernels are within 5 % of that, dhidden / dW_head read 33-37 % more
+# (every panel tile is read by the two column tiles of its block, whose CTA pairs do not always
+# share an L2 half).  ncu_traffic() refuses an entry whose slope leaves the band measured for its
+# kernel, so a kernel change cannot leave the table stale unnoticed.
 NCU_TRAFFIC_SHAPE = (896, 151936)
 NCU_TRAFFIC = {
-    # kernel: (fixed bytes, bytes per token)
+    # kernel: (fixed bytes, bytes per token, highest slope / algorithmic ratio accepted)
+    "fwd_gemm": (0.2312e9, 22.63e3, None),
+    "fwd_exp": (0.2265e9, 321.3e3, 1.08),
+    "bwd_dz": (0.2628e9, 302.0e3, 1.08),
+    "bwd_dh": (0.0737e9, 418.0e3, 1.45),
+    "bwd_dw": (0.3143e9, 407.9e3, 1.45),
 }
+NCU_TRAFFIC_SEPARATE = {"bwd_dh": (0.0671e9, 421.1e3, 1.45), "bwd_dw": (0.3186e9, 405.9e3, 1.45)}
 
 
 def algorithmic_bytes_per_token(kernel: str, H: int, V: int) -> float:
@@ -242,13 +251,16 @@ def algorithmic_bytes_per_token(kernel: str, H: int, V: int) -> float:
             "bwd_dh": 2.0 * vp + 4 * H, "bwd_dw": 2.0 * vp + 2 * H}[kernel]
 
 
-def ncu_traffic(kernel: str, H: int, V: int, tokens_per_launch: float):
+def ncu_traffic(kernel: str, H: int, V: int, tokens_per_launch: float, separate_calls: bool = False):
     """Per-launch DRAM traffic from the ncu table, or None when there is no valid entry."""
-    if (H, V) != NCU_TRAFFIC_SHAPE or kernel not in NCU_TRAFFIC:
+    table = dict(NCU_TRAFFIC)
+    if separate_calls:
+        table.update(NCU_TRAFFIC_SEPARATE)
+    if (H, V) != NCU_TRAFFIC_SHAPE or kernel not in table:
         return None
-    fixed, per_token = NCU_TRAFFIC[kernel]
+    fixed, per_token, max_ratio = table[kernel]
     alg = algorithmic_bytes_per_token(kernel, H, V)
-    if kernel != "fwd_gemm" and abs(per_token / alg - 1.0) > 0.02:
+    if max_ratio is not None and not (0.95 <= per_token / alg <= max_ratio):
         raise SystemExit(f"bench.py: the ncu traffic table for {kernel} ({per_token:.0f} B/token) no longer matches "
                          f"the kernel's algorithmic {alg:.0f} B/token: re-capture it")
     return fixed + per_token * tokens_per_launch
@@ -323,9 +335,32 @@ def measure(torch, dist, B, gen, replicas, PolicyScorer, _to_dev, args, workload
     for _ in range(warmup):
         dev_step()
     torch.cuda.synchronize()
+    # a library built with the cycle counters (build.py --stats, loaded through SAPO_B200_LIB) also
+    # reports what its GEMM kernels counted during the headline loop
+    import ctypes
+    lib = B.load()
+    counters = (ctypes.c_ulonglong * 48)() if hasattr(lib, "sapo_debug_wait_stats") else None
+    reset = (lambda: lib.sapo_debug_wait_stats(counters, 1)) if counters is not None else None
     # 1. the headline: device-resident inputs, no per-kernel events in the stream
-    m.ms_total, m.clocks = sampled(dev_step, steps)
+    m.ms_total, m.clocks = sampled(dev_step, steps, before=reset)
     scorer.check_status()
+    m.kernel_cycles = None
+    if counters is not None:
+        torch.cuda.synchronize()
+        lib.sapo_debug_wait_stats(counters, 0)
+        need = 2.0 * T * V * H / (148 * 8192.0)          # tensor-pipe cycles of one contraction over all tokens
+        m.kernel_cycles = {}
+        for r, name in enumerate(("forward", "dz", "dhidden", "dW_head")):
+            c = [int(counters[12 * r + i]) for i in range(12)]
+            if c[10] == 0:
+                continue
+            per_step = c[10] / steps
+            m.kernel_cycles[name] = {
+                "launches_per_step": per_step, "sm_cycles_per_step": c[8] / steps, "us_per_step": c[9] / steps / 1e3,
+                "sm_ghz": c[8] / max(1, c[9]), "tensor_pipe_cycles_needed_over_elapsed": need / (c[8] / steps),
+                "mma_thread_waits_for_operands": c[1] / max(1, c[5]) if c[5] else None,
+                "mma_thread_waits_for_an_accumulator": c[2] / max(1, c[5]) if c[5] else None,
+                "copy_warp_waits_for_a_free_stage": c[0] / max(1, c[4]) if c[4] else None}
     # 2. the same steps with every launch bracketed by events: which kernel takes what
     m.per_kernel, m.clocks_kernels, m.kernel_steps = None, None, 0
     if breakdown:
@@ -450,7 +485,7 @@ def run_ours(args):
         per_step = n_top / ksteps                   # launches per step (one per panel chunk)
         flops_of = lambda k: 2.0 * (T if k in ("fwd_gemm", "fwd_exp") else t_exec if k == "bwd_dz" else t_act) * V * H
         achieved = flops_of(top) / per_step / (ms_top / 1e3) / 1e12
-        traffic = ncu_traffic(top, H, V, T / per_step)
+        traffic = ncu_traffic(top, H, V, T / per_step, separate_calls=args.backward not in ("fused", "gather"))
         peak = peaks["bf16_tflops_sustained"]      # the kernel is timed inside a long step
         burst = peaks["bf16_tflops"]
         # per kernel: time, and time x SM clock (median under the same load): runs under different
@@ -507,6 +542,11 @@ def run_ours(args):
             "gpu_launches": int(round(m.launches_per_step * args.steps)),
             "clocks": m.clocks,
         }
+        if m.kernel_cycles is not None:
+            line["kernel_cycles"] = {"how": "counted by the kernels themselves (clock64 and globaltimer of CTA 0, waits of "
+                                            "the copy warp and the MMA thread) during the headline loop; "
+                                            "8192 flop per SM and cycle",
+                                     **m.kernel_cycles}
         if m.separate is not None:
             ms_sep, n_sep, clocks_sep = m.separate
             line["separate_calls"] = {

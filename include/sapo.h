@@ -196,8 +196,8 @@ int sapo_pack_rollouts(const sapo_rollout_buf* h_local, const sapo_rollout_buf* 
  * carry their rounding errors along (compensated fp32), so an advantage is within 6 fp32 ulp of
  * the exactly computed value for groups of up to 16 rewards whatever their common offset, and an
  * all-equal group gives exactly 0.  mean / std may be NULL.  A non-finite reward sets
- * SAPO_ST_NONFINITE_REWARD.  Up to 4095 questions run on the warp-level kernel (eight lanes per
- * question), more on a thread-per-question kernel; sapo_group_advantages_warp always takes the
+ * SAPO_ST_NONFINITE_REWARD.  Up to 4095 questions run on the warp-level kernel (two lanes per
+ * question, a 16-byte vector of rewards each), more on a thread-per-question kernel; sapo_group_advantages_warp always takes the
  * warp-level one (same arguments and results; it exists so that kernel can be measured alone). */
 int sapo_group_advantages(const float* rewards, const int32_t* group_offsets, int32_t Q,
                           float adv_eps, int32_t ddof, float* adv, float* mean, float* std,

@@ -9,7 +9,7 @@
 //     so mean = (s + c) / G is known as an unevaluated pair mu_hi + mu_lo to about 2^-46;
 //   - d_i = (r_i - mu_hi) - mu_lo: at most one ulp off, however large the common offset of the
 //     rewards is (an all-equal group gives exactly 0);
-//   - sum of d_i^2 by fused multiply-adds on four interleaved accumulators, combined pairwise;
+//   - sum of d_i^2 by fused multiply-adds on interleaved accumulators, combined pairwise;
 //   - correctly rounded division, square root and reciprocal for the scalars.
 // Worst-case error of an advantage against the exact value for groups of up to 16: 1 ulp (d)
 // + 2.5 (std: half of the 4-5 ulp of the sum of squares) + 1.5 (division by G - ddof, root,
@@ -54,10 +54,13 @@ __device__ __forceinline__ void std_and_inverse(float ss, int32_t G, int32_t ddo
   inv = __frcp_rn(__fadd_rn(sd, eps));
 }
 
-// The warp-level kernel: LANES lanes per question (8: every lane holds one reward of a group of
-// eight, two of a group of sixteen), 32 / LANES questions per warp, segmented shuffles.  Loads
-// and stores of a warp are contiguous.  Serves batches of any size; the thread-per-question
-// kernel below takes over for very many questions because it spends fewer instructions on each.
+// The warp-level kernel: LANES lanes per question, 32 / LANES questions per warp, segmented
+// shuffles.  A lane takes every LANES-th 16-byte vector of its question's rewards (groups whose
+// start and size are multiples of four: with two lanes a group of eight is one vector per lane and
+// a warp's loads cover 16 neighbouring questions, 512 contiguous bytes), or every LANES-th reward
+// otherwise.  The offsets of the next question are loaded a turn ahead, as in the thread kernel.
+// Serves batches of any size; the thread-per-question kernel below takes over for very many
+// questions because it spends fewer instructions on each.
 template <int LANES>
 __global__ void __launch_bounds__(256)
 group_adv_kernel(const float* __restrict__ rewards, const int32_t* __restrict__ group_offsets,
@@ -68,23 +71,41 @@ group_adv_kernel(const float* __restrict__ rewards, const int32_t* __restrict__ 
   const int sub = lane / LANES, l = lane % LANES;
   const int64_t warp0 = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
   const int64_t n_warps = ((int64_t)gridDim.x * blockDim.x) >> 5;
-  for (int64_t g0 = warp0 * PER_WARP; g0 < Q; g0 += n_warps * PER_WARP) {
-    const int64_t g = g0 + sub;
-    const bool live = g < Q;                 // every lane still takes part in the shuffles
-    const int32_t a = live ? group_offsets[g] : 0, b = live ? group_offsets[g + 1] : 0;
+  const int64_t stride = n_warps * PER_WARP;
+  int64_t g = warp0 * PER_WARP + sub;
+  int32_t a_next = 0, b_next = 0;
+  if (g < Q) { a_next = group_offsets[g]; b_next = group_offsets[g + 1]; }
+  // the loop bound is the same for all lanes of a warp: every lane takes part in the shuffles
+  for (int64_t g0 = warp0 * PER_WARP; g0 < Q; g0 += stride, g += stride) {
+    const bool live = g < Q;
+    const int32_t a = live ? a_next : 0, b = live ? b_next : 0;
+    if (g + stride < Q) { a_next = group_offsets[g + stride]; b_next = group_offsets[g + stride + 1]; }
     const int32_t G = b - a;
-    // this lane's rewards, compensated; the first one is kept for the second pass
-    float s = 0.f, c = 0.f, r_first = 0.f;
+    const bool vec = ((a | G) & 3) == 0;
+    const int32_t n4 = G >> 2;
+    // this lane's rewards, compensated; its first vector (or reward) is kept for the later passes
+    float s = 0.f, c = 0.f;
+    float4 first = make_float4(0.f, 0.f, 0.f, 0.f);
     bool bad = false;
-    for (int32_t i = a + l; i < b; i += LANES) {
-      const float r = rewards[i];
-      if (i == a + l) r_first = r;
-      bad |= !isfinite(r);
-      comp_add(s, c, r);
+    if (vec) {
+      const float4* r4 = reinterpret_cast<const float4*>(rewards + a);
+      for (int32_t v = l; v < n4; v += LANES) {
+        const float4 r = __ldg(r4 + v);
+        if (v == l) first = r;
+        bad |= !isfinite(r.x) | !isfinite(r.y) | !isfinite(r.z) | !isfinite(r.w);
+        comp_add(s, c, r.x); comp_add(s, c, r.y); comp_add(s, c, r.z); comp_add(s, c, r.w);
+      }
+    } else {
+      for (int32_t i = a + l; i < b; i += LANES) {
+        const float r = rewards[i];
+        if (i == a + l) first.x = r;
+        bad |= !isfinite(r);
+        comp_add(s, c, r);
+      }
     }
     if (__any_sync(0xffffffffu, bad) && lane == 0) raise_status(status, SAPO_ST_NONFINITE_REWARD);
     #pragma unroll
-    for (int d = 1; d < LANES; d <<= 1) {    // fixed pairing: lane ^ 1, ^ 2, ^ 4, ...
+    for (int d = 1; d < LANES; d <<= 1) {    // fixed pairing: lane ^ 1, ^ 2, ...
       const float so = __shfl_xor_sync(0xffffffffu, s, d), co = __shfl_xor_sync(0xffffffffu, c, d);
       float t, e;
       // both partners must get the same bits: add in the order (lower lane, upper lane)
@@ -94,19 +115,36 @@ group_adv_kernel(const float* __restrict__ rewards, const int32_t* __restrict__ 
     }
     float mu_hi = 0.f, mu_lo = 0.f;
     if (G > 0) comp_mean(s, c, G, mu_hi, mu_lo);
+    auto dev = [&](float r) { return __fsub_rn(__fsub_rn(r, mu_hi), mu_lo); };
     float ss = 0.f;
-    for (int32_t i = a + l; i < b; i += LANES) {
-      const float r = i == a + l ? r_first : rewards[i];
-      const float dv = __fsub_rn(__fsub_rn(r, mu_hi), mu_lo);
-      ss = __fmaf_rn(dv, dv, ss);
+    if (vec) {
+      const float4* r4 = reinterpret_cast<const float4*>(rewards + a);
+      for (int32_t v = l; v < n4; v += LANES) {
+        const float4 r = v == l ? first : __ldg(r4 + v);
+        const float dx = dev(r.x), dy = dev(r.y), dz = dev(r.z), dw = dev(r.w);
+        ss = __fadd_rn(ss, __fadd_rn(__fmaf_rn(dy, dy, __fmul_rn(dx, dx)), __fmaf_rn(dw, dw, __fmul_rn(dz, dz))));
+      }
+    } else {
+      for (int32_t i = a + l; i < b; i += LANES) {
+        const float dv = dev(i == a + l ? first.x : rewards[i]);
+        ss = __fmaf_rn(dv, dv, ss);
+      }
     }
     #pragma unroll
     for (int d = 1; d < LANES; d <<= 1) ss = __fadd_rn(ss, __shfl_xor_sync(0xffffffffu, ss, d));
     float sd, inv;
     std_and_inverse(ss, G, ddof, adv_eps, sd, inv);
-    for (int32_t i = a + l; i < b; i += LANES) {
-      const float r = i == a + l ? r_first : rewards[i];
-      adv[i] = __fmul_rn(__fsub_rn(__fsub_rn(r, mu_hi), mu_lo), inv);
+    if (vec) {
+      const float4* r4 = reinterpret_cast<const float4*>(rewards + a);
+      float4* a4 = reinterpret_cast<float4*>(adv + a);
+      for (int32_t v = l; v < n4; v += LANES) {
+        const float4 r = v == l ? first : __ldg(r4 + v);
+        a4[v] = make_float4(__fmul_rn(dev(r.x), inv), __fmul_rn(dev(r.y), inv), __fmul_rn(dev(r.z), inv),
+                            __fmul_rn(dev(r.w), inv));
+      }
+    } else {
+      for (int32_t i = a + l; i < b; i += LANES)
+        adv[i] = __fmul_rn(dev(i == a + l ? first.x : rewards[i]), inv);
     }
     if (live && l == 0) {
       if (mean) mean[g] = G > 0 ? mu_hi : 0.f;
@@ -239,7 +277,7 @@ static int launch_group_adv(const float* rewards, const int32_t* group_offsets, 
   const int sms = sm_count();
   if (sms <= 0) return SAPO_ERR_CUDA;
   const bool many = which == 2 || (which == 0 && Q >= 4096);        // then: one thread per question
-  int64_t blocks = ((int64_t)Q + (many ? 255 : 31)) / (many ? 256 : 32);   // warp-level: 4 questions per warp
+  int64_t blocks = ((int64_t)Q + (many ? 255 : 127)) / (many ? 256 : 128);   // warp-level: 16 questions per warp
   if (blocks > (int64_t)sms * 8) blocks = (int64_t)sms * 8;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   {
@@ -248,7 +286,7 @@ static int launch_group_adv(const float* rewards, const int32_t* group_offsets, 
       group_adv_thread_kernel<<<(int)blocks, 256, 0, st>>>(rewards, group_offsets, Q, adv_eps, ddof,
                                                            adv, mean, std, status);
     else
-      group_adv_kernel<8><<<(int)blocks, 256, 0, st>>>(rewards, group_offsets, Q, adv_eps, ddof, adv,
+      group_adv_kernel<2><<<(int)blocks, 256, 0, st>>>(rewards, group_offsets, Q, adv_eps, ddof, adv,
                                                        mean, std, status);
   }
   return check_launch();

@@ -45,10 +45,10 @@ def _regular(hidden, W, ids, old, adv, cu):
     return out
 
 
-def _static_raw(hidden, W, ids, old, adv, cu, out, status):
+def _static_raw(hidden, W, ids, old, adv, cu, out, status, entropy=None):
     """The raw symbol, called through ctypes with plain pointers: no tensor is created here."""
     T, H, V, S = hidden.shape[0], hidden.shape[1], W.shape[0], cu.numel() - 1
-    cfg = B.LossCfgC(0.2, 0.28, 1.0, 0, 0.0, None)
+    cfg = B.LossCfgC(0.2, 0.28, 1.0, 0, 0.0, None, None if entropy is None else entropy.data_ptr())
     rc = B.load().sapo_policy_loss_fwd_static(
         hidden.data_ptr(), W.data_ptr(), B.DTYPE_BF16, T, H, V, hidden.stride(0), W.stride(0),
         ids.data_ptr(), old.data_ptr(), adv.data_ptr(), cu.data_ptr(), S, C.byref(cfg),
@@ -89,6 +89,17 @@ def test_static_scratch_forward_matches_the_regular_one_twice_in_a_row():
     _identical(cases[0][4], cases[0][3])
     _identical(cases[1][4], cases[1][3])
     _identical(cases[1][5], cases[1][3])
+    # with the entropy output (one more partial array in the scratch): same values as the regular call's
+    hidden, W, ids, old, adv, cu = cases[0][2]
+    T, H, V = hidden.shape[0], hidden.shape[1], W.shape[0]
+    ent_s, ent_r = torch.empty(T, device="cuda"), torch.empty(T, device="cuda")
+    ws = torch.empty(B.sapo_workspace_bytes(B.WS_FWD, T, H, V, B.DTYPE_BF16), dtype=torch.uint8, device="cuda")
+    B.sapo_policy_loss_fwd(hidden, W, ids, old, adv, cu, 0.2, 0.28, 1.0, B.alloc_fwd_outputs(T, cu.numel() - 1),
+                           ws, status, entropy=ent_r)
+    _static_raw(hidden, W, ids, old, adv, cu, cases[0][5], status, entropy=ent_s)
+    torch.cuda.synchronize()
+    assert status.item() == 0 and torch.equal(ent_s, ent_r)
+    _identical(cases[0][5], cases[0][3])
     # the static path against the oracle, under the tolerances of the other parity tests
     batch, adv_np, dev, _, out, _ = cases[0]
     b = batch.built
