@@ -284,7 +284,7 @@ def measure(torch, dist, B, gen, replicas, PolicyScorer, _to_dev, args, workload
     # old log-probs = current + noise: "current" is one forward pass of the library itself
     # over the packed tokens (set-up, untimed); the noise comes from the seeded generator.
     scorer.make_host_batch(batch)
-    res = scorer.step_from_host(T, S)
+    res = scorer.step_from_host(T, S, prefetch_next=False)
     torch.cuda.synchronize()
     gen.install_old_logp(batch, res.fwd["logp"][:T].cpu().numpy())
     scorer.make_host_batch(batch)
@@ -535,6 +535,8 @@ def run_ours(args):
                                  "clocks": m.clocks_kernels},
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d,
                     "d2h_bytes_per_step": d2h, "ms_per_step": m.ms_e2e / args.steps,
+                    "overlap": "every step copies its inputs from pinned host memory into one of two device "
+                               "buffer sets on a copy stream; the copy for step i+1 runs while step i computes",
                     "returns": "loss and per-token log-probs go back to the host every step; dhidden and dW_head "
                                "stay in device memory, where the transformer backward and the optimiser step "
                                "read them",

@@ -181,12 +181,17 @@ struct ExpEpiT {
     __nv_bfloat16* panel;
     int64_t panel_rows;   // 128-byte rows the panel holds, and
     int32_t parts_cap;    // partials per token the arrays hold (checked builds)
+    // optional: one bit per 128-token block of the whole batch, set when some token of the block
+    // can have a gradient; the panel rows of a clear block are not written (its sums still are).
+    // blk0 = index of this launch's first block in that array
+    const uint32_t* need; int32_t blk0;
   };
-  float c, sum, sz; int32_t tile_row0; int r; bool valid, in_panel; int64_t row;
+  float c, sum, sz; int32_t tile_row0; int r; bool valid, in_panel, store; int64_t row;
   __device__ __forceinline__ void begin_unit(const Params& p, int mb, int r_) {
     row = (int64_t)mb * BM + r_;
     valid = row < p.M;
     in_panel = (int64_t)mb * BM < p.M;
+    store = p.need == nullptr || ((p.need[(p.blk0 + mb) >> 5] >> ((p.blk0 + mb) & 31)) & 1u) != 0u;
     r = r_;
     tile_row0 = mb * p.nvt * BM;
     c = valid ? p.c2[row] : 0.f;
@@ -197,6 +202,7 @@ struct ExpEpiT {
     if (!in_panel) return;
     uint32_t w[8];
     if (!valid || col0 >= p.V) {
+      if (!store) return;
       #pragma unroll
       for (int j = 0; j < 8; ++j) w[j] = 0u;
       store_panel_16(p.panel, p.panel_rows, r, tile_row0, col0, w);
@@ -221,12 +227,14 @@ struct ExpEpiT {
       #pragma unroll
       for (int j = 16 * h; j < 16 * h + 16; j += 4) { a0 += v[j]; a1 += v[j + 1]; a2 += v[j + 2]; a3 += v[j + 3]; }
       sum += (a0 + a1) + (a2 + a3);
-      #pragma unroll
-      for (int j = 0; j < 8; ++j) {
-        __nv_bfloat162 b2 = __floats2bfloat162_rn(v[16 * h + 2 * j], v[16 * h + 2 * j + 1]);
-        w[j] = *reinterpret_cast<uint32_t*>(&b2);
+      if (store) {
+        #pragma unroll
+        for (int j = 0; j < 8; ++j) {
+          __nv_bfloat162 b2 = __floats2bfloat162_rn(v[16 * h + 2 * j], v[16 * h + 2 * j + 1]);
+          w[j] = *reinterpret_cast<uint32_t*>(&b2);
+        }
+        store_panel_16(p.panel, p.panel_rows, r, tile_row0, col0 + 16 * h, w);
       }
-      store_panel_16(p.panel, p.panel_rows, r, tile_row0, col0 + 16 * h, w);
     }
   }
   __device__ __forceinline__ void group_end(const Params&, int) {}
@@ -291,6 +299,10 @@ struct StoreEpi {
   }
   template <int HALF>
   __device__ __forceinline__ void chunk(const Params& p, float (&v)[32], int col0) {
+    if (scale == 0.f) {                    // a row without a gradient: exact zeros, whatever was contracted
+      #pragma unroll
+      for (int j = 0; j < 32; ++j) v[j] = 0.f;
+    }
     if (part != nullptr) {
       float4* dst = reinterpret_cast<float4*>(part + (col0 - n0));
       #pragma unroll
@@ -360,6 +372,7 @@ streamk_fixup_kernel(const Sched s_arg, const StoreEpi::Params p_arg, int pairs)
       sum.x += v.x; sum.y += v.y; sum.z += v.z; sum.w += v.w;
     }
     float4 o = make_float4(scale * sum.x, scale * sum.y, scale * sum.z, scale * sum.w);
+    if (scale == 0.f) o = make_float4(0.f, 0.f, 0.f, 0.f);
     if (p.out_bf16) {
       __nv_bfloat162* dst = reinterpret_cast<__nv_bfloat162*>(reinterpret_cast<__nv_bfloat16*>(p.C) + row * p.ldc + n0 + 4 * c4);
       if (p.accumulate) {

@@ -508,8 +508,8 @@ umma_gemm2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
       // 128-byte swizzle) and leaves as one TMA store, or TMA add when accumulating, of
       // 128 rows x 32 columns: full lines, and rows / columns outside the output are clipped.
       auto emit = [&](float (&v)[32], int col0) {
-        if (!any) {
-          #pragma unroll
+        if (!any || epi.scale == 0.f) {    // (a row without a gradient gives exact zeros: its panel
+          #pragma unroll                   //  block may never have been written)
           for (int q = 0; q < 32; ++q) v[q] = 0.f;
         }
         if (epi.part != nullptr) { epi.template chunk<0>(ep, v, col0); return; }

@@ -382,7 +382,7 @@ static int64_t preferred_panel_rows(int64_t T) {
 // needs (row scales, partial sums, the scaled copy of hidden), the K-split scratch, the
 // per-sequence sums when the caller does not want them, and the panel of exponentials.
 constexpr int FUSED_MAX_SPLITS = 160;
-struct FusedLayout { size_t zy, c2, obj, seq, mask, partials, dw_acc, boxes, n_boxes, fixed; size_t bytes_per_row; };
+struct FusedLayout { size_t zy, c2, obj, seq, mask, need, partials, dw_acc, boxes, n_boxes, fixed; size_t bytes_per_row; };
 static FusedLayout fused_layout(int64_t T, int32_t H, int32_t V, int32_t S, bool out_bf16 = false,
                                 bool gather = false) {
   FusedLayout L{};
@@ -399,6 +399,7 @@ static FusedLayout fused_layout(int64_t T, int32_t H, int32_t V, int32_t S, bool
   L.obj = take((size_t)T * 4);
   L.seq = take((size_t)(S > 0 ? S : 1) * 4);
   L.mask = take((size_t)MASK_WORDS_MAX * 4);
+  L.need = take((size_t)ceil_div<int64_t>(ceil_div<int64_t>(T, BM), 32) * 4);
   L.partials = take(KSPLIT_SCRATCH_BYTES);
   L.fixed = off;
   // per chunk row: panel row, scaled hidden row, row scale, partial sums
@@ -1099,12 +1100,24 @@ static int fused_impl(const void* hidden, const HiddenSource* src, const void* W
                                                                                src->n_ext, boxes, n_boxes, status);
   }
 
+  // Blocks of 128 tokens whose sequences all have a zero advantage get log-probs but no gradient
+  // (without a KL term): the forward leaves their panel rows unwritten and both contractions
+  // skip them.  Only where the contractions do skip by block: wide tiles, a chunk's block bits
+  // within what those kernels hold.
+  uint32_t* need = nullptr;
+  if (use_wide_tiles(H) && h_cfg->kl_beta == 0.f &&
+      ceil_div<int64_t>(ceil_div<int64_t>(chunk_rows < T ? chunk_rows : T, BM), 32) <= MASK_WORDS_MAX) {
+    need = reinterpret_cast<uint32_t*>(ws + L.need);
+    if (cudaMemsetAsync(need, 0, (size_t)ceil_div<int64_t>(ceil_div<int64_t>(T, BM), 32) * 4, st) != cudaSuccess)
+      return SAPO_ERR_CUDA;
+  }
   // 1. chosen-token logits and the reference of the exponentials, all tokens
   {
     int64_t blocks = ceil_div<int64_t>(T, 8);
     if (blocks > (int64_t)sms * 8) blocks = (int64_t)sms * 8;
     KernelScope scope(SAPO_K_TARGET_LOGIT, st);
-    target_logit_kernel<<<(int)blocks, 256, 0, st>>>(rows, B, ld_W, ids, old_logp, T, H, V, zy, c2);
+    target_logit_kernel<<<(int)blocks, 256, 0, st>>>(rows, B, ld_W, ids, old_logp, T, H, V, zy, c2,
+                                                     adv, cu_seqlens, S, need);
   }
   CUtensorMap map_w_kmajor;
   if (!make_map(&map_w_kmajor, B, H, V, ld_W, 128)) return SAPO_ERR_CUDA;
@@ -1129,11 +1142,11 @@ static int fused_impl(const void* hidden, const HiddenSource* src, const void* W
     {
       int rc;
       if (want_entropy) {
-        ExpEpiT<true>::Params ep{c2 + t0, ps, pe, tc, V, nvt, panel, panel_rows, 2 * FUSED_MAX_SPLITS};
+        ExpEpiT<true>::Params ep{c2 + t0, ps, pe, tc, V, nvt, panel, panel_rows, 2 * FUSED_MAX_SPLITS, need, (int32_t)(t0 / BM)};
         rc = gather ? launch_gemm<0, false, ExpEpiT<true>, FWD_BK, FWD_STAGES, GatherArgs>(map_h_kmajor, map_w_kmajor, fs, ep, status, st, SAPO_K_FWD_EXP, ga)
                     : launch_gemm<0, false, ExpEpiT<true>, FWD_BK, FWD_STAGES>(map_h_kmajor, map_w_kmajor, fs, ep, status, st, SAPO_K_FWD_EXP);
       } else {
-        ExpEpi::Params ep{c2 + t0, ps, nullptr, tc, V, nvt, panel, panel_rows, 2 * FUSED_MAX_SPLITS};
+        ExpEpi::Params ep{c2 + t0, ps, nullptr, tc, V, nvt, panel, panel_rows, 2 * FUSED_MAX_SPLITS, need, (int32_t)(t0 / BM)};
         rc = gather ? launch_gemm<0, false, ExpEpi, FWD_BK, FWD_STAGES, GatherArgs>(map_h_kmajor, map_w_kmajor, fs, ep, status, st, SAPO_K_FWD_EXP, ga)
                     : launch_gemm<0, false, ExpEpi, FWD_BK, FWD_STAGES>(map_h_kmajor, map_w_kmajor, fs, ep, status, st, SAPO_K_FWD_EXP);
       }

@@ -246,10 +246,15 @@ gather_boxes_kernel(const int64_t* __restrict__ tok_src, int64_t T, int64_t n_ro
 // which equals lse_t when the policy has not moved since old_logp was taken and is off by
 // log(ratio_t) otherwise: exp(z - c_t) then stays within a few powers of e of a probability.
 // c2 is c_t * log2(e).  A token id outside [0, V) gets z_y = c = 0 (the tail reports it).
+// need (optional, zeroed by the caller): one bit per 128-token block, set when a token of the
+// block belongs to a sequence whose advantage is not zero.  Without a KL term every other token
+// has g_t = 0 whatever the pass finds, so the forward need not keep the block's exponentials.
 __global__ void __launch_bounds__(256)
 target_logit_kernel(const RowSource rows, const __nv_bfloat16* __restrict__ W,
                     int64_t ldw, const int32_t* __restrict__ ids, const float* __restrict__ old_logp,
-                    int64_t T, int32_t H, int32_t V, float* __restrict__ zy, float* __restrict__ c2) {
+                    int64_t T, int32_t H, int32_t V, float* __restrict__ zy, float* __restrict__ c2,
+                    const float* __restrict__ adv, const int32_t* __restrict__ cu, int32_t S,
+                    uint32_t* __restrict__ need) {
   const int lane = threadIdx.x & 31;
   const int64_t warp = (int64_t)blockIdx.x * 8 + (threadIdx.x >> 5);
   const int64_t n_warps = (int64_t)gridDim.x * 8;
@@ -279,6 +284,13 @@ target_logit_kernel(const RowSource rows, const __nv_bfloat16* __restrict__ W,
       zy[t] = ok ? acc : 0.f;
       // a non-finite old log-prob (the tail reports it and masks the token) must not reach the panel
       c2[t] = ok ? (isfinite(old) ? acc - old : acc) * LOG2E : 0.f;
+      if (need != nullptr) {
+        // the token's sequence (last s with cu[s] <= t) and whether its advantage can give a gradient
+        int lo = 0, hi = S - 1;
+        while (lo < hi) { const int mid = (lo + hi + 1) >> 1; if ((int64_t)cu[mid] <= t) lo = mid; else hi = mid - 1; }
+        const uint32_t bit = 1u << ((t >> 7) & 31);
+        if (adv[lo] != 0.f && (need[t >> 12] & bit) == 0u) atomicOr(&need[t >> 12], bit);
+      }
     }
   }
 }

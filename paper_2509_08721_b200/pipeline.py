@@ -124,6 +124,8 @@ class PolicyScorer:
     # -- one step from pinned host buffers -----------------------------------------------------
     def make_host_batch(self, batch: gen.Batch) -> Dict[str, torch.Tensor]:
         """Pinned host copies of everything a step consumes, plus matching device buffers."""
+        if getattr(self, "_copy_stream", None) is not None:
+            self._copy_stream.synchronize()          # no copy into the buffers this call replaces
         host, dev = {}, {}
         for side, buf in (("local", batch.local), ("ext", batch.ext)):
             for k in ("hidden", "ids", "old_logp", "offsets", "rewards"):
@@ -131,20 +133,49 @@ class PolicyScorer:
                 host[f"{side}.{k}"] = _pinned(a)
         for k in ("q_offsets_local", "local_idx", "q_offsets_ext", "ext_idx"):
             host[f"sel.{k}"] = _pinned(getattr(batch.sel, k))
+        # two sets of device buffers: while a step computes on one, the next step's inputs are
+        # copied into the other on a stream of their own
+        other = {}
         for k, t in host.items():
             dev[k] = torch.empty(t.shape, dtype=t.dtype, device=self.device)
+            other[k] = torch.empty(t.shape, dtype=t.dtype, device=self.device)
         self._host, self._dev = host, dev
+        self._dev_sets = [dev, other]
+        self._copy_stream = torch.cuda.Stream(device=self.device)
+        self._copied = [torch.cuda.Event(), torch.cuda.Event()]
+        self._consumed = [None, None]
+        self._in_flight = [False, False]
+        self._next_set = 0
         self._loss_host = torch.empty(1, dtype=torch.float32).pin_memory()
         self._logp_host = torch.empty(batch.T, dtype=torch.float32).pin_memory()
         self.h2d_bytes = sum(t.numel() * t.element_size() for t in host.values())
         self.d2h_bytes = 4 + 4 * batch.T
         return host
 
-    def step_from_host(self, T: int, S: int) -> StepResult:
-        """Copy the pinned inputs to the device, run the step, read loss and log-probs back."""
-        d = self._dev
-        for k, t in self._host.items():
-            d[k].copy_(t, non_blocking=True)
+    def _start_copy(self, i: int) -> None:
+        """Host -> device copy of the pinned inputs into buffer set i, on the copy stream, once
+        the step that last read that set has finished."""
+        with torch.cuda.stream(self._copy_stream):
+            if self._consumed[i] is not None:
+                self._copy_stream.wait_event(self._consumed[i])
+            for k, t in self._host.items():
+                self._dev_sets[i][k].copy_(t, non_blocking=True)
+            self._copied[i].record(self._copy_stream)
+        self._in_flight[i] = True
+
+    def step_from_host(self, T: int, S: int, prefetch_next: bool = True) -> StepResult:
+        """One step whose inputs start in pinned host memory: copy them to the device, run the
+        step, read loss and log-probs back.  Every call makes exactly one copy of the inputs; with
+        prefetch_next the copy it starts is the one the *next* call consumes (into the other buffer
+        set, overlapping this call's kernels), and its own inputs are those the previous call
+        fetched (or are copied now, on the first call)."""
+        i = self._next_set
+        if not self._in_flight[i]:
+            self._start_copy(i)
+        stream = torch.cuda.current_stream()
+        stream.wait_event(self._copied[i])
+        self._in_flight[i] = False
+        d = self._dev_sets[i]
         view = lambda t: t.view(torch.bfloat16) if (t.dtype == torch.int16) else t
         local = B.DeviceRollouts(view(d["local.hidden"]), d["local.ids"], d["local.old_logp"],
                                  d["local.offsets"], d["local.rewards"])
@@ -153,8 +184,14 @@ class PolicyScorer:
         sel = B.DeviceSelection(d["sel.q_offsets_local"], d["sel.local_idx"], d["sel.q_offsets_ext"],
                                 d["sel.ext_idx"])
         res = self.step(local, ext, sel, T, S)
+        if self._consumed[i] is None:
+            self._consumed[i] = torch.cuda.Event()
+        self._consumed[i].record(stream)
         self._loss_host.copy_(res.loss, non_blocking=True)
         self._logp_host.copy_(res.fwd["logp"][:T], non_blocking=True)
+        if prefetch_next:
+            self._start_copy(1 - i)
+            self._next_set = 1 - i
         return res
 
     def check_status(self) -> None:

@@ -26,7 +26,7 @@ def run_scorer(batch, recipe, backward="dense"):
     scorer = PolicyScorer(_to_dev(batch.W, "cuda"), batch.T, batch.S, recipe.Q,
                           eps_low=batch.eps_low, eps_high=batch.eps_high, backward=backward)
     scorer.make_host_batch(batch)
-    res = scorer.step_from_host(batch.T, batch.S)
+    res = scorer.step_from_host(batch.T, batch.S, prefetch_next=False)
     torch.cuda.synchronize()
     scorer.check_status()
     return scorer, res
@@ -162,7 +162,7 @@ def test_workloads_3_to_5_full_size(number, ext_fraction, backward):
     scorer = PolicyScorer(_to_dev(batch.W, "cuda"), T, S, recipe.Q, eps_low=batch.eps_low,
                           eps_high=batch.eps_high, backward=backward, want_entropy=True)
     scorer.make_host_batch(batch)
-    res = scorer.step_from_host(T, S)
+    res = scorer.step_from_host(T, S, prefetch_next=False)
     torch.cuda.synchronize()
     scorer.check_status()
     # pack and advantages

@@ -156,6 +156,56 @@ def test_edge_shapes_of_the_wide_backward_kernels(name, recipe):
         check_all(U.gpu_scores(*args, 0.2, 0.28, bwd_workspace_bytes=small_b), ref, adv, batch, 0.2, 0.28)
 
 
+@pytest.mark.parametrize("H", [256, 520])
+@pytest.mark.parametrize("pattern", ["leading", "alternating", "all_zero"])
+def test_blocks_of_zero_advantage_sequences_leave_no_trace(H, pattern):
+    """Runs of sequences whose advantage is exactly zero that cover whole 128-token blocks: the
+    forward writes no panel rows for them and the contractions leave them out.  The scratch is
+    filled with NaN patterns beforehand, so anything read from an unwritten block would show;
+    their log-probs must still be right and their dhidden rows exactly zero.  The patterns give
+    256-token tiles with one written and one unwritten block, in either order."""
+    recipe = small_recipe(H=H, V=1500, Q=8, I=2, J=2, length_law=("uniform", 100, 160))
+    batch = gen.make_batch(recipe, 91)
+    gen.install_old_logp(batch, U.oracle_current_logp(batch))
+    b = batch.built
+    S, T = batch.S, batch.T
+    adv = np.linspace(-1.5, 1.5, S).astype(np.float32)
+    adv[np.abs(adv) < 1e-3] = 0.25
+    q_of = np.repeat(np.arange(8), 4)
+    if pattern == "leading":
+        adv[q_of < 3] = 0.0                    # 12 sequences, about 1500 tokens, then live ones
+    elif pattern == "alternating":
+        adv[q_of % 2 == 1] = 0.0               # about 500 dead tokens between live stretches
+    else:
+        adv[:] = 0.0
+    h, W = gen.as_f32(b.hidden), gen.as_f32(batch.W)
+    ref = orc.policy_loss_fwd(h, W, b.ids, b.old_logp, adv, b.cu_seqlens, 0.2, 0.28)
+    ref.update(orc.policy_loss_bwd(h, W, b.ids, ref["lse"], ref["gscale"]))
+    args = device_inputs(batch, adv)
+    dead = np.repeat(adv == 0.0, np.diff(b.cu_seqlens))
+    blocks = dead[: (T // 128) * 128].reshape(-1, 128).all(axis=1)
+    assert pattern == "all_zero" or (blocks.any() and not blocks.all())
+    small = B.sapo_workspace_bytes_min(B.WS_FUSED, T, H, 1500, B.DTYPE_BF16)
+    three = small + 3 * 128 * (2 * 1536 + 2 * H + 4 + 2560)     # room for about three more blocks per chunk
+    for nbytes in (None, small, three):      # one chunk; chunks of one block; chunks of a few blocks
+        for out_dtype in (torch.float32, torch.bfloat16):
+            kw = {} if nbytes is None else {"workspace_bytes": nbytes + (
+                B.sapo_workspace_bytes_min(B.WS_FUSED | B.WS_OUT_BF16, T, H, 1500, B.DTYPE_BF16) - small
+                if out_dtype == torch.bfloat16 else 0)}
+            out = U.gpu_scores_fused(*args, 0.2, 0.28, out_dtype=out_dtype, **kw)
+            assert out["status"] == 0
+            U.check_forward(out, ref, adv.astype(np.float64), b.cu_seqlens, 0.2, 0.28)
+            dH = out["dhidden"].float()
+            assert torch.isfinite(dH).all() and torch.isfinite(out["dW"].float()).all()
+            assert not dH[torch.from_numpy(dead).cuda()].any()
+            if pattern == "all_zero":
+                assert not out["dW"].float().any()
+                continue
+            tol = U.TOL_GRAD_FRO
+            assert U.rel_fro(dH.cpu().numpy(), ref["dhidden"]) <= tol
+            assert U.rel_fro(out["dW"].float().cpu().numpy(), ref["dW"]) <= tol
+
+
 def _random_recipe(seed):
     rng = np.random.default_rng(1000 + seed)
     H = int(rng.choice([8, 16, 24, 64, 72, 248, 256, 264, 392, 512, 776, 1024, 1096]))
@@ -325,3 +375,35 @@ def test_fused_argument_errors():
         B.sapo_policy_loss_fwd_bwd(xb, Wb, i, f, f[:1], cu, 0.2, 0.2, 1.0, out, dH, dW, False, ws[:1024],
                                    B.new_status())
     assert B.sapo_workspace_bytes(B.WS_FUSED, 8, 16, 16, B.DTYPE_F32) == 0
+
+
+def test_steps_from_pinned_host_buffers_overlap_their_copies_and_repeat_bit_for_bit():
+    """PolicyScorer.step_from_host keeps two sets of device input buffers and copies the next
+    step's inputs while the current step computes: consecutive steps (which alternate between
+    the sets) must give the bits of a step over device-resident inputs."""
+    from paper_2509_08721_b200.pipeline import PolicyScorer
+    recipe = small_recipe(H=256, V=3000, Q=6, length_law=("uniform", 40, 120))
+    batch = gen.make_batch(recipe, 55)
+    gen.install_old_logp(batch, U.oracle_current_logp(batch))
+    scorer = PolicyScorer(U.to_torch(batch.W), batch.T, batch.S, recipe.Q, eps_low=0.2, eps_high=0.28,
+                          backward="fused")
+    scorer.make_host_batch(batch)
+    first = scorer.step_from_host(batch.T, batch.S)
+    torch.cuda.synchronize()
+    want = {k: first.fwd[k].clone() for k in ("logp", "ratio", "gscale", "loss")}
+    want_dW, want_dH = first.dW.clone(), first.dhidden.clone()
+    for _ in range(4):
+        res = scorer.step_from_host(batch.T, batch.S)
+    torch.cuda.synchronize()
+    scorer.check_status()
+    for k, v in want.items():
+        assert torch.equal(res.fwd[k], v), k
+    assert torch.equal(res.dW, want_dW) and torch.equal(res.dhidden, want_dH)
+    assert torch.equal(scorer._logp_host, want["logp"][:batch.T].cpu())
+    # and against the oracle, so that "the same bits" are the right ones
+    adv = orc.group_advantages(batch.built.rewards, batch.built.group_offsets,
+                               adv_eps=float(np.float32(batch.adv_eps)))["adv"]
+    ref = orc.policy_loss_fwd(gen.as_f32(batch.built.hidden), gen.as_f32(batch.W), batch.built.ids,
+                              batch.built.old_logp, adv, batch.built.cu_seqlens, 0.2, 0.28)
+    out = {k: res.fwd[k][:batch.T] for k in ("logp", "lse", "ratio", "surr", "gscale")}
+    U.check_forward(out, ref, adv, batch.built.cu_seqlens, 0.2, 0.28)

@@ -97,14 +97,14 @@ def gpu_scores(hidden, W, ids, old_logp, adv, cu, eps_low, eps_high, grad_scale=
     dcode = B.DTYPE_F32 if hidden.dtype == torch.float32 else B.DTYPE_BF16
     status = B.new_status()
     out = B.alloc_fwd_outputs(T, S)
-    ws_f = torch.empty(B.sapo_workspace_bytes(B.WS_FWD, T, H, V, dcode), dtype=torch.uint8, device="cuda")
+    ws_f = poisoned_workspace(B.sapo_workspace_bytes(B.WS_FWD, T, H, V, dcode))
     B.sapo_policy_loss_fwd(hidden, W, ids, old_logp, adv, cu, eps_low, eps_high, grad_scale, out,
                            ws_f, status)
     if want_bwd:
         kind = B.WS_BWD | (B.WS_OUT_BF16 if out_dtype == torch.bfloat16 else 0)
         nbytes = (B.sapo_workspace_bytes(kind, T, H, V, dcode)
                   if bwd_workspace_bytes is None else bwd_workspace_bytes)
-        ws_b = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
+        ws_b = poisoned_workspace(nbytes)
         out["dhidden"] = torch.empty(T, H, dtype=out_dtype, device="cuda")
         out["dW"] = torch.empty(V, H, dtype=out_dtype, device="cuda") if accumulate_into is None else accumulate_into
         B.sapo_policy_loss_bwd(hidden, W, ids, out["lse"], out["gscale"], out["dhidden"], out["dW"],
@@ -112,6 +112,12 @@ def gpu_scores(hidden, W, ids, old_logp, adv, cu, eps_low, eps_high, grad_scale=
     torch.cuda.synchronize()
     out["status"] = int(status.item())
     return out
+
+
+def poisoned_workspace(nbytes: int) -> torch.Tensor:
+    """Scratch for a library call with every byte 0xFF: any bf16 or fp32 read from a place the call
+    has not written first is a NaN, and shows in the outputs."""
+    return torch.full((nbytes,), 0xFF, dtype=torch.uint8, device="cuda")
 
 
 def gpu_scores_fused(hidden, W, ids, old_logp, adv, cu, eps_low, eps_high, grad_scale=1.0,
@@ -124,7 +130,7 @@ def gpu_scores_fused(hidden, W, ids, old_logp, adv, cu, eps_low, eps_high, grad_
     kind = B.WS_FUSED | (B.WS_OUT_BF16 if out_dtype == torch.bfloat16 else 0)
     nbytes = (B.sapo_workspace_bytes(kind, T, H, V, B.DTYPE_BF16)
               if workspace_bytes is None else workspace_bytes)
-    ws = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
+    ws = poisoned_workspace(nbytes)
     out["dhidden"] = torch.empty(T, H, dtype=out_dtype, device="cuda")
     out["dW"] = torch.empty(V, H, dtype=out_dtype, device="cuda") if accumulate_into is None else accumulate_into
     B.sapo_policy_loss_fwd_bwd(hidden, W, ids, old_logp, adv, cu, eps_low, eps_high, grad_scale, out,
