@@ -373,9 +373,37 @@ static int64_t equal_chunk_rows(int64_t T, int64_t max_rows) {     // max_rows: 
   const int64_t rows = round_up<int64_t>(ceil_div<int64_t>(T, n), BM);
   return rows < max_rows ? rows : max_rows;
 }
-static int64_t preferred_panel_rows(int64_t T) {
+// Waves of CTA pairs the dhidden contraction of a `rows`-token chunk takes, in units of one tile's
+// time, by the schedule's own rule for its last wave.  Of the three big kernels it is the one whose
+// tile count follows the chunk size (2 to 7 column tiles per 256-token block), so it decides how
+// well a chunk size fills the machine.
+static double dhidden_waves(int64_t rows, int32_t H, int32_t V, int pairs) {
+  Sched s = make_sched_wide(rows, H, padded_vocab(V));
+  s.k_split_ok = 1;
+  split_last_wave(s, pairs);
+  if (s.sk_tiles == 0) return (double)ceil_div(s.num_units, pairs);
+  const int rounds = ceil_div(s.sk_tiles * s.sk_parts, pairs);
+  return (double)(s.dp_units / pairs) + (double)rounds / s.sk_parts + 0.02 * rounds;
+}
+// Panel rows the workspace queries ask for.  A batch of up to 20 480 tokens is taken whole.  A
+// longer one is cut into equal chunks of at most 20 480 tokens when a chunk's hidden rows still
+// sit in the share of L2 the forward pass counts on (48 MB), of at most 16 384 otherwise; among
+// the five smallest chunk counts that allow, the one whose dhidden contraction wastes least of
+// its last wave (plus a twentieth of a tile's time per chunk for what every chunk costs anyway).
+static int64_t preferred_panel_rows(int64_t T, int32_t H, int32_t V) {
   if (T <= PANEL_ROWS_ONE_PIECE) return round_up<int64_t>(T, BM);
-  return equal_chunk_rows(T, PANEL_ROWS_TARGET);
+  const int64_t cap = PANEL_ROWS_ONE_PIECE * (int64_t)H * 2 <= (48ll << 20) ? PANEL_ROWS_ONE_PIECE : PANEL_ROWS_TARGET;
+  if (!use_wide_tiles(H)) return equal_chunk_rows(T, cap);
+  const int sms = sm_count();
+  const int pairs = sms >= 2 ? sms / 2 : 74;
+  const int64_t n_min = ceil_div<int64_t>(T, cap);
+  int64_t best_rows = 0; double best_cost = 0.0;
+  for (int64_t n = n_min; n < n_min + 5; ++n) {
+    const int64_t rows = round_up<int64_t>(ceil_div<int64_t>(T, n), BM);
+    const double cost = (double)n * (dhidden_waves(rows, H, V, pairs) + 0.05);
+    if (best_rows == 0 || cost < best_cost - 1e-9) { best_rows = rows; best_cost = cost; }
+  }
+  return best_rows;
 }
 
 // Scratch of the fused call: per-token vectors for all T tokens, then what one token chunk
@@ -511,12 +539,12 @@ extern "C" size_t sapo_workspace_bytes(int32_t which, int64_t T, int32_t H, int3
   if (which == SAPO_WS_FUSED) {
     if (dtype != SAPO_DTYPE_BF16) return 0;
     const FusedLayout L = fused_layout(T, H, V, /*S=*/(int32_t)(T < 0x7fffffff ? T : 0x7fffffff), out_bf16, gather);
-    return L.fixed + FUSED_CHUNK_SLACK + (size_t)preferred_panel_rows(T) * L.bytes_per_row;
+    return L.fixed + FUSED_CHUNK_SLACK + (size_t)preferred_panel_rows(T, H, V) * L.bytes_per_row;
   }
   if (which == SAPO_WS_BWD || which == SAPO_WS_BWD_ACTIVE) {
     const BwdLayout L = bwd_layout(T, H, V, dtype, out_bf16);
     const size_t extra = which == SAPO_WS_BWD_ACTIVE ? active_layout(T, H).total : 0;
-    return extra + L.fixed + (size_t)preferred_panel_rows(T) * L.bytes_per_row;
+    return extra + L.fixed + (size_t)preferred_panel_rows(T, H, V) * L.bytes_per_row;
   }
   return 0;
 }
