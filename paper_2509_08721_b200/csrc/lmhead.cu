@@ -129,11 +129,8 @@ static int fwd_splits(int64_t T, int32_t V, int64_t K, int sms) {
 }
 
 // Stage shape of the three projections hidden . W^T (forward, dz, single pass): K depth and ring length
-#ifdef SAPO_FWD_BK64
-constexpr int FWD_BK = 64, FWD_STAGES = 7;
-#else
+// (a ring of seven 64-deep stages was measured 15-20 % slower: twice the barrier rounds per MMA)
 constexpr int FWD_BK = BK, FWD_STAGES = STAGES;
-#endif
 
 template <int A_KIND, bool B_MN, class Epi, int BKT = BK, int NSTAGE = STAGES, class Gather = NoGather>
 static int launch_gemm(const CUtensorMap& ma, const CUtensorMap& mb, const Sched& sched,
