@@ -12,8 +12,8 @@ What it computes, and where the method states it:
   group_advantages    GRPO's group-relative advantage (paper Section 4.2 names GRPO);
                       A = (r - mean_group) / (std_group + eps)
   token_logprobs      log-prob of each chosen token under the policy's LM head
-                      (Section 3.2: nodes "re-encode and compute token-level values" for
-                      any rollout as if it were their own)
+                      (Section 3.2: a node encodes any rollout, received or its own, and
+                      scores its tokens under its own policy)
   token_entropy       entropy of that distribution per position (a logged by-product)
   policy_loss_fwd     the clipped-ratio surrogate with KL weight 0 and separate lower /
                       upper clip thresholds (Section 4.2)
