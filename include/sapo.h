@@ -1,8 +1,8 @@
 /*
  * sapo.h — C ABI of the SAPO policy-scoring library for NVIDIA B200 (sm_100a).
  *
- * One SAPO node's policy update (paper Algorithm 1, "Assemble training set" and
- * "Policy update") scores a batch made of I locally generated and J swarm-sampled
+ * One SAPO node's policy update (paper Algorithm 1: the steps that put the training set
+ * together and update the policy) scores a batch made of I locally generated and J swarm-sampled
  * rollouts per question.  This library runs the data-parallel part of that update:
  *
  *   sapo_pack_rollouts     training set T^n = {local picks} U {external picks}
@@ -13,7 +13,7 @@
  *                          node's own policy) + clipped-ratio surrogate, KL weight 0,
  *                          separate lower/upper clip thresholds (Section 4.2)
  *   sapo_policy_loss_bwd   gradient of that loss w.r.t. the final hidden states and the
- *                          LM-head weight (Algorithm 1, PolicyGradient)
+ *                          LM-head weight (Algorithm 1, the policy-gradient step)
  *   sapo_policy_loss_fwd_bwd  the two above in one call that passes over the logits once
  *                          (bf16 operands; the fastest way through a training step)
  *
@@ -173,7 +173,7 @@ typedef struct sapo_loss_cfg {
   float* entropy;
 } sapo_loss_cfg;
 
-/* Section 3.2, training-set equation / Algorithm 1 "Assemble training set".
+/* Section 3.2, training-set equation / Algorithm 1, where the training set is put together.
  * Gathers the selected rollouts into one token-major batch.  Sequence order: questions in
  * order; inside a question its local picks in list order, then its external picks in list
  * order.  Copies are byte-exact.  H is the row width in elements, `dtype` a SAPO_DTYPE_*.

@@ -7,8 +7,8 @@ product path never does.  It shares no code with the CUDA sources.
 What it computes, and where the method states it:
 
   pack_rollouts       the training set T^n = {I local samples} U {J external samples}
-                      (paper Section 3.2, training-set equation; Algorithm 1
-                      "Assemble training set"), as a varlen token layout
+                      (paper Section 3.2, training-set equation; Algorithm 1,
+                      where the training set is put together), as a varlen token layout
   group_advantages    GRPO's group-relative advantage (paper Section 4.2 names GRPO);
                       A = (r - mean_group) / (std_group + eps)
   token_logprobs      log-prob of each chosen token under the policy's LM head
