@@ -96,3 +96,28 @@ def test_pack_rejects_null_arrays_on_the_host():
         assert call(bufs(), bufs(), packed(**{member: None})) == -1, member
     assert call(bufs(), bufs(), packed(), B.SelectionC(None, x, x, x, 2)) == -1
     assert call(bufs(), bufs(), packed(), B.SelectionC(x, x, None, x, 2)) == -1
+
+
+def test_default_panel_size_fills_the_last_wave_of_the_dhidden_contraction():
+    """Batches beyond 20 480 tokens are cut into equal chunks whose count the workspace query
+    picks so that the dhidden contraction (2, 3 or 7 column tiles per 256-token block at H = 896,
+    1536, 3584; 74 CTA pairs) wastes least of its last wave.  The chunk rows follow from the size
+    of the dz panel, the only per-row part of the separate backward's scratch."""
+    def panel_rows(T, H, V):
+        full = B.sapo_workspace_bytes(B.WS_BWD, T, H, V, B.DTYPE_BF16)
+        least = B.sapo_workspace_bytes_min(B.WS_BWD, T, H, V, B.DTYPE_BF16)
+        vp = -(-V // 128) * 128
+        assert (full - least) % (2 * vp) == 0
+        return (full - least) // (2 * vp) + 128
+    assert panel_rows(16527, 896, 151936) == 16640            # up to 20 480 tokens: the whole batch
+    assert panel_rows(20480, 896, 151936) == 20480
+    # 332 751 tokens at H = 896: 18 chunks of 18 560 (146 tiles = two full waves), not 17 of 19 584
+    assert panel_rows(332751, 896, 151936) == 18560
+    # H = 1536 and 3584: chunks of at most 16 384 tokens (a chunk's hidden rows stay within 48 MB)
+    assert panel_rows(146382, 1536, 151936) == 13312          # 11 chunks; 9 of 16 384 waste a third of a wave
+    assert panel_rows(143347, 3584, 152064) == 14336          # 10 chunks
+    for T, H, V in ((146382, 1536, 151936), (143347, 3584, 152064), (332751, 896, 151936), (50000, 256, 4096)):
+        rows = panel_rows(T, H, V)
+        assert rows % 128 == 0 and 128 <= rows <= 20480
+        n = -(-T // rows)
+        assert (n - 1) * rows < T <= n * rows and n * rows - T < n * 128   # equal chunks, no short one at the end
