@@ -157,6 +157,17 @@ group_adv_kernel(const float* __restrict__ rewards, const int32_t* __restrict__ 
 // held in registers by one thread.  Loads and stores are 32 bytes wide, so a thread touches whole
 // sectors and a warp's accesses to neighbouring groups of eight are contiguous.
 template <int N4>
+__device__ __forceinline__ void group_finish(float (&r)[4 * N4], float* __restrict__ adv, int32_t a, int32_t G,
+                                             float adv_eps, int32_t ddof, float& mu_out, float& sd_out, bool& bad);
+
+// eight rewards of a group that starts on a 32-byte boundary
+__device__ __forceinline__ void load_eight(const float* __restrict__ p, float (&r)[8]) {
+  asm volatile("ld.global.nc.v8.f32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+               : "=f"(r[0]), "=f"(r[1]), "=f"(r[2]), "=f"(r[3]), "=f"(r[4]), "=f"(r[5]), "=f"(r[6]), "=f"(r[7])
+               : "l"(p));
+}
+
+template <int N4>
 __device__ __forceinline__ void group_in_registers(const float* __restrict__ rewards, float* __restrict__ adv,
                                                    int32_t a, int32_t G, float adv_eps, int32_t ddof,
                                                    float& mu_out, float& sd_out, bool& bad) {
@@ -186,6 +197,14 @@ __device__ __forceinline__ void group_in_registers(const float* __restrict__ rew
       for (int j = 0; j < 8; ++j) r[4 * i + j] = 0.f;
     }
   }
+  group_finish<N4>(r, adv, a, G, adv_eps, ddof, mu_out, sd_out, bad);
+}
+
+// the arithmetic and the stores of a group whose rewards are in r (padding zeros past G)
+template <int N4>
+__device__ __forceinline__ void group_finish(float (&r)[4 * N4], float* __restrict__ adv, int32_t a, int32_t G,
+                                             float adv_eps, int32_t ddof, float& mu_out, float& sd_out, bool& bad) {
+  constexpr int N = 4 * N4;
   float s = r[0], c = 0.f;
   bad = !isfinite(r[0]);
   #pragma unroll
@@ -225,25 +244,45 @@ __device__ __forceinline__ void group_in_registers(const float* __restrict__ rew
 // One thread per question, for batches of very many small groups: no shuffles and no idle lanes.
 // A group of up to 16 whose start and size are multiples of four lives in registers; other groups
 // take plain loops in fp64.
-__global__ void __launch_bounds__(256, 4)
+__global__ void __launch_bounds__(256, 3)
 group_adv_thread_kernel(const float* __restrict__ rewards, const int32_t* __restrict__ group_offsets,
                         int32_t Q, float adv_eps, int32_t ddof, float* __restrict__ adv,
                         float* __restrict__ mean, float* __restrict__ stdv, int32_t* status) {
   // The kernel is bound by how many loads it keeps in flight: a question's rewards can only be
-  // fetched once its offsets are known, so the offsets of the thread's next question are loaded
-  // one turn ahead and a turn waits for a single round trip to memory.
+  // fetched once its offsets are known.  So a thread runs two turns ahead with the offsets and one
+  // turn ahead with the rewards of a group of eight on a 32-byte boundary (the usual case): every
+  // turn has a 32-byte reward load and an offset load in flight while it computes and stores.
   const int64_t stride = (int64_t)gridDim.x * blockDim.x;
   int64_t g = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-  int32_t a_next = 0, b_next = 0;
-  if (g < Q) { a_next = group_offsets[g]; b_next = group_offsets[g + 1]; }
+  int32_t a1 = 0, b1 = 0, a2 = 0, b2 = 0;
+  if (g < Q) { a1 = group_offsets[g]; b1 = group_offsets[g + 1]; }
+  if (g + stride < Q) { a2 = group_offsets[g + stride]; b2 = group_offsets[g + stride + 1]; }
+  float ahead[8];
+  bool have = g < Q && (a1 & 7) == 0 && b1 - a1 == 8;
+  if (have) load_eight(rewards + a1, ahead);
   for (; g < Q; g += stride) {
-    const int32_t a = a_next, b = b_next;
-    if (g + stride < Q) { a_next = group_offsets[g + stride]; b_next = group_offsets[g + stride + 1]; }
+    const int32_t a = a1, b = b1;
+    a1 = a2; b1 = b2;
+    if (g + 2 * stride < Q) { a2 = group_offsets[g + 2 * stride]; b2 = group_offsets[g + 2 * stride + 1]; }
+    const bool had = have;
+    float r8[8];
+    #pragma unroll
+    for (int i = 0; i < 8; ++i) r8[i] = ahead[i];
+    have = g + stride < Q && (a1 & 7) == 0 && b1 - a1 == 8;
+    if (have) load_eight(rewards + a1, ahead);
     const int32_t G = b - a;
+    if (had) {
+      float mu, sd; bool bad;
+      group_finish<2>(r8, adv, a, 8, adv_eps, ddof, mu, sd, bad);
+      if (bad) raise_status(status, SAPO_ST_NONFINITE_REWARD);
+      if (mean) mean[g] = mu;
+      if (stdv) stdv[g] = sd;
+      continue;
+    }
     if (G <= 0) { if (mean) mean[g] = 0.f; if (stdv) stdv[g] = 0.f; continue; }
     const bool vec = ((a | G) & 3) == 0;
     if (vec && G <= 16) {
-      // the usual case (8 or 16 completions per question)
+      // 4, 12 or 16 completions, or eight off the 32-byte boundary
       float mu, sd; bool bad;
       if (G <= 8) group_in_registers<2>(rewards, adv, a, G, adv_eps, ddof, mu, sd, bad);
       else        group_in_registers<4>(rewards, adv, a, G, adv_eps, ddof, mu, sd, bad);
@@ -278,7 +317,9 @@ static int launch_group_adv(const float* rewards, const int32_t* group_offsets, 
   if (sms <= 0) return SAPO_ERR_CUDA;
   const bool many = which == 2 || (which == 0 && Q >= 4096);        // then: one thread per question
   int64_t blocks = ((int64_t)Q + (many ? 255 : 127)) / (many ? 256 : 128);   // warp-level: 16 questions per warp
-  if (blocks > (int64_t)sms * 8) blocks = (int64_t)sms * 8;
+  // the thread-per-question kernel: three blocks fit an SM, all of the grid resident at once
+  const int64_t cap = (int64_t)sms * (many ? 3 : 8);
+  if (blocks > cap) blocks = cap;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   {
     KernelScope scope(SAPO_K_GROUP_ADV, st);
