@@ -118,7 +118,7 @@ __global__ void __launch_bounds__(SCAN_THREADS) pack_scan_kernel(PackArgs a) {
 // per lane) are issued before the first store.
 constexpr int ROW_VECS_PER_LANE = 4;     // 16-byte vectors of one row a lane holds at a time
 
-__global__ void __launch_bounds__(256) pack_copy_kernel(PackArgs a) {
+__global__ void __launch_bounds__(256, 3) pack_copy_kernel(PackArgs a) {
   const int lane = threadIdx.x & 31;
   const int64_t warp0 = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
   const int64_t n_warps = ((int64_t)gridDim.x * blockDim.x) >> 5;
@@ -187,27 +187,42 @@ __global__ void __launch_bounds__(256) pack_copy_kernel(PackArgs a) {
       if (ta >= T) break;
       const bool have_b = tb < T;
       if (two_at_once) {
+        // all loads of the two tokens (rows, ids, old log-probs) are issued before the first store,
+        // so the pair costs one round trip to memory, not one per dependent load-store pair
         const int64_t sa = locate(ta);
+        const int32_t seq_a = s, side_a = side;
         const uint4* fa = reinterpret_cast<const uint4*>(a.hid[side] + sa * a.row_bytes);
         uint4 va[ROW_VECS_PER_LANE], vb[ROW_VECS_PER_LANE];
         #pragma unroll
         for (int q = 0; q < ROW_VECS_PER_LANE; ++q) if (lane + 32 * q < n4) va[q] = __ldg(fa + lane + 32 * q);
-        finish(ta, sa);
-        int64_t sb = 0;
+        const bool ok_a = lane == 0 && SAPO_IN_BOUNDS(ta < a.max_tokens && sa >= 0 && sa < a.off[side][a.n_roll[side]]);
+        int32_t id_a = 0, id_b = 0; float old_a = 0.f, old_b = 0.f;
+        if (ok_a) { id_a = a.ids[side][sa]; old_a = a.old[side][sa]; }
+        int64_t sb = 0; int32_t seq_b = 0, side_b = 0; bool ok_b = false;
         if (have_b) {
           sb = locate(tb);
+          seq_b = s; side_b = side;
           const uint4* fb = reinterpret_cast<const uint4*>(a.hid[side] + sb * a.row_bytes);
           #pragma unroll
           for (int q = 0; q < ROW_VECS_PER_LANE; ++q) if (lane + 32 * q < n4) vb[q] = __ldg(fb + lane + 32 * q);
+          ok_b = lane == 0 && SAPO_IN_BOUNDS(tb < a.max_tokens && sb >= 0 && sb < a.off[side][a.n_roll[side]]);
+          if (ok_b) { id_b = a.ids[side][sb]; old_b = a.old[side][sb]; }
         }
         uint4* oa = reinterpret_cast<uint4*>(a.o_hid + ta * a.row_bytes);
         #pragma unroll
         for (int q = 0; q < ROW_VECS_PER_LANE; ++q) if (lane + 32 * q < n4) oa[lane + 32 * q] = va[q];
+        if (ok_a) {
+          a.o_ids[ta] = id_a; a.o_old[ta] = old_a; a.tok_seq[ta] = seq_a; a.tok_mask[ta] = 1;
+          if (a.tok_src != nullptr) a.tok_src[ta] = sa | ((int64_t)side_a << 62);
+        }
         if (have_b) {
           uint4* ob = reinterpret_cast<uint4*>(a.o_hid + tb * a.row_bytes);
           #pragma unroll
           for (int q = 0; q < ROW_VECS_PER_LANE; ++q) if (lane + 32 * q < n4) ob[lane + 32 * q] = vb[q];
-          finish(tb, sb);
+          if (ok_b) {
+            a.o_ids[tb] = id_b; a.o_old[tb] = old_b; a.tok_seq[tb] = seq_b; a.tok_mask[tb] = 1;
+            if (a.tok_src != nullptr) a.tok_src[tb] = sb | ((int64_t)side_b << 62);
+          }
         }
         continue;
       }
@@ -302,7 +317,7 @@ extern "C" int sapo_pack_rollouts(const sapo_rollout_buf* h_local, const sapo_ro
     a.tokens_per_warp = a.max_tokens >= (int64_t)sms * 64 * 16 ? 16 : 8;
     const int64_t warps_wanted = (a.max_tokens + a.tokens_per_warp - 1) / a.tokens_per_warp;
     int blocks = (int)((warps_wanted + 7) / 8);
-    const int max_blocks = sms * 8;                 // 8 resident blocks of 256 threads per SM
+    const int max_blocks = sms * 3;                 // three blocks of 256 threads are resident per SM: the whole grid at once
     if (blocks > max_blocks) blocks = max_blocks;
     KernelScope scope(SAPO_K_PACK_COPY, st);
     pack_copy_kernel<<<blocks, 256, 0, st>>>(a);
