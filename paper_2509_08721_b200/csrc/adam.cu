@@ -68,6 +68,8 @@ extern "C" int sapo_adam_step(float* master, float* m, float* v, const float* gr
   if (sms <= 0) return SAPO_ERR_CUDA;
   const int64_t n4 = rows * (int64_t)(cols / 4);
   int64_t blocks = ceil_div<int64_t>(n4, 256);
+  // (a grid of only the resident blocks was measured slower here, 0.89 against 0.96 of copy bandwidth:
+  //  seven streams per thread, and short-lived blocks keep them closer together in memory)
   if (blocks > (int64_t)sms * 16) blocks = (int64_t)sms * 16;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   {

@@ -317,8 +317,9 @@ static int launch_group_adv(const float* rewards, const int32_t* group_offsets, 
   if (sms <= 0) return SAPO_ERR_CUDA;
   const bool many = which == 2 || (which == 0 && Q >= 4096);        // then: one thread per question
   int64_t blocks = ((int64_t)Q + (many ? 255 : 127)) / (many ? 256 : 128);   // warp-level: 16 questions per warp
-  // the thread-per-question kernel: three blocks fit an SM, all of the grid resident at once
-  const int64_t cap = (int64_t)sms * (many ? 3 : 8);
+  // at most the blocks the device holds at once (three per SM for the thread-per-question kernel)
+  const int64_t cap = (int64_t)sms * (many ? resident_blocks_per_sm(group_adv_thread_kernel, 256)
+                                           : resident_blocks_per_sm(group_adv_kernel<2>, 256));
   if (blocks > cap) blocks = cap;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   {

@@ -56,6 +56,16 @@ inline int sm_count() {
   return n[dev];
 }
 
+// Blocks of `threads` threads of `kernel` an SM holds at once.  The grid-stride kernels that stream
+// through device memory are launched with at most that many blocks per SM: a larger grid runs in
+// waves, and a last wave that is not full leaves bandwidth unused.
+template <class Kernel>
+inline int resident_blocks_per_sm(Kernel kernel, int threads) {
+  int n = 0;
+  if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, kernel, threads, 0) != cudaSuccess || n < 1) n = 1;
+  return n;
+}
+
 // Optional per-kernel timing and launch counting (see sapo_timing_* in sapo.h).
 // A KernelScope brackets one kernel launch with two CUDA events when timing is on.
 struct KernelTimer {

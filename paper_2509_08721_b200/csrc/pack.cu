@@ -317,7 +317,7 @@ extern "C" int sapo_pack_rollouts(const sapo_rollout_buf* h_local, const sapo_ro
     a.tokens_per_warp = a.max_tokens >= (int64_t)sms * 64 * 16 ? 16 : 8;
     const int64_t warps_wanted = (a.max_tokens + a.tokens_per_warp - 1) / a.tokens_per_warp;
     int blocks = (int)((warps_wanted + 7) / 8);
-    const int max_blocks = sms * 3;                 // three blocks of 256 threads are resident per SM: the whole grid at once
+    const int max_blocks = sms * resident_blocks_per_sm(pack_copy_kernel, 256);   // the whole grid resident at once (three per SM)
     if (blocks > max_blocks) blocks = max_blocks;
     KernelScope scope(SAPO_K_PACK_COPY, st);
     pack_copy_kernel<<<blocks, 256, 0, st>>>(a);
